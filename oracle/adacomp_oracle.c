@@ -1,0 +1,285 @@
+/*
+ * CPU oracle for AdaComp pack() and unpack()-and-sum.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded restatement of Algorithm 2 ("Details of pack()")
+ * and of the unpack()/sum half of Algorithm 1 of the AdaComp paper, in IEEE
+ * binary32 (the precision the method is stated in), written to be checked
+ * against the paper by eye.  It shares no code with the CUDA library and is
+ * only ever called from the tests, from the smoke check and from the
+ * benchmark's CPU-baseline leg.  Build: gcc -O2 -ffp-contract=off (no fast-math),
+ * so every add/sub is a single rounded binary32 operation and denormals are kept.
+ *
+ * Parity pins: hand-worked bins, closed-form special cases, brute force against
+ * an independent scalar Python restatement, and exact-sum checks against
+ * rational arithmetic live in the CPU test-suite.  No function here is unpinned.
+ *
+ * Where the paper is silent the following readings are taken (each is tested):
+ *   - the last bin may be short (Section 2.5 says Algorithm 2 assumes T | length);
+ *   - g_max(i) is the largest |G| in bin i (Algorithm 2, "largest absolute value");
+ *   - an element is sent when |H| >= g_max(i) (Algorithm 2) or when it IS the
+ *     bin maximum (Section 2.4: "In addition to this value ... several other
+ *     residues"); flag bit 0 drops the second clause (literal Algorithm 2);
+ *   - bins whose maximum is zero send nothing, and an element with G == 0 is
+ *     never sent (its ternary value would be 0);
+ *   - Quantize(G) = sign(G) * scale, scale = mean over ALL bins of g_max
+ *     (Section 2.5), the sum taken exactly, rounded once to double, divided by
+ *     the bin count in double and rounded to binary32;
+ *   - the wire word is (index_in_bin << 2) | code with code 01 = +scale and
+ *     11 = -scale, 8 bits wide for L_T <= 64 and 16 bits up to L_T = 16384
+ *     (Section "Experiment Results": 8-/16-bit sparse-indexed words, 2 bits of
+ *     which hold the ternary value);
+ *   - unpack() scatters +-scale_l; the sum over learners runs l = 0..k-1 in
+ *     order starting from +0.0f.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_MAGIC 0x31434441u /* "ADC1" little-endian */
+#define ORACLE_HEADER_BYTES 64u
+
+static uint64_t align16(uint64_t x) { return (x + 15u) & ~(uint64_t)15u; }
+
+/* ---- stream geometry: a pure function of (n, L_T) ------------------------ */
+
+typedef struct {
+    uint32_t w;          /* bytes per word */
+    uint32_t tile_bins;  /* bins per directory tile */
+    uint64_t n_bins;
+    uint64_t n_tiles;
+    uint64_t tile_off_at; /* byte offsets of the sections */
+    uint64_t bin_cnt_at;
+    uint64_t payload_at;
+} geometry;
+
+static geometry geometry_of(uint64_t n, uint32_t L_T)
+{
+    geometry g;
+    g.w = (L_T <= 64u) ? 1u : 2u;
+    g.tile_bins = (L_T <= 1000u) ? 4u * (1000u / L_T) : 1u;
+    g.n_bins = (n + L_T - 1u) / L_T;
+    g.n_tiles = (g.n_bins + g.tile_bins - 1u) / g.tile_bins;
+    g.tile_off_at = ORACLE_HEADER_BYTES;
+    g.bin_cnt_at = align16(g.tile_off_at + 8u * (g.n_tiles + 1u));
+    g.payload_at = align16(g.bin_cnt_at + g.n_bins * g.w);
+    return g;
+}
+
+uint64_t adacomp_oracle_stream_bytes(uint64_t n, uint32_t L_T, uint64_t n_sel)
+{
+    geometry g = geometry_of(n, L_T);
+    return g.payload_at + align16(n_sel * g.w);
+}
+
+/* ---- little-endian field access ------------------------------------------ */
+
+static void put_u16(uint8_t *p, uint16_t v) { p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); }
+static void put_u32(uint8_t *p, uint32_t v) { for (int i = 0; i < 4; i++) p[i] = (uint8_t)(v >> (8 * i)); }
+static void put_u64(uint8_t *p, uint64_t v) { for (int i = 0; i < 8; i++) p[i] = (uint8_t)(v >> (8 * i)); }
+static uint16_t get_u16(const uint8_t *p) { return (uint16_t)(p[0] | (p[1] << 8)); }
+static uint32_t get_u32(const uint8_t *p) { uint32_t v = 0; for (int i = 3; i >= 0; i--) v = (v << 8) | p[i]; return v; }
+static uint64_t get_u64(const uint8_t *p) { uint64_t v = 0; for (int i = 7; i >= 0; i--) v = (v << 8) | p[i]; return v; }
+
+/* ---- exact sum of non-negative binary32 values --------------------------- */
+/*
+ * Every finite binary32 value is an integer multiple of 2^-149 below 2^128,
+ * so a 320-bit unsigned integer holds the exact sum of up to 2^31 of them.
+ * The sum is then rounded once, to nearest-even, to a double.
+ */
+#define BIG_LIMBS 10
+
+static void big_add_f32(uint32_t limb[BIG_LIMBS], float v)
+{
+    uint32_t bits;
+    memcpy(&bits, &v, 4);
+    uint32_t e = (bits >> 23) & 0xffu;
+    uint32_t frac = bits & 0x7fffffu;
+    uint64_t m = e ? (frac | 0x800000u) : frac;   /* value = m * 2^(shift-149) */
+    uint32_t shift = e ? e - 1u : 0u;
+    uint32_t at = shift / 32u;
+    uint64_t add = m << (shift % 32u);            /* < 2^55 */
+    uint64_t carry = 0;
+    for (uint32_t i = at; i < BIG_LIMBS && (add || carry); i++) {
+        uint64_t s = (uint64_t)limb[i] + (add & 0xffffffffu) + carry;
+        limb[i] = (uint32_t)s;
+        carry = s >> 32;
+        add >>= 32;
+    }
+}
+
+static int big_bit(const uint32_t limb[BIG_LIMBS], int pos)
+{
+    return (limb[pos / 32] >> (pos % 32)) & 1u;
+}
+
+static double big_to_double_units(const uint32_t limb[BIG_LIMBS])
+{
+    /* returns the double nearest to (integer value) * 2^-149 */
+    int top = -1;
+    for (int pos = 32 * BIG_LIMBS - 1; pos >= 0; pos--)
+        if (big_bit(limb, pos)) { top = pos; break; }
+    if (top < 0) return 0.0;
+    uint64_t mant = 0;
+    int low = top - 52;               /* position of the last kept bit */
+    if (low <= 0) {
+        for (int pos = top; pos >= 0; pos--) mant = (mant << 1) | (uint64_t)big_bit(limb, pos);
+        return ldexp((double)mant, -149);
+    }
+    for (int pos = top; pos >= low; pos--) mant = (mant << 1) | (uint64_t)big_bit(limb, pos);
+    int round_bit = big_bit(limb, low - 1);
+    int sticky = 0;
+    for (int pos = low - 2; pos >= 0 && !sticky; pos--) sticky = big_bit(limb, pos);
+    if (round_bit && (sticky || (mant & 1u))) mant += 1;   /* ties to even */
+    return ldexp((double)mant, low - 149);
+}
+
+/* exposed so the tests can pin the summation by itself against rational arithmetic */
+double adacomp_oracle_exact_sum(const float *v, uint64_t count)
+{
+    uint32_t limb[BIG_LIMBS] = {0};
+    for (uint64_t i = 0; i < count; i++) big_add_f32(limb, v[i]);
+    return big_to_double_units(limb);
+}
+
+/* ---- pack(): Algorithm 2 -------------------------------------------------- */
+/*
+ * dW[n] in; residue[n] in/out; out[out_cap] receives the stream.
+ * g_max_out (optional, n_bins floats) receives the bin maxima.
+ * Returns 0, or -1 bad argument, -2 out of memory, -3 out_cap too small.
+ */
+int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_T,
+                        uint32_t flags, uint8_t *out, uint64_t out_cap, float *g_max_out)
+{
+    if (L_T == 0 || L_T > 16384u || !out || (n && (!dW || !residue))) return -1;
+    const int literal = (flags & 1u) != 0;
+    geometry geo = geometry_of(n, L_T);
+    if (out_cap < geo.payload_at) return -3;
+
+    float *G = (float *)malloc((n ? n : 1) * sizeof(float));
+    float *H = (float *)malloc((n ? n : 1) * sizeof(float));
+    float *g_max = (float *)malloc((geo.n_bins ? geo.n_bins : 1) * sizeof(float));
+    if (!G || !H || !g_max) { free(G); free(H); free(g_max); return -2; }
+
+    /* G <- residue + dW ;  H <- G + dW   (two rounded additions) */
+    for (uint64_t i = 0; i < n; i++) {
+        G[i] = residue[i] + dW[i];
+        H[i] = G[i] + dW[i];
+    }
+
+    /* first loop over all bins: the largest absolute value in each bin */
+    for (uint64_t b = 0; b < geo.n_bins; b++) {
+        uint64_t lo = b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+        float m = 0.0f;
+        for (uint64_t i = lo; i < hi; i++)
+            if (fabsf(G[i]) > m) m = fabsf(G[i]);
+        g_max[b] = m;
+        if (g_max_out) g_max_out[b] = m;
+    }
+
+    /* one scale for the layer: the average of the g_max vector */
+    float scale = 0.0f;
+    if (geo.n_bins) {
+        double S = adacomp_oracle_exact_sum(g_max, geo.n_bins);
+        scale = (float)(S / (double)geo.n_bins);
+    }
+
+    /* second loop over all bins and all indices within each bin */
+    memset(out, 0, geo.payload_at);
+    uint8_t *tile_off = out + geo.tile_off_at;
+    uint8_t *bin_cnt = out + geo.bin_cnt_at;
+    uint8_t *payload = out + geo.payload_at;
+    uint64_t n_sel = 0;
+    int overflow = 0;
+    for (uint64_t b = 0; b < geo.n_bins; b++) {
+        if (b % geo.tile_bins == 0) put_u64(tile_off + 8u * (b / geo.tile_bins), n_sel);
+        uint64_t lo = b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+        uint32_t count = 0;
+        for (uint64_t index = lo; index < hi; index++) {
+            int send = g_max[b] > 0.0f && G[index] != 0.0f &&
+                       (fabsf(H[index]) >= g_max[b] ||
+                        (!literal && fabsf(G[index]) == g_max[b]));
+            if (send) {
+                int negative = signbit(G[index]) != 0;
+                float Gq = negative ? -scale : scale;           /* Quantize(G(index)) */
+                uint32_t word = ((uint32_t)(index - lo) << 2) | (negative ? 3u : 1u);
+                uint64_t at = geo.payload_at + (n_sel + 1u) * geo.w;
+                if (at > out_cap) overflow = 1;
+                else if (geo.w == 1u) payload[n_sel] = (uint8_t)word;
+                else put_u16(payload + 2u * n_sel, (uint16_t)word);
+                residue[index] = G[index] - Gq;
+                n_sel++;
+                count++;
+            } else {
+                residue[index] = G[index];                       /* no transmission */
+            }
+        }
+        if (geo.w == 1u) bin_cnt[b] = (uint8_t)count;
+        else put_u16(bin_cnt + 2u * b, (uint16_t)count);
+    }
+    put_u64(tile_off + 8u * geo.n_tiles, n_sel);
+
+    uint64_t bytes_used = geo.payload_at + align16(n_sel * geo.w);
+    if (bytes_used > out_cap) overflow = 1;
+    if (!overflow) memset(payload + n_sel * geo.w, 0, bytes_used - geo.payload_at - n_sel * geo.w);
+
+    put_u32(out + 0, ORACLE_MAGIC);
+    put_u16(out + 4, 1);
+    out[6] = (uint8_t)geo.w;
+    out[7] = (uint8_t)(flags & 1u);
+    put_u32(out + 8, L_T);
+    put_u32(out + 12, geo.tile_bins);
+    put_u64(out + 16, n);
+    put_u64(out + 24, geo.n_bins);
+    put_u64(out + 32, geo.n_tiles);
+    put_u64(out + 40, n_sel);
+    uint32_t scale_bits;
+    memcpy(&scale_bits, &scale, 4);
+    put_u32(out + 48, scale_bits);
+    put_u32(out + 52, 0);
+    put_u64(out + 56, bytes_used);
+
+    free(G); free(H); free(g_max);
+    return overflow ? -3 : 0;
+}
+
+/* ---- unpack() and sum ----------------------------------------------------- */
+/*
+ * dst[n] is overwritten with the sum over the k streams, taken in stream
+ * order from +0.0f.  Returns 0, or -1 bad argument, -4 streams disagree on
+ * (n, L_T, word size) or are malformed, -5 reserved ternary code 10 met.
+ */
+int adacomp_oracle_unpack_sum(const uint8_t *const *streams, uint32_t k, float *dst, uint64_t n)
+{
+    if (!streams || k == 0 || (n && !dst)) return -1;
+    for (uint64_t i = 0; i < n; i++) dst[i] = 0.0f;
+    uint32_t L_T0 = get_u32(streams[0] + 8);
+    for (uint32_t l = 0; l < k; l++) {
+        const uint8_t *s = streams[l];
+        if (get_u32(s) != ORACLE_MAGIC || get_u16(s + 4) != 1) return -4;
+        uint32_t L_T = get_u32(s + 8);
+        if (L_T == 0 || L_T > 16384u || L_T != L_T0 || get_u64(s + 16) != n) return -4;
+        geometry geo = geometry_of(n, L_T);
+        if (s[6] != geo.w || get_u64(s + 24) != geo.n_bins) return -4;
+        uint32_t scale_bits = get_u32(s + 48);
+        float scale;
+        memcpy(&scale, &scale_bits, 4);
+        const uint8_t *bin_cnt = s + geo.bin_cnt_at;
+        const uint8_t *payload = s + geo.payload_at;
+        uint64_t at = 0;
+        for (uint64_t b = 0; b < geo.n_bins; b++) {
+            uint32_t count = geo.w == 1u ? bin_cnt[b] : get_u16(bin_cnt + 2u * b);
+            for (uint32_t j = 0; j < count; j++, at++) {
+                uint32_t word = geo.w == 1u ? payload[at] : get_u16(payload + 2u * at);
+                uint32_t code = word & 3u;
+                uint64_t index = b * L_T + (word >> 2);
+                if (code == 2u) return -5;
+                if (index >= n) return -4;
+                if (code == 1u) dst[index] = dst[index] + scale;
+                if (code == 3u) dst[index] = dst[index] - scale;
+            }
+        }
+        if (at != get_u64(s + 40)) return -4;
+    }
+    return 0;
+}

@@ -1,0 +1,122 @@
+"""ctypes front end of the C oracle, plus a reader for the stream it emits.
+
+TEST INFRASTRUCTURE ONLY: see the package docstring.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import struct
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build.build())
+        _lib.adacomp_oracle_stream_bytes.restype = C.c_uint64
+        _lib.adacomp_oracle_stream_bytes.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
+        _lib.adacomp_oracle_exact_sum.restype = C.c_double
+        _lib.adacomp_oracle_exact_sum.argtypes = [C.c_void_p, C.c_uint64]
+        _lib.adacomp_oracle_pack.restype = C.c_int
+        _lib.adacomp_oracle_pack.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32,
+                                             C.c_uint32, C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.adacomp_oracle_unpack_sum.restype = C.c_int
+        _lib.adacomp_oracle_unpack_sum.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
+    return _lib
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def stream_bytes(n: int, L_T: int, n_sel: int) -> int:
+    return int(lib().adacomp_oracle_stream_bytes(n, L_T, n_sel))
+
+
+def exact_sum(values: np.ndarray) -> float:
+    """Correctly rounded (to double) exact sum of non-negative float32 values."""
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    return float(lib().adacomp_oracle_exact_sum(_ptr(v), v.size))
+
+
+@dataclass
+class Packed:
+    """A parsed stream (Section 'Experiment Results': sparse-indexed words)."""
+
+    raw: np.ndarray          # uint8, exactly bytes_used long
+    n: int
+    L_T: int
+    w: int
+    flags: int
+    tile_bins: int
+    n_bins: int
+    n_tiles: int
+    n_sel: int
+    scale: np.float32
+    scale_bits: int
+    bytes_used: int
+    tile_off: np.ndarray     # uint64[n_tiles+1]
+    bin_cnt: np.ndarray      # uint8/uint16[n_bins]
+    words: np.ndarray        # uint8/uint16[n_sel]
+    g_max: Optional[np.ndarray] = None
+
+    def positions_and_codes(self):
+        """Flat element index and ternary code of every word, in stream order."""
+        bins = np.repeat(np.arange(self.n_bins, dtype=np.int64), self.bin_cnt.astype(np.int64))
+        idx = (self.words.astype(np.int64) >> 2)
+        return bins * self.L_T + idx, (self.words.astype(np.int64) & 3)
+
+
+def parse(raw: np.ndarray) -> Packed:
+    raw = np.ascontiguousarray(raw, dtype=np.uint8)
+    (magic, version, w, flags, L_T, tile_bins, n, n_bins, n_tiles, n_sel, scale_bits, _rsv,
+     bytes_used) = struct.unpack_from("<IHBBIIQQQQIIQ", raw.tobytes()[:64])
+    assert magic == 0x31434441 and version == 1, (hex(magic), version)
+    tile_off_at = 64
+    bin_cnt_at = (tile_off_at + 8 * (n_tiles + 1) + 15) & ~15
+    payload_at = (bin_cnt_at + n_bins * w + 15) & ~15
+    dt = np.uint8 if w == 1 else np.dtype("<u2")
+    tile_off = np.frombuffer(raw, dtype="<u8", count=n_tiles + 1, offset=tile_off_at).copy()
+    bin_cnt = np.frombuffer(raw, dtype=dt, count=n_bins, offset=bin_cnt_at).copy()
+    words = np.frombuffer(raw, dtype=dt, count=n_sel, offset=payload_at).copy()
+    scale = np.frombuffer(struct.pack("<I", scale_bits), dtype=np.float32)[0]
+    return Packed(raw[:bytes_used].copy(), n, L_T, w, flags, tile_bins, n_bins, n_tiles, n_sel,
+                  scale, scale_bits, bytes_used, tile_off, bin_cnt, words)
+
+
+def pack(dW: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0,
+         want_gmax: bool = False) -> Packed:
+    """Run Algorithm 2 on one layer.  `residue` (float32, contiguous) is updated in place."""
+    assert dW.dtype == np.float32 and residue.dtype == np.float32
+    assert dW.flags.c_contiguous and residue.flags.c_contiguous and dW.shape == residue.shape
+    n = dW.size
+    cap = stream_bytes(n, L_T, n)           # worst case: every element sent
+    out = np.empty(cap, dtype=np.uint8)
+    n_bins = (n + L_T - 1) // L_T
+    gmax = np.empty(max(n_bins, 1), dtype=np.float32) if want_gmax else None
+    rc = lib().adacomp_oracle_pack(_ptr(dW) if n else None, _ptr(residue) if n else None, n, L_T,
+                                   flags, _ptr(out), cap, _ptr(gmax) if want_gmax else None)
+    if rc != 0:
+        raise RuntimeError(f"adacomp_oracle_pack failed: {rc}")
+    p = parse(out)
+    if want_gmax:
+        p.g_max = gmax[:n_bins]
+    return p
+
+
+def unpack_sum(streams: Sequence[np.ndarray], n: int) -> np.ndarray:
+    """Sum k packed streams, in order, into a dense float32 vector."""
+    keep: List[np.ndarray] = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    ptrs = (C.c_void_p * len(keep))(*[_ptr(s) for s in keep])
+    dst = np.empty(n, dtype=np.float32)
+    rc = lib().adacomp_oracle_unpack_sum(ptrs, len(keep), _ptr(dst) if n else None, n)
+    if rc != 0:
+        raise RuntimeError(f"adacomp_oracle_unpack_sum failed: {rc}")
+    return dst
