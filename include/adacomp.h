@@ -1,0 +1,163 @@
+/*
+ * adacomp.h - C ABI of libadacomp: AdaComp residual gradient compression on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the two per-layer functions of the AdaComp paper
+ * (Chen et al., "AdaComp: Adaptive Residual Gradient Compression for
+ * Data-Parallel Distributed Training"): pack() of Algorithm 2 and the
+ * unpack()-then-sum half of Algorithm 1.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device pointers valid on the current device;
+ *     "host" pointers are ordinary process memory.  `stream` is a cudaStream_t
+ *     passed as void* (NULL = the legacy default stream).
+ *   - The caller owns every buffer.  The library allocates no memory and keeps
+ *     no per-call state; all work is enqueued on `stream` and the call returns
+ *     without synchronising (adacomp_device_status is the one exception).
+ *   - grad, residue, dst and packed buffers must be 16-byte aligned.
+ *   - Return value: ADACOMP_OK (0) or a negative ADACOMP_ERR_* code.  When an
+ *     error code is returned nothing has been enqueued.  Conditions only the
+ *     GPU can see set sticky bits (ADACOMP_DEV_*) read by adacomp_device_status;
+ *     a kernel that meets one skips the affected work and finishes normally.
+ *   - Arithmetic is IEEE binary32, round-to-nearest-even, denormals kept, no
+ *     fused multiply-add.  Results are deterministic: the same inputs give the
+ *     same bytes, whatever the launch geometry.
+ *
+ * Packed stream (little-endian; section offsets are a pure function of n, L_T)
+ *   header, 64 bytes:
+ *      0 u32 magic "ADC1" (0x31434441)    4 u16 version = 1
+ *      6 u8  w = bytes per word (1 if L_T <= 64, else 2)
+ *      7 u8  flags (bit 0: literal Algorithm-2 selection)
+ *      8 u32 L_T                         12 u32 tile_bins
+ *     16 u64 n                           24 u64 n_bins = ceil(n / L_T)
+ *     32 u64 n_tiles = ceil(n_bins / tile_bins)
+ *     40 u64 n_sel (elements sent)       48 f32 scale      52 u32 0
+ *     56 u64 bytes_used (header + sections, the bytes a receiver needs)
+ *   tile_off  u64[n_tiles + 1] at byte 64: index of each tile's first word
+ *             (exclusive scan of the per-tile counts; last entry = n_sel);
+ *             tile_bins = 4 * floor(1000 / L_T) for L_T <= 1000, else 1
+ *   bin_cnt   n_bins entries of w bytes, 16-byte aligned: words sent per bin
+ *   payload   n_sel words of w bytes, 16-byte aligned, zero padded to 16 bytes:
+ *             word = (index_in_bin << 2) | code, code 01 = +scale, 11 = -scale,
+ *             00 = no-op, 10 = reserved; bins in order, indices ascending.
+ *   The word widths and the 2-bit ternary value follow the paper's Section
+ *   "Experiment Results" (8-bit words below L_T = 64, 16-bit words up to 16K).
+ *   Beyond bytes_used the buffer holds scratch the compressor needs.
+ */
+#ifndef ADACOMP_H
+#define ADACOMP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ADACOMP_VERSION 1
+#define ADACOMP_MAX_L_T 16384u
+#define ADACOMP_MAX_STREAMS 64u
+
+/* host-detected errors */
+#define ADACOMP_OK 0
+#define ADACOMP_ERR_NULL (-1)      /* a required pointer is NULL */
+#define ADACOMP_ERR_L_T (-2)       /* L_T == 0 or L_T > ADACOMP_MAX_L_T */
+#define ADACOMP_ERR_ALIGN (-3)     /* a buffer is not 16-byte aligned */
+#define ADACOMP_ERR_STREAMS (-4)   /* k_streams == 0 or > ADACOMP_MAX_STREAMS */
+#define ADACOMP_ERR_SIZE (-5)      /* n too large (n_bins must stay below 2^31) */
+#define ADACOMP_ERR_FLAGS (-6)     /* unknown flag bits */
+#define ADACOMP_ERR_CUDA (-7)      /* a CUDA runtime call failed */
+
+/* device-detected conditions (sticky bits) */
+#define ADACOMP_DEV_NONFINITE 1u        /* a bin maximum was inf or NaN */
+#define ADACOMP_DEV_HEADER_MISMATCH 2u  /* streams disagree on n / L_T / w, or bad magic */
+#define ADACOMP_DEV_RESERVED_CODE 4u    /* ternary code 10 met while decoding */
+#define ADACOMP_DEV_TIMEOUT 8u          /* a bounded device-side wait gave up */
+#define ADACOMP_DEV_BAD_STREAM 16u      /* a word points outside its bin / tensor */
+
+/* flags of adacomp_compress_ex */
+#define ADACOMP_FLAG_LITERAL 1u       /* Algorithm 2 as printed: |H| >= g_max only */
+#define ADACOMP_FLAG_GENERIC_PATH 256u /* use the any-L_T kernel even for L_T = 50 / 500 */
+
+/* Library ABI version (ADACOMP_VERSION).  Host only, no CUDA call. */
+int adacomp_version(void);
+
+/* Static, human-readable text for an ADACOMP_ERR_* code.  Host only. */
+const char *adacomp_strerror(int code);
+
+/*
+ * Bytes the caller must allocate for `packed_out` of a layer of n elements:
+ * header + directory + bin counts + worst-case payload (every element sent) +
+ * the compressor's scratch.  Returns 0 for an invalid L_T.  Host only.
+ */
+size_t adacomp_packed_capacity(uint64_t n, uint32_t L_T);
+
+/*
+ * pack() - Algorithm 2 ("Details of pack()") with the scale of Section 2.5.
+ *   grad       device, const float[n]: dW of this step.
+ *   residue    device, float[n], in/out: the learner's residual gradient.
+ *              On return of the stream it holds G - Gq where sent, G elsewhere.
+ *   n, L_T     element count (0 is a valid no-op that writes only a header)
+ *              and bin length, 1 <= L_T <= 16384.
+ *   packed_out device, adacomp_packed_capacity(n, L_T) bytes; receives the stream.
+ *   count_out  device, uint64_t[2]: {n_sel, bytes_used}.
+ * Computes G = residue + dW, H = G + dW, g_max = per-bin max |G|,
+ * scale = mean of g_max over all bins (exact sum, rounded once), sends element i
+ * of bin b when g_max[b] > 0, G[i] != 0 and (|H[i]| >= g_max[b] or |G[i]| == g_max[b]),
+ * quantises it to sign(G) * scale and subtracts that from the residue.
+ */
+int adacomp_compress(const float *grad, float *residue, uint64_t n, uint32_t L_T,
+                     void *packed_out, uint64_t *count_out, void *stream);
+
+/* As adacomp_compress, with ADACOMP_FLAG_* bits. */
+int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t L_T,
+                        void *packed_out, uint64_t *count_out, void *stream, uint32_t flags);
+
+/*
+ * unpack() of k learners' streams and their sum (Algorithm 1: unpack(), and the
+ * summation inside averageGradients()).
+ *   packed     HOST array of k device pointers to packed streams of one layer.
+ *   k_streams  1 .. ADACOMP_MAX_STREAMS.
+ *   dst        device, float[n] (n is read from the first stream's header on the
+ *              device); fully overwritten: dst[i] = sum over l = 0..k-1, in that
+ *              order and starting from +0.0f, of +-scale_l where learner l sent i.
+ * Streams that disagree on n, L_T or word size set ADACOMP_DEV_HEADER_MISMATCH
+ * and dst is left untouched.
+ */
+int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams, float *dst,
+                                  void *stream);
+
+/* One tensor of a multi-tensor call; every tensor is its own layer (own bins, own scale). */
+typedef struct {
+    const float *grad;
+    float *residue;
+    uint64_t n;
+    uint32_t L_T;
+    uint32_t flags;
+    void *packed_out;
+    uint64_t *count_out;
+} adacomp_layer_desc;
+
+/* pack() of every layer in `layers` (HOST array of n_layers descriptors) on one stream. */
+int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream);
+
+/*
+ * unpack()-and-sum of every layer: packed[t * k_streams + l] (HOST array) is
+ * learner l's stream of layer t, dst[t] (HOST array of device pointers) its output.
+ */
+int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_streams,
+                                        float *const *dst, uint32_t n_layers, void *stream);
+
+/*
+ * Synchronises `stream`, then copies the current device's sticky ADACOMP_DEV_* bits to
+ * *host_out.  The bits stay set until adacomp_device_status_reset.
+ */
+int adacomp_device_status(uint32_t *host_out, void *stream);
+
+/* Enqueues a clear of the sticky bits on `stream`. */
+int adacomp_device_status_reset(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADACOMP_H */

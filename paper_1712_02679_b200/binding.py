@@ -1,0 +1,189 @@
+"""Thin ctypes binding of libadacomp.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  There is no CPU
+fallback: if the shared library has not been built, or a tensor is not on a
+CUDA device, the call raises.  PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libadacomp.so")
+
+ADACOMP_FLAG_LITERAL = 1
+ADACOMP_FLAG_GENERIC_PATH = 256
+ADACOMP_MAX_STREAMS = 64
+
+ADACOMP_DEV_NONFINITE = 1
+ADACOMP_DEV_HEADER_MISMATCH = 2
+ADACOMP_DEV_RESERVED_CODE = 4
+ADACOMP_DEV_TIMEOUT = 8
+ADACOMP_DEV_BAD_STREAM = 16
+
+
+class AdaCompError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what} failed: {code} ({adacomp_strerror(code)})")
+        self.code = code
+
+
+class adacomp_layer_desc(C.Structure):
+    _fields_ = [("grad", C.c_void_p), ("residue", C.c_void_p), ("n", C.c_uint64),
+                ("L_T", C.c_uint32), ("flags", C.c_uint32), ("packed_out", C.c_void_p),
+                ("count_out", C.c_void_p)]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_1712_02679_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.adacomp_version.restype = C.c_int
+        L.adacomp_strerror.restype = C.c_char_p
+        L.adacomp_strerror.argtypes = [C.c_int]
+        L.adacomp_packed_capacity.restype = C.c_size_t
+        L.adacomp_packed_capacity.argtypes = [C.c_uint64, C.c_uint32]
+        L.adacomp_compress.restype = C.c_int
+        L.adacomp_compress.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p,
+                                       C.c_void_p, C.c_void_p]
+        L.adacomp_compress_ex.restype = C.c_int
+        L.adacomp_compress_ex.argtypes = L.adacomp_compress.argtypes + [C.c_uint32]
+        L.adacomp_decompress_accumulate.restype = C.c_int
+        L.adacomp_decompress_accumulate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.adacomp_compress_multi.restype = C.c_int
+        L.adacomp_compress_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+        L.adacomp_decompress_accumulate_multi.restype = C.c_int
+        L.adacomp_decompress_accumulate_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p,
+                                                          C.c_uint32, C.c_void_p]
+        L.adacomp_device_status.restype = C.c_int
+        L.adacomp_device_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.adacomp_device_status_reset.restype = C.c_int
+        L.adacomp_device_status_reset.argtypes = [C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _dev_ptr(t: Optional[torch.Tensor], what: str, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{what} must be a CUDA tensor (no CPU path exists)")
+    if not t.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{what} must have dtype {dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise AdaCompError(rc, what)
+
+
+def adacomp_version() -> int:
+    return int(lib().adacomp_version())
+
+
+def adacomp_strerror(code: int) -> str:
+    return lib().adacomp_strerror(int(code)).decode()
+
+
+def adacomp_packed_capacity(n: int, L_T: int) -> int:
+    return int(lib().adacomp_packed_capacity(int(n), int(L_T)))
+
+
+def adacomp_compress(grad, residue, n: int, L_T: int, packed_out, count_out, stream=None) -> None:
+    """pack(): see include/adacomp.h.  count_out is an int64[2] CUDA tensor."""
+    _check(lib().adacomp_compress(_dev_ptr(grad, "grad", torch.float32),
+                                  _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                  _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                  _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
+           "adacomp_compress")
+
+
+def adacomp_compress_ex(grad, residue, n: int, L_T: int, packed_out, count_out, stream=None,
+                        flags: int = 0) -> None:
+    _check(lib().adacomp_compress_ex(_dev_ptr(grad, "grad", torch.float32),
+                                     _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                     _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                     _dev_ptr(count_out, "count_out", torch.int64), _stream(stream),
+                                     int(flags)),
+           "adacomp_compress_ex")
+
+
+def adacomp_decompress_accumulate(packed: Sequence[torch.Tensor], k_streams: int, dst,
+                                  stream=None) -> None:
+    """unpack()-and-sum of k streams into dst (fully overwritten)."""
+    ptrs = (C.c_void_p * max(int(k_streams), 1))(
+        *[_dev_ptr(p, "packed[l]", torch.uint8) for p in packed[:k_streams]])
+    _check(lib().adacomp_decompress_accumulate(ptrs, int(k_streams),
+                                               _dev_ptr(dst, "dst", torch.float32), _stream(stream)),
+           "adacomp_decompress_accumulate")
+
+
+def make_layer_descs(layers: Sequence[dict]):
+    """HOST array of adacomp_layer_desc from dicts with the struct's field names."""
+    arr = (adacomp_layer_desc * max(len(layers), 1))()
+    for i, d in enumerate(layers):
+        arr[i].grad = _dev_ptr(d["grad"], "grad", torch.float32)
+        arr[i].residue = _dev_ptr(d["residue"], "residue", torch.float32)
+        arr[i].n = int(d["n"])
+        arr[i].L_T = int(d["L_T"])
+        arr[i].flags = int(d.get("flags", 0))
+        arr[i].packed_out = _dev_ptr(d["packed_out"], "packed_out", torch.uint8)
+        arr[i].count_out = _dev_ptr(d["count_out"], "count_out", torch.int64)
+    return arr
+
+
+def adacomp_compress_multi(layers, n_layers: int, stream=None) -> None:
+    """layers: a ctypes array from make_layer_descs (or a list of dicts)."""
+    if not isinstance(layers, C.Array):
+        layers = make_layer_descs(layers)
+    _check(lib().adacomp_compress_multi(layers, int(n_layers), _stream(stream)),
+           "adacomp_compress_multi")
+
+
+def make_pointer_array(tensors: Sequence[torch.Tensor], dtype):
+    return (C.c_void_p * max(len(tensors), 1))(*[_dev_ptr(t, "tensor", dtype) for t in tensors])
+
+
+def adacomp_decompress_accumulate_multi(packed, k_streams: int, dst, n_layers: int,
+                                        stream=None) -> None:
+    """packed[t * k_streams + l]: learner l's stream of layer t; dst[t]: its output."""
+    if not isinstance(packed, C.Array):
+        packed = make_pointer_array(packed, torch.uint8)
+    if not isinstance(dst, C.Array):
+        dst = make_pointer_array(dst, torch.float32)
+    _check(lib().adacomp_decompress_accumulate_multi(packed, int(k_streams), dst, int(n_layers),
+                                                     _stream(stream)),
+           "adacomp_decompress_accumulate_multi")
+
+
+def adacomp_device_status(stream=None) -> int:
+    out = C.c_uint32(0)
+    _check(lib().adacomp_device_status(C.byref(out), _stream(stream)), "adacomp_device_status")
+    return int(out.value)
+
+
+def adacomp_device_status_reset(stream=None) -> None:
+    _check(lib().adacomp_device_status_reset(_stream(stream)), "adacomp_device_status_reset")

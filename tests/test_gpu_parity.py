@@ -1,0 +1,242 @@
+"""CUDA path vs the CPU oracle through the C ABI, element by element.
+
+Integer outputs (indices, signs, packed bytes, counts, directory) must match
+bit for bit; so must scale and residue: both sides take the same single
+binary32 operations and the scale comes from an exact sum, so the tolerance
+the task allows (1e-6 relative, 1e-7 absolute near zero) is only checked as a
+fallback statement of that bar."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cref
+from paper_1712_02679_b200 import binding as B
+from paper_1712_02679_b200 import synth
+from tests.gpu_util import GpuLayer, assert_f32_bits_equal, assert_stream_equal
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-6, 1e-7       # the stated floating-point bar; the tests below are stricter (bits)
+
+
+def run_steps(n, L_T, dws, flags=0, residue0=None):
+    """Carried-residue run on both sides; compares every step."""
+    r_cpu = np.zeros(n, np.float32) if residue0 is None else residue0.copy()
+    layer = GpuLayer(n, L_T, residue0)
+    streams = []
+    for step, dW in enumerate(dws):
+        want = cref.pack(dW, r_cpu, L_T, flags=flags & 1)
+        raw, n_sel, used = layer.compress(dW, flags)
+        what = f"n={n} L_T={L_T} flags={flags} step={step}"
+        assert (n_sel, used) == (want.n_sel, want.bytes_used), what
+        assert_stream_equal(raw, want, what)
+        got_r = layer.residue_host()
+        assert_f32_bits_equal(got_r, r_cpu, what + " residue")
+        np.testing.assert_allclose(got_r, r_cpu, rtol=RTOL, atol=ATOL)
+        streams.append(raw)
+    assert B.adacomp_device_status() == 0
+    return layer, streams
+
+
+def test_config1_fc_layer_ten_steps():
+    n, L_T = 100352, 50
+    dws = [synth.make_dw(1, 0, 0, s, n, heavy=False, sigma=1e-3) for s in range(10)]
+    run_steps(n, L_T, dws)
+    run_steps(n, L_T, dws[:3], flags=B.ADACOMP_FLAG_GENERIC_PATH)
+
+
+def test_config2_small_conv_net_twenty_steps():
+    for t, spec in enumerate(synth.config2_tensors()):
+        dws = [synth.make_dw(2, 0, t, s, spec.n, heavy=True) for s in range(20)]
+        run_steps(spec.n, spec.L_T, dws)
+
+
+@pytest.mark.parametrize("L_T", [1, 2, 3, 7, 25, 49, 50, 51, 63, 64, 65, 100, 333, 499, 500, 501,
+                                 1000, 1001, 4096, 5000, 16384])
+def test_bin_lengths_and_ragged_tails(L_T):
+    rng = np.random.default_rng(L_T)
+    for n in sorted({1, L_T - 1, L_T, L_T + 1, 4001, 3 * 4000 + 17, 10 * max(L_T, 40) + 3}):
+        if n <= 0:
+            continue
+        dws = [rng.normal(0, 1e-3, n).astype(np.float32) for _ in range(3)]
+        run_steps(n, L_T, dws)
+
+
+@pytest.mark.parametrize("L_T", [50, 500])
+@pytest.mark.parametrize("n", [4000, 8000, 7999, 8001, 4000 * 150 + 1, 4000 * 1500 - 3])
+def test_fast_path_tile_boundaries(L_T, n):
+    rng = np.random.default_rng(n + L_T)
+    dws = [synth.heavy_dw(n, 1e-3, rng) for _ in range(4)]
+    run_steps(n, L_T, dws)
+    run_steps(n, L_T, dws[:2], flags=B.ADACOMP_FLAG_LITERAL)
+    run_steps(n, L_T, dws[:2], flags=B.ADACOMP_FLAG_GENERIC_PATH | B.ADACOMP_FLAG_LITERAL)
+
+
+def test_empty_tensor_writes_a_header_only():
+    layer = GpuLayer(0, 50)
+    raw, n_sel, used = layer.compress(np.zeros(0, np.float32))
+    want = cref.pack(np.zeros(0, np.float32), np.zeros(0, np.float32), 50)
+    assert (n_sel, used) == (0, 80)
+    assert_stream_equal(raw, want)
+
+
+def test_degenerate_values():
+    n, L_T = 9000, 50
+    rng = np.random.default_rng(4)
+    zeros = np.zeros(n, np.float32)
+    run_steps(n, L_T, [zeros, zeros])                              # nothing to send at all
+    dw = rng.normal(0, 1e-3, n).astype(np.float32)
+    dw[:150] = 0                                                   # zero bins inside
+    dw[200:250] = np.float32(1e-3)                                 # a bin of ties: all sent
+    dw[300:350] = np.float32(-0.0)
+    run_steps(n, L_T, [dw, -dw, dw])                               # -dw cancels: exact zeros
+    tiny = (rng.normal(0, 1, n) * 1e-42).astype(np.float32)        # denormals must survive
+    run_steps(n, L_T, [tiny, tiny])
+    huge = (rng.normal(0, 1, n) * 1e37).astype(np.float32)
+    run_steps(n, L_T, [huge])
+    wide = (rng.normal(0, 1, n) * 10.0 ** rng.uniform(-40, 30, n)).astype(np.float32)
+    run_steps(n, 500, [wide, wide])                                # scale sum over 70 decades
+    res0 = rng.normal(0, 5e-3, n).astype(np.float32)
+    run_steps(n, 500, [np.zeros(n, np.float32)], residue0=res0)    # dW = 0: only maxima go
+
+
+def test_metamorphic_on_gpu_scale_is_order_independent():
+    L_T, Bn = 50, 4000
+    rng = np.random.default_rng(9)
+    dW = rng.normal(0, 1e-3, L_T * Bn).astype(np.float32)
+    dW[::977] *= np.float32(1e4)
+    perm = rng.permutation(Bn)
+    dWp = dW.reshape(Bn, L_T)[perm].ravel().copy()
+    a, _ = run_steps(L_T * Bn, L_T, [dW])
+    b, _ = run_steps(L_T * Bn, L_T, [dWp])
+    sa = a.packed[48:52].cpu().numpy().tobytes()
+    sb = b.packed[48:52].cpu().numpy().tobytes()
+    assert sa == sb
+
+
+def test_same_inputs_twice_give_the_same_bytes():
+    n = 4000 * 300 + 11
+    rng = np.random.default_rng(21)
+    dW = rng.normal(0, 1e-3, n).astype(np.float32)
+    res = rng.normal(0, 3e-3, n).astype(np.float32)
+    outs = []
+    for _ in range(3):
+        layer = GpuLayer(n, 50, res)
+        raw, _, _ = layer.compress(dW)
+        outs.append((raw.tobytes(), layer.residue_host().tobytes()))
+    assert outs[0] == outs[1] == outs[2]
+
+
+# --------------------------------------------------------------------------
+# unpack()-and-sum
+# --------------------------------------------------------------------------
+
+def gpu_decode(streams, n):
+    dev = torch.device("cuda:0")
+    bufs = [torch.from_numpy(s.copy()).to(dev) for s in streams]
+    # pad each to a 16-byte aligned allocation (torch already aligns to 512)
+    dst = torch.full((max(n, 4),), float("nan"), dtype=torch.float32, device=dev)
+    B.adacomp_decompress_accumulate(bufs, len(bufs), dst)
+    torch.cuda.synchronize()
+    return dst[:n].cpu().numpy()
+
+
+@pytest.mark.parametrize("L_T,n,k", [(50, 100352, 1), (50, 5120, 4), (500, 147456, 8), (50, 4000 * 40 + 7, 16),
+                                     (3, 9001, 3), (64, 70000, 2), (65, 70000, 2), (1000, 50001, 5),
+                                     (1001, 50001, 5), (5000, 123457, 3), (16384, 100001, 4),
+                                     (16384, 100, 2), (500, 12, 64)])
+def test_decode_sum_matches_oracle(L_T, n, k):
+    rng = np.random.default_rng(L_T + n + k)
+    streams_gpu, streams_cpu = [], []
+    for l in range(k):
+        r = rng.normal(0, 2e-3, n).astype(np.float32)
+        dW = rng.normal(0, 1e-3 * (1 + l), n).astype(np.float32)
+        want = cref.pack(dW, r.copy(), L_T)
+        raw, _, _ = GpuLayer(n, L_T, r).compress(dW)
+        assert_stream_equal(raw, want)
+        streams_gpu.append(raw)
+        streams_cpu.append(want.raw)
+    want_dst = cref.unpack_sum(streams_cpu, n)
+    got = gpu_decode(streams_gpu, n)
+    assert_f32_bits_equal(got, want_dst, f"decode L_T={L_T} n={n} k={k}")
+    np.testing.assert_allclose(got, want_dst, rtol=RTOL, atol=ATOL)
+    assert B.adacomp_device_status() == 0
+
+
+def test_decode_sum_seeded_four_learners_crosscheck():
+    import zlib
+    spec = synth.config2_tensors()[7]
+    streams = []
+    for l in range(4):
+        dW = synth.make_dw(2, l, 7, 0, spec.n, heavy=True)
+        raw, _, _ = GpuLayer(spec.n, spec.L_T).compress(dW)
+        streams.append(raw)
+    dst = gpu_decode(streams, spec.n)
+    assert zlib.crc32(dst.astype("<f4").tobytes()) & 0xFFFFFFFF == 0x4FC334F2
+    assert int(np.count_nonzero(dst)) == 2589
+
+
+def test_decoder_flags_bad_streams_without_faulting():
+    n, L_T = 20000, 50
+    rng = np.random.default_rng(2)
+    a = cref.pack(rng.normal(0, 1e-3, n).astype(np.float32), np.zeros(n, np.float32), L_T)
+    b = cref.pack(rng.normal(0, 1e-3, n + 50).astype(np.float32), np.zeros(n + 50, np.float32), L_T)
+    B.adacomp_device_status_reset()
+    assert B.adacomp_device_status() == 0
+    got = gpu_decode([a.raw, b.raw], n)                       # n differs between the streams
+    assert B.adacomp_device_status() & B.ADACOMP_DEV_HEADER_MISMATCH
+    assert np.all(np.isnan(got))                              # dst left untouched
+    B.adacomp_device_status_reset()
+    bad = a.raw.copy()
+    first_word = a.bytes_used - 16 * ((a.n_sel + 15) // 16)
+    bad[first_word] = (bad[first_word] & 0xFC) | 0b10         # reserved ternary code
+    got = gpu_decode([bad], n)
+    assert B.adacomp_device_status() == B.ADACOMP_DEV_RESERVED_CODE
+    want = cref.unpack_sum([a.raw], n)
+    pos, _ = a.positions_and_codes()
+    want[pos[0]] = 0.0                                        # the bad word is skipped
+    assert_f32_bits_equal(got, want)
+    B.adacomp_device_status_reset()
+    assert B.adacomp_device_status() == 0
+
+
+def test_nonfinite_gradient_sets_a_status_bit_and_returns():
+    n = 8000
+    dW = np.full(n, 1e-3, np.float32)
+    dW[17] = np.inf
+    dW[4100] = np.nan
+    B.adacomp_device_status_reset()
+    GpuLayer(n, 50).compress(dW)
+    assert B.adacomp_device_status() & B.ADACOMP_DEV_NONFINITE
+    B.adacomp_device_status_reset()
+
+
+def test_multi_tensor_calls_match_single_calls():
+    specs = synth.resnet50_tensors()[:30]
+    dev = torch.device("cuda:0")
+    layers, singles, dws = [], [], []
+    for t, spec in enumerate(specs):
+        dW = synth.make_dw(3, 0, t, 0, spec.n, heavy=True)
+        dws.append(dW)
+        L = GpuLayer(spec.n, spec.L_T)
+        L.grad[:spec.n].copy_(torch.from_numpy(dW))
+        layers.append(L)
+    descs = [dict(grad=L.grad, residue=L.residue, n=L.n, L_T=L.L_T, packed_out=L.packed,
+                  count_out=L.count) for L in layers]
+    B.adacomp_compress_multi(descs, len(descs))
+    torch.cuda.synchronize()
+    for t, (L, spec) in enumerate(zip(layers, specs)):
+        r = np.zeros(spec.n, np.float32)
+        want = cref.pack(dws[t], r, spec.L_T)
+        used = int(L.count[1])
+        assert_stream_equal(L.packed[:used].cpu().numpy(), want, f"tensor {t}")
+        assert_f32_bits_equal(L.residue_host(), r)
+    # decode every layer from two "learners" (the same stream twice) in one call
+    dsts = [torch.empty(max(L.n, 4), dtype=torch.float32, device=dev) for L in layers]
+    packed = [p for L in layers for p in (L.packed, L.packed)]
+    B.adacomp_decompress_accumulate_multi(packed, 2, dsts, len(layers))
+    torch.cuda.synchronize()
+    for t, L in enumerate(layers):
+        used = int(L.count[1])
+        raw = L.packed[:used].cpu().numpy()
+        assert_f32_bits_equal(dsts[t][:L.n].cpu().numpy(), cref.unpack_sum([raw, raw], L.n))
