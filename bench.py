@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the AdaComp hot path on B200: k learners' pack() + one unpack()-and-sum.
+
+One step = every learner compresses its own seeded gradient of n fp32 elements
+(residue pre-warmed by 5 steps and restored, untimed, before each step so that
+every repetition is "step 6" on identical data), then the k packed streams are
+decode-summed into one dense gradient.  Prints ONE JSON line (rank 0).
+
+  python bench.py                      # 1 GPU, n = 2^30, L_T = 50, 4 learners
+  python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 \
+         --master-port P bench.py --gpus N          # N independent ranks (weak scaling)
+  python bench.py --impl reference     # the CPU oracle on a bounded sample of the workload
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compress+pack GB/s of fp32 gradient"
+SIGMA = 1e-3
+PREWARM_STEPS = 5
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--log2n", type=int, default=30, help="elements per learner = 2^log2n")
+    ap.add_argument("--L_T", type=int, default=50)
+    ap.add_argument("--learners", type=int, default=4)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def workload_name(a):
+    return (f"bandwidth sweep point: flat fp32 gradient n=2^{a.log2n}, L_T={a.L_T}, "
+            f"dW~N(0,1e-3), residue pre-warmed {PREWARM_STEPS} steps, {a.learners} learners' "
+            f"streams decode-summed")
+
+
+# ----------------------------------------------------------------------------------
+# reference arm / cpu_baseline: the oracle as it stands, on a bounded sample
+# ----------------------------------------------------------------------------------
+
+def oracle_sample(a, steps, warmup):
+    """Times oracle pack() for `learners` learners plus one unpack-sum per step on a
+    sample of 2^cpu_log2n elements with the workload's distribution.  Single thread."""
+    import numpy as np
+    from oracle import cref
+
+    n = 1 << min(a.cpu_log2n, a.log2n)
+    k = a.learners
+    rng = np.random.default_rng(np.random.SeedSequence([1712, 2679, 5, 777]))
+    draw = lambda: (rng.standard_normal(n, dtype=np.float32) * np.float32(SIGMA))
+    residues = [np.zeros(n, np.float32) for _ in range(k)]
+    prewarm = 2                       # bounded: fewer pre-warm steps than the GPU arm's 5
+    for _ in range(prewarm):
+        for r in residues:
+            cref.pack(draw(), r, a.L_T)
+    dws = [draw() for _ in range(k)]
+    snaps = [r.copy() for r in residues]
+    t_pack, t_sum, t_step = [], [], []
+    for it in range(warmup + steps):
+        for r, s in zip(residues, snaps):
+            r[:] = s
+        t0 = time.perf_counter()
+        streams = [cref.pack(dws[l], residues[l], a.L_T).raw for l in range(k)]
+        t1 = time.perf_counter()
+        cref.unpack_sum(streams, n)
+        t2 = time.perf_counter()
+        if it >= warmup:
+            t_pack.append(t1 - t0)
+            t_sum.append(t2 - t1)
+            t_step.append(t2 - t0)
+    grad_bytes = 4.0 * n * k
+    return {
+        "n": n, "k": k,
+        "step_s": statistics.mean(t_step),
+        "step_gbs": grad_bytes / statistics.mean(t_step) / 1e9,
+        "pack_gbs": grad_bytes / statistics.mean(t_pack) / 1e9,
+        "sum_gbs": 4.0 * n / statistics.mean(t_sum) / 1e9,
+        "sample": (f"n=2^{n.bit_length() - 1} of the workload's 2^{a.log2n} elements per learner, "
+                   f"{k} learners, L_T={a.L_T}, residue pre-warmed {prewarm} steps, "
+                   f"{steps} timed steps after {warmup} warm-up"),
+    }
+
+
+def run_reference(a):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = min(a.steps, 3), min(a.warmup, 1)
+    r = oracle_sample(a, steps, warmup)
+    line = {
+        "impl": "reference",
+        "metric": METRIC, "value": r["step_gbs"], "unit": "GB/s",
+        "n_gpus": a.gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": 1e3 * r["step_s"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(a), "sampled": r["sample"]},
+        "cpu_baseline": {"value": r["step_gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": r["sample"], "pack_gbs": r["pack_gbs"],
+                         "unpack_sum_gbs": r["sum_gbs"]},
+        "e2e": {"value": r["step_gbs"], "unit": "GB/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------
+
+def run_ours(a):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1712_02679_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n, L_T, k = 1 << a.log2n, a.L_T, a.learners
+    K, W = a.steps, max(a.warmup, 3)
+    stream = torch.cuda.current_stream()
+
+    # ---- the workload: seeded on the device (host numpy needs ~15 s per 2^30 normals) ----
+    gen = torch.Generator(device=dev)
+    cap = B.adacomp_packed_capacity(n, L_T)
+    residue = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(k)]
+    packed = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(k)]
+    count = [torch.zeros(2, dtype=torch.int64, device=dev) for _ in range(k)]
+    dW = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(k)]
+    dst = torch.empty(n, dtype=torch.float32, device=dev)
+    for step in range(PREWARM_STEPS + 1):
+        for l in range(k):
+            gen.manual_seed(1712_02679 + 1000003 * rank + 1009 * l + step)
+            dW[l].normal_(0.0, SIGMA, generator=gen)
+            if step < PREWARM_STEPS:
+                B.adacomp_compress(dW[l], residue[l], n, L_T, packed[l], count[l], stream)
+    snap = [r.clone() for r in residue]
+    torch.cuda.synchronize()
+
+    def restore():
+        for r, s in zip(residue, snap):
+            r.copy_(s)
+
+    def step_events():
+        return [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+
+    # ---- timed region: device-resident inputs ----
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    evs = []
+    for it in range(W + K):
+        if it == W:
+            barrier()
+            if rank == 0:
+                sampler.start()
+        restore()
+        e = step_events()
+        e[0].record(stream)
+        for l in range(k):
+            B.adacomp_compress(dW[l], residue[l], n, L_T, packed[l], count[l], stream)
+        e[1].record(stream)
+        B.adacomp_decompress_accumulate(packed, k, dst, stream)
+        e[2].record(stream)
+        if it >= W:
+            evs.append(e)
+    barrier()
+    t_comp = [e[0].elapsed_time(e[1]) for e in evs]
+    t_dec = [e[1].elapsed_time(e[2]) for e in evs]
+    t_total_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
+
+    # ---- per-kernel durations of pack() (learner 0), same protocol, CUDA events ----
+    prof = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    for row in prof:
+        for e in row:
+            e.record(stream)           # creates the handles
+    for row in prof:
+        restore()
+        B.adacomp_compress_profile(dW[0], residue[0], n, L_T, packed[0], count[0], stream, 0, row)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    t_tile = statistics.mean(r[0].elapsed_time(r[1]) for r in prof)
+    t_fin = statistics.mean(r[1].elapsed_time(r[2]) for r in prof)
+    t_fix = statistics.mean(r[2].elapsed_time(r[3]) for r in prof)
+
+    status = B.adacomp_device_status(stream)
+    counts = [tuple(int(v) for v in c.cpu()) for c in count]
+    n_sel = [c[0] for c in counts]
+    used = [c[1] for c in counts]
+    w = 1 if L_T <= 64 else 2
+    n_bins = -(-n // L_T)
+    tile_bins = 4 * (1000 // L_T) if L_T <= 1000 else 1
+    n_tiles = -(-n_bins // tile_bins)
+
+    # ---- end to end through the host-buffer entry points ----
+    e2e = None
+    if not a.no_e2e:
+        Ke = max(1, min(K, 3))
+        h_dW = [torch.empty(n, dtype=torch.float32, pin_memory=True) for _ in range(k)]
+        for l in range(k):
+            h_dW[l].copy_(dW[l])
+        h_packed = [torch.empty(used[l] + (1 << 20), dtype=torch.uint8, pin_memory=True) for l in range(k)]
+        h_count = [torch.zeros(2, dtype=torch.int64, pin_memory=True) for _ in range(k)]
+        h_dst = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        stage = torch.empty(n, dtype=torch.float32, device=dev)
+        torch.cuda.synchronize()
+        spans = []
+        for it in range(1 + Ke):
+            restore()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for l in range(k):
+                B.adacomp_compress_host(h_dW[l], stage, residue[l], n, L_T, packed[l], count[l],
+                                        h_packed[l], h_count[l], stream)
+            nbytes = [int(c[1]) for c in h_count]
+            B.adacomp_decompress_accumulate_host(h_packed, nbytes, packed, k, dst, h_dst, n, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if it >= 1:
+                spans.append(e0.elapsed_time(e1))
+        e2e_ms = statistics.mean(spans)
+        e2e = {"ms": e2e_ms, "h2d": 4 * n * k + sum(used), "d2h": sum(used) + 16 * k + 4 * n,
+               "steps": Ke}
+        del h_dW, h_packed, h_dst, stage
+
+    # ---- max over ranks ----
+    if world > 1:
+        t = torch.tensor([t_total_ms, statistics.mean(t_comp), statistics.mean(t_dec),
+                          e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_total_ms, m_comp, m_dec, e2e_ms = (float(x) for x in t.cpu())
+        if e2e:
+            e2e["ms"] = e2e_ms
+    else:
+        m_comp, m_dec = statistics.mean(t_comp), statistics.mean(t_dec)
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        ms_per_step = t_total_ms / K
+        grad_bytes = 4.0 * n * k * world
+        value = grad_bytes / (ms_per_step * 1e-3) / 1e9
+        tile_bytes = 12.0 * n + n_bins * w + n_sel[0] * w + 8.0 * n_tiles
+        achieved = tile_bytes / (t_tile * 1e-3) / 1e9
+        call_bytes = [12.0 * n + u for u in used]
+        comp_frac = sum(call_bytes) / (m_comp * 1e-3) / 1e9 / peak
+        dec_bytes = 4.0 * n + sum(used)
+        dec_frac = dec_bytes / (m_dec * 1e-3) / 1e9 / peak
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": workload_name(a), "n": n, "L_T": L_T, "learners_per_gpu": k,
+                "l2": "no flush needed: each array is %.1f GiB, far beyond the 126 MB L2" % (4.0 * n / 2 ** 30)
+                      if 4 * n > (1 << 29) else "arrays are not much larger than L2: numbers are L2-assisted",
+                "timing": "sum over steps of the CUDA-event span [first pack launch, end of decode-sum]; "
+                          "residues restored from a snapshot between steps outside the span",
+                "step": "k x adacomp_compress + 1 x adacomp_decompress_accumulate",
+            },
+            "compress_gbs": 4.0 * n * k * world / (m_comp * 1e-3) / 1e9,
+            "decompress_sum_gbs": 4.0 * n * world / (m_dec * 1e-3) / 1e9,
+            "hbm_frac_compress_call": comp_frac,
+            "hbm_frac_decompress_sum": dec_frac,
+            "pack_kernels_ms": {"tile_pass": t_tile, "finalize": t_fin, "gather_fixup": t_fix},
+            "selected_fraction": n_sel[0] / n, "bytes_used": used[0], "device_status": status,
+            "roofline": {"bound": "hbm", "kernel": "tile_pass", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": tile_bytes},
+            "clocks": clocks,
+            "gpu_launches": K * (3 * k + 1),
+        }
+        if e2e:
+            line["e2e"] = {"value": grad_bytes / (e2e["ms"] * 1e-3) / 1e9, "unit": "GB/s",
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": e2e["ms"], "steps": e2e["steps"]}
+        if not a.no_cpu:
+            r = oracle_sample(a, 2, 1)
+            line["cpu_baseline"] = {"value": r["step_gbs"], "unit": "GB/s", "cores": 1,
+                                    "kind": "oracle", "sample": r["sample"],
+                                    "pack_gbs": r["pack_gbs"], "unpack_sum_gbs": r["sum_gbs"]}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
+
+
+if __name__ == "__main__":
+    main()

@@ -127,6 +127,41 @@ int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t 
 int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams, float *dst,
                                   void *stream);
 
+/*
+ * adacomp_compress_ex with four caller-created cudaEvent_t handles (HOST array, as
+ * void*) recorded on `stream` around the three kernels of pack(): events[0] before and
+ * events[1] after the tile pass, events[2] after the scale/scan kernel, events[3] after
+ * the gather / residue fix-up.  For measurement; the results are those of
+ * adacomp_compress_ex.  The paper reports no timing of pack() (Section "Experiments").
+ */
+int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T,
+                             void *packed_out, uint64_t *count_out, void *stream, uint32_t flags,
+                             void *const *events);
+
+/*
+ * pack() for a gradient that lives in HOST memory (Algorithm 1: serializeGrad() ->
+ * pack() -> exchange()).  Copies grad_host[n] (pinned memory advised) to the device
+ * staging buffer grad_stage[n], runs adacomp_compress on it, then copies count_dev to
+ * count_host[2] and the first bytes_used bytes of packed_dev to packed_host.
+ * UNLIKE the other calls this one synchronises `stream` before it returns.
+ * packed_host_cap smaller than bytes_used returns ADACOMP_ERR_SIZE (residue is then
+ * already updated).  residue, packed_dev, count_dev: as in adacomp_compress.
+ */
+int adacomp_compress_host(const float *grad_host, float *grad_stage, float *residue, uint64_t n,
+                          uint32_t L_T, void *packed_dev, uint64_t *count_dev, void *packed_host,
+                          uint64_t packed_host_cap, uint64_t *count_host, void *stream);
+
+/*
+ * unpack()-and-sum for streams received into HOST memory (Algorithm 1: exchange() ->
+ * unpack() -> averageGradients()).  Copies packed_host[l][0 .. packed_bytes[l]) to the
+ * device buffers packed_stage[l] (all three are HOST arrays of k entries), runs
+ * adacomp_decompress_accumulate into dst_dev[n] and copies it to dst_host[n].
+ * Synchronises `stream` before it returns.
+ */
+int adacomp_decompress_accumulate_host(const void *const *packed_host, const uint64_t *packed_bytes,
+                                       void *const *packed_stage, uint32_t k_streams, float *dst_dev,
+                                       float *dst_host, uint64_t n, void *stream);
+
 /* One tensor of a multi-tensor call; every tensor is its own layer (own bins, own scale). */
 typedef struct {
     const float *grad;

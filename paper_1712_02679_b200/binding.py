@@ -62,6 +62,16 @@ def lib() -> C.CDLL:
         L.adacomp_compress_ex.argtypes = L.adacomp_compress.argtypes + [C.c_uint32]
         L.adacomp_decompress_accumulate.restype = C.c_int
         L.adacomp_decompress_accumulate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.adacomp_compress_profile.restype = C.c_int
+        L.adacomp_compress_profile.argtypes = L.adacomp_compress_ex.argtypes + [C.c_void_p]
+        L.adacomp_compress_host.restype = C.c_int
+        L.adacomp_compress_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                            C.c_void_p, C.c_void_p]
+        L.adacomp_decompress_accumulate_host.restype = C.c_int
+        L.adacomp_decompress_accumulate_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p,
+                                                         C.c_uint32, C.c_void_p, C.c_void_p,
+                                                         C.c_uint64, C.c_void_p]
         L.adacomp_compress_multi.restype = C.c_int
         L.adacomp_compress_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.adacomp_decompress_accumulate_multi.restype = C.c_int
@@ -139,6 +149,56 @@ def adacomp_decompress_accumulate(packed: Sequence[torch.Tensor], k_streams: int
     _check(lib().adacomp_decompress_accumulate(ptrs, int(k_streams),
                                                _dev_ptr(dst, "dst", torch.float32), _stream(stream)),
            "adacomp_decompress_accumulate")
+
+
+def adacomp_compress_profile(grad, residue, n: int, L_T: int, packed_out, count_out, stream=None,
+                             flags: int = 0, events: Sequence[torch.cuda.Event] = ()) -> None:
+    """adacomp_compress_ex with four torch CUDA events (already recorded once, so that
+    their handles exist) recorded around the three kernels."""
+    assert len(events) == 4
+    handles = (C.c_void_p * 4)(*[int(e.cuda_event) for e in events])
+    _check(lib().adacomp_compress_profile(_dev_ptr(grad, "grad", torch.float32),
+                                          _dev_ptr(residue, "residue", torch.float32), int(n),
+                                          int(L_T), _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                          _dev_ptr(count_out, "count_out", torch.int64),
+                                          _stream(stream), int(flags), handles),
+           "adacomp_compress_profile")
+
+
+def _host_ptr(t: torch.Tensor, what: str, dtype) -> int:
+    if t.is_cuda or not t.is_contiguous() or t.dtype != dtype:
+        raise ValueError(f"{what} must be a contiguous host tensor of dtype {dtype}")
+    return t.data_ptr()
+
+
+def adacomp_compress_host(grad_host, grad_stage, residue, n: int, L_T: int, packed_dev, count_dev,
+                          packed_host, count_host, stream=None) -> None:
+    """pack() of a host-resident gradient; synchronises.  count_host: int64[2] host tensor."""
+    _check(lib().adacomp_compress_host(_host_ptr(grad_host, "grad_host", torch.float32),
+                                       _dev_ptr(grad_stage, "grad_stage", torch.float32),
+                                       _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                       _dev_ptr(packed_dev, "packed_dev", torch.uint8),
+                                       _dev_ptr(count_dev, "count_dev", torch.int64),
+                                       _host_ptr(packed_host, "packed_host", torch.uint8),
+                                       packed_host.numel(),
+                                       _host_ptr(count_host, "count_host", torch.int64),
+                                       _stream(stream)),
+           "adacomp_compress_host")
+
+
+def adacomp_decompress_accumulate_host(packed_host: Sequence[torch.Tensor],
+                                       packed_bytes: Sequence[int],
+                                       packed_stage: Sequence[torch.Tensor], k_streams: int,
+                                       dst_dev, dst_host, n: int, stream=None) -> None:
+    """unpack()-and-sum of host-resident streams into dst_host; synchronises."""
+    k = int(k_streams)
+    hp = (C.c_void_p * max(k, 1))(*[_host_ptr(p, "packed_host[l]", torch.uint8) for p in packed_host[:k]])
+    nb = (C.c_uint64 * max(k, 1))(*[int(b) for b in packed_bytes[:k]])
+    sp = (C.c_void_p * max(k, 1))(*[_dev_ptr(p, "packed_stage[l]", torch.uint8) for p in packed_stage[:k]])
+    _check(lib().adacomp_decompress_accumulate_host(hp, nb, sp, k, _dev_ptr(dst_dev, "dst_dev", torch.float32),
+                                                    _host_ptr(dst_host, "dst_host", torch.float32),
+                                                    int(n), _stream(stream)),
+           "adacomp_decompress_accumulate_host")
 
 
 def make_layer_descs(layers: Sequence[dict]):

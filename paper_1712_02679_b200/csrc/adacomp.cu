@@ -764,7 +764,7 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 }
 
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
-                  uint64_t *count_out, void *stream, uint32_t flags)
+                  uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
@@ -782,7 +782,9 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     unsigned char *packed = static_cast<unsigned char *>(packed_out);
 
     if (cudaMemsetAsync(packed + geo.ctl_at, 0, kCtlBytes, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
+    auto mark = [&](int i) { if (events) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st); };
 
+    mark(0);
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, geo, flags & ADACOMP_FLAG_LITERAL};
         const bool fast = (L_T == 50u || L_T == 500u) && !(flags & ADACOMP_FLAG_GENERIC_PATH);
@@ -803,13 +805,16 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
             if (rc != ADACOMP_OK) return rc;
         }
     }
+    mark(1);
     finalize<<<1, 1024, 0, st>>>(packed, geo, flags, reinterpret_cast<u64 *>(count_out));
+    mark(2);
     if (geo.n_tiles) {
         const u64 cap = (u64)info.sms * 8;
         const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
         if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
         else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
     }
+    mark(3);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
@@ -883,6 +888,54 @@ int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t 
 int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams, float *dst, void *stream)
 {
     return decompress_impl(packed, k_streams, dst, stream);
+}
+
+int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                             uint64_t *count_out, void *stream, uint32_t flags, void *const *events)
+{
+    if (!events) return ADACOMP_ERR_NULL;
+    for (int i = 0; i < 4; i++)
+        if (!events[i]) return ADACOMP_ERR_NULL;
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, flags, events);
+}
+
+int adacomp_compress_host(const float *grad_host, float *grad_stage, float *residue, uint64_t n, uint32_t L_T,
+                          void *packed_dev, uint64_t *count_dev, void *packed_host, uint64_t packed_host_cap,
+                          uint64_t *count_host, void *stream)
+{
+    if (!count_host || !packed_host || (n && (!grad_host || !grad_stage))) return ADACOMP_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n && cudaMemcpyAsync(grad_stage, grad_host, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return ADACOMP_ERR_CUDA;
+    int rc = compress_impl(grad_stage, residue, n, L_T, packed_dev, count_dev, stream, 0);
+    if (rc != ADACOMP_OK) return rc;
+    if (cudaMemcpyAsync(count_host, count_dev, 2 * sizeof(uint64_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return ADACOMP_ERR_CUDA;
+    if (count_host[1] > packed_host_cap) return ADACOMP_ERR_SIZE;
+    if (cudaMemcpyAsync(packed_host, packed_dev, count_host[1], cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return ADACOMP_ERR_CUDA;
+    return ADACOMP_OK;
+}
+
+int adacomp_decompress_accumulate_host(const void *const *packed_host, const uint64_t *packed_bytes,
+                                       void *const *packed_stage, uint32_t k_streams, float *dst_dev,
+                                       float *dst_host, uint64_t n, void *stream)
+{
+    if (!packed_host || !packed_bytes || !packed_stage || !dst_dev || (n && !dst_host)) return ADACOMP_ERR_NULL;
+    if (k_streams == 0 || k_streams > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (uint32_t l = 0; l < k_streams; l++) {
+        if (!packed_host[l] || !packed_stage[l]) return ADACOMP_ERR_NULL;
+        if (cudaMemcpyAsync(packed_stage[l], packed_host[l], packed_bytes[l], cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return ADACOMP_ERR_CUDA;
+    }
+    int rc = decompress_impl(packed_stage, k_streams, dst_dev, stream);
+    if (rc != ADACOMP_OK) return rc;
+    if (n && cudaMemcpyAsync(dst_host, dst_dev, n * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ADACOMP_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
 int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream)
