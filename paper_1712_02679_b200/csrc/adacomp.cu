@@ -4,9 +4,10 @@
 //   tile_pass     one read of dW and residue, one write of residue (= G everywhere);
 //                 per-bin max |G|, selection, words compacted per tile into a scratch
 //                 slot, per-bin counts, per-tile counts, exact partial sums of g_max
-//   finalize      exact sum -> scale, scan of the tile counts, header, count_out
-//   gather_fixup  moves each tile's words to their final place and subtracts
-//                 sign * scale from the residue of the sent elements only
+//   finalize      exact sum -> scale, scan of the tile-group counts, header, count_out
+//   gather_fixup  moves each tile's words to their final place, writes the tile
+//                 directory, and subtracts sign * scale from the residue of the sent
+//                 elements only
 // The layer-wide scale (Section 2.5: mean of the g_max vector) is needed by every
 // sent element's residue but is known only after every bin has been seen; that is
 // why the residue of sent elements is finished by the third kernel.
@@ -14,7 +15,10 @@
 // unpack()-and-sum is one kernel: each CTA owns an output tile in shared memory,
 // adds the k learners' words into it in learner order and stores it once.
 //
-// HBM-bandwidth bound; no tensor cores (nothing here is a contraction).
+// HBM-bandwidth bound; no tensor cores (nothing here is a contraction).  The fast
+// tile pass (L_T = 50 and 500) is a persistent kernel fed by 1-D bulk copies (TMA)
+// through a three-stage shared-memory ring guarded by mbarriers; every wait on a
+// barrier is bounded and reports ADACOMP_DEV_TIMEOUT instead of spinning forever.
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -30,15 +34,21 @@ constexpr u32 kMagic = 0x31434441u;
 constexpr u32 kHeaderBytes = 64;
 constexpr u32 kCtlBytes = 256;       // control block at the start of the scratch area
 constexpr int kWindows = 9;          // 32-bit windows of the exact g_max accumulator
+constexpr int kGroupTiles = 32;      // tiles per group of the two-level count scan
 constexpr int kSeg = 25;             // elements per thread on the fast path
 constexpr int kTileSegs = 160;       // segments per tile on the fast path
 constexpr int kFastTile = kSeg * kTileSegs;   // 4000 elements
-constexpr int kFastThreads = 192;
+constexpr int kFastThreads = 192;    // 5 compute warps + 1 service warp
+constexpr int kStages = 3;
+constexpr u32 kTileBytes = kFastTile * 4;     // 16000
+constexpr u32 kStageBytes = 2 * kTileBytes;   // dW + residue
 constexpr int kGenericThreads = 256;
 constexpr int kDecodeChunk = 4096;   // output elements per decode work item
-constexpr int kDecodeThreads = 256;
+constexpr int kDecodeThreads = 128;
 constexpr int kGatherThreads = 128;
 constexpr int kMaxTileBins = 4000;
+constexpr int kSmallBins = 96;       // tiles with at most this many bins take the fast decode / gather
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: bound of every device-side wait
 
 __device__ u32 g_status;             // sticky ADACOMP_DEV_* bits of this device
 
@@ -47,8 +57,9 @@ __host__ __device__ inline u64 align_up(u64 x, u64 a) { return (x + a - 1) / a *
 // Section offsets of a packed stream and of the scratch behind it.
 struct Geometry {
     u32 w, L_T, tile_bins, tile_elems;
-    u64 n, n_bins, n_tiles;
-    u64 tile_off_at, bin_cnt_at, payload_at, ctl_at, slots_at, slot_bytes, capacity;
+    u64 n, n_bins, n_tiles, n_groups;
+    u64 tile_off_at, bin_cnt_at, payload_at;                             // the stream
+    u64 ctl_at, group_at, tile_cnt_at, slots_at, slot_bytes, capacity;   // scratch
 };
 
 __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
@@ -61,11 +72,14 @@ __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
     g.tile_elems = g.tile_bins * L_T;
     g.n_bins = (n + L_T - 1) / L_T;
     g.n_tiles = (g.n_bins + g.tile_bins - 1) / g.tile_bins;
+    g.n_groups = (g.n_tiles + kGroupTiles - 1) / kGroupTiles;
     g.tile_off_at = kHeaderBytes;
     g.bin_cnt_at = align_up(g.tile_off_at + 8 * (g.n_tiles + 1), 16);
     g.payload_at = align_up(g.bin_cnt_at + g.n_bins * g.w, 16);
     g.ctl_at = align_up(g.payload_at + align_up(n * g.w, 16), 256);
-    g.slots_at = g.ctl_at + kCtlBytes;
+    g.group_at = g.ctl_at + kCtlBytes;                         // u64[n_groups], zeroed per call
+    g.tile_cnt_at = g.group_at + 8 * g.n_groups;               // u32[n_tiles]
+    g.slots_at = align_up(g.tile_cnt_at + 4 * g.n_tiles, 256);
     g.slot_bytes = align_up((u64)g.tile_elems * g.w, 16);
     g.capacity = g.slots_at + g.n_tiles * g.slot_bytes;
     return g;
@@ -77,6 +91,16 @@ __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
 
 __device__ inline void raise_status(u32 bits) { atomicOr(&g_status, bits); }
 
+__device__ inline u32 warp_inclusive_scan(u32 v, int lane)
+{
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const u32 t = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += t;
+    }
+    return v;
+}
+
 // Exclusive scan, in place, of a[0..count) in shared memory; a[count] receives the total.
 // Called by every thread of the CTA; contains barriers.
 __device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* >= 33 */)
@@ -86,29 +110,20 @@ __device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* 
     const int lo = min(tid * per, count), hi = min(lo + per, count);
     u32 sum = 0;
     for (int i = lo; i < hi; i++) sum += a[i];
-    // scan of the per-thread sums: warp shuffles, then the warp totals
     const int lane = tid & 31, warp = tid >> 5, nwarp = (nthr + 31) >> 5;
-    u32 inc = sum;
-    for (int d = 1; d < 32; d <<= 1) {
-        u32 t = __shfl_up_sync(0xffffffffu, inc, d);
-        if (lane >= d) inc += t;
-    }
+    const u32 inc = warp_inclusive_scan(sum, lane);
     if (lane == 31) warp_tmp[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        u32 v = lane < nwarp ? warp_tmp[lane] : 0u;
-        u32 s = v;
-        for (int d = 1; d < 32; d <<= 1) {
-            u32 t = __shfl_up_sync(0xffffffffu, s, d);
-            if (lane >= d) s += t;
-        }
+        const u32 v = lane < nwarp ? warp_tmp[lane] : 0u;
+        const u32 s = warp_inclusive_scan(v, lane);
         warp_tmp[lane] = s - v;
         if (lane == 31) warp_tmp[32] = s;
     }
     __syncthreads();
     u32 run = warp_tmp[warp] + inc - sum;
     for (int i = lo; i < hi; i++) {
-        u32 v = a[i];
+        const u32 v = a[i];
         a[i] = run;
         run += v;
     }
@@ -121,7 +136,7 @@ __device__ inline int bin_of_word(const u32 *prefix, int bins, u32 j)
 {
     int lo = 0, hi = bins;           // invariant: prefix[lo] <= j < prefix[hi]
     while (hi - lo > 1) {
-        int mid = (lo + hi) >> 1;
+        const int mid = (lo + hi) >> 1;
         if (prefix[mid] <= j) lo = mid; else hi = mid;
     }
     return lo;
@@ -169,11 +184,76 @@ __device__ inline void warp_accumulate(u64 *acc, float gm, bool valid)
     __syncwarp();
 }
 
+// ---- mbarrier / bulk-copy (TMA) wrappers; no cluster multicast anywhere ----
+
+__device__ inline u32 smem_addr(const void *p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(u64 *bar, u32 arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+
+__device__ inline void mbar_arrive_expect_tx(u64 *bar, u32 bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ inline bool mbar_try_wait(u64 *bar, u32 parity)
+{
+    u32 ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ inline bool mbar_wait(u64 *bar, u32 parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
+__device__ inline void bulk_load(void *smem_dst, const void *gmem_src, u32 bytes, u64 *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+                     "r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+__device__ inline void bulk_store(void *gmem_dst, const void *smem_src, u32 bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst),
+                 "r"(smem_addr(smem_src)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ inline void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ inline void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------------
 // tile_pass, fast path: L_T = 25 * SPB (50 and 500), tiles of 4000 elements.
+//
 // Thread t < 160 owns the 25 consecutive elements of segment t (stride 25 words in
-// shared memory: odd, so the warp's accesses are bank-conflict free); a bin is SPB
-// adjacent segments.  Warp 5 has no segment: it feeds the exact g_max accumulator.
+// shared memory: odd, so a warp's accesses are bank-conflict free); a bin is SPB
+// adjacent segments.  Warp 5 (the service warp) owns no segment: its lane 0 issues
+// every bulk copy, and the warp feeds the exact g_max accumulator and copies the
+// tile's words to the scratch slot.
+//
+// Ring: tile i of this CTA lives in stage i % 3.  Loads for tile i + 2 are issued
+// during tile i, after the bulk store that drained that stage (tile i - 1) has
+// finished reading shared memory.
 // ---------------------------------------------------------------------------------
 
 struct PassArgs {
@@ -184,155 +264,214 @@ struct PassArgs {
     u32 literal;
 };
 
+struct FastSmem {
+    static constexpr u32 kWordsAt = kStages * kStageBytes;            // 96000
+    static constexpr u32 kInclAt = kWordsAt + 2 * kFastTile;          // + 8000 (16-bit words)
+    static constexpr u32 kWtotAt = kInclAt + 4 * kTileSegs;
+    static constexpr u32 kSegmaxAt = kWtotAt + 4 * 8;
+    static constexpr u32 kBinmaxAt = kSegmaxAt + 4 * kTileSegs;
+    static constexpr u32 kAccAt = kBinmaxAt + 4 * 80;                 // 8-byte aligned
+    static constexpr u32 kBarAt = kAccAt + 8 * (kWindows + 1);
+    static constexpr u32 kAbortAt = kBarAt + 8 * kStages;
+    static constexpr u32 kBytes = kAbortAt + 16;
+};
+static_assert(FastSmem::kAccAt % 8 == 0, "accumulator must be 8-byte aligned");
+
 template <int SPB, typename Word>
-__global__ void __launch_bounds__(kFastThreads)
+__global__ void __launch_bounds__(kFastThreads, 2)
 tile_pass_fast(PassArgs a)
 {
-    __shared__ __align__(16) float s_d[kFastTile];     // dW, later the word staging area
-    __shared__ __align__(16) float s_r[kFastTile];     // residue, later G
-    __shared__ float s_segmax[kTileSegs];
-    __shared__ u32 s_off[kTileSegs + 1];
-    __shared__ u64 s_acc[kWindows + 1];
+    extern __shared__ __align__(128) unsigned char smem[];
+    Word *s_words = reinterpret_cast<Word *>(smem + FastSmem::kWordsAt);
+    u32 *s_incl = reinterpret_cast<u32 *>(smem + FastSmem::kInclAt);
+    u32 *s_wtot = reinterpret_cast<u32 *>(smem + FastSmem::kWtotAt);
+    float *s_segmax = reinterpret_cast<float *>(smem + FastSmem::kSegmaxAt);
+    float *s_binmax = reinterpret_cast<float *>(smem + FastSmem::kBinmaxAt);
+    u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
+    u64 *s_full = reinterpret_cast<u64 *>(smem + FastSmem::kBarAt);
+    volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FastSmem::kAbortAt);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool service = warp == 5;
     const Geometry &geo = a.geo;
     constexpr int kBins = kTileSegs / SPB;
-    u64 *tile_cnt = reinterpret_cast<u64 *>(a.packed + geo.tile_off_at);
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
-    Word *s_words = reinterpret_cast<Word *>(s_d);
+    u32 *tile_cnt = reinterpret_cast<u32 *>(a.packed + geo.tile_cnt_at);
+    u64 *group_cnt = reinterpret_cast<u64 *>(a.packed + geo.group_at);
+
+    // tiles of this CTA: blockIdx.x + i * gridDim.x
+    const u64 first = blockIdx.x, stride = gridDim.x;
+    const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
+    const u64 full_tiles = geo.n / kFastTile;       // tiles below this index are complete
 
     if (tid < kWindows + 1) s_acc[tid] = 0;
+    if (tid == 0) {
+        *s_abort = 0;
+        for (int s = 0; s < kStages; s++) mbar_init(&s_full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
-    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
+    u64 issued = 0;                     // service lane 0: loads issued for tiles [0, issued)
+    auto issue_load = [&](u64 i) {
+        const u64 tile = first + i * stride;
+        if (i >= my_tiles || tile >= full_tiles) return;
+        unsigned char *st = smem + (i % kStages) * kStageBytes;
+        u64 *bar = &s_full[i % kStages];
+        mbar_arrive_expect_tx(bar, kStageBytes);
+        bulk_load(st, a.grad + tile * (u64)kFastTile, kTileBytes, bar);
+        bulk_load(st + kTileBytes, a.residue + tile * (u64)kFastTile, kTileBytes, bar);
+        issued = i + 1;
+    };
+    if (service && lane == 0) {
+        issue_load(0);
+        issue_load(1);
+    }
+
+    u64 i = 0;
+    for (; i < my_tiles; i++) {
+        const u64 tile = first + i * stride;
         const u64 base = tile * (u64)kFastTile;
-        const u64 left = geo.n - base;
-        const int elems = left < (u64)kFastTile ? (int)left : kFastTile;
+        float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
+        float *s_r = s_d + kFastTile;
+        const bool whole = tile < full_tiles;
+        const int elems = whole ? kFastTile : (int)(geo.n - base);
 
-        // ---- load the tile (128-bit, coalesced; zero fill past the end) ----
-        const float4 *gd = reinterpret_cast<const float4 *>(a.grad + base);
-        const float4 *gr = reinterpret_cast<const float4 *>(a.residue + base);
-        for (int i = tid; i < kFastTile / 4; i += kFastThreads) {
-            float4 d = make_float4(0.f, 0.f, 0.f, 0.f), r = d;
-            if (4 * i + 3 < elems) {
-                d = __ldcs(gd + i);
-                r = __ldcs(gr + i);
-            } else {
-                float *pd = &d.x, *pr = &r.x;
-                for (int c = 0; c < 4; c++)
-                    if (4 * i + c < elems) {
-                        pd[c] = a.grad[base + 4 * i + c];
-                        pr[c] = a.residue[base + 4 * i + c];
-                    }
+        if (whole) {
+            if (!mbar_wait(&s_full[i % kStages], (u32)(i / kStages) & 1u)) {
+                *s_abort = 1;                      // every thread that times out says so
+                raise_status(ADACOMP_DEV_TIMEOUT);
             }
-            reinterpret_cast<float4 *>(s_d)[i] = d;
-            reinterpret_cast<float4 *>(s_r)[i] = r;
+        } else {
+            // the ragged last tile of the tensor: plain loads, zero fill past the end
+            for (int e = tid; e < kFastTile; e += kFastThreads) {
+                float d = 0.f, r = 0.f;
+                if (e < elems) { d = a.grad[base + e]; r = a.residue[base + e]; }
+                s_d[e] = d;
+                s_r[e] = r;
+            }
+            __syncthreads();
         }
-        __syncthreads();
 
-        // ---- G = residue + dW; maximum |G| of the segment ----
-        float g[kSeg];
-        if (tid < kTileSegs) {
+        // ---- G = residue + dW, H = G + dW; the segment's maximum |G| ----
+        float g[kSeg], key[kSeg];
+        float gm = 0.f;
+        u32 selmask = 0, cnt = 0, incl = 0;
+        if (!service) {
+            const float *pd = s_d + tid * kSeg;
+            const float *pr = s_r + tid * kSeg;
             float m = 0.f;
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
-                g[j] = __fadd_rn(s_r[tid * kSeg + j], s_d[tid * kSeg + j]);
+                const float d = pd[j];
+                g[j] = __fadd_rn(pr[j], d);
+                const float h = __fadd_rn(g[j], d);
                 m = fmaxf(m, fabsf(g[j]));
+                // |G| never exceeds the bin maximum, so "|H| >= g_max or |G| == g_max"
+                // is "max(|H|, |G|) >= g_max"
+                key[j] = fmaxf(fabsf(h), fabsf(g[j]));
             }
-            s_segmax[tid] = m;
-        }
-        __syncthreads();
-
-        // ---- bin maximum, selection; warp 5 adds the bin maxima to the exact sum ----
-        u32 selmask = 0, negmask = 0;
-        if (tid < kTileSegs) {
-            const int bin = tid / SPB;
-            float gm = 0.f;
-#pragma unroll
-            for (int s = 0; s < SPB; s++) gm = fmaxf(gm, s_segmax[bin * SPB + s]);
-            if (gm > 0.f) {
-#pragma unroll
-                for (int j = 0; j < kSeg; j++) {
-                    const float h = __fadd_rn(g[j], s_d[tid * kSeg + j]);
-                    const float ag = fabsf(g[j]);
-                    const bool sel = (g[j] != 0.f) &&
-                                     (fabsf(h) >= gm || (!a.literal && ag == gm));
-                    selmask |= (u32)sel << j;
-                    negmask |= (u32)(g[j] < 0.f) << j;
-                }
-            }
-            s_off[tid] = __popc(selmask);
-        } else {
-            for (int b0 = 0; b0 < kBins; b0 += 32) {    // every lane takes part each round
-                const int b = b0 + lane;
-                float gm = 0.f;
-                if (b < kBins) {
-#pragma unroll
-                    for (int s = 0; s < SPB; s++) gm = fmaxf(gm, s_segmax[b * SPB + s]);
-                }
-                const bool valid = b < kBins && tile * (u64)kBins + b < geo.n_bins;
-                warp_accumulate(s_acc, gm, valid);
+            if (SPB == 2) {
+                gm = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            } else {
+                s_segmax[tid] = m;
             }
         }
-        __syncthreads();    // s_d (dW) is dead from here on: it becomes the word staging area
-
-        // ---- exclusive scan of the 160 segment counts (warp 0, five per lane) ----
-        if (warp == 0) {
-            u32 c[5], sum = 0;
+        if (SPB != 2) {
+            __syncthreads();                                        // barrier A
+            if (!service) {
+                const int bin = tid / SPB;
 #pragma unroll
-            for (int q = 0; q < 5; q++) { c[q] = s_off[lane * 5 + q]; sum += c[q]; }
-            u32 inc = sum;
-            for (int d = 1; d < 32; d <<= 1) {
-                u32 t = __shfl_up_sync(0xffffffffu, inc, d);
-                if (lane >= d) inc += t;
+                for (int s = 0; s < SPB; s++) gm = fmaxf(gm, s_segmax[bin * SPB + s]);
             }
-            u32 run = inc - sum;
-#pragma unroll
-            for (int q = 0; q < 5; q++) { s_off[lane * 5 + q] = run; run += c[q]; }
-            if (lane == 31) s_off[kTileSegs] = inc;
         }
-        __syncthreads();
+        if (!service) {
+            if (tid % SPB == 0) s_binmax[tid / SPB] = gm;
+            // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
+#pragma unroll
+            for (int j = 0; j < kSeg; j++)
+                if (key[j] >= gm && g[j] != 0.f) selmask |= 1u << j;
+            cnt = __popc(selmask);
+            incl = warp_inclusive_scan(cnt, lane);
+            s_incl[tid] = incl;
+            if (lane == 31) s_wtot[warp] = incl;
+        }
+        __syncthreads();                                            // barrier B
 
-        // ---- words into the staging area, G back into shared memory, bin counts ----
-        if (tid < kTileSegs) {
-            u32 at = s_off[tid];
+        u32 total = 0;
+        if (!service) {
+            // ---- words into the staging area, G back into the residue stage ----
+            u32 wpre[6];
+            wpre[0] = 0;
+#pragma unroll
+            for (int wv = 0; wv < 5; wv++) wpre[wv + 1] = wpre[wv] + s_wtot[wv];
+            const u32 mine = wpre[warp] + incl;                     // inclusive position
+            float *pr = s_r + tid * kSeg;
+#pragma unroll
+            for (int j = 0; j < kSeg; j++) pr[j] = g[j];
+            u32 at = mine - cnt;
             const u32 seg_in_bin = (u32)(tid % SPB) * kSeg;
-#pragma unroll
-            for (int j = 0; j < kSeg; j++) {
-                if (selmask >> j & 1u) {
-                    const u32 code = (negmask >> j & 1u) ? 3u : 1u;
-                    s_words[at++] = (Word)(((seg_in_bin + j) << 2) | code);
-                }
-                s_r[tid * kSeg + j] = g[j];
+            u32 mask = selmask;
+            while (mask) {
+                const int j = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const u32 neg = __float_as_uint(pr[j]) >> 31;
+                s_words[at++] = (Word)(((seg_in_bin + j) << 2) | 1u | (neg << 1));
             }
             if (tid % SPB == 0) {
                 const u64 bin = tile * (u64)kBins + tid / SPB;
-                if (bin < geo.n_bins) bin_cnt[bin] = (Word)(s_off[tid + SPB] - s_off[tid]);
+                const int t1 = tid + SPB - 1;
+                const u32 last = wpre[t1 >> 5] + s_incl[t1];
+                if (bin < geo.n_bins) bin_cnt[bin] = (Word)(last - mine + cnt);
+            }
+            fence_async_smem();          // the bulk store below reads what was just written
+        } else {
+            total = s_wtot[0] + s_wtot[1] + s_wtot[2] + s_wtot[3] + s_wtot[4];
+            for (int b0 = 0; b0 < kBins; b0 += 32) {    // every lane takes part each round
+                const int b = b0 + lane;
+                const bool valid = b < kBins && tile * (u64)kBins + b < geo.n_bins;
+                warp_accumulate(s_acc, valid ? s_binmax[b] : 0.f, valid);
+            }
+            if (lane == 0) {
+                bulk_wait_read_all();    // the store of tile i - 1 has drained its stage
+                issue_load(i + 2);
             }
         }
-        __syncthreads();
+        __syncthreads();                                            // barrier D
 
-        // ---- store residue = G (coalesced) and the tile's words into its slot ----
-        float4 *out = reinterpret_cast<float4 *>(a.residue + base);
-        for (int i = tid; i < kFastTile / 4; i += kFastThreads) {
-            if (4 * i + 3 < elems) {
-                out[i] = reinterpret_cast<float4 *>(s_r)[i];
+        const bool aborted = *s_abort != 0;
+        if (service && !aborted) {
+            if (whole) {
+                if (lane == 0) {
+                    bulk_store(a.residue + base, s_r, kTileBytes);
+                    bulk_commit();
+                }
             } else {
-                for (int c = 0; c < 4; c++)
-                    if (4 * i + c < elems) a.residue[base + 4 * i + c] = s_r[4 * i + c];
+                for (int e = lane; e < elems; e += 32) a.residue[base + e] = s_r[e];
+            }
+            uint4 *slot = reinterpret_cast<uint4 *>(a.packed + geo.slots_at + tile * geo.slot_bytes);
+            const int chunks = (int)((total * sizeof(Word) + 15) / 16);
+            for (int c = lane; c < chunks; c += 32) slot[c] = reinterpret_cast<uint4 *>(s_words)[c];
+            if (lane == 0) {
+                tile_cnt[tile] = total;
+                if (total) atomicAdd(&group_cnt[tile / kGroupTiles], (u64)total);
             }
         }
-        const u32 total = s_off[kTileSegs];
-        uint4 *slot = reinterpret_cast<uint4 *>(a.packed + geo.slots_at + tile * geo.slot_bytes);
-        const int chunks = (int)((total * sizeof(Word) + 15) / 16);
-        for (int i = tid; i < chunks; i += kFastThreads) slot[i] = reinterpret_cast<uint4 *>(s_d)[i];
-        if (tid == 0) tile_cnt[tile + 1] = total;
-        __syncthreads();
+        if (aborted) break;          // uniform: the flag was set before barrier D
     }
 
-    // ---- this CTA's share of the exact sum of g_max ----
-    if (warp == 5 && lane < kWindows) {
-        const u64 v = s_acc[lane];
-        if (v) atomicAdd(reinterpret_cast<u64 *>(a.packed + geo.ctl_at) + lane, v);
+    if (service) {
+        if (lane == 0) {
+            bulk_wait_all();
+            // after a timeout: loads still in flight must land (or time out in turn)
+            // before this CTA's shared memory is given back
+            if (*s_abort)
+                for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % kStages], (u32)(j / kStages) & 1u);
+        }
+        if (lane < kWindows) {
+            const u64 v = s_acc[lane];
+            if (v) atomicAdd(reinterpret_cast<u64 *>(a.packed + geo.ctl_at) + lane, v);
+        }
     }
 }
 
@@ -359,8 +498,9 @@ tile_pass_generic(PassArgs a)
     u32 *s_cnt = reinterpret_cast<u32 *>(s_gmax + TB);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
-    u64 *tile_cnt = reinterpret_cast<u64 *>(a.packed + geo.tile_off_at);
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
+    u32 *tile_cnt = reinterpret_cast<u32 *>(a.packed + geo.tile_cnt_at);
+    u64 *group_cnt = reinterpret_cast<u64 *>(a.packed + geo.group_at);
 
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
@@ -442,7 +582,10 @@ tile_pass_generic(PassArgs a)
         const u32 total = s_cnt[TB];
         Word *slot = reinterpret_cast<Word *>(a.packed + geo.slots_at + tile * geo.slot_bytes);
         for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
-        if (tid == 0) tile_cnt[tile + 1] = total;
+        if (tid == 0) {
+            tile_cnt[tile] = total;
+            if (total) atomicAdd(&group_cnt[tile / kGroupTiles], (u64)total);
+        }
         __syncthreads();
     }
 
@@ -453,7 +596,7 @@ tile_pass_generic(PassArgs a)
 }
 
 // ---------------------------------------------------------------------------------
-// finalize: one CTA.  Exact sum -> scale; tile counts -> exclusive scan; header.
+// finalize: one CTA.  Exact sum -> scale; group counts -> exclusive scan; header.
 // ---------------------------------------------------------------------------------
 
 // The nine windows hold the exact sum of the bin maxima in units of 2^-149.  Returns the
@@ -495,41 +638,42 @@ finalize(unsigned char *packed, Geometry geo, u32 flags, u64 *count_out)
 {
     __shared__ u64 s_warp[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
+    u64 *group = reinterpret_cast<u64 *>(packed + geo.group_at);
 
-    // in-place exclusive scan of the tile counts held in tile_off[1 .. n_tiles]
-    const u64 per = (geo.n_tiles + 1023) / 1024;
-    const u64 lo = min((u64)tid * per, geo.n_tiles), hi = min(lo + per, geo.n_tiles);
+    // in-place exclusive scan of the per-group word counts
+    const u64 per = (geo.n_groups + 1023) / 1024;
+    const u64 lo = min((u64)tid * per, geo.n_groups), hi = min(lo + per, geo.n_groups);
     u64 sum = 0;
-    for (u64 i = lo; i < hi; i++) sum += tile_off[i + 1];
+    for (u64 i = lo; i < hi; i++) sum += group[i];
     u64 inc = sum;
     for (int d = 1; d < 32; d <<= 1) {
-        u64 t = __shfl_up_sync(0xffffffffu, inc, d);
+        const u64 t = __shfl_up_sync(0xffffffffu, inc, d);
         if (lane >= d) inc += t;
     }
     if (lane == 31) s_warp[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        u64 v = s_warp[lane], s = v;
+        const u64 v = s_warp[lane];
+        u64 s = v;
         for (int d = 1; d < 32; d <<= 1) {
-            u64 t = __shfl_up_sync(0xffffffffu, s, d);
+            const u64 t = __shfl_up_sync(0xffffffffu, s, d);
             if (lane >= d) s += t;
         }
         s_warp[lane] = s - v;
         if (lane == 31) s_warp[32] = s;
     }
     __syncthreads();
-    u64 run = s_warp[warp] + inc - sum;      // words before this thread's first tile
-    // entry i+1 must become the count of words before tile i+1 = run + count(tile i)
+    u64 run = s_warp[warp] + inc - sum;
     for (u64 i = lo; i < hi; i++) {
-        const u64 c = tile_off[i + 1];
+        const u64 c = group[i];
+        group[i] = run;
         run += c;
-        tile_off[i + 1] = run;
     }
     const u64 n_sel = s_warp[32];
 
     if (tid == 0) {
-        tile_off[0] = 0;
+        u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
+        tile_off[geo.n_tiles] = n_sel;
         const u64 *win = reinterpret_cast<const u64 *>(packed + geo.ctl_at);
         float scale = 0.f;
         if (geo.n_bins) {
@@ -564,27 +708,127 @@ finalize(unsigned char *packed, Geometry geo, u32 flags, u64 *count_out)
 }
 
 // ---------------------------------------------------------------------------------
-// gather_fixup: per tile, copy the slot's words to the payload and finish the residue
-// of the sent elements: residue = G - sign(G) * scale  (Algorithm 2, the "if" branch).
+// gather_fixup: per tile, copy the slot's words to the payload, write the tile's
+// directory entry and finish the residue of the sent elements:
+// residue = G - sign(G) * scale  (Algorithm 2, the "if" branch).
 // ---------------------------------------------------------------------------------
 
+// Words before `tile`: its group's scanned offset plus the counts of the tiles before it
+// in the group.  Warp-collective; also returns the tile's own count.
+__device__ inline u64 tile_offset(const unsigned char *packed, const Geometry &geo, u64 tile, int lane,
+                                  u32 &count)
+{
+    const u32 *tile_cnt = reinterpret_cast<const u32 *>(packed + geo.tile_cnt_at);
+    const u64 *group = reinterpret_cast<const u64 *>(packed + geo.group_at);
+    const u64 g = tile / kGroupTiles;
+    const int me = (int)(tile % kGroupTiles);
+    const u64 t = g * kGroupTiles + lane;
+    const u32 c = t < geo.n_tiles ? tile_cnt[t] : 0u;
+    u32 before = lane < me ? c : 0u;
+    for (int d = 16; d > 0; d >>= 1) before += __shfl_xor_sync(0xffffffffu, before, d);
+    count = __shfl_sync(0xffffffffu, c, me);
+    return group[g] + before;
+}
+
+// Tiles of at most 96 bins: one warp per tile.
+template <typename Word>
+__global__ void __launch_bounds__(kGatherThreads)
+gather_fixup_small(float *residue, unsigned char *packed, Geometry geo)
+{
+    __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    u32 *s_pre = s_pre_all[warp];
+    const int TB = (int)geo.tile_bins;
+    u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
+    const Word *bin_cnt = reinterpret_cast<const Word *>(packed + geo.bin_cnt_at);
+    Word *payload = reinterpret_cast<Word *>(packed + geo.payload_at);
+    const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
+    const u64 warps = (u64)gridDim.x * (kGatherThreads / 32);
+
+    for (u64 tile = (u64)blockIdx.x * (kGatherThreads / 32) + warp; tile < geo.n_tiles; tile += warps) {
+        u32 cnt;
+        const u64 off0 = tile_offset(packed, geo, tile, lane, cnt);
+        if (lane == 0) tile_off[tile] = off0;
+        if (cnt == 0) continue;
+        // exclusive scan of the tile's bin counts, three bins per lane
+        const u64 bin0 = tile * (u64)TB;
+        u32 c[3], sum = 0;
+#pragma unroll
+        for (int q = 0; q < 3; q++) {
+            const int b = lane * 3 + q;
+            c[q] = (b < TB && bin0 + b < geo.n_bins) ? (u32)bin_cnt[bin0 + b] : 0u;
+            sum += c[q];
+        }
+        const u32 inc = warp_inclusive_scan(sum, lane);
+        u32 run = inc - sum;
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 3; q++) {
+            const int b = lane * 3 + q;
+            if (b < TB) s_pre[b] = run;
+            run += c[q];
+        }
+        if (lane == 31) s_pre[TB] = inc;
+        __syncwarp();
+        const Word *slot = reinterpret_cast<const Word *>(packed + geo.slots_at + tile * geo.slot_bytes);
+        const u64 base = tile * (u64)geo.tile_elems;
+        for (u32 j0 = 0; j0 < cnt; j0 += 128) {
+            // four words per lane per round: their residue loads overlap
+            u32 word[4];
+            u64 pos[4];
+            float g[4];
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const u32 j = j0 + q * 32 + lane;
+                word[q] = 0;
+                pos[q] = 0;
+                g[q] = 0.f;
+                if (j < cnt) {
+                    word[q] = slot[j];
+                    const int b = bin_of_word(s_pre, TB, j);
+                    pos[q] = base + (u64)b * geo.L_T + (word[q] >> 2);
+                    g[q] = residue[pos[q]];
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const u32 j = j0 + q * 32 + lane;
+                if (j < cnt) {
+                    residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
+                    payload[off0 + j] = (Word)word[q];
+                }
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// Any tile shape: one CTA per tile.
 template <typename Word>
 __global__ void __launch_bounds__(kGatherThreads)
 gather_fixup(float *residue, unsigned char *packed, Geometry geo)
 {
     __shared__ u32 s_pre[kMaxTileBins + 1];
     __shared__ u32 s_tmp[33];
+    __shared__ u64 s_off0;
+    __shared__ u32 s_count;
     const int tid = threadIdx.x;
     const int TB = (int)geo.tile_bins;
-    const u64 *tile_off = reinterpret_cast<const u64 *>(packed + geo.tile_off_at);
+    u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
     const Word *bin_cnt = reinterpret_cast<const Word *>(packed + geo.bin_cnt_at);
     Word *payload = reinterpret_cast<Word *>(packed + geo.payload_at);
     const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
 
     for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
-        const u64 off0 = tile_off[tile];
-        const u32 cnt = (u32)(tile_off[tile + 1] - off0);
-        if (cnt == 0) continue;
+        if (tid < 32) {
+            u32 c;
+            const u64 o = tile_offset(packed, geo, tile, tid, c);
+            if (tid == 0) { s_off0 = o; s_count = c; tile_off[tile] = o; }
+        }
+        __syncthreads();
+        const u64 off0 = s_off0;
+        const u32 cnt = s_count;
+        if (cnt == 0) { __syncthreads(); continue; }
         const u64 bin0 = tile * (u64)TB;
         for (int b = tid; b < TB; b += kGatherThreads)
             s_pre[b] = bin0 + b < geo.n_bins ? (u32)bin_cnt[bin0 + b] : 0u;
@@ -605,7 +849,7 @@ gather_fixup(float *residue, unsigned char *packed, Geometry geo)
 }
 
 // ---------------------------------------------------------------------------------
-// decode_sum: unpack() of k streams and their ordered sum, one output chunk per CTA pass.
+// decode_sum: unpack() of k streams and their ordered sum.
 // ---------------------------------------------------------------------------------
 
 struct DecodeArgs {
@@ -614,38 +858,194 @@ struct DecodeArgs {
     u32 k;
 };
 
+struct DecodeSmem {
+    float acc[kDecodeChunk];                    // the output tile
+    u32 pre[kMaxTileBins + 1];                  // scanned bin counts
+    u32 tmp[40];
+    u64 off0[ADACOMP_MAX_STREAMS];              // first word of this tile in stream l
+    u64 n_sel[ADACOMP_MAX_STREAMS];             // words in stream l
+    float scale[ADACOMP_MAX_STREAMS];
+};
+
+__device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc)
+{
+    const int tid = threadIdx.x;
+    if ((out0 & 3u) == 0) {
+        float4 *o4 = reinterpret_cast<float4 *>(dst + out0);
+        float4 *s4 = reinterpret_cast<float4 *>(s_acc);
+        for (u32 i = tid; i < len / 4; i += kDecodeThreads) {
+            __stcs(o4 + i, s4[i]);
+            s4[i] = make_float4(0.f, 0.f, 0.f, 0.f);       // ready for the next tile
+        }
+        for (u32 i = (len & ~3u) + tid; i < len; i += kDecodeThreads) { dst[out0 + i] = s_acc[i]; s_acc[i] = 0.f; }
+    } else {
+        for (u32 i = tid; i < len; i += kDecodeThreads) { dst[out0 + i] = s_acc[i]; s_acc[i] = 0.f; }
+    }
+}
+
+// Tiles of 32..96 bins (L_T = 42..125): thread b owns bin b for every learner, so the
+// learners' contributions to an element are added by one thread, in learner order,
+// without any barrier between learners.
 template <typename Word>
-__device__ void decode_items(const DecodeArgs &a, const Geometry &geo, float *s_acc, u32 *s_pre,
-                             u32 *s_tmp)
+__device__ void decode_by_bin(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int TB = (int)geo.tile_bins;
+    u32 *s_wsum = sm.tmp;        // [4 warps][8 learners of a round]
+    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
+    if (tid < (int)a.k) {
+        sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
+        sm.n_sel[tid] = reinterpret_cast<const u64 *>(a.stream[tid])[5];
+    }
+    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
+        const u64 base = tile * (u64)geo.tile_elems;
+        const u64 bin = tile * (u64)TB + tid;
+        const bool live = tid < TB && bin < geo.n_bins;
+        if (tid < (int)a.k)
+            sm.off0[tid] = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at)[tile];
+        for (u32 l0 = 0; l0 < a.k; l0 += 8) {
+            const int round = (int)min(8u, a.k - l0);
+            u32 c[8], pre[8];
+#pragma unroll
+            for (int q = 0; q < 8; q++) {
+                c[q] = 0;
+                if (q < round && live)
+                    c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin], geo.L_T);
+                const u32 inc = warp_inclusive_scan(c[q], lane);
+                pre[q] = inc - c[q];
+                if (lane == 31) s_wsum[warp * 8 + q] = inc;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int q = 0; q < 8; q++)
+                for (int wv = 0; wv < warp; wv++) pre[q] += s_wsum[wv * 8 + q];
+            float *mine = sm.acc + tid * geo.L_T;
+#pragma unroll
+            for (int q = 0; q < 8; q++) {
+                if (q >= round || c[q] == 0) continue;
+                const u64 at0 = sm.off0[l0 + q] + pre[q];
+                if (at0 + c[q] > sm.n_sel[l0 + q]) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                const Word *p = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.payload_at) + at0;
+                const float scale = sm.scale[l0 + q];
+                for (u32 i = 0; i < c[q]; i++) {
+                    const u32 word = p[i];
+                    const u32 code = word & 3u, idx = word >> 2;
+                    if (code == 0u) continue;
+                    if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
+                    if (idx >= geo.L_T || base + (u64)tid * geo.L_T + idx >= geo.n) {
+                        raise_status(ADACOMP_DEV_BAD_STREAM);
+                        continue;
+                    }
+                    mine[idx] = code == 3u ? __fsub_rn(mine[idx], scale) : __fadd_rn(mine[idx], scale);
+                }
+            }
+            __syncthreads();
+        }
+        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
+        store_tile(a.dst, base, len, sm.acc);
+        __syncthreads();
+    }
+}
+
+// Tiles of 2..31 bins (L_T = 126..1000): the words of one learner are spread over the
+// threads; a barrier separates consecutive learners.
+template <typename Word>
+__device__ void decode_by_word(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int TB = (int)geo.tile_bins;
+    u32 (*s_pre)[33] = reinterpret_cast<u32 (*)[33]>(sm.pre);      // [learner of the round][bin]
+    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
+    if (tid < (int)a.k) {
+        sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
+        sm.n_sel[tid] = reinterpret_cast<const u64 *>(a.stream[tid])[5];
+    }
+    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
+        const u64 base = tile * (u64)geo.tile_elems;
+        const u64 bin0 = tile * (u64)TB;
+        for (u32 l0 = 0; l0 < a.k; l0 += 32) {
+            const int round = (int)min(32u, a.k - l0);
+            // warp wv scans the bin counts of learners wv, wv + 4, ... of this round
+            for (int q = warp; q < round; q += kDecodeThreads / 32) {
+                const unsigned char *s = a.stream[l0 + q];
+                u32 c = 0;
+                if (lane < TB && bin0 + lane < geo.n_bins)
+                    c = reinterpret_cast<const Word *>(s + geo.bin_cnt_at)[bin0 + lane];
+                const u32 inc = warp_inclusive_scan(c, lane);
+                s_pre[q][lane] = inc - c;
+                if (lane == 31) {
+                    s_pre[q][32] = inc;
+                    sm.off0[l0 + q] = reinterpret_cast<const u64 *>(s + geo.tile_off_at)[tile];
+                }
+            }
+            __syncthreads();
+            for (int q = 0; q < round; q++) {
+                const u32 cnt = s_pre[q][32];         // the same for every thread
+                if (cnt == 0) continue;
+                if (cnt > geo.tile_elems || sm.off0[l0 + q] + cnt > sm.n_sel[l0 + q]) {
+                    if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM);
+                    continue;
+                }
+                const Word *p = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.payload_at) + sm.off0[l0 + q];
+                const float scale = sm.scale[l0 + q];
+                for (u32 j = tid; j < cnt; j += kDecodeThreads) {
+                    const u32 word = p[j];
+                    const u32 code = word & 3u, idx = word >> 2;
+                    if (code == 0u) continue;
+                    if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
+                    int b = 0;
+                    for (int step = 16; step > 0; step >>= 1)       // at most 31 bins: five probes
+                        if (b + step < TB && s_pre[q][b + step] <= j) b += step;
+                    const u32 at = (u32)b * geo.L_T + idx;
+                    if (idx >= geo.L_T || base + at >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                    sm.acc[at] = code == 3u ? __fsub_rn(sm.acc[at], scale) : __fadd_rn(sm.acc[at], scale);
+                }
+                __syncthreads();
+            }
+            __syncthreads();
+        }
+        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
+        store_tile(a.dst, base, len, sm.acc);
+        __syncthreads();
+    }
+}
+
+// Any tile shape (also tiles larger than one output chunk).
+template <typename Word>
+__device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
 {
     const int tid = threadIdx.x;
     const int TB = (int)geo.tile_bins;
+    float *s_acc = sm.acc;
+    u32 *s_pre = sm.pre;
     const u32 chunks_per_tile = (geo.tile_elems + kDecodeChunk - 1) / kDecodeChunk;
     const u64 items = geo.n_tiles * chunks_per_tile;
+    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) s_acc[i] = 0.f;
+    __syncthreads();
     for (u64 item = blockIdx.x; item < items; item += gridDim.x) {
         const u64 tile = item / chunks_per_tile;
         const u32 c_lo = (u32)(item % chunks_per_tile) * kDecodeChunk;     // within the tile
         const u32 c_hi = min(c_lo + (u32)kDecodeChunk, geo.tile_elems);
         const u64 base = tile * (u64)geo.tile_elems;
-        for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) s_acc[i] = 0.f;
-        __syncthreads();
         for (u32 l = 0; l < a.k; l++) {
             const unsigned char *s = a.stream[l];
             const u64 *tile_off = reinterpret_cast<const u64 *>(s + geo.tile_off_at);
             const u64 off0 = tile_off[tile];
             const u32 cnt = (u32)(tile_off[tile + 1] - off0);
             if (cnt == 0) continue;
-            if (cnt > geo.tile_elems) { if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+            if (cnt > geo.tile_elems || off0 + cnt > reinterpret_cast<const u64 *>(s)[5]) {
+                if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM);
+                continue;
+            }
             const float scale = __uint_as_float(reinterpret_cast<const u32 *>(s)[12]);
             const Word *bin_cnt = reinterpret_cast<const Word *>(s + geo.bin_cnt_at);
             const Word *payload = reinterpret_cast<const Word *>(s + geo.payload_at);
             const u64 bin0 = tile * (u64)TB;
-            int b_fixed = 0;
             if (TB > 1) {
                 for (int b = tid; b < TB; b += kDecodeThreads)
                     s_pre[b] = bin0 + b < geo.n_bins ? (u32)bin_cnt[bin0 + b] : 0u;
                 __syncthreads();
-                block_exclusive_scan(s_pre, TB, s_tmp);
+                block_exclusive_scan(s_pre, TB, sm.tmp);
                 if (s_pre[TB] != cnt) { if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM); __syncthreads(); continue; }
             }
             for (u32 j = tid; j < cnt; j += kDecodeThreads) {
@@ -653,7 +1053,7 @@ __device__ void decode_items(const DecodeArgs &a, const Geometry &geo, float *s_
                 const u32 code = word & 3u;
                 if (code == 0u) continue;
                 if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                const int b = TB > 1 ? bin_of_word(s_pre, TB, j) : b_fixed;
+                const int b = TB > 1 ? bin_of_word(s_pre, TB, j) : 0;
                 const u32 idx = word >> 2;
                 const u32 at = (u32)b * geo.L_T + idx;          // within the tile
                 if (idx >= geo.L_T || base + at >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
@@ -666,14 +1066,7 @@ __device__ void decode_items(const DecodeArgs &a, const Geometry &geo, float *s_
         }
         const u64 out0 = base + c_lo;
         const u32 len = out0 < geo.n ? (u32)min((u64)(c_hi - c_lo), geo.n - out0) : 0u;
-        if ((out0 & 3u) == 0) {
-            float4 *o4 = reinterpret_cast<float4 *>(a.dst + out0);
-            for (u32 i = tid; i < len / 4; i += kDecodeThreads)
-                __stcs(o4 + i, reinterpret_cast<float4 *>(s_acc)[i]);
-            for (u32 i = (len & ~3u) + tid; i < len; i += kDecodeThreads) a.dst[out0 + i] = s_acc[i];
-        } else {
-            for (u32 i = tid; i < len; i += kDecodeThreads) a.dst[out0 + i] = s_acc[i];
-        }
+        store_tile(a.dst, out0, len, s_acc);
         __syncthreads();
     }
 }
@@ -681,9 +1074,7 @@ __device__ void decode_items(const DecodeArgs &a, const Geometry &geo, float *s_
 __global__ void __launch_bounds__(kDecodeThreads)
 decode_sum(DecodeArgs a)
 {
-    __shared__ __align__(16) float s_acc[kDecodeChunk];
-    __shared__ u32 s_pre[kMaxTileBins + 1];
-    __shared__ u32 s_tmp[33];
+    __shared__ __align__(16) DecodeSmem sm;
     __shared__ int s_bad;
 
     // every CTA reads and cross-checks the k headers itself: the decision is uniform
@@ -700,7 +1091,7 @@ decode_sum(DecodeArgs a)
         if (ok) {
             const Geometry g = make_geometry(n, L_T);
             ok = ((h[1] >> 16) & 0xffu) == g.w && h[3] == g.tile_bins && h64[3] == g.n_bins &&
-                 h64[4] == g.n_tiles;
+                 h64[4] == g.n_tiles && h64[5] <= n;
         }
         if (!ok) s_bad = 1;
     }
@@ -710,8 +1101,16 @@ decode_sum(DecodeArgs a)
         return;
     }
     const Geometry geo = make_geometry(n, L_T);
-    if (geo.w == 1u) decode_items<unsigned char>(a, geo, s_acc, s_pre, s_tmp);
-    else decode_items<unsigned short>(a, geo, s_acc, s_pre, s_tmp);
+    const bool by_bin = geo.tile_bins >= 32 && geo.tile_bins <= (u32)kSmallBins;
+    const bool by_word = geo.tile_bins >= 2 && geo.tile_bins <= 31;
+    if (geo.w == 1u) {
+        if (by_bin) decode_by_bin<unsigned char>(a, geo, sm);
+        else decode_generic<unsigned char>(a, geo, sm);
+    } else {
+        if (by_bin) decode_by_bin<unsigned short>(a, geo, sm);
+        else if (by_word) decode_by_word<unsigned short>(a, geo, sm);
+        else decode_generic<unsigned short>(a, geo, sm);
+    }
 }
 
 __global__ void reset_status_kernel() { g_status = 0; }
@@ -723,23 +1122,34 @@ __global__ void reset_status_kernel() { g_status = 0; }
 struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
+    int decode_per_sm = 0;
+    bool fast_ready = false;
 };
 
 DeviceInfo g_info[64];
 
-int device_info(DeviceInfo &out)
+int device_info(DeviceInfo *&out)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ADACOMP_ERR_CUDA;
-    if (g_info[dev].sms == 0) {
+    DeviceInfo &d = g_info[dev];
+    if (d.sms == 0) {
         int sms = 0, optin = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return ADACOMP_ERR_CUDA;
-        g_info[dev].smem_optin = optin;
-        g_info[dev].sms = sms;
+        d.smem_optin = optin;
+        int per_sm = 1;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
+        d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
+        d.fast_ready =
+            cudaFuncSetAttribute(tile_pass_fast<2, unsigned char>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)FastSmem::kBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(tile_pass_fast<20, unsigned short>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)FastSmem::kBytes) == cudaSuccess;
+        d.sms = sms;
     }
-    out = g_info[dev];
+    out = &d;
     return ADACOMP_OK;
 }
 
@@ -775,33 +1185,29 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     const Geometry geo = make_geometry(n, L_T);
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
 
-    DeviceInfo info;
+    DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char *packed = static_cast<unsigned char *>(packed_out);
 
-    if (cudaMemsetAsync(packed + geo.ctl_at, 0, kCtlBytes, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
+    // the exact-sum windows and the group counts start from zero
+    if (cudaMemsetAsync(packed + geo.ctl_at, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess)
+        return ADACOMP_ERR_CUDA;
     auto mark = [&](int i) { if (events) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st); };
 
     mark(0);
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, geo, flags & ADACOMP_FLAG_LITERAL};
-        const bool fast = (L_T == 50u || L_T == 500u) && !(flags & ADACOMP_FLAG_GENERIC_PATH);
+        const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
         if (fast) {
-            int per_sm = 1;
-            if (L_T == 50u)
-                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tile_pass_fast<2, unsigned char>, kFastThreads, 0);
-            else
-                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tile_pass_fast<20, unsigned short>, kFastThreads, 0);
-            if (per_sm < 1) per_sm = 1;
-            const u64 cap = (u64)info.sms * per_sm;
+            const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (L_T == 50u) tile_pass_fast<2, unsigned char><<<grid, kFastThreads, 0, st>>>(args);
-            else tile_pass_fast<20, unsigned short><<<grid, kFastThreads, 0, st>>>(args);
+            if (L_T == 50u) tile_pass_fast<2, unsigned char><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            else tile_pass_fast<20, unsigned short><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
         } else {
-            rc = geo.w == 1u ? launch_generic<unsigned char>(args, info, st)
-                             : launch_generic<unsigned short>(args, info, st);
+            rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
+                             : launch_generic<unsigned short>(args, *info, st);
             if (rc != ADACOMP_OK) return rc;
         }
     }
@@ -809,10 +1215,17 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     finalize<<<1, 1024, 0, st>>>(packed, geo, flags, reinterpret_cast<u64 *>(count_out));
     mark(2);
     if (geo.n_tiles) {
-        const u64 cap = (u64)info.sms * 8;
-        const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-        if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
-        else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+        if (geo.tile_bins <= (u32)kSmallBins) {
+            const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
+            const unsigned grid = (unsigned)(want < cap ? want : cap);
+            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+        } else {
+            const u64 cap = (u64)info->sms * 8;
+            const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
+            if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+            else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+        }
     }
     mark(3);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
@@ -832,13 +1245,11 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     if (misaligned(dst)) return ADACOMP_ERR_ALIGN;
     args.dst = dst;
     args.k = k;
-    DeviceInfo info;
+    DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
-    int per_sm = 1;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
-    if (per_sm < 1) per_sm = 1;
-    decode_sum<<<(unsigned)(info.sms * per_sm), kDecodeThreads, 0, static_cast<cudaStream_t>(stream)>>>(args);
+    decode_sum<<<(unsigned)(info->sms * info->decode_per_sm), kDecodeThreads, 0,
+                 static_cast<cudaStream_t>(stream)>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
