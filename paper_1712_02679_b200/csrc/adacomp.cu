@@ -58,8 +58,10 @@ __host__ __device__ inline u64 align_up(u64 x, u64 a) { return (x + a - 1) / a *
 struct Geometry {
     u32 w, L_T, tile_bins, tile_elems;
     u64 n, n_bins, n_tiles, n_groups;
-    u64 tile_off_at, bin_cnt_at, payload_at;                             // the stream
-    u64 ctl_at, group_at, tile_cnt_at, slots_at, slot_bytes, capacity;   // scratch
+    u64 tile_off_at, bin_cnt_at, payload_at;              // the stream, offsets in the packed buffer
+    u64 group_at, tile_cnt_at, slots_at, slot_bytes;      // the scratch, offsets from its base
+    u64 scratch_bytes;                                    // (the control block sits at offset 0)
+    u64 scratch_at, capacity;     // where the scratch starts when it follows the stream in one buffer
 };
 
 __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
@@ -76,12 +78,13 @@ __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
     g.tile_off_at = kHeaderBytes;
     g.bin_cnt_at = align_up(g.tile_off_at + 8 * (g.n_tiles + 1), 16);
     g.payload_at = align_up(g.bin_cnt_at + g.n_bins * g.w, 16);
-    g.ctl_at = align_up(g.payload_at + align_up(n * g.w, 16), 256);
-    g.group_at = g.ctl_at + kCtlBytes;                         // u64[n_groups], zeroed per call
+    g.group_at = kCtlBytes;                                    // u64[n_groups], zeroed per call
     g.tile_cnt_at = g.group_at + 8 * g.n_groups;               // u32[n_tiles]
     g.slots_at = align_up(g.tile_cnt_at + 4 * g.n_tiles, 256);
     g.slot_bytes = align_up((u64)g.tile_elems * g.w, 16);
-    g.capacity = g.slots_at + g.n_tiles * g.slot_bytes;
+    g.scratch_bytes = g.slots_at + g.n_tiles * g.slot_bytes;
+    g.scratch_at = align_up(g.payload_at + align_up(n * g.w, 16), 256);
+    g.capacity = g.scratch_at + g.scratch_bytes;
     return g;
 }
 
@@ -259,7 +262,8 @@ __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shar
 struct PassArgs {
     const float *grad;
     float *residue;
-    unsigned char *packed;
+    unsigned char *packed;      // the stream under construction
+    unsigned char *scratch;     // control block, group counts, tile counts, word slots
     Geometry geo;
     u32 literal;
 };
@@ -296,8 +300,8 @@ tile_pass_fast(PassArgs a)
     const Geometry &geo = a.geo;
     constexpr int kBins = kTileSegs / SPB;
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
-    u32 *tile_cnt = reinterpret_cast<u32 *>(a.packed + geo.tile_cnt_at);
-    u64 *group_cnt = reinterpret_cast<u64 *>(a.packed + geo.group_at);
+    u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
+    u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
 
     // tiles of this CTA: blockIdx.x + i * gridDim.x
     const u64 first = blockIdx.x, stride = gridDim.x;
@@ -449,7 +453,7 @@ tile_pass_fast(PassArgs a)
             } else {
                 for (int e = lane; e < elems; e += 32) a.residue[base + e] = s_r[e];
             }
-            uint4 *slot = reinterpret_cast<uint4 *>(a.packed + geo.slots_at + tile * geo.slot_bytes);
+            uint4 *slot = reinterpret_cast<uint4 *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
             const int chunks = (int)((total * sizeof(Word) + 15) / 16);
             for (int c = lane; c < chunks; c += 32) slot[c] = reinterpret_cast<uint4 *>(s_words)[c];
             if (lane == 0) {
@@ -470,7 +474,7 @@ tile_pass_fast(PassArgs a)
         }
         if (lane < kWindows) {
             const u64 v = s_acc[lane];
-            if (v) atomicAdd(reinterpret_cast<u64 *>(a.packed + geo.ctl_at) + lane, v);
+            if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + lane, v);
         }
     }
 }
@@ -499,8 +503,8 @@ tile_pass_generic(PassArgs a)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
-    u32 *tile_cnt = reinterpret_cast<u32 *>(a.packed + geo.tile_cnt_at);
-    u64 *group_cnt = reinterpret_cast<u64 *>(a.packed + geo.group_at);
+    u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
+    u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
 
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
@@ -580,7 +584,7 @@ tile_pass_generic(PassArgs a)
 
         for (int i = tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
         const u32 total = s_cnt[TB];
-        Word *slot = reinterpret_cast<Word *>(a.packed + geo.slots_at + tile * geo.slot_bytes);
+        Word *slot = reinterpret_cast<Word *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
         for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
         if (tid == 0) {
             tile_cnt[tile] = total;
@@ -591,7 +595,7 @@ tile_pass_generic(PassArgs a)
 
     if (tid < kWindows) {
         const u64 v = s_acc[tid];
-        if (v) atomicAdd(reinterpret_cast<u64 *>(a.packed + geo.ctl_at) + tid, v);
+        if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + tid, v);
     }
 }
 
@@ -634,11 +638,11 @@ __device__ double windows_to_double(const u64 *win)
 }
 
 __global__ void __launch_bounds__(1024)
-finalize(unsigned char *packed, Geometry geo, u32 flags, u64 *count_out)
+finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out)
 {
     __shared__ u64 s_warp[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    u64 *group = reinterpret_cast<u64 *>(packed + geo.group_at);
+    u64 *group = reinterpret_cast<u64 *>(scratch + geo.group_at);
 
     // in-place exclusive scan of the per-group word counts
     const u64 per = (geo.n_groups + 1023) / 1024;
@@ -674,7 +678,7 @@ finalize(unsigned char *packed, Geometry geo, u32 flags, u64 *count_out)
     if (tid == 0) {
         u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
         tile_off[geo.n_tiles] = n_sel;
-        const u64 *win = reinterpret_cast<const u64 *>(packed + geo.ctl_at);
+        const u64 *win = reinterpret_cast<const u64 *>(scratch);
         float scale = 0.f;
         if (geo.n_bins) {
             const double S = windows_to_double(win);
@@ -715,11 +719,11 @@ finalize(unsigned char *packed, Geometry geo, u32 flags, u64 *count_out)
 
 // Words before `tile`: its group's scanned offset plus the counts of the tiles before it
 // in the group.  Warp-collective; also returns the tile's own count.
-__device__ inline u64 tile_offset(const unsigned char *packed, const Geometry &geo, u64 tile, int lane,
+__device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &geo, u64 tile, int lane,
                                   u32 &count)
 {
-    const u32 *tile_cnt = reinterpret_cast<const u32 *>(packed + geo.tile_cnt_at);
-    const u64 *group = reinterpret_cast<const u64 *>(packed + geo.group_at);
+    const u32 *tile_cnt = reinterpret_cast<const u32 *>(scratch + geo.tile_cnt_at);
+    const u64 *group = reinterpret_cast<const u64 *>(scratch + geo.group_at);
     const u64 g = tile / kGroupTiles;
     const int me = (int)(tile % kGroupTiles);
     const u64 t = g * kGroupTiles + lane;
@@ -733,7 +737,7 @@ __device__ inline u64 tile_offset(const unsigned char *packed, const Geometry &g
 // Tiles of at most 96 bins: one warp per tile.
 template <typename Word>
 __global__ void __launch_bounds__(kGatherThreads)
-gather_fixup_small(float *residue, unsigned char *packed, Geometry geo)
+gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *scratch, Geometry geo)
 {
     __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -747,7 +751,7 @@ gather_fixup_small(float *residue, unsigned char *packed, Geometry geo)
 
     for (u64 tile = (u64)blockIdx.x * (kGatherThreads / 32) + warp; tile < geo.n_tiles; tile += warps) {
         u32 cnt;
-        const u64 off0 = tile_offset(packed, geo, tile, lane, cnt);
+        const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
         if (lane == 0) tile_off[tile] = off0;
         if (cnt == 0) continue;
         // exclusive scan of the tile's bin counts, three bins per lane
@@ -770,7 +774,7 @@ gather_fixup_small(float *residue, unsigned char *packed, Geometry geo)
         }
         if (lane == 31) s_pre[TB] = inc;
         __syncwarp();
-        const Word *slot = reinterpret_cast<const Word *>(packed + geo.slots_at + tile * geo.slot_bytes);
+        const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
         const u64 base = tile * (u64)geo.tile_elems;
         for (u32 j0 = 0; j0 < cnt; j0 += 128) {
             // four words per lane per round: their residue loads overlap
@@ -806,7 +810,7 @@ gather_fixup_small(float *residue, unsigned char *packed, Geometry geo)
 // Any tile shape: one CTA per tile.
 template <typename Word>
 __global__ void __launch_bounds__(kGatherThreads)
-gather_fixup(float *residue, unsigned char *packed, Geometry geo)
+gather_fixup(float *residue, unsigned char *packed, const unsigned char *scratch, Geometry geo)
 {
     __shared__ u32 s_pre[kMaxTileBins + 1];
     __shared__ u32 s_tmp[33];
@@ -822,7 +826,7 @@ gather_fixup(float *residue, unsigned char *packed, Geometry geo)
     for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
         if (tid < 32) {
             u32 c;
-            const u64 o = tile_offset(packed, geo, tile, tid, c);
+            const u64 o = tile_offset(scratch, geo, tile, tid, c);
             if (tid == 0) { s_off0 = o; s_count = c; tile_off[tile] = o; }
         }
         __syncthreads();
@@ -834,7 +838,7 @@ gather_fixup(float *residue, unsigned char *packed, Geometry geo)
             s_pre[b] = bin0 + b < geo.n_bins ? (u32)bin_cnt[bin0 + b] : 0u;
         __syncthreads();
         block_exclusive_scan(s_pre, TB, s_tmp);
-        const Word *slot = reinterpret_cast<const Word *>(packed + geo.slots_at + tile * geo.slot_bytes);
+        const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
         const u64 base = tile * (u64)geo.tile_elems;
         for (u32 j = tid; j < cnt; j += kGatherThreads) {
             const u32 word = slot[j];
@@ -1191,14 +1195,16 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char *packed = static_cast<unsigned char *>(packed_out);
 
+    unsigned char *scratch = packed + geo.scratch_at;
+
     // the exact-sum windows and the group counts start from zero
-    if (cudaMemsetAsync(packed + geo.ctl_at, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess)
+    if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess)
         return ADACOMP_ERR_CUDA;
     auto mark = [&](int i) { if (events) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st); };
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, geo, flags & ADACOMP_FLAG_LITERAL};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL};
         const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
         if (fast) {
             const u64 cap = (u64)info->sms * 2;
@@ -1212,19 +1218,19 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         }
     }
     mark(1);
-    finalize<<<1, 1024, 0, st>>>(packed, geo, flags, reinterpret_cast<u64 *>(count_out));
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags, reinterpret_cast<u64 *>(count_out));
     mark(2);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
             const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
             const unsigned grid = (unsigned)(want < cap ? want : cap);
-            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
-            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
         } else {
             const u64 cap = (u64)info->sms * 8;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
-            else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, geo);
+            if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
         }
     }
     mark(3);
