@@ -67,6 +67,10 @@ extern "C" {
 #define ADACOMP_ERR_SIZE (-5)      /* n too large (n_bins must stay below 2^31) */
 #define ADACOMP_ERR_FLAGS (-6)     /* unknown flag bits */
 #define ADACOMP_ERR_CUDA (-7)      /* a CUDA runtime call failed */
+#define ADACOMP_ERR_STATIC_SCRATCH (-8) /* adacomp_compress_static: tensor beyond the built-in scratch */
+
+/* size of the scratch array built into the library for adacomp_compress_static */
+#define ADACOMP_STATIC_SCRATCH_BYTES (8u << 20)
 
 /* device-detected conditions (sticky bits) */
 #define ADACOMP_DEV_NONFINITE 1u        /* a bin maximum was inf or NaN */
@@ -108,6 +112,38 @@ size_t adacomp_packed_capacity(uint64_t n, uint32_t L_T);
  */
 int adacomp_compress(const float *grad, float *residue, uint64_t n, uint32_t L_T,
                      void *packed_out, uint64_t *count_out, void *stream);
+
+/*
+ * adacomp_compress for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework that
+ * hands out a fixed arena and forbids further allocation, in a latency-critical loop
+ * where an allocation would synchronise the device, or in a component that is only ever
+ * given its input and output buffers.  adacomp_compress needs scratch behind the stream
+ * (roughly one more word per element, see adacomp_packed_capacity); here that scratch is
+ * an array of ADACOMP_STATIC_SCRATCH_BYTES (8 MiB) built into the library instead, so
+ *   packed_out needs only the stream itself: 64 + 8 * (n_tiles + 1) + w * n_bins +
+ *              w * n bytes with each section rounded up to 16 (adacomp_packed_capacity
+ *              is always a safe upper bound);
+ *   the tensor must be small enough for the array: about 8.3 M elements at L_T <= 64
+ *              and 4.1 M above (the scratch holds w bytes per element plus 4 bytes per
+ *              tile).  Larger tensors return ADACOMP_ERR_STATIC_SCRATCH and nothing is
+ *              enqueued; use adacomp_compress for those.
+ * Arguments, results and error codes are otherwise those of adacomp_compress, and the
+ * bytes written to packed_out, count_out and residue are identical.
+ *
+ * The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ * The array lives in the library's device image, so every GPU that loads the library
+ * holds the 8 MiB until the process exits.  The first call on each device looks up the
+ * array's device address (with that device current); make that first call before any
+ * stream capture.  Every call on a device shares the one array, and it keeps the previous
+ * call's contents: the call clears the part that must start from zero itself, but two
+ * calls that overlap on the GPU (different streams, no dependency between them) race on
+ * it and corrupt each other's output.  Calls on one stream are safe.
+ */
+int adacomp_compress_static(const float *grad, float *residue, uint64_t n, uint32_t L_T,
+                            void *packed_out, uint64_t *count_out, void *stream);
 
 /* As adacomp_compress, with ADACOMP_FLAG_* bits. */
 int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t L_T,

@@ -58,6 +58,8 @@ def lib() -> C.CDLL:
         L.adacomp_compress.restype = C.c_int
         L.adacomp_compress.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p,
                                        C.c_void_p, C.c_void_p]
+        L.adacomp_compress_static.restype = C.c_int
+        L.adacomp_compress_static.argtypes = L.adacomp_compress.argtypes
         L.adacomp_compress_ex.restype = C.c_int
         L.adacomp_compress_ex.argtypes = L.adacomp_compress.argtypes + [C.c_uint32]
         L.adacomp_decompress_accumulate.restype = C.c_int
@@ -129,6 +131,20 @@ def adacomp_compress(grad, residue, n: int, L_T: int, packed_out, count_out, str
                                   _dev_ptr(packed_out, "packed_out", torch.uint8),
                                   _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
            "adacomp_compress")
+
+
+def adacomp_compress_static(grad, residue, n: int, L_T: int, packed_out, count_out,
+                            stream=None) -> None:
+    """pack() for callers that may not allocate device memory: same results as
+    adacomp_compress, but the compressor's scratch is an 8 MiB array built into the library,
+    so packed_out only has to hold the stream.  Tensors that need more scratch raise
+    AdaCompError(-8).  Calls that overlap on the GPU share (and would corrupt) that array."""
+    _check(lib().adacomp_compress_static(_dev_ptr(grad, "grad", torch.float32),
+                                         _dev_ptr(residue, "residue", torch.float32), int(n),
+                                         int(L_T), _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                         _dev_ptr(count_out, "count_out", torch.int64),
+                                         _stream(stream)),
+           "adacomp_compress_static")
 
 
 def adacomp_compress_ex(grad, residue, n: int, L_T: int, packed_out, count_out, stream=None,

@@ -1259,6 +1259,80 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------
+// pack() with the library's own scratch: for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------
+
+// Built-in scratch of adacomp_compress_static.  It is part of the loaded module: every
+// GPU that loads the library holds these bytes until the process exits.  All calls on a
+// device share it and it keeps the previous call's contents.
+static __device__ __align__(256) unsigned char g_static_scratch[ADACOMP_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch per device, looked up on the first call there.  In
+// host code the array's name is only a handle for the runtime, never a device address.
+unsigned char *g_static_scratch_addr[64];
+
+int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                         uint64_t *count_out, void *stream)
+{
+    if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
+    if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    if (misaligned(grad) || misaligned(residue) || misaligned(packed_out) ||
+        (reinterpret_cast<uintptr_t>(count_out) & 7u))
+        return ADACOMP_ERR_ALIGN;
+    const Geometry geo = make_geometry(n, L_T);
+    if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
+    if (geo.scratch_bytes > (u64)ADACOMP_STATIC_SCRATCH_BYTES) return ADACOMP_ERR_STATIC_SCRATCH;
+
+    DeviceInfo *info = nullptr;
+    int rc = device_info(info);
+    if (rc != ADACOMP_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ADACOMP_ERR_CUDA;
+    if (!g_static_scratch_addr[dev]) {
+        // set-up, once per device, with that device current
+        unsigned char *ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
+            return ADACOMP_ERR_CUDA;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    unsigned char *scratch = g_static_scratch_addr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *packed = static_cast<unsigned char *>(packed_out);
+
+    // the array keeps the last call's contents: the exact-sum windows and the group counts
+    // must start from zero; tile counts and word slots are fully rewritten before they are read
+    if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
+    if (geo.n_tiles) {
+        PassArgs args{grad, residue, packed, scratch, geo, 0u};
+        if ((L_T == 50u || L_T == 500u) && info->fast_ready) {
+            const u64 cap = (u64)info->sms * 2;
+            const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
+            if (L_T == 50u) tile_pass_fast<2, unsigned char><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            else tile_pass_fast<20, unsigned short><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+        } else {
+            rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
+                             : launch_generic<unsigned short>(args, *info, st);
+            if (rc != ADACOMP_OK) return rc;
+        }
+    }
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, 0u, reinterpret_cast<u64 *>(count_out));
+    if (geo.n_tiles) {
+        if (geo.tile_bins <= (u32)kSmallBins) {
+            const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
+            const unsigned grid = (unsigned)(want < cap ? want : cap);
+            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+        } else {
+            const u64 cap = (u64)info->sms * 8;
+            const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
+            if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+        }
+    }
+    return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------
@@ -1280,6 +1354,8 @@ const char *adacomp_strerror(int code)
     case ADACOMP_ERR_SIZE: return "tensor too large for this bin length";
     case ADACOMP_ERR_FLAGS: return "unknown flag bits";
     case ADACOMP_ERR_CUDA: return "a CUDA runtime call failed";
+    case ADACOMP_ERR_STATIC_SCRATCH:
+        return "tensor needs more scratch than the library's built-in array holds; use adacomp_compress";
     default: return "unknown error code";
     }
 }
@@ -1294,6 +1370,12 @@ int adacomp_compress(const float *grad, float *residue, uint64_t n, uint32_t L_T
                      uint64_t *count_out, void *stream)
 {
     return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0);
+}
+
+int adacomp_compress_static(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                            uint64_t *count_out, void *stream)
+{
+    return compress_static_impl(grad, residue, n, L_T, packed_out, count_out, stream);
 }
 
 int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
