@@ -67,6 +67,7 @@ extern "C" {
 #define ADACOMP_ERR_SIZE (-5)      /* n too large (n_bins must stay below 2^31) */
 #define ADACOMP_ERR_FLAGS (-6)     /* unknown flag bits */
 #define ADACOMP_ERR_CUDA (-7)      /* a CUDA runtime call failed */
+#define ADACOMP_ERR_UNSUPPORTED (-9) /* lazy mode: L_T other than 50 / 500, or flags given */
 #define ADACOMP_ERR_STATIC_SCRATCH (-8) /* adacomp_compress_static: tensor beyond the built-in scratch */
 
 /* size of the scratch array built into the library for adacomp_compress_static */
@@ -172,7 +173,33 @@ int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams,
  */
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T,
                              void *packed_out, uint64_t *count_out, void *stream, uint32_t flags,
-                             void *const *events);
+                             void *const *events, void *lazy_state /* NULL: as adacomp_compress_ex */);
+
+/*
+ * Lazy-scale pack(): the same stream, bit for bit, in one pass over the residue.
+ *
+ * In Algorithm 2 the residue of a sent element is G - Gq, and Gq = sign(G) * scale needs the
+ * layer-wide scale (Section 2.5), known only after every bin has been seen.  adacomp_compress
+ * therefore revisits the sent elements once the scale exists.  The lazy form does not: it leaves
+ * G in `residue`, records which elements were sent (one bit each) and the scale in `state`, and the
+ * NEXT adacomp_compress_lazy applies "- sign(G) * scale" to those elements as it loads them - the
+ * same single binary32 subtraction, so every later stream, scale and residue is identical.
+ *
+ *   state    device, adacomp_lazy_state_bytes(n, L_T) bytes, 16-byte aligned, set up once per
+ *            tensor by adacomp_lazy_state_init and then passed to every call for that tensor.
+ *   residue  between calls it is NOT the paper's residue: run adacomp_residue_flush before
+ *            reading it (checkpointing), before handing it to adacomp_compress, or before
+ *            changing L_T.  After a flush it is exactly what adacomp_compress would have left.
+ * Only L_T = 50 and 500 (the paper's two settings) are supported: others return
+ * ADACOMP_ERR_UNSUPPORTED (adacomp_lazy_state_bytes returns 0).  A state that does not belong to
+ * (n, L_T) sets ADACOMP_DEV_HEADER_MISMATCH and nothing is written.
+ */
+size_t adacomp_lazy_state_bytes(uint64_t n, uint32_t L_T);
+int adacomp_lazy_state_init(void *state, uint64_t n, uint32_t L_T, void *stream);
+int adacomp_compress_lazy(const float *grad, float *residue, void *state, uint64_t n, uint32_t L_T,
+                          void *packed_out, uint64_t *count_out, void *stream);
+/* Applies the pending "- sign(G) * scale" to the elements the last lazy call sent; clears the marks. */
+int adacomp_residue_flush(float *residue, void *state, uint64_t n, uint32_t L_T, void *stream);
 
 /*
  * pack() for a gradient that lives in HOST memory (Algorithm 1: serializeGrad() ->

@@ -65,7 +65,16 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate.restype = C.c_int
         L.adacomp_decompress_accumulate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
         L.adacomp_compress_profile.restype = C.c_int
-        L.adacomp_compress_profile.argtypes = L.adacomp_compress_ex.argtypes + [C.c_void_p]
+        L.adacomp_compress_profile.argtypes = L.adacomp_compress_ex.argtypes + [C.c_void_p, C.c_void_p]
+        L.adacomp_lazy_state_bytes.restype = C.c_size_t
+        L.adacomp_lazy_state_bytes.argtypes = [C.c_uint64, C.c_uint32]
+        L.adacomp_lazy_state_init.restype = C.c_int
+        L.adacomp_lazy_state_init.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p]
+        L.adacomp_compress_lazy.restype = C.c_int
+        L.adacomp_compress_lazy.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32,
+                                            C.c_void_p, C.c_void_p, C.c_void_p]
+        L.adacomp_residue_flush.restype = C.c_int
+        L.adacomp_residue_flush.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p]
         L.adacomp_compress_host.restype = C.c_int
         L.adacomp_compress_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32,
                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
@@ -167,17 +176,46 @@ def adacomp_decompress_accumulate(packed: Sequence[torch.Tensor], k_streams: int
            "adacomp_decompress_accumulate")
 
 
+def adacomp_lazy_state_bytes(n: int, L_T: int) -> int:
+    return int(lib().adacomp_lazy_state_bytes(int(n), int(L_T)))
+
+
+def adacomp_lazy_state_init(state, n: int, L_T: int, stream=None) -> None:
+    _check(lib().adacomp_lazy_state_init(_dev_ptr(state, "state", torch.uint8), int(n), int(L_T),
+                                         _stream(stream)), "adacomp_lazy_state_init")
+
+
+def adacomp_compress_lazy(grad, residue, state, n: int, L_T: int, packed_out, count_out,
+                          stream=None) -> None:
+    """Lazy-scale pack(): same stream as adacomp_compress; `residue` keeps G until the next
+    call or adacomp_residue_flush (see include/adacomp.h)."""
+    _check(lib().adacomp_compress_lazy(_dev_ptr(grad, "grad", torch.float32),
+                                       _dev_ptr(residue, "residue", torch.float32),
+                                       _dev_ptr(state, "state", torch.uint8), int(n), int(L_T),
+                                       _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                       _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
+           "adacomp_compress_lazy")
+
+
+def adacomp_residue_flush(residue, state, n: int, L_T: int, stream=None) -> None:
+    _check(lib().adacomp_residue_flush(_dev_ptr(residue, "residue", torch.float32),
+                                       _dev_ptr(state, "state", torch.uint8), int(n), int(L_T),
+                                       _stream(stream)), "adacomp_residue_flush")
+
+
 def adacomp_compress_profile(grad, residue, n: int, L_T: int, packed_out, count_out, stream=None,
-                             flags: int = 0, events: Sequence[torch.cuda.Event] = ()) -> None:
-    """adacomp_compress_ex with four torch CUDA events (already recorded once, so that
-    their handles exist) recorded around the three kernels."""
+                             flags: int = 0, events: Sequence[torch.cuda.Event] = (),
+                             lazy_state=None) -> None:
+    """adacomp_compress_ex (or, with lazy_state, adacomp_compress_lazy) with four torch CUDA
+    events (already recorded once, so that their handles exist) recorded around the three kernels."""
     assert len(events) == 4
     handles = (C.c_void_p * 4)(*[int(e.cuda_event) for e in events])
     _check(lib().adacomp_compress_profile(_dev_ptr(grad, "grad", torch.float32),
                                           _dev_ptr(residue, "residue", torch.float32), int(n),
                                           int(L_T), _dev_ptr(packed_out, "packed_out", torch.uint8),
                                           _dev_ptr(count_out, "count_out", torch.int64),
-                                          _stream(stream), int(flags), handles),
+                                          _stream(stream), int(flags), handles,
+                                          _dev_ptr(lazy_state, "lazy_state", torch.uint8)),
            "adacomp_compress_profile")
 
 

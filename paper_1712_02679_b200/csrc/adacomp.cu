@@ -41,7 +41,8 @@ constexpr int kFastTile = kSeg * kTileSegs;   // 4000 elements
 constexpr int kFastThreads = 192;    // 5 compute warps + 1 service warp
 constexpr int kStages = 3;
 constexpr u32 kTileBytes = kFastTile * 4;     // 16000
-constexpr u32 kStageBytes = 2 * kTileBytes;   // dW + residue
+constexpr u32 kMaskBytes = kTileSegs * 4;      // lazy mode: one 25-bit "sent" mask per segment
+constexpr u32 kStageBytes = 2 * kTileBytes + kMaskBytes;   // dW + residue + previous step's masks
 constexpr int kGenericThreads = 256;
 constexpr int kDecodeChunk = 4096;   // output elements per decode work item
 constexpr int kDecodeThreads = 128;
@@ -266,7 +267,24 @@ struct PassArgs {
     unsigned char *scratch;     // control block, group counts, tile counts, word slots
     Geometry geo;
     u32 literal;
+    unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
 };
+
+// Lazy-mode state: 64-byte header, then one u32 per 25-element segment (bit j = element j
+// of the segment was sent by the last step and its residue still holds G).
+constexpr u32 kLazyMagic = 0x314c4441u;     // "ADL1"
+constexpr u32 kLazyHeaderBytes = 64;
+struct LazyHeader {
+    u32 magic, L_T;
+    u64 n;
+    float scale;        // last step's scale
+    u32 steps;          // lazy steps since the last flush
+};
+
+__host__ __device__ inline u64 lazy_state_bytes(const Geometry &g)
+{
+    return kLazyHeaderBytes + align_up(g.n_tiles * (u64)kMaskBytes, 16);
+}
 
 struct FastSmem {
     static constexpr u32 kWordsAt = kStages * kStageBytes;            // 96000
@@ -281,7 +299,7 @@ struct FastSmem {
 };
 static_assert(FastSmem::kAccAt % 8 == 0, "accumulator must be 8-byte aligned");
 
-template <int SPB, typename Word>
+template <int SPB, typename Word, bool LAZY>
 __global__ void __launch_bounds__(kFastThreads, 2)
 tile_pass_fast(PassArgs a)
 {
@@ -308,6 +326,27 @@ tile_pass_fast(PassArgs a)
     const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
     const u64 full_tiles = geo.n / kFastTile;       // tiles below this index are complete
 
+    // Lazy mode: the residue buffer holds last step's G; the elements sent then still owe
+    // "- sign(G) * scale" (Algorithm 2's G - Gq), applied here as they are loaded.
+    u32 prev_scale_bits = 0;
+    u32 *lazy_mask = nullptr;
+    if (LAZY) {
+        const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(a.lazy_state);
+        if (lh->magic != kLazyMagic || lh->n != a.geo.n || lh->L_T != a.geo.L_T) {
+            // not the state of this tensor (the same verdict in every CTA): touch neither residue
+            // nor state, and report every tile as empty so that the kernels after this one see a
+            // consistent, empty stream
+            if (threadIdx.x == 0) {
+                if (blockIdx.x == 0) raise_status(ADACOMP_DEV_HEADER_MISMATCH);
+                u32 *counts = reinterpret_cast<u32 *>(a.scratch + a.geo.tile_cnt_at);
+                for (u64 t = blockIdx.x; t < a.geo.n_tiles; t += gridDim.x) counts[t] = 0;
+            }
+            return;
+        }
+        prev_scale_bits = __float_as_uint(lh->scale) & 0x7fffffffu;
+        lazy_mask = reinterpret_cast<u32 *>(a.lazy_state + kLazyHeaderBytes);
+    }
+
     if (tid < kWindows + 1) s_acc[tid] = 0;
     if (tid == 0) {
         *s_abort = 0;
@@ -322,9 +361,10 @@ tile_pass_fast(PassArgs a)
         if (i >= my_tiles || tile >= full_tiles) return;
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        mbar_arrive_expect_tx(bar, kStageBytes);
+        mbar_arrive_expect_tx(bar, 2 * kTileBytes + (LAZY ? kMaskBytes : 0u));
         bulk_load(st, a.grad + tile * (u64)kFastTile, kTileBytes, bar);
         bulk_load(st + kTileBytes, a.residue + tile * (u64)kFastTile, kTileBytes, bar);
+        if (LAZY) bulk_load(st + 2 * kTileBytes, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
         issued = i + 1;
     };
     if (service && lane == 0) {
@@ -338,6 +378,7 @@ tile_pass_fast(PassArgs a)
         const u64 base = tile * (u64)kFastTile;
         float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
         float *s_r = s_d + kFastTile;
+        const u32 *s_prev = reinterpret_cast<const u32 *>(s_r + kFastTile);
         const bool whole = tile < full_tiles;
         const int elems = whole ? kFastTile : (int)(geo.n - base);
 
@@ -354,6 +395,8 @@ tile_pass_fast(PassArgs a)
                 s_d[e] = d;
                 s_r[e] = r;
             }
+            if (LAZY && tid < kTileSegs)
+                const_cast<u32 *>(s_prev)[tid] = lazy_mask[tile * (u64)kTileSegs + tid];
             __syncthreads();
         }
 
@@ -365,10 +408,18 @@ tile_pass_fast(PassArgs a)
             const float *pd = s_d + tid * kSeg;
             const float *pr = s_r + tid * kSeg;
             float m = 0.f;
+            const u32 prev = LAZY ? s_prev[tid] : 0u;
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
                 const float d = pd[j];
-                g[j] = __fadd_rn(pr[j], d);
+                float r = pr[j];
+                if (LAZY) {
+                    // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
+                    const float q = __uint_as_float(prev_scale_bits | (__float_as_uint(r) & 0x80000000u));
+                    const float fixed = __fsub_rn(r, q);
+                    r = (prev >> j & 1u) ? fixed : r;
+                }
+                g[j] = __fadd_rn(r, d);
                 const float h = __fadd_rn(g[j], d);
                 m = fmaxf(m, fabsf(g[j]));
                 // |G| never exceeds the bin maximum, so "|H| >= g_max or |G| == g_max"
@@ -422,6 +473,7 @@ tile_pass_fast(PassArgs a)
                 const u32 neg = __float_as_uint(pr[j]) >> 31;
                 s_words[at++] = (Word)(((seg_in_bin + j) << 2) | 1u | (neg << 1));
             }
+            if (LAZY) lazy_mask[tile * (u64)kTileSegs + tid] = selmask;
             if (tid % SPB == 0) {
                 const u64 bin = tile * (u64)kBins + tid / SPB;
                 const int t1 = tid + SPB - 1;
@@ -467,10 +519,13 @@ tile_pass_fast(PassArgs a)
     if (service) {
         if (lane == 0) {
             bulk_wait_all();
-            // after a timeout: loads still in flight must land (or time out in turn)
-            // before this CTA's shared memory is given back
-            if (*s_abort)
+            if (*s_abort) {
+                // after a timeout: loads still in flight must land (or time out in turn) before
+                // this CTA's shared memory is given back, and the tiles it never finished count
+                // as empty so that the kernels after this one stay inside their buffers
                 for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % kStages], (u32)(j / kStages) & 1u);
+                for (u64 j = i; j < my_tiles; j++) tile_cnt[first + j * stride] = 0;
+            }
         }
         if (lane < kWindows) {
             const u64 v = s_acc[lane];
@@ -638,7 +693,8 @@ __device__ double windows_to_double(const u64 *win)
 }
 
 __global__ void __launch_bounds__(1024)
-finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out)
+finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out,
+         unsigned char *lazy_state)
 {
     __shared__ u64 s_warp[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -700,6 +756,13 @@ finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags,
         h64[7] = bytes_used;
         count_out[0] = n_sel;
         count_out[1] = bytes_used;
+        if (lazy_state) {
+            LazyHeader *lh = reinterpret_cast<LazyHeader *>(lazy_state);
+            if (lh->magic == kLazyMagic && lh->n == geo.n && lh->L_T == geo.L_T) {
+                lh->scale = scale;      // the next step (or a flush) finishes the sent residues with it
+                lh->steps += 1;
+            }
+        }
     }
     // zero padding behind the last word, and the alignment gaps of the directory sections
     const u64 pay_end = geo.payload_at + n_sel * geo.w;
@@ -730,12 +793,12 @@ __device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &
     const u32 c = t < geo.n_tiles ? tile_cnt[t] : 0u;
     u32 before = lane < me ? c : 0u;
     for (int d = 16; d > 0; d >>= 1) before += __shfl_xor_sync(0xffffffffu, before, d);
-    count = __shfl_sync(0xffffffffu, c, me);
+    count = min(__shfl_sync(0xffffffffu, c, me), geo.tile_elems);
     return group[g] + before;
 }
 
 // Tiles of at most 96 bins: one warp per tile.
-template <typename Word>
+template <typename Word, bool FIXUP>
 __global__ void __launch_bounds__(kGatherThreads)
 gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *scratch, Geometry geo)
 {
@@ -754,9 +817,10 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
         const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
         if (lane == 0) tile_off[tile] = off0;
         if (cnt == 0) continue;
-        // exclusive scan of the tile's bin counts, three bins per lane
+        // exclusive scan of the tile's bin counts, three bins per lane (only the fix-up needs bins)
         const u64 bin0 = tile * (u64)TB;
         u32 c[3], sum = 0;
+        if (FIXUP) {
 #pragma unroll
         for (int q = 0; q < 3; q++) {
             const int b = lane * 3 + q;
@@ -774,6 +838,7 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
         }
         if (lane == 31) s_pre[TB] = inc;
         __syncwarp();
+        }
         const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
         const u64 base = tile * (u64)geo.tile_elems;
         for (u32 j0 = 0; j0 < cnt; j0 += 128) {
@@ -789,16 +854,18 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
                 g[q] = 0.f;
                 if (j < cnt) {
                     word[q] = slot[j];
-                    const int b = bin_of_word(s_pre, TB, j);
-                    pos[q] = base + (u64)b * geo.L_T + (word[q] >> 2);
-                    g[q] = residue[pos[q]];
+                    if (FIXUP) {
+                        const int b = bin_of_word(s_pre, TB, j);
+                        pos[q] = base + (u64)b * geo.L_T + (word[q] >> 2);
+                        g[q] = residue[pos[q]];
+                    }
                 }
             }
 #pragma unroll
             for (int q = 0; q < 4; q++) {
                 const u32 j = j0 + q * 32 + lane;
                 if (j < cnt) {
-                    residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
+                    if (FIXUP) residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
                     payload[off0 + j] = (Word)word[q];
                 }
             }
@@ -862,11 +929,21 @@ struct DecodeArgs {
     u32 k;
 };
 
+constexpr int kWbufBytes = 16384;    // staged words of one round of learners
+constexpr int kRoundMax = 8;         // learners per round
+
 struct DecodeSmem {
     float acc[kDecodeChunk];                    // the output tile
-    u32 pre[kMaxTileBins + 1];                  // scanned bin counts
+    union {
+        u32 pre[kMaxTileBins + 1];              // generic path: scanned bin counts of one stream
+        struct {
+            uint4 wbuf[kWbufBytes / 16];        // fast paths: the round's words, staged
+            u32 bin_pre[kRoundMax][33];         // by-word path: scanned bin counts per learner
+        } f;
+    };
     u32 tmp[40];
     u64 off0[ADACOMP_MAX_STREAMS];              // first word of this tile in stream l
+    u32 cnt[ADACOMP_MAX_STREAMS];               // words of this tile in stream l
     u64 n_sel[ADACOMP_MAX_STREAMS];             // words in stream l
     float scale[ADACOMP_MAX_STREAMS];
 };
@@ -887,126 +964,152 @@ __device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc)
     }
 }
 
-// Tiles of 32..96 bins (L_T = 42..125): thread b owns bin b for every learner, so the
-// learners' contributions to an element are added by one thread, in learner order,
-// without any barrier between learners.
-template <typename Word>
-__device__ void decode_by_bin(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
+// Fast decode for tiles of at most 96 bins and 4096 elements (L_T = 42..1000).
+//
+// Per tile: (1) each learner's word range comes from its directory; (2) the words of a
+// round of up to eight learners are staged in shared memory with 16-byte loads, all in
+// flight together; (3) the words are added into the output tile in learner order:
+//   BY_BIN  (32..96 bins): thread b owns bin b for every learner, so one thread adds all
+//           contributions to an element, in learner order, with no barrier in between;
+//   by word (2..31 bins): a learner's words are spread over the threads and a barrier
+//           separates consecutive learners;
+// (4) the tile is stored once with 128-bit streaming stores.
+template <typename Word, bool BY_BIN>
+__device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
-    u32 *s_wsum = sm.tmp;        // [4 warps][8 learners of a round]
+    u32 *s_wsum = sm.tmp;                      // BY_BIN: [4 warps][8 learners]
+    const unsigned char *s_bytes = reinterpret_cast<const unsigned char *>(sm.f.wbuf);
     for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
     if (tid < (int)a.k) {
         sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
         sm.n_sel[tid] = reinterpret_cast<const u64 *>(a.stream[tid])[5];
     }
-    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
-        const u64 base = tile * (u64)geo.tile_elems;
-        const u64 bin = tile * (u64)TB + tid;
-        const bool live = tid < TB && bin < geo.n_bins;
-        if (tid < (int)a.k)
-            sm.off0[tid] = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at)[tile];
-        for (u32 l0 = 0; l0 < a.k; l0 += 8) {
-            const int round = (int)min(8u, a.k - l0);
-            u32 c[8], pre[8];
-#pragma unroll
-            for (int q = 0; q < 8; q++) {
-                c[q] = 0;
-                if (q < round && live)
-                    c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin], geo.L_T);
-                const u32 inc = warp_inclusive_scan(c[q], lane);
-                pre[q] = inc - c[q];
-                if (lane == 31) s_wsum[warp * 8 + q] = inc;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int q = 0; q < 8; q++)
-                for (int wv = 0; wv < warp; wv++) pre[q] += s_wsum[wv * 8 + q];
-            float *mine = sm.acc + tid * geo.L_T;
-#pragma unroll
-            for (int q = 0; q < 8; q++) {
-                if (q >= round || c[q] == 0) continue;
-                const u64 at0 = sm.off0[l0 + q] + pre[q];
-                if (at0 + c[q] > sm.n_sel[l0 + q]) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                const Word *p = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.payload_at) + at0;
-                const float scale = sm.scale[l0 + q];
-                for (u32 i = 0; i < c[q]; i++) {
-                    const u32 word = p[i];
-                    const u32 code = word & 3u, idx = word >> 2;
-                    if (code == 0u) continue;
-                    if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                    if (idx >= geo.L_T || base + (u64)tid * geo.L_T + idx >= geo.n) {
-                        raise_status(ADACOMP_DEV_BAD_STREAM);
-                        continue;
-                    }
-                    mine[idx] = code == 3u ? __fsub_rn(mine[idx], scale) : __fadd_rn(mine[idx], scale);
-                }
-            }
-            __syncthreads();
-        }
-        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
-        store_tile(a.dst, base, len, sm.acc);
-        __syncthreads();
-    }
-}
-
-// Tiles of 2..31 bins (L_T = 126..1000): the words of one learner are spread over the
-// threads; a barrier separates consecutive learners.
-template <typename Word>
-__device__ void decode_by_word(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int TB = (int)geo.tile_bins;
-    u32 (*s_pre)[33] = reinterpret_cast<u32 (*)[33]>(sm.pre);      // [learner of the round][bin]
-    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
-    if (tid < (int)a.k) {
-        sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
-        sm.n_sel[tid] = reinterpret_cast<const u64 *>(a.stream[tid])[5];
+    // directory entries of the first tile; those of the next tile are fetched one tile ahead
+    u64 nx0 = 0, nx1 = 0;
+    if (tid < (int)a.k && blockIdx.x < geo.n_tiles) {
+        const u64 *dir = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at);
+        nx0 = dir[blockIdx.x];
+        nx1 = dir[blockIdx.x + 1];
     }
     for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
         const u64 base = tile * (u64)geo.tile_elems;
         const u64 bin0 = tile * (u64)TB;
-        for (u32 l0 = 0; l0 < a.k; l0 += 32) {
-            const int round = (int)min(32u, a.k - l0);
-            // warp wv scans the bin counts of learners wv, wv + 4, ... of this round
-            for (int q = warp; q < round; q += kDecodeThreads / 32) {
-                const unsigned char *s = a.stream[l0 + q];
-                u32 c = 0;
-                if (lane < TB && bin0 + lane < geo.n_bins)
-                    c = reinterpret_cast<const Word *>(s + geo.bin_cnt_at)[bin0 + lane];
-                const u32 inc = warp_inclusive_scan(c, lane);
-                s_pre[q][lane] = inc - c;
-                if (lane == 31) {
-                    s_pre[q][32] = inc;
-                    sm.off0[l0 + q] = reinterpret_cast<const u64 *>(s + geo.tile_off_at)[tile];
-                }
+        if (tid < (int)a.k) {
+            // a malformed directory must not send the copy below out of the stream
+            const bool ok = nx1 >= nx0 && nx1 - nx0 <= geo.tile_elems && nx1 <= sm.n_sel[tid];
+            if (!ok) raise_status(ADACOMP_DEV_BAD_STREAM);
+            sm.off0[tid] = nx0;
+            sm.cnt[tid] = ok ? (u32)(nx1 - nx0) : 0u;
+            const u64 next = tile + gridDim.x;
+            if (next < geo.n_tiles) {
+                const u64 *dir = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at);
+                nx0 = dir[next];
+                nx1 = dir[next + 1];
             }
-            __syncthreads();
-            for (int q = 0; q < round; q++) {
-                const u32 cnt = s_pre[q][32];         // the same for every thread
-                if (cnt == 0) continue;
-                if (cnt > geo.tile_elems || sm.off0[l0 + q] + cnt > sm.n_sel[l0 + q]) {
-                    if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM);
-                    continue;
+        }
+        __syncthreads();
+
+        u32 l0 = 0;
+        while (l0 < a.k) {
+            // ---- the round: learners [l0, l1) whose words fit the staging buffer ----
+            u32 at[kRoundMax + 1], head[kRoundMax];      // 16-byte chunk index / misalignment of each learner
+            u32 l1 = l0;
+            at[0] = 0;
+            while (l1 < a.k && l1 - l0 < (u32)kRoundMax) {
+                const u32 q = l1 - l0;
+                const u64 src = (u64)(uintptr_t)(a.stream[l1] + geo.payload_at) + sm.off0[l1] * sizeof(Word);
+                head[q] = (u32)(src & 15u);
+                const u32 chunks = sm.cnt[l1] ? (head[q] + sm.cnt[l1] * (u32)sizeof(Word) + 15u) / 16u : 0u;
+                if (at[q] + chunks > (u32)(kWbufBytes / 16)) break;
+                at[q + 1] = at[q] + chunks;
+                l1++;
+            }
+            const int round = (int)(l1 - l0);            // >= 1: one learner's tile always fits
+            // ---- stage the words: every 16-byte load of the round is issued before any is used ----
+            for (u32 c = tid; c < at[round]; c += kDecodeThreads) {
+                int q = 0;
+#pragma unroll
+                for (int t = 1; t < kRoundMax; t++)
+                    if (t < round && c >= at[t]) q = t;
+                const u64 src = ((u64)(uintptr_t)(a.stream[l0 + q] + geo.payload_at) +
+                                 sm.off0[l0 + q] * sizeof(Word)) & ~(u64)15u;
+                sm.f.wbuf[c] = __ldg(reinterpret_cast<const uint4 *>(src) + (c - at[q]));
+            }
+            if (BY_BIN) {
+                const u64 bin = bin0 + tid;
+                const bool live = tid < TB && bin < geo.n_bins;
+                u32 c[kRoundMax], pre[kRoundMax];
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    c[q] = 0;
+                    if (q < round && live)
+                        c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin], geo.L_T);
                 }
-                const Word *p = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.payload_at) + sm.off0[l0 + q];
-                const float scale = sm.scale[l0 + q];
-                for (u32 j = tid; j < cnt; j += kDecodeThreads) {
-                    const u32 word = p[j];
-                    const u32 code = word & 3u, idx = word >> 2;
-                    if (code == 0u) continue;
-                    if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                    int b = 0;
-                    for (int step = 16; step > 0; step >>= 1)       // at most 31 bins: five probes
-                        if (b + step < TB && s_pre[q][b + step] <= j) b += step;
-                    const u32 at = (u32)b * geo.L_T + idx;
-                    if (idx >= geo.L_T || base + at >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                    sm.acc[at] = code == 3u ? __fsub_rn(sm.acc[at], scale) : __fadd_rn(sm.acc[at], scale);
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    const u32 inc = warp_inclusive_scan(c[q], lane);
+                    pre[q] = inc - c[q];
+                    if (lane == 31) s_wsum[warp * kRoundMax + q] = inc;
                 }
                 __syncthreads();
+                float *mine = sm.acc + tid * geo.L_T;
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    if (q >= round || c[q] == 0) continue;
+                    for (int wv = 0; wv < warp; wv++) pre[q] += s_wsum[wv * kRoundMax + q];
+                    if (pre[q] + c[q] > sm.cnt[l0 + q]) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                    const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + head[q]) + pre[q];
+                    const float scale = sm.scale[l0 + q];
+                    for (u32 i = 0; i < c[q]; i++) {
+                        const u32 word = p[i];
+                        const u32 code = word & 3u, idx = word >> 2;
+                        if (code == 0u) continue;
+                        if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
+                        if (idx >= geo.L_T || base + (u64)tid * geo.L_T + idx >= geo.n) {
+                            raise_status(ADACOMP_DEV_BAD_STREAM);
+                            continue;
+                        }
+                        mine[idx] = code == 3u ? __fsub_rn(mine[idx], scale) : __fadd_rn(mine[idx], scale);
+                    }
+                }
+                __syncthreads();
+            } else {
+                // warp wv scans the bin counts of learners wv, wv + 4 of the round
+                for (int q = warp; q < round; q += kDecodeThreads / 32) {
+                    u32 c = 0;
+                    if (lane < TB && bin0 + lane < geo.n_bins)
+                        c = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin0 + lane];
+                    const u32 inc = warp_inclusive_scan(c, lane);
+                    sm.f.bin_pre[q][lane] = inc - c;
+                    if (lane == 31) sm.f.bin_pre[q][32] = inc;
+                }
+                __syncthreads();
+                for (int q = 0; q < round; q++) {
+                    const u32 cnt = sm.cnt[l0 + q];           // the same for every thread
+                    if (cnt == 0) continue;
+                    if (sm.f.bin_pre[q][32] != cnt) { if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                    const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + head[q]);
+                    const float scale = sm.scale[l0 + q];
+                    for (u32 j = tid; j < cnt; j += kDecodeThreads) {
+                        const u32 word = p[j];
+                        const u32 code = word & 3u, idx = word >> 2;
+                        if (code == 0u) continue;
+                        if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
+                        int b = 0;
+#pragma unroll
+                        for (int step = 16; step > 0; step >>= 1)       // at most 31 bins: five probes
+                            if (b + step < TB && sm.f.bin_pre[q][b + step] <= j) b += step;
+                        const u32 e = (u32)b * geo.L_T + idx;
+                        if (idx >= geo.L_T || base + e >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                        sm.acc[e] = code == 3u ? __fsub_rn(sm.acc[e], scale) : __fadd_rn(sm.acc[e], scale);
+                    }
+                    __syncthreads();
+                }
+                __syncthreads();     // bin_pre and wbuf are rewritten by the next round
             }
-            __syncthreads();
+            l0 = l1;
         }
         const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
         store_tile(a.dst, base, len, sm.acc);
@@ -1108,16 +1211,55 @@ decode_sum(DecodeArgs a)
     const bool by_bin = geo.tile_bins >= 32 && geo.tile_bins <= (u32)kSmallBins;
     const bool by_word = geo.tile_bins >= 2 && geo.tile_bins <= 31;
     if (geo.w == 1u) {
-        if (by_bin) decode_by_bin<unsigned char>(a, geo, sm);
+        if (by_bin) decode_staged<unsigned char, true>(a, geo, sm);
         else decode_generic<unsigned char>(a, geo, sm);
     } else {
-        if (by_bin) decode_by_bin<unsigned short>(a, geo, sm);
-        else if (by_word) decode_by_word<unsigned short>(a, geo, sm);
+        if (by_bin) decode_staged<unsigned short, true>(a, geo, sm);
+        else if (by_word) decode_staged<unsigned short, false>(a, geo, sm);
         else decode_generic<unsigned short>(a, geo, sm);
     }
 }
 
 __global__ void reset_status_kernel() { g_status = 0; }
+
+__global__ void lazy_init_kernel(unsigned char *state, u64 n, u32 L_T)
+{
+    LazyHeader *lh = reinterpret_cast<LazyHeader *>(state);
+    lh->magic = kLazyMagic;
+    lh->L_T = L_T;
+    lh->n = n;
+    lh->scale = 0.f;
+    lh->steps = 0;
+}
+
+// residue_flush: finish "residue = G - sign(G) * scale" for the elements the last lazy step sent,
+// and clear their marks.  One thread per 25-element segment.
+__global__ void __launch_bounds__(256)
+lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T)
+{
+    const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(state);
+    if (lh->magic != kLazyMagic || lh->n != n || lh->L_T != L_T) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) raise_status(ADACOMP_DEV_HEADER_MISMATCH);
+        return;
+    }
+    const u32 sbits = __float_as_uint(lh->scale) & 0x7fffffffu;
+    u32 *mask = reinterpret_cast<u32 *>(state + kLazyHeaderBytes);
+    const u64 segs = (n + kSeg - 1) / kSeg;
+    for (u64 sgm = (u64)blockIdx.x * blockDim.x + threadIdx.x; sgm < segs; sgm += (u64)gridDim.x * blockDim.x) {
+        u32 m = mask[sgm];
+        if (m == 0) continue;
+        mask[sgm] = 0;
+        while (m) {
+            const int j = __ffs(m) - 1;
+            m &= m - 1;
+            const u64 i = sgm * kSeg + j;
+            if (i < n) {
+                const float r = residue[i];
+                residue[i] = __fsub_rn(r, __uint_as_float(sbits | (__float_as_uint(r) & 0x80000000u)));
+            }
+        }
+    }
+}
 
 // ---------------------------------------------------------------------------------
 // host side
@@ -1146,11 +1288,12 @@ int device_info(DeviceInfo *&out)
         int per_sm = 1;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
-        d.fast_ready =
-            cudaFuncSetAttribute(tile_pass_fast<2, unsigned char>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)FastSmem::kBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(tile_pass_fast<20, unsigned short>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)FastSmem::kBytes) == cudaSuccess;
+        const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        const int bytes = (int)FastSmem::kBytes;
+        d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
+                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false>, at, bytes) == cudaSuccess &&
+                       cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, true>, at, bytes) == cudaSuccess &&
+                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, true>, at, bytes) == cudaSuccess;
         d.sms = sms;
     }
     out = &d;
@@ -1178,7 +1321,8 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 }
 
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
-                  uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr)
+                  uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
+                  void *lazy_state = nullptr)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
@@ -1188,13 +1332,18 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         return ADACOMP_ERR_ALIGN;
     const Geometry geo = make_geometry(n, L_T);
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
+    unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
+    if (lazy) {
+        if ((L_T != 50u && L_T != 500u) || flags != 0) return ADACOMP_ERR_UNSUPPORTED;
+        if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
+    }
 
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
+    if (lazy && !info->fast_ready) return ADACOMP_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char *packed = static_cast<unsigned char *>(packed_out);
-
     unsigned char *scratch = packed + geo.scratch_at;
 
     // the exact-sum windows and the group counts start from zero
@@ -1204,13 +1353,19 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy};
         const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
         if (fast) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (L_T == 50u) tile_pass_fast<2, unsigned char><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
-            else tile_pass_fast<20, unsigned short><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            const size_t sm = FastSmem::kBytes;
+            if (lazy) {
+                if (L_T == 50u) tile_pass_fast<2, unsigned char, true><<<grid, kFastThreads, sm, st>>>(args);
+                else tile_pass_fast<20, unsigned short, true><<<grid, kFastThreads, sm, st>>>(args);
+            } else {
+                if (L_T == 50u) tile_pass_fast<2, unsigned char, false><<<grid, kFastThreads, sm, st>>>(args);
+                else tile_pass_fast<20, unsigned short, false><<<grid, kFastThreads, sm, st>>>(args);
+            }
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
@@ -1218,14 +1373,19 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         }
     }
     mark(1);
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags, reinterpret_cast<u64 *>(count_out));
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags, reinterpret_cast<u64 *>(count_out), lazy);
     mark(2);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
             const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
             const unsigned grid = (unsigned)(want < cap ? want : cap);
-            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            if (lazy) {     // the residue keeps G; only the words move
+                if (geo.w == 1u) gather_fixup_small<unsigned char, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+                else gather_fixup_small<unsigned short, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            } else {
+                if (geo.w == 1u) gather_fixup_small<unsigned char, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+                else gather_fixup_small<unsigned short, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            }
         } else {
             const u64 cap = (u64)info->sms * 8;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
@@ -1304,25 +1464,25 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     // must start from zero; tile counts and word slots are fully rewritten before they are read
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, 0u};
+        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr};
         if ((L_T == 50u || L_T == 500u) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (L_T == 50u) tile_pass_fast<2, unsigned char><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
-            else tile_pass_fast<20, unsigned short><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            if (L_T == 50u) tile_pass_fast<2, unsigned char, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            else tile_pass_fast<20, unsigned short, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
             if (rc != ADACOMP_OK) return rc;
         }
     }
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, 0u, reinterpret_cast<u64 *>(count_out));
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, 0u, reinterpret_cast<u64 *>(count_out), nullptr);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
             const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
             const unsigned grid = (unsigned)(want < cap ? want : cap);
-            if (geo.w == 1u) gather_fixup_small<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-            else gather_fixup_small<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            if (geo.w == 1u) gather_fixup_small<unsigned char, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
+            else gather_fixup_small<unsigned short, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
         } else {
             const u64 cap = (u64)info->sms * 8;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
@@ -1354,6 +1514,7 @@ const char *adacomp_strerror(int code)
     case ADACOMP_ERR_SIZE: return "tensor too large for this bin length";
     case ADACOMP_ERR_FLAGS: return "unknown flag bits";
     case ADACOMP_ERR_CUDA: return "a CUDA runtime call failed";
+    case ADACOMP_ERR_UNSUPPORTED: return "lazy mode supports L_T = 50 and 500 without flags only";
     case ADACOMP_ERR_STATIC_SCRATCH:
         return "tensor needs more scratch than the library's built-in array holds; use adacomp_compress";
     default: return "unknown error code";
@@ -1390,12 +1551,52 @@ int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams,
 }
 
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
-                             uint64_t *count_out, void *stream, uint32_t flags, void *const *events)
+                             uint64_t *count_out, void *stream, uint32_t flags, void *const *events,
+                             void *lazy_state)
 {
     if (!events) return ADACOMP_ERR_NULL;
     for (int i = 0; i < 4; i++)
         if (!events[i]) return ADACOMP_ERR_NULL;
-    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, flags, events);
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, flags, events, lazy_state);
+}
+
+size_t adacomp_lazy_state_bytes(uint64_t n, uint32_t L_T)
+{
+    if (L_T != 50u && L_T != 500u) return 0;
+    return (size_t)lazy_state_bytes(make_geometry(n, L_T));
+}
+
+int adacomp_lazy_state_init(void *state, uint64_t n, uint32_t L_T, void *stream)
+{
+    if (!state) return ADACOMP_ERR_NULL;
+    if (L_T != 50u && L_T != 500u) return ADACOMP_ERR_UNSUPPORTED;
+    if (misaligned(state)) return ADACOMP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(state, 0, lazy_state_bytes(make_geometry(n, L_T)), st) != cudaSuccess) return ADACOMP_ERR_CUDA;
+    lazy_init_kernel<<<1, 1, 0, st>>>(static_cast<unsigned char *>(state), n, L_T);
+    return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+}
+
+int adacomp_compress_lazy(const float *grad, float *residue, void *state, uint64_t n, uint32_t L_T,
+                          void *packed_out, uint64_t *count_out, void *stream)
+{
+    if (!state) return ADACOMP_ERR_NULL;
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, state);
+}
+
+int adacomp_residue_flush(float *residue, void *state, uint64_t n, uint32_t L_T, void *stream)
+{
+    if (!state || (n && !residue)) return ADACOMP_ERR_NULL;
+    if (L_T != 50u && L_T != 500u) return ADACOMP_ERR_UNSUPPORTED;
+    if (misaligned(residue) || misaligned(state)) return ADACOMP_ERR_ALIGN;
+    DeviceInfo *info = nullptr;
+    int rc = device_info(info);
+    if (rc != ADACOMP_OK) return rc;
+    const u64 segs = (n + kSeg - 1) / kSeg;
+    const u64 want = (segs + 255) / 256, cap = (u64)info->sms * 8;
+    const unsigned grid = (unsigned)(want < 1 ? 1 : (want < cap ? want : cap));
+    lazy_flush_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(residue, static_cast<unsigned char *>(state), n, L_T);
+    return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
 int adacomp_compress_host(const float *grad_host, float *grad_stage, float *residue, uint64_t n, uint32_t L_T,
