@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--learners", type=int, default=4)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-lazy", action="store_true")
     ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
     return ap.parse_args()
 
@@ -234,9 +235,55 @@ def run_ours(a):
     snap = [r.clone() for r in residue]
     torch.cuda.synchronize()
 
-    def restore():
+    lazy_state, lazy_snap = [], []
+
+    def restore(lazy=False):
         for r, s in zip(residue, snap):
             r.copy_(s)
+        if lazy:
+            for st_, s in zip(lazy_state, lazy_snap):
+                st_.copy_(s)
+
+    def pack(l, lazy=False):
+        if lazy:
+            B.adacomp_compress_lazy(dW[l], residue[l], lazy_state[l], n, L_T, packed[l], count[l], stream)
+        else:
+            B.adacomp_compress(dW[l], residue[l], n, L_T, packed[l], count[l], stream)
+
+    def timed_steps(lazy, with_clocks):
+        """W warm-up + K timed steps; returns per-step (pack ms, decode ms) and the total ms."""
+        evs = []
+        for it in range(W + K):
+            if it == W:
+                barrier()
+                if with_clocks and rank == 0:
+                    sampler.start()
+            restore(lazy)
+            e = step_events()
+            e[0].record(stream)
+            for l in range(k):
+                pack(l, lazy)
+            e[1].record(stream)
+            B.adacomp_decompress_accumulate(packed, k, dst, stream)
+            e[2].record(stream)
+            if it >= W:
+                evs.append(e)
+        barrier()
+        return ([e[0].elapsed_time(e[1]) for e in evs], [e[1].elapsed_time(e[2]) for e in evs],
+                sum(e[0].elapsed_time(e[2]) for e in evs))
+
+    def profile_pack(lazy):
+        """Mean device time of the three kernels of one learner's pack(), CUDA events."""
+        prof = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+        for row in prof:
+            for e in row:
+                e.record(stream)           # creates the handles
+        for row in prof:
+            restore(lazy)
+            B.adacomp_compress_profile(dW[0], residue[0], n, L_T, packed[0], count[0], stream, 0, row,
+                                       lazy_state[0] if lazy else None)
+        torch.cuda.synchronize()
+        return tuple(statistics.mean(r[i].elapsed_time(r[i + 1]) for r in prof) for i in range(3))
 
     def step_events():
         return [torch.cuda.Event(enable_timing=True) for _ in range(3)]
@@ -244,40 +291,9 @@ def run_ours(a):
     # ---- timed region: device-resident inputs ----
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
                            else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
-    evs = []
-    for it in range(W + K):
-        if it == W:
-            barrier()
-            if rank == 0:
-                sampler.start()
-        restore()
-        e = step_events()
-        e[0].record(stream)
-        for l in range(k):
-            B.adacomp_compress(dW[l], residue[l], n, L_T, packed[l], count[l], stream)
-        e[1].record(stream)
-        B.adacomp_decompress_accumulate(packed, k, dst, stream)
-        e[2].record(stream)
-        if it >= W:
-            evs.append(e)
-    barrier()
-    t_comp = [e[0].elapsed_time(e[1]) for e in evs]
-    t_dec = [e[1].elapsed_time(e[2]) for e in evs]
-    t_total_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
-
-    # ---- per-kernel durations of pack() (learner 0), same protocol, CUDA events ----
-    prof = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    for row in prof:
-        for e in row:
-            e.record(stream)           # creates the handles
-    for row in prof:
-        restore()
-        B.adacomp_compress_profile(dW[0], residue[0], n, L_T, packed[0], count[0], stream, 0, row)
-    torch.cuda.synchronize()
+    t_comp, t_dec, t_total_ms = timed_steps(False, True)
+    t_tile, t_fin, t_fix = profile_pack(False)
     clocks = sampler.stop() if rank == 0 else None
-    t_tile = statistics.mean(r[0].elapsed_time(r[1]) for r in prof)
-    t_fin = statistics.mean(r[1].elapsed_time(r[2]) for r in prof)
-    t_fix = statistics.mean(r[2].elapsed_time(r[3]) for r in prof)
 
     status = B.adacomp_device_status(stream)
     counts = [tuple(int(v) for v in c.cpu()) for c in count]
@@ -320,16 +336,53 @@ def run_ours(a):
                "steps": Ke}
         del h_dW, h_packed, h_dst, stage
 
+    # ---- the same steps with lazy-scale pack(): identical streams, one pass over the residue ----
+    lazy = None
+    if L_T in (50, 500) and not a.no_lazy:
+        eager_counts = [tuple(int(v) for v in c.cpu()) for c in count]
+        for r in residue:
+            r.zero_()
+        nbytes = B.adacomp_lazy_state_bytes(n, L_T)
+        for l in range(k):
+            lazy_state.append(torch.empty(nbytes, dtype=torch.uint8, device=dev))
+            B.adacomp_lazy_state_init(lazy_state[l], n, L_T, stream)
+        keep = [d.clone() for d in dW] if 4 * n * k < (8 << 30) else None
+        for step in range(PREWARM_STEPS + 1):
+            for l in range(k):
+                gen.manual_seed(1712_02679 + 1000003 * rank + 1009 * l + step)
+                dW[l].normal_(0.0, SIGMA, generator=gen)
+                if step < PREWARM_STEPS:
+                    pack(l, True)
+        if keep is not None:
+            assert all(torch.equal(a_, b_) for a_, b_ in zip(keep, dW)), "seeded dW not reproducible"
+            del keep
+        for r, s_ in zip(residue, snap):
+            s_.copy_(r)                         # now holds step 5's G plus the pending marks in the state
+        lazy_snap.extend(st_.clone() for st_ in lazy_state)
+        torch.cuda.synchronize()
+        lz_comp, lz_dec, lz_total = timed_steps(True, False)
+        lz_tile, lz_fin, lz_gather = profile_pack(True)
+        lazy_counts = [tuple(int(v) for v in c.cpu()) for c in count]
+        lazy = {"same_counts_as_eager": lazy_counts == eager_counts, "t_comp": statistics.mean(lz_comp),
+                "t_dec": statistics.mean(lz_dec), "total_ms": lz_total,
+                "kernels": {"tile_pass": lz_tile, "finalize": lz_fin, "gather": lz_gather},
+                "state_bytes": nbytes}
+        restore(False)
+
+
     # ---- max over ranks ----
+    m_comp, m_dec = statistics.mean(t_comp), statistics.mean(t_dec)
     if world > 1:
-        t = torch.tensor([t_total_ms, statistics.mean(t_comp), statistics.mean(t_dec),
-                          e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        t = torch.tensor([t_total_ms, m_comp, m_dec, e2e["ms"] if e2e else 0.0,
+                          lazy["total_ms"] if lazy else 0.0, lazy["t_comp"] if lazy else 0.0,
+                          lazy["t_dec"] if lazy else 0.0], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_total_ms, m_comp, m_dec, e2e_ms = (float(x) for x in t.cpu())
+        v = [float(x) for x in t.cpu()]
+        t_total_ms, m_comp, m_dec = v[0], v[1], v[2]
         if e2e:
-            e2e["ms"] = e2e_ms
-    else:
-        m_comp, m_dec = statistics.mean(t_comp), statistics.mean(t_dec)
+            e2e["ms"] = v[3]
+        if lazy:
+            lazy["total_ms"], lazy["t_comp"], lazy["t_dec"] = v[4], v[5], v[6]
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -367,6 +420,19 @@ def run_ours(a):
             "clocks": clocks,
             "gpu_launches": K * (3 * k + 1),
         }
+        if lazy:
+            lz_call = [12.0 * n + u + 2 * lazy["state_bytes"] for u in used]
+            line["lazy_scale"] = {
+                "what": "same step with adacomp_compress_lazy (bit-identical streams; the sent elements' "
+                        "residue is finished on the next step's load instead of by a fix-up pass)",
+                "value": grad_bytes / (lazy["total_ms"] / K * 1e-3) / 1e9, "unit": "GB/s",
+                "ms_per_step": lazy["total_ms"] / K,
+                "compress_gbs": 4.0 * n * k * world / (lazy["t_comp"] * 1e-3) / 1e9,
+                "hbm_frac_compress_call": sum(lz_call) / (lazy["t_comp"] * 1e-3) / 1e9 / peak,
+                "pack_kernels_ms": lazy["kernels"],
+                "tile_pass_frac": (tile_bytes + 2 * lazy["state_bytes"]) / (lazy["kernels"]["tile_pass"] * 1e-3) / 1e9 / peak,
+                "same_counts_as_eager": lazy["same_counts_as_eager"],
+            }
         if e2e:
             line["e2e"] = {"value": grad_bytes / (e2e["ms"] * 1e-3) / 1e9, "unit": "GB/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],

@@ -812,7 +812,10 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
     const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
     const u64 warps = (u64)gridDim.x * (kGatherThreads / 32);
 
-    for (u64 tile = (u64)blockIdx.x * (kGatherThreads / 32) + warp; tile < geo.n_tiles; tile += warps) {
+    // Last tile first: the tile pass wrote the residue front to back, so its tail is what the
+    // L2 still holds when this kernel starts.
+    for (u64 item = (u64)blockIdx.x * (kGatherThreads / 32) + warp; item < geo.n_tiles; item += warps) {
+        const u64 tile = geo.n_tiles - 1 - item;
         u32 cnt;
         const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
         if (lane == 0) tile_off[tile] = off0;
@@ -929,13 +932,14 @@ struct DecodeArgs {
     u32 k;
 };
 
-constexpr int kWbufBytes = 16384;    // staged words of one round of learners
-constexpr int kRoundMax = 8;         // learners per round
+constexpr int kWbufBytes = 8192;     // staged words of one round of learners (one learner's worst case fits)
+constexpr int kRoundMax = 4;         // learners per round
+constexpr int kGenericSegBins = 1024;   // generic decode: bins scanned per pass
 
 struct DecodeSmem {
     float acc[kDecodeChunk];                    // the output tile
     union {
-        u32 pre[kMaxTileBins + 1];              // generic path: scanned bin counts of one stream
+        u32 pre[kGenericSegBins + 1];           // generic path: scanned bin counts of one stream
         struct {
             uint4 wbuf[kWbufBytes / 16];        // fast paths: the round's words, staged
             u32 bin_pre[kRoundMax][33];         // by-word path: scanned bin counts per learner
@@ -964,23 +968,62 @@ __device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc)
     }
 }
 
+// Number of malformed fields in four packed bytes (Word = u8) or two packed halfwords (u16)
+// of staged payload: the reserved ternary code 10, or an index >= L_T (field >= 4 * L_T).
+// Returns non-zero status bits instead of a count.
+template <typename Word>
+__device__ inline u32 check_fields(u32 x, u32 L_T)
+{
+    u32 bad = 0;
+    if (sizeof(Word) == 1) {
+        const u32 t = (x & 0x03030303u) ^ 0x02020202u;                    // zero byte <=> code 10
+        if ((t - 0x01010101u) & ~t & 0x80808080u) bad |= ADACOMP_DEV_RESERVED_CODE;
+        const u32 T = 4u * L_T;                                           // L_T <= 64
+        if (T < 256u) {
+            const u32 low = x & 0x7f7f7f7fu;
+            const u32 ge = T >= 128u ? ((low + (256u - T) * 0x01010101u) & x)
+                                     : ((low + (128u - T) * 0x01010101u) | x);
+            if (ge & 0x80808080u) bad |= ADACOMP_DEV_BAD_STREAM;
+        }
+    } else {
+        const u32 t = (x & 0x00030003u) ^ 0x00020002u;
+        if ((t - 0x00010001u) & ~t & 0x80008000u) bad |= ADACOMP_DEV_RESERVED_CODE;
+        const u32 T = 4u * L_T;                                           // L_T <= 16384
+        if (T < 65536u) {
+            const u32 low = x & 0x7fff7fffu;
+            const u32 ge = T >= 32768u ? ((low + (65536u - T) * 0x00010001u) & x)
+                                       : ((low + (32768u - T) * 0x00010001u) | x);
+            if (ge & 0x80008000u) bad |= ADACOMP_DEV_BAD_STREAM;
+        }
+    }
+    return bad;
+}
+
 // Fast decode for tiles of at most 96 bins and 4096 elements (L_T = 42..1000).
 //
-// Per tile: (1) each learner's word range comes from its directory; (2) the words of a
-// round of up to eight learners are staged in shared memory with 16-byte loads, all in
-// flight together; (3) the words are added into the output tile in learner order:
+// Per tile: (1) each learner's word range comes from its directory (fetched one tile ahead);
+// (2) the words of a round of up to four learners are staged in shared memory with 16-byte
+// loads, all in flight together, and checked as they pass (reserved code, index beyond the
+// bin); (3) the words are added into the output tile in learner order:
 //   BY_BIN  (32..96 bins): thread b owns bin b for every learner, so one thread adds all
 //           contributions to an element, in learner order, with no barrier in between;
 //   by word (2..31 bins): a learner's words are spread over the threads and a barrier
 //           separates consecutive learners;
 // (4) the tile is stored once with 128-bit streaming stores.
+// A stream that fails a check raises a status bit; its words are still applied with the index
+// clamped into the bin, so nothing is read or written out of bounds.
 template <typename Word, bool BY_BIN>
 __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
-    u32 *s_wsum = sm.tmp;                      // BY_BIN: [4 warps][8 learners]
+    const u32 L_T = geo.L_T;
+    u32 *s_wsum = sm.tmp;                      // BY_BIN: [4 warps][2 packed pairs of learners]
     const unsigned char *s_bytes = reinterpret_cast<const unsigned char *>(sm.f.wbuf);
+    constexpr u32 kCap = kWbufBytes / 16;
+    int top_probe = 1;                         // by word: highest power of two below the bin count
+    while (top_probe * 2 < TB) top_probe *= 2;
+
     for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
     if (tid < (int)a.k) {
         sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
@@ -993,13 +1036,14 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
         nx0 = dir[blockIdx.x];
         nx1 = dir[blockIdx.x + 1];
     }
+    u32 bad = 0;
     for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
         const u64 base = tile * (u64)geo.tile_elems;
         const u64 bin0 = tile * (u64)TB;
         if (tid < (int)a.k) {
             // a malformed directory must not send the copy below out of the stream
             const bool ok = nx1 >= nx0 && nx1 - nx0 <= geo.tile_elems && nx1 <= sm.n_sel[tid];
-            if (!ok) raise_status(ADACOMP_DEV_BAD_STREAM);
+            if (!ok) bad |= ADACOMP_DEV_BAD_STREAM;
             sm.off0[tid] = nx0;
             sm.cnt[tid] = ok ? (u32)(nx1 - nx0) : 0u;
             const u64 next = tile + gridDim.x;
@@ -1011,110 +1055,129 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
         }
         __syncthreads();
 
-        u32 l0 = 0;
-        while (l0 < a.k) {
-            // ---- the round: learners [l0, l1) whose words fit the staging buffer ----
-            u32 at[kRoundMax + 1], head[kRoundMax];      // 16-byte chunk index / misalignment of each learner
-            u32 l1 = l0;
-            at[0] = 0;
-            while (l1 < a.k && l1 - l0 < (u32)kRoundMax) {
-                const u32 q = l1 - l0;
-                const u64 src = (u64)(uintptr_t)(a.stream[l1] + geo.payload_at) + sm.off0[l1] * sizeof(Word);
-                head[q] = (u32)(src & 15u);
-                const u32 chunks = sm.cnt[l1] ? (head[q] + sm.cnt[l1] * (u32)sizeof(Word) + 15u) / 16u : 0u;
-                if (at[q] + chunks > (u32)(kWbufBytes / 16)) break;
-                at[q + 1] = at[q] + chunks;
-                l1++;
-            }
-            const int round = (int)(l1 - l0);            // >= 1: one learner's tile always fits
-            // ---- stage the words: every 16-byte load of the round is issued before any is used ----
-            for (u32 c = tid; c < at[round]; c += kDecodeThreads) {
-                int q = 0;
+        for (u32 g0 = 0; g0 < a.k; g0 += kRoundMax) {
+            // ---- a group of up to four learners: one round if its words fit the staging
+            //      buffer, else one round per learner (a single learner's tile always fits) ----
+            const int R = (int)min((u32)kRoundMax, a.k - g0);
+            u64 src[kRoundMax];
+            u32 chunks[kRoundMax], headb[kRoundMax], cnts[kRoundMax];
+            u32 total = 0;
 #pragma unroll
-                for (int t = 1; t < kRoundMax; t++)
-                    if (t < round && c >= at[t]) q = t;
-                const u64 src = ((u64)(uintptr_t)(a.stream[l0 + q] + geo.payload_at) +
-                                 sm.off0[l0 + q] * sizeof(Word)) & ~(u64)15u;
-                sm.f.wbuf[c] = __ldg(reinterpret_cast<const uint4 *>(src) + (c - at[q]));
-            }
-            if (BY_BIN) {
-                const u64 bin = bin0 + tid;
-                const bool live = tid < TB && bin < geo.n_bins;
-                u32 c[kRoundMax], pre[kRoundMax];
-#pragma unroll
-                for (int q = 0; q < kRoundMax; q++) {
-                    c[q] = 0;
-                    if (q < round && live)
-                        c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin], geo.L_T);
+            for (int q = 0; q < kRoundMax; q++) {
+                src[q] = 0; chunks[q] = 0; headb[q] = 0; cnts[q] = 0;
+                if (q < R) {
+                    const u64 p = (u64)(uintptr_t)(a.stream[g0 + q] + geo.payload_at) + sm.off0[g0 + q] * sizeof(Word);
+                    cnts[q] = sm.cnt[g0 + q];
+                    headb[q] = (u32)(p & 15u);
+                    src[q] = p & ~(u64)15u;
+                    chunks[q] = cnts[q] ? (headb[q] + cnts[q] * (u32)sizeof(Word) + 15u) / 16u : 0u;
+                    total += chunks[q];
                 }
+            }
+            const bool fits = total <= kCap;
+            const int nsub = fits ? 1 : R;
+            for (int sub = 0; sub < nsub; sub++) {
+                // learners of this round: q in [q_lo, q_hi); chunk offsets at[q] within the buffer
+                const int q_lo = fits ? 0 : sub, q_hi = fits ? R : sub + 1;
+                u32 at[kRoundMax + 1];
+                at[0] = 0;
 #pragma unroll
-                for (int q = 0; q < kRoundMax; q++) {
-                    const u32 inc = warp_inclusive_scan(c[q], lane);
-                    pre[q] = inc - c[q];
-                    if (lane == 31) s_wsum[warp * kRoundMax + q] = inc;
+                for (int q = 0; q < kRoundMax; q++)
+                    at[q + 1] = at[q] + ((q >= q_lo && q < q_hi) ? chunks[q] : 0u);
+
+                // ---- stage and check the words ----
+                for (u32 c = tid; c < at[kRoundMax]; c += kDecodeThreads) {
+                    u64 from = src[0];
+                    u32 first = 0;
+#pragma unroll
+                    for (int q = 1; q < kRoundMax; q++)
+                        if (c >= at[q]) { from = src[q]; first = at[q]; }
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(from) + (c - first));
+                    bad |= check_fields<Word>(v.x, L_T) | check_fields<Word>(v.y, L_T) |
+                           check_fields<Word>(v.z, L_T) | check_fields<Word>(v.w, L_T);
+                    sm.f.wbuf[c] = v;
                 }
-                __syncthreads();
-                float *mine = sm.acc + tid * geo.L_T;
+
+                if (BY_BIN) {
+                    // ---- bin counts -> word offsets: two learners per scan (16 bits each) ----
+                    const u64 bin = bin0 + tid;
+                    const bool live = tid < TB && bin < geo.n_bins;
+                    u32 c[kRoundMax];
 #pragma unroll
-                for (int q = 0; q < kRoundMax; q++) {
-                    if (q >= round || c[q] == 0) continue;
-                    for (int wv = 0; wv < warp; wv++) pre[q] += s_wsum[wv * kRoundMax + q];
-                    if (pre[q] + c[q] > sm.cnt[l0 + q]) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                    const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + head[q]) + pre[q];
-                    const float scale = sm.scale[l0 + q];
-                    for (u32 i = 0; i < c[q]; i++) {
-                        const u32 word = p[i];
-                        const u32 code = word & 3u, idx = word >> 2;
-                        if (code == 0u) continue;
-                        if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                        if (idx >= geo.L_T || base + (u64)tid * geo.L_T + idx >= geo.n) {
-                            raise_status(ADACOMP_DEV_BAD_STREAM);
-                            continue;
-                        }
-                        mine[idx] = code == 3u ? __fsub_rn(mine[idx], scale) : __fadd_rn(mine[idx], scale);
+                    for (int q = 0; q < kRoundMax; q++) {
+                        c[q] = 0;
+                        if (q >= q_lo && q < q_hi && live)
+                            c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[g0 + q] + geo.bin_cnt_at)[bin], L_T);
                     }
-                }
-                __syncthreads();
-            } else {
-                // warp wv scans the bin counts of learners wv, wv + 4 of the round
-                for (int q = warp; q < round; q += kDecodeThreads / 32) {
-                    u32 c = 0;
-                    if (lane < TB && bin0 + lane < geo.n_bins)
-                        c = reinterpret_cast<const Word *>(a.stream[l0 + q] + geo.bin_cnt_at)[bin0 + lane];
-                    const u32 inc = warp_inclusive_scan(c, lane);
-                    sm.f.bin_pre[q][lane] = inc - c;
-                    if (lane == 31) sm.f.bin_pre[q][32] = inc;
-                }
-                __syncthreads();
-                for (int q = 0; q < round; q++) {
-                    const u32 cnt = sm.cnt[l0 + q];           // the same for every thread
-                    if (cnt == 0) continue;
-                    if (sm.f.bin_pre[q][32] != cnt) { if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                    const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + head[q]);
-                    const float scale = sm.scale[l0 + q];
-                    for (u32 j = tid; j < cnt; j += kDecodeThreads) {
-                        const u32 word = p[j];
-                        const u32 code = word & 3u, idx = word >> 2;
-                        if (code == 0u) continue;
-                        if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                        int b = 0;
+                    u32 pair[2] = {c[0] | (c[1] << 16), c[2] | (c[3] << 16)};
+                    u32 excl[2];
 #pragma unroll
-                        for (int step = 16; step > 0; step >>= 1)       // at most 31 bins: five probes
-                            if (b + step < TB && sm.f.bin_pre[q][b + step] <= j) b += step;
-                        const u32 e = (u32)b * geo.L_T + idx;
-                        if (idx >= geo.L_T || base + e >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                        sm.acc[e] = code == 3u ? __fsub_rn(sm.acc[e], scale) : __fadd_rn(sm.acc[e], scale);
+                    for (int h = 0; h < 2; h++) {
+                        const u32 inc = warp_inclusive_scan(pair[h], lane);
+                        excl[h] = inc - pair[h];
+                        if (lane == 31) s_wsum[warp * 2 + h] = inc;
                     }
                     __syncthreads();
+                    if (tid < TB) {
+                        for (int wv = 0; wv < warp; wv++) {
+                            excl[0] += s_wsum[wv * 2];
+                            excl[1] += s_wsum[wv * 2 + 1];
+                        }
+                        const u32 pre[kRoundMax] = {excl[0] & 0xffffu, excl[0] >> 16, excl[1] & 0xffffu, excl[1] >> 16};
+                        float *mine = sm.acc + tid * L_T;
+#pragma unroll
+                        for (int q = 0; q < kRoundMax; q++) {
+                            if (c[q] == 0) continue;
+                            if (pre[q] + c[q] > cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
+                            const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]) + pre[q];
+                            const u32 sbits = __float_as_uint(sm.scale[g0 + q]);
+                            for (u32 i = 0; i < c[q]; i++) {
+                                const u32 word = p[i];
+                                const u32 e = min(word >> 2, L_T - 1u);
+                                const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
+                                mine[e] = __fadd_rn(mine[e], add);
+                            }
+                        }
+                    }
+                    __syncthreads();
+                } else {
+                    // warp wv scans the bin counts of learner wv of the round
+                    if (warp >= q_lo && warp < q_hi) {
+                        u32 c = 0;
+                        if (lane < TB && bin0 + lane < geo.n_bins)
+                            c = reinterpret_cast<const Word *>(a.stream[g0 + warp] + geo.bin_cnt_at)[bin0 + lane];
+                        const u32 inc = warp_inclusive_scan(c, lane);
+                        sm.f.bin_pre[warp][lane] = inc - c;
+                        if (lane == 31) sm.f.bin_pre[warp][32] = inc;
+                    }
+                    __syncthreads();
+#pragma unroll
+                    for (int q = 0; q < kRoundMax; q++) {
+                        if (q < q_lo || q >= q_hi || cnts[q] == 0) continue;      // the same for every thread
+                        if (sm.f.bin_pre[q][32] != cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
+                        const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]);
+                        const u32 sbits = __float_as_uint(sm.scale[g0 + q]);
+                        const u32 *pre = sm.f.bin_pre[q];
+                        for (u32 j = tid; j < cnts[q]; j += kDecodeThreads) {
+                            const u32 word = p[j];
+                            int b = 0;
+                            for (int step = top_probe; step > 0; step >>= 1)
+                                if (b + step < TB && pre[b + step] <= j) b += step;
+                            const u32 e = (u32)b * L_T + min(word >> 2, L_T - 1u);
+                            const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
+                            sm.acc[e] = __fadd_rn(sm.acc[e], add);
+                        }
+                        __syncthreads();
+                    }
+                    __syncthreads();     // bin_pre and wbuf are rewritten by the next round
                 }
-                __syncthreads();     // bin_pre and wbuf are rewritten by the next round
             }
-            l0 = l1;
         }
         const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
         store_tile(a.dst, base, len, sm.acc);
         __syncthreads();
     }
+    if (bad) raise_status(bad);
 }
 
 // Any tile shape (also tiles larger than one output chunk).
@@ -1148,28 +1211,40 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
             const Word *bin_cnt = reinterpret_cast<const Word *>(s + geo.bin_cnt_at);
             const Word *payload = reinterpret_cast<const Word *>(s + geo.payload_at);
             const u64 bin0 = tile * (u64)TB;
-            if (TB > 1) {
-                for (int b = tid; b < TB; b += kDecodeThreads)
-                    s_pre[b] = bin0 + b < geo.n_bins ? (u32)bin_cnt[bin0 + b] : 0u;
+            // the tile's bins are scanned kGenericSegBins at a time; `done` words precede the pass
+            u32 done = 0;
+            for (int seg = 0; seg < TB; seg += kGenericSegBins) {
+                const int bins = min(kGenericSegBins, TB - seg);
+                u32 words = cnt;                               // one bin per tile: all words are its
+                if (TB > 1) {
+                    for (int b = tid; b < bins; b += kDecodeThreads)
+                        s_pre[b] = bin0 + seg + b < geo.n_bins ? (u32)bin_cnt[bin0 + seg + b] : 0u;
+                    __syncthreads();
+                    block_exclusive_scan(s_pre, bins, sm.tmp);
+                    words = s_pre[bins];
+                }
+                if (done + words > cnt) {                       // counts and directory disagree
+                    if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM);
+                    __syncthreads();
+                    break;
+                }
+                for (u32 j = tid; j < words; j += kDecodeThreads) {
+                    const u32 word = payload[off0 + done + j];
+                    const u32 code = word & 3u;
+                    if (code == 0u) continue;
+                    if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
+                    const int b = seg + (TB > 1 ? bin_of_word(s_pre, bins, j) : 0);
+                    const u32 idx = word >> 2;
+                    const u32 at = (u32)b * geo.L_T + idx;          // within the tile
+                    if (idx >= geo.L_T || base + at >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
+                    if (at < c_lo || at >= c_hi) continue;
+                    // one word per element per learner: no two threads meet on one address here
+                    const float v = s_acc[at - c_lo];
+                    s_acc[at - c_lo] = code == 3u ? __fsub_rn(v, scale) : __fadd_rn(v, scale);
+                }
+                done += words;
                 __syncthreads();
-                block_exclusive_scan(s_pre, TB, sm.tmp);
-                if (s_pre[TB] != cnt) { if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM); __syncthreads(); continue; }
             }
-            for (u32 j = tid; j < cnt; j += kDecodeThreads) {
-                const u32 word = payload[off0 + j];
-                const u32 code = word & 3u;
-                if (code == 0u) continue;
-                if (code == 2u) { raise_status(ADACOMP_DEV_RESERVED_CODE); continue; }
-                const int b = TB > 1 ? bin_of_word(s_pre, TB, j) : 0;
-                const u32 idx = word >> 2;
-                const u32 at = (u32)b * geo.L_T + idx;          // within the tile
-                if (idx >= geo.L_T || base + at >= geo.n) { raise_status(ADACOMP_DEV_BAD_STREAM); continue; }
-                if (at < c_lo || at >= c_hi) continue;
-                // one word per element per learner: no two threads meet on one address here
-                const float v = s_acc[at - c_lo];
-                s_acc[at - c_lo] = code == 3u ? __fsub_rn(v, scale) : __fadd_rn(v, scale);
-            }
-            __syncthreads();
         }
         const u64 out0 = base + c_lo;
         const u32 len = out0 < geo.n ? (u32)min((u64)(c_hi - c_lo), geo.n - out0) : 0u;
