@@ -151,13 +151,25 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def merge(parts):
+        """One record from several sampled regions (median of all samples, union of reasons)."""
+        parts = [p for p in parts if p and p.get("samples")]
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not parts:
+            return out
+        sm = [v for p in parts for v in p["_sm"]]
+        out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(p["sm_max_mhz"] for p in parts),
+                   reasons=sorted({r for p in parts for r in p["reasons"]}), samples=len(sm))
+        return out
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "_sm": []}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -184,7 +196,7 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm), _sm=sm)
         out["reasons"] = sorted(reasons)
         return out
 
@@ -198,10 +210,9 @@ def run_ours(a):
     import torch.distributed as dist
 
     from paper_1712_02679_b200 import binding as B
+    from paper_1712_02679_b200 import ranks
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = ranks.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
@@ -228,7 +239,7 @@ def run_ours(a):
     dst = torch.empty(n, dtype=torch.float32, device=dev)
     for step in range(PREWARM_STEPS + 1):
         for l in range(k):
-            gen.manual_seed(1712_02679 + 1000003 * rank + 1009 * l + step)
+            gen.manual_seed(ranks.learner_seed(rank, l, step))
             dW[l].normal_(0.0, SIGMA, generator=gen)
             if step < PREWARM_STEPS:
                 B.adacomp_compress(dW[l], residue[l], n, L_T, packed[l], count[l], stream)
@@ -289,11 +300,12 @@ def run_ours(a):
         return [torch.cuda.Event(enable_timing=True) for _ in range(3)]
 
     # ---- timed region: device-resident inputs ----
-    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
-                           else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    gpu_index = (torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                 else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    sampler = ClockSampler(gpu_index)
     t_comp, t_dec, t_total_ms = timed_steps(False, True)
+    clock_parts = [sampler.stop()] if rank == 0 else []
     t_tile, t_fin, t_fix = profile_pack(False)
-    clocks = sampler.stop() if rank == 0 else None
 
     status = B.adacomp_device_status(stream)
     counts = [tuple(int(v) for v in c.cpu()) for c in count]
@@ -349,7 +361,7 @@ def run_ours(a):
         keep = [d.clone() for d in dW] if 4 * n * k < (8 << 30) else None
         for step in range(PREWARM_STEPS + 1):
             for l in range(k):
-                gen.manual_seed(1712_02679 + 1000003 * rank + 1009 * l + step)
+                gen.manual_seed(ranks.learner_seed(rank, l, step))
                 dW[l].normal_(0.0, SIGMA, generator=gen)
                 if step < PREWARM_STEPS:
                     pack(l, True)
@@ -360,7 +372,10 @@ def run_ours(a):
             s_.copy_(r)                         # now holds step 5's G plus the pending marks in the state
         lazy_snap.extend(st_.clone() for st_ in lazy_state)
         torch.cuda.synchronize()
-        lz_comp, lz_dec, lz_total = timed_steps(True, False)
+        sampler = ClockSampler(gpu_index)
+        lz_comp, lz_dec, lz_total = timed_steps(True, True)
+        if rank == 0:
+            clock_parts.append(sampler.stop())
         lz_tile, lz_fin, lz_gather = profile_pack(True)
         lazy_counts = [tuple(int(v) for v in c.cpu()) for c in count]
         lazy = {"same_counts_as_eager": lazy_counts == eager_counts, "t_comp": statistics.mean(lz_comp),
@@ -372,23 +387,20 @@ def run_ours(a):
 
     # ---- max over ranks ----
     m_comp, m_dec = statistics.mean(t_comp), statistics.mean(t_dec)
-    if world > 1:
-        t = torch.tensor([t_total_ms, m_comp, m_dec, e2e["ms"] if e2e else 0.0,
-                          lazy["total_ms"] if lazy else 0.0, lazy["t_comp"] if lazy else 0.0,
-                          lazy["t_dec"] if lazy else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        v = [float(x) for x in t.cpu()]
-        t_total_ms, m_comp, m_dec = v[0], v[1], v[2]
-        if e2e:
-            e2e["ms"] = v[3]
-        if lazy:
-            lazy["total_ms"], lazy["t_comp"], lazy["t_dec"] = v[4], v[5], v[6]
+    v = ranks.max_over_ranks([t_total_ms, m_comp, m_dec, e2e["ms"] if e2e else 0.0,
+                              lazy["total_ms"] if lazy else 0.0, lazy["t_comp"] if lazy else 0.0,
+                              lazy["t_dec"] if lazy else 0.0], device=dev)
+    t_total_ms, m_comp, m_dec = v[0], v[1], v[2]
+    if e2e:
+        e2e["ms"] = v[3]
+    if lazy:
+        lazy["total_ms"], lazy["t_comp"], lazy["t_dec"] = v[4], v[5], v[6]
 
     if rank == 0:
         peak, peak_src = measured_peak()
         ms_per_step = t_total_ms / K
         grad_bytes = 4.0 * n * k * world
-        value = grad_bytes / (ms_per_step * 1e-3) / 1e9
+        value = ranks.whole_job_throughput(4.0 * n * k, world, ms_per_step)
         tile_bytes = 12.0 * n + n_bins * w + n_sel[0] * w + 8.0 * n_tiles
         achieved = tile_bytes / (t_tile * 1e-3) / 1e9
         call_bytes = [12.0 * n + u for u in used]
@@ -417,7 +429,7 @@ def run_ours(a):
                          "unit": "GB/s", "frac": achieved / peak, "traffic": None,
                          "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": tile_bytes},
-            "clocks": clocks,
+            "clocks": ClockSampler.merge(clock_parts),
             "gpu_launches": K * (3 * k + 1),
         }
         if lazy:
