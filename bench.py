@@ -27,6 +27,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "compress+pack GB/s of fp32 gradient"
+# dram__bytes_read.sum + dram__bytes_write.sum per element of tile_pass_fast, from the ncu capture
+# at n = 2^26 summarised in profiles/tile_pass_fast_n2e26_LT50.md; traffic grows in proportion to n.
+TILE_PASS_DRAM_BYTES_PER_ELEM = {50: 11.50}
 SIGMA = 1e-3
 PREWARM_STEPS = 5
 FALLBACK_HBM_GBS = 6650.0
@@ -155,6 +158,16 @@ class ClockSampler:
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
+            return
+        # nvidia-smi needs a moment to start: wait (bounded) for its first sample
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < 3.0:
+            try:
+                if os.path.getsize(self.path) > 0:
+                    break
+            except OSError:
+                pass
+            time.sleep(0.02)
 
     @staticmethod
     def merge(parts):
@@ -264,11 +277,11 @@ def run_ours(a):
     def timed_steps(lazy, with_clocks):
         """W warm-up + K timed steps; returns per-step (pack ms, decode ms) and the total ms."""
         evs = []
+        if with_clocks and rank == 0:
+            sampler.start()              # sampling spans warm-up and timed steps of this arm
         for it in range(W + K):
             if it == W:
                 barrier()
-                if with_clocks and rank == 0:
-                    sampler.start()
             restore(lazy)
             e = step_events()
             e[0].record(stream)
@@ -426,7 +439,10 @@ def run_ours(a):
             "pack_kernels_ms": {"tile_pass": t_tile, "finalize": t_fin, "gather_fixup": t_fix},
             "selected_fraction": n_sel[0] / n, "bytes_used": used[0], "device_status": status,
             "roofline": {"bound": "hbm", "kernel": "tile_pass", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": (TILE_PASS_DRAM_BYTES_PER_ELEM[L_T] * n
+                                     if L_T in TILE_PASS_DRAM_BYTES_PER_ELEM else None),
+                         "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/tile_pass_fast_n2e26_LT50.md)",
                          "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": tile_bytes},
             "clocks": ClockSampler.merge(clock_parts),
