@@ -45,13 +45,29 @@ constexpr u32 kMaskBytes = kTileSegs * 4;      // lazy mode: one 25-bit "sent" m
 constexpr u32 kStageBytes = 2 * kTileBytes + kMaskBytes;   // dW + residue + previous step's masks
 constexpr int kGenericThreads = 256;
 constexpr int kDecodeChunk = 4096;   // output elements per decode work item
-constexpr int kDecodeThreads = 128;
+constexpr int kDecodeThreads = 128;  // decoding threads of a decode CTA (warps 0-3)
+constexpr int kDecodeLaunch = 160;   // launched threads: warp 4 is the pipelined path's producer
 constexpr int kGatherThreads = 128;
 constexpr int kMaxTileBins = 4000;
 constexpr int kSmallBins = 96;       // tiles with at most this many bins take the fast decode / gather
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: bound of every device-side wait
 
 __device__ u32 g_status;             // sticky ADACOMP_DEV_* bits of this device
+
+#ifdef ADACOMP_PHASE_CLOCKS
+// Development aid (not part of the ABI): cycles spent by one thread of one CTA in each phase.
+__device__ unsigned long long g_phase_clocks[16];
+#define PHASE_CLOCK(i, t0)                                                              \
+    do {                                                                               \
+        if (blockIdx.x == 3 && threadIdx.x == 32) {                                    \
+            const long long now_ = clock64();                                          \
+            g_phase_clocks[i] += (unsigned long long)(now_ - (t0));                    \
+            (t0) = now_;                                                               \
+        }                                                                              \
+    } while (0)
+#else
+#define PHASE_CLOCK(i, t0) do { } while (0)
+#endif
 
 __host__ __device__ inline u64 align_up(u64 x, u64 a) { return (x + a - 1) / a * a; }
 
@@ -107,9 +123,15 @@ __device__ inline u32 warp_inclusive_scan(u32 v, int lane)
 
 // Exclusive scan, in place, of a[0..count) in shared memory; a[count] receives the total.
 // Called by every thread of the CTA; contains barriers.
-__device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* >= 33 */)
+// With `decoders` set it is called by the 128 decoding threads of a decode CTA only and meets at
+// their named barrier.
+__device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* >= 33 */, bool decoders = false)
 {
-    const int tid = threadIdx.x, nthr = blockDim.x;
+    auto sync = [&]() {
+        if (decoders) asm volatile("bar.sync 1, 128;" ::: "memory");
+        else __syncthreads();
+    };
+    const int tid = threadIdx.x, nthr = decoders ? 128 : (int)blockDim.x;
     const int per = (count + nthr - 1) / nthr;
     const int lo = min(tid * per, count), hi = min(lo + per, count);
     u32 sum = 0;
@@ -117,14 +139,14 @@ __device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* 
     const int lane = tid & 31, warp = tid >> 5, nwarp = (nthr + 31) >> 5;
     const u32 inc = warp_inclusive_scan(sum, lane);
     if (lane == 31) warp_tmp[warp] = inc;
-    __syncthreads();
+    sync();
     if (warp == 0) {
         const u32 v = lane < nwarp ? warp_tmp[lane] : 0u;
         const u32 s = warp_inclusive_scan(v, lane);
         warp_tmp[lane] = s - v;
         if (lane == 31) warp_tmp[32] = s;
     }
-    __syncthreads();
+    sync();
     u32 run = warp_tmp[warp] + inc - sum;
     for (int i = lo; i < hi; i++) {
         const u32 v = a[i];
@@ -132,8 +154,11 @@ __device__ inline void block_exclusive_scan(u32 *a, int count, u32 *warp_tmp /* 
         run += v;
     }
     if (tid == 0) a[count] = warp_tmp[32];
-    __syncthreads();
+    sync();
 }
+
+// Barrier of the 128 decoding threads of a decode CTA (its producer warp never joins).
+__device__ inline void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Largest b in [0, bins) with prefix[b] <= j  (prefix is an exclusive scan, prefix[bins] > j).
 __device__ inline int bin_of_word(const u32 *prefix, int bins, u32 j)
@@ -936,18 +961,42 @@ constexpr int kWbufBytes = 8192;     // staged words of one round of learners (o
 constexpr int kRoundMax = 4;         // learners per round
 constexpr int kGenericSegBins = 1024;   // generic decode: bins scanned per pass
 
+constexpr u32 kPipeStageBytes = 8192 + 512;     // staged words + bin counts of one tile
+constexpr int kConsumers = 128;                 // threads of warps 0-3
+
+struct PipePlan {                               // where a tile's data sits in its stage
+    unsigned short woff[ADACOMP_MAX_STREAMS];   // stage byte offset of learner l's first word
+    unsigned short coff[ADACOMP_MAX_STREAMS];   // stage byte offset of its bin counts
+    unsigned short cnt[ADACOMP_MAX_STREAMS];    // its words in this tile (at most 4096)
+    u32 kf;                                     // learners [0, kf) were fetched into the stage
+    u32 bad;                                    // directory entries that failed their checks
+};
+
+struct PipeSmem {
+    uint4 stage[2][kPipeStageBytes / 16];
+    PipePlan plan[2];
+    unsigned short pre[kRoundMax][kSmallBins + 1];      // exclusive word offsets of the bins, per learner of a group
+    unsigned short pre0[2][kRoundMax][kSmallBins + 1];  // the same for the first group of each stage, made by the producer
+    u64 full[2], empty[2], ready[2];            // mbarriers of the two stages
+    u32 abort;
+};
+
 struct DecodeSmem {
     float acc[kDecodeChunk];                    // the output tile
     union {
-        u32 pre[kGenericSegBins + 1];           // generic path: scanned bin counts of one stream
         struct {
-            uint4 wbuf[kWbufBytes / 16];        // fast paths: the round's words, staged
-            u32 bin_pre[kRoundMax][33];         // by-word path: scanned bin counts per learner
+            u32 pre[kGenericSegBins + 1];       // generic path: scanned bin counts of one stream
+            u32 tmp[40];
+        } g;
+        struct {
+            u32 tmp[40];
+            uint4 wbuf[kWbufBytes / 16];        // staged path: the round's words
+            u32 bin_pre[kRoundMax][33];         // staged by-word path: scanned bin counts per learner
+            u64 off0[ADACOMP_MAX_STREAMS];      // first word of this tile in stream l
+            u32 cnt[ADACOMP_MAX_STREAMS];       // words of this tile in stream l
         } f;
+        PipeSmem pipe;                          // pipelined path
     };
-    u32 tmp[40];
-    u64 off0[ADACOMP_MAX_STREAMS];              // first word of this tile in stream l
-    u32 cnt[ADACOMP_MAX_STREAMS];               // words of this tile in stream l
     u64 n_sel[ADACOMP_MAX_STREAMS];             // words in stream l
     float scale[ADACOMP_MAX_STREAMS];
 };
@@ -1018,7 +1067,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
     const u32 L_T = geo.L_T;
-    u32 *s_wsum = sm.tmp;                      // BY_BIN: [4 warps][2 packed pairs of learners]
+    u32 *s_wsum = sm.f.tmp;                    // BY_BIN: [4 warps][2 packed pairs of learners]
     const unsigned char *s_bytes = reinterpret_cast<const unsigned char *>(sm.f.wbuf);
     constexpr u32 kCap = kWbufBytes / 16;
     int top_probe = 1;                         // by word: highest power of two below the bin count
@@ -1044,8 +1093,8 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
             // a malformed directory must not send the copy below out of the stream
             const bool ok = nx1 >= nx0 && nx1 - nx0 <= geo.tile_elems && nx1 <= sm.n_sel[tid];
             if (!ok) bad |= ADACOMP_DEV_BAD_STREAM;
-            sm.off0[tid] = nx0;
-            sm.cnt[tid] = ok ? (u32)(nx1 - nx0) : 0u;
+            sm.f.off0[tid] = nx0;
+            sm.f.cnt[tid] = ok ? (u32)(nx1 - nx0) : 0u;
             const u64 next = tile + gridDim.x;
             if (next < geo.n_tiles) {
                 const u64 *dir = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at);
@@ -1053,7 +1102,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
                 nx1 = dir[next + 1];
             }
         }
-        __syncthreads();
+        consumer_barrier();
 
         for (u32 g0 = 0; g0 < a.k; g0 += kRoundMax) {
             // ---- a group of up to four learners: one round if its words fit the staging
@@ -1066,8 +1115,8 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
             for (int q = 0; q < kRoundMax; q++) {
                 src[q] = 0; chunks[q] = 0; headb[q] = 0; cnts[q] = 0;
                 if (q < R) {
-                    const u64 p = (u64)(uintptr_t)(a.stream[g0 + q] + geo.payload_at) + sm.off0[g0 + q] * sizeof(Word);
-                    cnts[q] = sm.cnt[g0 + q];
+                    const u64 p = (u64)(uintptr_t)(a.stream[g0 + q] + geo.payload_at) + sm.f.off0[g0 + q] * sizeof(Word);
+                    cnts[q] = sm.f.cnt[g0 + q];
                     headb[q] = (u32)(p & 15u);
                     src[q] = p & ~(u64)15u;
                     chunks[q] = cnts[q] ? (headb[q] + cnts[q] * (u32)sizeof(Word) + 15u) / 16u : 0u;
@@ -1117,7 +1166,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
                         excl[h] = inc - pair[h];
                         if (lane == 31) s_wsum[warp * 2 + h] = inc;
                     }
-                    __syncthreads();
+                    consumer_barrier();
                     if (tid < TB) {
                         for (int wv = 0; wv < warp; wv++) {
                             excl[0] += s_wsum[wv * 2];
@@ -1139,7 +1188,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
                             }
                         }
                     }
-                    __syncthreads();
+                    consumer_barrier();
                 } else {
                     // warp wv scans the bin counts of learner wv of the round
                     if (warp >= q_lo && warp < q_hi) {
@@ -1150,7 +1199,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
                         sm.f.bin_pre[warp][lane] = inc - c;
                         if (lane == 31) sm.f.bin_pre[warp][32] = inc;
                     }
-                    __syncthreads();
+                    consumer_barrier();
 #pragma unroll
                     for (int q = 0; q < kRoundMax; q++) {
                         if (q < q_lo || q >= q_hi || cnts[q] == 0) continue;      // the same for every thread
@@ -1167,15 +1216,420 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
                             const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
                             sm.acc[e] = __fadd_rn(sm.acc[e], add);
                         }
-                        __syncthreads();
+                        consumer_barrier();
                     }
-                    __syncthreads();     // bin_pre and wbuf are rewritten by the next round
+                    consumer_barrier();     // bin_pre and wbuf are rewritten by the next round
                 }
             }
         }
         const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
         store_tile(a.dst, base, len, sm.acc);
-        __syncthreads();
+        consumer_barrier();
+    }
+    if (bad) raise_status(bad);
+}
+
+// ---------------------------------------------------------------------------------
+// decode, pipelined path: tiles of 2..96 bins whose bin-count run is a multiple of 16 bytes
+// (L_T = 50 and 500 among them).
+//
+// Warp 4 is a producer: for every tile of this CTA it reads the k directory entries (one lane
+// per learner, one tile ahead), lays the learners' bin counts and words out in one of two
+// shared-memory stages and starts the bulk copies (TMA, no multicast); it runs up to two tiles
+// ahead of the consumers and never touches the output.  Warps 0-3 are consumers: they wait for
+// the stage, turn the bin counts into word offsets, add the words into the output tile and
+// store it.  G threads share a bin (G = 1 for more than 64 bins, up to 32 for few bins); a
+// bin's G threads sit in one warp, so the learners' contributions to an element stay in learner
+// order with a __syncwarp() between learners.  The consumers meet at two named barriers per
+// tile; producer and consumers meet only through the stages' full / empty mbarriers, and every
+// wait on those is bounded.
+// ---------------------------------------------------------------------------------
+
+__device__ inline void mbar_arrive(u64 *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// Adds the words [0, c) at p (one learner's words of one bin) into the bin's 'mine' elements;
+// threads r, r + G, ... of the bin's G threads take every G-th word.  `seen` collects the ternary
+// codes met and `mx` the largest index, checked by the caller.
+// A thread that owns its bin alone (G == 1) handles words four at a time: a learner sends an
+// element at most once, so the four read-modify-writes are independent and their shared-memory
+// latencies overlap (slots past the end carry the no-op word 0).  With G > 1 a thread rarely has
+// more than one word, so it takes them singly.
+template <typename Word>
+__device__ inline void add_words(const Word *p, u32 c, int r, int G, u32 sbits, float *mine, u32 L_T,
+                                 u32 &seen, u32 &mx)
+{
+    if (G > 1) {
+        for (u32 j = r; j < c; j += (u32)G) {
+            const u32 word = p[j];
+            const u32 idx = word >> 2;
+            mx = max(mx, idx);
+            seen |= 1u << (word & 3u);
+            const u32 e = sizeof(Word) == 1 ? idx : min(idx, L_T - 1u);
+            if (word & 1u) mine[e] = __fadd_rn(mine[e], __uint_as_float(sbits ^ ((word & 2u) << 30)));
+        }
+        return;
+    }
+    constexpr int kBatch = 4;
+    for (u32 j0 = 0; j0 < c; j0 += kBatch) {
+        u32 word[kBatch], e[kBatch];
+        float v[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; i++) word[i] = j0 + i < c ? (u32)p[j0 + i] : 0u;
+#pragma unroll
+        for (int i = 0; i < kBatch; i++) {
+            const u32 idx = word[i] >> 2;
+            mx = max(mx, idx);
+            e[i] = sizeof(Word) == 1 ? idx : min(idx, L_T - 1u);      // 8-bit indices cannot leave the tile
+            v[i] = mine[e[i]];
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; i++) {
+            if (j0 + i < c) seen |= 1u << (word[i] & 3u);
+            if (word[i] & 1u) mine[e[i]] = __fadd_rn(v[i], __uint_as_float(sbits ^ ((word[i] & 2u) << 30)));
+        }
+    }
+}
+
+// Exclusive word offsets of bins 0..TB (TB <= 96) of up to four learners, written to pre[q][0..TB].
+// count(q, b) returns learner q's count of bin b.  Called by the warps that own bins (whole warps);
+// two 16-bit counts share a scan, and each warp adds up the bins of the warps before it itself.
+template <typename CountFn>
+__device__ inline void bin_offsets(CountFn count, int R, int TB, int tid, unsigned short (*pre)[kSmallBins + 1])
+{
+    const int lane = tid & 31, warp = tid >> 5;
+    u32 c[kRoundMax];
+#pragma unroll
+    for (int q = 0; q < kRoundMax; q++) c[q] = (q < R && tid < TB) ? count(q, tid) : 0u;
+    u32 pair[2] = {c[0] | (c[1] << 16), c[2] | (c[3] << 16)};
+    u32 basep[2] = {0u, 0u};
+    for (int wv = 0; wv < warp; wv++) {            // bins of the warps before this one
+        const int b = wv * 32 + lane;
+        u32 e[kRoundMax];
+#pragma unroll
+        for (int q = 0; q < kRoundMax; q++) e[q] = q < R ? count(q, b) : 0u;
+        basep[0] += e[0] | (e[1] << 16);
+        basep[1] += e[2] | (e[3] << 16);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+        if (warp > 0)
+            for (int d = 16; d > 0; d >>= 1) basep[h] += __shfl_xor_sync(0xffffffffu, basep[h], d);
+        const u32 inc = warp_inclusive_scan(pair[h], lane);
+        const u32 excl = basep[h] + inc - pair[h];
+        if (tid < TB) {
+            pre[2 * h][tid] = (unsigned short)(excl & 0xffffu);
+            pre[2 * h + 1][tid] = (unsigned short)(excl >> 16);
+            if (tid == TB - 1) {
+                pre[2 * h][TB] = (unsigned short)((excl + pair[h]) & 0xffffu);
+                pre[2 * h + 1][TB] = (unsigned short)((excl + pair[h]) >> 16);
+            }
+        }
+    }
+}
+
+template <typename Word>
+__device__ void decode_pipelined(const DecodeArgs &a, const Geometry &geo, float *s_acc, PipeSmem &ps,
+                                 const float *s_scale, const u64 *s_nsel)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int TB = (int)geo.tile_bins;
+    const u32 L_T = geo.L_T;
+    const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
+    const u64 first = blockIdx.x, stride = gridDim.x;
+    const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
+
+    if (tid == 0) {
+        mbar_init(&ps.full[0], 1);
+        mbar_init(&ps.full[1], 1);
+        mbar_init(&ps.empty[0], 1);
+        mbar_init(&ps.empty[1], 1);
+        mbar_init(&ps.ready[0], 1);
+        mbar_init(&ps.ready[1], 1);
+        ps.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
+    __syncthreads();
+
+    if (warp == 4) {
+        // =============================== producer warp ===============================
+        // lane l looks after learners l and l + 32
+        u64 d0[2] = {0, 0}, d1[2] = {0, 0};
+        auto load_dir = [&](u64 it) {
+            const u64 tile = first + it * stride;
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const u32 l = (u32)lane + 32u * h;
+                if (l < a.k && it < my_tiles) {
+                    const u64 *dir = reinterpret_cast<const u64 *>(a.stream[l] + geo.tile_off_at);
+                    d0[h] = dir[tile];
+                    d1[h] = dir[tile + 1];
+                }
+            }
+        };
+        load_dir(0);
+        u64 issued = 0;                 // copies were started for tiles [0, issued)
+        for (u64 it = 0; it < my_tiles; it++) {
+            const int s = (int)(it & 1);
+            const u64 tile = first + it * stride;
+            const u64 c0[2] = {d0[0], d0[1]}, c1[2] = {d1[0], d1[1]};
+            load_dir(it + 1);                       // next tile's entries travel while this one is laid out
+            if (it >= 2 && !mbar_wait(&ps.empty[s], (u32)((it >> 1) - 1) & 1u)) {
+                ps.abort = 1;
+                raise_status(ADACOMP_DEV_TIMEOUT);
+                break;                              // the consumers time out on the full barrier in turn
+            }
+            if (*reinterpret_cast<volatile u32 *>(&ps.abort)) break;
+            PipePlan &pl = ps.plan[s];
+            unsigned char *st = reinterpret_cast<unsigned char *>(ps.stage[s]);
+            const u64 bin0 = tile * (u64)TB;
+            const u64 bins_left = geo.n_bins - bin0;
+            const u32 cbytes = bins_left >= (u64)TB ? count_bytes
+                                                    : (u32)align_up(bins_left * sizeof(Word), 16);   // last tile
+            u32 used = 0, kf = 0, total = 0, bad = 0;
+            bool open = true;               // learners are staged as a prefix: once one does not fit, none after it is
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const u32 l = (u32)lane + 32u * h;
+                const bool active = l < a.k;
+                bool ok = true;
+                u32 cnt = 0, head = 0, wbytes = 0;
+                if (active) {
+                    ok = c1[h] >= c0[h] && c1[h] - c0[h] <= geo.tile_elems && c1[h] <= s_nsel[l];
+                    cnt = ok ? (u32)(c1[h] - c0[h]) : 0u;
+                    const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + c0[h] * sizeof(Word);
+                    head = (u32)(src & 15u);
+                    wbytes = cnt ? (u32)align_up(head + cnt * sizeof(Word), 16) : 0u;
+                    pl.cnt[l] = (unsigned short)cnt;
+                }
+                if (__any_sync(0xffffffffu, active && !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
+                const u32 need = active ? count_bytes + wbytes : 0u;
+                const u32 incl = used + warp_inclusive_scan(need, lane);
+                const u32 fits = __ballot_sync(0xffffffffu, active && open && incl <= kPipeStageBytes);
+                const int lead = __ffs(~fits) - 1;                  // first lane that is not staged
+                const int staged_lanes = lead < 0 ? 32 : lead;
+                const bool staged = lane < staged_lanes;
+                if (staged) {
+                    pl.coff[l] = (unsigned short)(incl - need);
+                    pl.woff[l] = (unsigned short)(incl - need + count_bytes + head);
+                }
+                u32 bytes = staged ? cbytes + wbytes : 0u;
+                for (int d = 16; d > 0; d >>= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, d);
+                total += bytes;
+                kf += (u32)staged_lanes;
+                if (staged_lanes > 0) used = __shfl_sync(0xffffffffu, incl, staged_lanes - 1);
+                if (staged_lanes < 32) open = false;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                pl.kf = kf;
+                pl.bad = bad;
+                mbar_arrive_expect_tx(&ps.full[s], total);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const u32 l = (u32)lane + 32u * h;
+                if (l < kf) {
+                    const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + c0[h] * sizeof(Word);
+                    const u32 head = (u32)(src & 15u);
+                    bulk_load(st + pl.coff[l], a.stream[l] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ps.full[s]);
+                    if (pl.cnt[l])
+                        bulk_load(st + pl.woff[l] - head, reinterpret_cast<const void *>(src & ~(u64)15u),
+                                  (u32)align_up(head + pl.cnt[l] * sizeof(Word), 16), &ps.full[s]);
+                }
+            }
+            issued = it + 1;
+
+            // ---- word offsets of the bins for the tile's first group of learners: done here, one
+            //      tile ahead of the decoding warps.  Lane i scans bins 3i .. 3i + 2. ----
+            if (!mbar_wait(&ps.full[s], (u32)(it >> 1) & 1u)) {
+                ps.abort = 1;
+                raise_status(ADACOMP_DEV_TIMEOUT);
+                break;
+            }
+            {
+                const int R = (int)min((u32)kRoundMax, kf);
+                const u32 live_bins = (u32)min((u64)TB, bins_left);
+                u32 c[3][kRoundMax], sum[2] = {0u, 0u};
+#pragma unroll
+                for (int t = 0; t < 3; t++) {
+                    const u32 b = (u32)lane * 3u + t;
+#pragma unroll
+                    for (int q = 0; q < kRoundMax; q++)
+                        c[t][q] = (q < R && b < live_bins)
+                                      ? min((u32)reinterpret_cast<const Word *>(st + pl.coff[q])[b], L_T) : 0u;
+                    sum[0] += c[t][0] | (c[t][1] << 16);
+                    sum[1] += c[t][2] | (c[t][3] << 16);
+                }
+#pragma unroll
+                for (int hh = 0; hh < 2; hh++) {
+                    const u32 inc = warp_inclusive_scan(sum[hh], lane);
+                    u32 run = inc - sum[hh];
+#pragma unroll
+                    for (int t = 0; t < 3; t++) {
+                        const int b = lane * 3 + t;
+                        if (b <= TB) {
+                            ps.pre0[s][2 * hh][b] = (unsigned short)(run & 0xffffu);
+                            ps.pre0[s][2 * hh + 1][b] = (unsigned short)(run >> 16);
+                        }
+                        run += c[t][2 * hh] | (c[t][2 * hh + 1] << 16);
+                    }
+                    if (lane == 31 && TB == 96) {
+                        ps.pre0[s][2 * hh][96] = (unsigned short)(inc & 0xffffu);
+                        ps.pre0[s][2 * hh + 1][96] = (unsigned short)(inc >> 16);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ps.ready[s]);
+            }
+        }
+        if (*reinterpret_cast<volatile u32 *>(&ps.abort)) {
+            // after a timeout the copies already started must land (or time out in turn) before
+            // this CTA's shared memory is given back
+            for (u64 j = issued >= 2 ? issued - 2 : 0; j < issued; j++)
+                mbar_wait(&ps.full[j & 1], (u32)(j >> 1) & 1u);
+        }
+        return;
+    }
+
+    // ================================== consumers ==================================
+    int G = 1;
+    while (G < 32 && 2 * G * TB <= kConsumers) G *= 2;
+    const int my_bin = tid / G, my_r = tid % G;
+    const bool scatterer = my_bin < TB;
+    const bool scanner = tid < ((TB + 31) & ~31);
+    const bool whole_tiles = geo.tile_elems == 4000u;
+    u32 bad = 0;
+    for (u64 it = 0; it < my_tiles; it++) {
+        const u64 tile = first + it * stride;
+        const u64 base = tile * (u64)geo.tile_elems;
+        const u64 bin0 = tile * (u64)TB;
+        const int s = (int)(it & 1);
+        const PipePlan &pl = ps.plan[s];
+        const unsigned char *st = reinterpret_cast<const unsigned char *>(ps.stage[s]);
+
+        long long t0 = clock64();
+        if (!mbar_wait(&ps.full[s], (u32)(it >> 1) & 1u)) {
+            ps.abort = 1;
+            bad |= ADACOMP_DEV_TIMEOUT;
+        }
+        if (!mbar_wait(&ps.ready[s], (u32)(it >> 1) & 1u)) {
+            ps.abort = 1;
+            bad |= ADACOMP_DEV_TIMEOUT;
+        }
+        PHASE_CLOCK(0, t0);
+        const u32 kf = pl.kf;
+        if (tid == 0) bad |= pl.bad;
+        const u32 live_bins = (u32)min((u64)TB, geo.n_bins - bin0);
+
+        // ---- the prefetched learners, four at a time ----
+        for (u32 g0 = 0; g0 < kf; g0 += kRoundMax) {
+            const int R = (int)min((u32)kRoundMax, kf - g0);
+            const unsigned short (*pre_of)[kSmallBins + 1] = g0 == 0 ? ps.pre0[s] : ps.pre;
+            if (g0 > 0 && scanner)      // (the first group's offsets were made by the producer warp)
+                bin_offsets([&](int q, int b) {
+                    return (u32)b < live_bins ? min((u32)reinterpret_cast<const Word *>(st + pl.coff[g0 + q])[b], L_T) : 0u;
+                }, R, TB, tid, ps.pre);
+            PHASE_CLOCK(1, t0);
+            consumer_barrier();     // offsets published; (first group) the previous tile is stored and zeroed
+            PHASE_CLOCK(2, t0);
+            if (scatterer) {
+                u32 seen = 0, mx = 0;
+                float *mine = s_acc + my_bin * L_T;
+                // everything the four learners need is read up front, so the loads overlap
+                u32 pre[kRoundMax], cq[kRoundMax], sb[kRoundMax];
+                const Word *wp[kRoundMax];
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    pre[q] = 0; cq[q] = 0; sb[q] = 0; wp[q] = nullptr;
+                    if (q < R) {
+                        const bool sane = pre_of[q][TB] <= pl.cnt[g0 + q];      // the same for every thread
+                        if (!sane) bad |= ADACOMP_DEV_BAD_STREAM;
+                        pre[q] = pre_of[q][my_bin];
+                        cq[q] = sane ? pre_of[q][my_bin + 1] - pre[q] : 0u;
+                        sb[q] = __float_as_uint(s_scale[g0 + q]);
+                        wp[q] = reinterpret_cast<const Word *>(st + pl.woff[g0 + q]) + pre[q];
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    if (q >= R) break;
+                    add_words(wp[q], cq[q], my_r, G, sb[q], mine, L_T, seen, mx);
+                    if (G > 1) __syncwarp();       // the bin's threads share a warp: learner order kept
+                }
+                if (seen & 4u) bad |= ADACOMP_DEV_RESERVED_CODE;
+                if (mx >= L_T) bad |= ADACOMP_DEV_BAD_STREAM;
+            }
+            PHASE_CLOCK(3, t0);
+            if (g0 + kRoundMax < kf) consumer_barrier();   // ps.pre is rewritten by the next group
+        }
+
+        // ---- learners that did not fit the stage: fetched and added one at a time ----
+        for (u32 l = kf; l < a.k; l++) {
+            consumer_barrier();                    // every reader of the stage is done
+            unsigned char *stw = reinterpret_cast<unsigned char *>(ps.stage[s]);
+            const u32 cnt = pl.cnt[l];
+            const u64 word0 = reinterpret_cast<const u64 *>(a.stream[l] + geo.tile_off_at)[tile];
+            const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + word0 * sizeof(Word);
+            const u32 head = (u32)(src & 15u);
+            const u32 chunks = cnt ? (head + cnt * (u32)sizeof(Word) + 15u) / 16u : 0u;
+            for (u32 c = tid; c < chunks; c += kConsumers)
+                reinterpret_cast<uint4 *>(stw + count_bytes)[c] = __ldg(reinterpret_cast<const uint4 *>(src & ~(u64)15u) + c);
+            if (tid < TB)
+                reinterpret_cast<Word *>(stw)[tid] =
+                    (u32)tid < live_bins ? reinterpret_cast<const Word *>(a.stream[l] + geo.bin_cnt_at)[bin0 + tid] : (Word)0;
+            consumer_barrier();
+            if (scanner)
+                bin_offsets([&](int q, int b) {
+                    return (q == 0 && b < TB) ? min((u32)reinterpret_cast<const Word *>(stw)[b], L_T) : 0u;
+                }, 1, TB, tid, ps.pre);
+            consumer_barrier();
+            if (scatterer) {
+                if (ps.pre[0][TB] > cnt) {
+                    bad |= ADACOMP_DEV_BAD_STREAM;
+                } else {
+                    u32 seen = 0, mx = 0;
+                    const u32 pre = ps.pre[0][my_bin];
+                    add_words(reinterpret_cast<const Word *>(stw + count_bytes + head) + pre, ps.pre[0][my_bin + 1] - pre,
+                              my_r, G, __float_as_uint(s_scale[l]), s_acc + my_bin * L_T, L_T, seen, mx);
+                    if (seen & 4u) bad |= ADACOMP_DEV_RESERVED_CODE;
+                    if (mx >= L_T) bad |= ADACOMP_DEV_BAD_STREAM;
+                }
+            }
+        }
+
+        consumer_barrier();                        // all words added; stage s and its plan are free
+        PHASE_CLOCK(4, t0);
+        const bool aborted = *reinterpret_cast<volatile u32 *>(&ps.abort) != 0;
+        if (tid == 0) mbar_arrive(&ps.empty[s]);
+        if (aborted) break;
+        // ---- store the tile (and leave it zeroed for the next one) ----
+        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
+        if (whole_tiles && len == 4000u) {
+            float4 *o4 = reinterpret_cast<float4 *>(a.dst + base);
+            float4 *s4 = reinterpret_cast<float4 *>(s_acc);
+            const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const int at = tid + i * kConsumers;
+                if (i < 7 || at < 1000) {
+                    __stcs(o4 + at, s4[at]);
+                    s4[at] = zero;
+                }
+            }
+        } else {
+            store_tile(a.dst, base, len, s_acc);
+        }
+        PHASE_CLOCK(5, t0);
+#ifdef ADACOMP_PHASE_CLOCKS
+        if (blockIdx.x == 3 && threadIdx.x == 32) g_phase_clocks[6] += 1;
+#endif
+        // (the next tile's first barrier orders this zeroing before its adds; every tile has one,
+        // because a single learner's words always fit the stage: kf >= 1)
     }
     if (bad) raise_status(bad);
 }
@@ -1187,11 +1641,11 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
     const int tid = threadIdx.x;
     const int TB = (int)geo.tile_bins;
     float *s_acc = sm.acc;
-    u32 *s_pre = sm.pre;
+    u32 *s_pre = sm.g.pre;
     const u32 chunks_per_tile = (geo.tile_elems + kDecodeChunk - 1) / kDecodeChunk;
     const u64 items = geo.n_tiles * chunks_per_tile;
     for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) s_acc[i] = 0.f;
-    __syncthreads();
+    consumer_barrier();
     for (u64 item = blockIdx.x; item < items; item += gridDim.x) {
         const u64 tile = item / chunks_per_tile;
         const u32 c_lo = (u32)(item % chunks_per_tile) * kDecodeChunk;     // within the tile
@@ -1219,13 +1673,13 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
                 if (TB > 1) {
                     for (int b = tid; b < bins; b += kDecodeThreads)
                         s_pre[b] = bin0 + seg + b < geo.n_bins ? (u32)bin_cnt[bin0 + seg + b] : 0u;
-                    __syncthreads();
-                    block_exclusive_scan(s_pre, bins, sm.tmp);
+                    consumer_barrier();
+                    block_exclusive_scan(s_pre, bins, sm.g.tmp, true);
                     words = s_pre[bins];
                 }
                 if (done + words > cnt) {                       // counts and directory disagree
                     if (tid == 0) raise_status(ADACOMP_DEV_BAD_STREAM);
-                    __syncthreads();
+                    consumer_barrier();
                     break;
                 }
                 for (u32 j = tid; j < words; j += kDecodeThreads) {
@@ -1243,17 +1697,17 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
                     s_acc[at - c_lo] = code == 3u ? __fsub_rn(v, scale) : __fadd_rn(v, scale);
                 }
                 done += words;
-                __syncthreads();
+                consumer_barrier();
             }
         }
         const u64 out0 = base + c_lo;
         const u32 len = out0 < geo.n ? (u32)min((u64)(c_hi - c_lo), geo.n - out0) : 0u;
         store_tile(a.dst, out0, len, s_acc);
-        __syncthreads();
+        consumer_barrier();
     }
 }
 
-__global__ void __launch_bounds__(kDecodeThreads)
+__global__ void __launch_bounds__(kDecodeLaunch, 6)
 decode_sum(DecodeArgs a)
 {
     __shared__ __align__(16) DecodeSmem sm;
@@ -1285,6 +1739,18 @@ decode_sum(DecodeArgs a)
     const Geometry geo = make_geometry(n, L_T);
     const bool by_bin = geo.tile_bins >= 32 && geo.tile_bins <= (u32)kSmallBins;
     const bool by_word = geo.tile_bins >= 2 && geo.tile_bins <= 31;
+    if (threadIdx.x < a.k) {
+        sm.scale[threadIdx.x] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[threadIdx.x])[12]);
+        sm.n_sel[threadIdx.x] = reinterpret_cast<const u64 *>(a.stream[threadIdx.x])[5];
+    }
+    if ((by_bin || by_word) && (geo.tile_bins * geo.w) % 16u == 0) {
+        // bin-count runs start on 16-byte boundaries: everything a tile needs can be bulk-copied ahead
+        if (geo.w == 1u) decode_pipelined<unsigned char>(a, geo, sm.acc, sm.pipe, sm.scale, sm.n_sel);
+        else decode_pipelined<unsigned short>(a, geo, sm.acc, sm.pipe, sm.scale, sm.n_sel);
+        return;
+    }
+    __syncthreads();                               // scales and word totals are in place
+    if (threadIdx.x >= kDecodeThreads) return;     // the other paths have no producer warp
     if (geo.w == 1u) {
         if (by_bin) decode_staged<unsigned char, true>(a, geo, sm);
         else decode_generic<unsigned char>(a, geo, sm);
@@ -1361,7 +1827,7 @@ int device_info(DeviceInfo *&out)
             return ADACOMP_ERR_CUDA;
         d.smem_optin = optin;
         int per_sm = 1;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeLaunch, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
@@ -1489,7 +1955,7 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
-    decode_sum<<<(unsigned)(info->sms * info->decode_per_sm), kDecodeThreads, 0,
+    decode_sum<<<(unsigned)(info->sms * info->decode_per_sm), kDecodeLaunch, 0,
                  static_cast<cudaStream_t>(stream)>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
@@ -1752,6 +2218,19 @@ int adacomp_device_status(uint32_t *host_out, void *stream)
     *host_out = v;
     return ADACOMP_OK;
 }
+
+#ifdef ADACOMP_PHASE_CLOCKS
+int adacomp_debug_phase_clocks(unsigned long long *host_out, int reset)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess) return ADACOMP_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(host_out, g_phase_clocks, sizeof(g_phase_clocks)) != cudaSuccess) return ADACOMP_ERR_CUDA;
+    if (reset) {
+        unsigned long long zero[16] = {0};
+        cudaMemcpyToSymbol(g_phase_clocks, zero, sizeof(zero));
+    }
+    return ADACOMP_OK;
+}
+#endif
 
 int adacomp_device_status_reset(void *stream)
 {

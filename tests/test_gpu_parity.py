@@ -163,6 +163,25 @@ def test_decode_sum_matches_oracle(L_T, n, k):
     assert B.adacomp_device_status() == 0
 
 
+def test_decode_sum_dense_streams_overflow_the_prefetch_stage():
+    """Every element sent (all ties): 4000 words per tile and learner, so only a few learners'
+    words fit the decoder's staging buffer and the rest take its one-at-a-time path."""
+    rng = np.random.default_rng(8)
+    for L_T, n, k in [(50, 4000 * 9 + 123, 12), (500, 4000 * 5 + 77, 7)]:
+        streams = []
+        for l in range(k):
+            sign = np.where(rng.random(n) < 0.5, -1.0, 1.0).astype(np.float32)
+            dW = sign * np.float32(2.0 ** -(l % 5))
+            want = cref.pack(dW, np.zeros(n, np.float32), L_T)
+            assert want.n_sel == n
+            raw, _, _ = GpuLayer(n, L_T).compress(dW)
+            assert_stream_equal(raw, want)
+            streams.append(raw)
+        got = gpu_decode(streams, n)
+        assert_f32_bits_equal(got, cref.unpack_sum(streams, n), f"dense decode L_T={L_T} k={k}")
+    assert B.adacomp_device_status() == 0
+
+
 def test_decode_sum_seeded_four_learners_crosscheck():
     import zlib
     spec = synth.config2_tensors()[7]
