@@ -565,6 +565,113 @@ tile_pass_fast(PassArgs a)
 // gmax[tile_bins], cnt[tile_bins + 1].
 // ---------------------------------------------------------------------------------
 
+// One tile of one layer.  Called by all 256 threads of the CTA; `s_acc` collects the CTA's share of
+// the layer's exact g_max sum.
+struct TileIo {                 // the buffers of one layer, as the generic tile code sees them
+    const float *grad;
+    float *residue;
+    unsigned char *packed, *scratch;
+    u32 literal;
+};
+
+template <typename Word>
+__device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, unsigned char *smem_raw, u32 *s_tmp,
+                             u64 *s_acc)
+{
+    const int T = (int)geo.tile_elems, TB = (int)geo.tile_bins, L = (int)geo.L_T;
+    float *s_d = reinterpret_cast<float *>(smem_raw);
+    float *s_g = s_d + T;
+    Word *s_words = reinterpret_cast<Word *>(s_g + T);
+    float *s_gmax = reinterpret_cast<float *>(smem_raw + align_up((u64)T * (8 + sizeof(Word)), 16));
+    u32 *s_cnt = reinterpret_cast<u32 *>(s_gmax + TB);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
+    Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
+    u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
+    u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
+
+    const u64 base = tile * (u64)T;
+    const u64 left = geo.n - base;
+    const int elems = left < (u64)T ? (int)left : T;
+
+    for (int i = tid; i < T; i += kGenericThreads) {
+        float d = 0.f, r = 0.f;
+        if (i < elems) { d = a.grad[base + i]; r = a.residue[base + i]; }
+        s_d[i] = d;
+        s_g[i] = __fadd_rn(r, d);
+    }
+    __syncthreads();
+
+    // bin maxima and per-bin counts
+    for (int b = warp; b < TB; b += nwarp) {
+        float m = 0.f;
+        for (int j = lane; j < L; j += 32) m = fmaxf(m, fabsf(s_g[b * L + j]));
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        u32 count = 0;
+        if (m > 0.f) {
+            for (int j0 = 0; j0 < L; j0 += 32) {
+                const int j = j0 + lane;
+                bool sel = false;
+                if (j < L) {
+                    const float g = s_g[b * L + j];
+                    const float h = __fadd_rn(g, s_d[b * L + j]);
+                    sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
+                }
+                count += __popc(__ballot_sync(0xffffffffu, sel));
+            }
+        }
+        if (lane == 0) {
+            s_gmax[b] = m;
+            s_cnt[b] = count;
+            const u64 bin = tile * (u64)TB + b;
+            if (bin < geo.n_bins) {
+                bin_cnt[bin] = (Word)count;
+                u32 window;
+                u64 lo, hi;
+                if (split_for_sum(m, window, lo, hi)) {
+                    atomicAdd(&s_acc[window], lo);
+                    atomicAdd(&s_acc[window + 1], hi);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    block_exclusive_scan(s_cnt, TB, s_tmp);
+
+    // words, in ascending order inside each bin
+    for (int b = warp; b < TB; b += nwarp) {
+        const float m = s_gmax[b];
+        if (!(m > 0.f)) continue;
+        u32 at = s_cnt[b];
+        for (int j0 = 0; j0 < L; j0 += 32) {
+            const int j = j0 + lane;
+            bool sel = false;
+            float g = 0.f;
+            if (j < L) {
+                g = s_g[b * L + j];
+                const float h = __fadd_rn(g, s_d[b * L + j]);
+                sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
+            }
+            const u32 mask = __ballot_sync(0xffffffffu, sel);
+            if (sel) {
+                const u32 pos = at + __popc(mask & ((1u << lane) - 1u));
+                s_words[pos] = (Word)(((u32)j << 2) | (g < 0.f ? 3u : 1u));
+            }
+            at += __popc(mask);
+        }
+    }
+    __syncthreads();
+
+    for (int i = tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
+    const u32 total = s_cnt[TB];
+    Word *slot = reinterpret_cast<Word *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
+    for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
+    if (tid == 0) {
+        tile_cnt[tile] = total;
+        if (total) atomicAdd(&group_cnt[tile / kGroupTiles], (u64)total);
+    }
+    __syncthreads();
+}
+
 template <typename Word>
 __global__ void __launch_bounds__(kGenericThreads)
 tile_pass_generic(PassArgs a)
@@ -572,107 +679,12 @@ tile_pass_generic(PassArgs a)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 s_tmp[33];
     __shared__ u64 s_acc[kWindows + 1];
-
-    const Geometry &geo = a.geo;
-    const int T = (int)geo.tile_elems, TB = (int)geo.tile_bins, L = (int)geo.L_T;
-    float *s_d = reinterpret_cast<float *>(smem_raw);
-    float *s_g = s_d + T;
-    Word *s_words = reinterpret_cast<Word *>(s_g + T);
-    float *s_gmax = reinterpret_cast<float *>(smem_raw + align_up((u64)T * (8 + sizeof(Word)), 16));
-    u32 *s_cnt = reinterpret_cast<u32 *>(s_gmax + TB);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
-    Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
-    u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
-    u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
-
+    const int tid = threadIdx.x;
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
-
-    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
-        const u64 base = tile * (u64)T;
-        const u64 left = geo.n - base;
-        const int elems = left < (u64)T ? (int)left : T;
-
-        for (int i = tid; i < T; i += kGenericThreads) {
-            float d = 0.f, r = 0.f;
-            if (i < elems) { d = a.grad[base + i]; r = a.residue[base + i]; }
-            s_d[i] = d;
-            s_g[i] = __fadd_rn(r, d);
-        }
-        __syncthreads();
-
-        // bin maxima and per-bin counts
-        for (int b = warp; b < TB; b += nwarp) {
-            float m = 0.f;
-            for (int j = lane; j < L; j += 32) m = fmaxf(m, fabsf(s_g[b * L + j]));
-            for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
-            u32 count = 0;
-            if (m > 0.f) {
-                for (int j0 = 0; j0 < L; j0 += 32) {
-                    const int j = j0 + lane;
-                    bool sel = false;
-                    if (j < L) {
-                        const float g = s_g[b * L + j];
-                        const float h = __fadd_rn(g, s_d[b * L + j]);
-                        sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
-                    }
-                    count += __popc(__ballot_sync(0xffffffffu, sel));
-                }
-            }
-            if (lane == 0) {
-                s_gmax[b] = m;
-                s_cnt[b] = count;
-                const u64 bin = tile * (u64)TB + b;
-                if (bin < geo.n_bins) {
-                    bin_cnt[bin] = (Word)count;
-                    u32 window;
-                    u64 lo, hi;
-                    if (split_for_sum(m, window, lo, hi)) {
-                        atomicAdd(&s_acc[window], lo);
-                        atomicAdd(&s_acc[window + 1], hi);
-                    }
-                }
-            }
-        }
-        __syncthreads();
-        block_exclusive_scan(s_cnt, TB, s_tmp);
-
-        // words, in ascending order inside each bin
-        for (int b = warp; b < TB; b += nwarp) {
-            const float m = s_gmax[b];
-            if (!(m > 0.f)) continue;
-            u32 at = s_cnt[b];
-            for (int j0 = 0; j0 < L; j0 += 32) {
-                const int j = j0 + lane;
-                bool sel = false;
-                float g = 0.f;
-                if (j < L) {
-                    g = s_g[b * L + j];
-                    const float h = __fadd_rn(g, s_d[b * L + j]);
-                    sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
-                }
-                const u32 mask = __ballot_sync(0xffffffffu, sel);
-                if (sel) {
-                    const u32 pos = at + __popc(mask & ((1u << lane) - 1u));
-                    s_words[pos] = (Word)(((u32)j << 2) | (g < 0.f ? 3u : 1u));
-                }
-                at += __popc(mask);
-            }
-        }
-        __syncthreads();
-
-        for (int i = tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
-        const u32 total = s_cnt[TB];
-        Word *slot = reinterpret_cast<Word *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
-        for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
-        if (tid == 0) {
-            tile_cnt[tile] = total;
-            if (total) atomicAdd(&group_cnt[tile / kGroupTiles], (u64)total);
-        }
-        __syncthreads();
-    }
-
+    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal};
+    for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x)
+        generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
     if (tid < kWindows) {
         const u64 v = s_acc[tid];
         if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + tid, v);
@@ -717,9 +729,8 @@ __device__ double windows_to_double(const u64 *win)
     return scalbn((double)mant, low - 149);
 }
 
-__global__ void __launch_bounds__(1024)
-finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out,
-         unsigned char *lazy_state)
+__device__ void finalize_body(unsigned char *packed, unsigned char *scratch, const Geometry &geo, u32 flags,
+                              u64 *count_out, unsigned char *lazy_state)
 {
     __shared__ u64 s_warp[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -799,6 +810,13 @@ finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags,
     if ((u64)tid < geo.payload_at - cnt_end) packed[cnt_end + tid] = 0;
 }
 
+__global__ void __launch_bounds__(1024)
+finalize(unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out,
+         unsigned char *lazy_state)
+{
+    finalize_body(packed, scratch, geo, flags, count_out, lazy_state);
+}
+
 // ---------------------------------------------------------------------------------
 // gather_fixup: per tile, copy the slot's words to the payload, write the tile's
 // directory entry and finish the residue of the sent elements:
@@ -822,6 +840,76 @@ __device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &
     return group[g] + before;
 }
 
+// One tile of at most 96 bins, handled by one warp.
+template <typename Word, bool FIXUP>
+__device__ void gather_tile_small(float *residue, unsigned char *packed, const unsigned char *scratch,
+                                  const Geometry &geo, u64 tile, int lane, u32 *s_pre)
+{
+    const int TB = (int)geo.tile_bins;
+    u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
+    const Word *bin_cnt = reinterpret_cast<const Word *>(packed + geo.bin_cnt_at);
+    Word *payload = reinterpret_cast<Word *>(packed + geo.payload_at);
+    const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
+    u32 cnt;
+    const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
+    if (lane == 0) tile_off[tile] = off0;
+    if (cnt == 0) return;
+    // exclusive scan of the tile's bin counts, three bins per lane (only the fix-up needs bins)
+    const u64 bin0 = tile * (u64)TB;
+    u32 c[3], sum = 0;
+    if (FIXUP) {
+#pragma unroll
+    for (int q = 0; q < 3; q++) {
+        const int b = lane * 3 + q;
+        c[q] = (b < TB && bin0 + b < geo.n_bins) ? (u32)bin_cnt[bin0 + b] : 0u;
+        sum += c[q];
+    }
+    const u32 inc = warp_inclusive_scan(sum, lane);
+    u32 run = inc - sum;
+    __syncwarp();
+#pragma unroll
+    for (int q = 0; q < 3; q++) {
+        const int b = lane * 3 + q;
+        if (b < TB) s_pre[b] = run;
+        run += c[q];
+    }
+    if (lane == 31) s_pre[TB] = inc;
+    __syncwarp();
+    }
+    const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
+    const u64 base = tile * (u64)geo.tile_elems;
+    for (u32 j0 = 0; j0 < cnt; j0 += 128) {
+        // four words per lane per round: their residue loads overlap
+        u32 word[4];
+        u64 pos[4];
+        float g[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            const u32 j = j0 + q * 32 + lane;
+            word[q] = 0;
+            pos[q] = 0;
+            g[q] = 0.f;
+            if (j < cnt) {
+                word[q] = slot[j];
+                if (FIXUP) {
+                    const int b = bin_of_word(s_pre, TB, j);
+                    pos[q] = base + (u64)b * geo.L_T + (word[q] >> 2);
+                    g[q] = residue[pos[q]];
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            const u32 j = j0 + q * 32 + lane;
+            if (j < cnt) {
+                if (FIXUP) residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
+                payload[off0 + j] = (Word)word[q];
+            }
+        }
+    }
+    __syncwarp();
+}
+
 // Tiles of at most 96 bins: one warp per tile.
 template <typename Word, bool FIXUP>
 __global__ void __launch_bounds__(kGatherThreads)
@@ -829,77 +917,11 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
 {
     __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    u32 *s_pre = s_pre_all[warp];
-    const int TB = (int)geo.tile_bins;
-    u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
-    const Word *bin_cnt = reinterpret_cast<const Word *>(packed + geo.bin_cnt_at);
-    Word *payload = reinterpret_cast<Word *>(packed + geo.payload_at);
-    const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
     const u64 warps = (u64)gridDim.x * (kGatherThreads / 32);
-
     // Last tile first: the tile pass wrote the residue front to back, so its tail is what the
     // L2 still holds when this kernel starts.
-    for (u64 item = (u64)blockIdx.x * (kGatherThreads / 32) + warp; item < geo.n_tiles; item += warps) {
-        const u64 tile = geo.n_tiles - 1 - item;
-        u32 cnt;
-        const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
-        if (lane == 0) tile_off[tile] = off0;
-        if (cnt == 0) continue;
-        // exclusive scan of the tile's bin counts, three bins per lane (only the fix-up needs bins)
-        const u64 bin0 = tile * (u64)TB;
-        u32 c[3], sum = 0;
-        if (FIXUP) {
-#pragma unroll
-        for (int q = 0; q < 3; q++) {
-            const int b = lane * 3 + q;
-            c[q] = (b < TB && bin0 + b < geo.n_bins) ? (u32)bin_cnt[bin0 + b] : 0u;
-            sum += c[q];
-        }
-        const u32 inc = warp_inclusive_scan(sum, lane);
-        u32 run = inc - sum;
-        __syncwarp();
-#pragma unroll
-        for (int q = 0; q < 3; q++) {
-            const int b = lane * 3 + q;
-            if (b < TB) s_pre[b] = run;
-            run += c[q];
-        }
-        if (lane == 31) s_pre[TB] = inc;
-        __syncwarp();
-        }
-        const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
-        const u64 base = tile * (u64)geo.tile_elems;
-        for (u32 j0 = 0; j0 < cnt; j0 += 128) {
-            // four words per lane per round: their residue loads overlap
-            u32 word[4];
-            u64 pos[4];
-            float g[4];
-#pragma unroll
-            for (int q = 0; q < 4; q++) {
-                const u32 j = j0 + q * 32 + lane;
-                word[q] = 0;
-                pos[q] = 0;
-                g[q] = 0.f;
-                if (j < cnt) {
-                    word[q] = slot[j];
-                    if (FIXUP) {
-                        const int b = bin_of_word(s_pre, TB, j);
-                        pos[q] = base + (u64)b * geo.L_T + (word[q] >> 2);
-                        g[q] = residue[pos[q]];
-                    }
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 4; q++) {
-                const u32 j = j0 + q * 32 + lane;
-                if (j < cnt) {
-                    if (FIXUP) residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
-                    payload[off0 + j] = (Word)word[q];
-                }
-            }
-        }
-        __syncwarp();
-    }
+    for (u64 item = (u64)blockIdx.x * (kGatherThreads / 32) + warp; item < geo.n_tiles; item += warps)
+        gather_tile_small<Word, FIXUP>(residue, packed, scratch, geo, geo.n_tiles - 1 - item, lane, s_pre_all[warp]);
 }
 
 // Any tile shape: one CTA per tile.
@@ -944,6 +966,117 @@ gather_fixup(float *residue, unsigned char *packed, const unsigned char *scratch
             payload[off0 + j] = (Word)word;
         }
         __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Batched pack(): many small layers in four launches instead of four launches per layer.
+// The layer table travels in the kernel parameters; a global tile index runs over the tiles
+// of all layers, and every CTA (tile pass) or warp (gather) looks its tile's layer up.
+// Layers of 42 <= L_T <= 1000 (tiles of at most 4000 elements and 96 bins) qualify.
+// ---------------------------------------------------------------------------------
+
+constexpr int kBatchMax = 160;                       // layers per batched launch (parameter space: 32 KB)
+constexpr u64 kBatchLayerMaxElems = 1ull << 22;      // larger layers take the single-layer kernels
+constexpr u32 kBatchSmemBytes = 4000 * 10 + 4 * kSmallBins + 4 * (kSmallBins + 1) + 16;
+
+struct BatchLayer {
+    const float *grad;
+    float *residue;
+    unsigned char *packed;
+    u64 *count_out;
+    Geometry geo;
+    u32 tile_first;                                  // global index of the layer's first tile
+    u32 pad;
+};
+
+// The table comes in two sizes: kernel parameters are copied at every launch, and a launch with the
+// full 27 KB table costs several microseconds more than one with the small table.
+constexpr int kBatchSmall = 16;
+
+template <int N>
+struct BatchArgsT {
+    u32 n_layers, total_tiles;
+    BatchLayer layer[N];
+};
+typedef BatchArgsT<kBatchMax> BatchArgs;
+
+// Largest i with layer[i].tile_first <= gt (layers without tiles are skipped by construction).
+template <int N>
+__device__ inline int batch_layer_of(const BatchArgsT<N> &b, u32 gt)
+{
+    int lo = 0, hi = (int)b.n_layers;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (b.layer[mid].tile_first <= gt) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <int N>
+__global__ void __launch_bounds__(128)
+batch_clear(const __grid_constant__ BatchArgsT<N> b)
+{
+    const BatchLayer &L = b.layer[blockIdx.x];
+    u64 *z = reinterpret_cast<u64 *>(L.packed + L.geo.scratch_at);
+    const u64 words = kCtlBytes / 8 + L.geo.n_groups;
+    for (u64 i = threadIdx.x; i < words; i += blockDim.x) z[i] = 0;
+}
+
+template <int N>
+__global__ void __launch_bounds__(kGenericThreads)
+batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ u32 s_tmp[33];
+    __shared__ u64 s_acc[kWindows + 1];
+    const int tid = threadIdx.x;
+    if (tid < kWindows + 1) s_acc[tid] = 0;
+    __syncthreads();
+    int cur = -1;
+    auto flush = [&]() {        // this CTA's share of the current layer's exact sum
+        if (cur >= 0 && tid < kWindows) {
+            const u64 v = s_acc[tid];
+            if (v) atomicAdd(reinterpret_cast<u64 *>(b.layer[cur].packed + b.layer[cur].geo.scratch_at) + tid, v);
+            s_acc[tid] = 0;
+        }
+    };
+    for (u32 gt = blockIdx.x; gt < b.total_tiles; gt += gridDim.x) {
+        const int li = batch_layer_of(b, gt);
+        if (li != cur) {
+            flush();
+            cur = li;
+        }
+        const BatchLayer &L = b.layer[li];
+        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u};
+        if (L.geo.w == 1u) generic_tile<unsigned char>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
+        else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
+    }
+    flush();
+}
+
+template <int N>
+__global__ void __launch_bounds__(1024)
+batch_finalize(const __grid_constant__ BatchArgsT<N> b)
+{
+    const BatchLayer &L = b.layer[blockIdx.x];
+    finalize_body(L.packed, L.packed + L.geo.scratch_at, L.geo, 0u, L.count_out, nullptr);
+}
+
+template <int N>
+__global__ void __launch_bounds__(kGatherThreads)
+batch_gather(const __grid_constant__ BatchArgsT<N> b)
+{
+    __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const u32 warps = gridDim.x * (kGatherThreads / 32);
+    for (u32 gt = blockIdx.x * (kGatherThreads / 32) + warp; gt < b.total_tiles; gt += warps) {
+        const BatchLayer &L = b.layer[batch_layer_of(b, gt)];
+        const unsigned char *scratch = L.packed + L.geo.scratch_at;
+        if (L.geo.w == 1u)
+            gather_tile_small<unsigned char, true>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
+        else
+            gather_tile_small<unsigned short, true>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
     }
 }
 
@@ -1810,6 +1943,7 @@ struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
     int decode_per_sm = 0;
+    int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
     bool fast_ready = false;
 };
 
@@ -1835,6 +1969,15 @@ int device_info(DeviceInfo *&out)
                        cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false>, at, bytes) == cudaSuccess &&
                        cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, true>, at, bytes) == cudaSuccess &&
                        cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, true>, at, bytes) == cudaSuccess;
+        if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kBatchSmemBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(batch_tile_pass<kBatchSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kBatchSmemBytes) == cudaSuccess) {
+            int per = 0;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, batch_tile_pass<kBatchMax>, kGenericThreads,
+                                                          kBatchSmemBytes);
+            d.batch_per_sm = per;
+        }
         d.sms = sms;
     }
     out = &d;
@@ -1958,6 +2101,47 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     decode_sum<<<(unsigned)(info->sms * info->decode_per_sm), kDecodeLaunch, 0,
                  static_cast<cudaStream_t>(stream)>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+}
+
+template <int N>
+int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStream_t st)
+{
+    batch_clear<N><<<b.n_layers, 128, 0, st>>>(b);
+    if (b.total_tiles) {
+        const u64 cap = (u64)info.sms * info.batch_per_sm;
+        const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
+        batch_tile_pass<N><<<grid, kGenericThreads, kBatchSmemBytes, st>>>(b);
+    }
+    batch_finalize<N><<<b.n_layers, 1024, 0, st>>>(b);
+    if (b.total_tiles) {
+        const u64 want = ((u64)b.total_tiles + 3) / 4, cap = (u64)info.sms * 16;
+        batch_gather<N><<<(unsigned)(want < cap ? want : cap), kGatherThreads, 0, st>>>(b);
+    }
+    return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+}
+
+// Launches one batch (at most kBatchMax layers, all batchable) on the stream.
+int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st)
+{
+    if (b.n_layers == 0) return ADACOMP_OK;
+    if (b.n_layers == 1) {      // a batch of one gains nothing over the single-layer kernels
+        const BatchLayer &L = b.layer[0];
+        return compress_impl(L.grad, L.residue, L.geo.n, L.geo.L_T, L.packed, reinterpret_cast<uint64_t *>(L.count_out),
+                             st, 0);
+    }
+    if (b.n_layers <= (u32)kBatchSmall) {
+        BatchArgsT<kBatchSmall> small;
+        small.n_layers = b.n_layers;
+        small.total_tiles = b.total_tiles;
+        for (u32 i = 0; i < b.n_layers; i++) small.layer[i] = b.layer[i];
+        return launch_batch_sized(small, info, st);
+    }
+    return launch_batch_sized(b, info, st);
+}
+
+inline bool batchable(const adacomp_layer_desc &d)
+{
+    return d.flags == 0 && d.L_T >= 42u && d.L_T <= 1000u && d.n < kBatchLayerMaxElems;
 }
 
 // ---------------------------------------------------------------------------------
@@ -2189,12 +2373,38 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
         if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
         if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out)) return ADACOMP_ERR_ALIGN;
     }
+    DeviceInfo *info = nullptr;
+    int rc = device_info(info);
+    if (rc != ADACOMP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // small layers share four launches per batch; the rest go through the single-layer path
+    static thread_local BatchArgs batch;
+    batch.n_layers = 0;
+    batch.total_tiles = 0;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        int rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags);
-        if (rc != ADACOMP_OK) return rc;
+        if (info->batch_per_sm > 0 && batchable(d)) {
+            BatchLayer &L = batch.layer[batch.n_layers++];
+            L.grad = d.grad;
+            L.residue = d.residue;
+            L.packed = static_cast<unsigned char *>(d.packed_out);
+            L.count_out = reinterpret_cast<u64 *>(d.count_out);
+            L.geo = make_geometry(d.n, d.L_T);
+            L.tile_first = batch.total_tiles;
+            L.pad = 0;
+            batch.total_tiles += (u32)L.geo.n_tiles;
+            if (batch.n_layers == (u32)kBatchMax) {
+                rc = launch_batch(batch, *info, st);
+                if (rc != ADACOMP_OK) return rc;
+                batch.n_layers = 0;
+                batch.total_tiles = 0;
+            }
+        } else {
+            rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags);
+            if (rc != ADACOMP_OK) return rc;
+        }
     }
-    return ADACOMP_OK;
+    return launch_batch(batch, *info, st);
 }
 
 int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_streams, float *const *dst,

@@ -231,7 +231,13 @@ def test_nonfinite_gradient_sets_a_status_bit_and_returns():
 
 
 def test_multi_tensor_calls_match_single_calls():
-    specs = synth.resnet50_tensors()[:30]
+    # a mix: small layers (batched launches), an empty one, bin lengths outside the batched range and
+    # one layer large enough for the single-layer fast path
+    specs = synth.resnet50_tensors()[:30] + [
+        synth.TensorSpec("empty", 0, 50, "fc"), synth.TensorSpec("odd_bins", 12345, 7, "fc"),
+        synth.TensorSpec("long_bins", 54321, 5000, "fc"), synth.TensorSpec("big", (1 << 22) + 4321, 50, "fc"),
+        synth.TensorSpec("tail_of_one", 4001, 500, "conv"), synth.TensorSpec("lt42", 9999, 42, "fc"),
+        synth.TensorSpec("lt1000", 99999, 1000, "fc")]
     dev = torch.device("cuda:0")
     layers, singles, dws = [], [], []
     for t, spec in enumerate(specs):
