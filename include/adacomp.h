@@ -165,6 +165,20 @@ int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams,
                                   void *stream);
 
 /*
+ * adacomp_decompress_accumulate for a caller that knows the tensor's shape on the host (the plain
+ * call reads n and L_T from the first stream's header on the device and must launch a full grid;
+ * here the grid is sized to the tensor, which matters for small layers).  Streams whose headers do
+ * not carry exactly (n, L_T) set ADACOMP_DEV_HEADER_MISMATCH and dst is left untouched.
+ */
+int adacomp_decompress_accumulate_ex(const void *const *packed, uint32_t k_streams, float *dst,
+                                     uint64_t n, uint32_t L_T, void *stream);
+
+/* adacomp_decompress_accumulate_multi with the layers' shapes (HOST arrays n[n_layers], L_T[n_layers]). */
+int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams,
+                                           float *const *dst, const uint64_t *n, const uint32_t *L_T,
+                                           uint32_t n_layers, void *stream);
+
+/*
  * adacomp_compress_ex with four caller-created cudaEvent_t handles (HOST array, as
  * void*) recorded on `stream` around the three kernels of pack(): events[0] before and
  * events[1] after the tile pass, events[2] after the scale/scan kernel, events[3] after

@@ -64,6 +64,12 @@ def lib() -> C.CDLL:
         L.adacomp_compress_ex.argtypes = L.adacomp_compress.argtypes + [C.c_uint32]
         L.adacomp_decompress_accumulate.restype = C.c_int
         L.adacomp_decompress_accumulate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.adacomp_decompress_accumulate_ex.restype = C.c_int
+        L.adacomp_decompress_accumulate_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64,
+                                                       C.c_uint32, C.c_void_p]
+        L.adacomp_decompress_accumulate_multi_ex.restype = C.c_int
+        L.adacomp_decompress_accumulate_multi_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
+                                                             C.c_void_p, C.c_uint32, C.c_void_p]
         L.adacomp_compress_profile.restype = C.c_int
         L.adacomp_compress_profile.argtypes = L.adacomp_compress_ex.argtypes + [C.c_void_p, C.c_void_p]
         L.adacomp_lazy_state_bytes.restype = C.c_size_t
@@ -174,6 +180,30 @@ def adacomp_decompress_accumulate(packed: Sequence[torch.Tensor], k_streams: int
     _check(lib().adacomp_decompress_accumulate(ptrs, int(k_streams),
                                                _dev_ptr(dst, "dst", torch.float32), _stream(stream)),
            "adacomp_decompress_accumulate")
+
+
+def adacomp_decompress_accumulate_ex(packed: Sequence[torch.Tensor], k_streams: int, dst, n: int,
+                                     L_T: int, stream=None) -> None:
+    """unpack()-and-sum when the caller knows (n, L_T): the grid is sized to the tensor."""
+    ptrs = (C.c_void_p * max(int(k_streams), 1))(
+        *[_dev_ptr(p, "packed[l]", torch.uint8) for p in packed[:k_streams]])
+    _check(lib().adacomp_decompress_accumulate_ex(ptrs, int(k_streams), _dev_ptr(dst, "dst", torch.float32),
+                                                  int(n), int(L_T), _stream(stream)),
+           "adacomp_decompress_accumulate_ex")
+
+
+def adacomp_decompress_accumulate_multi_ex(packed, k_streams: int, dst, n: Sequence[int],
+                                           L_T: Sequence[int], n_layers: int, stream=None) -> None:
+    """adacomp_decompress_accumulate_multi with the layers' shapes known on the host."""
+    if not isinstance(packed, C.Array):
+        packed = make_pointer_array(packed, torch.uint8)
+    if not isinstance(dst, C.Array):
+        dst = make_pointer_array(dst, torch.float32)
+    ns = (C.c_uint64 * max(int(n_layers), 1))(*[int(v) for v in n[:n_layers]])
+    lts = (C.c_uint32 * max(int(n_layers), 1))(*[int(v) for v in L_T[:n_layers]])
+    _check(lib().adacomp_decompress_accumulate_multi_ex(packed, int(k_streams), dst, ns, lts, int(n_layers),
+                                                        _stream(stream)),
+           "adacomp_decompress_accumulate_multi_ex")
 
 
 def adacomp_lazy_state_bytes(n: int, L_T: int) -> int:

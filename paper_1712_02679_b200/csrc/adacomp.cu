@@ -1088,7 +1088,18 @@ struct DecodeArgs {
     const unsigned char *stream[ADACOMP_MAX_STREAMS];
     float *dst;
     u32 k;
+    u32 hint_L_T;       // 0: the caller did not say; else the streams must carry exactly this shape
+    u64 hint_n;
 };
+
+// Work items of the decoder for a tensor: output tiles, split into chunks where a tile is larger.
+__host__ __device__ inline u64 decode_items(u64 n, u32 L_T)
+{
+    const u32 tile_bins = L_T <= 1000u ? 4u * (1000u / L_T) : 1u;
+    const u64 n_bins = (n + L_T - 1) / L_T;
+    const u64 n_tiles = (n_bins + tile_bins - 1) / tile_bins;
+    return n_tiles * (((u64)tile_bins * L_T + kDecodeChunk - 1) / kDecodeChunk);
+}
 
 constexpr int kWbufBytes = 8192;     // staged words of one round of learners (one learner's worst case fits)
 constexpr int kRoundMax = 4;         // learners per round
@@ -1850,7 +1861,9 @@ decode_sum(DecodeArgs a)
     const u32 *h0 = reinterpret_cast<const u32 *>(a.stream[0]);
     const u32 L_T = h0[2];
     const u64 n = reinterpret_cast<const u64 *>(a.stream[0])[2];
-    if (threadIdx.x == 0) s_bad = 0;
+    // CTAs beyond the tensor's last work item have nothing to do (CTA 0 stays to report bad headers)
+    if (blockIdx.x > 0 && L_T >= 1u && L_T <= ADACOMP_MAX_L_T && blockIdx.x >= decode_items(n, L_T)) return;
+    if (threadIdx.x == 0) s_bad = a.hint_L_T != 0 && (a.hint_L_T != L_T || a.hint_n != n);
     __syncthreads();
     if (threadIdx.x < a.k) {
         const u32 *h = reinterpret_cast<const u32 *>(a.stream[threadIdx.x]);
@@ -2081,7 +2094,8 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
-int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *stream)
+int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *stream, uint64_t hint_n = 0,
+                    uint32_t hint_L_T = 0)
 {
     if (!packed || !dst) return ADACOMP_ERR_NULL;
     if (k == 0 || k > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
@@ -2095,11 +2109,17 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     if (misaligned(dst)) return ADACOMP_ERR_ALIGN;
     args.dst = dst;
     args.k = k;
+    args.hint_n = hint_n;
+    args.hint_L_T = hint_L_T;
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
-    decode_sum<<<(unsigned)(info->sms * info->decode_per_sm), kDecodeLaunch, 0,
-                 static_cast<cudaStream_t>(stream)>>>(args);
+    u64 grid = (u64)info->sms * info->decode_per_sm;
+    if (hint_L_T) {             // the shape is known on the host: no more CTAs than work items
+        const u64 items = decode_items(hint_n, hint_L_T);
+        grid = items < grid ? (items ? items : 1) : grid;
+    }
+    decode_sum<<<(unsigned)grid, kDecodeLaunch, 0, static_cast<cudaStream_t>(stream)>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
@@ -2275,6 +2295,27 @@ int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams,
     return decompress_impl(packed, k_streams, dst, stream);
 }
 
+int adacomp_decompress_accumulate_ex(const void *const *packed, uint32_t k_streams, float *dst, uint64_t n,
+                                     uint32_t L_T, void *stream)
+{
+    if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    return decompress_impl(packed, k_streams, dst, stream, n, L_T);
+}
+
+int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams, float *const *dst,
+                                           const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream)
+{
+    if (n_layers && (!packed || !dst || !n || !L_T)) return ADACOMP_ERR_NULL;
+    if (k_streams == 0 || k_streams > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
+    for (uint32_t t = 0; t < n_layers; t++)
+        if (L_T[t] == 0 || L_T[t] > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    for (uint32_t t = 0; t < n_layers; t++) {
+        int rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, dst[t], stream, n[t], L_T[t]);
+        if (rc != ADACOMP_OK) return rc;
+    }
+    return ADACOMP_OK;
+}
+
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                              uint64_t *count_out, void *stream, uint32_t flags, void *const *events,
                              void *lazy_state)
@@ -2373,6 +2414,7 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
         if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
         if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out)) return ADACOMP_ERR_ALIGN;
     }
+    if (n_layers == 0) return ADACOMP_OK;
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;

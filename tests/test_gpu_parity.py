@@ -182,6 +182,31 @@ def test_decode_sum_dense_streams_overflow_the_prefetch_stage():
     assert B.adacomp_device_status() == 0
 
 
+def test_decode_with_shape_hint_matches_and_rejects_wrong_hints():
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(31)
+    for L_T, n in [(50, 777), (500, 4000 * 12 + 5), (7, 3000), (50, 4000 * 300)]:
+        raws = []
+        for l in range(3):
+            dW = rng.normal(0, 1e-3 * (l + 1), n).astype(np.float32)
+            raws.append(cref.pack(dW, np.zeros(n, np.float32), L_T).raw)
+        bufs = [torch.from_numpy(r.copy()).to(dev) for r in raws]
+        dst = torch.full((n,), float("nan"), device=dev)
+        B.adacomp_decompress_accumulate_ex(bufs, 3, dst, n, L_T)
+        torch.cuda.synchronize()
+        assert_f32_bits_equal(dst.cpu().numpy(), cref.unpack_sum(raws, n), f"hinted decode L_T={L_T} n={n}")
+        dsts = [torch.empty(n, device=dev) for _ in range(2)]
+        B.adacomp_decompress_accumulate_multi_ex(bufs + bufs, 3, dsts, [n, n], [L_T, L_T], 2)
+        torch.cuda.synchronize()
+        assert torch.equal(dsts[0], dst) and torch.equal(dsts[1], dst)
+        assert B.adacomp_device_status() == 0
+        dst.fill_(float("nan"))
+        B.adacomp_decompress_accumulate_ex(bufs, 3, dst, n + 1, L_T)       # wrong n: flagged, dst untouched
+        assert B.adacomp_device_status() & B.ADACOMP_DEV_HEADER_MISMATCH
+        assert bool(torch.isnan(dst).all())
+        B.adacomp_device_status_reset()
+
+
 def test_decode_sum_seeded_four_learners_crosscheck():
     import zlib
     spec = synth.config2_tensors()[7]
