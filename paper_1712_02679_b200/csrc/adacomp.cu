@@ -1194,7 +1194,7 @@ __device__ inline u32 check_fields(u32 x, u32 L_T)
 
 // Fast decode for tiles of at most 96 bins and 4096 elements (L_T = 42..1000).
 //
-// Per tile: (1) each learner's word range comes from its directory (fetched one tile ahead);
+// Per tile: (1) each learner's word range comes from its directory;
 // (2) the words of a round of up to four learners are staged in shared memory with 16-byte
 // loads, all in flight together, and checked as they pass (reserved code, index beyond the
 // bin); (3) the words are added into the output tile in learner order:
@@ -1206,7 +1206,8 @@ __device__ inline u32 check_fields(u32 x, u32 L_T)
 // A stream that fails a check raises a status bit; its words are still applied with the index
 // clamped into the bin, so nothing is read or written out of bounds.
 template <typename Word, bool BY_BIN>
-__device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
+__device__ void decode_item_staged(const unsigned char *const *streams, u32 k, const Geometry &geo, u64 tile,
+                                   float *dst, DecodeSmem &sm, u32 &bad)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
@@ -1216,160 +1217,153 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
     constexpr u32 kCap = kWbufBytes / 16;
     int top_probe = 1;                         // by word: highest power of two below the bin count
     while (top_probe * 2 < TB) top_probe *= 2;
+    const u64 base = tile * (u64)geo.tile_elems;
+    const u64 bin0 = tile * (u64)TB;
 
-    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
-    if (tid < (int)a.k) {
-        sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[tid])[12]);
-        sm.n_sel[tid] = reinterpret_cast<const u64 *>(a.stream[tid])[5];
+    if (tid < (int)k) {
+        const unsigned char *s = streams[tid];
+        const u64 n_sel = reinterpret_cast<const u64 *>(s)[5];
+        const u64 *dir = reinterpret_cast<const u64 *>(s + geo.tile_off_at);
+        const u64 o0 = dir[tile], o1 = dir[tile + 1];
+        // a malformed directory must not send the copy below out of the stream
+        const bool ok = o1 >= o0 && o1 - o0 <= geo.tile_elems && o1 <= n_sel;
+        if (!ok) bad |= ADACOMP_DEV_BAD_STREAM;
+        sm.scale[tid] = __uint_as_float(reinterpret_cast<const u32 *>(s)[12]);
+        sm.f.off0[tid] = o0;
+        sm.f.cnt[tid] = ok ? (u32)(o1 - o0) : 0u;
     }
-    // directory entries of the first tile; those of the next tile are fetched one tile ahead
-    u64 nx0 = 0, nx1 = 0;
-    if (tid < (int)a.k && blockIdx.x < geo.n_tiles) {
-        const u64 *dir = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at);
-        nx0 = dir[blockIdx.x];
-        nx1 = dir[blockIdx.x + 1];
-    }
-    u32 bad = 0;
-    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x) {
-        const u64 base = tile * (u64)geo.tile_elems;
-        const u64 bin0 = tile * (u64)TB;
-        if (tid < (int)a.k) {
-            // a malformed directory must not send the copy below out of the stream
-            const bool ok = nx1 >= nx0 && nx1 - nx0 <= geo.tile_elems && nx1 <= sm.n_sel[tid];
-            if (!ok) bad |= ADACOMP_DEV_BAD_STREAM;
-            sm.f.off0[tid] = nx0;
-            sm.f.cnt[tid] = ok ? (u32)(nx1 - nx0) : 0u;
-            const u64 next = tile + gridDim.x;
-            if (next < geo.n_tiles) {
-                const u64 *dir = reinterpret_cast<const u64 *>(a.stream[tid] + geo.tile_off_at);
-                nx0 = dir[next];
-                nx1 = dir[next + 1];
+    consumer_barrier();
+
+    for (u32 g0 = 0; g0 < k; g0 += kRoundMax) {
+        // ---- a group of up to four learners: one round if its words fit the staging
+        //      buffer, else one round per learner (a single learner's tile always fits) ----
+        const int R = (int)min((u32)kRoundMax, k - g0);
+        u64 src[kRoundMax];
+        u32 chunks[kRoundMax], headb[kRoundMax], cnts[kRoundMax];
+        u32 total = 0;
+#pragma unroll
+        for (int q = 0; q < kRoundMax; q++) {
+            src[q] = 0; chunks[q] = 0; headb[q] = 0; cnts[q] = 0;
+            if (q < R) {
+                const u64 p = (u64)(uintptr_t)(streams[g0 + q] + geo.payload_at) + sm.f.off0[g0 + q] * sizeof(Word);
+                cnts[q] = sm.f.cnt[g0 + q];
+                headb[q] = (u32)(p & 15u);
+                src[q] = p & ~(u64)15u;
+                chunks[q] = cnts[q] ? (headb[q] + cnts[q] * (u32)sizeof(Word) + 15u) / 16u : 0u;
+                total += chunks[q];
             }
         }
-        consumer_barrier();
-
-        for (u32 g0 = 0; g0 < a.k; g0 += kRoundMax) {
-            // ---- a group of up to four learners: one round if its words fit the staging
-            //      buffer, else one round per learner (a single learner's tile always fits) ----
-            const int R = (int)min((u32)kRoundMax, a.k - g0);
-            u64 src[kRoundMax];
-            u32 chunks[kRoundMax], headb[kRoundMax], cnts[kRoundMax];
-            u32 total = 0;
+        const bool fits = total <= kCap;
+        const int nsub = fits ? 1 : R;
+        for (int sub = 0; sub < nsub; sub++) {
+            // learners of this round: q in [q_lo, q_hi); chunk offsets at[q] within the buffer
+            const int q_lo = fits ? 0 : sub, q_hi = fits ? R : sub + 1;
+            u32 at[kRoundMax + 1];
+            at[0] = 0;
 #pragma unroll
-            for (int q = 0; q < kRoundMax; q++) {
-                src[q] = 0; chunks[q] = 0; headb[q] = 0; cnts[q] = 0;
-                if (q < R) {
-                    const u64 p = (u64)(uintptr_t)(a.stream[g0 + q] + geo.payload_at) + sm.f.off0[g0 + q] * sizeof(Word);
-                    cnts[q] = sm.f.cnt[g0 + q];
-                    headb[q] = (u32)(p & 15u);
-                    src[q] = p & ~(u64)15u;
-                    chunks[q] = cnts[q] ? (headb[q] + cnts[q] * (u32)sizeof(Word) + 15u) / 16u : 0u;
-                    total += chunks[q];
-                }
+            for (int q = 0; q < kRoundMax; q++)
+                at[q + 1] = at[q] + ((q >= q_lo && q < q_hi) ? chunks[q] : 0u);
+
+            // ---- stage and check the words ----
+            for (u32 c = tid; c < at[kRoundMax]; c += kDecodeThreads) {
+                u64 from = src[0];
+                u32 first = 0;
+#pragma unroll
+                for (int q = 1; q < kRoundMax; q++)
+                    if (c >= at[q]) { from = src[q]; first = at[q]; }
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(from) + (c - first));
+                bad |= check_fields<Word>(v.x, L_T) | check_fields<Word>(v.y, L_T) |
+                       check_fields<Word>(v.z, L_T) | check_fields<Word>(v.w, L_T);
+                sm.f.wbuf[c] = v;
             }
-            const bool fits = total <= kCap;
-            const int nsub = fits ? 1 : R;
-            for (int sub = 0; sub < nsub; sub++) {
-                // learners of this round: q in [q_lo, q_hi); chunk offsets at[q] within the buffer
-                const int q_lo = fits ? 0 : sub, q_hi = fits ? R : sub + 1;
-                u32 at[kRoundMax + 1];
-                at[0] = 0;
-#pragma unroll
-                for (int q = 0; q < kRoundMax; q++)
-                    at[q + 1] = at[q] + ((q >= q_lo && q < q_hi) ? chunks[q] : 0u);
 
-                // ---- stage and check the words ----
-                for (u32 c = tid; c < at[kRoundMax]; c += kDecodeThreads) {
-                    u64 from = src[0];
-                    u32 first = 0;
+            if (BY_BIN) {
+                // ---- bin counts -> word offsets: two learners per scan (16 bits each) ----
+                const u64 bin = bin0 + tid;
+                const bool live = tid < TB && bin < geo.n_bins;
+                u32 c[kRoundMax];
 #pragma unroll
-                    for (int q = 1; q < kRoundMax; q++)
-                        if (c >= at[q]) { from = src[q]; first = at[q]; }
-                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(from) + (c - first));
-                    bad |= check_fields<Word>(v.x, L_T) | check_fields<Word>(v.y, L_T) |
-                           check_fields<Word>(v.z, L_T) | check_fields<Word>(v.w, L_T);
-                    sm.f.wbuf[c] = v;
+                for (int q = 0; q < kRoundMax; q++) {
+                    c[q] = 0;
+                    if (q >= q_lo && q < q_hi && live)
+                        c[q] = min((u32)reinterpret_cast<const Word *>(streams[g0 + q] + geo.bin_cnt_at)[bin], L_T);
                 }
-
-                if (BY_BIN) {
-                    // ---- bin counts -> word offsets: two learners per scan (16 bits each) ----
-                    const u64 bin = bin0 + tid;
-                    const bool live = tid < TB && bin < geo.n_bins;
-                    u32 c[kRoundMax];
+                u32 pair[2] = {c[0] | (c[1] << 16), c[2] | (c[3] << 16)};
+                u32 excl[2];
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    const u32 inc = warp_inclusive_scan(pair[h], lane);
+                    excl[h] = inc - pair[h];
+                    if (lane == 31) s_wsum[warp * 2 + h] = inc;
+                }
+                consumer_barrier();
+                if (tid < TB) {
+                    for (int wv = 0; wv < warp; wv++) {
+                        excl[0] += s_wsum[wv * 2];
+                        excl[1] += s_wsum[wv * 2 + 1];
+                    }
+                    const u32 pre[kRoundMax] = {excl[0] & 0xffffu, excl[0] >> 16, excl[1] & 0xffffu, excl[1] >> 16};
+                    float *mine = sm.acc + tid * L_T;
 #pragma unroll
                     for (int q = 0; q < kRoundMax; q++) {
-                        c[q] = 0;
-                        if (q >= q_lo && q < q_hi && live)
-                            c[q] = min((u32)reinterpret_cast<const Word *>(a.stream[g0 + q] + geo.bin_cnt_at)[bin], L_T);
-                    }
-                    u32 pair[2] = {c[0] | (c[1] << 16), c[2] | (c[3] << 16)};
-                    u32 excl[2];
-#pragma unroll
-                    for (int h = 0; h < 2; h++) {
-                        const u32 inc = warp_inclusive_scan(pair[h], lane);
-                        excl[h] = inc - pair[h];
-                        if (lane == 31) s_wsum[warp * 2 + h] = inc;
-                    }
-                    consumer_barrier();
-                    if (tid < TB) {
-                        for (int wv = 0; wv < warp; wv++) {
-                            excl[0] += s_wsum[wv * 2];
-                            excl[1] += s_wsum[wv * 2 + 1];
-                        }
-                        const u32 pre[kRoundMax] = {excl[0] & 0xffffu, excl[0] >> 16, excl[1] & 0xffffu, excl[1] >> 16};
-                        float *mine = sm.acc + tid * L_T;
-#pragma unroll
-                        for (int q = 0; q < kRoundMax; q++) {
-                            if (c[q] == 0) continue;
-                            if (pre[q] + c[q] > cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
-                            const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]) + pre[q];
-                            const u32 sbits = __float_as_uint(sm.scale[g0 + q]);
-                            for (u32 i = 0; i < c[q]; i++) {
-                                const u32 word = p[i];
-                                const u32 e = min(word >> 2, L_T - 1u);
-                                const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
-                                mine[e] = __fadd_rn(mine[e], add);
-                            }
-                        }
-                    }
-                    consumer_barrier();
-                } else {
-                    // warp wv scans the bin counts of learner wv of the round
-                    if (warp >= q_lo && warp < q_hi) {
-                        u32 c = 0;
-                        if (lane < TB && bin0 + lane < geo.n_bins)
-                            c = reinterpret_cast<const Word *>(a.stream[g0 + warp] + geo.bin_cnt_at)[bin0 + lane];
-                        const u32 inc = warp_inclusive_scan(c, lane);
-                        sm.f.bin_pre[warp][lane] = inc - c;
-                        if (lane == 31) sm.f.bin_pre[warp][32] = inc;
-                    }
-                    consumer_barrier();
-#pragma unroll
-                    for (int q = 0; q < kRoundMax; q++) {
-                        if (q < q_lo || q >= q_hi || cnts[q] == 0) continue;      // the same for every thread
-                        if (sm.f.bin_pre[q][32] != cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
-                        const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]);
+                        if (c[q] == 0) continue;
+                        if (pre[q] + c[q] > cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
+                        const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]) + pre[q];
                         const u32 sbits = __float_as_uint(sm.scale[g0 + q]);
-                        const u32 *pre = sm.f.bin_pre[q];
-                        for (u32 j = tid; j < cnts[q]; j += kDecodeThreads) {
-                            const u32 word = p[j];
-                            int b = 0;
-                            for (int step = top_probe; step > 0; step >>= 1)
-                                if (b + step < TB && pre[b + step] <= j) b += step;
-                            const u32 e = (u32)b * L_T + min(word >> 2, L_T - 1u);
+                        for (u32 i = 0; i < c[q]; i++) {
+                            const u32 word = p[i];
+                            const u32 e = min(word >> 2, L_T - 1u);
                             const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
-                            sm.acc[e] = __fadd_rn(sm.acc[e], add);
+                            mine[e] = __fadd_rn(mine[e], add);
                         }
-                        consumer_barrier();
                     }
-                    consumer_barrier();     // bin_pre and wbuf are rewritten by the next round
                 }
+                consumer_barrier();
+            } else {
+                // warp wv scans the bin counts of learner wv of the round
+                if (warp >= q_lo && warp < q_hi) {
+                    u32 c = 0;
+                    if (lane < TB && bin0 + lane < geo.n_bins)
+                        c = reinterpret_cast<const Word *>(streams[g0 + warp] + geo.bin_cnt_at)[bin0 + lane];
+                    const u32 inc = warp_inclusive_scan(c, lane);
+                    sm.f.bin_pre[warp][lane] = inc - c;
+                    if (lane == 31) sm.f.bin_pre[warp][32] = inc;
+                }
+                consumer_barrier();
+#pragma unroll
+                for (int q = 0; q < kRoundMax; q++) {
+                    if (q < q_lo || q >= q_hi || cnts[q] == 0) continue;      // the same for every thread
+                    if (sm.f.bin_pre[q][32] != cnts[q]) { bad |= ADACOMP_DEV_BAD_STREAM; continue; }
+                    const Word *p = reinterpret_cast<const Word *>(s_bytes + at[q] * 16u + headb[q]);
+                    const u32 sbits = __float_as_uint(sm.scale[g0 + q]);
+                    const u32 *pre = sm.f.bin_pre[q];
+                    for (u32 j = tid; j < cnts[q]; j += kDecodeThreads) {
+                        const u32 word = p[j];
+                        int b = 0;
+                        for (int step = top_probe; step > 0; step >>= 1)
+                            if (b + step < TB && pre[b + step] <= j) b += step;
+                        const u32 e = (u32)b * L_T + min(word >> 2, L_T - 1u);
+                        const float add = (word & 1u) ? __uint_as_float(sbits ^ ((word & 2u) << 30)) : 0.f;
+                        sm.acc[e] = __fadd_rn(sm.acc[e], add);
+                    }
+                    consumer_barrier();
+                }
+                consumer_barrier();     // bin_pre and wbuf are rewritten by the next round
             }
         }
-        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
-        store_tile(a.dst, base, len, sm.acc);
-        consumer_barrier();
     }
+    const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
+    store_tile(dst, base, len, sm.acc);
+    consumer_barrier();
+}
+
+template <typename Word, bool BY_BIN>
+__device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
+{
+    for (int i = threadIdx.x; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
+    u32 bad = 0;
+    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x)
+        decode_item_staged<Word, BY_BIN>(a.stream, a.k, geo, tile, a.dst, sm, bad);
     if (bad) raise_status(bad);
 }
 
@@ -1907,6 +1901,86 @@ decode_sum(DecodeArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------
+// Batched decode-sum: many small layers in one launch.  The layer table (shapes, output and
+// stream pointers) travels in the kernel parameters; every CTA builds the same tile index over
+// all layers in shared memory and takes (layer, tile) items from it.  Layers of
+// 42 <= L_T <= 1000 qualify (tiles of at most 4096 elements and 2..96 bins).
+// ---------------------------------------------------------------------------------
+
+constexpr int kDecBatchLayers = 96;
+constexpr int kDecBatchPtrs = 2900;
+
+struct DecodeBatchArgs {
+    u32 n_layers, k;
+    u64 n[kDecBatchLayers];
+    u32 L_T[kDecBatchLayers];
+    float *dst[kDecBatchLayers];
+    const unsigned char *stream[kDecBatchPtrs];      // [layer * k + learner]
+};
+
+struct DecodeBatchSmem {
+    DecodeSmem d;
+    Geometry geo[kDecBatchLayers];
+    u32 first[kDecBatchLayers + 1];                  // global index of each layer's first tile
+};
+
+__global__ void __launch_bounds__(kDecodeThreads)
+decode_batch(const __grid_constant__ DecodeBatchArgs b)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DecodeBatchSmem &sm = *reinterpret_cast<DecodeBatchSmem *>(smem_raw);
+    const int tid = threadIdx.x;
+    u32 bad = 0;
+    // every CTA checks every layer's k headers against the shape the caller gave and indexes the
+    // tiles of the layers that pass; a layer that fails is skipped (dst untouched) and reported
+    for (int t = tid; t < (int)b.n_layers; t += kDecodeThreads) {
+        const Geometry g = make_geometry(b.n[t], b.L_T[t]);
+        bool ok = true;
+        for (u32 l = 0; l < b.k; l++) {
+            const u32 *h = reinterpret_cast<const u32 *>(b.stream[t * b.k + l]);
+            const u64 *h64 = reinterpret_cast<const u64 *>(h);
+            ok = ok && h[0] == kMagic && (h[1] & 0xffffu) == 1u && h[2] == g.L_T && h64[2] == g.n &&
+                 ((h[1] >> 16) & 0xffu) == g.w && h[3] == g.tile_bins && h64[3] == g.n_bins &&
+                 h64[4] == g.n_tiles && h64[5] <= g.n;
+        }
+        if (!ok) bad |= ADACOMP_DEV_HEADER_MISMATCH;
+        sm.geo[t] = g;
+        sm.first[t + 1] = ok ? (u32)g.n_tiles : 0u;
+    }
+    for (int i = tid; i < kDecodeChunk; i += kDecodeThreads) sm.d.acc[i] = 0.f;
+    consumer_barrier();
+    if (tid == 0) {
+        u32 run = 0;
+        sm.first[0] = 0;
+        for (u32 t = 0; t < b.n_layers; t++) {
+            run += sm.first[t + 1];
+            sm.first[t + 1] = run;
+        }
+    }
+    consumer_barrier();
+    const u32 total = sm.first[b.n_layers];
+    for (u32 gt = blockIdx.x; gt < total; gt += gridDim.x) {
+        int lo = 0, hi = (int)b.n_layers;            // largest t with first[t] <= gt and a tile of its own
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (sm.first[mid] <= gt) lo = mid; else hi = mid;
+        }
+        const Geometry &geo = sm.geo[lo];
+        const u64 tile = gt - sm.first[lo];
+        const unsigned char *const *streams = &b.stream[lo * b.k];
+        if (geo.w == 1u) {
+            decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+        } else if (geo.tile_bins >= 32) {
+            decode_item_staged<unsigned short, true>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+        } else {
+            decode_item_staged<unsigned short, false>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+        }
+    }
+    if (bad && blockIdx.x == 0) raise_status(bad & ADACOMP_DEV_HEADER_MISMATCH);
+    if (bad & ~ADACOMP_DEV_HEADER_MISMATCH) raise_status(bad & ~ADACOMP_DEV_HEADER_MISMATCH);
+}
+
 __global__ void reset_status_kernel() { g_status = 0; }
 
 __global__ void lazy_init_kernel(unsigned char *state, u64 n, u32 L_T)
@@ -1957,6 +2031,7 @@ struct DeviceInfo {
     int smem_optin = 0;
     int decode_per_sm = 0;
     int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
+    int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
 };
 
@@ -1990,6 +2065,12 @@ int device_info(DeviceInfo *&out)
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, batch_tile_pass<kBatchMax>, kGenericThreads,
                                                           kBatchSmemBytes);
             d.batch_per_sm = per;
+        }
+        if (cudaFuncSetAttribute(decode_batch, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(DecodeBatchSmem)) == cudaSuccess) {
+            int per = 0;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, decode_batch, kDecodeThreads, sizeof(DecodeBatchSmem));
+            d.dec_batch_per_sm = per;
         }
         d.sms = sms;
     }
@@ -2307,13 +2388,57 @@ int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k
 {
     if (n_layers && (!packed || !dst || !n || !L_T)) return ADACOMP_ERR_NULL;
     if (k_streams == 0 || k_streams > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
-    for (uint32_t t = 0; t < n_layers; t++)
-        if (L_T[t] == 0 || L_T[t] > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
     for (uint32_t t = 0; t < n_layers; t++) {
-        int rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, dst[t], stream, n[t], L_T[t]);
-        if (rc != ADACOMP_OK) return rc;
+        if (L_T[t] == 0 || L_T[t] > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+        if (!dst[t]) return ADACOMP_ERR_NULL;
+        if (misaligned(dst[t])) return ADACOMP_ERR_ALIGN;
+        for (uint32_t l = 0; l < k_streams; l++) {
+            if (!packed[(size_t)t * k_streams + l]) return ADACOMP_ERR_NULL;
+            if (misaligned(packed[(size_t)t * k_streams + l])) return ADACOMP_ERR_ALIGN;
+        }
     }
-    return ADACOMP_OK;
+    if (n_layers == 0) return ADACOMP_OK;
+    DeviceInfo *info = nullptr;
+    int rc = device_info(info);
+    if (rc != ADACOMP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // small layers of the paper's bin lengths share launches; the rest are decoded one by one
+    static thread_local DecodeBatchArgs batch;
+    batch.n_layers = 0;
+    batch.k = k_streams;
+    u64 batch_tiles = 0;
+    auto flush = [&]() -> int {
+        if (batch.n_layers == 0) return ADACOMP_OK;
+        const u64 cap = (u64)info->sms * info->dec_batch_per_sm;
+        const unsigned grid = (unsigned)(batch_tiles < cap ? (batch_tiles ? batch_tiles : 1) : cap);
+        decode_batch<<<grid, kDecodeThreads, sizeof(DecodeBatchSmem), st>>>(batch);
+        batch.n_layers = 0;
+        batch_tiles = 0;
+        return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+    };
+    const uint32_t per_batch = (uint32_t)kDecBatchPtrs / k_streams < (uint32_t)kDecBatchLayers
+                                   ? (uint32_t)kDecBatchPtrs / k_streams : (uint32_t)kDecBatchLayers;
+    for (uint32_t t = 0; t < n_layers; t++) {
+        const bool small = info->dec_batch_per_sm > 0 && L_T[t] >= 42u && L_T[t] <= 1000u &&
+                           n[t] < kBatchLayerMaxElems && n_layers > 1;
+        if (small) {
+            const u32 i = batch.n_layers++;
+            batch.n[i] = n[t];
+            batch.L_T[i] = L_T[t];
+            batch.dst[i] = dst[t];
+            for (uint32_t l = 0; l < k_streams; l++)
+                batch.stream[(size_t)i * k_streams + l] = static_cast<const unsigned char *>(packed[(size_t)t * k_streams + l]);
+            batch_tiles += decode_items(n[t], L_T[t]);
+            if (batch.n_layers == per_batch) {
+                rc = flush();
+                if (rc != ADACOMP_OK) return rc;
+            }
+        } else {
+            rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, dst[t], stream, n[t], L_T[t]);
+            if (rc != ADACOMP_OK) return rc;
+        }
+    }
+    return flush();
 }
 
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,

@@ -64,7 +64,8 @@ def _multi_tensor_case(cfg, specs, learners, heavy_sigma=None):
     # one decode-sum of the `learners` streams of every tensor
     _, dsts = carve(lambda s: max(s.n, 4), torch.float32)
     flat_packed = [packed_views[l][t] for t in range(n_t) for l in range(learners)]
-    B.adacomp_decompress_accumulate_multi(flat_packed, learners, dsts, n_t)
+    B.adacomp_decompress_accumulate_multi_ex(flat_packed, learners, dsts, [s.n for s in specs],
+                                             [s.L_T for s in specs], n_t)
     torch.cuda.synchronize()
     with ThreadPoolExecutor(8) as ex:
         refs = list(ex.map(lambda t: cref.unpack_sum(streams_cpu[t], specs[t].n), range(n_t)))
