@@ -28,8 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "compress+pack GB/s of fp32 gradient"
 # dram__bytes_read.sum + dram__bytes_write.sum per element of tile_pass_fast, from the ncu capture
-# at n = 2^26 summarised in profiles/tile_pass_fast_n2e26_LT50.md; traffic grows in proportion to n.
-TILE_PASS_DRAM_BYTES_PER_ELEM = {50: 11.50}
+# at n = 2^26 summarised in profiles/tile_pass_fast_n2e26_LT50.md (L_T = 50) and
+# profiles/tile_pass_and_gather_n2e26_LT500.md (L_T = 500); traffic grows in proportion to n.
+TILE_PASS_DRAM_BYTES_PER_ELEM = {50: 11.50, 500: 11.38}
 SIGMA = 1e-3
 PREWARM_STEPS = 5
 FALLBACK_HBM_GBS = 6650.0
@@ -442,7 +443,8 @@ def run_ours(a):
                          "unit": "GB/s", "frac": achieved / peak,
                          "traffic": (TILE_PASS_DRAM_BYTES_PER_ELEM[L_T] * n
                                      if L_T in TILE_PASS_DRAM_BYTES_PER_ELEM else None),
-                         "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/tile_pass_fast_n2e26_LT50.md)",
+                         "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/tile_pass_fast_n2e26_LT50.md, "
+                                           "profiles/tile_pass_and_gather_n2e26_LT500.md)",
                          "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": tile_bytes},
             "clocks": ClockSampler.merge(clock_parts),
