@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-lazy", action="store_true")
     ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4"],
+                    help="sweep: flat tensor of 2^log2n (the default bench); configN: the multi-tensor "
+                         "parameter lists, through the *_multi entry points")
     return ap.parse_args()
 
 
@@ -478,10 +481,74 @@ def run_ours(a):
         dist.destroy_process_group()
 
 
+def run_multi_workload(a):
+    """One step of a multi-tensor config: every learner packs its whole parameter list with one
+    adacomp_compress_multi call, then one adacomp_decompress_accumulate_multi_ex sums the learners'
+    streams of every tensor.  First step from a zero residue (the densest the codec emits)."""
+    import torch
+
+    from paper_1712_02679_b200 import binding as B
+    from paper_1712_02679_b200 import synth
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = int(a.workload[-1])
+    specs, learners = {1: (synth.config1_tensors(), 1), 2: (synth.config2_tensors(), 1),
+                       3: (synth.resnet50_tensors(), 8), 4: (synth.config4_tensors(), 16)}[cfg]
+    nl, total = len(specs), sum(s.n for s in specs)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1712_02679 + cfg)
+    layers = []
+    for l in range(learners):
+        for s in specs:
+            n = max(s.n, 4)
+            layers.append(dict(grad=torch.empty(n, device=dev).normal_(0.0, SIGMA, generator=gen),
+                               residue=torch.zeros(n, device=dev), n=s.n, L_T=s.L_T,
+                               packed_out=torch.empty(B.adacomp_packed_capacity(s.n, s.L_T), dtype=torch.uint8, device=dev),
+                               count_out=torch.zeros(2, dtype=torch.int64, device=dev)))
+    descs = [B.make_layer_descs(layers[l * nl:(l + 1) * nl]) for l in range(learners)]
+    dsts = [torch.empty(max(s.n, 4), device=dev) for s in specs]
+    packed = B.make_pointer_array([layers[l * nl + t]["packed_out"] for t in range(nl) for l in range(learners)], torch.uint8)
+    dst_arr = B.make_pointer_array(dsts, torch.float32)
+    ns, lts = [s.n for s in specs], [s.L_T for s in specs]
+    K, W = a.steps, max(a.warmup, 3)
+    evs = []
+    for it in range(W + K):
+        for d in layers:
+            d["residue"].zero_()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        for l in range(learners):
+            B.adacomp_compress_multi(descs[l], nl)
+        e[1].record()
+        B.adacomp_decompress_accumulate_multi_ex(packed, learners, dst_arr, ns, lts, nl)
+        e[2].record()
+        if it >= W:
+            evs.append(e)
+    torch.cuda.synchronize()
+    t_c = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    t_d = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    n_sel = sum(int(d["count_out"][0]) for d in layers[:nl])
+    line = {
+        "metric": METRIC, "value": 4.0 * total * learners / ((t_c + t_d) * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1,
+        "steps": K, "warmup": W, "ms_per_step": t_c + t_d, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"config {cfg}: {nl} tensors, {total} elements, {learners} learners, first step "
+                               f"from a zero residue, dW~N(0,1e-3); *_multi entry points",
+                   "l2": "working set %.0f MB" % (12.0 * total * learners / 1e6)},
+        "compress_ms": t_c, "compress_gbs": 4.0 * total * learners / (t_c * 1e-3) / 1e9,
+        "decompress_sum_ms": t_d, "decompress_sum_gbs": 4.0 * total / (t_d * 1e-3) / 1e9,
+        "selected_fraction_learner0": n_sel / max(total, 1), "device_status": B.adacomp_device_status(),
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.workload != "sweep":
+        run_multi_workload(a)
     else:
         run_ours(a)
 
