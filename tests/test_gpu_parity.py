@@ -290,3 +290,23 @@ def test_multi_tensor_calls_match_single_calls():
         used = int(L.count[1])
         raw = L.packed[:used].cpu().numpy()
         assert_f32_bits_equal(dsts[t][:L.n].cpu().numpy(), cref.unpack_sum([raw, raw], L.n))
+
+
+def test_random_shapes_against_the_oracle():
+    """Seeded fuzz over (n, L_T, k): two carried pack() steps per learner and one dense sum."""
+    rng = np.random.default_rng(20261125)
+    for case in range(40):
+        L_T = int(rng.choice([int(rng.integers(1, 130)), int(rng.integers(130, 1100)),
+                              int(rng.integers(1100, 16385)), 50, 500]))
+        n = int(rng.integers(1, 60000))
+        k = int(rng.integers(1, 7))
+        streams = []
+        for l in range(k):
+            sigma = 10.0 ** rng.uniform(-5, 1)
+            dws = [synth.heavy_dw(n, sigma, rng) if rng.random() < 0.5 else
+                   rng.normal(0, sigma, n).astype(np.float32) for _ in range(2)]
+            layer, raws = run_steps(n, L_T, dws)
+            streams.append(raws[-1])
+        got = gpu_decode(streams, n)
+        assert_f32_bits_equal(got, cref.unpack_sum(streams, n), f"fuzz case {case}: n={n} L_T={L_T} k={k}")
+    assert B.adacomp_device_status() == 0
