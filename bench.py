@@ -234,6 +234,7 @@ def run_ours(a):
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    B.adacomp_set_device(local)          # the library's own CUDA runtime follows torch's choice
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 

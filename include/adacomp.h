@@ -261,6 +261,14 @@ int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_st
                                         float *const *dst, uint32_t n_layers, void *stream);
 
 /*
+ * Makes `device` the calling host thread's current CUDA device for this library.  Every entry
+ * point works on the calling thread's current device; a process that selects its GPU through
+ * another copy of the CUDA runtime (PyTorch's, say) calls this once per thread with the same
+ * ordinal so that both agree.  Not needed in single-GPU processes.
+ */
+int adacomp_set_device(int device);
+
+/*
  * Synchronises `stream`, then copies the current device's sticky ADACOMP_DEV_* bits to
  * *host_out.  The bits stay set until adacomp_device_status_reset.
  */

@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate_multi.restype = C.c_int
         L.adacomp_decompress_accumulate_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p,
                                                           C.c_uint32, C.c_void_p]
+        L.adacomp_set_device.restype = C.c_int
+        L.adacomp_set_device.argtypes = [C.c_int]
         L.adacomp_device_status.restype = C.c_int
         L.adacomp_device_status.argtypes = [C.c_void_p, C.c_void_p]
         L.adacomp_device_status_reset.restype = C.c_int
@@ -321,6 +323,11 @@ def adacomp_decompress_accumulate_multi(packed, k_streams: int, dst, n_layers: i
     _check(lib().adacomp_decompress_accumulate_multi(packed, int(k_streams), dst, int(n_layers),
                                                      _stream(stream)),
            "adacomp_decompress_accumulate_multi")
+
+
+def adacomp_set_device(device: int) -> None:
+    """Select the calling thread's CUDA device inside the library (see include/adacomp.h)."""
+    _check(lib().adacomp_set_device(int(device)), "adacomp_set_device")
 
 
 def adacomp_device_status(stream=None) -> int:

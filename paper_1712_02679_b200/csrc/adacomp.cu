@@ -2586,6 +2586,11 @@ int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_st
     return ADACOMP_OK;
 }
 
+int adacomp_set_device(int device)
+{
+    return cudaSetDevice(device) == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+}
+
 int adacomp_device_status(uint32_t *host_out, void *stream)
 {
     if (!host_out) return ADACOMP_ERR_NULL;
