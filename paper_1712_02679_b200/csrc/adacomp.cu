@@ -55,18 +55,27 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: bound of every device
 __device__ u32 g_status;             // sticky ADACOMP_DEV_* bits of this device
 
 #ifdef ADACOMP_PHASE_CLOCKS
-// Development aid (not part of the ABI): cycles spent by one thread of one CTA in each phase.
+// Development aid (not part of the ABI): cycles spent by one decoding thread and by the producer's
+// first lane of one CTA in each phase, kept in registers and written out once at the end.
 __device__ unsigned long long g_phase_clocks[16];
+#define PHASE_DECL unsigned long long pc_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
 #define PHASE_CLOCK(i, t0)                                                              \
     do {                                                                               \
-        if (blockIdx.x == 3 && threadIdx.x == 32) {                                    \
-            const long long now_ = clock64();                                          \
-            g_phase_clocks[i] += (unsigned long long)(now_ - (t0));                    \
-            (t0) = now_;                                                               \
-        }                                                                              \
+        const long long now_ = clock64();                                              \
+        pc_[i] += (unsigned long long)(now_ - (t0));                                   \
+        (t0) = now_;                                                                   \
+    } while (0)
+#define PHASE_CLOCK_P(i, t0) PHASE_CLOCK(i, t0)
+#define PHASE_FLUSH(thread, lo, hi)                                                     \
+    do {                                                                               \
+        if (blockIdx.x == 3 && threadIdx.x == (thread))                                \
+            for (int i_ = (lo); i_ < (hi); i_++) g_phase_clocks[i_] += pc_[i_];        \
     } while (0)
 #else
+#define PHASE_DECL do { } while (0)
 #define PHASE_CLOCK(i, t0) do { } while (0)
+#define PHASE_CLOCK_P(i, t0) do { } while (0)
+#define PHASE_FLUSH(thread, lo, hi) do { } while (0)
 #endif
 
 __host__ __device__ inline u64 align_up(u64 x, u64 a) { return (x + a - 1) / a * a; }
@@ -239,6 +248,11 @@ __device__ inline bool mbar_try_wait(u64 *bar, u32 parity)
         : "r"(smem_addr(bar)), "r"(parity)
         : "memory");
     return ok != 0;
+}
+
+__device__ inline void mbar_arrive(u64 *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
 // Bounded wait: false if the phase did not complete within kWaitCycles.
@@ -1105,25 +1119,28 @@ constexpr int kWbufBytes = 8192;     // staged words of one round of learners (o
 constexpr int kRoundMax = 4;         // learners per round
 constexpr int kGenericSegBins = 1024;   // generic decode: bins scanned per pass
 
-constexpr u32 kPipeStageBytes = 8192 + 512;     // staged words + bin counts of one tile
-constexpr int kConsumers = 128;                 // threads of warps 0-3
+// shared memory of the warp path (described with decode_warps below)
+#ifndef ADACOMP_WARPS_PER_SM
+#define ADACOMP_WARPS_PER_SM 6
+#endif
+constexpr int kWarpsPerSm = ADACOMP_WARPS_PER_SM;    // CTAs of the warp decoder per SM
+constexpr int kSlots = 8;                       // tiles in flight per CTA at most
+constexpr u32 kRingBytes = 19200;
+constexpr u32 kSlotMax = kRingBytes / 2;        // a slot never takes more: two tiles are always in flight
 
-struct PipePlan {                               // where a tile's data sits in its stage
-    unsigned short woff[ADACOMP_MAX_STREAMS];   // stage byte offset of learner l's first word
-    unsigned short coff[ADACOMP_MAX_STREAMS];   // stage byte offset of its bin counts
-    unsigned short cnt[ADACOMP_MAX_STREAMS];    // its words in this tile (at most 4096)
-    u32 kf;                                     // learners [0, kf) were fetched into the stage
-    u32 bad;                                    // directory entries that failed their checks
+struct WarpDecSmem {
+    uint4 ring[kRingBytes / 16];
+    u32 tmp[4][32];                             // per decoding warp: output places of its non-empty bins
+    unsigned short coff[ADACOMP_MAX_STREAMS];   // byte offset in a slot of learner l's bin counts (its words follow them)
+    unsigned short wcap[ADACOMP_MAX_STREAMS];   // bytes of its word region
+    u64 full[kSlots], empty[kSlots];            // mbarriers of the slots
+    u32 slot_bytes, n_slots, kf, abort;         // kf: learners [0, kf) have a region
 };
 
-struct PipeSmem {
-    uint4 stage[2][kPipeStageBytes / 16];
-    PipePlan plan[2];
-    unsigned short pre[kRoundMax][kSmallBins + 1];      // exclusive word offsets of the bins, per learner of a group
-    unsigned short pre0[2][kRoundMax][kSmallBins + 1];  // the same for the first group of each stage, made by the producer
-    u64 full[2], empty[2], ready[2];            // mbarriers of the two stages
-    u32 abort;
-};
+// A slot starts with {u32 staged, u32 bad} (learners [0, staged) of this tile are in the slot;
+// failed directory checks), 8 bytes of padding, then u16 cnt[k8] and u16 head[k8]: words of the
+// learner in this tile and the byte offset of the first one in its word region.
+constexpr u32 kSlotHead = 16;
 
 struct DecodeSmem {
     float acc[kDecodeChunk];                    // the output tile
@@ -1139,7 +1156,6 @@ struct DecodeSmem {
             u64 off0[ADACOMP_MAX_STREAMS];      // first word of this tile in stream l
             u32 cnt[ADACOMP_MAX_STREAMS];       // words of this tile in stream l
         } f;
-        PipeSmem pipe;                          // pipelined path
     };
     u64 n_sel[ADACOMP_MAX_STREAMS];             // words in stream l
     float scale[ADACOMP_MAX_STREAMS];
@@ -1368,109 +1384,298 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
 }
 
 // ---------------------------------------------------------------------------------
-// decode, pipelined path: tiles of 2..96 bins whose bin-count run is a multiple of 16 bytes
+// decode, warp path: tiles of 4..96 bins whose bin-count run is a multiple of 16 bytes
 // (L_T = 50 and 500 among them).
 //
-// Warp 4 is a producer: for every tile of this CTA it reads the k directory entries (one lane
-// per learner, one tile ahead), lays the learners' bin counts and words out in one of two
-// shared-memory stages and starts the bulk copies (TMA, no multicast); it runs up to two tiles
-// ahead of the consumers and never touches the output.  Warps 0-3 are consumers: they wait for
-// the stage, turn the bin counts into word offsets, add the words into the output tile and
-// store it.  G threads share a bin (G = 1 for more than 64 bins, up to 32 for few bins); a
-// bin's G threads sit in one warp, so the learners' contributions to an element stay in learner
-// order with a __syncwarp() between learners.  The consumers meet at two named barriers per
-// tile; producer and consumers meet only through the stages' full / empty mbarriers, and every
-// wait on those is bounded.
+// Warp 4 is a loader: for every tile of this CTA, lane l reads learner l's two directory
+// entries (two tiles ahead) and bulk-copies (TMA, no multicast) that learner's bin counts and
+// words of the tile into the learner's fixed region of a shared-memory slot; the slots form a
+// ring of up to kSlots tiles in flight.  Region sizes are set once per launch from the streams'
+// word totals (1.5 times a tile's average plus slack); a learner whose words of some tile do not
+// fit its region, and every learner for which the slot has no region, is read by the decoding
+// warps straight from global memory for that tile.
+//
+// Warps 0-3 decode.  Each owns a quarter of the tile's bins and of the output tile and never
+// touches the rest, so the four need no barrier among themselves: a warp waits for the slot,
+// adds its words learner by learner (one __syncwarp() between learners keeps an element's
+// contributions in learner order), gives the slot back and stores its quarter.  Within a
+// learner the warp works by word, not by bin: lane j takes word j of the warp's run of words, 32
+// at a time.  The bin of a word comes from the bin counts: the lanes that hold the warp's bins
+// (at most 24) scan their counts, raise a flag bit at the position of each non-empty bin's first
+// word, and a word's bin is the number of flags at or before it (a population count), mapped to
+// the bin's place in the output tile by one shuffle.
+// Loader and decoding warps meet only through the slots' full / empty mbarriers, and every wait
+// on those is bounded.
 // ---------------------------------------------------------------------------------
 
-__device__ inline void mbar_arrive(u64 *bar)
+template <typename Word, bool SHARED>
+__device__ inline u32 load_word(u64 addr)
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+    u32 v;
+    if (SHARED) {
+        if (sizeof(Word) == 1) asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"((u32)addr) : "memory");
+        else asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"((u32)addr) : "memory");
+    } else {
+        if (sizeof(Word) == 1) asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+        else asm volatile("ld.global.nc.u16 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
+    }
+    return v;
 }
 
-// Adds the words [0, c) at p (one learner's words of one bin) into the bin's 'mine' elements;
-// threads r, r + G, ... of the bin's G threads take every G-th word.  `seen` collects the ternary
-// codes met and `mx` the largest index, checked by the caller.
-// A thread that owns its bin alone (G == 1) handles words four at a time: a learner sends an
-// element at most once, so the four read-modify-writes are independent and their shared-memory
-// latencies overlap (slots past the end carry the no-op word 0).  With G > 1 a thread rarely has
-// more than one word, so it takes them singly.
-template <typename Word>
-__device__ inline void add_words(const Word *p, u32 c, int r, int G, u32 sbits, float *mine, u32 L_T,
-                                 u32 &seen, u32 &mx)
+// out[e] += v (fp32, round to nearest even, denormals kept) for a word that carries a value
+// (bit 0 set) and an index inside its bin (word < 4 L_T); nothing is read or written otherwise.
+__device__ inline void add_at_if_valid(u32 e, float v, u32 word, u32 LT4)
 {
-    if (G > 1) {
-        for (u32 j = r; j < c; j += (u32)G) {
-            const u32 word = p[j];
-            const u32 idx = word >> 2;
-            mx = max(mx, idx);
-            seen |= 1u << (word & 3u);
-            const u32 e = sizeof(Word) == 1 ? idx : min(idx, L_T - 1u);
-            if (word & 1u) mine[e] = __fadd_rn(mine[e], __uint_as_float(sbits ^ ((word & 2u) << 30)));
-        }
-        return;
-    }
-    constexpr int kBatch = 4;
-    for (u32 j0 = 0; j0 < c; j0 += kBatch) {
-        u32 word[kBatch], e[kBatch];
-        float v[kBatch];
-#pragma unroll
-        for (int i = 0; i < kBatch; i++) word[i] = j0 + i < c ? (u32)p[j0 + i] : 0u;
-#pragma unroll
-        for (int i = 0; i < kBatch; i++) {
-            const u32 idx = word[i] >> 2;
-            mx = max(mx, idx);
-            e[i] = sizeof(Word) == 1 ? idx : min(idx, L_T - 1u);      // 8-bit indices cannot leave the tile
-            v[i] = mine[e[i]];
-        }
-#pragma unroll
-        for (int i = 0; i < kBatch; i++) {
-            if (j0 + i < c) seen |= 1u << (word[i] & 3u);
-            if (word[i] & 1u) mine[e[i]] = __fadd_rn(v[i], __uint_as_float(sbits ^ ((word[i] & 2u) << 30)));
-        }
-    }
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t.reg .f32 x;\n\t"
+        "and.b32 t, %2, 1;\n\t"
+        "setp.ne.u32 p, t, 0;\n\t"
+        "setp.lt.and.u32 p, %2, %3, p;\n\t"
+        "@p ld.shared.f32 x, [%0];\n\t"
+        "@p add.rn.f32 x, x, %1;\n\t"
+        "@p st.shared.f32 [%0], x;\n\t}"
+        ::"r"(e), "f"(v), "r"(word), "r"(LT4)
+        : "memory");
 }
 
-// Exclusive word offsets of bins 0..TB (TB <= 96) of up to four learners, written to pre[q][0..TB].
-// count(q, b) returns learner q's count of bin b.  Called by the warps that own bins (whole warps);
-// two 16-bit counts share a scan, and each warp adds up the bins of the warps before it itself.
-template <typename CountFn>
-__device__ inline void bin_offsets(CountFn count, int R, int TB, int tid, unsigned short (*pre)[kSmallBins + 1])
+// A group of up to four learners, as the decoding warp holds it: lane q (q < 4) has learner q's
+// addresses of its bin counts and first word of this tile, the words the directory gives it in
+// this tile, and its scale's bits; the other lanes get them by shuffle.
+template <typename Addr>
+struct GroupSrc {
+    Addr counts, words;
+    u32 limit, sbits;
+};
+__device__ inline u32 bcast(u32 v, int q) { return __shfl_sync(0xffffffffu, v, q); }
+__device__ inline u64 bcast(u64 v, int q)
 {
-    const int lane = tid & 31, warp = tid >> 5;
-    u32 c[kRoundMax];
+    return ((u64)__shfl_sync(0xffffffffu, (u32)(v >> 32), q) << 32) | __shfl_sync(0xffffffffu, (u32)v, q);
+}
+
+// 1 << d for d < 32, else 0 (PTX shifts clamp at the register width).
+__device__ inline u32 shl_clamped(u32 d)
+{
+    u32 r;
+    asm("shl.b32 %0, 1, %1;" : "=r"(r) : "r"(d));
+    return r;
+}
+
+// The warp's view of up to four learners' bin counts of one tile.  Two learners share a register
+// (16 bits each: a tile has at most 4096 words), so one scan and one reduction serve two
+// learners.  For learner q (field q & 1 of register q >> 1): `bef` = words of the tile in bins ahead
+// of the warp's (the same in every lane); lane i holds in `mine` the count of the warp's bin i
+// and in `ex` the words of the warp's bins ahead of it; `tot` = words of the warp's bins together.
+struct WarpBins {
+    u32 mine[2], ex[2], bef[2], tot[2];
+};
+__device__ inline u32 field(const u32 *x, int q) { return (x[q >> 1] >> (16 * (q & 1))) & 0xffffu; }
+
+//   counts(q)  address of learner q's bin counts of this tile (bin 0 of the tile)
+//   b0, nb     the warp's bins are [b0, b0 + nb) of the tile; `live` of the tile's bins exist
+template <typename Word, bool SHARED, typename CountsFn>
+__device__ inline void warp_bins(CountsFn counts, int R, int b0, int nb, u32 live, u32 L_T, int lane, WarpBins &wb)
+{
+    constexpr u32 full = 0xffffffffu;
+    u32 bef[2] = {0u, 0u};
+    wb.mine[0] = wb.mine[1] = 0u;
+    const u32 mb = (u32)(b0 + lane);
+    const bool have = lane < nb && mb < live;
 #pragma unroll
-    for (int q = 0; q < kRoundMax; q++) c[q] = (q < R && tid < TB) ? count(q, tid) : 0u;
-    u32 pair[2] = {c[0] | (c[1] << 16), c[2] | (c[3] << 16)};
-    u32 basep[2] = {0u, 0u};
-    for (int wv = 0; wv < warp; wv++) {            // bins of the warps before this one
-        const int b = wv * 32 + lane;
-        u32 e[kRoundMax];
+    for (int q = 0; q < kRoundMax; q++) {
+        if (q < R) {
+            const auto at = counts(q);
+            u32 cq = 0, bq = 0;
+            if (have) cq = min(load_word<Word, SHARED>(at + mb * (u32)sizeof(Word)), L_T);
 #pragma unroll
-        for (int q = 0; q < kRoundMax; q++) e[q] = q < R ? count(q, b) : 0u;
-        basep[0] += e[0] | (e[1] << 16);
-        basep[1] += e[2] | (e[3] << 16);
+            for (int r = 0; r < 3; r++) {           // bins before b0: at most 72
+                const u32 b = (u32)lane + 32u * r;
+                if (b < (u32)b0 && b < live) bq += min(load_word<Word, SHARED>(at + b * (u32)sizeof(Word)), L_T);
+            }
+            wb.mine[q >> 1] |= cq << (16 * (q & 1));
+            bef[q >> 1] += bq << (16 * (q & 1));
+        }
     }
 #pragma unroll
     for (int h = 0; h < 2; h++) {
-        if (warp > 0)
-            for (int d = 16; d > 0; d >>= 1) basep[h] += __shfl_xor_sync(0xffffffffu, basep[h], d);
-        const u32 inc = warp_inclusive_scan(pair[h], lane);
-        const u32 excl = basep[h] + inc - pair[h];
-        if (tid < TB) {
-            pre[2 * h][tid] = (unsigned short)(excl & 0xffffu);
-            pre[2 * h + 1][tid] = (unsigned short)(excl >> 16);
-            if (tid == TB - 1) {
-                pre[2 * h][TB] = (unsigned short)((excl + pair[h]) & 0xffffu);
-                pre[2 * h + 1][TB] = (unsigned short)((excl + pair[h]) >> 16);
-            }
+        wb.ex[h] = wb.bef[h] = wb.tot[h] = 0u;
+        if (2 * h < R) {
+            wb.bef[h] = b0 > 0 ? __reduce_add_sync(full, bef[h]) : 0u;
+            const u32 incl = warp_inclusive_scan(wb.mine[h], lane);
+            wb.ex[h] = incl - wb.mine[h];
+            wb.tot[h] = __shfl_sync(full, incl, 31);
         }
     }
 }
 
+// One learner's words of one warp's bins, added into the warp's part of the output tile.
+//   words    address of the first of them (word `before` of the learner's words of this tile)
+//   W, c, excl  as WarpBins gives them for this learner
+//   acc_at   shared-memory address of the first output element of the warp's first bin
+//   tmp      32 words of scratch of this warp
+// SHARED: `words` is a shared-memory address (a slot), else a global one.
+// Returns the ADACOMP_DEV_* bits of what was wrong with the data.
+template <typename Word, bool SHARED, typename Addr>
+__device__ inline u32 warp_add_words(Addr words, u32 W, u32 c, u32 excl, int nb, u32 L_T, u32 sbits, u32 acc_at,
+                                     u32 *tmp, int lane)
+{
+    constexpr u32 full = 0xffffffffu;
+    if (W == 0) return 0;
+    // ---- the output place of the r-th non-empty bin, held by lane r ----
+    const u32 LT4 = L_T * 4u;
+    u32 place = acc_at + (u32)lane * LT4;
+    const u32 ne = __ballot_sync(full, c != 0u);
+    if (ne != (1u << nb) - 1u) {                    // (nb <= 24)
+        __syncwarp();
+        if (c != 0u) tmp[__popc(ne & ((1u << lane) - 1u))] = place;
+        __syncwarp();
+        place = tmp[lane];
+    }
+
+    // ---- the words, 32 at a time: lane j takes word j0 + j ----
+    const u32 le_mask = (2u << lane) - 1u;
+    Addr wp = words + (Addr)((u32)lane * (u32)sizeof(Word));
+    u32 d = c != 0u ? excl : 0x80000000u;           // distance from j0 to the first word of my bin (none: far away)
+    u32 left = W - min(W, (u32)lane);               // words at or after mine
+    int rbase = -1;
+    u32 mx = 0, rsv = 0;
+    for (u32 j0 = 0; j0 < W; j0 += 32u) {
+        const u32 m = __reduce_or_sync(full, shl_clamped(d));         // first words of bins in this chunk
+        d -= 32u;
+        const int r = rbase + __popc(m & le_mask);
+        rbase += __popc(m);
+        const u32 bin_at = __shfl_sync(full, place, r);
+        u32 word = 0;
+        if (left != 0u) word = load_word<Word, SHARED>(wp);
+        left -= min(left, 32u);
+        wp += (Addr)(32u * (u32)sizeof(Word));
+        mx = max(mx, word);
+        rsv |= (word >> 1) & ~word;
+        // 4 * idx is the element's byte offset in its bin
+        add_at_if_valid(bin_at + (word & ~3u), __uint_as_float(sbits ^ ((word << 30) & 0x80000000u)), word, LT4);
+    }
+    u32 bad = 0;
+    if (__any_sync(full, (rsv & 1u) != 0u)) bad |= ADACOMP_DEV_RESERVED_CODE;
+    if (__any_sync(full, mx >= LT4)) bad |= ADACOMP_DEV_BAD_STREAM;
+    return bad;
+}
+
+// Up to four learners (a group, in learner order) of one warp's bins of one tile, by word.
+template <typename Word, bool SHARED, typename Addr>
+__device__ inline u32 warp_add_group(const GroupSrc<Addr> &src, int R, int b0, int nb, u32 live, u32 L_T, u32 acc_at,
+                                     u32 *tmp, int lane)
+{
+    WarpBins wb;
+    warp_bins<Word, SHARED>([&](int q) { return bcast(src.counts, q); }, R, b0, nb, live, L_T, lane, wb);
+    u32 bad = 0;
+#pragma unroll
+    for (int q = 0; q < kRoundMax; q++) {
+        if (q >= R) break;
+        const Addr words = bcast(src.words, q);
+        const u32 limit = bcast(src.limit, q), sbits = bcast(src.sbits, q);
+        const u32 before = field(wb.bef, q), W = field(wb.tot, q);
+        if (before + W > limit) {
+            bad |= ADACOMP_DEV_BAD_STREAM;          // counts and directory disagree: nothing is read
+        } else {
+            bad |= warp_add_words<Word, SHARED, Addr>(words + (Addr)(before * (u32)sizeof(Word)), W, field(wb.mine, q),
+                                                      field(wb.ex, q), nb, L_T, sbits, acc_at, tmp, lane);
+        }
+        __syncwarp();                               // learner order, element by element
+    }
+    return bad;
+}
+
+// Tiles of at most 64 bins: G = 32 / (a warp's bins, rounded up to a power of two) lanes share a
+// bin.  For a group of up to four learners (in learner order) every lane gets its bin's count and
+// the words of the tile ahead of that bin from two warp scans over the tile's bin counts (lane j
+// holds bins j and j + 32; two learners share a register, 16 bits each), then the bin's lanes
+// take every G-th word of the bin.
+//   bin      the lane's bin in the tile (>= TB: the lane has none), r its place among the bin's G lanes
+//   mine_at  shared-memory address of the bin's first output element
+template <typename Word, bool SHARED, typename Addr>
+__device__ inline u32 warp_add_group_by_bin(const GroupSrc<Addr> &src, int R, int TB, u32 live, u32 L_T, int bin, int r,
+                                            int G, u32 mine_at, int lane)
+{
+    constexpr u32 full = 0xffffffffu;
+    const u32 LT4 = L_T * 4u;
+    // ---- packed bin counts of the tile: lo = bin `lane`, hi = bin `lane + 32` ----
+    u32 lo[2] = {0u, 0u}, hi[2] = {0u, 0u};
+#pragma unroll
+    for (int q = 0; q < kRoundMax; q++) {
+        if (q < R) {
+            const Addr counts = bcast(src.counts, q);
+            if ((u32)lane < live) lo[q >> 1] |= min(load_word<Word, SHARED>(counts + (Addr)((u32)lane * (u32)sizeof(Word))), L_T) << (16 * (q & 1));
+            if (TB > 32 && (u32)lane + 32u < live)
+                hi[q >> 1] |= min(load_word<Word, SHARED>(counts + (Addr)(((u32)lane + 32u) * (u32)sizeof(Word))), L_T) << (16 * (q & 1));
+        }
+    }
+    // ---- per learner pair: words ahead of my bin, words of my bin, words of the tile ----
+    u32 ex[2] = {0u, 0u}, cm[2] = {0u, 0u}, tot[2] = {0u, 0u};
+    const int bsrc = bin & 31;
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+        if (2 * h < R) {
+            const u32 il = warp_inclusive_scan(lo[h], lane);
+            u32 t = __shfl_sync(full, il, 31);
+            u32 e = __shfl_sync(full, il - lo[h], bsrc), c = __shfl_sync(full, lo[h], bsrc);
+            if (TB > 32) {
+                const u32 ih = warp_inclusive_scan(hi[h], lane) + t;
+                const u32 e2 = __shfl_sync(full, ih - hi[h], bsrc), c2 = __shfl_sync(full, hi[h], bsrc);
+                t = __shfl_sync(full, ih, 31);
+                if (bin >= 32) {
+                    e = e2;
+                    c = c2;
+                }
+            }
+            ex[h] = e;
+            cm[h] = bin < TB ? c : 0u;
+            tot[h] = t;
+        }
+    }
+    // ---- the words ----
+    u32 bad = 0, mx = 0, rsv = 0;
+#pragma unroll
+    for (int q = 0; q < kRoundMax; q++) {
+        if (q >= R) break;
+        const Addr words = bcast(src.words, q);
+        const u32 limit = bcast(src.limit, q), sbits = bcast(src.sbits, q);
+        if (field(tot, q) > limit) {
+            bad |= ADACOMP_DEV_BAD_STREAM;          // counts and directory disagree: nothing is read
+        } else {
+            const u32 c = field(cm, q);
+            Addr wp = words + (Addr)((field(ex, q) + (u32)r) * (u32)sizeof(Word));
+            for (u32 j = (u32)r; j < c; j += (u32)G) {
+                const u32 word = load_word<Word, SHARED>(wp);
+                wp += (Addr)((u32)G * (u32)sizeof(Word));
+                mx = max(mx, word);
+                rsv |= (word >> 1) & ~word;
+                add_at_if_valid(mine_at + (word & ~3u), __uint_as_float(sbits ^ ((word << 30) & 0x80000000u)), word, LT4);
+            }
+        }
+        __syncwarp();                               // learner order, element by element
+    }
+    if (__any_sync(full, (rsv & 1u) != 0u)) bad |= ADACOMP_DEV_RESERVED_CODE;
+    if (__any_sync(full, mx >= LT4)) bad |= ADACOMP_DEV_BAD_STREAM;
+    return bad;
+}
+
+// The same for learners read from global memory: rare, so kept out of line (the decoding warps'
+// registers go to the path that reads the slots).
 template <typename Word>
-__device__ void decode_pipelined(const DecodeArgs &a, const Geometry &geo, float *s_acc, PipeSmem &ps,
-                                 const float *s_scale, const u64 *s_nsel)
+__device__ __noinline__ u32 warp_add_group_by_bin_global(GroupSrc<u64> src, int R, int TB, u32 live, u32 L_T, int bin, int r,
+                                                         int G, u32 mine_at, int lane)
+{
+    return warp_add_group_by_bin<Word, false, u64>(src, R, TB, live, L_T, bin, r, G, mine_at, lane);
+}
+template <typename Word>
+__device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int b0, int nb, u32 live, u32 L_T, u32 acc_at,
+                                                  u32 *tmp, int lane)
+{
+    return warp_add_group<Word, false, u64>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
+}
+
+template <typename Word>
+__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+                             const float *s_scale, const u64 *s_nsel)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
@@ -1478,297 +1683,277 @@ __device__ void decode_pipelined(const DecodeArgs &a, const Geometry &geo, float
     const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
     const u64 first = blockIdx.x, stride = gridDim.x;
     const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
+    const u32 k8 = (a.k + 7u) & ~7u;
+    const u32 meta_bytes = kSlotHead + 4u * k8;                    // slot header + cnt[k8] + head[k8]
+    unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
+    constexpr u32 full_mask = 0xffffffffu;
 
     if (tid == 0) {
-        mbar_init(&ps.full[0], 1);
-        mbar_init(&ps.full[1], 1);
-        mbar_init(&ps.empty[0], 1);
-        mbar_init(&ps.empty[1], 1);
-        mbar_init(&ps.ready[0], 1);
-        mbar_init(&ps.ready[1], 1);
-        ps.abort = 0;
+        for (int s = 0; s < kSlots; s++) {
+            mbar_init(&ws.full[s], 32);         // every lane of the loader arrives, with or without bytes to expect
+            mbar_init(&ws.empty[s], 4);         // every decoding warp arrives
+        }
+        ws.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
+    if (warp == 4) {
+        // the learners' regions of a slot: counts, then room for 1.5 times a tile's average words + slack
+        u32 used = meta_bytes, kf = 0;
+        bool open = true;
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            const u32 l = (u32)lane + 32u * h;
+            const bool active = l < a.k;
+            u32 wbytes = 0;
+            if (active) {
+                const u64 avg = s_nsel[l] / geo.n_tiles;
+                const u64 cap = min((u64)geo.tile_elems, avg + avg / 2 + 64);
+                wbytes = (u32)align_up(cap * sizeof(Word) + 16, 16);
+            }
+            const u32 need = active ? count_bytes + wbytes : 0u;
+            const u32 incl = used + warp_inclusive_scan(need, lane);
+            const u32 fits = __ballot_sync(full_mask, active && open && incl <= kSlotMax);
+            const int lead = __ffs(~fits) - 1;
+            const int staged_lanes = lead < 0 ? 32 : lead;
+            if (active) {
+                ws.coff[l] = (unsigned short)(incl - need);
+                ws.wcap[l] = (unsigned short)wbytes;
+            }
+            kf += (u32)staged_lanes;
+            if (staged_lanes > 0) used = __shfl_sync(full_mask, incl, staged_lanes - 1);
+            if (staged_lanes < 32) open = false;
+        }
+        if (lane == 0) {
+            ws.kf = kf;
+            ws.slot_bytes = used;
+            ws.n_slots = max(1u, min((u32)kSlots, kRingBytes / used));     // (kf == 0: one slot of headers only)
+        }
+    }
     __syncthreads();
+    const u32 kf = ws.kf, slot_bytes = ws.slot_bytes, S = ws.n_slots;
 
     if (warp == 4) {
-        // =============================== producer warp ===============================
-        // lane l looks after learners l and l + 32
-        u64 d0[2] = {0, 0}, d1[2] = {0, 0};
-        auto load_dir = [&](u64 it) {
-            const u64 tile = first + it * stride;
+        // ================================ loader warp ================================
+        u64 da0[2] = {0, 0}, da1[2] = {0, 0}, db0[2] = {0, 0}, db1[2] = {0, 0};
+        auto load_dir = [&](u64 t, u64 *d0, u64 *d1) {
+            const u64 tile = first + t * stride;
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const u32 l = (u32)lane + 32u * h;
-                if (l < a.k && it < my_tiles) {
+                if (l < kf && t < my_tiles) {
                     const u64 *dir = reinterpret_cast<const u64 *>(a.stream[l] + geo.tile_off_at);
                     d0[h] = dir[tile];
                     d1[h] = dir[tile + 1];
                 }
             }
         };
-        load_dir(0);
+        load_dir(0, da0, da1);
+        load_dir(1, db0, db1);
+        u32 my_coff[2], my_wcap[2];
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            const u32 l = (u32)lane + 32u * h;
+            my_coff[h] = l < kf ? ws.coff[l] : 0u;
+            my_wcap[h] = l < kf ? ws.wcap[l] : 0u;
+        }
         u64 issued = 0;                 // copies were started for tiles [0, issued)
-        for (u64 it = 0; it < my_tiles; it++) {
-            const int s = (int)(it & 1);
-            const u64 tile = first + it * stride;
-            const u64 c0[2] = {d0[0], d0[1]}, c1[2] = {d1[0], d1[1]};
-            load_dir(it + 1);                       // next tile's entries travel while this one is laid out
-            if (it >= 2 && !mbar_wait(&ps.empty[s], (u32)((it >> 1) - 1) & 1u)) {
-                ps.abort = 1;
+        PHASE_DECL;
+        long long tp = clock64();
+        // (no division by S in the loops: slot and use count step along with the tile)
+        u32 s = 0, use = 0;             // the tile's slot; how many times the slot was used before
+        u64 tile = first;
+        for (u64 it = 0; it < my_tiles; it++, tile += stride, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
+            PHASE_CLOCK(9, tp);
+            if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
+                ws.abort = 1;
                 raise_status(ADACOMP_DEV_TIMEOUT);
-                break;                              // the consumers time out on the full barrier in turn
+                break;                  // the decoding warps time out on the full barrier in turn
             }
-            if (*reinterpret_cast<volatile u32 *>(&ps.abort)) break;
-            PipePlan &pl = ps.plan[s];
-            unsigned char *st = reinterpret_cast<unsigned char *>(ps.stage[s]);
+            if (*reinterpret_cast<volatile u32 *>(&ws.abort)) break;
+            PHASE_CLOCK(7, tp);
+            unsigned char *sl = ring + s * slot_bytes;
             const u64 bin0 = tile * (u64)TB;
             const u64 bins_left = geo.n_bins - bin0;
-            const u32 cbytes = bins_left >= (u64)TB ? count_bytes
-                                                    : (u32)align_up(bins_left * sizeof(Word), 16);   // last tile
-            u32 used = 0, kf = 0, total = 0, bad = 0;
-            bool open = true;               // learners are staged as a prefix: once one does not fit, none after it is
+            const u32 cbytes = bins_left >= (u64)TB ? count_bytes : (u32)align_up(bins_left * sizeof(Word), 16);   // last tile
+            unsigned short *m_cnt = reinterpret_cast<unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
+            u64 src[2] = {0, 0};
+            u32 wbytes[2] = {0, 0};
+            u32 staged = 0, bad = 0;
+            bool open = true;
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const u32 l = (u32)lane + 32u * h;
-                const bool active = l < a.k;
-                bool ok = true;
-                u32 cnt = 0, head = 0, wbytes = 0;
+                const bool active = l < kf;
+                bool ok = true, fit = false;
                 if (active) {
-                    ok = c1[h] >= c0[h] && c1[h] - c0[h] <= geo.tile_elems && c1[h] <= s_nsel[l];
-                    cnt = ok ? (u32)(c1[h] - c0[h]) : 0u;
-                    const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + c0[h] * sizeof(Word);
-                    head = (u32)(src & 15u);
-                    wbytes = cnt ? (u32)align_up(head + cnt * sizeof(Word), 16) : 0u;
-                    pl.cnt[l] = (unsigned short)cnt;
+                    ok = da1[h] >= da0[h] && da1[h] - da0[h] <= geo.tile_elems && da1[h] <= s_nsel[l];
+                    const u32 cnt = ok ? (u32)(da1[h] - da0[h]) : 0u;
+                    src[h] = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + da0[h] * sizeof(Word);
+                    const u32 head = (u32)(src[h] & 15u);
+                    wbytes[h] = cnt ? (u32)align_up(head + cnt * sizeof(Word), 16) : 0u;
+                    fit = wbytes[h] <= my_wcap[h];
+                    m_cnt[l] = (unsigned short)cnt;
+                    m_head[l] = (unsigned short)head;
                 }
-                if (__any_sync(0xffffffffu, active && !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
-                const u32 need = active ? count_bytes + wbytes : 0u;
-                const u32 incl = used + warp_inclusive_scan(need, lane);
-                const u32 fits = __ballot_sync(0xffffffffu, active && open && incl <= kPipeStageBytes);
-                const int lead = __ffs(~fits) - 1;                  // first lane that is not staged
+                if (__any_sync(full_mask, active && !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
+                const u32 fits = __ballot_sync(full_mask, active && open && fit);
+                const int lead = __ffs(~fits) - 1;
                 const int staged_lanes = lead < 0 ? 32 : lead;
-                const bool staged = lane < staged_lanes;
-                if (staged) {
-                    pl.coff[l] = (unsigned short)(incl - need);
-                    pl.woff[l] = (unsigned short)(incl - need + count_bytes + head);
-                }
-                u32 bytes = staged ? cbytes + wbytes : 0u;
-                for (int d = 16; d > 0; d >>= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, d);
-                total += bytes;
-                kf += (u32)staged_lanes;
-                if (staged_lanes > 0) used = __shfl_sync(0xffffffffu, incl, staged_lanes - 1);
+                staged += (u32)staged_lanes;
                 if (staged_lanes < 32) open = false;
+                if (kf <= 32u) break;
             }
-            __syncwarp();
             if (lane == 0) {
-                pl.kf = kf;
-                pl.bad = bad;
-                mbar_arrive_expect_tx(&ps.full[s], total);
+                reinterpret_cast<u32 *>(sl)[0] = staged;
+                reinterpret_cast<u32 *>(sl)[1] = bad;
             }
             __syncwarp();
+            u32 expect = 0;
+#pragma unroll
+            for (int h = 0; h < 2; h++)
+                if ((u32)lane + 32u * h < staged) expect += cbytes + wbytes[h];
+            if (expect) mbar_arrive_expect_tx(&ws.full[s], expect);
+            else mbar_arrive(&ws.full[s]);
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const u32 l = (u32)lane + 32u * h;
-                if (l < kf) {
-                    const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + c0[h] * sizeof(Word);
-                    const u32 head = (u32)(src & 15u);
-                    bulk_load(st + pl.coff[l], a.stream[l] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ps.full[s]);
-                    if (pl.cnt[l])
-                        bulk_load(st + pl.woff[l] - head, reinterpret_cast<const void *>(src & ~(u64)15u),
-                                  (u32)align_up(head + pl.cnt[l] * sizeof(Word), 16), &ps.full[s]);
+                if (l < staged) {
+                    bulk_load(sl + my_coff[h], a.stream[l] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ws.full[s]);
+                    if (wbytes[h])
+                        bulk_load(sl + my_coff[h] + count_bytes, reinterpret_cast<const void *>(src[h] & ~(u64)15u),
+                                  wbytes[h], &ws.full[s]);
                 }
             }
             issued = it + 1;
-
-            // ---- word offsets of the bins for the tile's first group of learners: done here, one
-            //      tile ahead of the decoding warps.  Lane i scans bins 3i .. 3i + 2. ----
-            if (!mbar_wait(&ps.full[s], (u32)(it >> 1) & 1u)) {
-                ps.abort = 1;
-                raise_status(ADACOMP_DEV_TIMEOUT);
-                break;
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                da0[h] = db0[h];
+                da1[h] = db1[h];
             }
-            {
-                const int R = (int)min((u32)kRoundMax, kf);
-                const u32 live_bins = (u32)min((u64)TB, bins_left);
-                u32 c[3][kRoundMax], sum[2] = {0u, 0u};
-#pragma unroll
-                for (int t = 0; t < 3; t++) {
-                    const u32 b = (u32)lane * 3u + t;
-#pragma unroll
-                    for (int q = 0; q < kRoundMax; q++)
-                        c[t][q] = (q < R && b < live_bins)
-                                      ? min((u32)reinterpret_cast<const Word *>(st + pl.coff[q])[b], L_T) : 0u;
-                    sum[0] += c[t][0] | (c[t][1] << 16);
-                    sum[1] += c[t][2] | (c[t][3] << 16);
-                }
-#pragma unroll
-                for (int hh = 0; hh < 2; hh++) {
-                    const u32 inc = warp_inclusive_scan(sum[hh], lane);
-                    u32 run = inc - sum[hh];
-#pragma unroll
-                    for (int t = 0; t < 3; t++) {
-                        const int b = lane * 3 + t;
-                        if (b <= TB) {
-                            ps.pre0[s][2 * hh][b] = (unsigned short)(run & 0xffffu);
-                            ps.pre0[s][2 * hh + 1][b] = (unsigned short)(run >> 16);
-                        }
-                        run += c[t][2 * hh] | (c[t][2 * hh + 1] << 16);
-                    }
-                    if (lane == 31 && TB == 96) {
-                        ps.pre0[s][2 * hh][96] = (unsigned short)(inc & 0xffffu);
-                        ps.pre0[s][2 * hh + 1][96] = (unsigned short)(inc >> 16);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ps.ready[s]);
-            }
+            load_dir(it + 2, db0, db1);
+            PHASE_CLOCK(8, tp);
         }
-        if (*reinterpret_cast<volatile u32 *>(&ps.abort)) {
+        PHASE_FLUSH(128, 7, 10);
+        if (*reinterpret_cast<volatile u32 *>(&ws.abort)) {
             // after a timeout the copies already started must land (or time out in turn) before
             // this CTA's shared memory is given back
-            for (u64 j = issued >= 2 ? issued - 2 : 0; j < issued; j++)
-                mbar_wait(&ps.full[j & 1], (u32)(j >> 1) & 1u);
+            for (u64 j = issued > S ? issued - S : 0; j < issued; j++) mbar_wait(&ws.full[j % S], (u32)(j / S) & 1u);    // (rare)
         }
         return;
     }
 
-    // ================================== consumers ==================================
-    int G = 1;
-    while (G < 32 && 2 * G * TB <= kConsumers) G *= 2;
-    const int my_bin = tid / G, my_r = tid % G;
-    const bool scatterer = my_bin < TB;
-    const bool scanner = tid < ((TB + 31) & ~31);
-    const bool whole_tiles = geo.tile_elems == 4000u;
+    // =============================== decoding warps ===============================
+    const int nb = TB / 4;                          // bins of a warp (tile_bins is a multiple of 4)
+    const int b0 = warp * nb;
+    const u32 quarter = (u32)nb * L_T;              // output elements of a warp
+    const u32 acc_at = smem_addr(s_acc) + (u32)warp * quarter * 4u;
+    float *const my_acc = s_acc + (u32)warp * quarter;
+    u32 *const tmp = ws.tmp[warp];
+    const bool vec_store = (quarter & 3u) == 0 && (geo.tile_elems & 3u) == 0;
+    // tiles of at most 64 bins: G lanes share a bin
+    const bool by_bin = sizeof(Word) == 2 || TB <= 64;     // (16-bit words: L_T >= 65, at most 60 bins)
+    int G = 32;
+    while (G * nb > 32) G >>= 1;
+    const int my_local = lane / G, my_r = lane % G;
+    const int my_bin = my_local < nb ? b0 + my_local : TB;
+    const u32 mine_at = smem_addr(s_acc) + (u32)my_bin * L_T * 4u;
     u32 bad = 0;
-    for (u64 it = 0; it < my_tiles; it++) {
-        const u64 tile = first + it * stride;
-        const u64 base = tile * (u64)geo.tile_elems;
+    PHASE_DECL;
+    u32 s = 0, use = 0;                             // the tile's slot; how many times the slot was used before
+    u64 tile = first;
+    for (u64 it = 0; it < my_tiles; it++, tile += stride, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
         const u64 bin0 = tile * (u64)TB;
-        const int s = (int)(it & 1);
-        const PipePlan &pl = ps.plan[s];
-        const unsigned char *st = reinterpret_cast<const unsigned char *>(ps.stage[s]);
-
+        const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
         long long t0 = clock64();
-        if (!mbar_wait(&ps.full[s], (u32)(it >> 1) & 1u)) {
-            ps.abort = 1;
+        if (!mbar_wait(&ws.full[s], use & 1u)) {
+            ws.abort = 1;
             bad |= ADACOMP_DEV_TIMEOUT;
-        }
-        if (!mbar_wait(&ps.ready[s], (u32)(it >> 1) & 1u)) {
-            ps.abort = 1;
-            bad |= ADACOMP_DEV_TIMEOUT;
+            break;
         }
         PHASE_CLOCK(0, t0);
-        const u32 kf = pl.kf;
-        if (tid == 0) bad |= pl.bad;
-        const u32 live_bins = (u32)min((u64)TB, geo.n_bins - bin0);
+        const unsigned char *sl = ring + s * slot_bytes;
+        const u32 staged = reinterpret_cast<const u32 *>(sl)[0];
+        if (warp == 0) bad |= reinterpret_cast<const u32 *>(sl)[1];
+        const unsigned short *m_cnt = reinterpret_cast<const unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
+        const u32 sl_at = smem_addr(sl);
 
-        // ---- the prefetched learners, four at a time ----
-        for (u32 g0 = 0; g0 < kf; g0 += kRoundMax) {
-            const int R = (int)min((u32)kRoundMax, kf - g0);
-            const unsigned short (*pre_of)[kSmallBins + 1] = g0 == 0 ? ps.pre0[s] : ps.pre;
-            if (g0 > 0 && scanner)      // (the first group's offsets were made by the producer warp)
-                bin_offsets([&](int q, int b) {
-                    return (u32)b < live_bins ? min((u32)reinterpret_cast<const Word *>(st + pl.coff[g0 + q])[b], L_T) : 0u;
-                }, R, TB, tid, ps.pre);
-            PHASE_CLOCK(1, t0);
-            consumer_barrier();     // offsets published; (first group) the previous tile is stored and zeroed
-            PHASE_CLOCK(2, t0);
-            if (scatterer) {
-                u32 seen = 0, mx = 0;
-                float *mine = s_acc + my_bin * L_T;
-                // everything the four learners need is read up front, so the loads overlap
-                u32 pre[kRoundMax], cq[kRoundMax], sb[kRoundMax];
-                const Word *wp[kRoundMax];
-#pragma unroll
-                for (int q = 0; q < kRoundMax; q++) {
-                    pre[q] = 0; cq[q] = 0; sb[q] = 0; wp[q] = nullptr;
-                    if (q < R) {
-                        const bool sane = pre_of[q][TB] <= pl.cnt[g0 + q];      // the same for every thread
-                        if (!sane) bad |= ADACOMP_DEV_BAD_STREAM;
-                        pre[q] = pre_of[q][my_bin];
-                        cq[q] = sane ? pre_of[q][my_bin + 1] - pre[q] : 0u;
-                        sb[q] = __float_as_uint(s_scale[g0 + q]);
-                        wp[q] = reinterpret_cast<const Word *>(st + pl.woff[g0 + q]) + pre[q];
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < kRoundMax; q++) {
-                    if (q >= R) break;
-                    add_words(wp[q], cq[q], my_r, G, sb[q], mine, L_T, seen, mx);
-                    if (G > 1) __syncwarp();       // the bin's threads share a warp: learner order kept
-                }
-                if (seen & 4u) bad |= ADACOMP_DEV_RESERVED_CODE;
-                if (mx >= L_T) bad |= ADACOMP_DEV_BAD_STREAM;
+        // ---- the learners whose words wait in the slot, four at a time ----
+        for (u32 g0 = 0; g0 < staged; g0 += kRoundMax) {
+            const int R = (int)min((u32)kRoundMax, staged - g0);
+            GroupSrc<u32> src = {0u, 0u, 0u, 0u};
+            if (lane < R) {
+                const u32 l = g0 + (u32)lane;
+                src.counts = sl_at + ws.coff[l];
+                src.words = src.counts + count_bytes + m_head[l];
+                src.limit = m_cnt[l];
+                src.sbits = __float_as_uint(s_scale[l]);
             }
-            PHASE_CLOCK(3, t0);
-            if (g0 + kRoundMax < kf) consumer_barrier();   // ps.pre is rewritten by the next group
+            if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+            else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
         }
+        if (lane == 0) mbar_arrive(&ws.empty[s]);   // (the group's last __syncwarp orders the warp's reads before it)
+        PHASE_CLOCK(1, t0);
 
-        // ---- learners that did not fit the stage: fetched and added one at a time ----
-        for (u32 l = kf; l < a.k; l++) {
-            consumer_barrier();                    // every reader of the stage is done
-            unsigned char *stw = reinterpret_cast<unsigned char *>(ps.stage[s]);
-            const u32 cnt = pl.cnt[l];
-            const u64 word0 = reinterpret_cast<const u64 *>(a.stream[l] + geo.tile_off_at)[tile];
-            const u64 src = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + word0 * sizeof(Word);
-            const u32 head = (u32)(src & 15u);
-            const u32 chunks = cnt ? (head + cnt * (u32)sizeof(Word) + 15u) / 16u : 0u;
-            for (u32 c = tid; c < chunks; c += kConsumers)
-                reinterpret_cast<uint4 *>(stw + count_bytes)[c] = __ldg(reinterpret_cast<const uint4 *>(src & ~(u64)15u) + c);
-            if (tid < TB)
-                reinterpret_cast<Word *>(stw)[tid] =
-                    (u32)tid < live_bins ? reinterpret_cast<const Word *>(a.stream[l] + geo.bin_cnt_at)[bin0 + tid] : (Word)0;
-            consumer_barrier();
-            if (scanner)
-                bin_offsets([&](int q, int b) {
-                    return (q == 0 && b < TB) ? min((u32)reinterpret_cast<const Word *>(stw)[b], L_T) : 0u;
-                }, 1, TB, tid, ps.pre);
-            consumer_barrier();
-            if (scatterer) {
-                if (ps.pre[0][TB] > cnt) {
-                    bad |= ADACOMP_DEV_BAD_STREAM;
-                } else {
-                    u32 seen = 0, mx = 0;
-                    const u32 pre = ps.pre[0][my_bin];
-                    add_words(reinterpret_cast<const Word *>(stw + count_bytes + head) + pre, ps.pre[0][my_bin + 1] - pre,
-                              my_r, G, __float_as_uint(s_scale[l]), s_acc + my_bin * L_T, L_T, seen, mx);
-                    if (seen & 4u) bad |= ADACOMP_DEV_RESERVED_CODE;
-                    if (mx >= L_T) bad |= ADACOMP_DEV_BAD_STREAM;
-                }
+        // ---- the others: read from global memory ----
+        for (u32 g0 = staged; g0 < a.k; g0 += kRoundMax) {
+            const int R = (int)min((u32)kRoundMax, a.k - g0);
+            GroupSrc<u64> src = {0ull, 0ull, 0u, 0u};
+            bool ok = true;
+            if (lane < R) {
+                const u32 l = g0 + (u32)lane;
+                const unsigned char *st = a.stream[l];
+                const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
+                const u64 w0 = dir[tile], w1 = dir[tile + 1];
+                ok = w1 >= w0 && w1 - w0 <= geo.tile_elems && w1 <= s_nsel[l];
+                src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
+                src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
+                src.limit = ok ? (u32)(w1 - w0) : 0u;
+                src.sbits = __float_as_uint(s_scale[l]);
             }
+            if (__any_sync(full_mask, !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
+            if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+            else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
         }
+        PHASE_CLOCK(2, t0);
 
-        consumer_barrier();                        // all words added; stage s and its plan are free
-        PHASE_CLOCK(4, t0);
-        const bool aborted = *reinterpret_cast<volatile u32 *>(&ps.abort) != 0;
-        if (tid == 0) mbar_arrive(&ps.empty[s]);
-        if (aborted) break;
-        // ---- store the tile (and leave it zeroed for the next one) ----
-        const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
-        if (whole_tiles && len == 4000u) {
-            float4 *o4 = reinterpret_cast<float4 *>(a.dst + base);
-            float4 *s4 = reinterpret_cast<float4 *>(s_acc);
+        // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
+        const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
+        const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
+        if (vec_store && len == quarter) {
+            // one bulk copy (TMA) takes the quarter from shared memory: the warp's own stores stay
+            // out of the way of everybody's shared-memory traffic
+            fence_async_smem();                     // this lane's adds, for the copy engine
+            __syncwarp();
+            if (lane == 0) {
+                bulk_store(a.dst + out0, my_acc, quarter * 4u);
+                bulk_commit();
+                bulk_wait_read_all();               // shared memory has been read: it can be zeroed
+            }
+            __syncwarp();
+            float4 *s4 = reinterpret_cast<float4 *>(my_acc);
             const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (quarter == 1000u) {
 #pragma unroll
-            for (int i = 0; i < 8; i++) {
-                const int at = tid + i * kConsumers;
-                if (i < 7 || at < 1000) {
-                    __stcs(o4 + at, s4[at]);
-                    s4[at] = zero;
-                }
+                for (int i = 0; i < 8; i++)
+                    if (i < 7 || lane < 26) s4[lane + 32 * i] = zero;
+            } else {
+                for (int at = lane; at < (int)(quarter >> 2); at += 32) s4[at] = zero;
             }
         } else {
-            store_tile(a.dst, base, len, s_acc);
+            for (u32 i = lane; i < quarter; i += 32) {
+                if (i < len) a.dst[out0 + i] = my_acc[i];
+                my_acc[i] = 0.f;
+            }
         }
-        PHASE_CLOCK(5, t0);
+        __syncwarp();                               // zeroed before the next tile's adds
+        PHASE_CLOCK(3, t0);
 #ifdef ADACOMP_PHASE_CLOCKS
-        if (blockIdx.x == 3 && threadIdx.x == 32) g_phase_clocks[6] += 1;
+        pc_[6] += 1;
 #endif
-        // (the next tile's first barrier orders this zeroing before its adds; every tile has one,
-        // because a single learner's words always fit the stage: kf >= 1)
     }
+    if (lane == 0) bulk_wait_all();                // the last copies leave shared memory before the CTA ends
+    PHASE_FLUSH(32, 0, 7);
     if (bad) raise_status(bad);
 }
 
@@ -1845,19 +2030,26 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
     }
 }
 
-__global__ void __launch_bounds__(kDecodeLaunch, 6)
-decode_sum(DecodeArgs a)
+// Tiles the warp path takes: 4..96 bins, a multiple of 4, bin-count runs that are a multiple of 16
+// bytes (so that everything a tile needs can be bulk-copied), at most 4096 elements.
+__host__ __device__ inline bool warp_path(const Geometry &g)
 {
-    __shared__ __align__(16) DecodeSmem sm;
-    __shared__ int s_bad;
+    return g.tile_bins >= 4u && g.tile_bins <= (u32)kSmallBins && g.tile_bins % 4u == 0 && (g.tile_bins * g.w) % 16u == 0 &&
+           g.tile_elems <= (u32)kDecodeChunk;
+}
 
-    // every CTA reads and cross-checks the k headers itself: the decision is uniform
+// Every CTA of a decode kernel reads and cross-checks the k headers itself: the decision is
+// uniform.  Returns false when this CTA has nothing to do (bad headers, raised by CTA 0; or a
+// CTA beyond the tensor's last work item); else the shape in L_T and n, and the streams' scales
+// and word totals in shared memory (behind a barrier).
+__device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_scale, u64 *s_nsel, u32 &L_T, u64 &n)
+{
     const u32 *h0 = reinterpret_cast<const u32 *>(a.stream[0]);
-    const u32 L_T = h0[2];
-    const u64 n = reinterpret_cast<const u64 *>(a.stream[0])[2];
-    // CTAs beyond the tensor's last work item have nothing to do (CTA 0 stays to report bad headers)
-    if (blockIdx.x > 0 && L_T >= 1u && L_T <= ADACOMP_MAX_L_T && blockIdx.x >= decode_items(n, L_T)) return;
-    if (threadIdx.x == 0) s_bad = a.hint_L_T != 0 && (a.hint_L_T != L_T || a.hint_n != n);
+    L_T = h0[2];
+    n = reinterpret_cast<const u64 *>(a.stream[0])[2];
+    // (CTA 0 stays to report bad headers)
+    if (blockIdx.x > 0 && L_T >= 1u && L_T <= ADACOMP_MAX_L_T && blockIdx.x >= decode_items(n, L_T)) return false;
+    if (threadIdx.x == 0) *s_bad = a.hint_L_T != 0 && (a.hint_L_T != L_T || a.hint_n != n);
     __syncthreads();
     if (threadIdx.x < a.k) {
         const u32 *h = reinterpret_cast<const u32 *>(a.stream[threadIdx.x]);
@@ -1869,28 +2061,50 @@ decode_sum(DecodeArgs a)
             ok = ((h[1] >> 16) & 0xffu) == g.w && h[3] == g.tile_bins && h64[3] == g.n_bins &&
                  h64[4] == g.n_tiles && h64[5] <= n;
         }
-        if (!ok) s_bad = 1;
+        if (!ok) *s_bad = 1;
+        s_scale[threadIdx.x] = __uint_as_float(h[12]);
+        s_nsel[threadIdx.x] = h64[5];
     }
     __syncthreads();
-    if (s_bad) {
+    if (*s_bad) {
         if (threadIdx.x == 0 && blockIdx.x == 0) raise_status(ADACOMP_DEV_HEADER_MISMATCH);
-        return;
+        return false;
     }
+    return true;
+}
+
+// The decoder is two kernels, so that each gets the registers its path needs: decode_sum_warps
+// takes the shapes of warp_path() and returns at once for any other, decode_sum the reverse.  A
+// caller that knows the shape launches the one that works; one that does not launches both.
+__global__ void __launch_bounds__(kDecodeLaunch, kWarpsPerSm)
+decode_sum_warps(DecodeArgs a)
+{
+    __shared__ __align__(16) float s_acc[kDecodeChunk];
+    __shared__ __align__(16) WarpDecSmem ws;
+    __shared__ u64 s_nsel[ADACOMP_MAX_STREAMS];
+    __shared__ float s_scale[ADACOMP_MAX_STREAMS];
+    __shared__ int s_bad;
+    u32 L_T;
+    u64 n;
+    if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
+    if (!warp_path(geo)) return;
+    if (geo.w == 1u) decode_warps<unsigned char>(a, geo, s_acc, ws, s_scale, s_nsel);
+    else decode_warps<unsigned short>(a, geo, s_acc, ws, s_scale, s_nsel);
+}
+
+__global__ void __launch_bounds__(kDecodeThreads, 6)
+decode_sum(DecodeArgs a)
+{
+    __shared__ __align__(16) DecodeSmem sm;
+    __shared__ int s_bad;
+    u32 L_T;
+    u64 n;
+    if (!decode_headers(a, &s_bad, sm.scale, sm.n_sel, L_T, n)) return;
+    const Geometry geo = make_geometry(n, L_T);
+    if (warp_path(geo)) return;
     const bool by_bin = geo.tile_bins >= 32 && geo.tile_bins <= (u32)kSmallBins;
     const bool by_word = geo.tile_bins >= 2 && geo.tile_bins <= 31;
-    if (threadIdx.x < a.k) {
-        sm.scale[threadIdx.x] = __uint_as_float(reinterpret_cast<const u32 *>(a.stream[threadIdx.x])[12]);
-        sm.n_sel[threadIdx.x] = reinterpret_cast<const u64 *>(a.stream[threadIdx.x])[5];
-    }
-    if ((by_bin || by_word) && (geo.tile_bins * geo.w) % 16u == 0) {
-        // bin-count runs start on 16-byte boundaries: everything a tile needs can be bulk-copied ahead
-        if (geo.w == 1u) decode_pipelined<unsigned char>(a, geo, sm.acc, sm.pipe, sm.scale, sm.n_sel);
-        else decode_pipelined<unsigned short>(a, geo, sm.acc, sm.pipe, sm.scale, sm.n_sel);
-        return;
-    }
-    __syncthreads();                               // scales and word totals are in place
-    if (threadIdx.x >= kDecodeThreads) return;     // the other paths have no producer warp
     if (geo.w == 1u) {
         if (by_bin) decode_staged<unsigned char, true>(a, geo, sm);
         else decode_generic<unsigned char>(a, geo, sm);
@@ -2030,6 +2244,7 @@ struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
     int decode_per_sm = 0;
+    int decode_warps_per_sm = 0;
     int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
@@ -2049,8 +2264,10 @@ int device_info(DeviceInfo *&out)
             return ADACOMP_ERR_CUDA;
         d.smem_optin = optin;
         int per_sm = 1;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeLaunch, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps, kDecodeLaunch, 0);
+        d.decode_warps_per_sm = per_sm < 1 ? 1 : per_sm;
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
         d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
@@ -2195,12 +2412,17 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
-    u64 grid = (u64)info->sms * info->decode_per_sm;
-    if (hint_L_T) {             // the shape is known on the host: no more CTAs than work items
+    u64 grid = (u64)info->sms * info->decode_per_sm, grid_w = (u64)info->sms * info->decode_warps_per_sm;
+    bool warps = true, others = true;   // the shape is on the device: both kernels go, one of them returns at once
+    if (hint_L_T) {                     // the shape is known on the host: one kernel, no more CTAs than work items
         const u64 items = decode_items(hint_n, hint_L_T);
         grid = items < grid ? (items ? items : 1) : grid;
+        grid_w = items < grid_w ? (items ? items : 1) : grid_w;
+        warps = warp_path(make_geometry(hint_n, hint_L_T));
+        others = !warps;
     }
-    decode_sum<<<(unsigned)grid, kDecodeLaunch, 0, static_cast<cudaStream_t>(stream)>>>(args);
+    if (warps) decode_sum_warps<<<(unsigned)grid_w, kDecodeLaunch, 0, static_cast<cudaStream_t>(stream)>>>(args);
+    if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, static_cast<cudaStream_t>(stream)>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
