@@ -1133,13 +1133,17 @@ struct WarpDecSmem {
     u32 tmp[4][32];                             // per decoding warp: output places of its non-empty bins
     unsigned short coff[ADACOMP_MAX_STREAMS];   // byte offset in a slot of learner l's bin counts (its words follow them)
     unsigned short wcap[ADACOMP_MAX_STREAMS];   // bytes of its word region
+    unsigned char rfirst[ADACOMP_MAX_STREAMS];  // round r brings learners [rfirst[r], rfirst[r] + rcount[r]) of a tile
+    unsigned char rcount[ADACOMP_MAX_STREAMS];
     u64 full[kSlots], empty[kSlots];            // mbarriers of the slots
-    u32 slot_bytes, n_slots, kf, abort;         // kf: learners [0, kf) have a region
+    u32 slot_bytes, n_slots, n_rounds, abort;
 };
 
-// A slot starts with {u32 staged, u32 bad} (learners [0, staged) of this tile are in the slot;
-// failed directory checks), 8 bytes of padding, then u16 cnt[k8] and u16 head[k8]: words of the
-// learner in this tile and the byte offset of the first one in its word region.
+// A slot holds one round of one tile: the learners of the round, as many as fit a slot with their
+// regions (all k of them when k is small).  It starts with {u32 staged, u32 bad} (the first
+// `staged` learners of the round are in the slot; failed directory checks), 8 bytes of padding,
+// then u16 cnt[k8] and u16 head[k8], indexed by the learner's place in the round: its words in
+// this tile and the byte offset of the first one in its word region.
 constexpr u32 kSlotHead = 16;
 
 struct DecodeSmem {
@@ -1387,23 +1391,30 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
 // decode, warp path: tiles of 4..96 bins whose bin-count run is a multiple of 16 bytes
 // (L_T = 50 and 500 among them).
 //
-// Warp 4 is a loader: for every tile of this CTA, lane l reads learner l's two directory
-// entries (two tiles ahead) and bulk-copies (TMA, no multicast) that learner's bin counts and
-// words of the tile into the learner's fixed region of a shared-memory slot; the slots form a
-// ring of up to kSlots tiles in flight.  Region sizes are set once per launch from the streams'
-// word totals (1.5 times a tile's average plus slack); a learner whose words of some tile do not
-// fit its region, and every learner for which the slot has no region, is read by the decoding
-// warps straight from global memory for that tile.
+// Warp 4 is a loader: for every tile of this CTA, a lane per learner reads the learner's two
+// directory entries (two steps ahead) and bulk-copies (TMA, no multicast) that learner's bin
+// counts and words of the tile into the learner's fixed region of a shared-memory slot; the
+// slots form a ring of up to kSlots in flight.  Region sizes are set once per launch from the
+// streams' word totals (1.5 times a tile's average plus slack).  When the k regions do not fit
+// one slot together, a tile takes several rounds, each a slot of its own with the next learners
+// in order.  A learner whose words of some tile do not fit its region is read by the decoding
+// warps straight from global memory for that tile.  The loader does nothing else: it shares its
+// SM's issue slots with some thirty busy warps, so its chain of dependent instructions per
+// tile has to stay short.
 //
 // Warps 0-3 decode.  Each owns a quarter of the tile's bins and of the output tile and never
 // touches the rest, so the four need no barrier among themselves: a warp waits for the slot,
 // adds its words learner by learner (one __syncwarp() between learners keeps an element's
-// contributions in learner order), gives the slot back and stores its quarter.  Within a
-// learner the warp works by word, not by bin: lane j takes word j of the warp's run of words, 32
-// at a time.  The bin of a word comes from the bin counts: the lanes that hold the warp's bins
-// (at most 24) scan their counts, raise a flag bit at the position of each non-empty bin's first
-// word, and a word's bin is the number of flags at or before it (a population count), mapped to
-// the bin's place in the output tile by one shuffle.
+// contributions in learner order), gives the slot back, hands its quarter to one bulk copy
+// (TMA store: the output does not pass through the warps' load/store path, which the adds keep
+// busy) and zeroes it once the copy has read it.
+// Two schemes for the adds.  Tiles of at most 64 bins (16-bit words among them): G lanes share a
+// bin and take every G-th word of it.  Tiles of more bins (8-bit words, L_T <= 58): the warp works
+// by word, lane j takes word j of the warp's run of words, 32 at a time; the bin of a word comes
+// from the bin counts: the lanes that hold the warp's bins (at most 24) scan their counts, raise
+// a flag bit at the position of each non-empty bin's first word, and a word's bin is the number
+// of flags at or before it (a population count), mapped to the bin's place in the output tile by
+// one shuffle.
 // Loader and decoding warps meet only through the slots' full / empty mbarriers, and every wait
 // on those is bounded.
 // ---------------------------------------------------------------------------------
@@ -1673,21 +1684,20 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
     return warp_add_group<Word, false, u64>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
 }
 
-template <typename Word>
+// Lays the slots out (see WarpDecSmem), then decodes.
+template <typename Word, bool MULTI>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
-                             const float *s_scale, const u64 *s_nsel)
+                             const float *s_scale, const u64 *s_nsel);
+
+template <typename Word>
+__device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+                                 const float *s_scale, const u64 *s_nsel)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
-    const u32 L_T = geo.L_T;
     const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
-    const u64 first = blockIdx.x, stride = gridDim.x;
-    const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
     const u32 k8 = (a.k + 7u) & ~7u;
     const u32 meta_bytes = kSlotHead + 4u * k8;                    // slot header + cnt[k8] + head[k8]
-    unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
-    constexpr u32 full_mask = 0xffffffffu;
-
     if (tid == 0) {
         for (int s = 0; s < kSlots; s++) {
             mbar_init(&ws.full[s], 32);         // every lane of the loader arrives, with or without bytes to expect
@@ -1698,143 +1708,183 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     }
     for (int i = tid; i < kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
     if (warp == 4) {
-        // the learners' regions of a slot: counts, then room for 1.5 times a tile's average words + slack
-        u32 used = meta_bytes, kf = 0;
-        bool open = true;
+        // the learners' regions: counts, then room for 1.5 times a tile's average words + slack
 #pragma unroll
         for (int h = 0; h < 2; h++) {
             const u32 l = (u32)lane + 32u * h;
-            const bool active = l < a.k;
-            u32 wbytes = 0;
-            if (active) {
+            if (l < a.k) {
                 const u64 avg = s_nsel[l] / geo.n_tiles;
                 const u64 cap = min((u64)geo.tile_elems, avg + avg / 2 + 64);
-                wbytes = (u32)align_up(cap * sizeof(Word) + 16, 16);
+                ws.wcap[l] = (unsigned short)align_up(cap * sizeof(Word) + 16, 16);
             }
-            const u32 need = active ? count_bytes + wbytes : 0u;
-            const u32 incl = used + warp_inclusive_scan(need, lane);
-            const u32 fits = __ballot_sync(full_mask, active && open && incl <= kSlotMax);
-            const int lead = __ffs(~fits) - 1;
-            const int staged_lanes = lead < 0 ? 32 : lead;
-            if (active) {
-                ws.coff[l] = (unsigned short)(incl - need);
-                ws.wcap[l] = (unsigned short)wbytes;
-            }
-            kf += (u32)staged_lanes;
-            if (staged_lanes > 0) used = __shfl_sync(full_mask, incl, staged_lanes - 1);
-            if (staged_lanes < 32) open = false;
         }
+        __syncwarp();
         if (lane == 0) {
-            ws.kf = kf;
-            ws.slot_bytes = used;
-            ws.n_slots = max(1u, min((u32)kSlots, kRingBytes / used));     // (kf == 0: one slot of headers only)
+            // rounds: learners in order, as many per round as fit a slot (any one learner fits)
+            u32 r = 0, used = meta_bytes, most = 0, r0 = 0;
+            for (u32 l = 0; l < a.k; l++) {
+                const u32 need = count_bytes + ws.wcap[l];
+                if (used + need > kSlotMax && l > r0) {
+                    ws.rfirst[r] = (unsigned char)r0;
+                    ws.rcount[r] = (unsigned char)(l - r0);
+                    r++;
+                    r0 = l;
+                    used = meta_bytes;
+                }
+                ws.coff[l] = (unsigned short)used;
+                used += need;
+                most = max(most, used);
+            }
+            ws.rfirst[r] = (unsigned char)r0;
+            ws.rcount[r] = (unsigned char)(a.k - r0);
+            ws.n_rounds = r + 1u;
+            ws.slot_bytes = most;
+            ws.n_slots = min((u32)kSlots, kRingBytes / most);
         }
     }
     __syncthreads();
-    const u32 kf = ws.kf, slot_bytes = ws.slot_bytes, S = ws.n_slots;
+    if (ws.n_rounds > 1u) decode_warps<Word, true>(a, geo, s_acc, ws, s_scale, s_nsel);
+    else decode_warps<Word, false>(a, geo, s_acc, ws, s_scale, s_nsel);
+}
+
+// MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
+template <typename Word, bool MULTI>
+__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+                             const float *s_scale, const u64 *s_nsel)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int TB = (int)geo.tile_bins;
+    const u32 L_T = geo.L_T;
+    const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
+    const u64 first = blockIdx.x, stride = gridDim.x;
+    const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
+    const u32 k8 = (a.k + 7u) & ~7u;
+    unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
+    constexpr u32 full_mask = 0xffffffffu;
+
+    const u32 NR = MULTI ? ws.n_rounds : 1u, slot_bytes = ws.slot_bytes, S = ws.n_slots;
 
     if (warp == 4) {
         // ================================ loader warp ================================
+        // An item is one round of one tile; lane j (and j + 32) looks after the j-th learner of the
+        // round.  The learners' directory entries are read two items ahead.
         u64 da0[2] = {0, 0}, da1[2] = {0, 0}, db0[2] = {0, 0}, db1[2] = {0, 0};
-        auto load_dir = [&](u64 t, u64 *d0, u64 *d1) {
-            const u64 tile = first + t * stride;
+        auto load_dir = [&](u64 tile, u32 r, bool valid, u64 *d0, u64 *d1) {
 #pragma unroll
             for (int h = 0; h < 2; h++) {
-                const u32 l = (u32)lane + 32u * h;
-                if (l < kf && t < my_tiles) {
-                    const u64 *dir = reinterpret_cast<const u64 *>(a.stream[l] + geo.tile_off_at);
+                const u32 j = (u32)lane + 32u * h;
+                if (valid && j < (MULTI ? (u32)ws.rcount[r] : a.k)) {
+                    const u64 *dir = reinterpret_cast<const u64 *>(a.stream[(MULTI ? (u32)ws.rfirst[r] : 0u) + j] + geo.tile_off_at);
                     d0[h] = dir[tile];
                     d1[h] = dir[tile + 1];
                 }
             }
         };
-        load_dir(0, da0, da1);
-        load_dir(1, db0, db1);
-        u32 my_coff[2], my_wcap[2];
+        // (no division in the loops: slot, use count and the look-ahead position step along)
+        u64 ptile = first, pit = 0;     // the item two ahead: its tile and round
+        u32 pr = 0;
+        auto step_ahead = [&]() {
+            if (++pr == NR) {
+                pr = 0;
+                ptile += stride;
+                pit++;
+            }
+        };
+        load_dir(ptile, pr, pit < my_tiles, da0, da1);
+        step_ahead();
+        load_dir(ptile, pr, pit < my_tiles, db0, db1);
+        step_ahead();
+        u32 my_coff[2] = {0, 0}, my_wcap[2] = {0, 0};       // one round: the lane's learners stay the same
 #pragma unroll
         for (int h = 0; h < 2; h++) {
             const u32 l = (u32)lane + 32u * h;
-            my_coff[h] = l < kf ? ws.coff[l] : 0u;
-            my_wcap[h] = l < kf ? ws.wcap[l] : 0u;
-        }
-        u64 issued = 0;                 // copies were started for tiles [0, issued)
-        PHASE_DECL;
-        long long tp = clock64();
-        // (no division by S in the loops: slot and use count step along with the tile)
-        u32 s = 0, use = 0;             // the tile's slot; how many times the slot was used before
-        u64 tile = first;
-        for (u64 it = 0; it < my_tiles; it++, tile += stride, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
-            PHASE_CLOCK(9, tp);
-            if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
-                ws.abort = 1;
-                raise_status(ADACOMP_DEV_TIMEOUT);
-                break;                  // the decoding warps time out on the full barrier in turn
+            if (!MULTI && l < a.k) {
+                my_coff[h] = ws.coff[l];
+                my_wcap[h] = ws.wcap[l];
             }
-            if (*reinterpret_cast<volatile u32 *>(&ws.abort)) break;
-            PHASE_CLOCK(7, tp);
-            unsigned char *sl = ring + s * slot_bytes;
+        }
+        u64 issued = 0;                 // copies were started for items [0, issued)
+        u32 s = 0, use = 0;             // the item's slot; how many times the slot was used before
+        u64 tile = first;
+        bool failed = false;
+        for (u64 it = 0; it < my_tiles && !failed; it++, tile += stride) {
             const u64 bin0 = tile * (u64)TB;
             const u64 bins_left = geo.n_bins - bin0;
             const u32 cbytes = bins_left >= (u64)TB ? count_bytes : (u32)align_up(bins_left * sizeof(Word), 16);   // last tile
-            unsigned short *m_cnt = reinterpret_cast<unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
-            u64 src[2] = {0, 0};
-            u32 wbytes[2] = {0, 0};
-            u32 staged = 0, bad = 0;
-            bool open = true;
-#pragma unroll
-            for (int h = 0; h < 2; h++) {
-                const u32 l = (u32)lane + 32u * h;
-                const bool active = l < kf;
-                bool ok = true, fit = false;
-                if (active) {
-                    ok = da1[h] >= da0[h] && da1[h] - da0[h] <= geo.tile_elems && da1[h] <= s_nsel[l];
-                    const u32 cnt = ok ? (u32)(da1[h] - da0[h]) : 0u;
-                    src[h] = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + da0[h] * sizeof(Word);
-                    const u32 head = (u32)(src[h] & 15u);
-                    wbytes[h] = cnt ? (u32)align_up(head + cnt * sizeof(Word), 16) : 0u;
-                    fit = wbytes[h] <= my_wcap[h];
-                    m_cnt[l] = (unsigned short)cnt;
-                    m_head[l] = (unsigned short)head;
+            for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
+                if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
+                    ws.abort = 1;
+                    raise_status(ADACOMP_DEV_TIMEOUT);
+                    failed = true;      // the decoding warps time out on the full barrier in turn
+                    break;
                 }
-                if (__any_sync(full_mask, active && !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
-                const u32 fits = __ballot_sync(full_mask, active && open && fit);
-                const int lead = __ffs(~fits) - 1;
-                const int staged_lanes = lead < 0 ? 32 : lead;
-                staged += (u32)staged_lanes;
-                if (staged_lanes < 32) open = false;
-                if (kf <= 32u) break;
-            }
-            if (lane == 0) {
-                reinterpret_cast<u32 *>(sl)[0] = staged;
-                reinterpret_cast<u32 *>(sl)[1] = bad;
-            }
-            __syncwarp();
-            u32 expect = 0;
-#pragma unroll
-            for (int h = 0; h < 2; h++)
-                if ((u32)lane + 32u * h < staged) expect += cbytes + wbytes[h];
-            if (expect) mbar_arrive_expect_tx(&ws.full[s], expect);
-            else mbar_arrive(&ws.full[s]);
-#pragma unroll
-            for (int h = 0; h < 2; h++) {
-                const u32 l = (u32)lane + 32u * h;
-                if (l < staged) {
-                    bulk_load(sl + my_coff[h], a.stream[l] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ws.full[s]);
-                    if (wbytes[h])
-                        bulk_load(sl + my_coff[h] + count_bytes, reinterpret_cast<const void *>(src[h] & ~(u64)15u),
-                                  wbytes[h], &ws.full[s]);
+                if (*reinterpret_cast<volatile u32 *>(&ws.abort)) {
+                    failed = true;
+                    break;
                 }
-            }
-            issued = it + 1;
+                unsigned char *sl = ring + s * slot_bytes;
+                unsigned short *m_cnt = reinterpret_cast<unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
+                const u32 l0 = MULTI ? ws.rfirst[r] : 0u, nl = MULTI ? ws.rcount[r] : a.k;
+                u64 src[2] = {0, 0};
+                u32 wbytes[2] = {0, 0}, coff[2] = {0, 0};
+                u32 staged = 0, bad = 0;
+                bool open = true;
 #pragma unroll
-            for (int h = 0; h < 2; h++) {
-                da0[h] = db0[h];
-                da1[h] = db1[h];
+                for (int h = 0; h < 2; h++) {
+                    const u32 j = (u32)lane + 32u * h;
+                    const bool active = j < nl;
+                    bool ok = true, fit = false;
+                    if (active) {
+                        const u32 l = l0 + j;
+                        ok = da1[h] >= da0[h] && da1[h] - da0[h] <= geo.tile_elems && da1[h] <= s_nsel[l];
+                        const u32 cnt = ok ? (u32)(da1[h] - da0[h]) : 0u;
+                        src[h] = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + da0[h] * sizeof(Word);
+                        const u32 head = (u32)(src[h] & 15u);
+                        wbytes[h] = cnt ? (u32)align_up(head + cnt * sizeof(Word), 16) : 0u;
+                        fit = wbytes[h] <= (MULTI ? (u32)ws.wcap[l] : my_wcap[h]);
+                        coff[h] = MULTI ? (u32)ws.coff[l] : my_coff[h];
+                        m_cnt[j] = (unsigned short)cnt;
+                        m_head[j] = (unsigned short)head;
+                    }
+                    if (__any_sync(full_mask, active && !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
+                    const u32 fits = __ballot_sync(full_mask, active && open && fit);
+                    const int lead = __ffs(~fits) - 1;
+                    const int staged_lanes = lead < 0 ? 32 : lead;
+                    staged += (u32)staged_lanes;
+                    if (staged_lanes < 32) open = false;
+                    if (nl <= 32u) break;
+                }
+                if (lane == 0) {
+                    reinterpret_cast<u32 *>(sl)[0] = staged;
+                    reinterpret_cast<u32 *>(sl)[1] = bad;
+                }
+                __syncwarp();
+                u32 expect = 0;
+#pragma unroll
+                for (int h = 0; h < 2; h++)
+                    if ((u32)lane + 32u * h < staged) expect += cbytes + wbytes[h];
+                if (expect) mbar_arrive_expect_tx(&ws.full[s], expect);
+                else mbar_arrive(&ws.full[s]);
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    const u32 j = (u32)lane + 32u * h;
+                    if (j < staged) {
+                        bulk_load(sl + coff[h], a.stream[l0 + j] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ws.full[s]);
+                        if (wbytes[h])
+                            bulk_load(sl + coff[h] + count_bytes, reinterpret_cast<const void *>(src[h] & ~(u64)15u), wbytes[h],
+                                      &ws.full[s]);
+                    }
+                }
+                issued++;
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    da0[h] = db0[h];
+                    da1[h] = db1[h];
+                }
+                load_dir(ptile, pr, pit < my_tiles, db0, db1);
+                step_ahead();
             }
-            load_dir(it + 2, db0, db1);
-            PHASE_CLOCK(8, tp);
         }
-        PHASE_FLUSH(128, 7, 10);
         if (*reinterpret_cast<volatile u32 *>(&ws.abort)) {
             // after a timeout the copies already started must land (or time out in turn) before
             // this CTA's shared memory is given back
@@ -1860,62 +1910,69 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     const u32 mine_at = smem_addr(s_acc) + (u32)my_bin * L_T * 4u;
     u32 bad = 0;
     PHASE_DECL;
-    u32 s = 0, use = 0;                             // the tile's slot; how many times the slot was used before
+    u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
     u64 tile = first;
-    for (u64 it = 0; it < my_tiles; it++, tile += stride, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
+    bool failed = false;
+    for (u64 it = 0; it < my_tiles; it++, tile += stride) {
         const u64 bin0 = tile * (u64)TB;
         const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
+        for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
+            long long t0 = clock64();
+            if (!mbar_wait(&ws.full[s], use & 1u)) {
+                ws.abort = 1;
+                bad |= ADACOMP_DEV_TIMEOUT;
+                failed = true;
+                break;
+            }
+            PHASE_CLOCK(0, t0);
+            const unsigned char *sl = ring + s * slot_bytes;
+            const u32 l0 = MULTI ? ws.rfirst[r] : 0u, nl = MULTI ? ws.rcount[r] : a.k;
+            const u32 staged = min(reinterpret_cast<const u32 *>(sl)[0], nl);
+            if (warp == 0) bad |= reinterpret_cast<const u32 *>(sl)[1];
+            const unsigned short *m_cnt = reinterpret_cast<const unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
+            const u32 sl_at = smem_addr(sl);
+
+            // ---- the round's learners whose words wait in the slot, four at a time ----
+            for (u32 g0 = 0; g0 < staged; g0 += kRoundMax) {
+                const int R = (int)min((u32)kRoundMax, staged - g0);
+                GroupSrc<u32> src = {0u, 0u, 0u, 0u};
+                if (lane < R) {
+                    const u32 j = g0 + (u32)lane, l = l0 + j;
+                    src.counts = sl_at + ws.coff[l];
+                    src.words = src.counts + count_bytes + m_head[j];
+                    src.limit = m_cnt[j];
+                    src.sbits = __float_as_uint(s_scale[l]);
+                }
+                if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+                else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
+            }
+            if (lane == 0) mbar_arrive(&ws.empty[s]);   // (the group's last __syncwarp orders the warp's reads before it)
+            PHASE_CLOCK(1, t0);
+
+            // ---- the round's others: read from global memory ----
+            for (u32 g0 = staged; g0 < nl; g0 += kRoundMax) {
+                const int R = (int)min((u32)kRoundMax, nl - g0);
+                GroupSrc<u64> src = {0ull, 0ull, 0u, 0u};
+                bool ok = true;
+                if (lane < R) {
+                    const u32 l = l0 + g0 + (u32)lane;
+                    const unsigned char *st = a.stream[l];
+                    const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
+                    const u64 w0 = dir[tile], w1 = dir[tile + 1];
+                    ok = w1 >= w0 && w1 - w0 <= geo.tile_elems && w1 <= s_nsel[l];
+                    src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
+                    src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
+                    src.limit = ok ? (u32)(w1 - w0) : 0u;
+                    src.sbits = __float_as_uint(s_scale[l]);
+                }
+                if (__any_sync(full_mask, !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
+                if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+                else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
+            }
+            PHASE_CLOCK(2, t0);
+        }
+        if (failed) break;
         long long t0 = clock64();
-        if (!mbar_wait(&ws.full[s], use & 1u)) {
-            ws.abort = 1;
-            bad |= ADACOMP_DEV_TIMEOUT;
-            break;
-        }
-        PHASE_CLOCK(0, t0);
-        const unsigned char *sl = ring + s * slot_bytes;
-        const u32 staged = reinterpret_cast<const u32 *>(sl)[0];
-        if (warp == 0) bad |= reinterpret_cast<const u32 *>(sl)[1];
-        const unsigned short *m_cnt = reinterpret_cast<const unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
-        const u32 sl_at = smem_addr(sl);
-
-        // ---- the learners whose words wait in the slot, four at a time ----
-        for (u32 g0 = 0; g0 < staged; g0 += kRoundMax) {
-            const int R = (int)min((u32)kRoundMax, staged - g0);
-            GroupSrc<u32> src = {0u, 0u, 0u, 0u};
-            if (lane < R) {
-                const u32 l = g0 + (u32)lane;
-                src.counts = sl_at + ws.coff[l];
-                src.words = src.counts + count_bytes + m_head[l];
-                src.limit = m_cnt[l];
-                src.sbits = __float_as_uint(s_scale[l]);
-            }
-            if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
-            else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
-        }
-        if (lane == 0) mbar_arrive(&ws.empty[s]);   // (the group's last __syncwarp orders the warp's reads before it)
-        PHASE_CLOCK(1, t0);
-
-        // ---- the others: read from global memory ----
-        for (u32 g0 = staged; g0 < a.k; g0 += kRoundMax) {
-            const int R = (int)min((u32)kRoundMax, a.k - g0);
-            GroupSrc<u64> src = {0ull, 0ull, 0u, 0u};
-            bool ok = true;
-            if (lane < R) {
-                const u32 l = g0 + (u32)lane;
-                const unsigned char *st = a.stream[l];
-                const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
-                const u64 w0 = dir[tile], w1 = dir[tile + 1];
-                ok = w1 >= w0 && w1 - w0 <= geo.tile_elems && w1 <= s_nsel[l];
-                src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
-                src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
-                src.limit = ok ? (u32)(w1 - w0) : 0u;
-                src.sbits = __float_as_uint(s_scale[l]);
-            }
-            if (__any_sync(full_mask, !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
-            if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
-            else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
-        }
-        PHASE_CLOCK(2, t0);
 
         // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
         const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
@@ -2089,8 +2146,9 @@ decode_sum_warps(DecodeArgs a)
     if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
     if (!warp_path(geo)) return;
-    if (geo.w == 1u) decode_warps<unsigned char>(a, geo, s_acc, ws, s_scale, s_nsel);
-    else decode_warps<unsigned short>(a, geo, s_acc, ws, s_scale, s_nsel);
+    // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
+    if (geo.w == 1u) decode_warps_any<unsigned char>(a, geo, s_acc, ws, s_scale, s_nsel);
+    else decode_warps_any<unsigned short>(a, geo, s_acc, ws, s_scale, s_nsel);
 }
 
 __global__ void __launch_bounds__(kDecodeThreads, 6)
