@@ -182,6 +182,42 @@ def test_decode_sum_dense_streams_overflow_the_prefetch_stage():
     assert B.adacomp_device_status() == 0
 
 
+def test_decode_sum_uneven_density_and_many_learners():
+    """The decoder sizes a learner's staging region from its average words per tile.  A learner that is
+    dense in a few tiles only overflows it there; forty sparse learners share one staging slot (more
+    learners than a warp has lanes); forty denser ones need several slots per tile."""
+    rng = np.random.default_rng(77)
+    cases = []
+    for L_T in (50, 500):
+        n = 4000 * 12 + 5
+        layers = []
+        for l in range(5):
+            dW = rng.normal(0, 1e-3, n).astype(np.float32)
+            if l == 2:      # every element of tiles 3..5 ties for its bin's maximum: all of them are sent
+                dW[12000:24000] = np.where(rng.random(12000) < 0.5, -1.0, 1.0).astype(np.float32) * np.float32(0.25)
+            layers.append((dW, np.zeros(n, np.float32)))
+        cases.append((L_T, n, layers))
+    n = 4000 * 6 + 9
+    sparse = []
+    for l in range(40):     # a few large entries per learner on a floor of tiny ones: few words per tile
+        dW = rng.normal(0, 1e-6, n).astype(np.float32)
+        at = rng.choice(n, 60, replace=False)
+        dW[at] = rng.normal(0, 1.0, 60).astype(np.float32)
+        sparse.append((dW, rng.normal(0, 1e-6, n).astype(np.float32)))
+    cases.append((500, n, sparse))
+    cases.append((50, n, [(rng.normal(0, 1e-3, n).astype(np.float32), np.zeros(n, np.float32)) for _ in range(40)]))
+    for L_T, n, layers in cases:
+        streams = []
+        for dW, r in layers:
+            want = cref.pack(dW, r.copy(), L_T)
+            raw, _, _ = GpuLayer(n, L_T, r).compress(dW)
+            assert_stream_equal(raw, want)
+            streams.append(raw)
+        got = gpu_decode(streams, n)
+        assert_f32_bits_equal(got, cref.unpack_sum(streams, n), f"decode L_T={L_T} k={len(layers)}")
+    assert B.adacomp_device_status() == 0
+
+
 def test_decode_with_shape_hint_matches_and_rejects_wrong_hints():
     dev = torch.device("cuda:0")
     rng = np.random.default_rng(31)
