@@ -120,3 +120,29 @@ def unpack_sum(streams: Sequence[np.ndarray], n: int) -> np.ndarray:
     if rc != 0:
         raise RuntimeError(f"adacomp_oracle_unpack_sum failed: {rc}")
     return dst
+
+
+def average_sgd(streams: Sequence[np.ndarray], n: int, weights: np.ndarray, momentum: np.ndarray,
+                lr: float, mu: float):
+    """unpack(), averageGradients() and updateWeights() of Algorithm 1 ("Computation Steps") for one layer.
+
+    The paper trains with "the conventional SGD with momentum" (momentum 0.9, Section "Discussions") and
+    gives no formula; the reading taken here is the plain heavy-ball step with no dampening, Nesterov
+    term or weight decay, every operation rounded to binary32 on its own (no fused multiply-add):
+
+        s    = sum of the k decoded streams, in learner order, from +0.0f     (unpack, as unpack_sum)
+        mean = s / k                                                          (averageGradients: one division)
+        v'   = (mu * v) + mean                                                (updateWeights)
+        w'   = w - (lr * v')
+
+    Returns (w', v') as new float32 arrays; the inputs are not modified.
+    """
+    k = len(streams)
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    v = np.ascontiguousarray(momentum, dtype=np.float32)
+    s = unpack_sum(streams, n)
+    mean = s / np.float32(k)
+    v_new = np.float32(mu) * v[:n] + mean
+    w_new = w[:n] - np.float32(lr) * v_new
+    assert mean.dtype == v_new.dtype == w_new.dtype == np.float32
+    return w_new, v_new
