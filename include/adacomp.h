@@ -173,6 +173,31 @@ int adacomp_decompress_accumulate(const void *const *packed, uint32_t k_streams,
 int adacomp_decompress_accumulate_ex(const void *const *packed, uint32_t k_streams, float *dst,
                                      uint64_t n, uint32_t L_T, void *stream);
 
+/*
+ * unpack(), averageGradients() and updateWeights() of Algorithm 1 ("Computation Steps") in one
+ * pass over the layer: the k streams are decoded and summed as adacomp_decompress_accumulate does,
+ * and each finished piece of the sum feeds the optimizer step on the spot, so that the dense
+ * gradient is never written to memory.  The paper names "SGD with momentum" (momentum 0.9,
+ * Section "Discussions") and prints no formula; the step taken is the plain heavy-ball one, every
+ * operation rounded to binary32 on its own (no fused multiply-add):
+ *     s    = ordered sum of the k decoded streams, from +0.0f
+ *     mean = s / k                      (one IEEE division by float(k))
+ *     v'   = (mu * v) + mean
+ *     w'   = w - (lr * v')
+ * for every element of the layer, the ones nobody sent included (mean = +0 there).
+ *   packed     HOST array of k device pointers to packed streams of one layer.
+ *   weights    device, float[n], read and written in place (w).
+ *   momentum   device, float[n], read and written in place (v).
+ *   n, L_T     the layer's shape; streams whose headers do not carry exactly (n, L_T) set
+ *              ADACOMP_DEV_HEADER_MISMATCH and neither array is touched.
+ *   lr, mu     learning rate and momentum coefficient.
+ * weights and momentum must be 16-byte aligned, must not overlap each other or the streams, and
+ * stay owned by the caller.  Asynchronous on `stream`; errors as for the other entry points.
+ */
+int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams, float *weights,
+                                   float *momentum, uint64_t n, uint32_t L_T, float lr, float mu,
+                                   void *stream);
+
 /* adacomp_decompress_accumulate_multi with the layers' shapes (HOST arrays n[n_layers], L_T[n_layers]). */
 int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams,
                                            float *const *dst, const uint64_t *n, const uint32_t *L_T,

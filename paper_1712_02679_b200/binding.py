@@ -67,6 +67,9 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate_ex.restype = C.c_int
         L.adacomp_decompress_accumulate_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64,
                                                        C.c_uint32, C.c_void_p]
+        L.adacomp_decompress_average_sgd.restype = C.c_int
+        L.adacomp_decompress_average_sgd.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64,
+                                                     C.c_uint32, C.c_float, C.c_float, C.c_void_p]
         L.adacomp_decompress_accumulate_multi_ex.restype = C.c_int
         L.adacomp_decompress_accumulate_multi_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
                                                              C.c_void_p, C.c_uint32, C.c_void_p]
@@ -192,6 +195,18 @@ def adacomp_decompress_accumulate_ex(packed: Sequence[torch.Tensor], k_streams: 
     _check(lib().adacomp_decompress_accumulate_ex(ptrs, int(k_streams), _dev_ptr(dst, "dst", torch.float32),
                                                   int(n), int(L_T), _stream(stream)),
            "adacomp_decompress_accumulate_ex")
+
+
+def adacomp_decompress_average_sgd(packed: Sequence[torch.Tensor], k_streams: int, weights, momentum, n: int,
+                                   L_T: int, lr: float, mu: float, stream=None) -> None:
+    """unpack(), averageGradients() and updateWeights() (SGD with momentum) in one pass; weights and
+    momentum are updated in place."""
+    ptrs = (C.c_void_p * max(int(k_streams), 1))(
+        *[_dev_ptr(p, "packed[l]", torch.uint8) for p in packed[:k_streams]])
+    _check(lib().adacomp_decompress_average_sgd(ptrs, int(k_streams), _dev_ptr(weights, "weights", torch.float32),
+                                                _dev_ptr(momentum, "momentum", torch.float32), int(n), int(L_T),
+                                                C.c_float(lr), C.c_float(mu), _stream(stream)),
+           "adacomp_decompress_average_sgd")
 
 
 def adacomp_decompress_accumulate_multi_ex(packed, k_streams: int, dst, n: Sequence[int],

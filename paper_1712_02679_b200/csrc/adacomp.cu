@@ -1098,8 +1098,40 @@ batch_gather(const __grid_constant__ BatchArgsT<N> b)
 // decode_sum: unpack() of k streams and their ordered sum.
 // ---------------------------------------------------------------------------------
 
+// What becomes of a finished tile of the ordered sum s: stored to dst (unpack() alone), or, with
+// `weights` set, averageGradients() and updateWeights() of Algorithm 1 on the spot:
+//     mean = s / k,  v' = (mu * v) + mean,  w' = w - (lr * v'),
+// every operation rounded to binary32 on its own (the paper names "SGD with momentum" and prints
+// no formula: this is the plain heavy-ball step).  The dense gradient then never reaches memory.
+struct Epilogue {
+    float *weights, *momentum;
+    float lr, mu, k;
+};
+
+// (s / k without the division where the quotient is known without it: a zero sum, which is what
+// most elements have, stays the same zero; for k a power of two the product with 1 / k is the
+// correctly rounded quotient too.)
+__device__ inline void sgd_step(float s, float &w, float &v, const Epilogue &ep)
+{
+    const bool pow2 = (__float_as_uint(ep.k) & 0x007fffffu) == 0u;
+    const float mean = s == 0.f ? s : pow2 ? __fmul_rn(s, __frcp_rn(ep.k)) : __fdiv_rn(s, ep.k);
+    v = __fadd_rn(__fmul_rn(ep.mu, v), mean);
+    w = __fsub_rn(w, __fmul_rn(ep.lr, v));
+}
+
+// Four elements at once.
+__device__ inline void sgd_step4(float4 s, float4 &w, float4 &v, float lr, float mu, float k)
+{
+    const Epilogue ep = {nullptr, nullptr, lr, mu, k};
+    sgd_step(s.x, w.x, v.x, ep);
+    sgd_step(s.y, w.y, v.y, ep);
+    sgd_step(s.z, w.z, v.z, ep);
+    sgd_step(s.w, w.w, v.w, ep);
+}
+
 struct DecodeArgs {
     const unsigned char *stream[ADACOMP_MAX_STREAMS];
+    Epilogue ep;
     float *dst;
     u32 k;
     u32 hint_L_T;       // 0: the caller did not say; else the streams must carry exactly this shape
@@ -1136,6 +1168,7 @@ struct WarpDecSmem {
     unsigned char rfirst[ADACOMP_MAX_STREAMS];  // round r brings learners [rfirst[r], rfirst[r] + rcount[r]) of a tile
     unsigned char rcount[ADACOMP_MAX_STREAMS];
     u64 full[kSlots], empty[kSlots];            // mbarriers of the slots
+    u64 wv_full[4];                             // optimizer epilogue: a warp's weight and momentum quarters have landed
     u32 slot_bytes, n_slots, n_rounds, abort;
 };
 
@@ -1165,9 +1198,19 @@ struct DecodeSmem {
     float scale[ADACOMP_MAX_STREAMS];
 };
 
-__device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc)
+__device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc, const Epilogue &ep)
 {
     const int tid = threadIdx.x;
+    if (ep.weights) {
+        for (u32 i = tid; i < len; i += kDecodeThreads) {
+            float w = ep.weights[out0 + i], v = ep.momentum[out0 + i];
+            sgd_step(s_acc[i], w, v, ep);
+            ep.momentum[out0 + i] = v;
+            ep.weights[out0 + i] = w;
+            s_acc[i] = 0.f;
+        }
+        return;
+    }
     if ((out0 & 3u) == 0) {
         float4 *o4 = reinterpret_cast<float4 *>(dst + out0);
         float4 *s4 = reinterpret_cast<float4 *>(s_acc);
@@ -1227,7 +1270,7 @@ __device__ inline u32 check_fields(u32 x, u32 L_T)
 // clamped into the bin, so nothing is read or written out of bounds.
 template <typename Word, bool BY_BIN>
 __device__ void decode_item_staged(const unsigned char *const *streams, u32 k, const Geometry &geo, u64 tile,
-                                   float *dst, DecodeSmem &sm, u32 &bad)
+                                   float *dst, const Epilogue &ep, DecodeSmem &sm, u32 &bad)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
@@ -1373,7 +1416,7 @@ __device__ void decode_item_staged(const unsigned char *const *streams, u32 k, c
         }
     }
     const u32 len = (u32)min((u64)geo.tile_elems, geo.n - base);
-    store_tile(dst, base, len, sm.acc);
+    store_tile(dst, base, len, sm.acc, ep);
     consumer_barrier();
 }
 
@@ -1383,7 +1426,7 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
     for (int i = threadIdx.x; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
     u32 bad = 0;
     for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x)
-        decode_item_staged<Word, BY_BIN>(a.stream, a.k, geo, tile, a.dst, sm, bad);
+        decode_item_staged<Word, BY_BIN>(a.stream, a.k, geo, tile, a.dst, a.ep, sm, bad);
     if (bad) raise_status(bad);
 }
 
@@ -1685,13 +1728,14 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
 }
 
 // Lays the slots out (see WarpDecSmem), then decodes.
-template <typename Word, bool MULTI>
+template <typename Word, bool MULTI, bool SGD>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
-                             const float *s_scale, const u64 *s_nsel);
+                             const float *s_scale, const u64 *s_nsel, float *s_wv);
 
-template <typename Word>
+//   s_wv   (SGD) shared memory for a tile of weights followed by a tile of momentum, 2 x kDecodeChunk floats
+template <typename Word, bool SGD>
 __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
-                                 const float *s_scale, const u64 *s_nsel)
+                                 const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
@@ -1703,6 +1747,7 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
             mbar_init(&ws.full[s], 32);         // every lane of the loader arrives, with or without bytes to expect
             mbar_init(&ws.empty[s], 4);         // every decoding warp arrives
         }
+        for (int w = 0; w < 4; w++) mbar_init(&ws.wv_full[w], 1);
         ws.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -1743,14 +1788,15 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         }
     }
     __syncthreads();
-    if (ws.n_rounds > 1u) decode_warps<Word, true>(a, geo, s_acc, ws, s_scale, s_nsel);
-    else decode_warps<Word, false>(a, geo, s_acc, ws, s_scale, s_nsel);
+    if (ws.n_rounds > 1u) decode_warps<Word, true, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    else decode_warps<Word, false, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
 }
 
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
-template <typename Word, bool MULTI>
+// SGD: the finished quarter feeds the optimizer step of a.ep instead of going to a.dst.
+template <typename Word, bool MULTI, bool SGD>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
-                             const float *s_scale, const u64 *s_nsel)
+                             const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int TB = (int)geo.tile_bins;
@@ -1913,9 +1959,21 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
     u64 tile = first;
     bool failed = false;
+    float *const wq = s_wv + (u32)warp * quarter, *const vq = s_wv + kDecodeChunk + (u32)warp * quarter;     // (SGD)
+    u32 wv_use = 0;                                 // (SGD) fetches of the quarters so far
     for (u64 it = 0; it < my_tiles; it++, tile += stride) {
         const u64 bin0 = tile * (u64)TB;
         const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
+        const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
+        const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
+        const bool whole = vec_store && len == quarter;
+        if (SGD && whole && lane == 0) {
+            // the warp's quarters of the weights and the momentum travel while the words are added
+            bulk_wait_read_all();                   // the previous tile's copies out have read the buffers
+            mbar_arrive_expect_tx(&ws.wv_full[warp], 2u * quarter * 4u);
+            bulk_load(wq, a.ep.weights + out0, quarter * 4u, &ws.wv_full[warp]);
+            bulk_load(vq, a.ep.momentum + out0, quarter * 4u, &ws.wv_full[warp]);
+        }
         for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
             long long t0 = clock64();
             if (!mbar_wait(&ws.full[s], use & 1u)) {
@@ -1975,9 +2033,45 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         long long t0 = clock64();
 
         // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
-        const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
-        const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
-        if (vec_store && len == quarter) {
+        if (SGD) {
+            // averageGradients() + updateWeights() on the warp's quarter, in shared memory; two bulk
+            // copies take the new weights and momentum back
+            if (whole) {
+                if (!mbar_wait(&ws.wv_full[warp], wv_use & 1u)) {
+                    ws.abort = 1;
+                    bad |= ADACOMP_DEV_TIMEOUT;
+                    break;
+                }
+                wv_use++;
+                float4 *w4 = reinterpret_cast<float4 *>(wq), *v4 = reinterpret_cast<float4 *>(vq);
+                float4 *s4 = reinterpret_cast<float4 *>(my_acc);
+                const int n4 = (int)(quarter >> 2);
+                for (int at = lane; at < n4; at += 32) {
+                    float4 w = w4[at], v = v4[at];
+                    sgd_step4(s4[at], w, v, a.ep.lr, a.ep.mu, a.ep.k);
+                    s4[at] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    v4[at] = v;
+                    w4[at] = w;
+                }
+                fence_async_smem();                 // this lane's results, for the copy engine
+                __syncwarp();
+                if (lane == 0) {
+                    bulk_store(a.ep.weights + out0, wq, quarter * 4u);
+                    bulk_store(a.ep.momentum + out0, vq, quarter * 4u);
+                    bulk_commit();
+                }
+            } else {
+                for (u32 i = lane; i < quarter; i += 32) {
+                    if (i < len) {
+                        float w = a.ep.weights[out0 + i], v = a.ep.momentum[out0 + i];
+                        sgd_step(my_acc[i], w, v, a.ep);
+                        a.ep.momentum[out0 + i] = v;
+                        a.ep.weights[out0 + i] = w;
+                    }
+                    my_acc[i] = 0.f;
+                }
+            }
+        } else if (whole) {
             // one bulk copy (TMA) takes the quarter from shared memory: the warp's own stores stay
             // out of the way of everybody's shared-memory traffic
             fence_async_smem();                     // this lane's adds, for the copy engine
@@ -2082,7 +2176,7 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
         }
         const u64 out0 = base + c_lo;
         const u32 len = out0 < geo.n ? (u32)min((u64)(c_hi - c_lo), geo.n - out0) : 0u;
-        store_tile(a.dst, out0, len, s_acc);
+        store_tile(a.dst, out0, len, s_acc, a.ep);
         consumer_barrier();
     }
 }
@@ -2133,7 +2227,10 @@ __device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_
 // The decoder is two kernels, so that each gets the registers its path needs: decode_sum_warps
 // takes the shapes of warp_path() and returns at once for any other, decode_sum the reverse.  A
 // caller that knows the shape launches the one that works; one that does not launches both.
-__global__ void __launch_bounds__(kDecodeLaunch, kWarpsPerSm)
+constexpr u32 kSgdSmemBytes = 2u * kDecodeChunk * 4u;    // dynamic shared memory of decode_sum_warps<true>
+
+template <bool SGD>
+__global__ void __launch_bounds__(kDecodeLaunch, SGD ? 3 : kWarpsPerSm)
 decode_sum_warps(DecodeArgs a)
 {
     __shared__ __align__(16) float s_acc[kDecodeChunk];
@@ -2147,8 +2244,9 @@ decode_sum_warps(DecodeArgs a)
     const Geometry geo = make_geometry(n, L_T);
     if (!warp_path(geo)) return;
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
-    if (geo.w == 1u) decode_warps_any<unsigned char>(a, geo, s_acc, ws, s_scale, s_nsel);
-    else decode_warps_any<unsigned short>(a, geo, s_acc, ws, s_scale, s_nsel);
+    extern __shared__ __align__(16) float s_dyn[];     // (SGD) a tile of weights and a tile of momentum
+    if (geo.w == 1u) decode_warps_any<unsigned char, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, SGD ? s_dyn : nullptr);
+    else decode_warps_any<unsigned short, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, SGD ? s_dyn : nullptr);
 }
 
 __global__ void __launch_bounds__(kDecodeThreads, 6)
@@ -2232,6 +2330,7 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
     }
     consumer_barrier();
     const u32 total = sm.first[b.n_layers];
+    const Epilogue no_ep = {nullptr, nullptr, 0.f, 0.f, 0.f};
     for (u32 gt = blockIdx.x; gt < total; gt += gridDim.x) {
         int lo = 0, hi = (int)b.n_layers;            // largest t with first[t] <= gt and a tile of its own
         while (hi - lo > 1) {
@@ -2242,11 +2341,11 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
         const u64 tile = gt - sm.first[lo];
         const unsigned char *const *streams = &b.stream[lo * b.k];
         if (geo.w == 1u) {
-            decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+            decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
         } else if (geo.tile_bins >= 32) {
-            decode_item_staged<unsigned short, true>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+            decode_item_staged<unsigned short, true>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
         } else {
-            decode_item_staged<unsigned short, false>(streams, b.k, geo, tile, b.dst[lo], sm.d, bad);
+            decode_item_staged<unsigned short, false>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
         }
     }
     if (bad && blockIdx.x == 0) raise_status(bad & ADACOMP_DEV_HEADER_MISMATCH);
@@ -2303,6 +2402,7 @@ struct DeviceInfo {
     int smem_optin = 0;
     int decode_per_sm = 0;
     int decode_warps_per_sm = 0;
+    int decode_sgd_per_sm = 0;  // 0: the optimizer decoder is unavailable on this device
     int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
@@ -2324,8 +2424,14 @@ int device_info(DeviceInfo *&out)
         int per_sm = 1;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps, kDecodeLaunch, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<false>, kDecodeLaunch, 0);
         d.decode_warps_per_sm = per_sm < 1 ? 1 : per_sm;
+        if (cudaFuncSetAttribute(decode_sum_warps<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kSgdSmemBytes) == cudaSuccess) {
+            per_sm = 0;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<true>, kDecodeLaunch, kSgdSmemBytes);
+            d.decode_sgd_per_sm = per_sm;
+        }
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
         d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
@@ -2450,10 +2556,11 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
+// `ep` (optional): the optimizer step that takes the place of the store to dst (dst is null then).
 int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *stream, uint64_t hint_n = 0,
-                    uint32_t hint_L_T = 0)
+                    uint32_t hint_L_T = 0, const Epilogue *ep = nullptr)
 {
-    if (!packed || !dst) return ADACOMP_ERR_NULL;
+    if (!packed || (!dst && !ep)) return ADACOMP_ERR_NULL;
     if (k == 0 || k > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
     DecodeArgs args;
     for (uint32_t l = 0; l < ADACOMP_MAX_STREAMS; l++) args.stream[l] = nullptr;
@@ -2462,7 +2569,14 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         if (misaligned(packed[l])) return ADACOMP_ERR_ALIGN;
         args.stream[l] = static_cast<const unsigned char *>(packed[l]);
     }
-    if (misaligned(dst)) return ADACOMP_ERR_ALIGN;
+    if (dst && misaligned(dst)) return ADACOMP_ERR_ALIGN;
+    args.ep = Epilogue{nullptr, nullptr, 0.f, 0.f, (float)k};
+    if (ep) {
+        if (!ep->weights || !ep->momentum) return ADACOMP_ERR_NULL;
+        if (misaligned(ep->weights) || misaligned(ep->momentum)) return ADACOMP_ERR_ALIGN;
+        args.ep = *ep;
+        args.ep.k = (float)k;
+    }
     args.dst = dst;
     args.k = k;
     args.hint_n = hint_n;
@@ -2479,8 +2593,18 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         warps = warp_path(make_geometry(hint_n, hint_L_T));
         others = !warps;
     }
-    if (warps) decode_sum_warps<<<(unsigned)grid_w, kDecodeLaunch, 0, static_cast<cudaStream_t>(stream)>>>(args);
-    if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, static_cast<cudaStream_t>(stream)>>>(args);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (warps && ep) {
+        if (!info->decode_sgd_per_sm) return ADACOMP_ERR_CUDA;
+        u64 grid_s = (u64)info->sms * info->decode_sgd_per_sm;
+        if (hint_L_T) {
+            const u64 items = decode_items(hint_n, hint_L_T);
+            grid_s = items < grid_s ? (items ? items : 1) : grid_s;
+        }
+        decode_sum_warps<true><<<(unsigned)grid_s, kDecodeLaunch, kSgdSmemBytes, st>>>(args);
+    }
+    else if (warps) decode_sum_warps<false><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
+    if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, st>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
@@ -2864,6 +2988,14 @@ int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_st
         if (rc != ADACOMP_OK) return rc;
     }
     return ADACOMP_OK;
+}
+
+int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams, float *weights, float *momentum,
+                                   uint64_t n, uint32_t L_T, float lr, float mu, void *stream)
+{
+    if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    const Epilogue ep = {weights, momentum, lr, mu, 0.f};
+    return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
 }
 
 int adacomp_set_device(int device)

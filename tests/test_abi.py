@@ -85,6 +85,16 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     odd = (C.c_void_p * 1)(A + 2)
     assert g(odd, 1, A, None) == -3
     assert g(ptrs, 2, A + 4, None) == -3
+    u = lib.adacomp_decompress_average_sgd
+    lr, mu = C.c_float(0.1), C.c_float(0.9)
+    assert u(ptrs, 2, None, A, 10, 50, lr, mu, None) == -1
+    assert u(ptrs, 2, A, None, 10, 50, lr, mu, None) == -1
+    assert u(None, 2, A, A, 10, 50, lr, mu, None) == -1
+    assert u(ptrs, 2, A, A, 10, 0, lr, mu, None) == -2
+    assert u(ptrs, 2, A, A, 10, 16385, lr, mu, None) == -2
+    assert u(ptrs, 2, A + 4, A, 10, 50, lr, mu, None) == -3
+    assert u(ptrs, 2, A, A + 8, 10, 50, lr, mu, None) == -3
+    assert u(ptrs, 0, A, A, 10, 50, lr, mu, None) == -4
     assert lib.adacomp_device_status(None, None) == -1
     descs = (binding.adacomp_layer_desc * 1)()
     descs[0].grad, descs[0].residue, descs[0].n, descs[0].L_T = A, A, 5, 0
