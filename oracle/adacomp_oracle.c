@@ -148,10 +148,31 @@ double adacomp_oracle_exact_sum(const float *v, uint64_t count)
  * g_max_out (optional, n_bins floats) receives the bin maxima.
  * Returns 0, or -1 bad argument, -2 out of memory, -3 out_cap too small.
  */
+/*
+ * `factor`: the scale-factor of the self-adjusting selection (Section 2.4: "the sum of its previous
+ * residue plus the latest gradient multiplied by a scale-factor", studied from 1.5 to 3.0, 2 chosen
+ * "for computational ease (simple additions vs. multiplications)").  0 selects the paper's choice as
+ * Algorithm 2 writes it, H = G + dW with two additions; any other value takes the general form
+ * H = residue + factor * dW, one rounded multiplication and one rounded addition (for factor 2 the
+ * two forms can differ in the last place, which is why they are kept apart).  Factor 1 makes H = G:
+ * only the bin maxima are sent, the local-selection scheme "without soft-threshold" the paper
+ * compares against (Section 5, "LS").  Streams made with a factor carry bit 1 in the header's flags.
+ */
+int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint32_t L_T,
+                               uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out);
+
 int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_T,
                         uint32_t flags, uint8_t *out, uint64_t out_cap, float *g_max_out)
 {
+    return adacomp_oracle_pack_scaled(dW, residue, n, L_T, flags, 0.0f, out, out_cap, g_max_out);
+}
+
+int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint32_t L_T,
+                               uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out)
+{
     if (L_T == 0 || L_T > 16384u || !out || (n && (!dW || !residue))) return -1;
+    if (factor != 0.0f && !(factor > 0.0f && factor <= 1e30f)) return -1;
+    flags = (flags & 1u) | (factor != 0.0f ? 2u : 0u);
     const int literal = (flags & 1u) != 0;
     geometry geo = geometry_of(n, L_T);
     if (out_cap < geo.payload_at) return -3;
@@ -161,10 +182,15 @@ int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_
     float *g_max = (float *)malloc((geo.n_bins ? geo.n_bins : 1) * sizeof(float));
     if (!G || !H || !g_max) { free(G); free(H); free(g_max); return -2; }
 
-    /* G <- residue + dW ;  H <- G + dW   (two rounded additions) */
+    /* G <- residue + dW ;  H <- G + dW   (two rounded additions), or H <- residue + factor * dW */
     for (uint64_t i = 0; i < n; i++) {
         G[i] = residue[i] + dW[i];
-        H[i] = G[i] + dW[i];
+        if (factor == 0.0f) {
+            H[i] = G[i] + dW[i];
+        } else {
+            const float scaled = factor * dW[i];
+            H[i] = residue[i] + scaled;
+        }
     }
 
     /* first loop over all bins: the largest absolute value in each bin */
@@ -226,7 +252,7 @@ int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_
     put_u32(out + 0, ORACLE_MAGIC);
     put_u16(out + 4, 1);
     out[6] = (uint8_t)geo.w;
-    out[7] = (uint8_t)(flags & 1u);
+    out[7] = (uint8_t)(flags & 3u);
     put_u32(out + 8, L_T);
     put_u32(out + 12, geo.tile_bins);
     put_u64(out + 16, n);

@@ -20,13 +20,17 @@ def _tile_bins(L_T: int) -> int:
     return 4 * (1000 // L_T) if L_T <= 1000 else 1
 
 
-def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool = False):
-    """Returns (bin_cnt, words, scale, new_residue, g_max)."""
+def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool = False, factor: float = 0.0):
+    """Returns (bin_cnt, words, scale, new_residue, g_max).  `factor` other than 0 replaces the paper's
+    H = G + dW by H = residue + factor * dW (the scale-factor of Section 2.4; 1 = local selection only)."""
     n = len(dW)
     dW = [f32(x) for x in dW]
     residue = [f32(x) for x in residue]
     G = [f32(residue[i] + dW[i]) for i in range(n)]          # G <- residue + dW
-    H = [f32(G[i] + dW[i]) for i in range(n)]                # H <- G + dW
+    if factor == 0.0:
+        H = [f32(G[i] + dW[i]) for i in range(n)]            # H <- G + dW
+    else:
+        H = [f32(residue[i] + f32(f32(factor) * dW[i])) for i in range(n)]
     n_bins = -(-n // L_T)
     g_max = []
     for i in range(n_bins):                                  # over all bins
@@ -60,7 +64,7 @@ def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool 
 
 
 def to_stream(n: int, L_T: int, bin_cnt: Sequence[int], words: Sequence[int], scale,
-              literal: bool = False) -> bytes:
+              literal: bool = False, factor: float = 0.0) -> bytes:
     """Serialise to the wire layout: header, tile directory, bin counts, words."""
     w = 1 if L_T <= 64 else 2
     tb = _tile_bins(L_T)
@@ -74,7 +78,7 @@ def to_stream(n: int, L_T: int, bin_cnt: Sequence[int], words: Sequence[int], sc
     body += pad16(struct.pack(f"<{len(words)}{fmt}", *words))
     bytes_used = 64 + len(body)
     scale_bits = struct.unpack("<I", struct.pack("<f", float(scale)))[0]
-    head = struct.pack("<IHBBIIQQQQIIQ", 0x31434441, 1, w, 1 if literal else 0, L_T, tb, n, n_bins,
+    head = struct.pack("<IHBBIIQQQQIIQ", 0x31434441, 1, w, (1 if literal else 0) | (2 if factor != 0.0 else 0), L_T, tb, n, n_bins,
                        n_tiles, len(words), scale_bits, 0, bytes_used)
     return head + body
 
