@@ -151,6 +151,21 @@ int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t 
                         void *packed_out, uint64_t *count_out, void *stream, uint32_t flags);
 
 /*
+ * adacomp_compress with the scale-factor of the paper's self-adjusting selection (Section 2.4:
+ * an element is also sent when "its previous residue plus the latest gradient multiplied by a
+ * scale-factor exceeds the maximum of the bin"; 1.5 to 3.0 were studied, 2 was chosen).  The test
+ * value becomes H = residue + factor * dW, one rounded multiplication and one rounded addition in
+ * binary32; everything else (G, bin maxima, scale, forced bin maximum, quantisation, residue,
+ * stream layout) is as in adacomp_compress, which keeps Algorithm 2's H = G + dW with two additions
+ * (for factor 2 the two can differ in the last place).  factor = 1 makes H = G: only the bin maxima
+ * are sent, the "local selection" scheme without soft-threshold of Section 5.
+ *   factor   0 < factor <= 1e30, else ADACOMP_ERR_FLAGS.
+ * The stream's header carries bit 1 in its flags byte.  Runs at the speed of adacomp_compress.
+ */
+int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint32_t L_T,
+                            void *packed_out, uint64_t *count_out, void *stream, float factor);
+
+/*
  * unpack() of k learners' streams and their sum (Algorithm 1: unpack(), and the
  * summation inside averageGradients()).
  *   packed     HOST array of k device pointers to packed streams of one layer.

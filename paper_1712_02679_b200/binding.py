@@ -67,6 +67,9 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate_ex.restype = C.c_int
         L.adacomp_decompress_accumulate_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64,
                                                        C.c_uint32, C.c_void_p]
+        L.adacomp_compress_scaled.restype = C.c_int
+        L.adacomp_compress_scaled.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
+                                              C.c_void_p, C.c_float]
         L.adacomp_decompress_average_sgd.restype = C.c_int
         L.adacomp_decompress_average_sgd.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64,
                                                      C.c_uint32, C.c_float, C.c_float, C.c_void_p]
@@ -175,6 +178,14 @@ def adacomp_compress_ex(grad, residue, n: int, L_T: int, packed_out, count_out, 
                                      _dev_ptr(count_out, "count_out", torch.int64), _stream(stream),
                                      int(flags)),
            "adacomp_compress_ex")
+
+
+def adacomp_compress_scaled(grad, residue, n: int, L_T: int, packed_out, count_out, factor: float, stream=None) -> None:
+    """pack() with the selection's scale-factor: H = residue + factor * dW (factor 1: bin maxima only)."""
+    _check(lib().adacomp_compress_scaled(_dev_ptr(grad, "grad", torch.float32), _dev_ptr(residue, "residue", torch.float32),
+                                         int(n), int(L_T), _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                         _dev_ptr(count_out, "count_out", torch.int64), _stream(stream), C.c_float(factor)),
+           "adacomp_compress_scaled")
 
 
 def adacomp_decompress_accumulate(packed: Sequence[torch.Tensor], k_streams: int, dst,

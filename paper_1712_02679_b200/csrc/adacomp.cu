@@ -31,6 +31,7 @@ typedef unsigned long long u64;
 typedef unsigned int u32;
 
 constexpr u32 kMagic = 0x31434441u;
+constexpr u32 kFlagFactor = 2u;       // header flag (set by the library): the stream was made with a scale-factor
 constexpr u32 kHeaderBytes = 64;
 constexpr u32 kCtlBytes = 256;       // control block at the start of the scratch area
 constexpr int kWindows = 9;          // 32-bit windows of the exact g_max accumulator
@@ -307,6 +308,7 @@ struct PassArgs {
     Geometry geo;
     u32 literal;
     unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
+    float factor;               // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW (Section 2.4's scale-factor)
 };
 
 // Lazy-mode state: 64-byte header, then one u32 per 25-element segment (bit j = element j
@@ -459,7 +461,7 @@ tile_pass_fast(PassArgs a)
                     r = (prev >> j & 1u) ? fixed : r;
                 }
                 g[j] = __fadd_rn(r, d);
-                const float h = __fadd_rn(g[j], d);
+                const float h = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g[j], d);
                 m = fmaxf(m, fabsf(g[j]));
                 // |G| never exceeds the bin maximum, so "|H| >= g_max or |G| == g_max"
                 // is "max(|H|, |G|) >= g_max"
@@ -586,6 +588,7 @@ struct TileIo {                 // the buffers of one layer, as the generic tile
     float *residue;
     unsigned char *packed, *scratch;
     u32 literal;
+    float factor;               // as in PassArgs
 };
 
 template <typename Word>
@@ -610,8 +613,9 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     for (int i = tid; i < T; i += kGenericThreads) {
         float d = 0.f, r = 0.f;
         if (i < elems) { d = a.grad[base + i]; r = a.residue[base + i]; }
-        s_d[i] = d;
-        s_g[i] = __fadd_rn(r, d);
+        const float g = __fadd_rn(r, d);
+        s_g[i] = g;
+        s_d[i] = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g, d);      // H: dW is not needed again
     }
     __syncthreads();
 
@@ -627,7 +631,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
                 bool sel = false;
                 if (j < L) {
                     const float g = s_g[b * L + j];
-                    const float h = __fadd_rn(g, s_d[b * L + j]);
+                    const float h = s_d[b * L + j];
                     sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
                 }
                 count += __popc(__ballot_sync(0xffffffffu, sel));
@@ -662,7 +666,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
             float g = 0.f;
             if (j < L) {
                 g = s_g[b * L + j];
-                const float h = __fadd_rn(g, s_d[b * L + j]);
+                const float h = s_d[b * L + j];
                 sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
             }
             const u32 mask = __ballot_sync(0xffffffffu, sel);
@@ -696,7 +700,7 @@ tile_pass_generic(PassArgs a)
     const int tid = threadIdx.x;
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
-    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal};
+    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor};
     for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x)
         generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
     if (tid < kWindows) {
@@ -794,7 +798,7 @@ __device__ void finalize_body(unsigned char *packed, unsigned char *scratch, con
         u32 *h32 = reinterpret_cast<u32 *>(packed);
         u64 *h64 = reinterpret_cast<u64 *>(packed);
         h32[0] = kMagic;
-        h32[1] = 1u | (geo.w << 16) | ((flags & ADACOMP_FLAG_LITERAL) << 24);
+        h32[1] = 1u | (geo.w << 16) | ((flags & (ADACOMP_FLAG_LITERAL | kFlagFactor)) << 24);
         h32[2] = geo.L_T;
         h32[3] = geo.tile_bins;
         h64[2] = geo.n;
@@ -1062,7 +1066,7 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
             cur = li;
         }
         const BatchLayer &L = b.layer[li];
-        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u};
+        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, 0.f};
         if (L.geo.w == 1u) generic_tile<unsigned char>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
         else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
     }
@@ -2481,11 +2485,12 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
-                  void *lazy_state = nullptr)
+                  void *lazy_state = nullptr, float factor = 0.f)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
     if (flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
+    if (factor != 0.f && !(factor > 0.f && factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
     if (misaligned(grad) || misaligned(residue) || misaligned(packed_out) ||
         (reinterpret_cast<uintptr_t>(count_out) & 7u))
         return ADACOMP_ERR_ALIGN;
@@ -2493,7 +2498,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
     if (lazy) {
-        if ((L_T != 50u && L_T != 500u) || flags != 0) return ADACOMP_ERR_UNSUPPORTED;
+        if ((L_T != 50u && L_T != 500u) || flags != 0 || factor != 0.f) return ADACOMP_ERR_UNSUPPORTED;
         if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
     }
 
@@ -2512,7 +2517,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor};
         const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
         if (fast) {
             const u64 cap = (u64)info->sms * 2;
@@ -2532,7 +2537,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         }
     }
     mark(1);
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags, reinterpret_cast<u64 *>(count_out), lazy);
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags | (factor != 0.f ? kFlagFactor : 0u), reinterpret_cast<u64 *>(count_out), lazy);
     mark(2);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
@@ -2694,7 +2699,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     // must start from zero; tile counts and word slots are fully rewritten before they are read
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr};
+        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f};
         if ((L_T == 50u || L_T == 500u) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
@@ -2988,6 +2993,13 @@ int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_st
         if (rc != ADACOMP_OK) return rc;
     }
     return ADACOMP_OK;
+}
+
+int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                            uint64_t *count_out, void *stream, float factor)
+{
+    if (!(factor > 0.f && factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, nullptr, factor);
 }
 
 int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams, float *weights, float *momentum,

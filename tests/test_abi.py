@@ -85,6 +85,13 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     odd = (C.c_void_p * 1)(A + 2)
     assert g(odd, 1, A, None) == -3
     assert g(ptrs, 2, A + 4, None) == -3
+    sc = lib.adacomp_compress_scaled
+    assert sc(A, A, 10, 50, A, A, None, C.c_float(0.0)) == -6
+    assert sc(A, A, 10, 50, A, A, None, C.c_float(-1.5)) == -6
+    assert sc(A, A, 10, 50, A, A, None, C.c_float(float("nan"))) == -6
+    assert sc(None, A, 10, 50, A, A, None, C.c_float(1.5)) == -1
+    assert sc(A, A, 10, 0, A, A, None, C.c_float(1.5)) == -2
+    assert sc(A + 4, A, 10, 50, A, A, None, C.c_float(1.5)) == -3
     u = lib.adacomp_decompress_average_sgd
     lr, mu = C.c_float(0.1), C.c_float(0.9)
     assert u(ptrs, 2, None, A, 10, 50, lr, mu, None) == -1
