@@ -151,3 +151,17 @@ def average_sgd(streams: Sequence[np.ndarray], n: int, weights: np.ndarray, mome
     w_new = w[:n] - np.float32(lr) * v_new
     assert mean.dtype == v_new.dtype == w_new.dtype == np.float32
     return w_new, v_new
+
+
+def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) as float32 values: a bfloat16 is the upper half of a binary32, so the
+    conversion appends sixteen zero bits and is exact (NaNs keep their payload)."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def pack_bf16(dW_bits: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0, want_gmax: bool = False) -> Packed:
+    """pack() for a gradient that arrives in bfloat16 (the paper's motivation is reduced-precision
+    accelerators, Section 1; the residue, and all of Algorithm 2's arithmetic, stay binary32): the
+    gradient is widened exactly and Algorithm 2 runs as for any binary32 gradient."""
+    return pack(bf16_to_f32(dW_bits), residue, L_T, flags=flags, want_gmax=want_gmax)
