@@ -166,6 +166,18 @@ int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint3
                             void *packed_out, uint64_t *count_out, void *stream, float factor);
 
 /*
+ * adacomp_compress for a gradient that arrives in bfloat16 (the paper's setting is training on
+ * reduced-precision accelerators, Section 1; it fixes no format).  Each value is widened exactly
+ * to binary32 (a bfloat16 is the upper half of a binary32) as it is read, and Algorithm 2 then runs
+ * unchanged: the residue, the scale and the stream are what adacomp_compress gives for the widened
+ * gradient.  The call reads 2 bytes per element of gradient instead of 4.
+ *   grad_bf16   device, n bfloat16 values (uint16 bit patterns), 16-byte aligned; read-only.
+ * Other arguments, ownership and errors as for adacomp_compress.
+ */
+int adacomp_compress_bf16(const void *grad_bf16, float *residue, uint64_t n, uint32_t L_T,
+                          void *packed_out, uint64_t *count_out, void *stream);
+
+/*
  * unpack() of k learners' streams and their sum (Algorithm 1: unpack(), and the
  * summation inside averageGradients()).
  *   packed     HOST array of k device pointers to packed streams of one layer.

@@ -67,6 +67,9 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate_ex.restype = C.c_int
         L.adacomp_decompress_accumulate_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64,
                                                        C.c_uint32, C.c_void_p]
+        L.adacomp_compress_bf16.restype = C.c_int
+        L.adacomp_compress_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
+                                            C.c_void_p]
         L.adacomp_compress_scaled.restype = C.c_int
         L.adacomp_compress_scaled.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                               C.c_void_p, C.c_float]
@@ -178,6 +181,15 @@ def adacomp_compress_ex(grad, residue, n: int, L_T: int, packed_out, count_out, 
                                      _dev_ptr(count_out, "count_out", torch.int64), _stream(stream),
                                      int(flags)),
            "adacomp_compress_ex")
+
+
+def adacomp_compress_bf16(grad_bf16, residue, n: int, L_T: int, packed_out, count_out, stream=None) -> None:
+    """pack() of a bfloat16 gradient (widened exactly on load); residue and stream as for a binary32 gradient."""
+    _check(lib().adacomp_compress_bf16(_dev_ptr(grad_bf16, "grad_bf16", torch.bfloat16),
+                                       _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                       _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                       _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
+           "adacomp_compress_bf16")
 
 
 def adacomp_compress_scaled(grad, residue, n: int, L_T: int, packed_out, count_out, factor: float, stream=None) -> None:

@@ -121,6 +121,12 @@ __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
 
 __device__ inline void raise_status(u32 bits) { atomicOr(&g_status, bits); }
 
+// Element i of a gradient that is binary32, or bfloat16 widened exactly (sixteen zero bits appended).
+__device__ inline float load_grad(const float *grad, u64 i, u32 bf16)
+{
+    return bf16 ? __uint_as_float((u32)reinterpret_cast<const unsigned short *>(grad)[i] << 16) : grad[i];
+}
+
 __device__ inline u32 warp_inclusive_scan(u32 v, int lane)
 {
 #pragma unroll
@@ -309,6 +315,7 @@ struct PassArgs {
     u32 literal;
     unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
     float factor;               // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW (Section 2.4's scale-factor)
+    u32 grad_bf16;              // `grad` points to bfloat16 values (widened exactly on load)
 };
 
 // Lazy-mode state: 64-byte header, then one u32 per 25-element segment (bit j = element j
@@ -340,7 +347,8 @@ struct FastSmem {
 };
 static_assert(FastSmem::kAccAt % 8 == 0, "accumulator must be 8-byte aligned");
 
-template <int SPB, typename Word, bool LAZY>
+// BF16: the gradient arrives as bfloat16 (8000-byte tiles, widened as they are read).
+template <int SPB, typename Word, bool LAZY, bool BF16 = false>
 __global__ void __launch_bounds__(kFastThreads, 2)
 tile_pass_fast(PassArgs a)
 {
@@ -402,8 +410,9 @@ tile_pass_fast(PassArgs a)
         if (i >= my_tiles || tile >= full_tiles) return;
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        mbar_arrive_expect_tx(bar, 2 * kTileBytes + (LAZY ? kMaskBytes : 0u));
-        bulk_load(st, a.grad + tile * (u64)kFastTile, kTileBytes, bar);
+        constexpr u32 kGradBytes = BF16 ? kTileBytes / 2 : kTileBytes;
+        mbar_arrive_expect_tx(bar, kGradBytes + kTileBytes + (LAZY ? kMaskBytes : 0u));
+        bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)kGradBytes, kGradBytes, bar);
         bulk_load(st + kTileBytes, a.residue + tile * (u64)kFastTile, kTileBytes, bar);
         if (LAZY) bulk_load(st + 2 * kTileBytes, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
         issued = i + 1;
@@ -432,8 +441,9 @@ tile_pass_fast(PassArgs a)
             // the ragged last tile of the tensor: plain loads, zero fill past the end
             for (int e = tid; e < kFastTile; e += kFastThreads) {
                 float d = 0.f, r = 0.f;
-                if (e < elems) { d = a.grad[base + e]; r = a.residue[base + e]; }
-                s_d[e] = d;
+                if (e < elems) { d = load_grad(a.grad, base + e, BF16); r = a.residue[base + e]; }
+                if (BF16) reinterpret_cast<unsigned short *>(s_d)[e] = (unsigned short)(__float_as_uint(d) >> 16);
+                else s_d[e] = d;
                 s_r[e] = r;
             }
             if (LAZY && tid < kTileSegs)
@@ -450,9 +460,23 @@ tile_pass_fast(PassArgs a)
             const float *pr = s_r + tid * kSeg;
             float m = 0.f;
             const u32 prev = LAZY ? s_prev[tid] : 0u;
+            // bfloat16: the segment's 50 bytes start on a 4-byte boundary for even threads and two bytes
+            // past one for odd threads; thirteen aligned 32-bit loads cover them either way, and a funnel
+            // shift by 0 or 16 bits lines the pairs up (half as many shared-memory accesses as 25 16-bit loads)
+            u32 pair[BF16 ? 13 : 1];
+            if (BF16) {
+                const u32 *pw = reinterpret_cast<const u32 *>(s_d) + ((tid * kSeg) >> 1);
+                const u32 sh = (tid & 1) * 16u;
+                u32 w[14];
+#pragma unroll
+                for (int q = 0; q < 13; q++) w[q] = pw[q];
+                w[13] = 0;
+#pragma unroll
+                for (int q = 0; q < 13; q++) pair[q] = __funnelshift_r(w[q], w[q + 1], sh);    // elements 2q, 2q + 1
+            }
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
-                const float d = pd[j];
+                const float d = BF16 ? __uint_as_float((j & 1) ? pair[j >> 1] & 0xffff0000u : pair[j >> 1] << 16) : pd[j];
                 float r = pr[j];
                 if (LAZY) {
                     // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
@@ -589,6 +613,7 @@ struct TileIo {                 // the buffers of one layer, as the generic tile
     unsigned char *packed, *scratch;
     u32 literal;
     float factor;               // as in PassArgs
+    u32 grad_bf16;
 };
 
 template <typename Word>
@@ -612,7 +637,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
 
     for (int i = tid; i < T; i += kGenericThreads) {
         float d = 0.f, r = 0.f;
-        if (i < elems) { d = a.grad[base + i]; r = a.residue[base + i]; }
+        if (i < elems) { d = load_grad(a.grad, base + i, a.grad_bf16); r = a.residue[base + i]; }
         const float g = __fadd_rn(r, d);
         s_g[i] = g;
         s_d[i] = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g, d);      // H: dW is not needed again
@@ -700,7 +725,7 @@ tile_pass_generic(PassArgs a)
     const int tid = threadIdx.x;
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
-    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor};
+    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_bf16};
     for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x)
         generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
     if (tid < kWindows) {
@@ -1066,7 +1091,7 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
             cur = li;
         }
         const BatchLayer &L = b.layer[li];
-        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, 0.f};
+        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, 0.f, 0u};
         if (L.geo.w == 1u) generic_tile<unsigned char>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
         else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
     }
@@ -2441,7 +2466,9 @@ int device_info(DeviceInfo *&out)
         d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
                        cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false>, at, bytes) == cudaSuccess &&
                        cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, true>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, true>, at, bytes) == cudaSuccess;
+                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, true>, at, bytes) == cudaSuccess &&
+                       cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false, true>, at, bytes) == cudaSuccess &&
+                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false, true>, at, bytes) == cudaSuccess;
         if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kBatchSmemBytes) == cudaSuccess &&
             cudaFuncSetAttribute(batch_tile_pass<kBatchSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -2485,7 +2512,7 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
-                  void *lazy_state = nullptr, float factor = 0.f)
+                  void *lazy_state = nullptr, float factor = 0.f, bool grad_bf16 = false)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
@@ -2498,7 +2525,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
     if (lazy) {
-        if ((L_T != 50u && L_T != 500u) || flags != 0 || factor != 0.f) return ADACOMP_ERR_UNSUPPORTED;
+        if ((L_T != 50u && L_T != 500u) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
         if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
     }
 
@@ -2517,7 +2544,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_bf16 ? 1u : 0u};
         const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
         if (fast) {
             const u64 cap = (u64)info->sms * 2;
@@ -2526,6 +2553,9 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
             if (lazy) {
                 if (L_T == 50u) tile_pass_fast<2, unsigned char, true><<<grid, kFastThreads, sm, st>>>(args);
                 else tile_pass_fast<20, unsigned short, true><<<grid, kFastThreads, sm, st>>>(args);
+            } else if (grad_bf16) {
+                if (L_T == 50u) tile_pass_fast<2, unsigned char, false, true><<<grid, kFastThreads, sm, st>>>(args);
+                else tile_pass_fast<20, unsigned short, false, true><<<grid, kFastThreads, sm, st>>>(args);
             } else {
                 if (L_T == 50u) tile_pass_fast<2, unsigned char, false><<<grid, kFastThreads, sm, st>>>(args);
                 else tile_pass_fast<20, unsigned short, false><<<grid, kFastThreads, sm, st>>>(args);
@@ -2699,7 +2729,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     // must start from zero; tile counts and word slots are fully rewritten before they are read
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f};
+        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f, 0u};
         if ((L_T == 50u || L_T == 500u) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
@@ -2993,6 +3023,13 @@ int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_st
         if (rc != ADACOMP_OK) return rc;
     }
     return ADACOMP_OK;
+}
+
+int adacomp_compress_bf16(const void *grad_bf16, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                          uint64_t *count_out, void *stream)
+{
+    return compress_impl(static_cast<const float *>(grad_bf16), residue, n, L_T, packed_out, count_out, stream, 0, nullptr,
+                         nullptr, 0.f, true);
 }
 
 int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,

@@ -85,6 +85,10 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     odd = (C.c_void_p * 1)(A + 2)
     assert g(odd, 1, A, None) == -3
     assert g(ptrs, 2, A + 4, None) == -3
+    hb = lib.adacomp_compress_bf16
+    assert hb(None, A, 10, 50, A, A, None) == -1
+    assert hb(A, A, 10, 0, A, A, None) == -2
+    assert hb(A + 2, A, 10, 50, A, A, None) == -3
     sc = lib.adacomp_compress_scaled
     assert sc(A, A, 10, 50, A, A, None, C.c_float(0.0)) == -6
     assert sc(A, A, 10, 50, A, A, None, C.c_float(-1.5)) == -6
