@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--no-lazy", action="store_true")
     ap.add_argument("--no-update", action="store_true", help="skip the fused unpack + average + SGD measurement")
     ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4", "lstm"],
                     help="sweep: flat tensor of 2^log2n (the default bench); configN: the multi-tensor "
                          "parameter lists, through the *_multi entry points")
     return ap.parse_args()
@@ -519,9 +519,10 @@ def run_multi_workload(a):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
-    cfg = int(a.workload[-1])
+    cfg = 6 if a.workload == "lstm" else int(a.workload[-1])
     specs, learners = {1: (synth.config1_tensors(), 1), 2: (synth.config2_tensors(), 1),
-                       3: (synth.resnet50_tensors(), 8), 4: (synth.config4_tensors(), 16)}[cfg]
+                       3: (synth.resnet50_tensors(), 8), 4: (synth.config4_tensors(), 16),
+                       6: (synth.lstm_tensors(), 8)}[cfg]
     nl, total = len(specs), sum(s.n for s in specs)
     gen = torch.Generator(device=dev)
     gen.manual_seed(1712_02679 + cfg)
@@ -560,7 +561,7 @@ def run_multi_workload(a):
         "metric": METRIC, "value": 4.0 * total * learners / ((t_c + t_d) * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1,
         "steps": K, "warmup": W, "ms_per_step": t_c + t_d, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"config {cfg}: {nl} tensors, {total} elements, {learners} learners, first step "
+        "config": {"workload": f"{'LSTM list (67-512-512-67)' if cfg == 6 else 'config ' + str(cfg)}: {nl} tensors, {total} elements, {learners} learners, first step "
                                f"from a zero residue, dW~N(0,1e-3); *_multi entry points",
                    "l2": "working set %.0f MB" % (12.0 * total * learners / 1e6)},
         "compress_ms": t_c, "compress_gbs": 4.0 * total * learners / (t_c * 1e-3) / 1e9,

@@ -118,6 +118,22 @@ def config4_tensors(hidden: int = 2048) -> List[TensorSpec]:
             for i in range(len(dims) - 1)]
 
 
+def lstm_tensors(vocab: int = 67, hidden: int = 512) -> List[TensorSpec]:
+    """Character-level LSTM of the paper's model list: two LSTM layers (67 -> 512, 512 -> 512) and a fully
+    connected layer (512 -> 67).  The paper names the layers by their input and output widths; the tensors
+    here are the gate-stacked matrices a framework keeps for them (input-to-hidden and hidden-to-hidden
+    weights of four gates, their biases) and the output layer with its bias, all with the bin length the
+    paper uses for LSTM and fully connected layers."""
+    out = []
+    for i, width in enumerate((vocab, hidden)):
+        out += [TensorSpec(f"lstm{i}_w_ih_{4 * hidden}x{width}", 4 * hidden * width, 500, "lstm"),
+                TensorSpec(f"lstm{i}_w_hh_{4 * hidden}x{hidden}", 4 * hidden * hidden, 500, "lstm"),
+                TensorSpec(f"lstm{i}_b_ih", 4 * hidden, 500, "lstm"),
+                TensorSpec(f"lstm{i}_b_hh", 4 * hidden, 500, "lstm")]
+    out += [TensorSpec(f"fc_{vocab}x{hidden}", vocab * hidden, 500, "fc"), TensorSpec("fc_bias", vocab, 500, "fc")]
+    return out
+
+
 def config5_sizes() -> List[int]:
     """Flat gradient sizes of the bandwidth sweep: 2^20 ... 2^30 in 4x steps."""
     return [1 << (20 + 2 * j) for j in range(6)]

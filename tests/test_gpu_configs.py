@@ -87,6 +87,12 @@ def test_config4_speech_dnn_sixteen_learners():
     _multi_tensor_case(4, specs, learners=16, heavy_sigma=1e-3)
 
 
+def test_lstm_parameter_list_eight_learners():
+    specs = synth.lstm_tensors()
+    assert len(specs) == 10 and sum(s.n for s in specs) == 2048 * (67 + 512 + 512 + 512) + 4 * 2048 + 67 * 512 + 67
+    _multi_tensor_case(6, specs, learners=8)
+
+
 @pytest.mark.parametrize("L_T", [50, 500])
 @pytest.mark.parametrize("log2n", [20, 22, 24])
 def test_config5_sweep_point_prewarmed_eager_and_lazy(L_T, log2n):
