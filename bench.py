@@ -554,6 +554,20 @@ def run_multi_workload(a):
         if it >= W:
             evs.append(e)
     torch.cuda.synchronize()
+    # the same streams, averaged and applied to weights and momentum in one call
+    wts = [torch.randn(max(s.n, 4), device=dev) for s in specs]
+    mom = [torch.zeros(max(s.n, 4), device=dev) for s in specs]
+    w_arr, m_arr = B.make_pointer_array(wts, torch.float32), B.make_pointer_array(mom, torch.float32)
+    evf = []
+    for it in range(W + K):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        e[0].record()
+        B.adacomp_decompress_average_sgd_multi(packed, learners, w_arr, m_arr, ns, lts, nl, 0.1, 0.9)
+        e[1].record()
+        if it >= W:
+            evf.append(e)
+    torch.cuda.synchronize()
+    t_f = statistics.mean(e[0].elapsed_time(e[1]) for e in evf)
     t_c = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     t_d = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     n_sel = sum(int(d["count_out"][0]) for d in layers[:nl])
@@ -565,7 +579,7 @@ def run_multi_workload(a):
                                f"from a zero residue, dW~N(0,1e-3); *_multi entry points",
                    "l2": "working set %.0f MB" % (12.0 * total * learners / 1e6)},
         "compress_ms": t_c, "compress_gbs": 4.0 * total * learners / (t_c * 1e-3) / 1e9,
-        "decompress_sum_ms": t_d, "decompress_sum_gbs": 4.0 * total / (t_d * 1e-3) / 1e9,
+        "decompress_sum_ms": t_d, "fused_update_ms": t_f, "decompress_sum_gbs": 4.0 * total / (t_d * 1e-3) / 1e9,
         "selected_fraction_learner0": n_sel / max(total, 1), "device_status": B.adacomp_device_status(),
     }
     print(json.dumps(line), flush=True)

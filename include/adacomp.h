@@ -225,6 +225,21 @@ int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams
                                    float *momentum, uint64_t n, uint32_t L_T, float lr, float mu,
                                    void *stream);
 
+/*
+ * adacomp_decompress_average_sgd for a list of layers (a model's parameter list) in one call, as
+ * adacomp_decompress_accumulate_multi_ex is to adacomp_decompress_accumulate_ex: small layers of
+ * the paper's bin lengths share launches, the others take the single-layer kernels.
+ *   packed     HOST array of n_layers * k_streams device pointers, packed[t * k_streams + l] =
+ *              learner l's stream of layer t.
+ *   weights, momentum   HOST arrays of n_layers device pointers (float[n[t]] each), updated in place.
+ *   n, L_T     HOST arrays of n_layers shapes.
+ * One learning rate and one momentum coefficient serve every layer of the call.
+ */
+int adacomp_decompress_average_sgd_multi(const void *const *packed, uint32_t k_streams,
+                                         float *const *weights, float *const *momentum,
+                                         const uint64_t *n, const uint32_t *L_T, uint32_t n_layers,
+                                         float lr, float mu, void *stream);
+
 /* adacomp_decompress_accumulate_multi with the layers' shapes (HOST arrays n[n_layers], L_T[n_layers]). */
 int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams,
                                            float *const *dst, const uint64_t *n, const uint32_t *L_T,

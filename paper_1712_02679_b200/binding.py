@@ -67,6 +67,9 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_accumulate_ex.restype = C.c_int
         L.adacomp_decompress_accumulate_ex.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64,
                                                        C.c_uint32, C.c_void_p]
+        L.adacomp_decompress_average_sgd_multi.restype = C.c_int
+        L.adacomp_decompress_average_sgd_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                           C.c_void_p, C.c_uint32, C.c_float, C.c_float, C.c_void_p]
         L.adacomp_compress_bf16.restype = C.c_int
         L.adacomp_compress_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p]
@@ -230,6 +233,22 @@ def adacomp_decompress_average_sgd(packed: Sequence[torch.Tensor], k_streams: in
                                                 _dev_ptr(momentum, "momentum", torch.float32), int(n), int(L_T),
                                                 C.c_float(lr), C.c_float(mu), _stream(stream)),
            "adacomp_decompress_average_sgd")
+
+
+def adacomp_decompress_average_sgd_multi(packed, k_streams: int, weights, momentum, n: Sequence[int],
+                                         L_T: Sequence[int], n_layers: int, lr: float, mu: float, stream=None) -> None:
+    """adacomp_decompress_average_sgd for a list of layers; weights[t] and momentum[t] are updated in place."""
+    if not isinstance(packed, C.Array):
+        packed = make_pointer_array(packed, torch.uint8)
+    if not isinstance(weights, C.Array):
+        weights = make_pointer_array(weights, torch.float32)
+    if not isinstance(momentum, C.Array):
+        momentum = make_pointer_array(momentum, torch.float32)
+    ns = (C.c_uint64 * max(int(n_layers), 1))(*[int(v) for v in n[:n_layers]])
+    lts = (C.c_uint32 * max(int(n_layers), 1))(*[int(v) for v in L_T[:n_layers]])
+    _check(lib().adacomp_decompress_average_sgd_multi(packed, int(k_streams), weights, momentum, ns, lts, int(n_layers),
+                                                      C.c_float(lr), C.c_float(mu), _stream(stream)),
+           "adacomp_decompress_average_sgd_multi")
 
 
 def adacomp_decompress_accumulate_multi_ex(packed, k_streams: int, dst, n: Sequence[int],

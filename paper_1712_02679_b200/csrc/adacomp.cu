@@ -2314,7 +2314,10 @@ struct DecodeBatchArgs {
     u32 n_layers, k;
     u64 n[kDecBatchLayers];
     u32 L_T[kDecBatchLayers];
-    float *dst[kDecBatchLayers];
+    float *dst[kDecBatchLayers];                     // the layer's output; with `sgd` its weights
+    float *aux[kDecBatchLayers];                     // with `sgd`: its momentum
+    float lr, mu;
+    u32 sgd;                                         // the optimizer step takes the place of the store (see Epilogue)
     const unsigned char *stream[kDecBatchPtrs];      // [layer * k + learner]
 };
 
@@ -2359,7 +2362,6 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
     }
     consumer_barrier();
     const u32 total = sm.first[b.n_layers];
-    const Epilogue no_ep = {nullptr, nullptr, 0.f, 0.f, 0.f};
     for (u32 gt = blockIdx.x; gt < total; gt += gridDim.x) {
         int lo = 0, hi = (int)b.n_layers;            // largest t with first[t] <= gt and a tile of its own
         while (hi - lo > 1) {
@@ -2369,12 +2371,13 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
         const Geometry &geo = sm.geo[lo];
         const u64 tile = gt - sm.first[lo];
         const unsigned char *const *streams = &b.stream[lo * b.k];
+        const Epilogue ep = {b.sgd ? b.dst[lo] : nullptr, b.sgd ? b.aux[lo] : nullptr, b.lr, b.mu, (float)b.k};
         if (geo.w == 1u) {
-            decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
+            decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], ep, sm.d, bad);
         } else if (geo.tile_bins >= 32) {
-            decode_item_staged<unsigned short, true>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
+            decode_item_staged<unsigned short, true>(streams, b.k, geo, tile, b.dst[lo], ep, sm.d, bad);
         } else {
-            decode_item_staged<unsigned short, false>(streams, b.k, geo, tile, b.dst[lo], no_ep, sm.d, bad);
+            decode_item_staged<unsigned short, false>(streams, b.k, geo, tile, b.dst[lo], ep, sm.d, bad);
         }
     }
     if (bad && blockIdx.x == 0) raise_status(bad & ADACOMP_DEV_HEADER_MISMATCH);
@@ -2822,15 +2825,17 @@ int adacomp_decompress_accumulate_ex(const void *const *packed, uint32_t k_strea
     return decompress_impl(packed, k_streams, dst, stream, n, L_T);
 }
 
-int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams, float *const *dst,
-                                           const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream)
+// Decode-sum of a list of layers whose shapes the caller knows.  `aux` (optional): the layers' momentum
+// arrays; `dst` then holds their weights and every layer gets the optimizer step instead of a store.
+int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *const *dst, float *const *aux,
+                          const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream, float lr, float mu)
 {
     if (n_layers && (!packed || !dst || !n || !L_T)) return ADACOMP_ERR_NULL;
     if (k_streams == 0 || k_streams > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
     for (uint32_t t = 0; t < n_layers; t++) {
         if (L_T[t] == 0 || L_T[t] > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-        if (!dst[t]) return ADACOMP_ERR_NULL;
-        if (misaligned(dst[t])) return ADACOMP_ERR_ALIGN;
+        if (!dst[t] || (aux && !aux[t])) return ADACOMP_ERR_NULL;
+        if (misaligned(dst[t]) || (aux && misaligned(aux[t]))) return ADACOMP_ERR_ALIGN;
         for (uint32_t l = 0; l < k_streams; l++) {
             if (!packed[(size_t)t * k_streams + l]) return ADACOMP_ERR_NULL;
             if (misaligned(packed[(size_t)t * k_streams + l])) return ADACOMP_ERR_ALIGN;
@@ -2845,6 +2850,9 @@ int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k
     static thread_local DecodeBatchArgs batch;
     batch.n_layers = 0;
     batch.k = k_streams;
+    batch.sgd = aux ? 1u : 0u;
+    batch.lr = lr;
+    batch.mu = mu;
     u64 batch_tiles = 0;
     auto flush = [&]() -> int {
         if (batch.n_layers == 0) return ADACOMP_OK;
@@ -2865,6 +2873,7 @@ int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k
             batch.n[i] = n[t];
             batch.L_T[i] = L_T[t];
             batch.dst[i] = dst[t];
+            batch.aux[i] = aux ? aux[t] : nullptr;
             for (uint32_t l = 0; l < k_streams; l++)
                 batch.stream[(size_t)i * k_streams + l] = static_cast<const unsigned char *>(packed[(size_t)t * k_streams + l]);
             batch_tiles += decode_items(n[t], L_T[t]);
@@ -2872,12 +2881,30 @@ int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k
                 rc = flush();
                 if (rc != ADACOMP_OK) return rc;
             }
+        } else if (aux) {
+            const Epilogue ep = {dst[t], aux[t], lr, mu, 0.f};
+            rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, nullptr, stream, n[t], L_T[t], &ep);
+            if (rc != ADACOMP_OK) return rc;
         } else {
             rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, dst[t], stream, n[t], L_T[t]);
             if (rc != ADACOMP_OK) return rc;
         }
     }
     return flush();
+}
+
+int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams, float *const *dst,
+                                           const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream)
+{
+    return decompress_multi_impl(packed, k_streams, dst, nullptr, n, L_T, n_layers, stream, 0.f, 0.f);
+}
+
+int adacomp_decompress_average_sgd_multi(const void *const *packed, uint32_t k_streams, float *const *weights,
+                                         float *const *momentum, const uint64_t *n, const uint32_t *L_T,
+                                         uint32_t n_layers, float lr, float mu, void *stream)
+{
+    if (n_layers && !momentum) return ADACOMP_ERR_NULL;
+    return decompress_multi_impl(packed, k_streams, weights, momentum, n, L_T, n_layers, stream, lr, mu);
 }
 
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,

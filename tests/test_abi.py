@@ -85,6 +85,13 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     odd = (C.c_void_p * 1)(A + 2)
     assert g(odd, 1, A, None) == -3
     assert g(ptrs, 2, A + 4, None) == -3
+    um = lib.adacomp_decompress_average_sgd_multi
+    one64, one32 = (C.c_uint64 * 1)(10), (C.c_uint32 * 1)(50)
+    wl, bad_w = (C.c_void_p * 1)(A), (C.c_void_p * 1)(A + 4)
+    assert um(ptrs, 2, wl, None, one64, one32, 1, lr, mu, None) == -1
+    assert um(ptrs, 2, bad_w, wl, one64, one32, 1, lr, mu, None) == -3
+    assert um(ptrs, 2, wl, wl, one64, (C.c_uint32 * 1)(0), 1, lr, mu, None) == -2
+    assert um(None, 2, None, None, None, None, 0, lr, mu, None) == 0
     hb = lib.adacomp_compress_bf16
     assert hb(None, A, 10, 50, A, A, None) == -1
     assert hb(A, A, 10, 0, A, A, None) == -2

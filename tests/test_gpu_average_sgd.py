@@ -83,3 +83,33 @@ def test_wrong_shape_leaves_the_arrays_alone_and_sets_a_status_bit():
     np.testing.assert_array_equal(got_w, w)
     np.testing.assert_array_equal(got_v, v)
     B.adacomp_device_status_reset()
+
+
+def test_layer_list_in_one_call_matches_per_layer_oracle():
+    """Small layers share a batched launch, the large ones take the single-layer kernels; bin lengths mixed."""
+    rng = np.random.default_rng(6)
+    shapes = [(864, 500), (9216, 500), (5120, 50), (4000 * 1100 + 7, 50), (147456, 500), (67, 500), (2048, 50),
+              (4000 * 1060, 500), (100, 7)]
+    k = 3
+    dev = torch.device("cuda:0")
+    streams_cpu, bufs, ws, vs, w_dev, v_dev = [], [], [], [], [], []
+    for n, L_T in shapes:
+        layer_streams = _streams(rng, n, L_T, k)
+        streams_cpu.append(layer_streams)
+        bufs += [torch.from_numpy(s.copy()).to(dev) for s in layer_streams]
+        w = rng.normal(0, 1, n).astype(np.float32)
+        v = rng.normal(0, 1e-2, n).astype(np.float32)
+        ws.append(w)
+        vs.append(v)
+        w_dev.append(torch.from_numpy(np.concatenate([w, np.full(4, 7.0, np.float32)])).to(dev))
+        v_dev.append(torch.from_numpy(np.concatenate([v, np.full(4, -7.0, np.float32)])).to(dev))
+    B.adacomp_decompress_average_sgd_multi(bufs, k, w_dev, v_dev, [n for n, _ in shapes], [L for _, L in shapes],
+                                           len(shapes), 0.1, 0.9)
+    torch.cuda.synchronize()
+    for t, (n, L_T) in enumerate(shapes):
+        want_w, want_v = cref.average_sgd(streams_cpu[t], n, ws[t], vs[t], 0.1, 0.9)
+        got_w, got_v = w_dev[t].cpu().numpy(), v_dev[t].cpu().numpy()
+        assert np.all(got_w[n:] == 7.0) and np.all(got_v[n:] == -7.0), f"layer {t}: wrote past the layer"
+        assert_f32_bits_equal(got_v[:n], want_v, f"momentum layer {t} n={n} L_T={L_T}")
+        assert_f32_bits_equal(got_w[:n], want_w, f"weights layer {t} n={n} L_T={L_T}")
+    assert B.adacomp_device_status() == 0
