@@ -86,6 +86,7 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert g(odd, 1, A, None) == -3
     assert g(ptrs, 2, A + 4, None) == -3
     um = lib.adacomp_decompress_average_sgd_multi
+    lr, mu = C.c_float(0.1), C.c_float(0.9)
     one64, one32 = (C.c_uint64 * 1)(10), (C.c_uint32 * 1)(50)
     wl, bad_w = (C.c_void_p * 1)(A), (C.c_void_p * 1)(A + 4)
     assert um(ptrs, 2, wl, None, one64, one32, 1, lr, mu, None) == -1
