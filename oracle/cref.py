@@ -165,3 +165,33 @@ def pack_bf16(dW_bits: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0
     accelerators, Section 1; the residue, and all of Algorithm 2's arithmetic, stay binary32): the
     gradient is widened exactly and Algorithm 2 runs as for any binary32 gradient."""
     return pack(bf16_to_f32(dW_bits), residue, L_T, flags=flags, want_gmax=want_gmax)
+
+
+def average_adam(streams: Sequence[np.ndarray], n: int, weights: np.ndarray, m: np.ndarray, v: np.ndarray,
+                 step_size: float, beta1: float, beta2: float, eps: float):
+    """unpack(), averageGradients() and an Adam step for one layer (the paper reports AdaComp with Adam too,
+    Section "Experiments"; it prints no formula).  The step is Kingma and Ba's Algorithm 1 in the order
+    its Section 2 suggests for efficiency, every operation rounded to binary32 on its own:
+
+        mean = s / k
+        m'   = (beta1 * m) + ((1 - beta1) * mean)
+        v'   = (beta2 * v) + ((1 - beta2) * (mean * mean))
+        w'   = w - ((step_size * m') / (sqrt(v') + eps))
+
+    with 1 - beta computed in binary32 and step_size = alpha * sqrt(1 - beta2^t) / (1 - beta1^t) supplied by the
+    caller (the bias correction belongs to the training loop, which knows t).  Returns (w', m', v')."""
+    k = len(streams)
+    f = np.float32
+    w = np.ascontiguousarray(weights, dtype=np.float32)[:n]
+    m0 = np.ascontiguousarray(m, dtype=np.float32)[:n]
+    v0 = np.ascontiguousarray(v, dtype=np.float32)[:n]
+    s = unpack_sum(streams, n)
+    mean = s / f(k)
+    c1 = f(1) - f(beta1)
+    c2 = f(1) - f(beta2)
+    m_new = f(beta1) * m0 + c1 * mean
+    v_new = f(beta2) * v0 + c2 * (mean * mean)
+    den = np.sqrt(v_new) + f(eps)
+    w_new = w - (f(step_size) * m_new) / den
+    assert m_new.dtype == v_new.dtype == w_new.dtype == den.dtype == np.float32
+    return w_new, m_new, v_new
