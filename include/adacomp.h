@@ -240,6 +240,31 @@ int adacomp_decompress_average_sgd_multi(const void *const *packed, uint32_t k_s
                                          const uint64_t *n, const uint32_t *L_T, uint32_t n_layers,
                                          float lr, float mu, void *stream);
 
+/*
+ * As adacomp_decompress_average_sgd, with an Adam step in place of the SGD step (the paper reports
+ * AdaComp with Adam as well, Section "Experiments", and prints no formula).  The step is Kingma and
+ * Ba's Algorithm 1 in the order its Section 2 suggests, every operation rounded to binary32 on its
+ * own (IEEE division and square root, no fused multiply-add):
+ *     mean = s / k
+ *     m'   = (beta1 * m) + ((1 - beta1) * mean)
+ *     v'   = (beta2 * v) + ((1 - beta2) * (mean * mean))
+ *     w'   = w - ((step_size * m') / (sqrt(v') + eps))
+ *   weights, m, v   device, float[n] each, read and written in place (v must be >= 0).
+ *   step_size       alpha * sqrt(1 - beta2^t) / (1 - beta1^t): the bias correction is the caller's,
+ *                   who knows the step count t.
+ *   eps             > 0.
+ * Everything else as for adacomp_decompress_average_sgd; the _multi form takes a list of layers as
+ * adacomp_decompress_average_sgd_multi does.
+ */
+int adacomp_decompress_average_adam(const void *const *packed, uint32_t k_streams, float *weights,
+                                    float *m, float *v, uint64_t n, uint32_t L_T, float step_size,
+                                    float beta1, float beta2, float eps, void *stream);
+int adacomp_decompress_average_adam_multi(const void *const *packed, uint32_t k_streams,
+                                          float *const *weights, float *const *m, float *const *v,
+                                          const uint64_t *n, const uint32_t *L_T, uint32_t n_layers,
+                                          float step_size, float beta1, float beta2, float eps,
+                                          void *stream);
+
 /* adacomp_decompress_accumulate_multi with the layers' shapes (HOST arrays n[n_layers], L_T[n_layers]). */
 int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams,
                                            float *const *dst, const uint64_t *n, const uint32_t *L_T,

@@ -70,6 +70,13 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_average_sgd_multi.restype = C.c_int
         L.adacomp_decompress_average_sgd_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                                            C.c_void_p, C.c_uint32, C.c_float, C.c_float, C.c_void_p]
+        L.adacomp_decompress_average_adam.restype = C.c_int
+        L.adacomp_decompress_average_adam.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64,
+                                                      C.c_uint32, C.c_float, C.c_float, C.c_float, C.c_float, C.c_void_p]
+        L.adacomp_decompress_average_adam_multi.restype = C.c_int
+        L.adacomp_decompress_average_adam_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                            C.c_void_p, C.c_void_p, C.c_uint32, C.c_float, C.c_float,
+                                                            C.c_float, C.c_float, C.c_void_p]
         L.adacomp_compress_bf16.restype = C.c_int
         L.adacomp_compress_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p]
@@ -233,6 +240,33 @@ def adacomp_decompress_average_sgd(packed: Sequence[torch.Tensor], k_streams: in
                                                 _dev_ptr(momentum, "momentum", torch.float32), int(n), int(L_T),
                                                 C.c_float(lr), C.c_float(mu), _stream(stream)),
            "adacomp_decompress_average_sgd")
+
+
+def adacomp_decompress_average_adam(packed: Sequence[torch.Tensor], k_streams: int, weights, m, v, n: int, L_T: int,
+                                    step_size: float, beta1: float, beta2: float, eps: float, stream=None) -> None:
+    """unpack(), averageGradients() and an Adam step in one pass; weights, m and v are updated in place."""
+    ptrs = (C.c_void_p * max(int(k_streams), 1))(
+        *[_dev_ptr(p, "packed[l]", torch.uint8) for p in packed[:k_streams]])
+    _check(lib().adacomp_decompress_average_adam(ptrs, int(k_streams), _dev_ptr(weights, "weights", torch.float32),
+                                                 _dev_ptr(m, "m", torch.float32), _dev_ptr(v, "v", torch.float32),
+                                                 int(n), int(L_T), C.c_float(step_size), C.c_float(beta1),
+                                                 C.c_float(beta2), C.c_float(eps), _stream(stream)),
+           "adacomp_decompress_average_adam")
+
+
+def adacomp_decompress_average_adam_multi(packed, k_streams: int, weights, m, v, n: Sequence[int], L_T: Sequence[int],
+                                          n_layers: int, step_size: float, beta1: float, beta2: float, eps: float,
+                                          stream=None) -> None:
+    """adacomp_decompress_average_adam for a list of layers."""
+    if not isinstance(packed, C.Array):
+        packed = make_pointer_array(packed, torch.uint8)
+    arrs = [a if isinstance(a, C.Array) else make_pointer_array(a, torch.float32) for a in (weights, m, v)]
+    ns = (C.c_uint64 * max(int(n_layers), 1))(*[int(x) for x in n[:n_layers]])
+    lts = (C.c_uint32 * max(int(n_layers), 1))(*[int(x) for x in L_T[:n_layers]])
+    _check(lib().adacomp_decompress_average_adam_multi(packed, int(k_streams), arrs[0], arrs[1], arrs[2], ns, lts,
+                                                       int(n_layers), C.c_float(step_size), C.c_float(beta1),
+                                                       C.c_float(beta2), C.c_float(eps), _stream(stream)),
+           "adacomp_decompress_average_adam_multi")
 
 
 def adacomp_decompress_average_sgd_multi(packed, k_streams: int, weights, momentum, n: Sequence[int],

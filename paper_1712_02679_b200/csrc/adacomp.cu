@@ -1128,34 +1128,62 @@ batch_gather(const __grid_constant__ BatchArgsT<N> b)
 // ---------------------------------------------------------------------------------
 
 // What becomes of a finished tile of the ordered sum s: stored to dst (unpack() alone), or, with
-// `weights` set, averageGradients() and updateWeights() of Algorithm 1 on the spot:
-//     mean = s / k,  v' = (mu * v) + mean,  w' = w - (lr * v'),
-// every operation rounded to binary32 on its own (the paper names "SGD with momentum" and prints
-// no formula: this is the plain heavy-ball step).  The dense gradient then never reaches memory.
+// `weights` set, averageGradients() and updateWeights() of Algorithm 1 on the spot, every operation
+// rounded to binary32 on its own, so that the dense gradient never reaches memory.  The paper
+// names its optimizers ("SGD with momentum", Adam) and prints no formula:
+//   SGD (adam == 0): the plain heavy-ball step
+//       mean = s / k,  v' = (mu * v) + mean,  w' = w - (lr * v')
+//   Adam (adam != 0): Kingma and Ba's Algorithm 1 in its "efficient" order; `momentum` is the first
+//       moment m, `second` the second moment v, `mu` beta1, `lr` the bias-corrected step size
+//       alpha * sqrt(1 - beta2^t) / (1 - beta1^t), which the caller computes
+//       mean = s / k,  m' = (beta1 * m) + ((1 - beta1) * mean),  v' = (beta2 * v) + ((1 - beta2) * (mean * mean)),
+//       w' = w - ((lr * m') / (sqrt(v') + eps))
 struct Epilogue {
-    float *weights, *momentum;
-    float lr, mu, k;
+    float *weights, *momentum, *second;
+    float lr, mu, beta2, eps, k;
+    u32 adam;
 };
 
-// (s / k without the division where the quotient is known without it: a zero sum, which is what
+// s / k without the division where the quotient is known without it: a zero sum, which is what
 // most elements have, stays the same zero; for k a power of two the product with 1 / k is the
-// correctly rounded quotient too.)
+// correctly rounded quotient too.
+__device__ inline float mean_of(float s, float k)
+{
+    const bool pow2 = (__float_as_uint(k) & 0x007fffffu) == 0u;
+    return s == 0.f ? s : pow2 ? __fmul_rn(s, __frcp_rn(k)) : __fdiv_rn(s, k);
+}
+
 __device__ inline void sgd_step(float s, float &w, float &v, const Epilogue &ep)
 {
-    const bool pow2 = (__float_as_uint(ep.k) & 0x007fffffu) == 0u;
-    const float mean = s == 0.f ? s : pow2 ? __fmul_rn(s, __frcp_rn(ep.k)) : __fdiv_rn(s, ep.k);
+    const float mean = mean_of(s, ep.k);
     v = __fadd_rn(__fmul_rn(ep.mu, v), mean);
     w = __fsub_rn(w, __fmul_rn(ep.lr, v));
+}
+
+__device__ inline void adam_step(float s, float &w, float &m, float &v, const Epilogue &ep)
+{
+    const float mean = mean_of(s, ep.k);
+    m = __fadd_rn(__fmul_rn(ep.mu, m), __fmul_rn(__fsub_rn(1.f, ep.mu), mean));
+    v = __fadd_rn(__fmul_rn(ep.beta2, v), __fmul_rn(__fsub_rn(1.f, ep.beta2), __fmul_rn(mean, mean)));
+    const float num = __fmul_rn(ep.lr, m), den = __fadd_rn(__fsqrt_rn(v), ep.eps);
+    w = __fsub_rn(w, num == 0.f ? num : __fdiv_rn(num, den));      // (0 / den is that zero: den > 0 for eps > 0)
 }
 
 // Four elements at once.
 __device__ inline void sgd_step4(float4 s, float4 &w, float4 &v, float lr, float mu, float k)
 {
-    const Epilogue ep = {nullptr, nullptr, lr, mu, k};
+    const Epilogue ep = {nullptr, nullptr, nullptr, lr, mu, 0.f, 0.f, k, 0u};
     sgd_step(s.x, w.x, v.x, ep);
     sgd_step(s.y, w.y, v.y, ep);
     sgd_step(s.z, w.z, v.z, ep);
     sgd_step(s.w, w.w, v.w, ep);
+}
+__device__ inline void adam_step4(float4 s, float4 &w, float4 &m, float4 &v, const Epilogue &ep)
+{
+    adam_step(s.x, w.x, m.x, v.x, ep);
+    adam_step(s.y, w.y, m.y, v.y, ep);
+    adam_step(s.z, w.z, m.z, v.z, ep);
+    adam_step(s.w, w.w, m.w, v.w, ep);
 }
 
 struct DecodeArgs {
@@ -1233,7 +1261,13 @@ __device__ inline void store_tile(float *dst, u64 out0, u32 len, float *s_acc, c
     if (ep.weights) {
         for (u32 i = tid; i < len; i += kDecodeThreads) {
             float w = ep.weights[out0 + i], v = ep.momentum[out0 + i];
-            sgd_step(s_acc[i], w, v, ep);
+            if (ep.adam) {
+                float v2 = ep.second[out0 + i];
+                adam_step(s_acc[i], w, v, v2, ep);
+                ep.second[out0 + i] = v2;
+            } else {
+                sgd_step(s_acc[i], w, v, ep);
+            }
             ep.momentum[out0 + i] = v;
             ep.weights[out0 + i] = w;
             s_acc[i] = 0.f;
@@ -1757,12 +1791,12 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
 }
 
 // Lays the slots out (see WarpDecSmem), then decodes.
-template <typename Word, bool MULTI, bool SGD>
+template <typename Word, bool MULTI, int OPT>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv);
 
-//   s_wv   (SGD) shared memory for a tile of weights followed by a tile of momentum, 2 x kDecodeChunk floats
-template <typename Word, bool SGD>
+//   s_wv   (OPT != 0) shared memory for a tile of weights, a tile of momentum and (Adam) a tile of second moments
+template <typename Word, int OPT>
 __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
                                  const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
@@ -1817,13 +1851,13 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         }
     }
     __syncthreads();
-    if (ws.n_rounds > 1u) decode_warps<Word, true, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-    else decode_warps<Word, false, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    else decode_warps<Word, false, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
 }
 
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
-// SGD: the finished quarter feeds the optimizer step of a.ep instead of going to a.dst.
-template <typename Word, bool MULTI, bool SGD>
+// OPT: 0 the finished quarter goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
+template <typename Word, bool MULTI, int OPT>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
@@ -1988,20 +2022,23 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
     u64 tile = first;
     bool failed = false;
-    float *const wq = s_wv + (u32)warp * quarter, *const vq = s_wv + kDecodeChunk + (u32)warp * quarter;     // (SGD)
-    u32 wv_use = 0;                                 // (SGD) fetches of the quarters so far
+    // (OPT != 0) the warp's quarters of the staged weights, momentum and second moments
+    float *const wq = s_wv + (u32)warp * quarter, *const vq = s_wv + kDecodeChunk + (u32)warp * quarter;
+    float *const uq = s_wv + 2 * kDecodeChunk + (u32)warp * quarter;
+    u32 wv_use = 0;                                 // fetches of the quarters so far
     for (u64 it = 0; it < my_tiles; it++, tile += stride) {
         const u64 bin0 = tile * (u64)TB;
         const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
         const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
         const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
         const bool whole = vec_store && len == quarter;
-        if (SGD && whole && lane == 0) {
-            // the warp's quarters of the weights and the momentum travel while the words are added
+        if (OPT != 0 && whole && lane == 0) {
+            // the warp's quarters of the optimizer's arrays travel while the words are added
             bulk_wait_read_all();                   // the previous tile's copies out have read the buffers
-            mbar_arrive_expect_tx(&ws.wv_full[warp], 2u * quarter * 4u);
+            mbar_arrive_expect_tx(&ws.wv_full[warp], (OPT == 2 ? 3u : 2u) * quarter * 4u);
             bulk_load(wq, a.ep.weights + out0, quarter * 4u, &ws.wv_full[warp]);
             bulk_load(vq, a.ep.momentum + out0, quarter * 4u, &ws.wv_full[warp]);
+            if (OPT == 2) bulk_load(uq, a.ep.second + out0, quarter * 4u, &ws.wv_full[warp]);
         }
         for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
             long long t0 = clock64();
@@ -2062,7 +2099,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         long long t0 = clock64();
 
         // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
-        if (SGD) {
+        if (OPT != 0) {
             // averageGradients() + updateWeights() on the warp's quarter, in shared memory; two bulk
             // copies take the new weights and momentum back
             if (whole) {
@@ -2075,9 +2112,16 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 float4 *w4 = reinterpret_cast<float4 *>(wq), *v4 = reinterpret_cast<float4 *>(vq);
                 float4 *s4 = reinterpret_cast<float4 *>(my_acc);
                 const int n4 = (int)(quarter >> 2);
+                float4 *u4 = reinterpret_cast<float4 *>(uq);
                 for (int at = lane; at < n4; at += 32) {
                     float4 w = w4[at], v = v4[at];
-                    sgd_step4(s4[at], w, v, a.ep.lr, a.ep.mu, a.ep.k);
+                    if (OPT == 2) {
+                        float4 u = u4[at];
+                        adam_step4(s4[at], w, v, u, a.ep);
+                        u4[at] = u;
+                    } else {
+                        sgd_step4(s4[at], w, v, a.ep.lr, a.ep.mu, a.ep.k);
+                    }
                     s4[at] = make_float4(0.f, 0.f, 0.f, 0.f);
                     v4[at] = v;
                     w4[at] = w;
@@ -2087,13 +2131,20 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 if (lane == 0) {
                     bulk_store(a.ep.weights + out0, wq, quarter * 4u);
                     bulk_store(a.ep.momentum + out0, vq, quarter * 4u);
+                    if (OPT == 2) bulk_store(a.ep.second + out0, uq, quarter * 4u);
                     bulk_commit();
                 }
             } else {
                 for (u32 i = lane; i < quarter; i += 32) {
                     if (i < len) {
                         float w = a.ep.weights[out0 + i], v = a.ep.momentum[out0 + i];
-                        sgd_step(my_acc[i], w, v, a.ep);
+                        if (OPT == 2) {
+                            float u = a.ep.second[out0 + i];
+                            adam_step(my_acc[i], w, v, u, a.ep);
+                            a.ep.second[out0 + i] = u;
+                        } else {
+                            sgd_step(my_acc[i], w, v, a.ep);
+                        }
                         a.ep.momentum[out0 + i] = v;
                         a.ep.weights[out0 + i] = w;
                     }
@@ -2256,10 +2307,11 @@ __device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_
 // The decoder is two kernels, so that each gets the registers its path needs: decode_sum_warps
 // takes the shapes of warp_path() and returns at once for any other, decode_sum the reverse.  A
 // caller that knows the shape launches the one that works; one that does not launches both.
-constexpr u32 kSgdSmemBytes = 2u * kDecodeChunk * 4u;    // dynamic shared memory of decode_sum_warps<true>
+// dynamic shared memory of decode_sum_warps<OPT>: a tile per array of the optimizer
+constexpr u32 opt_smem_bytes(int opt) { return opt == 0 ? 0u : (opt == 2 ? 3u : 2u) * kDecodeChunk * 4u; }
 
-template <bool SGD>
-__global__ void __launch_bounds__(kDecodeLaunch, SGD ? 3 : kWarpsPerSm)
+template <int OPT>
+__global__ void __launch_bounds__(kDecodeLaunch, OPT == 0 ? kWarpsPerSm : OPT == 1 ? 3 : 2)
 decode_sum_warps(DecodeArgs a)
 {
     __shared__ __align__(16) float s_acc[kDecodeChunk];
@@ -2273,9 +2325,9 @@ decode_sum_warps(DecodeArgs a)
     const Geometry geo = make_geometry(n, L_T);
     if (!warp_path(geo)) return;
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
-    extern __shared__ __align__(16) float s_dyn[];     // (SGD) a tile of weights and a tile of momentum
-    if (geo.w == 1u) decode_warps_any<unsigned char, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, SGD ? s_dyn : nullptr);
-    else decode_warps_any<unsigned short, SGD>(a, geo, s_acc, ws, s_scale, s_nsel, SGD ? s_dyn : nullptr);
+    extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles
+    if (geo.w == 1u) decode_warps_any<unsigned char, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
+    else decode_warps_any<unsigned short, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
 }
 
 __global__ void __launch_bounds__(kDecodeThreads, 6)
@@ -2315,9 +2367,10 @@ struct DecodeBatchArgs {
     u64 n[kDecBatchLayers];
     u32 L_T[kDecBatchLayers];
     float *dst[kDecBatchLayers];                     // the layer's output; with `sgd` its weights
-    float *aux[kDecBatchLayers];                     // with `sgd`: its momentum
-    float lr, mu;
-    u32 sgd;                                         // the optimizer step takes the place of the store (see Epilogue)
+    float *aux[kDecBatchLayers];                     // with `opt`: its momentum (Adam: first moments)
+    float *aux2[kDecBatchLayers];                    // Adam: its second moments
+    float lr, mu, beta2, eps;
+    u32 opt;                                         // 1 SGD, 2 Adam: the optimizer step takes the place of the store (see Epilogue)
     const unsigned char *stream[kDecBatchPtrs];      // [layer * k + learner]
 };
 
@@ -2371,7 +2424,8 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
         const Geometry &geo = sm.geo[lo];
         const u64 tile = gt - sm.first[lo];
         const unsigned char *const *streams = &b.stream[lo * b.k];
-        const Epilogue ep = {b.sgd ? b.dst[lo] : nullptr, b.sgd ? b.aux[lo] : nullptr, b.lr, b.mu, (float)b.k};
+        const Epilogue ep = {b.opt ? b.dst[lo] : nullptr, b.opt ? b.aux[lo] : nullptr, b.opt == 2u ? b.aux2[lo] : nullptr,
+                             b.lr, b.mu, b.beta2, b.eps, (float)b.k, b.opt == 2u ? 1u : 0u};
         if (geo.w == 1u) {
             decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], ep, sm.d, bad);
         } else if (geo.tile_bins >= 32) {
@@ -2435,6 +2489,7 @@ struct DeviceInfo {
     int decode_per_sm = 0;
     int decode_warps_per_sm = 0;
     int decode_sgd_per_sm = 0;  // 0: the optimizer decoder is unavailable on this device
+    int decode_adam_per_sm = 0;
     int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
@@ -2456,13 +2511,19 @@ int device_info(DeviceInfo *&out)
         int per_sm = 1;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<false>, kDecodeLaunch, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<0>, kDecodeLaunch, 0);
         d.decode_warps_per_sm = per_sm < 1 ? 1 : per_sm;
-        if (cudaFuncSetAttribute(decode_sum_warps<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSgdSmemBytes) == cudaSuccess) {
+        if (cudaFuncSetAttribute(decode_sum_warps<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)opt_smem_bytes(1)) == cudaSuccess) {
             per_sm = 0;
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<true>, kDecodeLaunch, kSgdSmemBytes);
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<1>, kDecodeLaunch, opt_smem_bytes(1));
             d.decode_sgd_per_sm = per_sm;
+        }
+        if (cudaFuncSetAttribute(decode_sum_warps<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)opt_smem_bytes(2)) == cudaSuccess) {
+            per_sm = 0;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<2>, kDecodeLaunch, opt_smem_bytes(2));
+            d.decode_adam_per_sm = per_sm;
         }
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
@@ -2608,10 +2669,11 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         args.stream[l] = static_cast<const unsigned char *>(packed[l]);
     }
     if (dst && misaligned(dst)) return ADACOMP_ERR_ALIGN;
-    args.ep = Epilogue{nullptr, nullptr, 0.f, 0.f, (float)k};
+    args.ep = Epilogue{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f, 0.f, (float)k, 0u};
     if (ep) {
-        if (!ep->weights || !ep->momentum) return ADACOMP_ERR_NULL;
-        if (misaligned(ep->weights) || misaligned(ep->momentum)) return ADACOMP_ERR_ALIGN;
+        if (!ep->weights || !ep->momentum || (ep->adam && !ep->second)) return ADACOMP_ERR_NULL;
+        if (misaligned(ep->weights) || misaligned(ep->momentum) || (ep->adam && misaligned(ep->second)))
+            return ADACOMP_ERR_ALIGN;
         args.ep = *ep;
         args.ep.k = (float)k;
     }
@@ -2633,15 +2695,17 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (warps && ep) {
-        if (!info->decode_sgd_per_sm) return ADACOMP_ERR_CUDA;
-        u64 grid_s = (u64)info->sms * info->decode_sgd_per_sm;
+        const int per = ep->adam ? info->decode_adam_per_sm : info->decode_sgd_per_sm;
+        if (!per) return ADACOMP_ERR_CUDA;
+        u64 grid_s = (u64)info->sms * per;
         if (hint_L_T) {
             const u64 items = decode_items(hint_n, hint_L_T);
             grid_s = items < grid_s ? (items ? items : 1) : grid_s;
         }
-        decode_sum_warps<true><<<(unsigned)grid_s, kDecodeLaunch, kSgdSmemBytes, st>>>(args);
+        if (ep->adam) decode_sum_warps<2><<<(unsigned)grid_s, kDecodeLaunch, opt_smem_bytes(2), st>>>(args);
+        else decode_sum_warps<1><<<(unsigned)grid_s, kDecodeLaunch, opt_smem_bytes(1), st>>>(args);
     }
-    else if (warps) decode_sum_warps<false><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
+    else if (warps) decode_sum_warps<0><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
     if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, st>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
@@ -2825,17 +2889,21 @@ int adacomp_decompress_accumulate_ex(const void *const *packed, uint32_t k_strea
     return decompress_impl(packed, k_streams, dst, stream, n, L_T);
 }
 
-// Decode-sum of a list of layers whose shapes the caller knows.  `aux` (optional): the layers' momentum
-// arrays; `dst` then holds their weights and every layer gets the optimizer step instead of a store.
+// Decode-sum of a list of layers whose shapes the caller knows.  `opt` (optional; its pointers unused):
+// `dst` then holds the layers' weights, `aux` their momentum (Adam: first moments), `aux2` (Adam) their
+// second moments, and every layer gets the optimizer step instead of a store.
 int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *const *dst, float *const *aux,
-                          const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream, float lr, float mu)
+                          float *const *aux2, const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream,
+                          const Epilogue *opt)
 {
+    if (opt && n_layers && (!aux || (opt->adam && !aux2))) return ADACOMP_ERR_NULL;
     if (n_layers && (!packed || !dst || !n || !L_T)) return ADACOMP_ERR_NULL;
     if (k_streams == 0 || k_streams > ADACOMP_MAX_STREAMS) return ADACOMP_ERR_STREAMS;
     for (uint32_t t = 0; t < n_layers; t++) {
         if (L_T[t] == 0 || L_T[t] > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-        if (!dst[t] || (aux && !aux[t])) return ADACOMP_ERR_NULL;
-        if (misaligned(dst[t]) || (aux && misaligned(aux[t]))) return ADACOMP_ERR_ALIGN;
+        if (!dst[t] || (opt && !aux[t]) || (opt && opt->adam && !aux2[t])) return ADACOMP_ERR_NULL;
+        if (misaligned(dst[t]) || (opt && misaligned(aux[t])) || (opt && opt->adam && misaligned(aux2[t])))
+            return ADACOMP_ERR_ALIGN;
         for (uint32_t l = 0; l < k_streams; l++) {
             if (!packed[(size_t)t * k_streams + l]) return ADACOMP_ERR_NULL;
             if (misaligned(packed[(size_t)t * k_streams + l])) return ADACOMP_ERR_ALIGN;
@@ -2850,9 +2918,11 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
     static thread_local DecodeBatchArgs batch;
     batch.n_layers = 0;
     batch.k = k_streams;
-    batch.sgd = aux ? 1u : 0u;
-    batch.lr = lr;
-    batch.mu = mu;
+    batch.opt = !opt ? 0u : opt->adam ? 2u : 1u;
+    batch.lr = opt ? opt->lr : 0.f;
+    batch.mu = opt ? opt->mu : 0.f;
+    batch.beta2 = opt ? opt->beta2 : 0.f;
+    batch.eps = opt ? opt->eps : 0.f;
     u64 batch_tiles = 0;
     auto flush = [&]() -> int {
         if (batch.n_layers == 0) return ADACOMP_OK;
@@ -2873,7 +2943,8 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
             batch.n[i] = n[t];
             batch.L_T[i] = L_T[t];
             batch.dst[i] = dst[t];
-            batch.aux[i] = aux ? aux[t] : nullptr;
+            batch.aux[i] = opt ? aux[t] : nullptr;
+            batch.aux2[i] = opt && opt->adam ? aux2[t] : nullptr;
             for (uint32_t l = 0; l < k_streams; l++)
                 batch.stream[(size_t)i * k_streams + l] = static_cast<const unsigned char *>(packed[(size_t)t * k_streams + l]);
             batch_tiles += decode_items(n[t], L_T[t]);
@@ -2881,8 +2952,11 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
                 rc = flush();
                 if (rc != ADACOMP_OK) return rc;
             }
-        } else if (aux) {
-            const Epilogue ep = {dst[t], aux[t], lr, mu, 0.f};
+        } else if (opt) {
+            Epilogue ep = *opt;
+            ep.weights = dst[t];
+            ep.momentum = aux[t];
+            ep.second = opt->adam ? aux2[t] : nullptr;
             rc = decompress_impl(packed + (size_t)t * k_streams, k_streams, nullptr, stream, n[t], L_T[t], &ep);
             if (rc != ADACOMP_OK) return rc;
         } else {
@@ -2896,15 +2970,24 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
 int adacomp_decompress_accumulate_multi_ex(const void *const *packed, uint32_t k_streams, float *const *dst,
                                            const uint64_t *n, const uint32_t *L_T, uint32_t n_layers, void *stream)
 {
-    return decompress_multi_impl(packed, k_streams, dst, nullptr, n, L_T, n_layers, stream, 0.f, 0.f);
+    return decompress_multi_impl(packed, k_streams, dst, nullptr, nullptr, n, L_T, n_layers, stream, nullptr);
 }
 
 int adacomp_decompress_average_sgd_multi(const void *const *packed, uint32_t k_streams, float *const *weights,
                                          float *const *momentum, const uint64_t *n, const uint32_t *L_T,
                                          uint32_t n_layers, float lr, float mu, void *stream)
 {
-    if (n_layers && !momentum) return ADACOMP_ERR_NULL;
-    return decompress_multi_impl(packed, k_streams, weights, momentum, n, L_T, n_layers, stream, lr, mu);
+    const Epilogue opt = {nullptr, nullptr, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u};
+    return decompress_multi_impl(packed, k_streams, weights, momentum, nullptr, n, L_T, n_layers, stream, &opt);
+}
+
+int adacomp_decompress_average_adam_multi(const void *const *packed, uint32_t k_streams, float *const *weights,
+                                          float *const *m, float *const *v, const uint64_t *n, const uint32_t *L_T,
+                                          uint32_t n_layers, float step_size, float beta1, float beta2, float eps,
+                                          void *stream)
+{
+    const Epilogue opt = {nullptr, nullptr, nullptr, step_size, beta1, beta2, eps, 0.f, 1u};
+    return decompress_multi_impl(packed, k_streams, weights, m, v, n, L_T, n_layers, stream, &opt);
 }
 
 int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
@@ -3070,7 +3153,16 @@ int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams
                                    uint64_t n, uint32_t L_T, float lr, float mu, void *stream)
 {
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-    const Epilogue ep = {weights, momentum, lr, mu, 0.f};
+    const Epilogue ep = {weights, momentum, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u};
+    return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
+}
+
+int adacomp_decompress_average_adam(const void *const *packed, uint32_t k_streams, float *weights, float *m, float *v,
+                                    uint64_t n, uint32_t L_T, float step_size, float beta1, float beta2, float eps,
+                                    void *stream)
+{
+    if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    const Epilogue ep = {weights, m, v, step_size, beta1, beta2, eps, 0.f, 1u};
     return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
 }
 

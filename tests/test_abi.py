@@ -93,6 +93,13 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert um(ptrs, 2, bad_w, wl, one64, one32, 1, lr, mu, None) == -3
     assert um(ptrs, 2, wl, wl, one64, (C.c_uint32 * 1)(0), 1, lr, mu, None) == -2
     assert um(None, 2, None, None, None, None, 0, lr, mu, None) == 0
+    ad = lib.adacomp_decompress_average_adam
+    hy = (C.c_float(1e-3), C.c_float(0.9), C.c_float(0.999), C.c_float(1e-8))
+    assert ad(ptrs, 2, A, A, None, 10, 50, *hy, None) == -1
+    assert ad(ptrs, 2, A, A, A + 4, 10, 50, *hy, None) == -3
+    assert ad(ptrs, 2, A, A, A, 10, 0, *hy, None) == -2
+    assert ad(ptrs, 65, A, A, A, 10, 50, *hy, None) == -4
+    assert lib.adacomp_decompress_average_adam_multi(ptrs, 2, wl, wl, None, one64, one32, 1, *hy, None) == -1
     hb = lib.adacomp_compress_bf16
     assert hb(None, A, 10, 50, A, A, None) == -1
     assert hb(A, A, 10, 0, A, A, None) == -2
