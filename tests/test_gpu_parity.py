@@ -144,7 +144,12 @@ def gpu_decode(streams, n):
 @pytest.mark.parametrize("L_T,n,k", [(50, 100352, 1), (50, 5120, 4), (500, 147456, 8), (50, 4000 * 40 + 7, 16),
                                      (3, 9001, 3), (64, 70000, 2), (65, 70000, 2), (1000, 50001, 5),
                                      (1001, 50001, 5), (5000, 123457, 3), (16384, 100001, 4),
-                                     (16384, 100, 2), (500, 12, 64)])
+                                     (16384, 100, 2), (500, 12, 64),
+                                     # every lane-to-bin arrangement of the warp decoder: 24 / 20 bins per warp by word,
+                                     # then 16, 10, 8, 4, 2 and 1 bins per warp with 2 .. 32 lanes per bin
+                                     (41, 96 * 41 * 9 + 5, 3), (48, 80 * 48 * 7 + 1, 4), (49, 80 * 49 * 5, 2),
+                                     (62, 64 * 62 * 6 + 9, 3), (100, 40 * 100 * 5 + 7, 3), (125, 32 * 125 * 5 + 3, 5),
+                                     (250, 16 * 250 * 6 + 11, 3), (400, 8 * 400 * 7 + 2, 9), (1000, 4 * 1000 * 6 + 13, 3)])
 def test_decode_sum_matches_oracle(L_T, n, k):
     rng = np.random.default_rng(L_T + n + k)
     streams_gpu, streams_cpu = [], []
