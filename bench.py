@@ -233,11 +233,19 @@ def run_ours(a):
     rank, world, local = ranks.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    # (two switches for exercising the multi-rank control flow on a box with one GPU: ranks share the
+    # device and meet over gloo; a measurement needs one GPU per rank and NCCL, the defaults)
+    if os.environ.get("ADACOMP_BENCH_SHARE_GPU") == "1":
+        local %= torch.cuda.device_count()
+    backend = os.environ.get("ADACOMP_BENCH_BACKEND", "nccl")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     B.adacomp_set_device(local)          # the library's own CUDA runtime follows torch's choice
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
 
     def barrier():
         if world > 1:
