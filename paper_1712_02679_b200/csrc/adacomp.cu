@@ -382,7 +382,7 @@ tile_pass_fast(PassArgs a)
     if (LAZY) {
         const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(a.lazy_state);
         if (lh->magic != kLazyMagic || lh->n != a.geo.n || lh->L_T != a.geo.L_T) {
-            // not the state of this tensor (the same verdict in every CTA): touch neither residue
+            // not the state of this tensor (the same decision in every CTA): touch neither residue
             // nor state, and report every tile as empty so that the kernels after this one see a
             // consistent, empty stream
             if (threadIdx.x == 0) {
