@@ -1217,15 +1217,16 @@ constexpr int kSlots = 8;                       // tiles in flight per CTA at mo
 constexpr u32 kRingBytes = 19200;
 constexpr u32 kSlotMax = kRingBytes / 2;        // a slot never takes more: two tiles are always in flight
 
+template <int NW>
 struct WarpDecSmem {
     uint4 ring[kRingBytes / 16];
-    u32 tmp[4][32];                             // per decoding warp: output places of its non-empty bins
+    u32 tmp[NW][32];                            // per decoding warp: output places of its non-empty bins
     unsigned short coff[ADACOMP_MAX_STREAMS];   // byte offset in a slot of learner l's bin counts (its words follow them)
     unsigned short wcap[ADACOMP_MAX_STREAMS];   // bytes of its word region
     unsigned char rfirst[ADACOMP_MAX_STREAMS];  // round r brings learners [rfirst[r], rfirst[r] + rcount[r]) of a tile
     unsigned char rcount[ADACOMP_MAX_STREAMS];
     u64 full[kSlots], empty[kSlots];            // mbarriers of the slots
-    u64 wv_full[4];                             // optimizer epilogue: a warp's weight and momentum quarters have landed
+    u64 wv_full[NW];                            // optimizer epilogue: a warp's share of the optimizer's arrays has landed
     u32 slot_bytes, n_slots, n_rounds, abort;
 };
 
@@ -1791,13 +1792,13 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
 }
 
 // Lays the slots out (see WarpDecSmem), then decodes.
-template <typename Word, bool MULTI, int OPT>
-__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+template <typename Word, bool MULTI, int OPT, int NW>
+__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv);
 
 //   s_wv   (OPT != 0) shared memory for a tile of weights, a tile of momentum and (Adam) a tile of second moments
-template <typename Word, int OPT>
-__device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+template <typename Word, int OPT, int NW>
+__device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                                  const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1808,14 +1809,14 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
     if (tid == 0) {
         for (int s = 0; s < kSlots; s++) {
             mbar_init(&ws.full[s], 32);         // every lane of the loader arrives, with or without bytes to expect
-            mbar_init(&ws.empty[s], 4);         // every decoding warp arrives
+            mbar_init(&ws.empty[s], NW);        // every decoding warp arrives
         }
-        for (int w = 0; w < 4; w++) mbar_init(&ws.wv_full[w], 1);
+        for (int w = 0; w < NW; w++) mbar_init(&ws.wv_full[w], 1);
         ws.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
-    if (warp == 4) {
+    if (warp == NW) {
         // the learners' regions: counts, then room for 1.5 times a tile's average words + slack
 #pragma unroll
         for (int h = 0; h < 2; h++) {
@@ -1851,14 +1852,15 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         }
     }
     __syncthreads();
-    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-    else decode_warps<Word, false, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    else decode_warps<Word, false, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
 }
 
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
-// OPT: 0 the finished quarter goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
-template <typename Word, bool MULTI, int OPT>
-__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem &ws,
+// OPT: 0 the finished share goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
+// NW: decoding warps (warp NW is the loader); each owns 1/NW of the tile's bins ("quarter" below, whatever NW is).
+template <typename Word, bool MULTI, int OPT, int NW>
+__device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1873,7 +1875,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
 
     const u32 NR = MULTI ? ws.n_rounds : 1u, slot_bytes = ws.slot_bytes, S = ws.n_slots;
 
-    if (warp == 4) {
+    if (warp == NW) {
         // ================================ loader warp ================================
         // An item is one round of one tile; lane j (and j + 32) looks after the j-th learner of the
         // round.  The learners' directory entries are read two items ahead.
@@ -2003,7 +2005,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     }
 
     // =============================== decoding warps ===============================
-    const int nb = TB / 4;                          // bins of a warp (tile_bins is a multiple of 4)
+    const int nb = TB / NW;                         // bins of a warp (the launcher picks NW to divide tile_bins)
     const int b0 = warp * nb;
     const u32 quarter = (u32)nb * L_T;              // output elements of a warp
     const u32 acc_at = smem_addr(s_acc) + (u32)warp * quarter * 4u;
@@ -2310,12 +2312,14 @@ __device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_
 // dynamic shared memory of decode_sum_warps<OPT>: a tile per array of the optimizer
 constexpr u32 opt_smem_bytes(int opt) { return opt == 0 ? 0u : (opt == 2 ? 3u : 2u) * kDecodeChunk * 4u; }
 
-template <int OPT>
-__global__ void __launch_bounds__(kDecodeLaunch, OPT == 0 ? kWarpsPerSm : OPT == 1 ? 3 : 2)
+// NW decoding warps and the loader warp: 4 for plain decoding; with an optimizer step, whose staged tiles
+// leave room for fewer CTAs per SM, 8 where they divide the tile's bins (more warps to hide the adds' latency).
+template <int OPT, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, OPT == 0 ? kWarpsPerSm : OPT == 1 ? 3 : 2)
 decode_sum_warps(DecodeArgs a)
 {
     __shared__ __align__(16) float s_acc[kDecodeChunk];
-    __shared__ __align__(16) WarpDecSmem ws;
+    __shared__ __align__(16) WarpDecSmem<NW> ws;
     __shared__ u64 s_nsel[ADACOMP_MAX_STREAMS];
     __shared__ float s_scale[ADACOMP_MAX_STREAMS];
     __shared__ int s_bad;
@@ -2323,11 +2327,11 @@ decode_sum_warps(DecodeArgs a)
     u64 n;
     if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
-    if (!warp_path(geo)) return;
+    if (!warp_path(geo) || geo.tile_bins % (u32)NW != 0) return;      // (the launcher picks NW from the shape it was given)
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
     extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles
-    if (geo.w == 1u) decode_warps_any<unsigned char, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
-    else decode_warps_any<unsigned short, OPT>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
+    if (geo.w == 1u) decode_warps_any<unsigned char, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
+    else decode_warps_any<unsigned short, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
 }
 
 __global__ void __launch_bounds__(kDecodeThreads, 6)
@@ -2488,8 +2492,7 @@ struct DeviceInfo {
     int smem_optin = 0;
     int decode_per_sm = 0;
     int decode_warps_per_sm = 0;
-    int decode_sgd_per_sm = 0;  // 0: the optimizer decoder is unavailable on this device
-    int decode_adam_per_sm = 0;
+    int decode_opt_per_sm[2][2] = {{0, 0}, {0, 0}};     // [SGD, Adam][4, 8 decoding warps]; 0: unavailable on this device
     int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
@@ -2511,20 +2514,18 @@ int device_info(DeviceInfo *&out)
         int per_sm = 1;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum, kDecodeThreads, 0);
         d.decode_per_sm = per_sm < 1 ? 1 : per_sm;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<0>, kDecodeLaunch, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<0, 4>, kDecodeLaunch, 0);
         d.decode_warps_per_sm = per_sm < 1 ? 1 : per_sm;
-        if (cudaFuncSetAttribute(decode_sum_warps<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)opt_smem_bytes(1)) == cudaSuccess) {
-            per_sm = 0;
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<1>, kDecodeLaunch, opt_smem_bytes(1));
-            d.decode_sgd_per_sm = per_sm;
-        }
-        if (cudaFuncSetAttribute(decode_sum_warps<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)opt_smem_bytes(2)) == cudaSuccess) {
-            per_sm = 0;
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_sum_warps<2>, kDecodeLaunch, opt_smem_bytes(2));
-            d.decode_adam_per_sm = per_sm;
-        }
+        auto opt_ready = [&](auto kernel, int threads, u32 smem) -> int {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+            int per = 0;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, kernel, threads, smem);
+            return per;
+        };
+        d.decode_opt_per_sm[0][0] = opt_ready(decode_sum_warps<1, 4>, 5 * 32, opt_smem_bytes(1));
+        d.decode_opt_per_sm[0][1] = opt_ready(decode_sum_warps<1, 8>, 9 * 32, opt_smem_bytes(1));
+        d.decode_opt_per_sm[1][0] = opt_ready(decode_sum_warps<2, 4>, 5 * 32, opt_smem_bytes(2));
+        d.decode_opt_per_sm[1][1] = opt_ready(decode_sum_warps<2, 8>, 9 * 32, opt_smem_bytes(2));
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
         d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
@@ -2695,17 +2696,22 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (warps && ep) {
-        const int per = ep->adam ? info->decode_adam_per_sm : info->decode_sgd_per_sm;
+        // (the optimizer entry points always pass the shape)
+        const bool eight = hint_L_T && make_geometry(hint_n, hint_L_T).tile_bins % 8u == 0;
+        const int per = info->decode_opt_per_sm[ep->adam ? 1 : 0][eight ? 1 : 0];
         if (!per) return ADACOMP_ERR_CUDA;
         u64 grid_s = (u64)info->sms * per;
         if (hint_L_T) {
             const u64 items = decode_items(hint_n, hint_L_T);
             grid_s = items < grid_s ? (items ? items : 1) : grid_s;
         }
-        if (ep->adam) decode_sum_warps<2><<<(unsigned)grid_s, kDecodeLaunch, opt_smem_bytes(2), st>>>(args);
-        else decode_sum_warps<1><<<(unsigned)grid_s, kDecodeLaunch, opt_smem_bytes(1), st>>>(args);
+        const unsigned g = (unsigned)grid_s;
+        if (ep->adam && eight) decode_sum_warps<2, 8><<<g, 9 * 32, opt_smem_bytes(2), st>>>(args);
+        else if (ep->adam) decode_sum_warps<2, 4><<<g, 5 * 32, opt_smem_bytes(2), st>>>(args);
+        else if (eight) decode_sum_warps<1, 8><<<g, 9 * 32, opt_smem_bytes(1), st>>>(args);
+        else decode_sum_warps<1, 4><<<g, 5 * 32, opt_smem_bytes(1), st>>>(args);
     }
-    else if (warps) decode_sum_warps<0><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
+    else if (warps) decode_sum_warps<0, 4><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
     if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, st>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
