@@ -1142,27 +1142,28 @@ struct Epilogue {
     float *weights, *momentum, *second;
     float lr, mu, beta2, eps, k;
     u32 adam;
+    float inv_k;        // 1 / k where k is a power of two (the product with it is the correctly rounded quotient), else 0
 };
 
-// s / k without the division where the quotient is known without it: a zero sum, which is what
-// most elements have, stays the same zero; for k a power of two the product with 1 / k is the
-// correctly rounded quotient too.
-__device__ inline float mean_of(float s, float k)
+// s / k without the division where the quotient is known without it: for k a power of two the product
+// with 1 / k is the correctly rounded quotient; otherwise a zero sum, which is what most elements have,
+// stays the same zero (and spares the division its slow path).
+__device__ inline float mean_of(float s, const Epilogue &ep)
 {
-    const bool pow2 = (__float_as_uint(k) & 0x007fffffu) == 0u;
-    return s == 0.f ? s : pow2 ? __fmul_rn(s, __frcp_rn(k)) : __fdiv_rn(s, k);
+    if (ep.inv_k != 0.f) return __fmul_rn(s, ep.inv_k);
+    return s == 0.f ? s : __fdiv_rn(s, ep.k);
 }
 
 __device__ inline void sgd_step(float s, float &w, float &v, const Epilogue &ep)
 {
-    const float mean = mean_of(s, ep.k);
+    const float mean = mean_of(s, ep);
     v = __fadd_rn(__fmul_rn(ep.mu, v), mean);
     w = __fsub_rn(w, __fmul_rn(ep.lr, v));
 }
 
 __device__ inline void adam_step(float s, float &w, float &m, float &v, const Epilogue &ep)
 {
-    const float mean = mean_of(s, ep.k);
+    const float mean = mean_of(s, ep);
     m = __fadd_rn(__fmul_rn(ep.mu, m), __fmul_rn(__fsub_rn(1.f, ep.mu), mean));
     v = __fadd_rn(__fmul_rn(ep.beta2, v), __fmul_rn(__fsub_rn(1.f, ep.beta2), __fmul_rn(mean, mean)));
     const float num = __fmul_rn(ep.lr, m), den = __fadd_rn(__fsqrt_rn(v), ep.eps);
@@ -1170,9 +1171,8 @@ __device__ inline void adam_step(float s, float &w, float &m, float &v, const Ep
 }
 
 // Four elements at once.
-__device__ inline void sgd_step4(float4 s, float4 &w, float4 &v, float lr, float mu, float k)
+__device__ inline void sgd_step4(float4 s, float4 &w, float4 &v, const Epilogue &ep)
 {
-    const Epilogue ep = {nullptr, nullptr, nullptr, lr, mu, 0.f, 0.f, k, 0u};
     sgd_step(s.x, w.x, v.x, ep);
     sgd_step(s.y, w.y, v.y, ep);
     sgd_step(s.z, w.z, v.z, ep);
@@ -2122,7 +2122,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                         adam_step4(s4[at], w, v, u, a.ep);
                         u4[at] = u;
                     } else {
-                        sgd_step4(s4[at], w, v, a.ep.lr, a.ep.mu, a.ep.k);
+                        sgd_step4(s4[at], w, v, a.ep);
                     }
                     s4[at] = make_float4(0.f, 0.f, 0.f, 0.f);
                     v4[at] = v;
@@ -2429,7 +2429,8 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
         const u64 tile = gt - sm.first[lo];
         const unsigned char *const *streams = &b.stream[lo * b.k];
         const Epilogue ep = {b.opt ? b.dst[lo] : nullptr, b.opt ? b.aux[lo] : nullptr, b.opt == 2u ? b.aux2[lo] : nullptr,
-                             b.lr, b.mu, b.beta2, b.eps, (float)b.k, b.opt == 2u ? 1u : 0u};
+                             b.lr, b.mu, b.beta2, b.eps, (float)b.k, b.opt == 2u ? 1u : 0u,
+                             (b.k & (b.k - 1u)) == 0u ? __frcp_rn((float)b.k) : 0.f};
         if (geo.w == 1u) {
             decode_item_staged<unsigned char, true>(streams, b.k, geo, tile, b.dst[lo], ep, sm.d, bad);
         } else if (geo.tile_bins >= 32) {
@@ -2670,13 +2671,14 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         args.stream[l] = static_cast<const unsigned char *>(packed[l]);
     }
     if (dst && misaligned(dst)) return ADACOMP_ERR_ALIGN;
-    args.ep = Epilogue{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f, 0.f, (float)k, 0u};
+    args.ep = Epilogue{nullptr, nullptr, nullptr, 0.f, 0.f, 0.f, 0.f, (float)k, 0u, 0.f};
     if (ep) {
         if (!ep->weights || !ep->momentum || (ep->adam && !ep->second)) return ADACOMP_ERR_NULL;
         if (misaligned(ep->weights) || misaligned(ep->momentum) || (ep->adam && misaligned(ep->second)))
             return ADACOMP_ERR_ALIGN;
         args.ep = *ep;
         args.ep.k = (float)k;
+        args.ep.inv_k = (k & (k - 1u)) == 0u ? 1.0f / (float)k : 0.f;
     }
     args.dst = dst;
     args.k = k;
@@ -2983,7 +2985,7 @@ int adacomp_decompress_average_sgd_multi(const void *const *packed, uint32_t k_s
                                          float *const *momentum, const uint64_t *n, const uint32_t *L_T,
                                          uint32_t n_layers, float lr, float mu, void *stream)
 {
-    const Epilogue opt = {nullptr, nullptr, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u};
+    const Epilogue opt = {nullptr, nullptr, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u, 0.f};
     return decompress_multi_impl(packed, k_streams, weights, momentum, nullptr, n, L_T, n_layers, stream, &opt);
 }
 
@@ -2992,7 +2994,7 @@ int adacomp_decompress_average_adam_multi(const void *const *packed, uint32_t k_
                                           uint32_t n_layers, float step_size, float beta1, float beta2, float eps,
                                           void *stream)
 {
-    const Epilogue opt = {nullptr, nullptr, nullptr, step_size, beta1, beta2, eps, 0.f, 1u};
+    const Epilogue opt = {nullptr, nullptr, nullptr, step_size, beta1, beta2, eps, 0.f, 1u, 0.f};
     return decompress_multi_impl(packed, k_streams, weights, m, v, n, L_T, n_layers, stream, &opt);
 }
 
@@ -3159,7 +3161,7 @@ int adacomp_decompress_average_sgd(const void *const *packed, uint32_t k_streams
                                    uint64_t n, uint32_t L_T, float lr, float mu, void *stream)
 {
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-    const Epilogue ep = {weights, momentum, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u};
+    const Epilogue ep = {weights, momentum, nullptr, lr, mu, 0.f, 0.f, 0.f, 0u, 0.f};
     return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
 }
 
@@ -3168,7 +3170,7 @@ int adacomp_decompress_average_adam(const void *const *packed, uint32_t k_stream
                                     void *stream)
 {
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-    const Epilogue ep = {weights, m, v, step_size, beta1, beta2, eps, 0.f, 1u};
+    const Epilogue ep = {weights, m, v, step_size, beta1, beta2, eps, 0.f, 1u, 0.f};
     return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
 }
 
