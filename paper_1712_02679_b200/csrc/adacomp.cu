@@ -1702,8 +1702,7 @@ __device__ inline u32 warp_add_group(const GroupSrc<Addr> &src, int R, int b0, i
     return bad;
 }
 
-// Tiles of at most 64 bins: G = 32 / (a warp's bins, rounded up to a power of two) lanes share a
-// bin.  For a group of up to four learners (in learner order) every lane gets its bin's count and
+// Tiles of at most 64 bins: G = 32 / (a warp's bins), rounded down, lanes share a bin.  For a group of up to four learners (in learner order) every lane gets its bin's count and
 // the words of the tile ahead of that bin from two warp scans over the tile's bin counts (lane j
 // holds bins j and j + 32; two learners share a register, 16 bits each), then the bin's lanes
 // take every G-th word of the bin.
@@ -1776,6 +1775,71 @@ __device__ inline u32 warp_add_group_by_bin(const GroupSrc<Addr> &src, int R, in
     return bad;
 }
 
+// out[e] += v (as add_at_if_valid) when `go` is not zero; nothing is read or written otherwise.
+__device__ inline void add_at_if(u32 e, float v, u32 go)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .f32 x;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "@p ld.shared.f32 x, [%0];\n\t"
+        "@p add.rn.f32 x, x, %1;\n\t"
+        "@p st.shared.f32 [%0], x;\n\t}"
+        ::"r"(e), "f"(v), "r"(go)
+        : "memory");
+}
+
+// L_T > 1000 (a tile is one bin): an item is up to four whole bins (GROUPED), or one bin, or a chunk of one,
+// and the decoding warps split its elements between them whatever the bins are.  For a group of up to four
+// learners (in learner order) the warp reads all the words of the item's `live` bins and adds those of its
+// own elements, [lo, lo + len) counted from the first bin's first element, at shared-memory address acc_at onwards.
+template <typename Word, bool SHARED, bool GROUPED, typename Addr>
+__device__ inline u32 warp_add_group_one_bin(const GroupSrc<Addr> &src, int R, u32 live, u32 lo, u32 len, u32 L_T, u32 acc_at,
+                                             int lane)
+{
+    constexpr u32 full = 0xffffffffu;
+    const u32 LT4 = L_T * 4u;
+    // lane q looks at learner q's bin counts: words ahead of the second, third and fourth bin, and all of them
+    u32 e[4] = {0u, 0u, 0u, 0u};
+    bool ok = true;
+    if (lane < R) {
+#pragma unroll
+        for (u32 b = 0; b < (GROUPED ? 4u : 1u); b++)
+            e[b] = (b ? e[b - 1] : 0u) + (b < live ? min(load_word<Word, SHARED>(src.counts + (Addr)(b * (u32)sizeof(Word))), L_T) : 0u);
+        ok = e[GROUPED ? 3 : 0] <= src.limit;
+    }
+    u32 bad = __any_sync(full, !ok) ? ADACOMP_DEV_BAD_STREAM : 0u;      // counts and directory disagree: nothing is read
+    const u32 mine_w = ok ? e[GROUPED ? 3 : 0] : 0u;
+    const u32 base = acc_at - 4u * lo;              // (wraps: only offsets of the warp's own elements are used)
+    u32 mx = 0, rsv = 0;
+#pragma unroll
+    for (int q = 0; q < kRoundMax; q++) {
+        if (q >= R) break;
+        const Addr words = bcast(src.words, q);
+        const u32 sbits = bcast(src.sbits, q), W = bcast(mine_w, q);
+        u32 e0 = 0, e1 = 0, e2 = 0;
+        if (GROUPED) {
+            e0 = bcast(e[0], q);
+            e1 = bcast(e[1], q);
+            e2 = bcast(e[2], q);
+        }
+        Addr wp = words + (Addr)((u32)lane * (u32)sizeof(Word));
+        for (u32 j = (u32)lane; j < W; j += 32u) {
+            const u32 word = load_word<Word, SHARED>(wp);
+            wp += (Addr)(32u * (u32)sizeof(Word));
+            mx = max(mx, word);
+            rsv |= (word >> 1) & ~word;
+            u32 off = word & ~3u;                   // 4 * (the element's place in the item)
+            if (GROUPED) off += ((u32)(j >= e0) + (u32)(j >= e1) + (u32)(j >= e2)) * LT4;
+            add_at_if(base + off, __uint_as_float(sbits ^ ((word << 30) & 0x80000000u)),
+                      (u32)((word & 1u) != 0u && (off >> 2) - lo < len && word < LT4));
+        }
+        __syncwarp();                               // learner order, element by element
+    }
+    if (__any_sync(full, (rsv & 1u) != 0u)) bad |= ADACOMP_DEV_RESERVED_CODE;
+    if (__any_sync(full, mx >= LT4)) bad |= ADACOMP_DEV_BAD_STREAM;
+    return bad;
+}
+
 // The same for learners read from global memory: rare, so kept out of line (the decoding warps'
 // registers go to the path that reads the slots).
 template <typename Word>
@@ -1791,19 +1855,80 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
     return warp_add_group<Word, false, u64>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
 }
 
+template <typename Word>
+__device__ __noinline__ u32 warp_add_group_one_bin_global(GroupSrc<u64> src, int R, u32 live, u32 lo, u32 len, u32 L_T,
+                                                          u32 acc_at, int lane)
+{
+    return warp_add_group_one_bin<Word, false, true, u64>(src, R, live, lo, len, L_T, acc_at, lane);
+}
+
+// How the warp path cuts a tensor into work items.  L_T <= 1000: an item is a tile.  L_T > 1000 (a tile is one
+// bin): an item is `group` consecutive tiles of at most 4096 elements together or, for L_T > 4096, one of
+// the `nchunks` chunks of at most 4096 elements of a tile (the tile's words are brought for each of them).
+struct WarpItems {
+    u32 group, nchunks, bins, elems, chunk_elems;   // tiles, chunks, bins and output elements of a group; elements of a chunk
+    u64 n_groups, n_items;
+};
+__host__ __device__ inline WarpItems warp_items(const Geometry &g)
+{
+    WarpItems w;
+    w.group = g.tile_bins == 1u && g.L_T <= (u32)kDecodeChunk ? (u32)kDecodeChunk / g.L_T : 1u;
+#ifdef ADACOMP_ONE_SIMPLE
+    w.group = 1u;
+#endif
+    w.bins = g.tile_bins * w.group;
+    w.elems = g.tile_elems * w.group;
+    w.nchunks = (w.elems + (u32)kDecodeChunk - 1u) / (u32)kDecodeChunk;
+    w.chunk_elems = g.tile_bins == 1u ? (u32)align_up((w.elems + w.nchunks - 1u) / w.nchunks, 16) : w.elems;
+    w.n_groups = (g.n_tiles + w.group - 1) / w.group;
+    w.n_items = w.n_groups * w.nchunks;
+    return w;
+}
+
+// A CTA's work items in turn: item v = group * nchunks + chunk, the CTA takes every stride-th.
+// (Stepped, not divided: a 64-bit division per item and warp costs more than a small tile.)
+struct ItemAt {
+    u64 tile;       // the tile (the group of tiles, where items are groups)
+    u32 chunk;
+};
+struct ItemStep {
+    u64 tiles;
+    u32 chunks, nchunks;
+};
+__device__ inline void next_item(ItemAt &p, const ItemStep &st)
+{
+    p.tile += st.tiles;
+    p.chunk += st.chunks;
+    if (p.chunk >= st.nchunks) {
+        p.chunk -= st.nchunks;
+        p.tile++;
+    }
+}
+
+// Room of one learner's bin counts of a tile in a slot.  The counts are bulk-copied from the
+// 16-byte boundary at or below their first byte, so a run that is not a multiple of 16 bytes
+// starts up to 15 bytes into its room.
+template <typename Word>
+__device__ inline u32 count_room(int TB)
+{
+    const u32 run = (u32)TB * (u32)sizeof(Word);
+    return run % 16u == 0 ? run : (u32)align_up(run + 15u, 16);
+}
+
 // Lays the slots out (see WarpDecSmem), then decodes.
-template <typename Word, bool MULTI, int OPT, int NW>
+template <typename Word, bool MULTI, int OPT, int NW, bool ONE>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv);
 
 //   s_wv   (OPT != 0) shared memory for a tile of weights, a tile of momentum and (Adam) a tile of second moments
-template <typename Word, int OPT, int NW>
+template <typename Word, int OPT, int NW, bool ONE>
 __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                                  const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int TB = (int)geo.tile_bins;
-    const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
+    const WarpItems wi = warp_items(geo);
+    const int TB = (int)wi.bins;
+    const u32 count_bytes = count_room<Word>(TB);
     const u32 k8 = (a.k + 7u) & ~7u;
     const u32 meta_bytes = kSlotHead + 4u * k8;                    // slot header + cnt[k8] + head[k8]
     if (tid == 0) {
@@ -1822,9 +1947,10 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         for (int h = 0; h < 2; h++) {
             const u32 l = (u32)lane + 32u * h;
             if (l < a.k) {
-                const u64 avg = s_nsel[l] / geo.n_tiles;
-                const u64 cap = min((u64)geo.tile_elems, avg + avg / 2 + 64);
-                ws.wcap[l] = (unsigned short)align_up(cap * sizeof(Word) + 16, 16);
+                const u64 avg = s_nsel[l] / wi.n_groups;
+                const u64 cap = min((u64)wi.elems, avg + avg / 2 + 64);
+                // (a learner alone always fits a slot; tiles of more than 4096 elements can have more words than that)
+                ws.wcap[l] = (unsigned short)min(align_up(cap * sizeof(Word) + 16, 16), (u64)((kSlotMax - meta_bytes - count_bytes) & ~15u));
             }
         }
         __syncwarp();
@@ -1852,23 +1978,29 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         }
     }
     __syncthreads();
-    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-    else decode_warps<Word, false, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT, NW, ONE>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    else decode_warps<Word, false, OPT, NW, ONE>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
 }
 
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
 // OPT: 0 the finished share goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
 // NW: decoding warps (warp NW is the loader); each owns 1/NW of the tile's bins ("quarter" below, whatever NW is).
-template <typename Word, bool MULTI, int OPT, int NW>
+// ONE: tiles of one bin (L_T > 1000, see WarpItems): each warp owns 1/NW of the item's elements instead.
+template <typename Word, bool MULTI, int OPT, int NW, bool ONE>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int TB = (int)geo.tile_bins;
+    const WarpItems wi = warp_items(geo);
+    const u32 group = ONE ? wi.group : 1u, nchunks = ONE ? wi.nchunks : 1u;
+    const u32 item_elems = ONE ? wi.elems : geo.tile_elems;        // output elements of an item's tiles
+    const int TB = ONE ? (int)wi.bins : (int)geo.tile_bins;        // bins of an item
     const u32 L_T = geo.L_T;
-    const u32 count_bytes = (u32)TB * (u32)sizeof(Word);           // a multiple of 16 on this path
-    const u64 first = blockIdx.x, stride = gridDim.x;
-    const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
+    const u32 count_bytes = count_room<Word>(TB);                  // room of a learner's bin counts in a slot
+    const u64 first = blockIdx.x, stride = gridDim.x, n_items = ONE ? wi.n_items : geo.n_tiles;
+    const u64 my_tiles = n_items > first ? (n_items - first + stride - 1) / stride : 0;     // items of this CTA
+    const ItemStep item_step = {stride / nchunks, (u32)(stride % nchunks), nchunks};
+    const ItemAt item0 = {first / nchunks, (u32)(first % nchunks)};
     const u32 k8 = (a.k + 7u) & ~7u;
     unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
     constexpr u32 full_mask = 0xffffffffu;
@@ -1886,24 +2018,25 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 const u32 j = (u32)lane + 32u * h;
                 if (valid && j < (MULTI ? (u32)ws.rcount[r] : a.k)) {
                     const u64 *dir = reinterpret_cast<const u64 *>(a.stream[(MULTI ? (u32)ws.rfirst[r] : 0u) + j] + geo.tile_off_at);
-                    d0[h] = dir[tile];
-                    d1[h] = dir[tile + 1];
+                    d0[h] = dir[tile * group];
+                    d1[h] = dir[ONE ? min((tile + 1) * group, geo.n_tiles) : tile + 1];
                 }
             }
         };
         // (no division in the loops: slot, use count and the look-ahead position step along)
-        u64 ptile = first, pit = 0;     // the item two ahead: its tile and round
+        ItemAt pa = item0;              // the item two ahead: its tile and round
+        u64 pit = 0;
         u32 pr = 0;
         auto step_ahead = [&]() {
             if (++pr == NR) {
                 pr = 0;
-                ptile += stride;
+                next_item(pa, item_step);
                 pit++;
             }
         };
-        load_dir(ptile, pr, pit < my_tiles, da0, da1);
+        load_dir(pa.tile, pr, pit < my_tiles, da0, da1);
         step_ahead();
-        load_dir(ptile, pr, pit < my_tiles, db0, db1);
+        load_dir(pa.tile, pr, pit < my_tiles, db0, db1);
         step_ahead();
         u32 my_coff[2] = {0, 0}, my_wcap[2] = {0, 0};       // one round: the lane's learners stay the same
 #pragma unroll
@@ -1916,12 +2049,14 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         }
         u64 issued = 0;                 // copies were started for items [0, issued)
         u32 s = 0, use = 0;             // the item's slot; how many times the slot was used before
-        u64 tile = first;
+        ItemAt cur = item0;
         bool failed = false;
-        for (u64 it = 0; it < my_tiles && !failed; it++, tile += stride) {
+        for (u64 it = 0; it < my_tiles && !failed; it++, next_item(cur, item_step)) {
+            const u64 tile = cur.tile;
             const u64 bin0 = tile * (u64)TB;
-            const u64 bins_left = geo.n_bins - bin0;
-            const u32 cbytes = bins_left >= (u64)TB ? count_bytes : (u32)align_up(bins_left * sizeof(Word), 16);   // last tile
+            // the tile's bin counts start `clead` bytes behind a 16-byte boundary: the copy starts at the boundary
+            const u32 clead = (u32)(bin0 * sizeof(Word)) & 15u;
+            const u32 cbytes = (u32)align_up(clead + min((u64)TB, geo.n_bins - bin0) * sizeof(Word), 16);
             for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
                 if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
                     ws.abort = 1;
@@ -1947,7 +2082,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     bool ok = true, fit = false;
                     if (active) {
                         const u32 l = l0 + j;
-                        ok = da1[h] >= da0[h] && da1[h] - da0[h] <= geo.tile_elems && da1[h] <= s_nsel[l];
+                        ok = da1[h] >= da0[h] && da1[h] - da0[h] <= item_elems && da1[h] <= s_nsel[l];
                         const u32 cnt = ok ? (u32)(da1[h] - da0[h]) : 0u;
                         src[h] = (u64)(uintptr_t)(a.stream[l] + geo.payload_at) + da0[h] * sizeof(Word);
                         const u32 head = (u32)(src[h] & 15u);
@@ -1980,7 +2115,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 for (int h = 0; h < 2; h++) {
                     const u32 j = (u32)lane + 32u * h;
                     if (j < staged) {
-                        bulk_load(sl + coff[h], a.stream[l0 + j] + geo.bin_cnt_at + bin0 * sizeof(Word), cbytes, &ws.full[s]);
+                        bulk_load(sl + coff[h], a.stream[l0 + j] + geo.bin_cnt_at + (bin0 * sizeof(Word) - clead), cbytes, &ws.full[s]);
                         if (wbytes[h])
                             bulk_load(sl + coff[h] + count_bytes, reinterpret_cast<const void *>(src[h] & ~(u64)15u), wbytes[h],
                                       &ws.full[s]);
@@ -1992,7 +2127,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     da0[h] = db0[h];
                     da1[h] = db1[h];
                 }
-                load_dir(ptile, pr, pit < my_tiles, db0, db1);
+                load_dir(pa.tile, pr, pit < my_tiles, db0, db1);
                 step_ahead();
             }
         }
@@ -2005,34 +2140,37 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     }
 
     // =============================== decoding warps ===============================
-    const int nb = TB / NW;                         // bins of a warp (the launcher picks NW to divide tile_bins)
+    const int nb = ONE ? 1 : TB / NW;               // bins of a warp (the launcher picks NW to divide tile_bins)
     const int b0 = warp * nb;
-    const u32 quarter = (u32)nb * L_T;              // output elements of a warp
+    const u32 quarter = ONE ? wi.chunk_elems / NW : (u32)nb * L_T;      // output elements of a warp
     const u32 acc_at = smem_addr(s_acc) + (u32)warp * quarter * 4u;
     float *const my_acc = s_acc + (u32)warp * quarter;
     u32 *const tmp = ws.tmp[warp];
     const bool vec_store = (quarter & 3u) == 0 && (geo.tile_elems & 3u) == 0;
     // tiles of at most 64 bins: G lanes share a bin
     const bool by_bin = sizeof(Word) == 2 || TB <= 64;     // (16-bit words: L_T >= 65, at most 60 bins)
-    int G = 32;
-    while (G * nb > 32) G >>= 1;
+    const int G = nb <= 32 ? 32 / nb : 1;           // (need not be a power of two: 5 bins take 6 lanes each)
     const int my_local = lane / G, my_r = lane % G;
     const int my_bin = my_local < nb ? b0 + my_local : TB;
     const u32 mine_at = smem_addr(s_acc) + (u32)my_bin * L_T * 4u;
     u32 bad = 0;
     PHASE_DECL;
     u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
-    u64 tile = first;
+    ItemAt cur = item0;
     bool failed = false;
     // (OPT != 0) the warp's quarters of the staged weights, momentum and second moments
     float *const wq = s_wv + (u32)warp * quarter, *const vq = s_wv + kDecodeChunk + (u32)warp * quarter;
     float *const uq = s_wv + 2 * kDecodeChunk + (u32)warp * quarter;
     u32 wv_use = 0;                                 // fetches of the quarters so far
-    for (u64 it = 0; it < my_tiles; it++, tile += stride) {
+    for (u64 it = 0; it < my_tiles; it++, next_item(cur, item_step)) {
+        const u64 tile = cur.tile;
         const u64 bin0 = tile * (u64)TB;
         const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
-        const u64 out0 = tile * (u64)geo.tile_elems + (u64)warp * quarter;
-        const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
+        const u32 clead = (u32)(bin0 * sizeof(Word)) & 15u;          // where the counts start in their room (see the loader)
+        const u32 lo = (ONE ? cur.chunk * wi.chunk_elems : 0u) + (u32)warp * quarter;       // the warp's first element, in the item
+        const u64 out0 = tile * (u64)item_elems + lo;
+        const u32 in_tile = lo < item_elems ? min(quarter, item_elems - lo) : 0u;
+        const u32 len = out0 < geo.n ? (u32)min((u64)in_tile, geo.n - out0) : 0u;
         const bool whole = vec_store && len == quarter;
         if (OPT != 0 && whole && lane == 0) {
             // the warp's quarters of the optimizer's arrays travel while the words are added
@@ -2064,12 +2202,14 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 GroupSrc<u32> src = {0u, 0u, 0u, 0u};
                 if (lane < R) {
                     const u32 j = g0 + (u32)lane, l = l0 + j;
-                    src.counts = sl_at + ws.coff[l];
-                    src.words = src.counts + count_bytes + m_head[j];
+                    src.counts = sl_at + ws.coff[l] + clead;
+                    src.words = sl_at + ws.coff[l] + count_bytes + m_head[j];
                     src.limit = m_cnt[j];
                     src.sbits = __float_as_uint(s_scale[l]);
                 }
-                if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+                if (ONE && TB == 1) bad |= warp_add_group_one_bin<Word, true, false, u32>(src, R, live, lo, len, L_T, acc_at, lane);
+                else if (ONE) bad |= warp_add_group_one_bin<Word, true, true, u32>(src, R, live, lo, len, L_T, acc_at, lane);
+                else if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
                 else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
             if (lane == 0) mbar_arrive(&ws.empty[s]);   // (the group's last __syncwarp orders the warp's reads before it)
@@ -2084,15 +2224,16 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     const u32 l = l0 + g0 + (u32)lane;
                     const unsigned char *st = a.stream[l];
                     const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
-                    const u64 w0 = dir[tile], w1 = dir[tile + 1];
-                    ok = w1 >= w0 && w1 - w0 <= geo.tile_elems && w1 <= s_nsel[l];
+                    const u64 w0 = dir[tile * group], w1 = dir[ONE ? min((tile + 1) * group, geo.n_tiles) : tile + 1];
+                    ok = w1 >= w0 && w1 - w0 <= item_elems && w1 <= s_nsel[l];
                     src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
                     src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
                     src.limit = ok ? (u32)(w1 - w0) : 0u;
                     src.sbits = __float_as_uint(s_scale[l]);
                 }
                 if (__any_sync(full_mask, !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
-                if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
+                if (ONE) bad |= warp_add_group_one_bin_global<Word>(src, R, live, lo, len, L_T, acc_at, lane);
+                else if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
                 else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
             PHASE_CLOCK(2, t0);
@@ -2263,12 +2404,12 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
     }
 }
 
-// Tiles the warp path takes: 4..96 bins, a multiple of 4, bin-count runs that are a multiple of 16
-// bytes (so that everything a tile needs can be bulk-copied), at most 4096 elements.
+// Tiles the warp path takes: 4..96 bins, a multiple of 4, at most 4096 elements (L_T = 41..1000); and the
+// tiles of one bin (L_T > 1000).
 __host__ __device__ inline bool warp_path(const Geometry &g)
 {
-    return g.tile_bins >= 4u && g.tile_bins <= (u32)kSmallBins && g.tile_bins % 4u == 0 && (g.tile_bins * g.w) % 16u == 0 &&
-           g.tile_elems <= (u32)kDecodeChunk;
+    if (g.tile_bins == 1u) return g.L_T > 1000u;
+    return g.tile_bins >= 4u && g.tile_bins <= (u32)kSmallBins && g.tile_bins % 4u == 0 && g.tile_elems <= (u32)kDecodeChunk;
 }
 
 // Every CTA of a decode kernel reads and cross-checks the k headers itself: the decision is
@@ -2327,11 +2468,18 @@ decode_sum_warps(DecodeArgs a)
     u64 n;
     if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
-    if (!warp_path(geo) || geo.tile_bins % (u32)NW != 0) return;      // (the launcher picks NW from the shape it was given)
+    // (the launcher picks NW from the shape it was given: a divisor of the tile's bins; 4 for tiles of one bin)
+    if (!warp_path(geo) || (geo.tile_bins == 1u ? NW != 4 : geo.tile_bins % (u32)NW != 0)) return;
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
     extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles
-    if (geo.w == 1u) decode_warps_any<unsigned char, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
-    else decode_warps_any<unsigned short, OPT, NW>(a, geo, s_acc, ws, s_scale, s_nsel, OPT ? s_dyn : nullptr);
+    float *const s_wv = OPT ? s_dyn : nullptr;
+    if (geo.w == 1u) {
+        decode_warps_any<unsigned char, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    } else if (geo.tile_bins == 1u) {
+        if constexpr (NW == 4) decode_warps_any<unsigned short, OPT, NW, true>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    } else {
+        decode_warps_any<unsigned short, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    }
 }
 
 __global__ void __launch_bounds__(kDecodeThreads, 6)
@@ -2690,11 +2838,12 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     u64 grid = (u64)info->sms * info->decode_per_sm, grid_w = (u64)info->sms * info->decode_warps_per_sm;
     bool warps = true, others = true;   // the shape is on the device: both kernels go, one of them returns at once
     if (hint_L_T) {                     // the shape is known on the host: one kernel, no more CTAs than work items
-        const u64 items = decode_items(hint_n, hint_L_T);
+        const Geometry hg = make_geometry(hint_n, hint_L_T);
+        warps = warp_path(hg);
+        others = !warps;
+        const u64 items = warps ? warp_items(hg).n_items : decode_items(hint_n, hint_L_T);
         grid = items < grid ? (items ? items : 1) : grid;
         grid_w = items < grid_w ? (items ? items : 1) : grid_w;
-        warps = warp_path(make_geometry(hint_n, hint_L_T));
-        others = !warps;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (warps && ep) {
@@ -2704,7 +2853,7 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         if (!per) return ADACOMP_ERR_CUDA;
         u64 grid_s = (u64)info->sms * per;
         if (hint_L_T) {
-            const u64 items = decode_items(hint_n, hint_L_T);
+            const u64 items = warp_items(make_geometry(hint_n, hint_L_T)).n_items;
             grid_s = items < grid_s ? (items ? items : 1) : grid_s;
         }
         const unsigned g = (unsigned)grid_s;

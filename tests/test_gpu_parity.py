@@ -149,7 +149,15 @@ def gpu_decode(streams, n):
                                      # then 16, 10, 8, 4, 2 and 1 bins per warp with 2 .. 32 lanes per bin
                                      (41, 96 * 41 * 9 + 5, 3), (48, 80 * 48 * 7 + 1, 4), (49, 80 * 49 * 5, 2),
                                      (62, 64 * 62 * 6 + 9, 3), (100, 40 * 100 * 5 + 7, 3), (125, 32 * 125 * 5 + 3, 5),
-                                     (250, 16 * 250 * 6 + 11, 3), (400, 8 * 400 * 7 + 2, 9), (1000, 4 * 1000 * 6 + 13, 3)])
+                                     (250, 16 * 250 * 6 + 11, 3), (400, 8 * 400 * 7 + 2, 9), (1000, 4 * 1000 * 6 + 13, 3),
+                                     # bin-count runs of a tile that are not a multiple of 16 bytes; 3, 5 and 15 bins per warp
+                                     (52, 76 * 52 * 9 + 3, 4), (58, 68 * 58 * 7 + 50, 3), (63, 60 * 63 * 8 + 1, 5),
+                                     (66, 60 * 66 * 5 + 65, 2), (200, 20 * 200 * 9 + 199, 4), (300, 12 * 300 * 7 + 8, 3),
+                                     (800, 4 * 800 * 11 + 5, 6),
+                                     # one bin per tile: the warps share it, in one to four chunks
+                                     (1001, 1001 * 23 + 17, 5), (2000, 2000 * 40 + 3, 4), (2001, 2001 * 21 + 1999, 3),
+                                     (4096, 4096 * 9 + 1, 3), (4097, 4097 * 7 + 5, 3), (5000, 5000 * 30 + 123, 6),
+                                     (8192, 8192 * 5, 2), (12345, 12345 * 9 + 12000, 3), (16384, 16384 * 6 + 11, 4)])
 def test_decode_sum_matches_oracle(L_T, n, k):
     rng = np.random.default_rng(L_T + n + k)
     streams_gpu, streams_cpu = [], []
@@ -172,7 +180,7 @@ def test_decode_sum_dense_streams_overflow_the_prefetch_stage():
     """Every element sent (all ties): 4000 words per tile and learner, so only a few learners'
     words fit the decoder's staging buffer and the rest take its one-at-a-time path."""
     rng = np.random.default_rng(8)
-    for L_T, n, k in [(50, 4000 * 9 + 123, 12), (500, 4000 * 5 + 77, 7)]:
+    for L_T, n, k in [(50, 4000 * 9 + 123, 12), (500, 4000 * 5 + 77, 7), (5000, 5000 * 5 + 77, 5), (16384, 16384 * 3 + 5, 3)]:
         streams = []
         for l in range(k):
             sign = np.where(rng.random(n) < 0.5, -1.0, 1.0).astype(np.float32)
