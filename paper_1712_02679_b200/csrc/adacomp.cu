@@ -1231,9 +1231,10 @@ struct WarpDecSmem {
 };
 
 // A slot holds one round of one tile: the learners of the round, as many as fit a slot with their
-// regions (all k of them when k is small).  It starts with {u32 staged, u32 bad} (the first
-// `staged` learners of the round are in the slot; failed directory checks), 8 bytes of padding,
-// then u16 cnt[k8] and u16 head[k8], indexed by the learner's place in the round: its words in
+// regions (all k of them when k is small).  It starts with {u32 staged, u32 bad, u32 item} (the first
+// `staged` learners of the round are in the slot; failed directory checks; where items are 4096
+// elements: the first one's place in its bin, the bins of the item << 16, the counts' offset in
+// their room << 24), 4 bytes of padding, then u16 cnt[k8] and u16 head[k8], indexed by the learner's place in the round: its words in
 // this tile and the byte offset of the first one in its word region.
 constexpr u32 kSlotHead = 16;
 
@@ -1495,13 +1496,15 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
 }
 
 // ---------------------------------------------------------------------------------
-// decode, warp path: tiles of 4..96 bins whose bin-count run is a multiple of 16 bytes
-// (L_T = 50 and 500 among them).
+// decode, warp path: every L_T above 40.  A work item is a tile of 4..96 bins (L_T <= 1000) or,
+// where a tile is one bin (L_T > 1000), 4096 consecutive output elements and the 1 to 6 bins
+// they lie in.
 //
-// Warp 4 is a loader: for every tile of this CTA, a lane per learner reads the learner's two
+// Warp 4 is a loader: for every item of this CTA, a lane per learner reads the learner's two
 // directory entries (two steps ahead) and bulk-copies (TMA, no multicast) that learner's bin
-// counts and words of the tile into the learner's fixed region of a shared-memory slot; the
-// slots form a ring of up to kSlots in flight.  Region sizes are set once per launch from the
+// counts and words of the item into the learner's fixed region of a shared-memory slot; the
+// slots form a ring of up to kSlots in flight.  (A bulk copy starts on a 16-byte boundary: counts
+// and words are copied from the boundary at or below their first byte and found at the offset.)  Region sizes are set once per launch from the
 // streams' word totals (1.5 times a tile's average plus slack).  When the k regions do not fit
 // one slot together, a tile takes several rounds, each a slot of its own with the next learners
 // in order.  A learner whose words of some tile do not fit its region is read by the decoding
@@ -1515,7 +1518,9 @@ __device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSm
 // contributions in learner order), gives the slot back, hands its quarter to one bulk copy
 // (TMA store: the output does not pass through the warps' load/store path, which the adds keep
 // busy) and zeroes it once the copy has read it.
-// Two schemes for the adds.  Tiles of at most 64 bins (16-bit words among them): G lanes share a
+// Three schemes for the adds.  Items of 4096 elements (L_T > 1000): a warp owns a quarter of the
+// elements whatever the bins are, reads the words of the bins its elements lie in and adds those
+// that are its own.  Tiles of at most 64 bins (16-bit words among them): G lanes share a
 // bin and take every G-th word of it.  Tiles of more bins (8-bit words, L_T <= 58): the warp works
 // by word, lane j takes word j of the warp's run of words, 32 at a time; the bin of a word comes
 // from the bin counts: the lanes that hold the warp's bins (at most 24) scan their counts, raise
@@ -1788,50 +1793,65 @@ __device__ inline void add_at_if(u32 e, float v, u32 go)
         : "memory");
 }
 
-// L_T > 1000 (a tile is one bin): an item is up to four whole bins (GROUPED), or one bin, or a chunk of one,
-// and the decoding warps split its elements between them whatever the bins are.  For a group of up to four
-// learners (in learner order) the warp reads all the words of the item's `live` bins and adds those of its
-// own elements, [lo, lo + len) counted from the first bin's first element, at shared-memory address acc_at onwards.
-template <typename Word, bool SHARED, bool GROUPED, typename Addr>
-__device__ inline u32 warp_add_group_one_bin(const GroupSrc<Addr> &src, int R, u32 live, u32 lo, u32 len, u32 L_T, u32 acc_at,
-                                             int lane)
+// L_T > 1000 (a tile is one bin): an item is 4096 consecutive output elements, which lie in `live` bins (at
+// most 6), and the decoding warps split the elements between them whatever the bins are.  For a group of
+// up to four learners (in learner order) the warp reads the words of the bins its own elements lie in (at
+// most 3), bin by bin, and adds those that are its own: elements [lo, lo + len) counted from the first
+// bin's first element, at shared-memory address acc_at onwards.
+template <typename Word, bool SHARED, typename Addr>
+__device__ inline u32 warp_add_group_flat(const GroupSrc<Addr> &src, int R, u32 live, u32 lo, u32 len, u32 L_T, u32 acc_at,
+                                          int lane)
 {
     constexpr u32 full = 0xffffffffu;
+    constexpr u32 kBins = 6;
     const u32 LT4 = L_T * 4u;
-    // lane q looks at learner q's bin counts: words ahead of the second, third and fourth bin, and all of them
-    u32 e[4] = {0u, 0u, 0u, 0u};
+    // the bins (of the item) of the warp's first and last element
+    u32 wf = 0, wl = 0;
+#pragma unroll
+    for (u32 i = 1; i < kBins; i++) {
+        wf += (u32)(lo >= i * L_T);
+        wl += (u32)(lo + len > i * L_T);
+    }
+    // lane q looks at learner q's bin counts: P[t] words lie in the bins ahead of bin wf + t
+    u32 P[4] = {0u, 0u, 0u, 0u};
     bool ok = true;
     if (lane < R) {
+        u32 run = 0;
 #pragma unroll
-        for (u32 b = 0; b < (GROUPED ? 4u : 1u); b++)
-            e[b] = (b ? e[b - 1] : 0u) + (b < live ? min(load_word<Word, SHARED>(src.counts + (Addr)(b * (u32)sizeof(Word))), L_T) : 0u);
-        ok = e[GROUPED ? 3 : 0] <= src.limit;
+        for (u32 b = 0; b < kBins; b++) {
+            const u32 c = b < live ? min(load_word<Word, SHARED>(src.counts + (Addr)(b * (u32)sizeof(Word))), L_T) : 0u;
+#pragma unroll
+            for (u32 t = 0; t < 4u; t++)
+                if (b < wf + t) P[t] += c;
+            run += c;
+        }
+        ok = run <= src.limit;
+        if (!ok || len == 0u) P[0] = P[1] = P[2] = P[3] = 0u;
     }
     u32 bad = __any_sync(full, !ok) ? ADACOMP_DEV_BAD_STREAM : 0u;      // counts and directory disagree: nothing is read
-    const u32 mine_w = ok ? e[GROUPED ? 3 : 0] : 0u;
-    const u32 base = acc_at - 4u * lo;              // (wraps: only offsets of the warp's own elements are used)
     u32 mx = 0, rsv = 0;
 #pragma unroll
     for (int q = 0; q < kRoundMax; q++) {
         if (q >= R) break;
         const Addr words = bcast(src.words, q);
-        const u32 sbits = bcast(src.sbits, q), W = bcast(mine_w, q);
-        u32 e0 = 0, e1 = 0, e2 = 0;
-        if (GROUPED) {
-            e0 = bcast(e[0], q);
-            e1 = bcast(e[1], q);
-            e2 = bcast(e[2], q);
-        }
-        Addr wp = words + (Addr)((u32)lane * (u32)sizeof(Word));
-        for (u32 j = (u32)lane; j < W; j += 32u) {
-            const u32 word = load_word<Word, SHARED>(wp);
-            wp += (Addr)(32u * (u32)sizeof(Word));
-            mx = max(mx, word);
-            rsv |= (word >> 1) & ~word;
-            u32 off = word & ~3u;                   // 4 * (the element's place in the item)
-            if (GROUPED) off += ((u32)(j >= e0) + (u32)(j >= e1) + (u32)(j >= e2)) * LT4;
-            add_at_if(base + off, __uint_as_float(sbits ^ ((word << 30) & 0x80000000u)),
-                      (u32)((word & 1u) != 0u && (off >> 2) - lo < len && word < LT4));
+        const u32 sbits = bcast(src.sbits, q);
+        u32 j1 = bcast(P[0], q);
+#pragma unroll
+        for (u32 t = 0; t < 3u; t++) {
+            const u32 j0 = j1;
+            j1 = bcast(P[t + 1], q);
+            if (wf + t > wl) continue;
+            const u32 first = (wf + t) * L_T - lo;          // the bin's first element, counted from the warp's (wraps)
+            const u32 base = acc_at + 4u * first;
+            Addr wp = words + (Addr)((j0 + (u32)lane) * (u32)sizeof(Word));
+            for (u32 j = j0 + (u32)lane; j < j1; j += 32u) {
+                const u32 word = load_word<Word, SHARED>(wp);
+                wp += (Addr)(32u * (u32)sizeof(Word));
+                mx = max(mx, word);
+                rsv |= (word >> 1) & ~word;
+                add_at_if(base + (word & ~3u), __uint_as_float(sbits ^ ((word << 30) & 0x80000000u)),
+                          (u32)((word & 1u) != 0u && first + (word >> 2) < len && word < LT4));
+            }
         }
         __syncwarp();                               // learner order, element by element
     }
@@ -1856,53 +1876,62 @@ __device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int 
 }
 
 template <typename Word>
-__device__ __noinline__ u32 warp_add_group_one_bin_global(GroupSrc<u64> src, int R, u32 live, u32 lo, u32 len, u32 L_T,
-                                                          u32 acc_at, int lane)
+__device__ __noinline__ u32 warp_add_group_flat_global(GroupSrc<u64> src, int R, u32 live, u32 lo, u32 len, u32 L_T,
+                                                       u32 acc_at, int lane)
 {
-    return warp_add_group_one_bin<Word, false, true, u64>(src, R, live, lo, len, L_T, acc_at, lane);
+    return warp_add_group_flat<Word, false, u64>(src, R, live, lo, len, L_T, acc_at, lane);
 }
 
 // How the warp path cuts a tensor into work items.  L_T <= 1000: an item is a tile.  L_T > 1000 (a tile is one
-// bin): an item is `group` consecutive tiles of at most 4096 elements together or, for L_T > 4096, one of
-// the `nchunks` chunks of at most 4096 elements of a tile (the tile's words are brought for each of them).
+// bin of up to 16384 elements): item v is the output elements [4096 v, 4096 v + 4096), whatever bins they lie in;
+// it needs the words of every bin it touches, at most `max_bins` of them.
 struct WarpItems {
-    u32 group, nchunks, bins, elems, chunk_elems;   // tiles, chunks, bins and output elements of a group; elements of a chunk
-    u64 n_groups, n_items;
+    u64 n_items;
+    u32 max_bins;   // bins an item needs the counts of
 };
 __host__ __device__ inline WarpItems warp_items(const Geometry &g)
 {
     WarpItems w;
-    w.group = g.tile_bins == 1u && g.L_T <= (u32)kDecodeChunk ? (u32)kDecodeChunk / g.L_T : 1u;
-#ifdef ADACOMP_ONE_SIMPLE
-    w.group = 1u;
-#endif
-    w.bins = g.tile_bins * w.group;
-    w.elems = g.tile_elems * w.group;
-    w.nchunks = (w.elems + (u32)kDecodeChunk - 1u) / (u32)kDecodeChunk;
-    w.chunk_elems = g.tile_bins == 1u ? (u32)align_up((w.elems + w.nchunks - 1u) / w.nchunks, 16) : w.elems;
-    w.n_groups = (g.n_tiles + w.group - 1) / w.group;
-    w.n_items = w.n_groups * w.nchunks;
+    if (g.tile_bins == 1u) {
+        w.n_items = (g.n + (u64)kDecodeChunk - 1) / (u64)kDecodeChunk;
+        w.max_bins = ((u32)kDecodeChunk - 2u) / g.L_T + 2u;
+    } else {
+        w.n_items = g.n_tiles;
+        w.max_bins = g.tile_bins;
+    }
     return w;
 }
 
-// A CTA's work items in turn: item v = group * nchunks + chunk, the CTA takes every stride-th.
-// (Stepped, not divided: a 64-bit division per item and warp costs more than a small tile.)
+// A CTA's work items in turn: it takes every stride-th.  Where items are tiles, `tile` is all there is to
+// one.  Where they are 4096 output elements (L_T > 1000), `tile` is the bin (= tile) of the item's first
+// element and `at` that element's place in the bin.  (Stepped, not divided: a 64-bit division per item and
+// warp costs more than a small item.)
+// (32 bits do: the warp path takes tensors of less than 2^40 elements)
 struct ItemAt {
-    u64 tile;       // the tile (the group of tiles, where items are groups)
-    u32 chunk;
+    u32 v, tile, at;
 };
 struct ItemStep {
-    u64 tiles;
-    u32 chunks, nchunks;
+    u32 items, tiles, at, L_T;
 };
 __device__ inline void next_item(ItemAt &p, const ItemStep &st)
 {
+    p.v += st.items;
     p.tile += st.tiles;
-    p.chunk += st.chunks;
-    if (p.chunk >= st.nchunks) {
-        p.chunk -= st.nchunks;
+    p.at += st.at;
+    if (p.at >= st.L_T) {
+        p.at -= st.L_T;
         p.tile++;
     }
+}
+// Bins that `len` (> 0) elements touch, the first of them element `at` of its bin.
+__device__ inline u32 bins_touched(u32 at, u32 len, u32 L_T)
+{
+    u32 last = at + len - 1u, bins = 1u;
+    while (last >= L_T) {
+        last -= L_T;
+        bins++;
+    }
+    return bins;
 }
 
 // Room of one learner's bin counts of a tile in a slot.  The counts are bulk-copied from the
@@ -1927,7 +1956,7 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const WarpItems wi = warp_items(geo);
-    const int TB = (int)wi.bins;
+    const int TB = (int)wi.max_bins;
     const u32 count_bytes = count_room<Word>(TB);
     const u32 k8 = (a.k + 7u) & ~7u;
     const u32 meta_bytes = kSlotHead + 4u * k8;                    // slot header + cnt[k8] + head[k8]
@@ -1947,8 +1976,9 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         for (int h = 0; h < 2; h++) {
             const u32 l = (u32)lane + 32u * h;
             if (l < a.k) {
-                const u64 avg = s_nsel[l] / wi.n_groups;
-                const u64 cap = min((u64)wi.elems, avg + avg / 2 + 64);
+                // (an item of 4096 elements brings the words of the bins at its ends whole: L_T more elements, on average)
+                const u64 per = s_nsel[l] / wi.n_items, avg = ONE ? per + per * geo.L_T / (u64)kDecodeChunk : per;
+                const u64 cap = min(ONE ? (u64)wi.max_bins * geo.L_T : (u64)geo.tile_elems, avg + avg / 2 + 64);
                 // (a learner alone always fits a slot; tiles of more than 4096 elements can have more words than that)
                 ws.wcap[l] = (unsigned short)min(align_up(cap * sizeof(Word) + 16, 16), (u64)((kSlotMax - meta_bytes - count_bytes) & ~15u));
             }
@@ -1985,22 +2015,18 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
 // OPT: 0 the finished share goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
 // NW: decoding warps (warp NW is the loader); each owns 1/NW of the tile's bins ("quarter" below, whatever NW is).
-// ONE: tiles of one bin (L_T > 1000, see WarpItems): each warp owns 1/NW of the item's elements instead.
+// ONE: tiles of one bin (L_T > 1000): an item is 4096 output elements (see WarpItems) and each warp owns 1/NW of them.
 template <typename Word, bool MULTI, int OPT, int NW, bool ONE>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const WarpItems wi = warp_items(geo);
-    const u32 group = ONE ? wi.group : 1u, nchunks = ONE ? wi.nchunks : 1u;
-    const u32 item_elems = ONE ? wi.elems : geo.tile_elems;        // output elements of an item's tiles
-    const int TB = ONE ? (int)wi.bins : (int)geo.tile_bins;        // bins of an item
+    const int TB = ONE ? (int)wi.max_bins : (int)geo.tile_bins;    // bins of an item (ONE: at most)
     const u32 L_T = geo.L_T;
     const u32 count_bytes = count_room<Word>(TB);                  // room of a learner's bin counts in a slot
     const u64 first = blockIdx.x, stride = gridDim.x, n_items = ONE ? wi.n_items : geo.n_tiles;
     const u64 my_tiles = n_items > first ? (n_items - first + stride - 1) / stride : 0;     // items of this CTA
-    const ItemStep item_step = {stride / nchunks, (u32)(stride % nchunks), nchunks};
-    const ItemAt item0 = {first / nchunks, (u32)(first % nchunks)};
     const u32 k8 = (a.k + 7u) & ~7u;
     unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
     constexpr u32 full_mask = 0xffffffffu;
@@ -2011,32 +2037,47 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         // ================================ loader warp ================================
         // An item is one round of one tile; lane j (and j + 32) looks after the j-th learner of the
         // round.  The learners' directory entries are read two items ahead.
+        // With them travels (ONE) the item's first bin and {place of the item's first element in that bin,
+        // bins of the item << 16, offset of the counts in their room << 24}: the loader steps through the
+        // bins once, for the item two ahead.
         u64 da0[2] = {0, 0}, da1[2] = {0, 0}, db0[2] = {0, 0}, db1[2] = {0, 0};
-        auto load_dir = [&](u64 tile, u32 r, bool valid, u64 *d0, u64 *d1) {
+        u32 ta = 0, ia = 0, tb = 0, ib = 0;
+        const u32 last_item = (u32)(n_items - 1), last_len = (u32)(geo.n - (n_items - 1) * (u64)kDecodeChunk);   // (ONE)
+        auto load_dir = [&](u64 tile, const ItemAt &p, u32 r, bool valid, u64 *d0, u64 *d1, u32 &t, u32 &info) {
+            u32 tiles = 1u;             // tiles (each a bin) of the item
+            if (ONE && valid) {
+                tiles = bins_touched(p.at, p.v == last_item ? last_len : (u32)kDecodeChunk, L_T);
+                t = p.tile;
+                info = p.at | (tiles << 16) | (((p.tile * (u32)sizeof(Word)) & 15u) << 24);
+                tile = p.tile;
+            }
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const u32 j = (u32)lane + 32u * h;
                 if (valid && j < (MULTI ? (u32)ws.rcount[r] : a.k)) {
                     const u64 *dir = reinterpret_cast<const u64 *>(a.stream[(MULTI ? (u32)ws.rfirst[r] : 0u) + j] + geo.tile_off_at);
-                    d0[h] = dir[tile * group];
-                    d1[h] = dir[ONE ? min((tile + 1) * group, geo.n_tiles) : tile + 1];
+                    d0[h] = dir[tile];
+                    d1[h] = dir[tile + tiles];
                 }
             }
         };
         // (no division in the loops: slot, use count and the look-ahead position step along)
-        ItemAt pa = item0;              // the item two ahead: its tile and round
-        u64 pit = 0;
+        // the item two ahead: its tile (ONE: its place, stepped in elements: the stride as whole bins and a rest) and round
+        u64 ptile = first, pit = 0;
+        const ItemStep item_step = {(u32)stride, (u32)(stride * (u64)kDecodeChunk / L_T), (u32)(stride * (u64)kDecodeChunk % L_T), L_T};
+        ItemAt pa = {(u32)first, (u32)(first * (u64)kDecodeChunk / L_T), (u32)(first * (u64)kDecodeChunk % L_T)};
         u32 pr = 0;
         auto step_ahead = [&]() {
             if (++pr == NR) {
                 pr = 0;
-                next_item(pa, item_step);
+                if (ONE) next_item(pa, item_step);
+                else ptile += stride;
                 pit++;
             }
         };
-        load_dir(pa.tile, pr, pit < my_tiles, da0, da1);
+        load_dir(ptile, pa, pr, pit < my_tiles, da0, da1, ta, ia);
         step_ahead();
-        load_dir(pa.tile, pr, pit < my_tiles, db0, db1);
+        load_dir(ptile, pa, pr, pit < my_tiles, db0, db1, tb, ib);
         step_ahead();
         u32 my_coff[2] = {0, 0}, my_wcap[2] = {0, 0};       // one round: the lane's learners stay the same
 #pragma unroll
@@ -2049,15 +2090,16 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         }
         u64 issued = 0;                 // copies were started for items [0, issued)
         u32 s = 0, use = 0;             // the item's slot; how many times the slot was used before
-        ItemAt cur = item0;
+        u64 tile = first;
         bool failed = false;
-        for (u64 it = 0; it < my_tiles && !failed; it++, next_item(cur, item_step)) {
-            const u64 tile = cur.tile;
-            const u64 bin0 = tile * (u64)TB;
-            // the tile's bin counts start `clead` bytes behind a 16-byte boundary: the copy starts at the boundary
-            const u32 clead = (u32)(bin0 * sizeof(Word)) & 15u;
-            const u32 cbytes = (u32)align_up(clead + min((u64)TB, geo.n_bins - bin0) * sizeof(Word), 16);
+        for (u64 it = 0; it < my_tiles && !failed; it++, tile += stride) {
             for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
+                const u64 bin0 = ONE ? (u64)ta : tile * (u64)TB;
+                const u32 live = ONE ? (ia >> 16) & 0xffu : (u32)min((u64)TB, geo.n_bins - bin0);
+                const u32 item_elems = ONE ? live * L_T : geo.tile_elems;      // more words than that are an error
+                // the item's bin counts start `clead` bytes behind a 16-byte boundary: the copy starts at the boundary
+                const u32 clead = ONE ? ia >> 24 : (u32)(bin0 * sizeof(Word)) & 15u;
+                const u32 cbytes = (u32)align_up(clead + live * (u32)sizeof(Word), 16);
                 if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
                     ws.abort = 1;
                     raise_status(ADACOMP_DEV_TIMEOUT);
@@ -2103,6 +2145,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 if (lane == 0) {
                     reinterpret_cast<u32 *>(sl)[0] = staged;
                     reinterpret_cast<u32 *>(sl)[1] = bad;
+                    if (ONE) reinterpret_cast<u32 *>(sl)[2] = ia;
                 }
                 __syncwarp();
                 u32 expect = 0;
@@ -2127,7 +2170,9 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     da0[h] = db0[h];
                     da1[h] = db1[h];
                 }
-                load_dir(pa.tile, pr, pit < my_tiles, db0, db1);
+                ta = tb;
+                ia = ib;
+                load_dir(ptile, pa, pr, pit < my_tiles, db0, db1, tb, ib);
                 step_ahead();
             }
         }
@@ -2142,11 +2187,11 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     // =============================== decoding warps ===============================
     const int nb = ONE ? 1 : TB / NW;               // bins of a warp (the launcher picks NW to divide tile_bins)
     const int b0 = warp * nb;
-    const u32 quarter = ONE ? wi.chunk_elems / NW : (u32)nb * L_T;      // output elements of a warp
+    const u32 quarter = ONE ? (u32)kDecodeChunk / NW : (u32)nb * L_T;   // output elements of a warp
     const u32 acc_at = smem_addr(s_acc) + (u32)warp * quarter * 4u;
     float *const my_acc = s_acc + (u32)warp * quarter;
     u32 *const tmp = ws.tmp[warp];
-    const bool vec_store = (quarter & 3u) == 0 && (geo.tile_elems & 3u) == 0;
+    const bool vec_store = (quarter & 3u) == 0 && (ONE || (geo.tile_elems & 3u) == 0);
     // tiles of at most 64 bins: G lanes share a bin
     const bool by_bin = sizeof(Word) == 2 || TB <= 64;     // (16-bit words: L_T >= 65, at most 60 bins)
     const int G = nb <= 32 ? 32 / nb : 1;           // (need not be a power of two: 5 bins take 6 lanes each)
@@ -2156,21 +2201,19 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     u32 bad = 0;
     PHASE_DECL;
     u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
-    ItemAt cur = item0;
+    u64 v = first;                                  // the item
     bool failed = false;
     // (OPT != 0) the warp's quarters of the staged weights, momentum and second moments
     float *const wq = s_wv + (u32)warp * quarter, *const vq = s_wv + kDecodeChunk + (u32)warp * quarter;
     float *const uq = s_wv + 2 * kDecodeChunk + (u32)warp * quarter;
     u32 wv_use = 0;                                 // fetches of the quarters so far
-    for (u64 it = 0; it < my_tiles; it++, next_item(cur, item_step)) {
-        const u64 tile = cur.tile;
-        const u64 bin0 = tile * (u64)TB;
-        const u32 live = (u32)min((u64)TB, geo.n_bins - bin0);
-        const u32 clead = (u32)(bin0 * sizeof(Word)) & 15u;          // where the counts start in their room (see the loader)
-        const u32 lo = (ONE ? cur.chunk * wi.chunk_elems : 0u) + (u32)warp * quarter;       // the warp's first element, in the item
-        const u64 out0 = tile * (u64)item_elems + lo;
-        const u32 in_tile = lo < item_elems ? min(quarter, item_elems - lo) : 0u;
-        const u32 len = out0 < geo.n ? (u32)min((u64)in_tile, geo.n - out0) : 0u;
+    for (u64 it = 0; it < my_tiles; it++, v += stride) {
+        // (ONE: the loader, which steps through the bins anyway, leaves these in the slot's header)
+        u32 live = ONE ? 0u : (u32)min((u64)TB, geo.n_bins - v * (u64)TB);      // bins of the item
+        u32 clead = ONE ? 0u : (u32)(v * (u64)TB * sizeof(Word)) & 15u;          // where the counts start in their room (see the loader)
+        u32 lo = 0;                                 // (ONE) the warp's first element, counted from the first bin's
+        const u64 out0 = v * (u64)(ONE ? (u32)kDecodeChunk : geo.tile_elems) + (u64)warp * quarter;
+        const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
         const bool whole = vec_store && len == quarter;
         if (OPT != 0 && whole && lane == 0) {
             // the warp's quarters of the optimizer's arrays travel while the words are added
@@ -2193,6 +2236,12 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             const u32 l0 = MULTI ? ws.rfirst[r] : 0u, nl = MULTI ? ws.rcount[r] : a.k;
             const u32 staged = min(reinterpret_cast<const u32 *>(sl)[0], nl);
             if (warp == 0) bad |= reinterpret_cast<const u32 *>(sl)[1];
+            if (ONE) {
+                const u32 info = reinterpret_cast<const u32 *>(sl)[2];
+                lo = (info & 0xffffu) + (u32)warp * quarter;
+                live = (info >> 16) & 0xffu;
+                clead = info >> 24;
+            }
             const unsigned short *m_cnt = reinterpret_cast<const unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
             const u32 sl_at = smem_addr(sl);
 
@@ -2207,8 +2256,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     src.limit = m_cnt[j];
                     src.sbits = __float_as_uint(s_scale[l]);
                 }
-                if (ONE && TB == 1) bad |= warp_add_group_one_bin<Word, true, false, u32>(src, R, live, lo, len, L_T, acc_at, lane);
-                else if (ONE) bad |= warp_add_group_one_bin<Word, true, true, u32>(src, R, live, lo, len, L_T, acc_at, lane);
+                if (ONE) bad |= warp_add_group_flat<Word, true, u32>(src, R, live, lo, len, L_T, acc_at, lane);
                 else if (by_bin) bad |= warp_add_group_by_bin<Word, true, u32>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
                 else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
@@ -2224,15 +2272,17 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     const u32 l = l0 + g0 + (u32)lane;
                     const unsigned char *st = a.stream[l];
                     const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
-                    const u64 w0 = dir[tile * group], w1 = dir[ONE ? min((tile + 1) * group, geo.n_tiles) : tile + 1];
-                    ok = w1 >= w0 && w1 - w0 <= item_elems && w1 <= s_nsel[l];
+                    // (ONE: the first tile, that is bin, of the item, by division on this rare path)
+                    const u64 tile = ONE ? (v * (u64)kDecodeChunk) / L_T : v, bin0 = ONE ? tile : tile * (u64)TB;
+                    const u64 w0 = dir[tile], w1 = dir[tile + (ONE ? live : 1u)];
+                    ok = w1 >= w0 && w1 - w0 <= (ONE ? live * L_T : geo.tile_elems) && w1 <= s_nsel[l];
                     src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
                     src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
                     src.limit = ok ? (u32)(w1 - w0) : 0u;
                     src.sbits = __float_as_uint(s_scale[l]);
                 }
                 if (__any_sync(full_mask, !ok)) bad |= ADACOMP_DEV_BAD_STREAM;
-                if (ONE) bad |= warp_add_group_one_bin_global<Word>(src, R, live, lo, len, L_T, acc_at, lane);
+                if (ONE) bad |= warp_add_group_flat_global<Word>(src, R, live, lo, len, L_T, acc_at, lane);
                 else if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
                 else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
@@ -2408,7 +2458,7 @@ __device__ void decode_generic(const DecodeArgs &a, const Geometry &geo, DecodeS
 // tiles of one bin (L_T > 1000).
 __host__ __device__ inline bool warp_path(const Geometry &g)
 {
-    if (g.tile_bins == 1u) return g.L_T > 1000u;
+    if (g.tile_bins == 1u) return g.L_T > 1000u && g.n < (1ull << 40);
     return g.tile_bins >= 4u && g.tile_bins <= (u32)kSmallBins && g.tile_bins % 4u == 0 && g.tile_elems <= (u32)kDecodeChunk;
 }
 

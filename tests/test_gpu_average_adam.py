@@ -27,7 +27,9 @@ def _dev(a, fill):
 
 
 @pytest.mark.parametrize("L_T,n,k", [(50, 100352, 1), (50, 4000 * 37 + 11, 4), (500, 147456, 8), (500, 4000 * 20 + 3, 3),
-                                     (50, 4000 * 6 + 1, 16), (3, 9001, 3), (64, 70000, 2), (1001, 50001, 2), (500, 12, 2)])
+                                     (50, 4000 * 6 + 1, 16), (3, 9001, 3), (64, 70000, 2), (1001, 50001, 2), (500, 12, 2),
+                                     (58, 68 * 58 * 5 + 3, 3), (300, 12 * 300 * 9 + 7, 4), (3000, 3000 * 21 + 2, 3),
+                                     (16384, 16384 * 4 + 5000, 2)])
 def test_fused_adam_matches_oracle_over_two_steps(L_T, n, k):
     rng = np.random.default_rng(2000 * L_T + n + k)
     w, m, v = _state(rng, n)

@@ -40,7 +40,11 @@ def _gpu_step(streams, n, L_T, w, v, lr, mu):
 
 @pytest.mark.parametrize("L_T,n,k", [(50, 100352, 1), (50, 4000 * 37 + 11, 4), (500, 147456, 8), (500, 4000 * 20 + 3, 3),
                                      (50, 4000 * 6 + 1, 16), (3, 9001, 3), (64, 70000, 2), (62, 31 * 3968 + 5, 3),
-                                     (100, 50007, 5), (1001, 50001, 2), (16384, 100001, 3), (500, 12, 2)])
+                                     (100, 50007, 5), (1001, 50001, 2), (16384, 100001, 3), (500, 12, 2),
+                                     # bin-count runs that are no multiple of 16 bytes; 5 and 15 bins per warp
+                                     (52, 76 * 52 * 5 + 9, 3), (63, 60 * 63 * 6 + 2, 4), (200, 20 * 200 * 7 + 3, 3),
+                                     # one bin per tile: items of 4096 elements over 1 to 6 bins
+                                     (1003, 4096 * 9 + 700, 4), (2000, 2000 * 30 + 1, 3), (5000, 5000 * 17 + 4097, 5)])
 def test_fused_update_matches_oracle(L_T, n, k):
     rng = np.random.default_rng(1000 * L_T + n + k)
     streams = _streams(rng, n, L_T, k)
