@@ -67,7 +67,7 @@ extern "C" {
 #define ADACOMP_ERR_SIZE (-5)      /* n too large (n_bins must stay below 2^31) */
 #define ADACOMP_ERR_FLAGS (-6)     /* unknown flag bits */
 #define ADACOMP_ERR_CUDA (-7)      /* a CUDA runtime call failed */
-#define ADACOMP_ERR_UNSUPPORTED (-9) /* lazy mode: L_T other than 50 / 500, or flags given */
+#define ADACOMP_ERR_UNSUPPORTED (-9) /* lazy mode: an L_T it does not take (see adacomp_compress_lazy), or flags given */
 #define ADACOMP_ERR_STATIC_SCRATCH (-8) /* adacomp_compress_static: tensor beyond the built-in scratch */
 
 /* size of the scratch array built into the library for adacomp_compress_static */
@@ -82,7 +82,7 @@ extern "C" {
 
 /* flags of adacomp_compress_ex */
 #define ADACOMP_FLAG_LITERAL 1u       /* Algorithm 2 as printed: |H| >= g_max only */
-#define ADACOMP_FLAG_GENERIC_PATH 256u /* use the any-L_T kernel even for L_T = 50 / 500 */
+#define ADACOMP_FLAG_GENERIC_PATH 256u /* use the any-L_T kernel even where a specialised one exists */
 
 /* Library ABI version (ADACOMP_VERSION).  Host only, no CUDA call. */
 int adacomp_version(void);
@@ -296,7 +296,8 @@ int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint
  *   residue  between calls it is NOT the paper's residue: run adacomp_residue_flush before
  *            reading it (checkpointing), before handing it to adacomp_compress, or before
  *            changing L_T.  After a flush it is exactly what adacomp_compress would have left.
- * Only L_T = 50 and 500 (the paper's two settings) are supported: others return
+ * Only L_T = 50, 100, 125, 200, 250, 500 and 1000 are supported (the paper's two settings, 50 and 500,
+ * among them: the bin lengths whose tiles are exactly 4000 elements): others return
  * ADACOMP_ERR_UNSUPPORTED (adacomp_lazy_state_bytes returns 0).  A state that does not belong to
  * (n, L_T) sets ADACOMP_DEV_HEADER_MISMATCH and nothing is written.
  */

@@ -293,7 +293,7 @@ __device__ inline void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 
 __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------
-// tile_pass, fast path: L_T = 25 * SPB (50 and 500), tiles of 4000 elements.
+// tile_pass, fast path: L_T = 25 * SPB for SPB = 2, 4, 5, 8, 10, 20, 40 (L_T = 50 ... 1000), tiles of 4000 elements.
 //
 // Thread t < 160 owns the 25 consecutive elements of segment t (stride 25 words in
 // shared memory: odd, so a warp's accesses are bank-conflict free); a bin is SPB
@@ -2686,6 +2686,29 @@ lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T)
 // host side
 // ---------------------------------------------------------------------------------
 
+// The fast tile pass takes L_T = 25 * SPB for the divisors SPB of 40 but 1 (tiles of exactly 4000 elements):
+// 50, 100, 125, 200, 250, 500 and 1000.
+__host__ __device__ inline bool fast_L_T(u32 L_T)
+{
+    return L_T == 50u || L_T == 100u || L_T == 125u || L_T == 200u || L_T == 250u || L_T == 500u || L_T == 1000u;
+}
+// Calls f(kernel) for the fast tile pass of L_T (LAZY, BF16 as given); false when there is none.
+template <bool LAZY, bool BF16, typename F>
+bool with_fast_kernel(u32 L_T, F f)
+{
+    switch (L_T) {
+    case 50u: f(tile_pass_fast<2, unsigned char, LAZY, BF16>); return true;
+    case 100u: f(tile_pass_fast<4, unsigned short, LAZY, BF16>); return true;
+    case 125u: f(tile_pass_fast<5, unsigned short, LAZY, BF16>); return true;
+    case 200u: f(tile_pass_fast<8, unsigned short, LAZY, BF16>); return true;
+    case 250u: f(tile_pass_fast<10, unsigned short, LAZY, BF16>); return true;
+    case 500u: f(tile_pass_fast<20, unsigned short, LAZY, BF16>); return true;
+    case 1000u: f(tile_pass_fast<40, unsigned short, LAZY, BF16>); return true;
+    default: return false;
+    }
+}
+constexpr u32 kFastL_T[] = {50u, 100u, 125u, 200u, 250u, 500u, 1000u};
+
 struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
@@ -2727,12 +2750,14 @@ int device_info(DeviceInfo *&out)
         d.decode_opt_per_sm[1][1] = opt_ready(decode_sum_warps<2, 8>, 9 * 32, opt_smem_bytes(2));
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
-        d.fast_ready = cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, true>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, true>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<2, unsigned char, false, true>, at, bytes) == cudaSuccess &&
-                       cudaFuncSetAttribute(tile_pass_fast<20, unsigned short, false, true>, at, bytes) == cudaSuccess;
+        bool ready = true;
+        auto allow = [&](auto kernel) { ready = ready && cudaFuncSetAttribute(kernel, at, bytes) == cudaSuccess; };
+        for (u32 L_T : kFastL_T) {
+            with_fast_kernel<false, false>(L_T, allow);
+            with_fast_kernel<true, false>(L_T, allow);
+            with_fast_kernel<false, true>(L_T, allow);
+        }
+        d.fast_ready = ready;
         if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kBatchSmemBytes) == cudaSuccess &&
             cudaFuncSetAttribute(batch_tile_pass<kBatchSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -2789,7 +2814,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
     if (lazy) {
-        if ((L_T != 50u && L_T != 500u) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
+        if (!fast_L_T(L_T) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
         if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
     }
 
@@ -2809,21 +2834,14 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     mark(0);
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_bf16 ? 1u : 0u};
-        const bool fast = (L_T == 50u || L_T == 500u) && flags == 0 && info->fast_ready;
+        const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
         if (fast) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            const size_t sm = FastSmem::kBytes;
-            if (lazy) {
-                if (L_T == 50u) tile_pass_fast<2, unsigned char, true><<<grid, kFastThreads, sm, st>>>(args);
-                else tile_pass_fast<20, unsigned short, true><<<grid, kFastThreads, sm, st>>>(args);
-            } else if (grad_bf16) {
-                if (L_T == 50u) tile_pass_fast<2, unsigned char, false, true><<<grid, kFastThreads, sm, st>>>(args);
-                else tile_pass_fast<20, unsigned short, false, true><<<grid, kFastThreads, sm, st>>>(args);
-            } else {
-                if (L_T == 50u) tile_pass_fast<2, unsigned char, false><<<grid, kFastThreads, sm, st>>>(args);
-                else tile_pass_fast<20, unsigned short, false><<<grid, kFastThreads, sm, st>>>(args);
-            }
+            auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
+            if (lazy) with_fast_kernel<true, false>(L_T, launch);
+            else if (grad_bf16) with_fast_kernel<false, true>(L_T, launch);
+            else with_fast_kernel<false, false>(L_T, launch);
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
@@ -3004,11 +3022,10 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f, 0u};
-        if ((L_T == 50u || L_T == 500u) && info->fast_ready) {
+        if (fast_L_T(L_T) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (L_T == 50u) tile_pass_fast<2, unsigned char, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
-            else tile_pass_fast<20, unsigned short, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(args);
+            with_fast_kernel<false, false>(L_T, [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); });
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
@@ -3209,14 +3226,14 @@ int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint
 
 size_t adacomp_lazy_state_bytes(uint64_t n, uint32_t L_T)
 {
-    if (L_T != 50u && L_T != 500u) return 0;
+    if (!fast_L_T(L_T)) return 0;
     return (size_t)lazy_state_bytes(make_geometry(n, L_T));
 }
 
 int adacomp_lazy_state_init(void *state, uint64_t n, uint32_t L_T, void *stream)
 {
     if (!state) return ADACOMP_ERR_NULL;
-    if (L_T != 50u && L_T != 500u) return ADACOMP_ERR_UNSUPPORTED;
+    if (!fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
     if (misaligned(state)) return ADACOMP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(state, 0, lazy_state_bytes(make_geometry(n, L_T)), st) != cudaSuccess) return ADACOMP_ERR_CUDA;
@@ -3234,7 +3251,7 @@ int adacomp_compress_lazy(const float *grad, float *residue, void *state, uint64
 int adacomp_residue_flush(float *residue, void *state, uint64_t n, uint32_t L_T, void *stream)
 {
     if (!state || (n && !residue)) return ADACOMP_ERR_NULL;
-    if (L_T != 50u && L_T != 500u) return ADACOMP_ERR_UNSUPPORTED;
+    if (!fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
     if (misaligned(residue) || misaligned(state)) return ADACOMP_ERR_ALIGN;
     DeviceInfo *info = nullptr;
     int rc = device_info(info);

@@ -28,7 +28,9 @@ def _compress(layer, bits):
 
 
 @pytest.mark.parametrize("L_T,n", [(50, 100352), (50, 4000 * 33), (50, 4000 * 3 + 1999), (500, 147456 + 3), (500, 4000 * 21),
-                                   (7, 1000), (64, 70000), (65, 70001), (1001, 50001), (500, 5), (50, 0)])
+                                   (7, 1000), (64, 70000), (65, 70001), (1001, 50001), (500, 5), (50, 0),
+                                   (100, 4000 * 17 + 50), (125, 4000 * 8 + 124), (200, 4000 * 11), (250, 4000 * 6 + 1),
+                                   (1000, 4000 * 9 + 999)])
 def test_bf16_gradient_matches_oracle_over_three_steps(L_T, n):
     rng = np.random.default_rng(7000 + L_T + n)
     r_cpu = rng.normal(0, 2e-3, n).astype(np.float32)

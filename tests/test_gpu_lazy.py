@@ -41,7 +41,8 @@ class LazyLayer:
 
 @pytest.mark.parametrize("L_T,n,heavy", [(50, 100352, False), (500, 147456, True), (50, 4000 * 37 + 1234, True),
                                          (500, 4000 * 300 - 7, False), (50, 3999, False), (500, 17, False),
-                                         (50, 4000 * 296, False)])
+                                         (50, 4000 * 296, False), (100, 4000 * 31 + 99, True), (125, 4000 * 12 + 1, False),
+                                         (200, 4000 * 40, False), (250, 4000 * 9 + 3999, True), (1000, 4000 * 25 + 500, False)])
 def test_lazy_steps_match_oracle_and_flush_restores_the_residue(L_T, n, heavy):
     rng = np.random.default_rng(n + L_T)
     res0 = rng.normal(0, 2e-3, n).astype(np.float32)

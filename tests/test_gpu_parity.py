@@ -62,7 +62,7 @@ def test_bin_lengths_and_ragged_tails(L_T):
         run_steps(n, L_T, dws)
 
 
-@pytest.mark.parametrize("L_T", [50, 500])
+@pytest.mark.parametrize("L_T", [50, 100, 125, 200, 250, 500, 1000])
 @pytest.mark.parametrize("n", [4000, 8000, 7999, 8001, 4000 * 150 + 1, 4000 * 1500 - 3])
 def test_fast_path_tile_boundaries(L_T, n):
     rng = np.random.default_rng(n + L_T)

@@ -21,7 +21,7 @@ def _compress_scaled(layer, dW, factor):
 
 @pytest.mark.parametrize("factor", [1.0, 1.5, 2.0, 3.0])
 @pytest.mark.parametrize("L_T,n", [(50, 100352), (500, 147456 + 3), (50, 4000 * 30), (7, 1000), (64, 70000),
-                                   (1001, 50001), (500, 77)])
+                                   (1001, 50001), (500, 77), (100, 4000 * 9 + 7), (250, 4000 * 5 + 249), (1000, 4000 * 7 + 1)])
 def test_scaled_selection_matches_oracle_over_three_steps(L_T, n, factor):
     rng = np.random.default_rng(int(1000 * factor) + L_T + n)
     r_cpu = rng.normal(0, 2e-3, n).astype(np.float32)
