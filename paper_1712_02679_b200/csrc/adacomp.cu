@@ -293,11 +293,14 @@ __device__ inline void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 
 __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------
-// tile_pass, fast path: L_T = 25 * SPB for SPB = 2, 4, 5, 8, 10, 20, 40 (L_T = 50 ... 1000), tiles of 4000 elements.
+// tile_pass, fast path: L_T = 25 * SPB for SPB = 2, 4, 5, 8, 10, 20, 40 (L_T = 50 ... 1000), tiles of 4000 elements;
+// and, as SPB = 0, every other L_T from 41 to 1000 (tiles of 3200 to 4000 elements, bins anywhere).
 //
 // Thread t < 160 owns the 25 consecutive elements of segment t (stride 25 words in
 // shared memory: odd, so a warp's accesses are bank-conflict free); a bin is SPB
-// adjacent segments.  Warp 5 (the service warp) owns no segment: its lane 0 issues
+// adjacent segments.  SPB = 0: a bin is L_T consecutive elements wherever the segments' edges
+// are; L_T > 25, so a segment lies in one bin or straddles one edge between two, and the
+// threads meet in shared-memory atomics on per-bin maxima and counts.  Warp 5 (the service warp) owns no segment: its lane 0 issues
 // every bulk copy, and the warp feeds the exact g_max accumulator and copies the
 // tile's words to the scratch slot.
 //
@@ -340,7 +343,7 @@ struct FastSmem {
     static constexpr u32 kWtotAt = kInclAt + 4 * kTileSegs;
     static constexpr u32 kSegmaxAt = kWtotAt + 4 * 8;
     static constexpr u32 kBinmaxAt = kSegmaxAt + 4 * kTileSegs;
-    static constexpr u32 kAccAt = kBinmaxAt + 4 * 80;                 // 8-byte aligned
+    static constexpr u32 kAccAt = kBinmaxAt + 4 * 4 * kSmallBins;     // (SPB = 0: two buffers each of bin maxima and counts) 8-byte aligned
     static constexpr u32 kBarAt = kAccAt + 8 * (kWindows + 1);
     static constexpr u32 kAbortAt = kBarAt + 8 * kStages;
     static constexpr u32 kBytes = kAbortAt + 16;
@@ -365,7 +368,24 @@ tile_pass_fast(PassArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == 5;
     const Geometry &geo = a.geo;
-    constexpr int kBins = kTileSegs / SPB;
+    constexpr bool ANY = SPB == 0;
+    static_assert(!ANY || (!LAZY && !BF16), "the any-L_T form takes fp32 gradients, eagerly");
+    constexpr int kBins = ANY ? kSmallBins : kTileSegs / (ANY ? 1 : SPB);
+    const int T = ANY ? (int)geo.tile_elems : kFastTile;            // elements of a tile (a multiple of 4)
+    const int TB = ANY ? (int)geo.tile_bins : kBins;
+    const u32 tile_bytes = (u32)T * 4u;
+    // ANY: the thread's elements [0, cut) lie in bin b0 of the tile, from place off0 of it on, the
+    // others in bin b0 + 1; only the first `vcount` of them exist (tiles of less than 4000 elements)
+    int b0 = 0, cut = kSeg, off0 = 0, vcount = kSeg;
+    if (ANY) {
+        const int L = (int)geo.L_T, e0 = tid * kSeg;
+        b0 = e0 / L;
+        off0 = e0 - b0 * L;
+        cut = min(kSeg, L - off0);
+        vcount = max(0, min(kSeg, T - e0));
+    }
+    u32 *s_anymax = reinterpret_cast<u32 *>(s_binmax);              // ANY: [2][kSmallBins] bits of the bin maxima, by tile parity
+    u32 *s_anycnt = s_anymax + 2 * kSmallBins;                      // ANY: [2][kSmallBins] words per bin
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
     u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
     u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
@@ -373,7 +393,7 @@ tile_pass_fast(PassArgs a)
     // tiles of this CTA: blockIdx.x + i * gridDim.x
     const u64 first = blockIdx.x, stride = gridDim.x;
     const u64 my_tiles = geo.n_tiles > first ? (geo.n_tiles - first + stride - 1) / stride : 0;
-    const u64 full_tiles = geo.n / kFastTile;       // tiles below this index are complete
+    const u64 full_tiles = geo.n / (u64)T;          // tiles below this index are complete
 
     // Lazy mode: the residue buffer holds last step's G; the elements sent then still owe
     // "- sign(G) * scale" (Algorithm 2's G - Gq), applied here as they are loaded.
@@ -397,6 +417,8 @@ tile_pass_fast(PassArgs a)
     }
 
     if (tid < kWindows + 1) s_acc[tid] = 0;
+    if (ANY)
+        for (int b = tid; b < 4 * kSmallBins; b += kFastThreads) s_anymax[b] = 0;
     if (tid == 0) {
         *s_abort = 0;
         for (int s = 0; s < kStages; s++) mbar_init(&s_full[s], 1);
@@ -410,10 +432,10 @@ tile_pass_fast(PassArgs a)
         if (i >= my_tiles || tile >= full_tiles) return;
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        constexpr u32 kGradBytes = BF16 ? kTileBytes / 2 : kTileBytes;
-        mbar_arrive_expect_tx(bar, kGradBytes + kTileBytes + (LAZY ? kMaskBytes : 0u));
-        bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)kGradBytes, kGradBytes, bar);
-        bulk_load(st + kTileBytes, a.residue + tile * (u64)kFastTile, kTileBytes, bar);
+        const u32 grad_bytes = BF16 ? kTileBytes / 2 : tile_bytes;
+        mbar_arrive_expect_tx(bar, grad_bytes + tile_bytes + (LAZY ? kMaskBytes : 0u));
+        bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)grad_bytes, grad_bytes, bar);
+        bulk_load(st + kTileBytes, a.residue + tile * (u64)T, tile_bytes, bar);
         if (LAZY) bulk_load(st + 2 * kTileBytes, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
         issued = i + 1;
     };
@@ -425,12 +447,13 @@ tile_pass_fast(PassArgs a)
     u64 i = 0;
     for (; i < my_tiles; i++) {
         const u64 tile = first + i * stride;
-        const u64 base = tile * (u64)kFastTile;
+        const u64 base = tile * (u64)T;
         float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
         float *s_r = s_d + kFastTile;
         const u32 *s_prev = reinterpret_cast<const u32 *>(s_r + kFastTile);
         const bool whole = tile < full_tiles;
-        const int elems = whole ? kFastTile : (int)(geo.n - base);
+        const int elems = whole ? T : (int)(geo.n - base);
+        u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
 
         if (whole) {
             if (!mbar_wait(&s_full[i % kStages], (u32)(i / kStages) & 1u)) {
@@ -453,12 +476,12 @@ tile_pass_fast(PassArgs a)
 
         // ---- G = residue + dW, H = G + dW; the segment's maximum |G| ----
         float g[kSeg], key[kSeg];
-        float gm = 0.f;
+        float gm = 0.f, gm1 = 0.f;      // the bin maximum (ANY: of the segment's first and second bin)
         u32 selmask = 0, cnt = 0, incl = 0;
         if (!service) {
             const float *pd = s_d + tid * kSeg;
             const float *pr = s_r + tid * kSeg;
-            float m = 0.f;
+            float m = 0.f, m1 = 0.f;
             const u32 prev = LAZY ? s_prev[tid] : 0u;
             // bfloat16: the segment's 50 bytes start on a 4-byte boundary for even threads and two bytes
             // past one for odd threads; thirteen aligned 32-bit loads cover them either way, and a funnel
@@ -476,8 +499,9 @@ tile_pass_fast(PassArgs a)
             }
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
-                const float d = BF16 ? __uint_as_float((j & 1) ? pair[j >> 1] & 0xffff0000u : pair[j >> 1] << 16) : pd[j];
+                float d = BF16 ? __uint_as_float((j & 1) ? pair[j >> 1] & 0xffff0000u : pair[j >> 1] << 16) : pd[j];
                 float r = pr[j];
+                if (ANY && j >= vcount) d = r = 0.f;        // past the tile's end
                 if (LAZY) {
                     // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
                     const float q = __uint_as_float(prev_scale_bits | (__float_as_uint(r) & 0x80000000u));
@@ -486,12 +510,17 @@ tile_pass_fast(PassArgs a)
                 }
                 g[j] = __fadd_rn(r, d);
                 const float h = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g[j], d);
-                m = fmaxf(m, fabsf(g[j]));
+                if (ANY && j >= cut) m1 = fmaxf(m1, fabsf(g[j]));
+                else m = fmaxf(m, fabsf(g[j]));
                 // |G| never exceeds the bin maximum, so "|H| >= g_max or |G| == g_max"
                 // is "max(|H|, |G|) >= g_max"
                 key[j] = fmaxf(fabsf(h), fabsf(g[j]));
             }
-            if (SPB == 2) {
+            if (ANY) {
+                // (non-negative floats order like their bits)
+                if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
+                if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
+            } else if (SPB == 2) {
                 gm = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
             } else {
                 s_segmax[tid] = m;
@@ -499,19 +528,34 @@ tile_pass_fast(PassArgs a)
         }
         if (SPB != 2) {
             __syncthreads();                                        // barrier A
-            if (!service) {
-                const int bin = tid / SPB;
+            if (ANY) {
+                // the other parity's buffers are free: tile i - 1 is done with them, tile i + 1 starts after barrier D
+                if (tid < kSmallBins) {
+                    s_anymax[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+                    s_anycnt[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+                }
+                if (!service) {
+                    gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
+                    gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
+                }
+            } else if (!service) {
+                const int bin = tid / (ANY ? 1 : SPB);
 #pragma unroll
                 for (int s = 0; s < SPB; s++) gm = fmaxf(gm, s_segmax[bin * SPB + s]);
             }
         }
         if (!service) {
-            if (tid % SPB == 0) s_binmax[tid / SPB] = gm;
+            if (!ANY && tid % (ANY ? 1 : SPB) == 0) s_binmax[tid / (ANY ? 1 : SPB)] = gm;
             // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
 #pragma unroll
             for (int j = 0; j < kSeg; j++)
-                if (key[j] >= gm && g[j] != 0.f) selmask |= 1u << j;
+                if (key[j] >= (ANY && j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
             cnt = __popc(selmask);
+            if (ANY) {
+                const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
+                if (c0) atomicAdd(&any_cnt[b0], c0);
+                if (cnt - c0) atomicAdd(&any_cnt[b0 + 1], cnt - c0);
+            }
             incl = warp_inclusive_scan(cnt, lane);
             s_incl[tid] = incl;
             if (lane == 31) s_wtot[warp] = incl;
@@ -530,17 +574,23 @@ tile_pass_fast(PassArgs a)
 #pragma unroll
             for (int j = 0; j < kSeg; j++) pr[j] = g[j];
             u32 at = mine - cnt;
-            const u32 seg_in_bin = (u32)(tid % SPB) * kSeg;
+            const u32 seg_in_bin = ANY ? (u32)off0 : (u32)(tid % (ANY ? 1 : SPB)) * kSeg;
             u32 mask = selmask;
             while (mask) {
                 const int j = __ffs(mask) - 1;
                 mask &= mask - 1;
                 const u32 neg = __float_as_uint(pr[j]) >> 31;
-                s_words[at++] = (Word)(((seg_in_bin + j) << 2) | 1u | (neg << 1));
+                const u32 idx = ANY && j >= cut ? (u32)(j - cut) : seg_in_bin + j;      // the element's place in its bin
+                s_words[at++] = (Word)((idx << 2) | 1u | (neg << 1));
             }
             if (LAZY) lazy_mask[tile * (u64)kTileSegs + tid] = selmask;
-            if (tid % SPB == 0) {
-                const u64 bin = tile * (u64)kBins + tid / SPB;
+            if (ANY) {
+                if (tid < TB) {
+                    const u64 bin = tile * (u64)TB + tid;
+                    if (bin < geo.n_bins) bin_cnt[bin] = (Word)any_cnt[tid];
+                }
+            } else if (tid % (ANY ? 1 : SPB) == 0) {
+                const u64 bin = tile * (u64)kBins + tid / (ANY ? 1 : SPB);
                 const int t1 = tid + SPB - 1;
                 const u32 last = wpre[t1 >> 5] + s_incl[t1];
                 if (bin < geo.n_bins) bin_cnt[bin] = (Word)(last - mine + cnt);
@@ -548,10 +598,10 @@ tile_pass_fast(PassArgs a)
             fence_async_smem();          // the bulk store below reads what was just written
         } else {
             total = s_wtot[0] + s_wtot[1] + s_wtot[2] + s_wtot[3] + s_wtot[4];
-            for (int b0 = 0; b0 < kBins; b0 += 32) {    // every lane takes part each round
-                const int b = b0 + lane;
-                const bool valid = b < kBins && tile * (u64)kBins + b < geo.n_bins;
-                warp_accumulate(s_acc, valid ? s_binmax[b] : 0.f, valid);
+            for (int bb = 0; bb < TB; bb += 32) {       // every lane takes part each round
+                const int b = bb + lane;
+                const bool valid = b < TB && tile * (u64)TB + b < geo.n_bins;
+                warp_accumulate(s_acc, valid ? (ANY ? __uint_as_float(any_max[b]) : s_binmax[b]) : 0.f, valid);
             }
             if (lane == 0) {
                 bulk_wait_read_all();    // the store of tile i - 1 has drained its stage
@@ -564,7 +614,7 @@ tile_pass_fast(PassArgs a)
         if (service && !aborted) {
             if (whole) {
                 if (lane == 0) {
-                    bulk_store(a.residue + base, s_r, kTileBytes);
+                    bulk_store(a.residue + base, s_r, tile_bytes);
                     bulk_commit();
                 }
             } else {
@@ -2708,6 +2758,15 @@ bool with_fast_kernel(u32 L_T, F f)
     }
 }
 constexpr u32 kFastL_T[] = {50u, 100u, 125u, 200u, 250u, 500u, 1000u};
+// Every other L_T from 41 to 1000 (tiles of at most 96 bins, bins longer than a thread's 25 elements) takes
+// the same kernel in its any-bin form (fp32 gradient, eager).
+__host__ __device__ inline bool any_fast_L_T(u32 L_T) { return L_T >= 41u && L_T <= 1000u && !fast_L_T(L_T); }
+template <typename F>
+void with_any_fast_kernel(u32 L_T, F f)
+{
+    if (L_T <= 64u) f(tile_pass_fast<0, unsigned char, false, false>);
+    else f(tile_pass_fast<0, unsigned short, false, false>);
+}
 
 struct DeviceInfo {
     int sms = 0;
@@ -2757,6 +2816,8 @@ int device_info(DeviceInfo *&out)
             with_fast_kernel<true, false>(L_T, allow);
             with_fast_kernel<false, true>(L_T, allow);
         }
+        with_any_fast_kernel(41u, allow);
+        with_any_fast_kernel(65u, allow);
         d.fast_ready = ready;
         if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kBatchSmemBytes) == cudaSuccess &&
@@ -2835,11 +2896,13 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_bf16 ? 1u : 0u};
         const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
-        if (fast) {
+        const bool any_fast = any_fast_L_T(L_T) && flags == 0 && !grad_bf16 && info->fast_ready;
+        if (fast || any_fast) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
             auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
-            if (lazy) with_fast_kernel<true, false>(L_T, launch);
+            if (any_fast) with_any_fast_kernel(L_T, launch);
+            else if (lazy) with_fast_kernel<true, false>(L_T, launch);
             else if (grad_bf16) with_fast_kernel<false, true>(L_T, launch);
             else with_fast_kernel<false, false>(L_T, launch);
         } else {
@@ -3022,10 +3085,12 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f, 0u};
-        if (fast_L_T(L_T) && info->fast_ready) {
+        if ((fast_L_T(L_T) || any_fast_L_T(L_T)) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            with_fast_kernel<false, false>(L_T, [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); });
+            auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
+            if (fast_L_T(L_T)) with_fast_kernel<false, false>(L_T, launch);
+            else with_any_fast_kernel(L_T, launch);
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
