@@ -651,8 +651,8 @@ tile_pass_fast(PassArgs a)
 
 // ---------------------------------------------------------------------------------
 // tile_pass, any L_T: a warp per bin, lanes strided over the bin's elements.
-// Dynamic shared memory: dW[tile_elems], G[tile_elems], words[tile_elems],
-// gmax[tile_bins], cnt[tile_bins + 1].
+// Dynamic shared memory: H[tile_elems], G[tile_elems], words[tile_elems],
+// gmax[units], cnt[units + 1], units = max(tile_bins, 8).
 // ---------------------------------------------------------------------------------
 
 // One tile of one layer.  Called by all 256 threads of the CTA; `s_acc` collects the CTA's share of
@@ -671,12 +671,18 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
                              u64 *s_acc)
 {
     const int T = (int)geo.tile_elems, TB = (int)geo.tile_bins, L = (int)geo.L_T;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
+    // A unit is a warp's work: a bin or, in tiles of fewer bins than the CTA has warps, one of P equal
+    // parts of a bin (whole 32-element steps each, so that the parts' words stay in ascending order).
+    // (tiles have 1 bin or a multiple of 4: P is 8, 2 or 1)
+    const int P = TB >= nwarp ? 1 : TB >= 4 ? 2 : 8, pshift = P == 8 ? 3 : P == 2 ? 1 : 0;
+    const int part = P == 1 ? L : (((L + P - 1) / P + 31) & ~31);
+    const int units = TB * P;
     float *s_d = reinterpret_cast<float *>(smem_raw);
     float *s_g = s_d + T;
     Word *s_words = reinterpret_cast<Word *>(s_g + T);
-    float *s_gmax = reinterpret_cast<float *>(smem_raw + align_up((u64)T * (8 + sizeof(Word)), 16));
-    u32 *s_cnt = reinterpret_cast<u32 *>(s_gmax + TB);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGenericThreads / 32;
+    float *s_gmax = reinterpret_cast<float *>(smem_raw + align_up((u64)T * (8 + sizeof(Word)), 16));    // [units]
+    u32 *s_cnt = reinterpret_cast<u32 *>(s_gmax + units);                                                  // [units + 1]
     Word *bin_cnt = reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at);
     u32 *tile_cnt = reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at);
     u64 *group_cnt = reinterpret_cast<u64 *>(a.scratch + geo.group_at);
@@ -685,7 +691,23 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     const u64 left = geo.n - base;
     const int elems = left < (u64)T ? (int)left : T;
 
-    for (int i = tid; i < T; i += kGenericThreads) {
+    // G and H of the tile: four elements a thread and step where 4 divides the tile's length (every tile, and
+    // the G array behind the H array in shared memory, then start on a 16-byte boundary)
+    const int quads = (T & 3) == 0 && !a.grad_bf16 ? elems >> 2 : 0;
+    for (int i = tid; i < quads; i += kGenericThreads) {
+        const float4 d = reinterpret_cast<const float4 *>(a.grad + base)[i];
+        const float4 r = reinterpret_cast<const float4 *>(a.residue + base)[i];
+        const float dv[4] = {d.x, d.y, d.z, d.w}, rv[4] = {r.x, r.y, r.z, r.w};
+        float gv[4], hv[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            gv[q] = __fadd_rn(rv[q], dv[q]);
+            hv[q] = a.factor != 0.f ? __fadd_rn(rv[q], __fmul_rn(a.factor, dv[q])) : __fadd_rn(gv[q], dv[q]);
+        }
+        reinterpret_cast<float4 *>(s_g)[i] = make_float4(gv[0], gv[1], gv[2], gv[3]);
+        reinterpret_cast<float4 *>(s_d)[i] = make_float4(hv[0], hv[1], hv[2], hv[3]);
+    }
+    for (int i = 4 * quads + tid; i < T; i += kGenericThreads) {
         float d = 0.f, r = 0.f;
         if (i < elems) { d = load_grad(a.grad, base + i, a.grad_bf16); r = a.residue[base + i]; }
         const float g = __fadd_rn(r, d);
@@ -694,17 +716,15 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     }
     __syncthreads();
 
-    // bin maxima and per-bin counts
-    for (int b = warp; b < TB; b += nwarp) {
-        float m = 0.f;
-        for (int j = lane; j < L; j += 32) m = fmaxf(m, fabsf(s_g[b * L + j]));
-        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    // words of unit u, whose bin's maximum is m; the bin's maximum joins the exact sum once
+    auto count_unit = [&](int u, float m) {
+        const int b = u >> pshift, j_lo = (u & (P - 1)) * part, j_hi = min(L, j_lo + part);
         u32 count = 0;
         if (m > 0.f) {
-            for (int j0 = 0; j0 < L; j0 += 32) {
+            for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
                 const int j = j0 + lane;
                 bool sel = false;
-                if (j < L) {
+                if (j < j_hi) {
                     const float g = s_g[b * L + j];
                     const float h = s_d[b * L + j];
                     sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
@@ -713,11 +733,8 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
             }
         }
         if (lane == 0) {
-            s_gmax[b] = m;
-            s_cnt[b] = count;
-            const u64 bin = tile * (u64)TB + b;
-            if (bin < geo.n_bins) {
-                bin_cnt[bin] = (Word)count;
+            s_cnt[u] = count;
+            if ((u & (P - 1)) == 0 && tile * (u64)TB + b < geo.n_bins) {
                 u32 window;
                 u64 lo, hi;
                 if (split_for_sum(m, window, lo, hi)) {
@@ -726,20 +743,43 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
                 }
             }
         }
+    };
+    // maxima of the units (a unit that is a whole bin goes on to count its words at once)
+    for (int u = warp; u < units; u += nwarp) {
+        const int b = u >> pshift, j_lo = (u & (P - 1)) * part, j_hi = min(L, j_lo + part);
+        float m = 0.f;
+        for (int j = j_lo + lane; j < j_hi; j += 32) m = fmaxf(m, fabsf(s_g[b * L + j]));
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        if (lane == 0) s_gmax[u] = m;
+        if (P == 1) count_unit(u, m);
+    }
+    if (P > 1) {
+        __syncthreads();
+        for (int u = warp; u < units; u += nwarp) {
+            float m = 0.f;
+            for (int q = 0; q < P; q++) m = fmaxf(m, s_gmax[(u & ~(P - 1)) + q]);
+            count_unit(u, m);
+        }
     }
     __syncthreads();
-    block_exclusive_scan(s_cnt, TB, s_tmp);
+    block_exclusive_scan(s_cnt, units, s_tmp);
+    for (int b = tid; b < TB; b += kGenericThreads) {
+        const u64 bin = tile * (u64)TB + b;
+        if (bin < geo.n_bins) bin_cnt[bin] = (Word)(s_cnt[(b + 1) << pshift] - s_cnt[b << pshift]);
+    }
 
     // words, in ascending order inside each bin
-    for (int b = warp; b < TB; b += nwarp) {
-        const float m = s_gmax[b];
+    for (int u = warp; u < units; u += nwarp) {
+        const int b = u >> pshift, j_lo = (u & (P - 1)) * part, j_hi = min(L, j_lo + part);
+        float m = 0.f;
+        for (int q = 0; q < P; q++) m = fmaxf(m, s_gmax[(u & ~(P - 1)) + q]);
         if (!(m > 0.f)) continue;
-        u32 at = s_cnt[b];
-        for (int j0 = 0; j0 < L; j0 += 32) {
+        u32 at = s_cnt[u];
+        for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
             const int j = j0 + lane;
             bool sel = false;
             float g = 0.f;
-            if (j < L) {
+            if (j < j_hi) {
                 g = s_g[b * L + j];
                 const float h = s_d[b * L + j];
                 sel = (g != 0.f) && (fabsf(h) >= m || (!a.literal && fabsf(g) == m));
@@ -754,8 +794,14 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     }
     __syncthreads();
 
-    for (int i = tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
-    const u32 total = s_cnt[TB];
+    if (quads) {
+        for (int i = tid; i < quads; i += kGenericThreads)
+            reinterpret_cast<float4 *>(a.residue + base)[i] = reinterpret_cast<const float4 *>(s_g)[i];
+        for (int i = 4 * quads + tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
+    } else {
+        for (int i = tid; i < elems; i += kGenericThreads) a.residue[base + i] = s_g[i];
+    }
+    const u32 total = s_cnt[units];
     Word *slot = reinterpret_cast<Word *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
     for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
     if (tid == 0) {
@@ -2846,8 +2892,8 @@ template <typename Word>
 int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st)
 {
     const Geometry &geo = args.geo;
-    const size_t smem = (size_t)align_up((u64)geo.tile_elems * (8 + sizeof(Word)), 16) +
-                        (size_t)geo.tile_bins * 4 + ((size_t)geo.tile_bins + 1) * 4;
+    const size_t units = geo.tile_bins < 8u ? 8u : geo.tile_bins;      // generic_tile: a bin or a part of one per warp
+    const size_t smem = (size_t)align_up((u64)geo.tile_elems * (8 + sizeof(Word)), 16) + units * 4 + (units + 1) * 4;
     if (smem > (size_t)info.smem_optin) return ADACOMP_ERR_SIZE;
     if (cudaFuncSetAttribute(tile_pass_generic<Word>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
