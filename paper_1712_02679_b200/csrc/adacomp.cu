@@ -1956,23 +1956,22 @@ __device__ inline u32 warp_add_group_flat(const GroupSrc<Addr> &src, int R, u32 
     return bad;
 }
 
-// The same for learners read from global memory: rare, so kept out of line (the decoding warps'
-// registers go to the path that reads the slots).
+// The same for learners read from global memory (rare).
 template <typename Word>
-__device__ __noinline__ u32 warp_add_group_by_bin_global(GroupSrc<u64> src, int R, int TB, u32 live, u32 L_T, int bin, int r,
+__device__ u32 warp_add_group_by_bin_global(GroupSrc<u64> src, int R, int TB, u32 live, u32 L_T, int bin, int r,
                                                          int G, u32 mine_at, int lane)
 {
     return warp_add_group_by_bin<Word, false, u64>(src, R, TB, live, L_T, bin, r, G, mine_at, lane);
 }
 template <typename Word>
-__device__ __noinline__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int b0, int nb, u32 live, u32 L_T, u32 acc_at,
+__device__ u32 warp_add_group_global(GroupSrc<u64> src, int R, int b0, int nb, u32 live, u32 L_T, u32 acc_at,
                                                   u32 *tmp, int lane)
 {
     return warp_add_group<Word, false, u64>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
 }
 
 template <typename Word>
-__device__ __noinline__ u32 warp_add_group_flat_global(GroupSrc<u64> src, int R, u32 live, u32 lo, u32 len, u32 L_T,
+__device__ u32 warp_add_group_flat_global(GroupSrc<u64> src, int R, u32 live, u32 lo, u32 len, u32 L_T,
                                                        u32 acc_at, int lane)
 {
     return warp_add_group_flat<Word, false, u64>(src, R, live, lo, len, L_T, acc_at, lane);
@@ -2593,18 +2592,22 @@ __device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_
     return true;
 }
 
-// The decoder is two kernels, so that each gets the registers its path needs: decode_sum_warps
-// takes the shapes of warp_path() and returns at once for any other, decode_sum the reverse.  A
-// caller that knows the shape launches the one that works; one that does not launches both.
+// The decoder is three kernels, so that each gets the registers its path needs: decode_sum_warps
+// takes the shapes of warp_path() (its ONE form the tiles of one bin, its other form the rest) and
+// returns at once for any other, decode_sum the reverse.  A caller that knows the shape launches
+// the one that works; one that does not launches all three.
 // dynamic shared memory of decode_sum_warps<OPT>: a tile per array of the optimizer
 constexpr u32 opt_smem_bytes(int opt) { return opt == 0 ? 0u : (opt == 2 ? 3u : 2u) * kDecodeChunk * 4u; }
 
 // NW decoding warps and the loader warp: 4 for plain decoding; with an optimizer step, whose staged tiles
 // leave room for fewer CTAs per SM, 8 where they divide the tile's bins (more warps to hide the adds' latency).
-template <int OPT, int NW>
+// ONE: the kernel of the tiles of one bin (L_T > 1000): a kernel of its own, so that its registers are
+// allotted apart from the other shapes'.
+template <int OPT, int NW, bool ONE = false>
 __global__ void __launch_bounds__((NW + 1) * 32, OPT == 0 ? kWarpsPerSm : OPT == 1 ? 3 : 2)
 decode_sum_warps(DecodeArgs a)
 {
+    static_assert(!ONE || NW == 4, "tiles of one bin are split between four warps");
     __shared__ __align__(16) float s_acc[kDecodeChunk];
     __shared__ __align__(16) WarpDecSmem<NW> ws;
     __shared__ u64 s_nsel[ADACOMP_MAX_STREAMS];
@@ -2615,16 +2618,15 @@ decode_sum_warps(DecodeArgs a)
     if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
     // (the launcher picks NW from the shape it was given: a divisor of the tile's bins; 4 for tiles of one bin)
-    if (!warp_path(geo) || (geo.tile_bins == 1u ? NW != 4 : geo.tile_bins % (u32)NW != 0)) return;
+    if (!warp_path(geo) || ONE != (geo.tile_bins == 1u) || (!ONE && geo.tile_bins % (u32)NW != 0)) return;
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
     extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles
     float *const s_wv = OPT ? s_dyn : nullptr;
-    if (geo.w == 1u) {
-        decode_warps_any<unsigned char, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-    } else if (geo.tile_bins == 1u) {
-        if constexpr (NW == 4) decode_warps_any<unsigned short, OPT, NW, true>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    if constexpr (ONE) {
+        decode_warps_any<unsigned short, OPT, NW, true>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
     } else {
-        decode_warps_any<unsigned short, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+        if (geo.w == 1u) decode_warps_any<unsigned char, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+        else decode_warps_any<unsigned short, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
     }
 }
 
@@ -2853,6 +2855,9 @@ int device_info(DeviceInfo *&out)
         d.decode_opt_per_sm[0][1] = opt_ready(decode_sum_warps<1, 8>, 9 * 32, opt_smem_bytes(1));
         d.decode_opt_per_sm[1][0] = opt_ready(decode_sum_warps<2, 4>, 5 * 32, opt_smem_bytes(2));
         d.decode_opt_per_sm[1][1] = opt_ready(decode_sum_warps<2, 8>, 9 * 32, opt_smem_bytes(2));
+        // (the kernels of the one-bin tiles: same shared memory and launch bounds as their four-warp siblings)
+        if (!opt_ready(decode_sum_warps<1, 4, true>, 5 * 32, opt_smem_bytes(1))) d.decode_opt_per_sm[0][0] = 0;
+        if (!opt_ready(decode_sum_warps<2, 4, true>, 5 * 32, opt_smem_bytes(2))) d.decode_opt_per_sm[1][0] = 0;
         const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
         const int bytes = (int)FastSmem::kBytes;
         bool ready = true;
@@ -3034,12 +3039,18 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
             grid_s = items < grid_s ? (items ? items : 1) : grid_s;
         }
         const unsigned g = (unsigned)grid_s;
+        const bool one = hint_L_T > 1000u;
         if (ep->adam && eight) decode_sum_warps<2, 8><<<g, 9 * 32, opt_smem_bytes(2), st>>>(args);
+        else if (ep->adam && one) decode_sum_warps<2, 4, true><<<g, 5 * 32, opt_smem_bytes(2), st>>>(args);
         else if (ep->adam) decode_sum_warps<2, 4><<<g, 5 * 32, opt_smem_bytes(2), st>>>(args);
         else if (eight) decode_sum_warps<1, 8><<<g, 9 * 32, opt_smem_bytes(1), st>>>(args);
+        else if (one) decode_sum_warps<1, 4, true><<<g, 5 * 32, opt_smem_bytes(1), st>>>(args);
         else decode_sum_warps<1, 4><<<g, 5 * 32, opt_smem_bytes(1), st>>>(args);
+    } else if (warps) {
+        // (without the shape both go and one of them returns at once)
+        if (!hint_L_T || hint_L_T <= 1000u) decode_sum_warps<0, 4><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
+        if (!hint_L_T || hint_L_T > 1000u) decode_sum_warps<0, 4, true><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
     }
-    else if (warps) decode_sum_warps<0, 4><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
     if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, st>>>(args);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
