@@ -377,7 +377,7 @@ def run_ours(a):
 
     # ---- the same steps with lazy-scale pack(): identical streams, one pass over the residue ----
     lazy = None
-    if L_T in (50, 100, 125, 200, 250, 500, 1000) and not a.no_lazy:
+    if 41 <= L_T <= 1000 and not a.no_lazy:
         eager_counts = [tuple(int(v) for v in c.cpu()) for c in count]
         for r in residue:
             r.zero_()

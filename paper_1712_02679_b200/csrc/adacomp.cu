@@ -369,7 +369,7 @@ tile_pass_fast(PassArgs a)
     const bool service = warp == 5;
     const Geometry &geo = a.geo;
     constexpr bool ANY = SPB == 0;
-    static_assert(!ANY || (!LAZY && !BF16), "the any-L_T form takes fp32 gradients, eagerly");
+    static_assert(!ANY || !BF16, "the any-L_T form takes fp32 gradients");
     constexpr int kBins = ANY ? kSmallBins : kTileSegs / (ANY ? 1 : SPB);
     const int T = ANY ? (int)geo.tile_elems : kFastTile;            // elements of a tile (a multiple of 4)
     const int TB = ANY ? (int)geo.tile_bins : kBins;
@@ -2754,7 +2754,7 @@ __global__ void lazy_init_kernel(unsigned char *state, u64 n, u32 L_T)
 // residue_flush: finish "residue = G - sign(G) * scale" for the elements the last lazy step sent,
 // and clear their marks.  One thread per 25-element segment.
 __global__ void __launch_bounds__(256)
-lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T)
+lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T, u32 tile_elems)
 {
     const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(state);
     if (lh->magic != kLazyMagic || lh->n != n || lh->L_T != L_T) {
@@ -2763,15 +2763,17 @@ lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T)
     }
     const u32 sbits = __float_as_uint(lh->scale) & 0x7fffffffu;
     u32 *mask = reinterpret_cast<u32 *>(state + kLazyHeaderBytes);
-    const u64 segs = (n + kSeg - 1) / kSeg;
+    // segment s of tile t starts at element t * tile_elems + 25 s (tiles of 4000 elements: 25 (160 t + s))
+    const u64 segs = (n + tile_elems - 1) / tile_elems * (u64)kTileSegs;
     for (u64 sgm = (u64)blockIdx.x * blockDim.x + threadIdx.x; sgm < segs; sgm += (u64)gridDim.x * blockDim.x) {
         u32 m = mask[sgm];
         if (m == 0) continue;
         mask[sgm] = 0;
+        const u64 first = sgm / kTileSegs * tile_elems + sgm % kTileSegs * kSeg;
         while (m) {
             const int j = __ffs(m) - 1;
             m &= m - 1;
-            const u64 i = sgm * kSeg + j;
+            const u64 i = first + j;
             if (i < n) {
                 const float r = residue[i];
                 residue[i] = __fsub_rn(r, __uint_as_float(sbits | (__float_as_uint(r) & 0x80000000u)));
@@ -2809,11 +2811,11 @@ constexpr u32 kFastL_T[] = {50u, 100u, 125u, 200u, 250u, 500u, 1000u};
 // Every other L_T from 41 to 1000 (tiles of at most 96 bins, bins longer than a thread's 25 elements) takes
 // the same kernel in its any-bin form (fp32 gradient, eager).
 __host__ __device__ inline bool any_fast_L_T(u32 L_T) { return L_T >= 41u && L_T <= 1000u && !fast_L_T(L_T); }
-template <typename F>
+template <bool LAZY, typename F>
 void with_any_fast_kernel(u32 L_T, F f)
 {
-    if (L_T <= 64u) f(tile_pass_fast<0, unsigned char, false, false>);
-    else f(tile_pass_fast<0, unsigned short, false, false>);
+    if (L_T <= 64u) f(tile_pass_fast<0, unsigned char, LAZY, false>);
+    else f(tile_pass_fast<0, unsigned short, LAZY, false>);
 }
 
 struct DeviceInfo {
@@ -2867,8 +2869,10 @@ int device_info(DeviceInfo *&out)
             with_fast_kernel<true, false>(L_T, allow);
             with_fast_kernel<false, true>(L_T, allow);
         }
-        with_any_fast_kernel(41u, allow);
-        with_any_fast_kernel(65u, allow);
+        with_any_fast_kernel<false>(41u, allow);
+        with_any_fast_kernel<false>(65u, allow);
+        with_any_fast_kernel<true>(41u, allow);
+        with_any_fast_kernel<true>(65u, allow);
         d.fast_ready = ready;
         if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kBatchSmemBytes) == cudaSuccess &&
@@ -2926,7 +2930,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
     if (lazy) {
-        if (!fast_L_T(L_T) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
+        if (!(fast_L_T(L_T) || any_fast_L_T(L_T)) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
         if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
     }
 
@@ -2952,7 +2956,8 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
             auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
-            if (any_fast) with_any_fast_kernel(L_T, launch);
+            if (any_fast && lazy) with_any_fast_kernel<true>(L_T, launch);
+            else if (any_fast) with_any_fast_kernel<false>(L_T, launch);
             else if (lazy) with_fast_kernel<true, false>(L_T, launch);
             else if (grad_bf16) with_fast_kernel<false, true>(L_T, launch);
             else with_fast_kernel<false, false>(L_T, launch);
@@ -3147,7 +3152,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
             auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
             if (fast_L_T(L_T)) with_fast_kernel<false, false>(L_T, launch);
-            else with_any_fast_kernel(L_T, launch);
+            else with_any_fast_kernel<false>(L_T, launch);
         } else {
             rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
                              : launch_generic<unsigned short>(args, *info, st);
@@ -3348,14 +3353,14 @@ int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint
 
 size_t adacomp_lazy_state_bytes(uint64_t n, uint32_t L_T)
 {
-    if (!fast_L_T(L_T)) return 0;
+    if (!fast_L_T(L_T) && !any_fast_L_T(L_T)) return 0;
     return (size_t)lazy_state_bytes(make_geometry(n, L_T));
 }
 
 int adacomp_lazy_state_init(void *state, uint64_t n, uint32_t L_T, void *stream)
 {
     if (!state) return ADACOMP_ERR_NULL;
-    if (!fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
+    if (!fast_L_T(L_T) && !any_fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
     if (misaligned(state)) return ADACOMP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(state, 0, lazy_state_bytes(make_geometry(n, L_T)), st) != cudaSuccess) return ADACOMP_ERR_CUDA;
@@ -3373,7 +3378,7 @@ int adacomp_compress_lazy(const float *grad, float *residue, void *state, uint64
 int adacomp_residue_flush(float *residue, void *state, uint64_t n, uint32_t L_T, void *stream)
 {
     if (!state || (n && !residue)) return ADACOMP_ERR_NULL;
-    if (!fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
+    if (!fast_L_T(L_T) && !any_fast_L_T(L_T)) return ADACOMP_ERR_UNSUPPORTED;
     if (misaligned(residue) || misaligned(state)) return ADACOMP_ERR_ALIGN;
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
@@ -3381,7 +3386,8 @@ int adacomp_residue_flush(float *residue, void *state, uint64_t n, uint32_t L_T,
     const u64 segs = (n + kSeg - 1) / kSeg;
     const u64 want = (segs + 255) / 256, cap = (u64)info->sms * 8;
     const unsigned grid = (unsigned)(want < 1 ? 1 : (want < cap ? want : cap));
-    lazy_flush_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(residue, static_cast<unsigned char *>(state), n, L_T);
+    lazy_flush_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(residue, static_cast<unsigned char *>(state), n, L_T,
+                                                                          make_geometry(n, L_T).tile_elems);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 

@@ -42,7 +42,10 @@ class LazyLayer:
 @pytest.mark.parametrize("L_T,n,heavy", [(50, 100352, False), (500, 147456, True), (50, 4000 * 37 + 1234, True),
                                          (500, 4000 * 300 - 7, False), (50, 3999, False), (500, 17, False),
                                          (50, 4000 * 296, False), (100, 4000 * 31 + 99, True), (125, 4000 * 12 + 1, False),
-                                         (200, 4000 * 40, False), (250, 4000 * 9 + 3999, True), (1000, 4000 * 25 + 500, False)])
+                                         (200, 4000 * 40, False), (250, 4000 * 9 + 3999, True), (1000, 4000 * 25 + 500, False),
+                                         # bins that do not line up with the 25-element segments (tiles of 3936, 3840, 3600, 3996 elements)
+                                         (41, 3936 * 21 + 40, True), (64, 3840 * 30, False), (300, 3600 * 17 + 1801, True),
+                                         (999, 3996 * 12 + 5, False), (65, 3900 * 3 - 1, False)])
 def test_lazy_steps_match_oracle_and_flush_restores_the_residue(L_T, n, heavy):
     rng = np.random.default_rng(n + L_T)
     res0 = rng.normal(0, 2e-3, n).astype(np.float32)
@@ -83,15 +86,16 @@ def test_unflushed_residue_holds_G_and_eager_continues_after_a_flush():
 
 def test_lazy_rejects_other_bin_lengths_and_foreign_state():
     dev = torch.device("cuda:0")
-    assert B.adacomp_lazy_state_bytes(1000, 64) == 0
+    assert B.adacomp_lazy_state_bytes(1000, 40) == 0
+    assert B.adacomp_lazy_state_bytes(100000, 1001) == 0
     assert B.adacomp_lazy_state_bytes(100352, 50) == 64 + 26 * 640
     n = 8000
     t = torch.zeros(n, device=dev)
-    packed = torch.empty(B.adacomp_packed_capacity(n, 64), dtype=torch.uint8, device=dev)
+    packed = torch.empty(B.adacomp_packed_capacity(n, 40), dtype=torch.uint8, device=dev)
     cnt = torch.zeros(2, dtype=torch.int64, device=dev)
     state = torch.zeros(4096, dtype=torch.uint8, device=dev)
     with pytest.raises(B.AdaCompError) as e:
-        B.adacomp_compress_lazy(t, t.clone(), state, n, 64, packed, cnt)
+        B.adacomp_compress_lazy(t, t.clone(), state, n, 40, packed, cnt)
     assert e.value.code == -9
     # a state initialised for another tensor: status bit, nothing written
     layer = LazyLayer(n, 50)
