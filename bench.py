@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--no-lazy", action="store_true")
     ap.add_argument("--no-update", action="store_true", help="skip the fused unpack + average + SGD measurement")
     ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4", "lstm"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4", "lstm", "ratecurve"],
                     help="sweep: flat tensor of 2^log2n (the default bench); configN: the multi-tensor "
                          "parameter lists, through the *_multi entry points")
     return ap.parse_args()
@@ -377,7 +377,7 @@ def run_ours(a):
 
     # ---- the same steps with lazy-scale pack(): identical streams, one pass over the residue ----
     lazy = None
-    if 41 <= L_T <= 1000 and not a.no_lazy:
+    if (41 <= L_T <= 1000 or (L_T <= 4000 and L_T % 4 == 0)) and not a.no_lazy:
         eager_counts = [tuple(int(v) for v in c.cpu()) for c in count]
         for r in residue:
             r.zero_()
@@ -615,10 +615,76 @@ def run_multi_workload(a):
     print(json.dumps(line), flush=True)
 
 
+def run_rate_curve(a):
+    """Compression rate against the bin length L_T (the axis of the paper's rate figures) on the synthetic
+    Gaussian run: for each L_T, k learners are pre-warmed PREWARM_STEPS steps from a zero residue, then one
+    step is timed (eager pack() per learner, one decode-sum with the shape known).  Rates: by the paper's
+    accounting (32 bits per element over 8 or 16 bits per sent element) and on the wire (4 n bytes over the
+    stream's bytes, which also carry the bin counts and the tile directory)."""
+    import torch
+
+    from paper_1712_02679_b200 import binding as B
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.adacomp_set_device(0)
+    n, k = 1 << min(a.log2n, 28), a.learners
+    K, W = max(a.steps, 1), max(a.warmup, 3)
+    rows = []
+    for L_T in (50, 64, 100, 200, 300, 500, 1000, 2000, 5000, 16384):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1712_02679 + L_T)
+        cap = B.adacomp_packed_capacity(n, L_T)
+        packed = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(k)]
+        count = [torch.zeros(2, dtype=torch.int64, device=dev) for _ in range(k)]
+        residue = [torch.zeros(n, device=dev) for _ in range(k)]
+        dW = torch.empty(n, device=dev)
+        dst = torch.empty(n, device=dev)
+        for _ in range(PREWARM_STEPS):
+            for l in range(k):
+                dW.normal_(0.0, SIGMA, generator=gen)
+                B.adacomp_compress(dW, residue[l], n, L_T, packed[l], count[l])
+        snap = [r.clone() for r in residue]
+        dW.normal_(0.0, SIGMA, generator=gen)
+        t_c, t_d = [], []
+        for it in range(W + K):
+            for l in range(k):
+                residue[l].copy_(snap[l])
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            for l in range(k):
+                B.adacomp_compress(dW, residue[l], n, L_T, packed[l], count[l])
+            ev[1].record()
+            B.adacomp_decompress_accumulate_ex(packed, k, dst, n, L_T)
+            ev[2].record()
+            torch.cuda.synchronize()
+            if it >= W:
+                t_c.append(ev[0].elapsed_time(ev[1]) / k)
+                t_d.append(ev[1].elapsed_time(ev[2]))
+        n_sel, used = (int(v) for v in count[0].cpu())
+        word_bits = 8 if L_T <= 64 else 16
+        rows.append({"L_T": L_T, "selected_fraction": n_sel / n,
+                     "rate_paper_accounting": 32.0 * n / max(word_bits * n_sel, 1), "rate_on_the_wire": 4.0 * n / used,
+                     "pack_ms": statistics.mean(t_c), "pack_gbs": 4.0 * n / (statistics.mean(t_c) * 1e-3) / 1e9,
+                     "decode_sum_ms": statistics.mean(t_d),
+                     "decode_sum_gbs": (4.0 * n + sum(int(c[1]) for c in count)) / (statistics.mean(t_d) * 1e-3) / 1e9})
+        del packed, residue, snap, dW, dst
+    line = {"metric": METRIC, "value": statistics.mean(r["pack_gbs"] for r in rows), "unit": "GB/s", "n_gpus": 1, "steps": K,
+            "warmup": W, "ms_per_step": sum(r["pack_ms"] * k + r["decode_sum_ms"] for r in rows), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"rate against L_T: flat fp32 gradient n=2^{min(a.log2n, 28)}, dW~N(0,1e-3), step {PREWARM_STEPS + 1} "
+                                   f"of a run from a zero residue, {k} learners (the same dW, their own residues)",
+                       "l2": "inputs far beyond the 126 MB L2" if n >= 1 << 26 else "small case"},
+            "rate_curve": rows, "device_status": B.adacomp_device_status()}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.workload == "ratecurve":
+        run_rate_curve(a)
     elif a.workload != "sweep":
         run_multi_workload(a)
     else:

@@ -296,9 +296,9 @@ int adacomp_compress_profile(const float *grad, float *residue, uint64_t n, uint
  *   residue  between calls it is NOT the paper's residue: run adacomp_residue_flush before
  *            reading it (checkpointing), before handing it to adacomp_compress, or before
  *            changing L_T.  After a flush it is exactly what adacomp_compress would have left.
- * L_T from 41 to 1000 is supported (the paper's two settings, 50 and 500, among them: the bin lengths
- * the pipelined tile pass takes): others return ADACOMP_ERR_UNSUPPORTED (adacomp_lazy_state_bytes
- * returns 0).  A state that does not belong to
+ * L_T from 41 to 1000, and the multiples of 4 from 1004 to 4000, are supported (the paper's two
+ * settings, 50 and 500, among them: the bin lengths the pipelined tile pass takes): others return
+ * ADACOMP_ERR_UNSUPPORTED (adacomp_lazy_state_bytes returns 0).  A state that does not belong to
  * (n, L_T) sets ADACOMP_DEV_HEADER_MISMATCH and nothing is written.
  */
 size_t adacomp_lazy_state_bytes(uint64_t n, uint32_t L_T);

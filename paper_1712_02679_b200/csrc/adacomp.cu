@@ -294,7 +294,8 @@ __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shar
 
 // ---------------------------------------------------------------------------------
 // tile_pass, fast path: L_T = 25 * SPB for SPB = 2, 4, 5, 8, 10, 20, 40 (L_T = 50 ... 1000), tiles of 4000 elements;
-// and, as SPB = 0, every other L_T from 41 to 1000 (tiles of 3200 to 4000 elements, bins anywhere).
+// and, as SPB = 0, every other L_T from 41 to 1000 (tiles of 3200 to 4000 elements, bins anywhere) and the
+// multiples of 4 up to 4000 (a tile is one bin).
 //
 // Thread t < 160 owns the 25 consecutive elements of segment t (stride 25 words in
 // shared memory: odd, so a warp's accesses are bank-conflict free); a bin is SPB
@@ -2811,8 +2812,12 @@ bool with_fast_kernel(u32 L_T, F f)
 }
 constexpr u32 kFastL_T[] = {50u, 100u, 125u, 200u, 250u, 500u, 1000u};
 // Every other L_T from 41 to 1000 (tiles of at most 96 bins, bins longer than a thread's 25 elements) takes
-// the same kernel in its any-bin form (fp32 gradient, eager).
-__host__ __device__ inline bool any_fast_L_T(u32 L_T) { return L_T >= 41u && L_T <= 1000u && !fast_L_T(L_T); }
+// the same kernel in its any-bin form (fp32 gradient), and so do the one-bin tiles of at most 4000 elements
+// that start on 16-byte boundaries (L_T up to 4000, a multiple of 4).
+__host__ __device__ inline bool any_fast_L_T(u32 L_T)
+{
+    return (L_T >= 41u && L_T <= 1000u && !fast_L_T(L_T)) || (L_T > 1000u && L_T <= (u32)kFastTile && L_T % 4u == 0);
+}
 template <bool LAZY, typename F>
 void with_any_fast_kernel(u32 L_T, F f)
 {

@@ -45,7 +45,9 @@ class LazyLayer:
                                          (200, 4000 * 40, False), (250, 4000 * 9 + 3999, True), (1000, 4000 * 25 + 500, False),
                                          # bins that do not line up with the 25-element segments (tiles of 3936, 3840, 3600, 3996 elements)
                                          (41, 3936 * 21 + 40, True), (64, 3840 * 30, False), (300, 3600 * 17 + 1801, True),
-                                         (999, 3996 * 12 + 5, False), (65, 3900 * 3 - 1, False)])
+                                         (999, 3996 * 12 + 5, False), (65, 3900 * 3 - 1, False),
+                                         # a tile is one bin
+                                         (1004, 1004 * 41 + 3, False), (2000, 2000 * 33 + 1999, True), (4000, 4000 * 9 + 1, False)])
 def test_lazy_steps_match_oracle_and_flush_restores_the_residue(L_T, n, heavy):
     rng = np.random.default_rng(n + L_T)
     res0 = rng.normal(0, 2e-3, n).astype(np.float32)

@@ -72,12 +72,12 @@ def test_fast_path_tile_boundaries(L_T, n):
     run_steps(n, L_T, dws[:2], flags=B.ADACOMP_FLAG_GENERIC_PATH | B.ADACOMP_FLAG_LITERAL)
 
 
-@pytest.mark.parametrize("L_T", [41, 52, 64, 65, 96, 300, 333, 400, 800, 999])
+@pytest.mark.parametrize("L_T", [41, 52, 64, 65, 96, 300, 333, 400, 800, 999, 1004, 1500, 2000, 3000, 3996, 4000])
 def test_any_bin_tile_pass_tile_boundaries(L_T):
     """Bin lengths whose bins do not line up with the threads' 25-element segments: the tile pass
     finds each segment's one or two bins at run time.  Whole tiles, ragged tails, many tiles; with a
     scale-factor; and against the warp-per-bin kernel on the same inputs."""
-    T = 4 * (1000 // L_T) * L_T
+    T = 4 * (1000 // L_T) * L_T if L_T <= 1000 else L_T        # a tile (one bin where L_T > 1000)
     for n in (T, 2 * T, 2 * T - 1, 2 * T + 1, T * 150 + 1, T * 301 - L_T - 3):
         rng = np.random.default_rng(n + L_T)
         dws = [synth.heavy_dw(n, 1e-3, rng) for _ in range(3)]
