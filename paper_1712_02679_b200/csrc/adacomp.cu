@@ -812,6 +812,106 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     __syncthreads();
 }
 
+// A tile that is one bin (L_T > 1000), by the whole CTA.  Per element only a signed key stays in shared
+// memory: max(|H|, |G|) (|H| alone under the literal flag) with G's sign, zero where G is zero; an element
+// goes out when the key's magnitude reaches the bin's maximum, which is known once all of G has gone by.
+// G itself is written to the residue as it is formed.  Dynamic shared memory: key[L_T], words[L_T].
+template <typename Word>
+__device__ void generic_tile_one_bin(const TileIo &a, const Geometry &geo, u64 tile, unsigned char *smem_raw, u32 *s_tmp,
+                                     u64 *s_acc)
+{
+    const int L = (int)geo.L_T;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int nwarp = kGenericThreads / 32;
+    float *s_key = reinterpret_cast<float *>(smem_raw);
+    Word *s_words = reinterpret_cast<Word *>(s_key + L);
+    const u64 base = tile * (u64)L;
+    const u64 left = geo.n - base;
+    const int elems = left < (u64)L ? (int)left : L;
+
+    auto key_of = [&](float r, float d, float &g) {
+        g = __fadd_rn(r, d);
+        const float h = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g, d);
+        const float k = a.literal ? fabsf(h) : fmaxf(fabsf(h), fabsf(g));
+        return g == 0.f ? 0.f : copysignf(k, g);
+    };
+    float m = 0.f;
+    // (four elements a step where the bin starts on a 16-byte boundary)
+    const int quads = (base & 3u) == 0 && !a.grad_bf16 ? elems >> 2 : 0;
+    for (int i = tid; i < quads; i += kGenericThreads) {
+        const float4 d = reinterpret_cast<const float4 *>(a.grad + base)[i];
+        const float4 r = reinterpret_cast<const float4 *>(a.residue + base)[i];
+        float4 g, k;
+        k.x = key_of(r.x, d.x, g.x);
+        k.y = key_of(r.y, d.y, g.y);
+        k.z = key_of(r.z, d.z, g.z);
+        k.w = key_of(r.w, d.w, g.w);
+        m = fmaxf(fmaxf(m, fmaxf(fabsf(g.x), fabsf(g.y))), fmaxf(fabsf(g.z), fabsf(g.w)));
+        reinterpret_cast<float4 *>(a.residue + base)[i] = g;
+        reinterpret_cast<float4 *>(s_key)[i] = k;
+    }
+    for (int i = 4 * quads + tid; i < L; i += kGenericThreads) {
+        float k = 0.f;
+        if (i < elems) {
+            float g;
+            k = key_of(a.residue[base + i], load_grad(a.grad, base + i, a.grad_bf16), g);
+            m = fmaxf(m, fabsf(g));
+            a.residue[base + i] = g;
+        }
+        s_key[i] = k;
+    }
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    if (lane == 0) s_tmp[warp] = __float_as_uint(m);
+    __syncthreads();
+    m = 0.f;
+    for (int q = 0; q < nwarp; q++) m = fmaxf(m, __uint_as_float(s_tmp[q]));
+    __syncthreads();                                   // s_tmp is reused for the counts
+
+    // a warp per eighth of the bin (whole 32-element steps, so that the words stay in ascending order)
+    const int part = ((L + nwarp - 1) / nwarp + 31) & ~31;
+    const int j_lo = warp * part, j_hi = min(L, j_lo + part);
+    u32 count = 0;
+    if (m > 0.f)
+        for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
+            const int j = j0 + lane;
+            const float k = j < j_hi ? s_key[j] : 0.f;
+            count += __popc(__ballot_sync(0xffffffffu, fabsf(k) >= m && k != 0.f));
+        }
+    if (lane == 0) s_tmp[warp] = count;
+    __syncthreads();
+    u32 at = 0, total = 0;
+    for (int q = 0; q < nwarp; q++) {
+        const u32 c = s_tmp[q];
+        if (q < warp) at += c;
+        total += c;
+    }
+    if (m > 0.f)
+        for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
+            const int j = j0 + lane;
+            const float k = j < j_hi ? s_key[j] : 0.f;
+            const bool sel = fabsf(k) >= m && k != 0.f;
+            const u32 mask = __ballot_sync(0xffffffffu, sel);
+            if (sel) s_words[at + __popc(mask & ((1u << lane) - 1u))] = (Word)(((u32)j << 2) | (k < 0.f ? 3u : 1u));
+            at += __popc(mask);
+        }
+    __syncthreads();
+
+    Word *slot = reinterpret_cast<Word *>(a.scratch + geo.slots_at + tile * geo.slot_bytes);
+    for (u32 i = tid; i < total; i += kGenericThreads) slot[i] = s_words[i];
+    if (tid == 0) {
+        reinterpret_cast<Word *>(a.packed + geo.bin_cnt_at)[tile] = (Word)total;       // (a tile is a bin)
+        reinterpret_cast<u32 *>(a.scratch + geo.tile_cnt_at)[tile] = total;
+        if (total) atomicAdd(&reinterpret_cast<u64 *>(a.scratch + geo.group_at)[tile / kGroupTiles], (u64)total);
+        u32 window;
+        u64 lo, hi;
+        if (split_for_sum(m, window, lo, hi)) {
+            atomicAdd(&s_acc[window], lo);
+            atomicAdd(&s_acc[window + 1], hi);
+        }
+    }
+    __syncthreads();
+}
+
 template <typename Word>
 __global__ void __launch_bounds__(kGenericThreads)
 tile_pass_generic(PassArgs a)
@@ -823,8 +923,10 @@ tile_pass_generic(PassArgs a)
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
     const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_bf16};
-    for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x)
-        generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
+    for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x) {
+        if (a.geo.tile_bins == 1u && sizeof(Word) == 2) generic_tile_one_bin<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
+        else generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
+    }
     if (tid < kWindows) {
         const u64 v = s_acc[tid];
         if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + tid, v);
@@ -2911,7 +3013,9 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 {
     const Geometry &geo = args.geo;
     const size_t units = geo.tile_bins < 8u ? 8u : geo.tile_bins;      // generic_tile: a bin or a part of one per warp
-    const size_t smem = (size_t)align_up((u64)geo.tile_elems * (8 + sizeof(Word)), 16) + units * 4 + (units + 1) * 4;
+    const size_t smem = geo.tile_bins == 1u && sizeof(Word) == 2
+                            ? (size_t)align_up((u64)geo.tile_elems * (4 + sizeof(Word)), 16)      // generic_tile_one_bin
+                            : (size_t)align_up((u64)geo.tile_elems * (8 + sizeof(Word)), 16) + units * 4 + (units + 1) * 4;
     if (smem > (size_t)info.smem_optin) return ADACOMP_ERR_SIZE;
     if (cudaFuncSetAttribute(tile_pass_generic<Word>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
@@ -2960,7 +3064,10 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_bf16 ? 1u : 0u};
         const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
-        const bool any_fast = any_fast_L_T(L_T) && flags == 0 && !grad_bf16 && info->fast_ready;
+        // (one-bin tiles fill the pipelined kernel's 4000-element stages only in part: below 2800 elements the
+        // warp-per-part kernel is faster, measured; lazy-scale mode exists in the pipelined kernel only)
+        const bool any_fast = any_fast_L_T(L_T) && flags == 0 && !grad_bf16 && info->fast_ready &&
+                              (lazy || L_T <= 1000u || L_T >= 2800u);
         if (fast || any_fast) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
@@ -3158,7 +3265,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f, 0u};
-        if ((fast_L_T(L_T) || any_fast_L_T(L_T)) && info->fast_ready) {
+        if ((fast_L_T(L_T) || (any_fast_L_T(L_T) && (L_T <= 1000u || L_T >= 2800u))) && info->fast_ready) {
             const u64 cap = (u64)info->sms * 2;
             const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
             auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
