@@ -306,6 +306,54 @@ def test_decoder_flags_bad_streams_without_faulting():
     assert B.adacomp_device_status() == 0
 
 
+@pytest.mark.parametrize("L_T,n", [(50, 4000 * 6 + 77), (62, 3968 * 5 + 9), (200, 4000 * 4 + 150), (500, 4000 * 5 + 3),
+                                   (1001, 4096 * 5 + 100), (5000, 5000 * 7 + 11), (16384, 16384 * 3 + 5)])
+def test_decoder_flags_out_of_range_words_and_inflated_counts(L_T, n):
+    """Streams that disagree with themselves (every read they ask for stays inside the stream): a word
+    whose index is past its bin is skipped and flagged; a bin count that makes a tile's counts exceed
+    its directory entry is flagged and costs at most that tile's neighbourhood."""
+    rng = np.random.default_rng(L_T + n)
+    good = cref.pack(rng.normal(0, 1e-3, n).astype(np.float32), np.zeros(n, np.float32), L_T)
+    a = cref.pack(rng.normal(0, 1e-3, n).astype(np.float32), np.zeros(n, np.float32), L_T)
+    w = a.w
+    n_tiles_bytes = 8 * (a.n_tiles + 1)
+    bin_cnt_at = (64 + n_tiles_bytes + 15) & ~15
+    payload_at = (bin_cnt_at + a.n_bins * w + 15) & ~15
+    pos, codes = a.positions_and_codes()
+    alone = cref.unpack_sum([good.raw], n)
+    both = cref.unpack_sum([good.raw, a.raw], n)
+
+    # a word in the middle of the stream gets the index L_T (one past its bin's last element)
+    j = a.n_sel // 2
+    word = (L_T << 2) | int(codes[j])
+    if word < (1 << (8 * w)):                                 # (L_T = 16384: every index a word can hold is inside the bin)
+        bad = a.raw.copy()
+        bad[payload_at + j * w: payload_at + (j + 1) * w] = np.frombuffer(int(word).to_bytes(w, "little"), dtype=np.uint8)
+        B.adacomp_device_status_reset()
+        got = gpu_decode([good.raw, bad], n)
+        assert B.adacomp_device_status() == B.ADACOMP_DEV_BAD_STREAM
+        want = both.copy()
+        want[pos[j]] = alone[pos[j]]                          # the bad word is skipped
+        assert_f32_bits_equal(got, want, f"L_T={L_T} out-of-range word")
+
+    # a bin of a middle tile claims one word more than it has
+    b = (a.n_bins // 2)
+    bad = a.raw.copy()
+    cnt = int(a.bin_cnt[b]) + 1
+    bad[bin_cnt_at + b * w: bin_cnt_at + (b + 1) * w] = np.frombuffer(cnt.to_bytes(w, "little"), dtype=np.uint8)
+    B.adacomp_device_status_reset()
+    got = gpu_decode([good.raw, bad], n)
+    assert B.adacomp_device_status() & B.ADACOMP_DEV_BAD_STREAM
+    # everything farther than a tile (and a 4096-element work item) from that bin is untouched by it
+    reach = max(a.tile_bins * L_T, 4096) + L_T
+    lo, hi = max(0, b * L_T - reach), min(n, (b + 1) * L_T + reach)
+    assert_f32_bits_equal(got[:lo], both[:lo], f"L_T={L_T} inflated count, before")
+    assert_f32_bits_equal(got[hi:], both[hi:], f"L_T={L_T} inflated count, after")
+    assert np.all(np.isfinite(got))
+    B.adacomp_device_status_reset()
+    assert B.adacomp_device_status() == 0
+
+
 def test_nonfinite_gradient_sets_a_status_bit_and_returns():
     n = 8000
     dW = np.full(n, 1e-3, np.float32)
