@@ -1219,7 +1219,11 @@ gather_fixup(float *residue, unsigned char *packed, const unsigned char *scratch
 // ---------------------------------------------------------------------------------
 
 constexpr int kBatchMax = 160;                       // layers per batched launch (parameter space: 32 KB)
-constexpr u64 kBatchLayerMaxElems = 1ull << 22;      // larger layers take the single-layer kernels
+constexpr u64 kBatchLayerMaxElems = 1ull << 22;      // decode: larger layers take the single-layer kernels
+// pack(): layers up to this size share a batch's launches when the pipelined batch tile pass is there (a
+// layer alone ramps its pipeline up and down over a few tiles per CTA and pays four launches and a finalize
+// of its own: below 2^24 elements it runs at under half the speed it has inside a batch)
+constexpr u64 kPackBatchMaxElems = 1ull << 25;
 constexpr u32 kBatchSmemBytes = 4000 * 10 + 4 * kSmallBins + 4 * (kSmallBins + 1) + 16;
 
 struct BatchLayer {
@@ -1295,6 +1299,260 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
         else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
     }
     flush();
+}
+
+// The pipelined tile pass (any-bin form: fp32 gradient, eager, no flags) over the tiles of a whole batch of
+// layers: global tile gt belongs to the layer whose tile_first is the largest not above it.  The CTA's
+// tiles go up, so each thread (and, for the loads two tiles ahead, the service lane) keeps a cursor
+// into the layer table; what depends on the layer's bin length (the place of a thread's 25 elements among
+// the bins) is recomputed when the cursor moves, and the CTA's share of a layer's exact g_max sum is added
+// to that layer's windows when the CTA leaves the layer.  Every layer here has 41 <= L_T <= 1000.
+template <int N>
+__global__ void __launch_bounds__(kFastThreads, 2)
+batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *s_words = smem + FastSmem::kWordsAt;
+    u32 *s_incl = reinterpret_cast<u32 *>(smem + FastSmem::kInclAt);
+    u32 *s_wtot = reinterpret_cast<u32 *>(smem + FastSmem::kWtotAt);
+    u32 *s_anymax = reinterpret_cast<u32 *>(smem + FastSmem::kBinmaxAt);    // [2][kSmallBins] bits of the bin maxima, by tile parity
+    u32 *s_anycnt = s_anymax + 2 * kSmallBins;                               // [2][kSmallBins] words per bin
+    u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
+    u64 *s_full = reinterpret_cast<u64 *>(smem + FastSmem::kBarAt);
+    volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FastSmem::kAbortAt);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool service = warp == 5;
+    const u32 first = blockIdx.x, stride = gridDim.x;
+    const u32 my_tiles = b.total_tiles > first ? (b.total_tiles - first + stride - 1) / stride : 0;
+    const int n_layers = (int)b.n_layers;
+    auto seek = [&](u32 gt, int &li) {      // (tiles only go up)
+        while (li + 1 < n_layers && b.layer[li + 1].tile_first <= gt) li++;
+    };
+
+    if (tid < kWindows + 1) s_acc[tid] = 0;
+    for (int i = tid; i < 4 * kSmallBins; i += kFastThreads) s_anymax[i] = 0;
+    if (tid == 0) {
+        *s_abort = 0;
+        for (int st = 0; st < kStages; st++) mbar_init(&s_full[st], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    u32 issued = 0;                     // service lane 0: loads issued for tiles [0, issued)
+    int load_li = 0;
+    auto issue_load = [&](u32 i) {
+        if (i >= my_tiles) return;
+        const u32 gt = first + i * stride;
+        seek(gt, load_li);
+        const BatchLayer &L = b.layer[load_li];
+        const u32 lt = gt - L.tile_first, T = L.geo.tile_elems;
+        if ((u64)lt >= L.geo.n / T) return;             // a ragged last tile is read with plain loads
+        unsigned char *st = smem + (i % kStages) * kStageBytes;
+        u64 *bar = &s_full[i % kStages];
+        mbar_arrive_expect_tx(bar, 8u * T);
+        bulk_load(st, L.grad + (u64)lt * T, 4u * T, bar);
+        bulk_load(st + kTileBytes, L.residue + (u64)lt * T, 4u * T, bar);
+        issued = i + 1;
+    };
+    if (service && lane == 0) {
+        issue_load(0);
+        issue_load(1);
+    }
+
+    int li = 0, at_li = -1;             // the tile's layer; the layer the values below belong to
+    u32 phase = 0;                      // bit s: parity of stage s's next completion (ragged tiles use no barrier)
+    int T = 0, TB = 0, b0 = 0, cut = kSeg, off0 = 0, vcount = 0;
+    u32 full_tiles = 0, wbytes = 1;
+    auto flush = [&]() {                // (service warp) this CTA's share of layer at_li's exact sum
+        if (at_li >= 0 && lane < kWindows) {
+            const u64 v = s_acc[lane];
+            if (v) atomicAdd(reinterpret_cast<u64 *>(b.layer[at_li].packed + b.layer[at_li].geo.scratch_at) + lane, v);
+            s_acc[lane] = 0;
+        }
+        __syncwarp();
+    };
+    u32 i = 0;
+    for (; i < my_tiles; i++) {
+        const u32 gt = first + i * stride;
+        seek(gt, li);
+        const BatchLayer &L = b.layer[li];
+        const Geometry &geo = L.geo;
+        if (li != at_li) {
+            if (service) flush();
+            at_li = li;
+            T = (int)geo.tile_elems;
+            TB = (int)geo.tile_bins;
+            full_tiles = (u32)(geo.n / (u64)T);
+            wbytes = geo.w;
+            // the thread's elements [0, cut) lie in bin b0 of the tile, from place off0 of it on, the others
+            // in bin b0 + 1; only the first `vcount` of them exist (tiles of less than 4000 elements)
+            const int Lt = (int)geo.L_T, e0 = tid * kSeg;
+            b0 = e0 / Lt;
+            off0 = e0 - b0 * Lt;
+            cut = min(kSeg, Lt - off0);
+            vcount = max(0, min(kSeg, T - e0));
+        }
+        unsigned char *scratch = L.packed + geo.scratch_at;
+        const u32 lt = gt - L.tile_first;
+        const u64 base = (u64)lt * (u64)T;
+        float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
+        float *s_r = s_d + kFastTile;
+        const bool whole = lt < full_tiles;
+        const int elems = whole ? T : (int)(geo.n - base);
+        u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
+
+        if (whole) {
+            const u32 stage = i % kStages;
+            if (!mbar_wait(&s_full[stage], (phase >> stage) & 1u)) {
+                *s_abort = 1;                      // every thread that times out says so
+                raise_status(ADACOMP_DEV_TIMEOUT);
+            }
+            phase ^= 1u << stage;
+        } else {
+            // the ragged last tile of a layer: plain loads, zero fill past the end
+            for (int e = tid; e < kFastTile; e += kFastThreads) {
+                float d = 0.f, r = 0.f;
+                if (e < elems) { d = L.grad[base + e]; r = L.residue[base + e]; }
+                s_d[e] = d;
+                s_r[e] = r;
+            }
+            __syncthreads();
+        }
+
+        // ---- G = residue + dW, H = G + dW; the maxima of |G| over the segment's part of each bin ----
+        float g[kSeg], key[kSeg];
+        float gm = 0.f, gm1 = 0.f;
+        u32 selmask = 0, cnt = 0, incl = 0;
+        if (!service) {
+            const float *pd = s_d + tid * kSeg;
+            const float *pr = s_r + tid * kSeg;
+            float m = 0.f, m1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < kSeg; j++) {
+                float d = pd[j], r = pr[j];
+                if (j >= vcount) d = r = 0.f;               // past the tile's end
+                g[j] = __fadd_rn(r, d);
+                const float h = __fadd_rn(g[j], d);
+                if (j >= cut) m1 = fmaxf(m1, fabsf(g[j]));
+                else m = fmaxf(m, fabsf(g[j]));
+                key[j] = fmaxf(fabsf(h), fabsf(g[j]));
+            }
+            // (non-negative floats order like their bits)
+            if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
+            if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
+        }
+        __syncthreads();                                            // barrier A
+        // the other parity's buffers are free: tile i - 1 is done with them, tile i + 1 starts after barrier D
+        if (tid < kSmallBins) {
+            s_anymax[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+            s_anycnt[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+        }
+        if (!service) {
+            gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
+            gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
+            // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
+#pragma unroll
+            for (int j = 0; j < kSeg; j++)
+                if (key[j] >= (j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
+            cnt = __popc(selmask);
+            const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
+            if (c0) atomicAdd(&any_cnt[b0], c0);
+            if (cnt - c0) atomicAdd(&any_cnt[b0 + 1], cnt - c0);
+            incl = warp_inclusive_scan(cnt, lane);
+            s_incl[tid] = incl;
+            if (lane == 31) s_wtot[warp] = incl;
+        }
+        __syncthreads();                                            // barrier B
+
+        u32 total = 0;
+        if (!service) {
+            // ---- words into the staging area, G back into the residue stage ----
+            u32 wpre = 0;
+#pragma unroll
+            for (int wv = 0; wv < 5; wv++)
+                if (wv < warp) wpre += s_wtot[wv];
+            float *pr = s_r + tid * kSeg;
+#pragma unroll
+            for (int j = 0; j < kSeg; j++) pr[j] = g[j];
+            u32 at = wpre + incl - cnt;
+            u32 mask = selmask;
+            while (mask) {
+                const int j = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const u32 neg = __float_as_uint(pr[j]) >> 31;
+                const u32 idx = j >= cut ? (u32)(j - cut) : (u32)(off0 + j);        // the element's place in its bin
+                const u32 word = (idx << 2) | 1u | (neg << 1);
+                if (wbytes == 1u) s_words[at] = (unsigned char)word;
+                else reinterpret_cast<unsigned short *>(s_words)[at] = (unsigned short)word;
+                at++;
+            }
+            if (tid < TB) {
+                const u64 bin = (u64)lt * (u64)TB + tid;
+                if (bin < geo.n_bins) {
+                    unsigned char *bc = L.packed + geo.bin_cnt_at;
+                    if (wbytes == 1u) bc[bin] = (unsigned char)any_cnt[tid];
+                    else reinterpret_cast<unsigned short *>(bc)[bin] = (unsigned short)any_cnt[tid];
+                }
+            }
+            fence_async_smem();          // the bulk store below reads what was just written
+        } else {
+            total = s_wtot[0] + s_wtot[1] + s_wtot[2] + s_wtot[3] + s_wtot[4];
+            for (int bb = 0; bb < TB; bb += 32) {       // every lane takes part each round
+                const int bq = bb + lane;
+                const bool valid = bq < TB && (u64)lt * (u64)TB + bq < geo.n_bins;
+                warp_accumulate(s_acc, valid ? __uint_as_float(any_max[bq]) : 0.f, valid);
+            }
+            if (lane == 0) {
+                bulk_wait_read_all();    // the store of tile i - 1 has drained its stage
+                issue_load(i + 2);
+            }
+        }
+        __syncthreads();                                            // barrier D
+
+        const bool aborted = *s_abort != 0;
+        if (service && !aborted) {
+            if (whole) {
+                if (lane == 0) {
+                    bulk_store(L.residue + base, s_r, 4u * (u32)T);
+                    bulk_commit();
+                }
+            } else {
+                for (int e = lane; e < elems; e += 32) L.residue[base + e] = s_r[e];
+            }
+            uint4 *slot = reinterpret_cast<uint4 *>(scratch + geo.slots_at + (u64)lt * geo.slot_bytes);
+            const int chunks = (int)((total * wbytes + 15) / 16);
+            for (int c = lane; c < chunks; c += 32) slot[c] = reinterpret_cast<uint4 *>(s_words)[c];
+            if (lane == 0) {
+                reinterpret_cast<u32 *>(scratch + geo.tile_cnt_at)[lt] = total;
+                if (total) atomicAdd(&reinterpret_cast<u64 *>(scratch + geo.group_at)[lt / kGroupTiles], (u64)total);
+            }
+        }
+        if (aborted) break;          // uniform: the flag was set before barrier D
+    }
+
+    if (service) {
+        if (lane == 0) {
+            bulk_wait_all();
+            if (*s_abort) {
+                // after a timeout: loads still in flight must land (or time out in turn) before this CTA's
+                // shared memory is given back, and the tiles it never finished count as empty so that the
+                // kernels after this one stay inside their buffers
+                int zl = 0;
+                for (u32 j = i; j < my_tiles; j++) {
+                    const u32 gt = first + j * stride;
+                    seek(gt, zl);
+                    const BatchLayer &Z = b.layer[zl];
+                    const u32 zt = gt - Z.tile_first;
+                    if (j > i && j < issued && (u64)zt < Z.geo.n / Z.geo.tile_elems)       // (a load was started for it)
+                        mbar_wait(&s_full[j % kStages], (phase >> (j % kStages)) & 1u);
+                    reinterpret_cast<u32 *>(Z.packed + Z.geo.scratch_at + Z.geo.tile_cnt_at)[zt] = 0;
+                }
+            }
+        }
+        __syncwarp();
+        flush();
+    }
 }
 
 template <int N>
@@ -2933,7 +3191,8 @@ struct DeviceInfo {
     int decode_per_sm = 0;
     int decode_warps_per_sm = 0, decode_one_per_sm = 0;
     int decode_opt_per_sm[2][2] = {{0, 0}, {0, 0}};     // [SGD, Adam][4, 8 decoding warps]; 0: unavailable on this device
-    int batch_per_sm = 0;       // 0: batched pack() unavailable on this device
+    int batch_per_sm = 0;
+    bool batch_fast_ready = false;      // the pipelined batch tile pass can be launched       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     bool fast_ready = false;
 };
@@ -2994,6 +3253,9 @@ int device_info(DeviceInfo *&out)
                                                           kBatchSmemBytes);
             d.batch_per_sm = per;
         }
+        d.batch_fast_ready = d.fast_ready &&
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax>, at, bytes) == cudaSuccess &&
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall>, at, bytes) == cudaSuccess;
         if (cudaFuncSetAttribute(decode_batch, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sizeof(DecodeBatchSmem)) == cudaSuccess) {
             int per = 0;
@@ -3183,9 +3445,15 @@ int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStrea
 {
     batch_clear<N><<<b.n_layers, 128, 0, st>>>(b);
     if (b.total_tiles) {
-        const u64 cap = (u64)info.sms * info.batch_per_sm;
-        const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
-        batch_tile_pass<N><<<grid, kGenericThreads, kBatchSmemBytes, st>>>(b);
+        if (info.batch_fast_ready) {
+            const u64 cap = (u64)info.sms * 2;
+            const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
+            batch_tile_pass_fast<N><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+        } else {
+            const u64 cap = (u64)info.sms * info.batch_per_sm;
+            const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
+            batch_tile_pass<N><<<grid, kGenericThreads, kBatchSmemBytes, st>>>(b);
+        }
     }
     batch_finalize<N><<<b.n_layers, 1024, 0, st>>>(b);
     if (b.total_tiles) {
@@ -3214,9 +3482,9 @@ int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st)
     return launch_batch_sized(b, info, st);
 }
 
-inline bool batchable(const adacomp_layer_desc &d)
+inline bool batchable(const adacomp_layer_desc &d, const DeviceInfo &info)
 {
-    return d.flags == 0 && d.L_T >= 42u && d.L_T <= 1000u && d.n < kBatchLayerMaxElems;
+    return d.flags == 0 && d.L_T >= 42u && d.L_T <= 1000u && d.n < (info.batch_fast_ready ? kPackBatchMaxElems : kBatchLayerMaxElems);
 }
 
 // ---------------------------------------------------------------------------------
@@ -3569,7 +3837,7 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
     batch.total_tiles = 0;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (info->batch_per_sm > 0 && batchable(d)) {
+        if (info->batch_per_sm > 0 && batchable(d, *info)) {
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
