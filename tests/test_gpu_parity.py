@@ -366,13 +366,15 @@ def test_nonfinite_gradient_sets_a_status_bit_and_returns():
 
 
 def test_multi_tensor_calls_match_single_calls():
-    # a mix: small layers (batched launches), an empty one, bin lengths outside the batched range and
-    # one layer large enough for the single-layer fast path
+    # a mix: small and mid-size layers (batched launches: the layer and its bin length change from tile to
+    # tile), an empty one, bin lengths outside the batched range and one layer beyond the batch's size limit
+    # (the single-layer kernels)
     specs = synth.resnet50_tensors()[:30] + [
         synth.TensorSpec("empty", 0, 50, "fc"), synth.TensorSpec("odd_bins", 12345, 7, "fc"),
         synth.TensorSpec("long_bins", 54321, 5000, "fc"), synth.TensorSpec("big", (1 << 22) + 4321, 50, "fc"),
         synth.TensorSpec("tail_of_one", 4001, 500, "conv"), synth.TensorSpec("lt42", 9999, 42, "fc"),
-        synth.TensorSpec("lt1000", 99999, 1000, "fc")]
+        synth.TensorSpec("lt1000", 99999, 1000, "fc"), synth.TensorSpec("lt333", 3996 * 7 + 5, 333, "fc"),
+        synth.TensorSpec("alone", (1 << 25) + 7, 500, "fc"), synth.TensorSpec("lt64", 3840 * 3, 64, "conv")]
     dev = torch.device("cuda:0")
     layers, singles, dws = [], [], []
     for t, spec in enumerate(specs):
