@@ -598,6 +598,28 @@ def run_multi_workload(a):
             evf.append(e)
     torch.cuda.synchronize()
     t_f = statistics.mean(e[0].elapsed_time(e[1]) for e in evf)
+    # pack() of the same step in lazy-scale mode (identical streams; no fix-up of the sent residues)
+    t_lz = None
+    if all(41 <= s.L_T <= 1000 for s in specs):
+        states = [[torch.empty(B.adacomp_lazy_state_bytes(s.n, s.L_T), dtype=torch.uint8, device=dev) for s in specs]
+                  for _ in range(learners)]
+        state_arr = [B.make_pointer_array(st, torch.uint8) for st in states]
+        evl = []
+        for it in range(W + K):
+            for d in layers:
+                d["residue"].zero_()
+            for l in range(learners):
+                for st, s in zip(states[l], specs):
+                    B.adacomp_lazy_state_init(st, s.n, s.L_T)
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            e[0].record()
+            for l in range(learners):
+                B.adacomp_compress_multi_lazy(descs[l], state_arr[l], nl)
+            e[1].record()
+            if it >= W:
+                evl.append(e)
+        torch.cuda.synchronize()
+        t_lz = statistics.mean(e[0].elapsed_time(e[1]) for e in evl)
     t_c = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     t_d = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     n_sel = sum(int(d["count_out"][0]) for d in layers[:nl])
@@ -608,7 +630,7 @@ def run_multi_workload(a):
         "config": {"workload": f"{'LSTM list (67-512-512-67)' if cfg == 6 else 'config ' + str(cfg)}: {nl} tensors, {total} elements, {learners} learners, first step "
                                f"from a zero residue, dW~N(0,1e-3); *_multi entry points",
                    "l2": "working set %.0f MB" % (12.0 * total * learners / 1e6)},
-        "compress_ms": t_c, "compress_gbs": 4.0 * total * learners / (t_c * 1e-3) / 1e9,
+        "compress_ms": t_c, "compress_gbs": 4.0 * total * learners / (t_c * 1e-3) / 1e9, "compress_lazy_ms": t_lz,
         "decompress_sum_ms": t_d, "fused_update_ms": t_f, "graph_replay_ms_per_step": t_g, "decompress_sum_gbs": 4.0 * total / (t_d * 1e-3) / 1e9,
         "selected_fraction_learner0": n_sel / max(total, 1), "device_status": B.adacomp_device_status(),
     }

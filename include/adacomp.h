@@ -347,6 +347,18 @@ typedef struct {
 int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream);
 
 /*
+ * adacomp_compress_multi in lazy-scale mode (see adacomp_compress_lazy): states[t] (HOST array of device
+ * pointers) is layer t's state, adacomp_lazy_state_bytes(n, L_T) bytes, set up once by
+ * adacomp_lazy_state_init; every layer's residue holds G between calls until adacomp_residue_flush.
+ * Streams, scales and (flushed) residues are those of adacomp_compress_multi, bit for bit.
+ * Every layer needs flags 0 and a bin length the lazy mode takes, else ADACOMP_ERR_UNSUPPORTED and
+ * nothing is launched.  A state that is not its layer's sets ADACOMP_DEV_HEADER_MISMATCH; that
+ * layer is left untouched and its stream is empty.
+ */
+int adacomp_compress_multi_lazy(const adacomp_layer_desc *layers, void *const *states, uint32_t n_layers,
+                                void *stream);
+
+/*
  * unpack()-and-sum of every layer: packed[t * k_streams + l] (HOST array) is
  * learner l's stream of layer t, dst[t] (HOST array of device pointers) its output.
  */

@@ -110,6 +110,8 @@ def lib() -> C.CDLL:
                                                          C.c_uint64, C.c_void_p]
         L.adacomp_compress_multi.restype = C.c_int
         L.adacomp_compress_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+        L.adacomp_compress_multi_lazy.restype = C.c_int
+        L.adacomp_compress_multi_lazy.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
         L.adacomp_decompress_accumulate_multi.restype = C.c_int
         L.adacomp_decompress_accumulate_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p,
                                                           C.c_uint32, C.c_void_p]
@@ -398,6 +400,16 @@ def adacomp_compress_multi(layers, n_layers: int, stream=None) -> None:
         layers = make_layer_descs(layers)
     _check(lib().adacomp_compress_multi(layers, int(n_layers), _stream(stream)),
            "adacomp_compress_multi")
+
+
+def adacomp_compress_multi_lazy(layers, states, n_layers: int, stream=None) -> None:
+    """adacomp_compress_multi in lazy-scale mode; states[t]: layer t's lazy state (uint8 CUDA tensors)."""
+    if not isinstance(layers, C.Array):
+        layers = make_layer_descs(layers)
+    if not isinstance(states, C.Array):
+        states = make_pointer_array(states, torch.uint8)
+    _check(lib().adacomp_compress_multi_lazy(layers, states, int(n_layers), _stream(stream)),
+           "adacomp_compress_multi_lazy")
 
 
 def make_pointer_array(tensors: Sequence[torch.Tensor], dtype):

@@ -16,9 +16,10 @@
 // adds the k learners' words into it in learner order and stores it once.
 //
 // HBM-bandwidth bound; no tensor cores (nothing here is a contraction).  The fast
-// tile pass (L_T = 50 and 500) is a persistent kernel fed by 1-D bulk copies (TMA)
-// through a three-stage shared-memory ring guarded by mbarriers; every wait on a
-// barrier is bounded and reports ADACOMP_DEV_TIMEOUT instead of spinning forever.
+// tile pass (every L_T from 41 to 1000, the paper's 50 and 500 among them) is a persistent
+// kernel fed by 1-D bulk copies (TMA) through a three-stage shared-memory ring guarded by
+// mbarriers, and so is the decoder (every L_T from 41 up) with its ring of slots; every wait
+// on a barrier is bounded and reports ADACOMP_DEV_TIMEOUT instead of spinning forever.
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -1234,6 +1235,7 @@ struct BatchLayer {
     Geometry geo;
     u32 tile_first;                                  // global index of the layer's first tile
     u32 pad;
+    unsigned char *lazy;                             // lazy-scale mode: the layer's state (else null)
 };
 
 // The table comes in two sizes: kernel parameters are copied at every launch, and a launch with the
@@ -1307,7 +1309,9 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
 // into the layer table; what depends on the layer's bin length (the place of a thread's 25 elements among
 // the bins) is recomputed when the cursor moves, and the CTA's share of a layer's exact g_max sum is added
 // to that layer's windows when the CTA leaves the layer.  Every layer here has 41 <= L_T <= 1000.
-template <int N>
+// LAZY: lazy-scale mode, every layer with its own state (see tile_pass_fast); a layer whose state is not its
+// own is flagged, left untouched and reports empty tiles.
+template <int N, bool LAZY>
 __global__ void __launch_bounds__(kFastThreads, 2)
 batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
 {
@@ -1329,6 +1333,10 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     auto seek = [&](u32 gt, int &li) {      // (tiles only go up)
         while (li + 1 < n_layers && b.layer[li + 1].tile_first <= gt) li++;
     };
+    auto state_ok = [&](const BatchLayer &L) {      // (LAZY) the state is this layer's
+        const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(L.lazy);
+        return lh->magic == kLazyMagic && lh->n == L.geo.n && lh->L_T == L.geo.L_T;
+    };
 
     if (tid < kWindows + 1) s_acc[tid] = 0;
     for (int i = tid; i < 4 * kSmallBins; i += kFastThreads) s_anymax[i] = 0;
@@ -1340,19 +1348,26 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     __syncthreads();
 
     u32 issued = 0;                     // service lane 0: loads issued for tiles [0, issued)
-    int load_li = 0;
+    int load_li = 0, load_checked = -1;
+    bool load_ok = true;
     auto issue_load = [&](u32 i) {
         if (i >= my_tiles) return;
         const u32 gt = first + i * stride;
         seek(gt, load_li);
         const BatchLayer &L = b.layer[load_li];
+        if (LAZY && load_li != load_checked) {
+            load_checked = load_li;
+            load_ok = state_ok(L);
+        }
+        if (LAZY && !load_ok) return;                   // nothing of such a layer is read
         const u32 lt = gt - L.tile_first, T = L.geo.tile_elems;
         if ((u64)lt >= L.geo.n / T) return;             // a ragged last tile is read with plain loads
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        mbar_arrive_expect_tx(bar, 8u * T);
+        mbar_arrive_expect_tx(bar, 8u * T + (LAZY ? kMaskBytes : 0u));
         bulk_load(st, L.grad + (u64)lt * T, 4u * T, bar);
         bulk_load(st + kTileBytes, L.residue + (u64)lt * T, 4u * T, bar);
+        if (LAZY) bulk_load(st + 2 * kTileBytes, L.lazy + kLazyHeaderBytes + (u64)lt * kMaskBytes, kMaskBytes, bar);
         issued = i + 1;
     };
     if (service && lane == 0) {
@@ -1364,6 +1379,9 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     u32 phase = 0;                      // bit s: parity of stage s's next completion (ragged tiles use no barrier)
     int T = 0, TB = 0, b0 = 0, cut = kSeg, off0 = 0, vcount = 0;
     u32 full_tiles = 0, wbytes = 1;
+    bool layer_ok = true;               // (LAZY) the layer's state is its own
+    u32 prev_scale_bits = 0;            // (LAZY) last step's scale of the layer
+    u32 *lazy_mask = nullptr;
     auto flush = [&]() {                // (service warp) this CTA's share of layer at_li's exact sum
         if (at_li >= 0 && lane < kWindows) {
             const u64 v = s_acc[lane];
@@ -1392,9 +1410,33 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             off0 = e0 - b0 * Lt;
             cut = min(kSeg, Lt - off0);
             vcount = max(0, min(kSeg, T - e0));
+            if (LAZY) {
+                layer_ok = state_ok(L);
+                if (layer_ok) {
+                    prev_scale_bits = __float_as_uint(reinterpret_cast<const LazyHeader *>(L.lazy)->scale) & 0x7fffffffu;
+                    lazy_mask = reinterpret_cast<u32 *>(L.lazy + kLazyHeaderBytes);
+                } else if (tid == 0) {
+                    raise_status(ADACOMP_DEV_HEADER_MISMATCH);
+                }
+            }
         }
         unsigned char *scratch = L.packed + geo.scratch_at;
         const u32 lt = gt - L.tile_first;
+        if (LAZY && !layer_ok) {
+            // the same hand-over as for a real tile, nothing read or computed: the tile counts as empty
+            __syncthreads();
+            if (tid < kSmallBins) {
+                s_anymax[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+                s_anycnt[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+            }
+            if (service && lane == 0) {
+                reinterpret_cast<u32 *>(scratch + geo.tile_cnt_at)[lt] = 0;
+                bulk_wait_read_all();
+                issue_load(i + 2);
+            }
+            __syncthreads();
+            continue;
+        }
         const u64 base = (u64)lt * (u64)T;
         float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
         float *s_r = s_d + kFastTile;
@@ -1417,6 +1459,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 s_d[e] = d;
                 s_r[e] = r;
             }
+            if (LAZY && tid < kTileSegs) reinterpret_cast<u32 *>(s_r + kFastTile)[tid] = lazy_mask[(u64)lt * kTileSegs + tid];
             __syncthreads();
         }
 
@@ -1428,10 +1471,17 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             const float *pd = s_d + tid * kSeg;
             const float *pr = s_r + tid * kSeg;
             float m = 0.f, m1 = 0.f;
+            const u32 prev = LAZY ? reinterpret_cast<const u32 *>(s_r + kFastTile)[tid] : 0u;
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
                 float d = pd[j], r = pr[j];
                 if (j >= vcount) d = r = 0.f;               // past the tile's end
+                if (LAZY) {
+                    // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
+                    const float q = __uint_as_float(prev_scale_bits | (__float_as_uint(r) & 0x80000000u));
+                    const float fixed = __fsub_rn(r, q);
+                    r = (prev >> j & 1u) ? fixed : r;
+                }
                 g[j] = __fadd_rn(r, d);
                 const float h = __fadd_rn(g[j], d);
                 if (j >= cut) m1 = fmaxf(m1, fabsf(g[j]));
@@ -1487,6 +1537,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 else reinterpret_cast<unsigned short *>(s_words)[at] = (unsigned short)word;
                 at++;
             }
+            if (LAZY) lazy_mask[(u64)lt * kTileSegs + tid] = selmask;
             if (tid < TB) {
                 const u64 bin = (u64)lt * (u64)TB + tid;
                 if (bin < geo.n_bins) {
@@ -1560,10 +1611,11 @@ __global__ void __launch_bounds__(1024)
 batch_finalize(const __grid_constant__ BatchArgsT<N> b)
 {
     const BatchLayer &L = b.layer[blockIdx.x];
-    finalize_body(L.packed, L.packed + L.geo.scratch_at, L.geo, 0u, L.count_out, nullptr);
+    finalize_body(L.packed, L.packed + L.geo.scratch_at, L.geo, 0u, L.count_out, L.lazy);
 }
 
-template <int N>
+// FIXUP: also finishes the sent elements' residues (eager mode; lazy-scale mode leaves G).
+template <int N, bool FIXUP>
 __global__ void __launch_bounds__(kGatherThreads)
 batch_gather(const __grid_constant__ BatchArgsT<N> b)
 {
@@ -1574,9 +1626,9 @@ batch_gather(const __grid_constant__ BatchArgsT<N> b)
         const BatchLayer &L = b.layer[batch_layer_of(b, gt)];
         const unsigned char *scratch = L.packed + L.geo.scratch_at;
         if (L.geo.w == 1u)
-            gather_tile_small<unsigned char, true>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
+            gather_tile_small<unsigned char, FIXUP>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
         else
-            gather_tile_small<unsigned short, true>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
+            gather_tile_small<unsigned short, FIXUP>(L.residue, L.packed, scratch, L.geo, gt - L.tile_first, lane, s_pre_all[warp]);
     }
 }
 
@@ -3254,8 +3306,10 @@ int device_info(DeviceInfo *&out)
             d.batch_per_sm = per;
         }
         d.batch_fast_ready = d.fast_ready &&
-                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax>, at, bytes) == cudaSuccess &&
-                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall>, at, bytes) == cudaSuccess;
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false>, at, bytes) == cudaSuccess &&
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false>, at, bytes) == cudaSuccess &&
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true>, at, bytes) == cudaSuccess &&
+                             cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true>, at, bytes) == cudaSuccess;
         if (cudaFuncSetAttribute(decode_batch, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sizeof(DecodeBatchSmem)) == cudaSuccess) {
             int per = 0;
@@ -3402,7 +3456,7 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     if (rc != ADACOMP_OK) return rc;
     u64 grid = (u64)info->sms * info->decode_per_sm, grid_w = (u64)info->sms * info->decode_warps_per_sm;
     u64 grid_one = (u64)info->sms * info->decode_one_per_sm;
-    bool warps = true, others = true;   // the shape is on the device: both kernels go, one of them returns at once
+    bool warps = true, others = true;   // the shape is on the device: every kernel goes, all but one return at once
     if (hint_L_T) {                     // the shape is known on the host: one kernel, no more CTAs than work items
         const Geometry hg = make_geometry(hint_n, hint_L_T);
         warps = warp_path(hg);
@@ -3440,15 +3494,17 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
+// lazy: lazy-scale mode (every layer carries its state; needs the pipelined batch tile pass).
 template <int N>
-int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStream_t st)
+int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStream_t st, bool lazy)
 {
     batch_clear<N><<<b.n_layers, 128, 0, st>>>(b);
     if (b.total_tiles) {
         if (info.batch_fast_ready) {
             const u64 cap = (u64)info.sms * 2;
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
-            batch_tile_pass_fast<N><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            if (lazy) batch_tile_pass_fast<N, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            else batch_tile_pass_fast<N, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
         } else {
             const u64 cap = (u64)info.sms * info.batch_per_sm;
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
@@ -3458,28 +3514,30 @@ int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStrea
     batch_finalize<N><<<b.n_layers, 1024, 0, st>>>(b);
     if (b.total_tiles) {
         const u64 want = ((u64)b.total_tiles + 3) / 4, cap = (u64)info.sms * 16;
-        batch_gather<N><<<(unsigned)(want < cap ? want : cap), kGatherThreads, 0, st>>>(b);
+        const unsigned grid = (unsigned)(want < cap ? want : cap);
+        if (lazy) batch_gather<N, false><<<grid, kGatherThreads, 0, st>>>(b);
+        else batch_gather<N, true><<<grid, kGatherThreads, 0, st>>>(b);
     }
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
 // Launches one batch (at most kBatchMax layers, all batchable) on the stream.
-int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st)
+int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st, bool lazy = false)
 {
     if (b.n_layers == 0) return ADACOMP_OK;
     if (b.n_layers == 1) {      // a batch of one gains nothing over the single-layer kernels
         const BatchLayer &L = b.layer[0];
         return compress_impl(L.grad, L.residue, L.geo.n, L.geo.L_T, L.packed, reinterpret_cast<uint64_t *>(L.count_out),
-                             st, 0);
+                             st, 0, nullptr, L.lazy);
     }
     if (b.n_layers <= (u32)kBatchSmall) {
         BatchArgsT<kBatchSmall> small;
         small.n_layers = b.n_layers;
         small.total_tiles = b.total_tiles;
         for (u32 i = 0; i < b.n_layers; i++) small.layer[i] = b.layer[i];
-        return launch_batch_sized(small, info, st);
+        return launch_batch_sized(small, info, st, lazy);
     }
-    return launch_batch_sized(b, info, st);
+    return launch_batch_sized(b, info, st, lazy);
 }
 
 inline bool batchable(const adacomp_layer_desc &d, const DeviceInfo &info)
@@ -3583,7 +3641,7 @@ const char *adacomp_strerror(int code)
     case ADACOMP_ERR_SIZE: return "tensor too large for this bin length";
     case ADACOMP_ERR_FLAGS: return "unknown flag bits";
     case ADACOMP_ERR_CUDA: return "a CUDA runtime call failed";
-    case ADACOMP_ERR_UNSUPPORTED: return "lazy mode supports L_T = 50 and 500 without flags only";
+    case ADACOMP_ERR_UNSUPPORTED: return "lazy mode supports L_T = 41..1000 (and multiples of 4 up to 4000) without flags only";
     case ADACOMP_ERR_STATIC_SCRATCH:
         return "tensor needs more scratch than the library's built-in array holds; use adacomp_compress";
     default: return "unknown error code";
@@ -3816,7 +3874,8 @@ int adacomp_decompress_accumulate_host(const void *const *packed_host, const uin
     return cudaStreamSynchronize(st) == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
-int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream)
+// `states` (optional): lazy-scale mode, states[t] the state of layer t.
+static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *states, uint32_t n_layers, void *stream)
 {
     if (n_layers && !layers) return ADACOMP_ERR_NULL;
     for (uint32_t t = 0; t < n_layers; t++) {
@@ -3825,6 +3884,11 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
         if (d.L_T == 0 || d.L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
         if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
         if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out)) return ADACOMP_ERR_ALIGN;
+        if (states) {
+            if (!states[t]) return ADACOMP_ERR_NULL;
+            if (misaligned(states[t])) return ADACOMP_ERR_ALIGN;
+            if (d.flags != 0 || !(fast_L_T(d.L_T) || any_fast_L_T(d.L_T))) return ADACOMP_ERR_UNSUPPORTED;
+        }
     }
     if (n_layers == 0) return ADACOMP_OK;
     DeviceInfo *info = nullptr;
@@ -3837,7 +3901,7 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
     batch.total_tiles = 0;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (info->batch_per_sm > 0 && batchable(d, *info)) {
+        if (info->batch_per_sm > 0 && batchable(d, *info) && (!states || info->batch_fast_ready)) {
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
@@ -3846,19 +3910,32 @@ int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, 
             L.geo = make_geometry(d.n, d.L_T);
             L.tile_first = batch.total_tiles;
             L.pad = 0;
+            L.lazy = states ? static_cast<unsigned char *>(states[t]) : nullptr;
             batch.total_tiles += (u32)L.geo.n_tiles;
             if (batch.n_layers == (u32)kBatchMax) {
-                rc = launch_batch(batch, *info, st);
+                rc = launch_batch(batch, *info, st, states != nullptr);
                 if (rc != ADACOMP_OK) return rc;
                 batch.n_layers = 0;
                 batch.total_tiles = 0;
             }
         } else {
-            rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags);
+            rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags, nullptr,
+                               states ? states[t] : nullptr);
             if (rc != ADACOMP_OK) return rc;
         }
     }
-    return launch_batch(batch, *info, st);
+    return launch_batch(batch, *info, st, states != nullptr);
+}
+
+int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream)
+{
+    return compress_multi_impl(layers, nullptr, n_layers, stream);
+}
+
+int adacomp_compress_multi_lazy(const adacomp_layer_desc *layers, void *const *states, uint32_t n_layers, void *stream)
+{
+    if (n_layers && !states) return ADACOMP_ERR_NULL;
+    return compress_multi_impl(layers, states, n_layers, stream);
 }
 
 int adacomp_decompress_accumulate_multi(const void *const *packed, uint32_t k_streams, float *const *dst,

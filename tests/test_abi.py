@@ -128,6 +128,8 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.adacomp_compress_multi(descs, 1, None) == -2
     assert lib.adacomp_compress_multi(None, 1, None) == -1
     assert lib.adacomp_compress_multi(None, 0, None) == 0
+    assert lib.adacomp_compress_multi_lazy(descs, None, 1, None) == -1
+    assert lib.adacomp_compress_multi_lazy(None, None, 0, None) == 0
 
 
 def test_binding_refuses_cpu_tensors():

@@ -111,3 +111,53 @@ def test_lazy_rejects_other_bin_lengths_and_foreign_state():
     assert B.adacomp_device_status() & B.ADACOMP_DEV_HEADER_MISMATCH
     assert torch.all(layer.residue == 1.0)
     B.adacomp_device_status_reset()
+
+
+def test_lazy_multi_matches_oracle_over_steps_and_flags_a_foreign_state():
+    """adacomp_compress_multi_lazy on a parameter list (layers and bin lengths change from tile to tile inside
+    one batch; one layer beyond the batch's size limit, one with one-bin tiles): every stream equals the
+    oracle's at every step, and after a flush every residue does.  Then one layer is given another layer's
+    state: flagged, left untouched, its stream empty, the others unaffected."""
+    specs = synth.resnet50_tensors()[:12] + [
+        synth.TensorSpec("lt64", 3840 * 5 + 77, 64, "conv"), synth.TensorSpec("lt333", 3996 * 3 + 5, 333, "fc"),
+        synth.TensorSpec("mid", (1 << 22) + 99, 500, "fc"), synth.TensorSpec("tiny", 17, 50, "conv"),
+        synth.TensorSpec("lt1000", 4000 * 6 + 999, 1000, "fc"), synth.TensorSpec("one_bin", 3000 * 9 + 1, 3000, "fc"),
+        synth.TensorSpec("alone", (1 << 25) + 3, 50, "conv")]
+    layers = [LazyLayer(s.n, s.L_T) for s in specs]
+    r_cpu = [np.zeros(s.n, np.float32) for s in specs]
+    descs = [dict(grad=L.grad, residue=L.residue, n=L.n, L_T=L.L_T, packed_out=L.packed, count_out=L.count)
+             for L in layers]
+    states = [L.state for L in layers]
+    for step in range(3):
+        wants = []
+        for t, s in enumerate(specs):
+            dW = synth.make_dw(3, step, t, 1, s.n, heavy=(t % 2 == 0))
+            layers[t].grad.copy_(torch.from_numpy(dW))
+            wants.append(cref.pack(dW, r_cpu[t], s.L_T))
+        B.adacomp_compress_multi_lazy(descs, states, len(descs))
+        torch.cuda.synchronize()
+        for t, L in enumerate(layers):
+            assert_stream_equal(L.packed[:int(L.count[1])].cpu().numpy(), wants[t], f"step {step} tensor {t} ({specs[t].name})")
+    for t, L in enumerate(layers):
+        assert_f32_bits_equal(L.flushed_residue(), r_cpu[t], f"flushed residue of tensor {t}")
+    assert B.adacomp_device_status() == 0
+
+    # layer 3 gets layer 4's state
+    before = [L.residue.clone() for L in layers]
+    swapped = list(states)
+    swapped[3] = states[4]
+    wants = []
+    for t, s in enumerate(specs):
+        dW = synth.make_dw(3, 7, t, 1, s.n, heavy=False)
+        layers[t].grad.copy_(torch.from_numpy(dW))
+        wants.append(None if t == 3 else cref.pack(dW, r_cpu[t], s.L_T))
+    B.adacomp_compress_multi_lazy(descs, swapped, len(descs))
+    torch.cuda.synchronize()
+    assert B.adacomp_device_status() & B.ADACOMP_DEV_HEADER_MISMATCH
+    B.adacomp_device_status_reset()
+    assert torch.equal(layers[3].residue, before[3])
+    assert int(layers[3].count[0]) == 0
+    for t, L in enumerate(layers):
+        if t != 3:
+            assert_stream_equal(L.packed[:int(L.count[1])].cpu().numpy(), wants[t], f"after the swap, tensor {t}")
+    assert B.adacomp_device_status() == 0
