@@ -3107,12 +3107,12 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
     for (int t = tid; t < (int)b.n_layers; t += kDecodeThreads) {
         const Geometry g = make_geometry(b.n[t], b.L_T[t]);
         bool ok = true;
-        for (u32 l = 0; l < b.k; l++) {
+        for (u32 l = 0; l < b.k; l++) {     // (no early exit: the k headers' loads go out together)
             const u32 *h = reinterpret_cast<const u32 *>(b.stream[t * b.k + l]);
             const u64 *h64 = reinterpret_cast<const u64 *>(h);
-            ok = ok && h[0] == kMagic && (h[1] & 0xffffu) == 1u && h[2] == g.L_T && h64[2] == g.n &&
-                 ((h[1] >> 16) & 0xffu) == g.w && h[3] == g.tile_bins && h64[3] == g.n_bins &&
-                 h64[4] == g.n_tiles && h64[5] <= g.n;
+            ok &= h[0] == kMagic && (h[1] & 0xffffu) == 1u && h[2] == g.L_T && h64[2] == g.n &&
+                  ((h[1] >> 16) & 0xffu) == g.w && h[3] == g.tile_bins && h64[3] == g.n_bins &&
+                  h64[4] == g.n_tiles && h64[5] <= g.n;
         }
         if (!ok) bad |= ADACOMP_DEV_HEADER_MISMATCH;
         sm.geo[t] = g;
