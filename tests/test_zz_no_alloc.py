@@ -40,7 +40,8 @@ def test_oversized_tensor_is_refused_on_the_host():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("L_T,n", [(50, 100352), (500, 2359296), (7, 30011), (5000, 123457)])
+@pytest.mark.parametrize("L_T,n", [(50, 100352), (500, 2359296), (7, 30011), (5000, 123457), (64, 3840 * 31 + 5), (333, 3996 * 9 + 1),
+                                   (200, 4000 * 12 + 150), (3000, 3000 * 17 + 2), (1001, 50001)])
 def test_static_scratch_matches_adacomp_compress_on_two_calls_in_a_row(L_T, n):
     dev = torch.device("cuda:0")
     rng = np.random.default_rng(L_T * 31 + n)
