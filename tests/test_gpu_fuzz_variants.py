@@ -78,3 +78,37 @@ def test_fuzz_fused_optimizer_steps():
         assert_f32_bits_equal(vd.cpu().numpy()[:n], want_v, "v " + what)
         assert_f32_bits_equal(wd.cpu().numpy()[:n], want_w, "w " + what)
     assert B.adacomp_device_status() == 0
+
+
+def test_fuzz_lazy_scale_pack():
+    """Lazy-scale pack() on random shapes over the bin lengths it takes (41..1000 and the multiples of 4 up to
+    4000): three carried steps equal the oracle's streams, a flush gives the oracle's residue, and the eager
+    entry point carries on from there."""
+    rng = np.random.default_rng(4242)
+    for case in range(24):
+        L_T = int(rng.integers(41, 1001)) if case % 3 else 4 * int(rng.integers(251, 1001))
+        n = int(rng.integers(1, 120000))
+        sigma = 10.0 ** rng.uniform(-4, 0)
+        r_cpu = rng.normal(0, sigma, n).astype(np.float32)
+        layer = GpuLayer(n, L_T, r_cpu)
+        state = torch.empty(B.adacomp_lazy_state_bytes(n, L_T), dtype=torch.uint8, device=DEV)
+        assert state.numel() > 0
+        B.adacomp_lazy_state_init(state, n, L_T)
+        for step in range(3):
+            g = rng.normal(0, sigma, n).astype(np.float32)
+            want = cref.pack(g, r_cpu, L_T)
+            layer.grad[:n].copy_(torch.from_numpy(g))
+            layer.packed.fill_(0xAB)
+            B.adacomp_compress_lazy(layer.grad, layer.residue, state, n, L_T, layer.packed, layer.count)
+            torch.cuda.synchronize()
+            assert_stream_equal(layer.packed[:int(layer.count[1])].cpu().numpy(), want, f"case {case} step {step} n={n} L_T={L_T}")
+        B.adacomp_residue_flush(layer.residue, state, n, L_T)
+        assert_f32_bits_equal(layer.residue_host(), r_cpu, f"flushed residue case {case} n={n} L_T={L_T}")
+        g = rng.normal(0, sigma, n).astype(np.float32)
+        want = cref.pack(g, r_cpu, L_T)
+        layer.grad[:n].copy_(torch.from_numpy(g))
+        B.adacomp_compress(layer.grad, layer.residue, n, L_T, layer.packed, layer.count)
+        torch.cuda.synchronize()
+        assert_stream_equal(layer.packed[:int(layer.count[1])].cpu().numpy(), want, f"eager after flush, case {case}")
+        assert_f32_bits_equal(layer.residue_host(), r_cpu, f"eager residue case {case}")
+    assert B.adacomp_device_status() == 0
