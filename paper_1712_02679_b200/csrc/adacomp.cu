@@ -3161,8 +3161,9 @@ decode_batch(const __grid_constant__ DecodeBatchArgs b)
 // per layer in shared memory; the slots are laid out once per launch, with the learners' word regions
 // sized from the batch-wide average bytes per tile (1.5 times it plus slack) and the room for the bin
 // counts from the largest count run among the layers; a learner's scale and word total come into the
-// slot with its directory entries.  Every layer here has 42 <= L_T <= 1000; the finished tiles go to
-// memory (no optimizer step on this path).
+// slot with its directory entries.  Every layer here has 42 <= L_T <= 1000.  OPT: 0 the finished tiles go
+// to dst; 1 (SGD) / 2 (Adam) they feed the optimizer step on the layer's weights instead (see Epilogue), the
+// warp reading and writing its share of the optimizer's arrays itself.
 // ---------------------------------------------------------------------------------
 struct BatchLayerCtx {
     u64 n, n_bins, bin_cnt_at, payload_at;
@@ -3185,6 +3186,7 @@ struct WarpBatchSmem {
     u32 count_room_max, bad;
 };
 
+template <int OPT>
 __global__ void __launch_bounds__(kDecodeLaunch, 4)
 decode_batch_warps(const __grid_constant__ DecodeBatchArgs b, u32 ring_bytes)
 {
@@ -3543,7 +3545,45 @@ decode_batch_warps(const __grid_constant__ DecodeBatchArgs b, u32 ring_bytes)
         if (failed) break;
 
         // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
-        if (whole) {
+        if (OPT != 0) {
+            // averageGradients() + updateWeights() on the warp's quarter; dst is the layer's weights
+            const Epilogue ep = {dst, b.aux[li], OPT == 2 ? b.aux2[li] : nullptr, b.lr, b.mu, b.beta2, b.eps, (float)k,
+                                 OPT == 2 ? 1u : 0u, (k & (k - 1u)) == 0u ? __frcp_rn((float)k) : 0.f};
+            if (whole) {
+                float4 *w4 = reinterpret_cast<float4 *>(ep.weights + out0), *v4 = reinterpret_cast<float4 *>(ep.momentum + out0);
+                float4 *u4 = OPT == 2 ? reinterpret_cast<float4 *>(ep.second + out0) : nullptr;
+                float4 *s4 = reinterpret_cast<float4 *>(my_acc);
+                for (int at = lane; at < (int)(quarter >> 2); at += 32) {
+                    float4 w = w4[at], v = v4[at];
+                    if (OPT == 2) {
+                        float4 u = u4[at];
+                        adam_step4(s4[at], w, v, u, ep);
+                        u4[at] = u;
+                    } else {
+                        sgd_step4(s4[at], w, v, ep);
+                    }
+                    s4[at] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    v4[at] = v;
+                    w4[at] = w;
+                }
+            } else {
+                for (u32 i = lane; i < quarter; i += 32) {
+                    if (i < len) {
+                        float w = ep.weights[out0 + i], v = ep.momentum[out0 + i];
+                        if (OPT == 2) {
+                            float u = ep.second[out0 + i];
+                            adam_step(my_acc[i], w, v, u, ep);
+                            ep.second[out0 + i] = u;
+                        } else {
+                            sgd_step(my_acc[i], w, v, ep);
+                        }
+                        ep.momentum[out0 + i] = v;
+                        ep.weights[out0 + i] = w;
+                    }
+                    my_acc[i] = 0.f;
+                }
+            }
+        } else if (whole) {
             fence_async_smem();                     // this lane's adds, for the copy engine
             __syncwarp();
             if (lane == 0) {
@@ -3663,7 +3703,7 @@ struct DeviceInfo {
     int batch_per_sm = 0;
     bool batch_fast_ready = false;      // the pipelined batch tile pass can be launched       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
-    int dec_batch_warps_per_sm[3] = {0, 0, 0};      // CTAs of the batched warp decoder per SM, by ring size
+    int dec_batch_warps_per_sm[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};      // CTAs of the batched warp decoder per SM, by optimizer form and ring size
     bool fast_ready = false;
 };
 
@@ -3733,13 +3773,18 @@ int device_info(DeviceInfo *&out)
             int per = 0;
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, decode_batch, kDecodeThreads, sizeof(DecodeBatchSmem));
             d.dec_batch_per_sm = per;
-            if (cudaFuncSetAttribute(decode_batch_warps, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kBatchRingBytes[2]) == cudaSuccess)
+            auto batch_warps_ready = [&](auto kernel, int o) {
+                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBatchRingBytes[2]) != cudaSuccess)
+                    return;
                 for (int i = 0; i < 3; i++) {
-                    per = 0;
-                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, decode_batch_warps, kDecodeLaunch, kBatchRingBytes[i]);
-                    d.dec_batch_warps_per_sm[i] = per;
+                    int q = 0;
+                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kernel, kDecodeLaunch, kBatchRingBytes[i]);
+                    d.dec_batch_warps_per_sm[o][i] = q;
                 }
+            };
+            batch_warps_ready(decode_batch_warps<0>, 0);
+            batch_warps_ready(decode_batch_warps<1>, 1);
+            batch_warps_ready(decode_batch_warps<2>, 2);
         }
         d.sms = sms;
     }
@@ -4144,17 +4189,20 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
     batch.beta2 = opt ? opt->beta2 : 0.f;
     batch.eps = opt ? opt->eps : 0.f;
     u64 batch_tiles = 0;
-    // (plain decode-sum takes the batched warp decoder, and with it layers of up to 2^25 elements; the forms
-    // with an optimizer step keep the staged one)
-    const bool warps_batch = !opt && info->dec_batch_warps_per_sm[0] > 0 && info->dec_batch_warps_per_sm[2] > 0;
-    const u64 batch_max_elems = warps_batch ? kPackBatchMaxElems : kBatchLayerMaxElems;
+    // (the batched warp decoder, and with it layers of up to 2^25 elements for plain decode-sum; with an
+    // optimizer step larger layers keep the single-tensor kernels, which stage the optimizer's arrays by bulk copies)
+    const int opt_form = !opt ? 0 : opt->adam ? 2 : 1;
+    const bool warps_batch = info->dec_batch_warps_per_sm[opt_form][0] > 0 && info->dec_batch_warps_per_sm[opt_form][1] > 0;
+    const u64 batch_max_elems = warps_batch && !opt ? kPackBatchMaxElems : kBatchLayerMaxElems;
     auto flush = [&]() -> int {
         if (batch.n_layers == 0) return ADACOMP_OK;
         if (warps_batch) {
             const u32 ring = batch_ring_bytes(k_streams);
-            const u64 cap = (u64)info->sms * info->dec_batch_warps_per_sm[ring == kBatchRingBytes[0] ? 0 : ring == kBatchRingBytes[1] ? 1 : 2];
+            const u64 cap = (u64)info->sms * info->dec_batch_warps_per_sm[batch.opt][ring == kBatchRingBytes[0] ? 0 : ring == kBatchRingBytes[1] ? 1 : 2];
             const unsigned grid = (unsigned)(batch_tiles < cap ? (batch_tiles ? batch_tiles : 1) : cap);
-            decode_batch_warps<<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
+            if (batch.opt == 2u) decode_batch_warps<2><<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
+            else if (batch.opt == 1u) decode_batch_warps<1><<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
+            else decode_batch_warps<0><<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
         } else {
             const u64 cap = (u64)info->sms * info->dec_batch_per_sm;
             const unsigned grid = (unsigned)(batch_tiles < cap ? (batch_tiles ? batch_tiles : 1) : cap);

@@ -51,7 +51,8 @@ def test_fused_adam_matches_oracle_over_two_steps(L_T, n, k):
 
 def test_layer_list_in_one_call():
     rng = np.random.default_rng(8)
-    shapes = [(864, 500), (5120, 50), (4000 * 1100 + 7, 50), (147456, 500), (67, 500), (100, 7)]
+    shapes = [(864, 500), (5120, 50), (4000 * 1100 + 7, 50), (147456, 500), (67, 500), (100, 7), (3996 * 3 + 5, 333),
+              (3840 * 2 + 7, 64)]
     k = 3
     streams_cpu, bufs, st, dv = [], [], [], []
     for n, L_T in shapes:

@@ -93,7 +93,7 @@ def test_layer_list_in_one_call_matches_per_layer_oracle():
     """Small layers share a batched launch, the large ones take the single-layer kernels; bin lengths mixed."""
     rng = np.random.default_rng(6)
     shapes = [(864, 500), (9216, 500), (5120, 50), (4000 * 1100 + 7, 50), (147456, 500), (67, 500), (2048, 50),
-              (4000 * 1060, 500), (100, 7)]
+              (4000 * 1060, 500), (100, 7), (3996 * 3 + 5, 333), (3840 * 2 + 7, 64), (4000 * 2 + 999, 1000)]
     k = 3
     dev = torch.device("cuda:0")
     streams_cpu, bufs, ws, vs, w_dev, v_dev = [], [], [], [], [], []
