@@ -1994,16 +1994,6 @@ __device__ void decode_item_staged(const unsigned char *const *streams, u32 k, c
     consumer_barrier();
 }
 
-template <typename Word, bool BY_BIN>
-__device__ void decode_staged(const DecodeArgs &a, const Geometry &geo, DecodeSmem &sm)
-{
-    for (int i = threadIdx.x; i < kDecodeChunk; i += kDecodeThreads) sm.acc[i] = 0.f;
-    u32 bad = 0;
-    for (u64 tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x)
-        decode_item_staged<Word, BY_BIN>(a.stream, a.k, geo, tile, a.dst, a.ep, sm, bad);
-    if (bad) raise_status(bad);
-}
-
 // ---------------------------------------------------------------------------------
 // decode, warp path: every L_T above 40.  A work item is a tile of 4..96 bins (L_T <= 1000) or,
 // where a tile is one bin (L_T > 1000), 4096 consecutive output elements and the 1 to 6 bins
@@ -3055,16 +3045,9 @@ decode_sum(DecodeArgs a)
     if (!decode_headers(a, &s_bad, sm.scale, sm.n_sel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
     if (warp_path(geo)) return;
-    const bool by_bin = geo.tile_bins >= 32 && geo.tile_bins <= (u32)kSmallBins;
-    const bool by_word = geo.tile_bins >= 2 && geo.tile_bins <= 31;
-    if (geo.w == 1u) {
-        if (by_bin) decode_staged<unsigned char, true>(a, geo, sm);
-        else decode_generic<unsigned char>(a, geo, sm);
-    } else {
-        if (by_bin) decode_staged<unsigned short, true>(a, geo, sm);
-        else if (by_word) decode_staged<unsigned short, false>(a, geo, sm);
-        else decode_generic<unsigned short>(a, geo, sm);
-    }
+    // (what is left: tiles of 100 bins and more, L_T <= 40; and tensors beyond the warp path's 2^40 elements)
+    if (geo.w == 1u) decode_generic<unsigned char>(a, geo, sm);
+    else decode_generic<unsigned short>(a, geo, sm);
 }
 
 // ---------------------------------------------------------------------------------
