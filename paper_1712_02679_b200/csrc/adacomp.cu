@@ -311,6 +311,9 @@ __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shar
 // finished reading shared memory.
 // ---------------------------------------------------------------------------------
 
+struct TrueType { static constexpr bool value = true; };
+struct FalseType { static constexpr bool value = false; };
+
 struct PassArgs {
     const float *grad;
     float *residue;
@@ -1379,6 +1382,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     u32 phase = 0;                      // bit s: parity of stage s's next completion (ragged tiles use no barrier)
     int T = 0, TB = 0, b0 = 0, cut = kSeg, off0 = 0, vcount = 0;
     u32 full_tiles = 0, wbytes = 1;
+    bool aligned = false;               // every segment of the layer's tiles lies in one bin and exists whole
     bool layer_ok = true;               // (LAZY) the layer's state is its own
     u32 prev_scale_bits = 0;            // (LAZY) last step's scale of the layer
     u32 *lazy_mask = nullptr;
@@ -1410,6 +1414,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             off0 = e0 - b0 * Lt;
             cut = min(kSeg, Lt - off0);
             vcount = max(0, min(kSeg, T - e0));
+            aligned = T == kFastTile && Lt % kSeg == 0;     // (then cut = vcount = 25 in every thread)
             if (LAZY) {
                 layer_ok = state_ok(L);
                 if (layer_ok) {
@@ -1472,22 +1477,30 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             const float *pr = s_r + tid * kSeg;
             float m = 0.f, m1 = 0.f;
             const u32 prev = LAZY ? reinterpret_cast<const u32 *>(s_r + kFastTile)[tid] : 0u;
+            // (the loop twice: where the segments line up with the bins, as in the lists' bin lengths 50 and
+            // 500, the tests on `vcount` and `cut` fold away)
+            auto form = [&](auto lined_up) {
+                constexpr bool AL = decltype(lined_up)::value;
+                const int vc = AL ? kSeg : vcount, ct = AL ? kSeg : cut;
 #pragma unroll
-            for (int j = 0; j < kSeg; j++) {
-                float d = pd[j], r = pr[j];
-                if (j >= vcount) d = r = 0.f;               // past the tile's end
-                if (LAZY) {
-                    // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
-                    const float q = __uint_as_float(prev_scale_bits | (__float_as_uint(r) & 0x80000000u));
-                    const float fixed = __fsub_rn(r, q);
-                    r = (prev >> j & 1u) ? fixed : r;
+                for (int j = 0; j < kSeg; j++) {
+                    float d = pd[j], r = pr[j];
+                    if (j >= vc) d = r = 0.f;               // past the tile's end
+                    if (LAZY) {
+                        // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
+                        const float q = __uint_as_float(prev_scale_bits | (__float_as_uint(r) & 0x80000000u));
+                        const float fixed = __fsub_rn(r, q);
+                        r = (prev >> j & 1u) ? fixed : r;
+                    }
+                    g[j] = __fadd_rn(r, d);
+                    const float h = __fadd_rn(g[j], d);
+                    if (j >= ct) m1 = fmaxf(m1, fabsf(g[j]));
+                    else m = fmaxf(m, fabsf(g[j]));
+                    key[j] = fmaxf(fabsf(h), fabsf(g[j]));
                 }
-                g[j] = __fadd_rn(r, d);
-                const float h = __fadd_rn(g[j], d);
-                if (j >= cut) m1 = fmaxf(m1, fabsf(g[j]));
-                else m = fmaxf(m, fabsf(g[j]));
-                key[j] = fmaxf(fabsf(h), fabsf(g[j]));
-            }
+            };
+            if (aligned) form(TrueType{});
+            else form(FalseType{});
             // (non-negative floats order like their bits)
             if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
             if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
@@ -1502,9 +1515,15 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
             gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
             // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
+            if (aligned) {
 #pragma unroll
-            for (int j = 0; j < kSeg; j++)
-                if (key[j] >= (j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
+                for (int j = 0; j < kSeg; j++)
+                    if (key[j] >= gm && g[j] != 0.f) selmask |= 1u << j;
+            } else {
+#pragma unroll
+                for (int j = 0; j < kSeg; j++)
+                    if (key[j] >= (j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
+            }
             cnt = __popc(selmask);
             const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
             if (c0) atomicAdd(&any_cnt[b0], c0);
