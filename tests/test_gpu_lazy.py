@@ -161,3 +161,26 @@ def test_lazy_multi_matches_oracle_over_steps_and_flags_a_foreign_state():
         if t != 3:
             assert_stream_equal(L.packed[:int(L.count[1])].cpu().numpy(), wants[t], f"after the swap, tensor {t}")
     assert B.adacomp_device_status() == 0
+
+
+def test_lazy_multi_with_a_single_layer_is_the_single_tensor_call():
+    n, L_T = 4000 * 9 + 41, 50
+    rng = np.random.default_rng(31)
+    r_cpu = np.zeros(n, np.float32)
+    layer = LazyLayer(n, L_T)
+    desc = [dict(grad=layer.grad, residue=layer.residue, n=n, L_T=L_T, packed_out=layer.packed, count_out=layer.count)]
+    for step in range(3):
+        dW = rng.normal(0, 1e-3, n).astype(np.float32)
+        want = cref.pack(dW, r_cpu, L_T)
+        layer.grad.copy_(torch.from_numpy(dW))
+        B.adacomp_compress_multi_lazy(desc, [layer.state], 1)
+        torch.cuda.synchronize()
+        assert_stream_equal(layer.packed[:int(layer.count[1])].cpu().numpy(), want, f"step {step}")
+    assert_f32_bits_equal(layer.flushed_residue(), r_cpu)
+    # a bin length the lazy mode does not take: refused on the host, nothing launched
+    other = LazyLayer(n, 50)
+    bad = [dict(grad=other.grad, residue=other.residue, n=n, L_T=40, packed_out=other.packed, count_out=other.count)]
+    with pytest.raises(B.AdaCompError) as e:
+        B.adacomp_compress_multi_lazy(bad, [other.state], 1)
+    assert e.value.code == -9
+    assert B.adacomp_device_status() == 0
