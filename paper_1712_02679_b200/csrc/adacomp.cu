@@ -3656,9 +3656,10 @@ lazy_flush_kernel(float *residue, unsigned char *state, u64 n, u32 L_T, u32 tile
 // host side
 // ---------------------------------------------------------------------------------
 
-// The batched warp decoder's ring of slots: deeper for more learners, so that a few tiles stay in flight.
-constexpr u32 kBatchRingBytes[3] = {19200u, 38400u, 57600u};
-inline u32 batch_ring_bytes(u32 k) { return kBatchRingBytes[k <= 4u ? 0 : k <= 8u ? 1 : 0]; }
+// The batched warp decoder's ring of slots (dynamic shared memory).  Deeper rings for more learners were
+// measured: they cost a CTA per SM and the decode of a list is bound by the warps' fixed work per learner and
+// tile, so more warps beat more tiles in flight (8 learners: 0.20 ms with this ring, 0.21 ms with twice it).
+constexpr u32 kBatchRingBytes = 19200u;
 
 // The fast tile pass takes L_T = 25 * SPB for the divisors SPB of 40 but 1 (tiles of exactly 4000 elements):
 // 50, 100, 125, 200, 250, 500 and 1000.
@@ -3705,7 +3706,7 @@ struct DeviceInfo {
     int batch_per_sm = 0;
     bool batch_fast_ready = false;      // the pipelined batch tile pass can be launched       // 0: batched pack() unavailable on this device
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
-    int dec_batch_warps_per_sm[3][3] = {{0, 0, 0}, {0, 0, 0}, {0, 0, 0}};      // CTAs of the batched warp decoder per SM, by optimizer form and ring size
+    int dec_batch_warps_per_sm[3] = {0, 0, 0};      // CTAs of the batched warp decoder per SM, by optimizer form
     bool fast_ready = false;
 };
 
@@ -3776,13 +3777,9 @@ int device_info(DeviceInfo *&out)
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, decode_batch, kDecodeThreads, sizeof(DecodeBatchSmem));
             d.dec_batch_per_sm = per;
             auto batch_warps_ready = [&](auto kernel, int o) {
-                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBatchRingBytes[2]) != cudaSuccess)
-                    return;
-                for (int i = 0; i < 3; i++) {
-                    int q = 0;
-                    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kernel, kDecodeLaunch, kBatchRingBytes[i]);
-                    d.dec_batch_warps_per_sm[o][i] = q;
-                }
+                int q = 0;
+                cudaOccupancyMaxActiveBlocksPerMultiprocessor(&q, kernel, kDecodeLaunch, kBatchRingBytes);
+                d.dec_batch_warps_per_sm[o] = q;
             };
             batch_warps_ready(decode_batch_warps<0>, 0);
             batch_warps_ready(decode_batch_warps<1>, 1);
@@ -4194,13 +4191,13 @@ int decompress_multi_impl(const void *const *packed, uint32_t k_streams, float *
     // (the batched warp decoder, and with it layers of up to 2^25 elements for plain decode-sum; with an
     // optimizer step larger layers keep the single-tensor kernels, which stage the optimizer's arrays by bulk copies)
     const int opt_form = !opt ? 0 : opt->adam ? 2 : 1;
-    const bool warps_batch = info->dec_batch_warps_per_sm[opt_form][0] > 0 && info->dec_batch_warps_per_sm[opt_form][1] > 0;
+    const bool warps_batch = info->dec_batch_warps_per_sm[opt_form] > 0;
     const u64 batch_max_elems = warps_batch && !opt ? kPackBatchMaxElems : kBatchLayerMaxElems;
     auto flush = [&]() -> int {
         if (batch.n_layers == 0) return ADACOMP_OK;
         if (warps_batch) {
-            const u32 ring = batch_ring_bytes(k_streams);
-            const u64 cap = (u64)info->sms * info->dec_batch_warps_per_sm[batch.opt][ring == kBatchRingBytes[0] ? 0 : ring == kBatchRingBytes[1] ? 1 : 2];
+            const u32 ring = kBatchRingBytes;
+            const u64 cap = (u64)info->sms * info->dec_batch_warps_per_sm[batch.opt];
             const unsigned grid = (unsigned)(batch_tiles < cap ? (batch_tiles ? batch_tiles : 1) : cap);
             if (batch.opt == 2u) decode_batch_warps<2><<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
             else if (batch.opt == 1u) decode_batch_warps<1><<<grid, kDecodeLaunch, ring, st>>>(batch, ring);
