@@ -3076,7 +3076,7 @@ decode_sum(DecodeArgs a)
 // 42 <= L_T <= 1000 qualify (tiles of at most 4096 elements and 2..96 bins).
 // ---------------------------------------------------------------------------------
 
-constexpr int kDecBatchLayers = 96;
+constexpr int kDecBatchLayers = 192;
 constexpr int kDecBatchPtrs = 2900;
 
 struct DecodeBatchArgs {
