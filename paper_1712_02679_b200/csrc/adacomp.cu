@@ -1222,7 +1222,7 @@ gather_fixup(float *residue, unsigned char *packed, const unsigned char *scratch
 // Layers of 42 <= L_T <= 1000 (tiles of at most 4000 elements and 96 bins) qualify.
 // ---------------------------------------------------------------------------------
 
-constexpr int kBatchMax = 160;                       // layers per batched launch (parameter space: 32 KB)
+constexpr int kBatchMax = 184;                       // layers per batched launch (the table is 32392 of the 32764 bytes of kernel parameters)
 constexpr u64 kBatchLayerMaxElems = 1ull << 22;      // decode: larger layers take the single-layer kernels
 // pack(): layers up to this size share a batch's launches when the pipelined batch tile pass is there (a
 // layer alone ramps its pipeline up and down over a few tiles per CTA and pays four launches and a finalize
