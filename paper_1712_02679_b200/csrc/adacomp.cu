@@ -4382,9 +4382,17 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
     static thread_local BatchArgs batch;
     batch.n_layers = 0;
     batch.total_tiles = 0;
+    auto batched = [&](const adacomp_layer_desc &d) {
+        return info->batch_per_sm > 0 && batchable(d, *info) && (!states || info->batch_fast_ready);
+    };
+    // (more layers than a table holds: batches of equal size, so that none is left with a layer or two)
+    uint32_t to_batch = 0;
+    for (uint32_t t = 0; t < n_layers; t++) to_batch += batched(layers[t]) ? 1u : 0u;
+    const uint32_t n_batches = (to_batch + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
+    const uint32_t per_batch = n_batches ? (to_batch + n_batches - 1) / n_batches : (uint32_t)kBatchMax;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (info->batch_per_sm > 0 && batchable(d, *info) && (!states || info->batch_fast_ready)) {
+        if (batched(d)) {
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
@@ -4395,7 +4403,7 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
             L.pad = 0;
             L.lazy = states ? static_cast<unsigned char *>(states[t]) : nullptr;
             batch.total_tiles += (u32)L.geo.n_tiles;
-            if (batch.n_layers == (u32)kBatchMax) {
+            if (batch.n_layers == per_batch) {
                 rc = launch_batch(batch, *info, st, states != nullptr);
                 if (rc != ADACOMP_OK) return rc;
                 batch.n_layers = 0;

@@ -404,6 +404,38 @@ def test_multi_tensor_calls_match_single_calls():
         assert_f32_bits_equal(dsts[t][:L.n].cpu().numpy(), cref.unpack_sum([raw, raw], L.n))
 
 
+def test_multi_tensor_calls_with_more_layers_than_one_batch_holds():
+    """200 small layers: two pack batches of 100 and two decode launches; every stream and sum equals the oracle's."""
+    rng = np.random.default_rng(200)
+    dev = torch.device("cuda:0")
+    shapes = [(int(rng.integers(1, 9000)), int(rng.choice([50, 500, 64, 333]))) for _ in range(200)]
+    layers, dws = [], []
+    for n, L_T in shapes:
+        L = GpuLayer(n, L_T)
+        dW = rng.normal(0, 1e-3, n).astype(np.float32)
+        L.grad[:n].copy_(torch.from_numpy(dW))
+        layers.append(L)
+        dws.append(dW)
+    descs = [dict(grad=L.grad, residue=L.residue, n=L.n, L_T=L.L_T, packed_out=L.packed, count_out=L.count) for L in layers]
+    B.adacomp_compress_multi(descs, len(descs))
+    torch.cuda.synchronize()
+    raws = []
+    for t, (L, (n, L_T)) in enumerate(zip(layers, shapes)):
+        r = np.zeros(n, np.float32)
+        want = cref.pack(dws[t], r, L_T)
+        raw = L.packed[:int(L.count[1])].cpu().numpy()
+        assert_stream_equal(raw, want, f"tensor {t} n={n} L_T={L_T}")
+        assert_f32_bits_equal(L.residue_host(), r, f"residue {t}")
+        raws.append(raw)
+    dsts = [torch.empty(max(L.n, 4), dtype=torch.float32, device=dev) for L in layers]
+    packed = [p for L in layers for p in (L.packed, L.packed)]
+    B.adacomp_decompress_accumulate_multi_ex(packed, 2, dsts, [n for n, _ in shapes], [l for _, l in shapes], len(layers))
+    torch.cuda.synchronize()
+    for t, L in enumerate(layers):
+        assert_f32_bits_equal(dsts[t][:L.n].cpu().numpy(), cref.unpack_sum([raws[t], raws[t]], L.n), f"sum {t}")
+    assert B.adacomp_device_status() == 0
+
+
 def test_random_shapes_against_the_oracle():
     """Seeded fuzz over (n, L_T, k): two carried pack() steps per learner and one dense sum."""
     rng = np.random.default_rng(20261125)
