@@ -1719,6 +1719,7 @@ struct DecodeArgs {
     Epilogue ep;
     float *dst;
     u32 k;
+    u32 pairs;          // the kernel of pair_path() is launched too: its shapes are left to it
     u32 hint_L_T;       // 0: the caller did not say; else the streams must carry exactly this shape
     u64 hint_n;
 };
@@ -1744,10 +1745,15 @@ constexpr int kWarpsPerSm = ADACOMP_WARPS_PER_SM;    // CTAs of the warp decoder
 constexpr int kSlots = 8;                       // tiles in flight per CTA at most
 constexpr u32 kRingBytes = 19200;
 constexpr u32 kSlotMax = kRingBytes / 2;        // a slot never takes more: two tiles are always in flight
+// (five decoding warps: the kernel of the pairs of tiles, whose items are twice as large; what four CTAs per SM leave)
+#ifndef ADACOMP_PAIR_RING
+#define ADACOMP_PAIR_RING 21504
+#endif
+__host__ __device__ constexpr u32 ring_bytes(int nw) { return nw == 5 ? (u32)ADACOMP_PAIR_RING : kRingBytes; }
 
 template <int NW>
 struct WarpDecSmem {
-    uint4 ring[kRingBytes / 16];
+    uint4 ring[ring_bytes(NW) / 16];
     u32 tmp[NW][32];                            // per decoding warp: output places of its non-empty bins
     unsigned short coff[ADACOMP_MAX_STREAMS];   // byte offset in a slot of learner l's bin counts (its words follow them)
     unsigned short wcap[ADACOMP_MAX_STREAMS];   // bytes of its word region
@@ -2036,7 +2042,11 @@ __device__ void decode_item_staged(const unsigned char *const *streams, u32 k, c
 // contributions in learner order), gives the slot back, hands its quarter to one bulk copy
 // (TMA store: the output does not pass through the warps' load/store path, which the adds keep
 // busy) and zeroes it once the copy has read it.
-// Three schemes for the adds.  Items of 4096 elements (L_T > 1000): a warp owns a quarter of the
+// Tiles of 80 bins of 8-bit words (L_T = 48, 49, 50; tensors of 256 tiles and more) are taken in pairs by a
+// kernel of its own with five decoding warps: an item is then 160 bins, 32 per warp (see pair_path()).
+// Four schemes for the adds.  Where a warp's share of the item is a multiple of 4 and at most 32 bins of
+// 8-bit words (the pairs; the 80- and 96-bin tiles in the kernels with an optimizer step): a lane per
+// bin, see warp_add_lanes_all().  Items of 4096 elements (L_T > 1000): a warp owns a quarter of the
 // elements whatever the bins are, reads the words of the bins its elements lie in and adds those
 // that are its own.  Tiles of at most 64 bins (16-bit words among them): G lanes share a
 // bin and take every G-th word of it.  Tiles of more bins (8-bit words, L_T <= 58): the warp works
@@ -2127,10 +2137,21 @@ __device__ inline void warp_bins(CountsFn counts, int R, int b0, int nb, u32 liv
             const auto at = counts(q);
             u32 cq = 0, bq = 0;
             if (have) cq = min(load_word<Word, SHARED>(at + mb * (u32)sizeof(Word)), L_T);
+            if (SHARED && sizeof(Word) == 1 && ((((u32)at) | (u32)b0) & 3u) == 0u && (u32)b0 <= live) {
+                // four 8-bit counts per load (the counts' run and the warp's first bin are 4-byte aligned);
+                // a count beyond L_T (a malformed stream) is clamped like the others: bytes are compared pairwise
+                if ((u32)lane < ((u32)b0 >> 2)) {
+                    u32 x;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x) : "r"((u32)at + 4u * (u32)lane) : "memory");
+                    x = __vminu4(x, L_T * 0x01010101u);
+                    bq = __dp4a(x, 0x01010101u, 0u);
+                }
+            } else {
 #pragma unroll
-            for (int r = 0; r < 3; r++) {           // bins before b0: at most 72
-                const u32 b = (u32)lane + 32u * r;
-                if (b < (u32)b0 && b < live) bq += min(load_word<Word, SHARED>(at + b * (u32)sizeof(Word)), L_T);
+                for (int r = 0; r < 4; r++) {       // bins before b0: at most 128
+                    const u32 b = (u32)lane + 32u * r;
+                    if (b < (u32)b0 && b < live) bq += min(load_word<Word, SHARED>(at + b * (u32)sizeof(Word)), L_T);
+                }
             }
             wb.mine[q >> 1] |= cq << (16 * (q & 1));
             bef[q >> 1] += bq << (16 * (q & 1));
@@ -2165,7 +2186,7 @@ __device__ inline u32 warp_add_words(Addr words, u32 W, u32 c, u32 excl, int nb,
     const u32 LT4 = L_T * 4u;
     u32 place = acc_at + (u32)lane * LT4;
     const u32 ne = __ballot_sync(full, c != 0u);
-    if (ne != (1u << nb) - 1u) {                    // (nb <= 24)
+    if (ne & (ne + 1u)) {                           // (the non-empty bins are not the warp's first ones in a row)
         __syncwarp();
         if (c != 0u) tmp[__popc(ne & ((1u << lane) - 1u))] = place;
         __syncwarp();
@@ -2222,6 +2243,141 @@ __device__ inline u32 warp_add_group(const GroupSrc<Addr> &src, int R, int b0, i
         }
         __syncwarp();                               // learner order, element by element
     }
+    return bad;
+}
+
+// out[e] += v (as add_at_if_valid) when `go` is not zero; nothing is read or written otherwise.
+__device__ inline void add_at_if(u32 e, float v, u32 go)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .f32 x;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "@p ld.shared.f32 x, [%0];\n\t"
+        "@p add.rn.f32 x, x, %1;\n\t"
+        "@p st.shared.f32 [%0], x;\n\t}"
+        ::"r"(e), "f"(v), "r"(go)
+        : "memory");
+}
+
+// Four 8-bit words of one bin (distinct indices; the no-op word 0 where there is none) added to the bin whose
+// first element is at shared-memory address `bin_at`: byte b carries idx << 2 | code, the element is at
+// bin_at + 4 idx = bin_at + (b & 0xfc), and the value is sb + (b << 30) as a bit pattern: sb is the scale's
+// pattern minus 0x40000000, so code 01 gives +scale and code 11 -scale.  Loads first, stores last.
+__device__ inline void add4_words(u32 bin_at, u32 w4, u32 sb)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, p2, p3;\n\t.reg .f32 x0, x1, x2, x3;\n\t.reg .b32 t, a4, e0, e1, e2, e3, v0, v1, v2, v3;\n\t"
+        "and.b32 t, %1, 0x00000001;\n\tsetp.ne.u32 p0, t, 0;\n\t"
+        "and.b32 t, %1, 0x00000100;\n\tsetp.ne.u32 p1, t, 0;\n\t"
+        "and.b32 t, %1, 0x00010000;\n\tsetp.ne.u32 p2, t, 0;\n\t"
+        "and.b32 t, %1, 0x01000000;\n\tsetp.ne.u32 p3, t, 0;\n\t"
+        "and.b32 a4, %1, 0xfcfcfcfc;\n\t"
+        "prmt.b32 e0, a4, 0, 0x4440;\n\tadd.u32 e0, e0, %0;\n\t"
+        "prmt.b32 e1, a4, 0, 0x4441;\n\tadd.u32 e1, e1, %0;\n\t"
+        "prmt.b32 e2, a4, 0, 0x4442;\n\tadd.u32 e2, e2, %0;\n\t"
+        "prmt.b32 e3, a4, 0, 0x4443;\n\tadd.u32 e3, e3, %0;\n\t"
+        "mad.lo.u32 v0, %1, 0x40000000, %2;\n\t"
+        "and.b32 t, %1, 0x00000300;\n\tmad.lo.u32 v1, t, 0x00400000, %2;\n\t"
+        "and.b32 t, %1, 0x00030000;\n\tmad.lo.u32 v2, t, 0x00004000, %2;\n\t"
+        "and.b32 t, %1, 0x03000000;\n\tmad.lo.u32 v3, t, 0x00000040, %2;\n\t"
+        "@p0 ld.shared.f32 x0, [e0];\n\t"
+        "@p1 ld.shared.f32 x1, [e1];\n\t"
+        "@p2 ld.shared.f32 x2, [e2];\n\t"
+        "@p3 ld.shared.f32 x3, [e3];\n\t"
+        "{\n\t.reg .f32 f0, f1, f2, f3;\n\t"
+        "mov.b32 f0, v0;\n\tmov.b32 f1, v1;\n\tmov.b32 f2, v2;\n\tmov.b32 f3, v3;\n\t"
+        "@p0 add.rn.f32 x0, x0, f0;\n\t"
+        "@p1 add.rn.f32 x1, x1, f1;\n\t"
+        "@p2 add.rn.f32 x2, x2, f2;\n\t"
+        "@p3 add.rn.f32 x3, x3, f3;\n\t}\n\t"
+        "@p0 st.shared.f32 [e0], x0;\n\t"
+        "@p1 st.shared.f32 [e1], x1;\n\t"
+        "@p2 st.shared.f32 [e2], x2;\n\t"
+        "@p3 st.shared.f32 [e3], x3;\n\t}"
+        ::"r"(bin_at), "r"(w4), "r"(sb)
+        : "memory");
+}
+
+// All the learners staged in a slot, a lane per bin, for the shapes whose bin counts line up with 32-bit
+// loads: 8-bit counts whose run in the slot starts on a 16-byte boundary (the item's bins times one byte is a
+// multiple of 16), nb a multiple of 4 and at most 32, and all nb bins of the warp inside the tensor.
+// Lane t owns bin b0 + t of the item for every learner, so one thread adds all contributions to an
+// element, in learner order, and no look-up from word to bin is needed.
+// Per learner: lane i < nb / 4 loads the warp's counts 4 i .. 4 i + 3 as one word: a dot product gives
+// their total, a scan over nb / 4 lanes the words ahead of each four, and one multiplication the running
+// sums inside a four (bytes: a well-formed count is at most 64); the lanes below b0 / 4 sum the bins ahead of
+// the warp's the same way.  Then every lane reads its bin's words four at a time (two aligned 32-bit
+// loads and a funnel shift), turns the bytes past its count into the no-op word 0, skips (and reports) the
+// malformed ones, and adds the others: four loads, four additions, four stores, the elements being distinct.
+// Counts are not clamped to L_T: a count beyond it belongs to a stream that is flagged for its sums or
+// whose words are skipped one by one, and every read it leads to stays inside the CTA's shared memory.
+__device__ inline u32 warp_add_lanes_all(u32 sl_at, const unsigned short *coff, const unsigned short *m_cnt,
+                                         const unsigned short *m_head, const float *s_scale, u32 l0, u32 staged,
+                                         u32 count_bytes, int b0, int nb, u32 L_T, u32 acc_at, int lane)
+{
+    constexpr u32 full = 0xffffffffu;
+    const u32 LT4 = L_T * 4u;
+    const u32 mine_at = acc_at + (u32)lane * LT4;
+    const u32 range_add = (256u - LT4) * 0x01010101u;       // (4 L_T is 164..256 here; 256: the term is 0 and no byte is out of range)
+    const int nq = nb >> 2, src_lane = lane >> 2;
+    const u32 sel = 0x4440u | ((u32)lane & 3u);             // byte (lane & 3) of a register, zero-extended
+    const bool own = lane < nq, ahead = (u32)lane < ((u32)b0 >> 2);
+    u32 bad = 0, rsv = 0, oor = 0;
+#pragma unroll 1
+    for (u32 j = 0; j < staged; j++) {
+        const u32 l = l0 + j;
+        const u32 counts = sl_at + coff[l];
+        const u32 limit = m_cnt[j];
+        const u32 words = counts + count_bytes + m_head[j];
+        const u32 sb = __float_as_uint(s_scale[l]) - 0x40000000u;   // + (word << 30): +scale for code 01, -scale for code 11
+        u32 x = 0, y = 0;
+        if (own) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x) : "r"(counts + (u32)(b0 + 4 * lane)) : "memory");
+        if (ahead) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(y) : "r"(counts + 4u * (u32)lane) : "memory");
+        const u32 t4 = __dp4a(x, 0x01010101u, 0u);
+        const u32 before = b0 > 0 ? __reduce_add_sync(full, __dp4a(y, 0x01010101u, 0u)) : 0u;
+        u32 v = t4;
+#pragma unroll
+        for (int d = 1; d < 8; d <<= 1) {
+            const u32 t = __shfl_up_sync(full, v, d);
+            if (lane >= d) v += t;
+        }
+        const u32 W = __shfl_sync(full, v, nq - 1);
+        const u32 base = __shfl_sync(full, v - t4, src_lane);
+        const u32 xs = __shfl_sync(full, x, src_lane);
+        const u32 c = lane < nb ? __byte_perm(xs, 0u, sel) : 0u;
+        if (before + W > limit) {
+            bad |= ADACOMP_DEV_BAD_STREAM;          // counts and directory disagree: nothing is read
+            continue;
+        }
+        u32 p = words + before + base + __byte_perm(xs * 0x01010100u, 0u, sel);     // my first word
+        const u32 sh = (p & 3u) * 8u;
+        p &= ~3u;
+        const u32 groups = (__reduce_max_sync(full, c) + 3u) >> 2;
+        int left8 = (int)(8u * c);                  // bits of my words still to come
+        u32 x0;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x0) : "r"(p) : "memory");
+#pragma unroll 1
+        for (u32 g = 0; g < groups; g++) {
+            u32 x1, past;
+            p += 4u;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x1) : "r"(p) : "memory");
+            u32 w4 = __funnelshift_r(x0, x1, sh);
+            x0 = x1;
+            asm("shl.b32 %0, %1, %2;" : "=r"(past) : "r"(full), "r"((u32)left8));     // (a shift by 32 or more gives 0)
+            left8 = max(left8 - 32, 0);
+            w4 &= ~past;                                                            // bytes past my count: the no-op word
+            rsv |= (w4 >> 1) & ~w4;                                                 // bit 0 of a byte: reserved code 10
+            const u32 ge = ((w4 & 0x7f7f7f7fu) + range_add) & w4 & 0x80808080u;     // bit 7 of a byte: index >= L_T
+            if (ge) {
+                oor |= ge;
+                w4 &= ~((ge >> 7) * 0xffu);                                         // those are skipped
+            }
+            // the four elements are distinct (a bin's words carry distinct indices): loads first, stores last
+            add4_words(mine_at, w4, sb);
+        }
+    }
+    if (__any_sync(full, (rsv & 0x01010101u) != 0u)) bad |= ADACOMP_DEV_RESERVED_CODE;
+    if (__any_sync(full, LT4 < 256u && oor != 0u)) bad |= ADACOMP_DEV_BAD_STREAM;
     return bad;
 }
 
@@ -2296,19 +2452,6 @@ __device__ inline u32 warp_add_group_by_bin(const GroupSrc<Addr> &src, int R, in
     if (__any_sync(full, (rsv & 1u) != 0u)) bad |= ADACOMP_DEV_RESERVED_CODE;
     if (__any_sync(full, mx >= LT4)) bad |= ADACOMP_DEV_BAD_STREAM;
     return bad;
-}
-
-// out[e] += v (as add_at_if_valid) when `go` is not zero; nothing is read or written otherwise.
-__device__ inline void add_at_if(u32 e, float v, u32 go)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .f32 x;\n\t"
-        "setp.ne.u32 p, %2, 0;\n\t"
-        "@p ld.shared.f32 x, [%0];\n\t"
-        "@p add.rn.f32 x, x, %1;\n\t"
-        "@p st.shared.f32 [%0], x;\n\t}"
-        ::"r"(e), "f"(v), "r"(go)
-        : "memory");
 }
 
 // L_T > 1000 (a tile is one bin): an item is 4096 consecutive output elements, which lie in `live` bins (at
@@ -2406,17 +2549,40 @@ struct WarpItems {
     u64 n_items;
     u32 max_bins;   // bins an item needs the counts of
 };
-__host__ __device__ inline WarpItems warp_items(const Geometry &g)
+// M (tiles of more than one bin only): an item is M consecutive tiles of the stream, decoded as one tile of
+// M * tile_bins bins (their bin counts and their words are contiguous in the stream).
+__host__ __device__ inline WarpItems warp_items(const Geometry &g, u32 M = 1u)
 {
     WarpItems w;
     if (g.tile_bins == 1u) {
         w.n_items = (g.n + (u64)kDecodeChunk - 1) / (u64)kDecodeChunk;
         w.max_bins = ((u32)kDecodeChunk - 2u) / g.L_T + 2u;
     } else {
-        w.n_items = g.n_tiles;
-        w.max_bins = g.tile_bins;
+        w.n_items = (g.n_tiles + M - 1u) / M;
+        w.max_bins = M * g.tile_bins;
     }
     return w;
+}
+
+// Tiles of 80 bins of 8-bit words (L_T = 48, 49, 50) go in pairs: 160 bins split between five decoding
+// warps give every lane of a warp a bin, and a warp's run of words per learner is long enough to
+// spread the per-learner set-up (counts to offsets, flags) over six 32-word steps instead of four.
+#ifndef ADACOMP_PAIR_MIN_TILES
+#define ADACOMP_PAIR_MIN_TILES 256
+#endif
+constexpr long long kPairMinTiles = ADACOMP_PAIR_MIN_TILES;
+
+// Items whose adds run a lane per bin (see warp_add_lanes_all): more than 64 bins of 8-bit words, split between
+// nw warps into shares of a multiple of 4 and at most 32 bins, the item's run of counts a multiple of 16 bytes.
+__host__ __device__ inline bool lanes_shape(u32 item_bins, u32 nw, u32 word_bytes)
+{
+    const u32 nb = item_bins / nw;
+    return word_bytes == 1u && item_bins > 64u && item_bins % nw == 0u && (nb & 3u) == 0u && nb <= 32u && (item_bins & 15u) == 0u;
+}
+__host__ __device__ inline bool pair_path(const Geometry &g)
+{
+    // (small tensors keep single tiles: more items to spread over the SMs)
+    return g.w == 1u && g.tile_bins == 80u && g.tile_elems <= (u32)kDecodeChunk && g.n_tiles >= (u64)kPairMinTiles;
 }
 
 // A CTA's work items in turn: it takes every stride-th.  Where items are tiles, `tile` is all there is to
@@ -2462,17 +2628,17 @@ __device__ inline u32 count_room(int TB)
 }
 
 // Lays the slots out (see WarpDecSmem), then decodes.
-template <typename Word, bool MULTI, int OPT, int NW, bool ONE>
+template <typename Word, bool MULTI, int OPT, int NW, bool ONE, int M>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv);
 
 //   s_wv   (OPT != 0) shared memory for a tile of weights, a tile of momentum and (Adam) a tile of second moments
-template <typename Word, int OPT, int NW, bool ONE>
+template <typename Word, int OPT, int NW, bool ONE, int M>
 __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                                  const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const WarpItems wi = warp_items(geo);
+    const WarpItems wi = warp_items(geo, (u32)M);
     const int TB = (int)wi.max_bins;
     const u32 count_bytes = count_room<Word>(TB);
     const u32 k8 = (a.k + 7u) & ~7u;
@@ -2486,7 +2652,7 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
         ws.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
+    for (int i = tid; i < M * kDecodeChunk; i += blockDim.x) s_acc[i] = 0.f;
     if (warp == NW) {
         // the learners' regions: counts, then room for 1.5 times a tile's average words + slack
 #pragma unroll
@@ -2495,7 +2661,7 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
             if (l < a.k) {
                 // (an item of 4096 elements brings the words of the bins at its ends whole: L_T more elements, on average)
                 const u64 per = s_nsel[l] / wi.n_items, avg = ONE ? per + per * geo.L_T / (u64)kDecodeChunk : per;
-                const u64 cap = min(ONE ? (u64)wi.max_bins * geo.L_T : (u64)geo.tile_elems, avg + avg / 2 + 64);
+                const u64 cap = min(ONE ? (u64)wi.max_bins * geo.L_T : (u64)M * geo.tile_elems, avg + avg / 2 + 64);
                 // (a learner alone always fits a slot; tiles of more than 4096 elements can have more words than that)
                 ws.wcap[l] = (unsigned short)min(align_up(cap * sizeof(Word) + 16, 16), (u64)((kSlotMax - meta_bytes - count_bytes) & ~15u));
             }
@@ -2521,28 +2687,31 @@ __device__ void decode_warps_any(const DecodeArgs &a, const Geometry &geo, float
             ws.rcount[r] = (unsigned char)(a.k - r0);
             ws.n_rounds = r + 1u;
             ws.slot_bytes = most;
-            ws.n_slots = min((u32)kSlots, kRingBytes / most);
+            ws.n_slots = min((u32)kSlots, ring_bytes(NW) / most);
         }
     }
     __syncthreads();
-    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT, NW, ONE>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-    else decode_warps<Word, false, OPT, NW, ONE>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    if (ws.n_rounds > 1u) decode_warps<Word, true, OPT, NW, ONE, M>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    else decode_warps<Word, false, OPT, NW, ONE, M>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
 }
 
 // MULTI: a tile takes several rounds (the learners' regions do not fit one slot together).
 // OPT: 0 the finished share goes to a.dst; 1 (SGD) / 2 (Adam) it feeds the optimizer step of a.ep instead.
 // NW: decoding warps (warp NW is the loader); each owns 1/NW of the tile's bins ("quarter" below, whatever NW is).
 // ONE: tiles of one bin (L_T > 1000): an item is 4096 output elements (see WarpItems) and each warp owns 1/NW of them.
-template <typename Word, bool MULTI, int OPT, int NW, bool ONE>
+// M: tiles of the stream per item (see warp_items); an item is decoded as one tile of M * tile_bins bins.
+template <typename Word, bool MULTI, int OPT, int NW, bool ONE, int M>
 __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_acc, WarpDecSmem<NW> &ws,
                              const float *s_scale, const u64 *s_nsel, float *s_wv)
 {
+    static_assert(M == 1 || !ONE, "items of several tiles are for tiles of more than one bin");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const WarpItems wi = warp_items(geo);
-    const int TB = ONE ? (int)wi.max_bins : (int)geo.tile_bins;    // bins of an item (ONE: at most)
+    const WarpItems wi = warp_items(geo, (u32)M);
+    const int TB = (int)wi.max_bins;                               // bins of an item (ONE: at most)
     const u32 L_T = geo.L_T;
+    const u32 item_len = (u32)M * geo.tile_elems;                  // (!ONE) output elements of an item
     const u32 count_bytes = count_room<Word>(TB);                  // room of a learner's bin counts in a slot
-    const u64 first = blockIdx.x, stride = gridDim.x, n_items = ONE ? wi.n_items : geo.n_tiles;
+    const u64 first = blockIdx.x, stride = gridDim.x, n_items = wi.n_items;
     const u64 my_tiles = n_items > first ? (n_items - first + stride - 1) / stride : 0;     // items of this CTA
     const u32 k8 = (a.k + 7u) & ~7u;
     unsigned char *const ring = reinterpret_cast<unsigned char *>(ws.ring);
@@ -2561,7 +2730,11 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         u32 ta = 0, ia = 0, tb = 0, ib = 0;
         const u32 last_item = (u32)(n_items - 1), last_len = (u32)(geo.n - (n_items - 1) * (u64)kDecodeChunk);   // (ONE)
         auto load_dir = [&](u64 tile, const ItemAt &p, u32 r, bool valid, u64 *d0, u64 *d1, u32 &t, u32 &info) {
-            u32 tiles = 1u;             // tiles (each a bin) of the item
+            u32 tiles = 1u;             // tiles of the item (ONE: each a bin)
+            if (!ONE && M > 1 && valid) {
+                tile *= (u64)M;         // the item's first tile
+                tiles = (u32)min((u64)M, geo.n_tiles - tile);
+            }
             if (ONE && valid) {
                 tiles = bins_touched(p.at, p.v == last_item ? last_len : (u32)kDecodeChunk, L_T);
                 t = p.tile;
@@ -2613,7 +2786,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
                 const u64 bin0 = ONE ? (u64)ta : tile * (u64)TB;
                 const u32 live = ONE ? (ia >> 16) & 0xffu : (u32)min((u64)TB, geo.n_bins - bin0);
-                const u32 item_elems = ONE ? live * L_T : geo.tile_elems;      // more words than that are an error
+                const u32 item_elems = ONE ? live * L_T : item_len;            // more words than that are an error
                 // the item's bin counts start `clead` bytes behind a 16-byte boundary: the copy starts at the boundary
                 const u32 clead = ONE ? ia >> 24 : (u32)(bin0 * sizeof(Word)) & 15u;
                 const u32 cbytes = (u32)align_up(clead + live * (u32)sizeof(Word), 16);
@@ -2710,8 +2883,11 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     u32 *const tmp = ws.tmp[warp];
     const bool vec_store = (quarter & 3u) == 0 && (ONE || (geo.tile_elems & 3u) == 0);
     // tiles of at most 64 bins: G lanes share a bin
-    const bool by_bin = sizeof(Word) == 2 || TB <= 64;     // (16-bit words: L_T >= 65, at most 60 bins)
+    const bool by_bin = M == 1 && (sizeof(Word) == 2 || TB <= 64);     // (16-bit words: L_T >= 65, at most 60 bins)
     const int G = nb <= 32 ? 32 / nb : 1;           // (need not be a power of two: 5 bins take 6 lanes each)
+    // tiles of more than 64 bins of 8-bit words whose counts line up with 32-bit loads: a lane per bin
+    // (not in the plain decoder of single tiles: at its 64 registers the lane-per-bin loop spills and is slower than by word)
+    const bool lanes_ok = (M == 2 || OPT != 0) && lanes_shape((u32)TB, (u32)NW, sizeof(Word));
     const int my_local = lane / G, my_r = lane % G;
     const int my_bin = my_local < nb ? b0 + my_local : TB;
     const u32 mine_at = smem_addr(s_acc) + (u32)my_bin * L_T * 4u;
@@ -2729,7 +2905,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         u32 live = ONE ? 0u : (u32)min((u64)TB, geo.n_bins - v * (u64)TB);      // bins of the item
         u32 clead = ONE ? 0u : (u32)(v * (u64)TB * sizeof(Word)) & 15u;          // where the counts start in their room (see the loader)
         u32 lo = 0;                                 // (ONE) the warp's first element, counted from the first bin's
-        const u64 out0 = v * (u64)(ONE ? (u32)kDecodeChunk : geo.tile_elems) + (u64)warp * quarter;
+        const u64 out0 = v * (u64)(ONE ? (u32)kDecodeChunk : item_len) + (u64)warp * quarter;
         const u32 len = out0 < geo.n ? (u32)min((u64)quarter, geo.n - out0) : 0u;
         const bool whole = vec_store && len == quarter;
         if (OPT != 0 && whole && lane == 0) {
@@ -2762,7 +2938,12 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             const unsigned short *m_cnt = reinterpret_cast<const unsigned short *>(sl + kSlotHead), *m_head = m_cnt + k8;
             const u32 sl_at = smem_addr(sl);
 
-            // ---- the round's learners whose words wait in the slot, four at a time ----
+            // ---- the round's learners whose words wait in the slot ----
+            if (lanes_ok && (u32)(b0 + nb) <= live) {
+                bad |= warp_add_lanes_all(sl_at, ws.coff, m_cnt, m_head, s_scale, l0, staged, count_bytes, b0, nb, L_T, acc_at, lane);
+                __syncwarp();
+            } else
+            // (the other shapes: four learners at a time)
             for (u32 g0 = 0; g0 < staged; g0 += kRoundMax) {
                 const int R = (int)min((u32)kRoundMax, staged - g0);
                 GroupSrc<u32> src = {0u, 0u, 0u, 0u};
@@ -2790,9 +2971,9 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     const unsigned char *st = a.stream[l];
                     const u64 *dir = reinterpret_cast<const u64 *>(st + geo.tile_off_at);
                     // (ONE: the first tile, that is bin, of the item, by division on this rare path)
-                    const u64 tile = ONE ? (v * (u64)kDecodeChunk) / L_T : v, bin0 = ONE ? tile : tile * (u64)TB;
-                    const u64 w0 = dir[tile], w1 = dir[tile + (ONE ? live : 1u)];
-                    ok = w1 >= w0 && w1 - w0 <= (ONE ? live * L_T : geo.tile_elems) && w1 <= s_nsel[l];
+                    const u64 tile = ONE ? (v * (u64)kDecodeChunk) / L_T : v * (u64)M, bin0 = ONE ? tile : v * (u64)TB;
+                    const u64 w0 = dir[tile], w1 = dir[tile + (ONE ? live : (u32)min((u64)M, geo.n_tiles - tile))];
+                    ok = w1 >= w0 && w1 - w0 <= (ONE ? live * L_T : item_len) && w1 <= s_nsel[l];
                     src.counts = (u64)__cvta_generic_to_global(st + geo.bin_cnt_at) + bin0 * sizeof(Word);
                     src.words = (u64)__cvta_generic_to_global(st + geo.payload_at) + (ok ? w0 : 0) * sizeof(Word);
                     src.limit = ok ? (u32)(w1 - w0) : 0u;
@@ -3020,6 +3201,7 @@ __device__ inline bool decode_headers(const DecodeArgs &a, int *s_bad, float *s_
 // the one that works; one that does not launches all three.
 // dynamic shared memory of decode_sum_warps<OPT>: a tile per array of the optimizer
 constexpr u32 opt_smem_bytes(int opt) { return opt == 0 ? 0u : (opt == 2 ? 3u : 2u) * kDecodeChunk * 4u; }
+constexpr u32 kPairSmemBytes = 2u * kDecodeChunk * 4u;     // dynamic shared memory of the M = 2 kernel: its output tile
 
 // NW decoding warps and the loader warp: 4 for plain decoding; with an optimizer step, whose staged tiles
 // leave room for fewer CTAs per SM, 8 where they divide the tile's bins (more warps to hide the adds' latency).
@@ -3027,12 +3209,15 @@ constexpr u32 opt_smem_bytes(int opt) { return opt == 0 ? 0u : (opt == 2 ? 3u : 
 // allotted apart from the other shapes'.
 // (The one-bin form runs four CTAs per SM: with 96 registers it keeps everything in registers, and its few
 // words per item leave it less to hide than the other shapes have; measured 3 % faster than six CTAs of 64.)
-template <int OPT, int NW, bool ONE = false>
-__global__ void __launch_bounds__((NW + 1) * 32, OPT == 0 ? (ONE ? 4 : kWarpsPerSm) : OPT == 1 ? 3 : 2)
+// M = 2 (plain decoding only): the pairs of 80-bin tiles of pair_path(), five decoding warps, four CTAs per SM; the
+// output tile of 2 x 4096 elements is dynamic shared memory.
+template <int OPT, int NW, bool ONE = false, int M = 1>
+__global__ void __launch_bounds__((NW + 1) * 32, M == 2 ? 4 : OPT == 0 ? (ONE ? 4 : kWarpsPerSm) : OPT == 1 ? 3 : 2)
 decode_sum_warps(DecodeArgs a)
 {
     static_assert(!ONE || NW == 4, "tiles of one bin are split between four warps");
-    __shared__ __align__(16) float s_acc[kDecodeChunk];
+    static_assert(M == 1 || (M == 2 && OPT == 0 && !ONE && NW == 5), "pairs of tiles: plain decoding, five warps");
+    __shared__ __align__(16) float s_acc_static[M == 1 ? kDecodeChunk : 4];
     __shared__ __align__(16) WarpDecSmem<NW> ws;
     __shared__ u64 s_nsel[ADACOMP_MAX_STREAMS];
     __shared__ float s_scale[ADACOMP_MAX_STREAMS];
@@ -3042,15 +3227,20 @@ decode_sum_warps(DecodeArgs a)
     if (!decode_headers(a, &s_bad, s_scale, s_nsel, L_T, n)) return;
     const Geometry geo = make_geometry(n, L_T);
     // (the launcher picks NW from the shape it was given: a divisor of the tile's bins; 4 for tiles of one bin)
-    if (!warp_path(geo) || ONE != (geo.tile_bins == 1u) || (!ONE && geo.tile_bins % (u32)NW != 0)) return;
+    if (!warp_path(geo) || ONE != (geo.tile_bins == 1u) || (!ONE && (M * geo.tile_bins) % (u32)NW != 0)) return;
+    // plain decoding: the shapes of pair_path() belong to the M = 2 kernel, all others to the M = 1 kernels
+    if (OPT == 0 && !ONE && (M == 2) != (a.pairs != 0u && pair_path(geo))) return;
     // (the rounds are laid out inside; the first thing decode_warps does after that is uniform)
-    extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles
+    extern __shared__ __align__(16) float s_dyn[];     // (OPT != 0) the optimizer's staged tiles; (M == 2) the output tile
     float *const s_wv = OPT ? s_dyn : nullptr;
+    float *const s_acc = M == 1 ? s_acc_static : s_dyn;
     if constexpr (ONE) {
-        decode_warps_any<unsigned short, OPT, NW, true>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+        decode_warps_any<unsigned short, OPT, NW, true, 1>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+    } else if constexpr (M == 2) {
+        decode_warps_any<unsigned char, OPT, NW, false, 2>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
     } else {
-        if (geo.w == 1u) decode_warps_any<unsigned char, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
-        else decode_warps_any<unsigned short, OPT, NW, false>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+        if (geo.w == 1u) decode_warps_any<unsigned char, OPT, NW, false, 1>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
+        else decode_warps_any<unsigned short, OPT, NW, false, 1>(a, geo, s_acc, ws, s_scale, s_nsel, s_wv);
     }
 }
 
@@ -3702,6 +3892,7 @@ struct DeviceInfo {
     int smem_optin = 0;
     int decode_per_sm = 0;
     int decode_warps_per_sm = 0, decode_one_per_sm = 0;
+    int decode_pair_per_sm = 0;         // 0: the kernel of pair_path() cannot be launched on this device
     int decode_opt_per_sm[2][2] = {{0, 0}, {0, 0}};     // [SGD, Adam][4, 8 decoding warps]; 0: unavailable on this device
     int batch_per_sm = 0;
     bool batch_fast_ready = false;      // the pipelined batch tile pass can be launched       // 0: batched pack() unavailable on this device
@@ -3736,6 +3927,7 @@ int device_info(DeviceInfo *&out)
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, kernel, threads, smem);
             return per;
         };
+        d.decode_pair_per_sm = opt_ready(decode_sum_warps<0, 5, false, 2>, 6 * 32, kPairSmemBytes);
         d.decode_opt_per_sm[0][0] = opt_ready(decode_sum_warps<1, 4>, 5 * 32, opt_smem_bytes(1));
         d.decode_opt_per_sm[0][1] = opt_ready(decode_sum_warps<1, 8>, 9 * 32, opt_smem_bytes(1));
         d.decode_opt_per_sm[1][0] = opt_ready(decode_sum_warps<2, 4>, 5 * 32, opt_smem_bytes(2));
@@ -3923,6 +4115,7 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;
+    args.pairs = !ep && info->decode_pair_per_sm > 0 ? 1u : 0u;
     u64 grid = (u64)info->sms * info->decode_per_sm, grid_w = (u64)info->sms * info->decode_warps_per_sm;
     u64 grid_one = (u64)info->sms * info->decode_one_per_sm;
     bool warps = true, others = true;   // the shape is on the device: every kernel goes, all but one return at once
@@ -3938,7 +4131,9 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (warps && ep) {
         // (the optimizer entry points always pass the shape)
-        const bool eight = hint_L_T && make_geometry(hint_n, hint_L_T).tile_bins % 8u == 0;
+        // (eight warps where they divide the tile's bins, unless four can work a lane per bin)
+        const Geometry og = make_geometry(hint_n, hint_L_T ? hint_L_T : 1u);
+        const bool eight = hint_L_T && og.tile_bins % 8u == 0 && !lanes_shape(og.tile_bins, 4u, og.w);
         const int per = info->decode_opt_per_sm[ep->adam ? 1 : 0][eight ? 1 : 0];
         if (!per) return ADACOMP_ERR_CUDA;
         u64 grid_s = (u64)info->sms * per;
@@ -3955,8 +4150,19 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
         else if (one) decode_sum_warps<1, 4, true><<<g, 5 * 32, opt_smem_bytes(1), st>>>(args);
         else decode_sum_warps<1, 4><<<g, 5 * 32, opt_smem_bytes(1), st>>>(args);
     } else if (warps) {
-        // (without the shape both go and one of them returns at once)
-        if (!hint_L_T || hint_L_T <= 1000u) decode_sum_warps<0, 4><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
+        // (without the shape all three go and two of them return at once; the pairs of 80-bin tiles have a
+        // kernel of their own, see pair_path())
+        const bool pairs_ok = info->decode_pair_per_sm > 0;
+        const bool pair = pairs_ok && hint_L_T && pair_path(make_geometry(hint_n, hint_L_T));
+        if (pairs_ok && (!hint_L_T || pair)) {
+            u64 grid_p = (u64)info->sms * info->decode_pair_per_sm;
+            if (hint_L_T) {
+                const u64 items = warp_items(make_geometry(hint_n, hint_L_T), 2u).n_items;
+                grid_p = items < grid_p ? (items ? items : 1) : grid_p;
+            }
+            decode_sum_warps<0, 5, false, 2><<<(unsigned)grid_p, 6 * 32, kPairSmemBytes, st>>>(args);
+        }
+        if (!hint_L_T || (hint_L_T <= 1000u && !pair)) decode_sum_warps<0, 4><<<(unsigned)grid_w, kDecodeLaunch, 0, st>>>(args);
         if (!hint_L_T || hint_L_T > 1000u) decode_sum_warps<0, 4, true><<<(unsigned)grid_one, kDecodeLaunch, 0, st>>>(args);
     }
     if (others) decode_sum<<<(unsigned)grid, kDecodeThreads, 0, st>>>(args);
