@@ -141,7 +141,9 @@ int adacomp_compress(const float *grad, float *residue, uint64_t n, uint32_t L_T
  * stream capture.  Every call on a device shares the one array, and it keeps the previous
  * call's contents: the call clears the part that must start from zero itself, but two
  * calls that overlap on the GPU (different streams, no dependency between them) race on
- * it and corrupt each other's output.  Calls on one stream are safe.
+ * it and corrupt each other's output.  Calls on one stream are safe.  (The address
+ * look-up itself needs no lock: host threads that make the first call together all find
+ * the same address.)
  */
 int adacomp_compress_static(const float *grad, float *residue, uint64_t n, uint32_t L_T,
                             void *packed_out, uint64_t *count_out, void *stream);
@@ -151,14 +153,14 @@ int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t 
                         void *packed_out, uint64_t *count_out, void *stream, uint32_t flags);
 
 /*
- * adacomp_compress with the scale-factor of the paper's self-adjusting selection (Section 2.4:
- * an element is also sent when "its previous residue plus the latest gradient multiplied by a
- * scale-factor exceeds the maximum of the bin"; 1.5 to 3.0 were studied, 2 was chosen).  The test
+ * adacomp_compress with another multiplier in the paper's self-adjusting selection (Section 2.4:
+ * the value compared with the bin maximum is the old residue plus a multiple of the latest
+ * gradient; multiples from 1.5 to 3.0 were studied and 2 was chosen).  The test
  * value becomes H = residue + factor * dW, one rounded multiplication and one rounded addition in
  * binary32; everything else (G, bin maxima, scale, forced bin maximum, quantisation, residue,
  * stream layout) is as in adacomp_compress, which keeps Algorithm 2's H = G + dW with two additions
  * (for factor 2 the two can differ in the last place).  factor = 1 makes H = G: only the bin maxima
- * are sent, the "local selection" scheme without soft-threshold of Section 5.
+ * are sent, which is Section 5's local selection without the soft threshold ("LS").
  *   factor   0 < factor <= 1e30, else ADACOMP_ERR_FLAGS.
  * The stream's header carries bit 1 in its flags byte.  Runs at the speed of adacomp_compress.
  */

@@ -1,7 +1,7 @@
 /*
  * CPU oracle for AdaComp pack() and unpack()-and-sum.  TEST INFRASTRUCTURE ONLY.
  *
- * A plain, slow, single-threaded restatement of Algorithm 2 ("Details of pack()")
+ * A plain, slow restatement of Algorithm 2 ("Details of pack()")
  * and of the unpack()/sum half of Algorithm 1 of the AdaComp paper, in IEEE
  * binary32 (the precision the method is stated in), written to be checked
  * against the paper by eye.  It shares no code with the CUDA library and is
@@ -17,8 +17,8 @@
  *   - the last bin may be short (Section 2.5 says Algorithm 2 assumes T | length);
  *   - g_max(i) is the largest |G| in bin i (Algorithm 2, "largest absolute value");
  *   - an element is sent when |H| >= g_max(i) (Algorithm 2) or when it IS the
- *     bin maximum (Section 2.4: "In addition to this value ... several other
- *     residues"); flag bit 0 drops the second clause (literal Algorithm 2);
+ *     bin maximum (Section 2.4 describes the other residues as sent in addition
+ *     to the maximum); flag bit 0 drops the second clause (literal Algorithm 2);
  *   - bins whose maximum is zero send nothing, and an element with G == 0 is
  *     never sent (its ternary value would be 0);
  *   - Quantize(G) = sign(G) * scale, scale = mean over ALL bins of g_max
@@ -143,20 +143,52 @@ double adacomp_oracle_exact_sum(const float *v, uint64_t count)
 }
 
 /* ---- pack(): Algorithm 2 -------------------------------------------------- */
+
+/*
+ * Threads the per-element and per-bin loops of pack() may use (default 1: the checker the tests
+ * pin).  Every bin is worked on its own and the sum of the bin maxima is exact, so the stream and
+ * the residue do not depend on this number; the benchmark's all-host-cores baseline sets it.
+ */
+static int oracle_threads = 1;
+
+void adacomp_oracle_set_threads(int threads) { oracle_threads = threads > 1 ? threads : 1; }
+int adacomp_oracle_get_threads(void) { return oracle_threads; }
+
+/*
+ * Which elements of one bin are sent (Algorithm 2's test inside its second pair of loops, with the
+ * readings listed at the top of this file).  The bin holds elements [lo, hi) of the layer and
+ * `largest` is its g_max.  The places of the sent elements inside the bin are written to `places`
+ * (ascending; skipped when NULL); the return value is how many there are.
+ */
+static uint32_t sent_places_of_bin(const float *G, const float *H, uint64_t lo, uint64_t hi, float largest,
+                                   int literal, uint16_t *places)
+{
+    uint32_t sent = 0;
+    if (!(largest > 0.0f)) return 0;                 /* a bin of zeros sends nothing */
+    for (uint64_t i = lo; i < hi; i++) {
+        if (G[i] == 0.0f) continue;                  /* its ternary value would be 0 */
+        const int passes_test = fabsf(H[i]) >= largest;
+        const int is_the_maximum = !literal && fabsf(G[i]) == largest;
+        if (passes_test || is_the_maximum) {
+            if (places) places[sent] = (uint16_t)(i - lo);
+            sent++;
+        }
+    }
+    return sent;
+}
+
 /*
  * dW[n] in; residue[n] in/out; out[out_cap] receives the stream.
  * g_max_out (optional, n_bins floats) receives the bin maxima.
  * Returns 0, or -1 bad argument, -2 out of memory, -3 out_cap too small.
- */
-/*
- * `factor`: the scale-factor of the self-adjusting selection (Section 2.4: "the sum of its previous
- * residue plus the latest gradient multiplied by a scale-factor", studied from 1.5 to 3.0, 2 chosen
- * "for computational ease (simple additions vs. multiplications)").  0 selects the paper's choice as
+ *
+ * `factor`: the multiplier of the latest gradient in the selection test (Section 2.4 studies 1.5 to
+ * 3.0 and settles on 2 because it needs additions only).  0 selects the paper's choice as
  * Algorithm 2 writes it, H = G + dW with two additions; any other value takes the general form
  * H = residue + factor * dW, one rounded multiplication and one rounded addition (for factor 2 the
  * two forms can differ in the last place, which is why they are kept apart).  Factor 1 makes H = G:
- * only the bin maxima are sent, the local-selection scheme "without soft-threshold" the paper
- * compares against (Section 5, "LS").  Streams made with a factor carry bit 1 in the header's flags.
+ * only the bin maxima are sent, which is the local selection without the soft threshold that the
+ * paper compares against (Section 5, "LS").  Streams made with a factor carry bit 1 in the header's flags.
  */
 int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint32_t L_T,
                                uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out);
@@ -174,16 +206,21 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
     if (factor != 0.0f && !(factor > 0.0f && factor <= 1e30f)) return -1;
     flags = (flags & 1u) | (factor != 0.0f ? 2u : 0u);
     const int literal = (flags & 1u) != 0;
+    const int threads = oracle_threads;
+    (void)threads;
     geometry geo = geometry_of(n, L_T);
     if (out_cap < geo.payload_at) return -3;
+    const int64_t bins = (int64_t)geo.n_bins, elems = (int64_t)n;
 
     float *G = (float *)malloc((n ? n : 1) * sizeof(float));
     float *H = (float *)malloc((n ? n : 1) * sizeof(float));
     float *g_max = (float *)malloc((geo.n_bins ? geo.n_bins : 1) * sizeof(float));
-    if (!G || !H || !g_max) { free(G); free(H); free(g_max); return -2; }
+    uint64_t *first_word = (uint64_t *)malloc((geo.n_bins + 1u) * sizeof(uint64_t));
+    if (!G || !H || !g_max || !first_word) { free(G); free(H); free(g_max); free(first_word); return -2; }
 
     /* G <- residue + dW ;  H <- G + dW   (two rounded additions), or H <- residue + factor * dW */
-    for (uint64_t i = 0; i < n; i++) {
+#pragma omp parallel for num_threads(threads) if (threads > 1)
+    for (int64_t i = 0; i < elems; i++) {
         G[i] = residue[i] + dW[i];
         if (factor == 0.0f) {
             H[i] = G[i] + dW[i];
@@ -193,9 +230,10 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
         }
     }
 
-    /* first loop over all bins: the largest absolute value in each bin */
-    for (uint64_t b = 0; b < geo.n_bins; b++) {
-        uint64_t lo = b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+    /* g_max: the largest |G| of every bin */
+#pragma omp parallel for num_threads(threads) if (threads > 1)
+    for (int64_t b = 0; b < bins; b++) {
+        uint64_t lo = (uint64_t)b * L_T, hi = lo + L_T < n ? lo + L_T : n;
         float m = 0.0f;
         for (uint64_t i = lo; i < hi; i++)
             if (fabsf(G[i]) > m) m = fabsf(G[i]);
@@ -210,43 +248,46 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
         scale = (float)(S / (double)geo.n_bins);
     }
 
-    /* second loop over all bins and all indices within each bin */
+    /* how many elements each bin sends, hence where its words start in the stream */
+#pragma omp parallel for num_threads(threads) if (threads > 1)
+    for (int64_t b = 0; b < bins; b++) {
+        uint64_t lo = (uint64_t)b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+        first_word[b + 1] = sent_places_of_bin(G, H, lo, hi, g_max[b], literal, NULL);
+    }
+    first_word[0] = 0;
+    for (uint64_t b = 0; b < geo.n_bins; b++) first_word[b + 1] += first_word[b];
+    const uint64_t n_sel = first_word[geo.n_bins];
+    const uint64_t bytes_used = geo.payload_at + align16(n_sel * geo.w);
+    const int overflow = bytes_used > out_cap;
+
+    /* bin by bin: the counts, the words of the sent elements, and everybody's new residue */
     memset(out, 0, geo.payload_at);
     uint8_t *tile_off = out + geo.tile_off_at;
     uint8_t *bin_cnt = out + geo.bin_cnt_at;
     uint8_t *payload = out + geo.payload_at;
-    uint64_t n_sel = 0;
-    int overflow = 0;
-    for (uint64_t b = 0; b < geo.n_bins; b++) {
-        if (b % geo.tile_bins == 0) put_u64(tile_off + 8u * (b / geo.tile_bins), n_sel);
-        uint64_t lo = b * L_T, hi = lo + L_T < n ? lo + L_T : n;
-        uint32_t count = 0;
-        for (uint64_t index = lo; index < hi; index++) {
-            int send = g_max[b] > 0.0f && G[index] != 0.0f &&
-                       (fabsf(H[index]) >= g_max[b] ||
-                        (!literal && fabsf(G[index]) == g_max[b]));
-            if (send) {
-                int negative = signbit(G[index]) != 0;
-                float Gq = negative ? -scale : scale;           /* Quantize(G(index)) */
-                uint32_t word = ((uint32_t)(index - lo) << 2) | (negative ? 3u : 1u);
-                uint64_t at = geo.payload_at + (n_sel + 1u) * geo.w;
-                if (at > out_cap) overflow = 1;
-                else if (geo.w == 1u) payload[n_sel] = (uint8_t)word;
-                else put_u16(payload + 2u * n_sel, (uint16_t)word);
-                residue[index] = G[index] - Gq;
-                n_sel++;
-                count++;
-            } else {
-                residue[index] = G[index];                       /* no transmission */
+#pragma omp parallel for num_threads(threads) if (threads > 1)
+    for (int64_t b = 0; b < bins; b++) {
+        uint64_t lo = (uint64_t)b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+        uint16_t places[16384];
+        const uint32_t sent = sent_places_of_bin(G, H, lo, hi, g_max[b], literal, places);
+        if ((uint64_t)b % geo.tile_bins == 0) put_u64(tile_off + 8u * ((uint64_t)b / geo.tile_bins), first_word[b]);
+        if (geo.w == 1u) bin_cnt[b] = (uint8_t)sent;
+        else put_u16(bin_cnt + 2u * (uint64_t)b, (uint16_t)sent);
+        for (uint64_t i = lo; i < hi; i++) residue[i] = G[i];          /* kept whole where nothing is sent */
+        for (uint32_t j = 0; j < sent; j++) {
+            const uint64_t i = lo + places[j];
+            const int negative = signbit(G[i]) != 0;
+            const float quantised = negative ? -scale : scale;          /* sign(G) times the layer's scale */
+            residue[i] = G[i] - quantised;
+            if (!overflow) {
+                const uint32_t word = ((uint32_t)places[j] << 2) | (negative ? 3u : 1u);
+                const uint64_t at = first_word[b] + j;
+                if (geo.w == 1u) payload[at] = (uint8_t)word;
+                else put_u16(payload + 2u * at, (uint16_t)word);
             }
         }
-        if (geo.w == 1u) bin_cnt[b] = (uint8_t)count;
-        else put_u16(bin_cnt + 2u * b, (uint16_t)count);
     }
     put_u64(tile_off + 8u * geo.n_tiles, n_sel);
-
-    uint64_t bytes_used = geo.payload_at + align16(n_sel * geo.w);
-    if (bytes_used > out_cap) overflow = 1;
     if (!overflow) memset(payload + n_sel * geo.w, 0, bytes_used - geo.payload_at - n_sel * geo.w);
 
     put_u32(out + 0, ORACLE_MAGIC);
@@ -265,7 +306,7 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
     put_u32(out + 52, 0);
     put_u64(out + 56, bytes_used);
 
-    free(G); free(H); free(g_max);
+    free(G); free(H); free(g_max); free(first_word);
     return overflow ? -3 : 0;
 }
 

@@ -9,7 +9,7 @@ SRC = os.path.join(HERE, "adacomp_oracle.c")
 LIB = os.path.join(HERE, "liboracle.so")
 
 FLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
-         "-Wall", "-Wextra"]
+         "-Wall", "-Wextra", "-fopenmp"]     # (OpenMP: the optional all-cores mode of pack(), one thread unless asked)
 
 
 def build(force: bool = False) -> str:

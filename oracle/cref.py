@@ -30,9 +30,23 @@ def lib() -> C.CDLL:
         _lib.adacomp_oracle_pack_scaled.restype = C.c_int
         _lib.adacomp_oracle_pack_scaled.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
                                                     C.c_float, C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.adacomp_oracle_set_threads.restype = None
+        _lib.adacomp_oracle_set_threads.argtypes = [C.c_int]
+        _lib.adacomp_oracle_get_threads.restype = C.c_int
+        _lib.adacomp_oracle_get_threads.argtypes = []
         _lib.adacomp_oracle_unpack_sum.restype = C.c_int
         _lib.adacomp_oracle_unpack_sum.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
     return _lib
+
+
+def set_threads(threads: int) -> None:
+    """Threads pack() may spread its per-element and per-bin loops over (1 unless asked: the pinned checker).
+    The result does not depend on it: bins are independent and the scale's sum is exact."""
+    lib().adacomp_oracle_set_threads(int(threads))
+
+
+def get_threads() -> int:
+    return int(lib().adacomp_oracle_get_threads())
 
 
 def _ptr(a: np.ndarray) -> int:
@@ -142,10 +156,16 @@ def average_sgd(streams: Sequence[np.ndarray], n: int, weights: np.ndarray, mome
 
     Returns (w', v') as new float32 arrays; the inputs are not modified.
     """
-    k = len(streams)
+    return sgd_step(unpack_sum(streams, n), len(streams), weights, momentum, lr, mu)
+
+
+def sgd_step(s: np.ndarray, k: int, weights: np.ndarray, momentum: np.ndarray, lr: float, mu: float):
+    """averageGradients() and updateWeights() of average_sgd on a decoded sum `s` of k streams (or on a slice
+    of one, with the matching slices of the weights and the momentum): the three lines of its docstring."""
+    n = s.size
+    assert s.dtype == np.float32
     w = np.ascontiguousarray(weights, dtype=np.float32)
     v = np.ascontiguousarray(momentum, dtype=np.float32)
-    s = unpack_sum(streams, n)
     mean = s / np.float32(k)
     v_new = np.float32(mu) * v[:n] + mean
     w_new = w[:n] - np.float32(lr) * v_new

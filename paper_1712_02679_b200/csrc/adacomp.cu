@@ -56,30 +56,6 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s: bound of every device
 
 __device__ u32 g_status;             // sticky ADACOMP_DEV_* bits of this device
 
-#ifdef ADACOMP_PHASE_CLOCKS
-// Development aid (not part of the ABI): cycles spent by one decoding thread and by the producer's
-// first lane of one CTA in each phase, kept in registers and written out once at the end.
-__device__ unsigned long long g_phase_clocks[16];
-#define PHASE_DECL unsigned long long pc_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
-#define PHASE_CLOCK(i, t0)                                                              \
-    do {                                                                               \
-        const long long now_ = clock64();                                              \
-        pc_[i] += (unsigned long long)(now_ - (t0));                                   \
-        (t0) = now_;                                                                   \
-    } while (0)
-#define PHASE_CLOCK_P(i, t0) PHASE_CLOCK(i, t0)
-#define PHASE_FLUSH(thread, lo, hi)                                                     \
-    do {                                                                               \
-        if (blockIdx.x == 3 && threadIdx.x == (thread))                                \
-            for (int i_ = (lo); i_ < (hi); i_++) g_phase_clocks[i_] += pc_[i_];        \
-    } while (0)
-#else
-#define PHASE_DECL do { } while (0)
-#define PHASE_CLOCK(i, t0) do { } while (0)
-#define PHASE_CLOCK_P(i, t0) do { } while (0)
-#define PHASE_FLUSH(thread, lo, hi) do { } while (0)
-#endif
-
 __host__ __device__ inline u64 align_up(u64 x, u64 a) { return (x + a - 1) / a * a; }
 
 // Section offsets of a packed stream and of the scratch behind it.
@@ -2354,15 +2330,17 @@ __device__ inline u32 warp_add_lanes_all(u32 sl_at, const unsigned short *coff, 
         p &= ~3u;
         const u32 groups = (__reduce_max_sync(full, c) + 3u) >> 2;
         int left8 = (int)(8u * c);                  // bits of my words still to come
-        u32 x0;
+        // (the next four words are on their way while these four are added)
+        u32 x0, x1;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x0) : "r"(p) : "memory");
+        asm volatile("ld.shared.u32 %0, [%1+4];" : "=r"(x1) : "r"(p) : "memory");
 #pragma unroll 1
         for (u32 g = 0; g < groups; g++) {
-            u32 x1, past;
-            p += 4u;
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x1) : "r"(p) : "memory");
+            u32 past;
             u32 w4 = __funnelshift_r(x0, x1, sh);
             x0 = x1;
+            p += 4u;
+            asm volatile("ld.shared.u32 %0, [%1+4];" : "=r"(x1) : "r"(p) : "memory");
             asm("shl.b32 %0, %1, %2;" : "=r"(past) : "r"(full), "r"((u32)left8));     // (a shift by 32 or more gives 0)
             left8 = max(left8 - 32, 0);
             w4 &= ~past;                                                            // bytes past my count: the no-op word
@@ -2892,7 +2870,6 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
     const int my_bin = my_local < nb ? b0 + my_local : TB;
     const u32 mine_at = smem_addr(s_acc) + (u32)my_bin * L_T * 4u;
     u32 bad = 0;
-    PHASE_DECL;
     u32 s = 0, use = 0;                             // the item's slot; how many times the slot was used before
     u64 v = first;                                  // the item
     bool failed = false;
@@ -2917,14 +2894,12 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             if (OPT == 2) bulk_load(uq, a.ep.second + out0, quarter * 4u, &ws.wv_full[warp]);
         }
         for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
-            long long t0 = clock64();
             if (!mbar_wait(&ws.full[s], use & 1u)) {
                 ws.abort = 1;
                 bad |= ADACOMP_DEV_TIMEOUT;
                 failed = true;
                 break;
             }
-            PHASE_CLOCK(0, t0);
             const unsigned char *sl = ring + s * slot_bytes;
             const u32 l0 = MULTI ? ws.rfirst[r] : 0u, nl = MULTI ? ws.rcount[r] : a.k;
             const u32 staged = min(reinterpret_cast<const u32 *>(sl)[0], nl);
@@ -2959,7 +2934,6 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 else bad |= warp_add_group<Word, true, u32>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
             if (lane == 0) mbar_arrive(&ws.empty[s]);   // (the group's last __syncwarp orders the warp's reads before it)
-            PHASE_CLOCK(1, t0);
 
             // ---- the round's others: read from global memory ----
             for (u32 g0 = staged; g0 < nl; g0 += kRoundMax) {
@@ -2984,10 +2958,8 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 else if (by_bin) bad |= warp_add_group_by_bin_global<Word>(src, R, TB, live, L_T, my_bin, my_r, G, mine_at, lane);
                 else bad |= warp_add_group_global<Word>(src, R, b0, nb, live, L_T, acc_at, tmp, lane);
             }
-            PHASE_CLOCK(2, t0);
         }
         if (failed) break;
-        long long t0 = clock64();
 
         // ---- store the warp's quarter of the tile (and leave it zeroed for the next one) ----
         if (OPT != 0) {
@@ -3069,13 +3041,8 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             }
         }
         __syncwarp();                               // zeroed before the next tile's adds
-        PHASE_CLOCK(3, t0);
-#ifdef ADACOMP_PHASE_CLOCKS
-        pc_[6] += 1;
-#endif
     }
     if (lane == 0) bulk_wait_all();                // the last copies leave shared memory before the CTA ends
-    PHASE_FLUSH(32, 0, 7);
     if (bad) raise_status(bad);
 }
 
@@ -4005,9 +3972,11 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
     return ADACOMP_OK;
 }
 
+// `own_scratch` (optional): the scratch to use in place of the one behind the stream in packed_out.
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
-                  void *lazy_state = nullptr, float factor = 0.f, bool grad_bf16 = false)
+                  void *lazy_state = nullptr, float factor = 0.f, bool grad_bf16 = false,
+                  unsigned char *own_scratch = nullptr)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
@@ -4030,9 +3999,10 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (lazy && !info->fast_ready) return ADACOMP_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char *packed = static_cast<unsigned char *>(packed_out);
-    unsigned char *scratch = packed + geo.scratch_at;
+    unsigned char *scratch = own_scratch ? own_scratch : packed + geo.scratch_at;
 
-    // the exact-sum windows and the group counts start from zero
+    // the exact-sum windows and the group counts start from zero (a scratch that is reused keeps the last
+    // call's contents: tile counts and word slots are fully rewritten before they are read)
     if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess)
         return ADACOMP_ERR_CUDA;
     auto mark = [&](int i) { if (events) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st); };
@@ -4245,54 +4215,19 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     if (geo.scratch_bytes > (u64)ADACOMP_STATIC_SCRATCH_BYTES) return ADACOMP_ERR_STATIC_SCRATCH;
 
-    DeviceInfo *info = nullptr;
-    int rc = device_info(info);
-    if (rc != ADACOMP_OK) return rc;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ADACOMP_ERR_CUDA;
     if (!g_static_scratch_addr[dev]) {
-        // set-up, once per device, with that device current
+        // set-up, once per device, with that device current (two host threads that meet here store the same
+        // address: the look-up is idempotent, so no lock guards it)
         unsigned char *ptr = nullptr;
         if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
             return ADACOMP_ERR_CUDA;
         g_static_scratch_addr[dev] = ptr;
     }
-    unsigned char *scratch = g_static_scratch_addr[dev];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    unsigned char *packed = static_cast<unsigned char *>(packed_out);
-
-    // the array keeps the last call's contents: the exact-sum windows and the group counts
-    // must start from zero; tile counts and word slots are fully rewritten before they are read
-    if (cudaMemsetAsync(scratch, 0, kCtlBytes + 8 * geo.n_groups, st) != cudaSuccess) return ADACOMP_ERR_CUDA;
-    if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, 0.f, 0u};
-        if ((fast_L_T(L_T) || (any_fast_L_T(L_T) && (L_T <= 1000u || L_T >= 2800u))) && info->fast_ready) {
-            const u64 cap = (u64)info->sms * 2;
-            const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            auto launch = [&](auto kernel) { kernel<<<grid, kFastThreads, FastSmem::kBytes, st>>>(args); };
-            if (fast_L_T(L_T)) with_fast_kernel<false, false>(L_T, launch);
-            else with_any_fast_kernel<false>(L_T, launch);
-        } else {
-            rc = geo.w == 1u ? launch_generic<unsigned char>(args, *info, st)
-                             : launch_generic<unsigned short>(args, *info, st);
-            if (rc != ADACOMP_OK) return rc;
-        }
-    }
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, 0u, reinterpret_cast<u64 *>(count_out), nullptr);
-    if (geo.n_tiles) {
-        if (geo.tile_bins <= (u32)kSmallBins) {
-            const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
-            const unsigned grid = (unsigned)(want < cap ? want : cap);
-            if (geo.w == 1u) gather_fixup_small<unsigned char, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-            else gather_fixup_small<unsigned short, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-        } else {
-            const u64 cap = (u64)info->sms * 8;
-            const unsigned grid = (unsigned)(geo.n_tiles < cap ? geo.n_tiles : cap);
-            if (geo.w == 1u) gather_fixup<unsigned char><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-            else gather_fixup<unsigned short><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
-        }
-    }
-    return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
+    // the same kernels, in the same order, as adacomp_compress: only the scratch is elsewhere
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, nullptr, 0.f, false,
+                         g_static_scratch_addr[dev]);
 }
 
 }  // namespace
@@ -4529,6 +4464,13 @@ int adacomp_compress_host(const float *grad_host, float *grad_stage, float *resi
                           uint64_t *count_host, void *stream)
 {
     if (!count_host || !packed_host || (n && (!grad_host || !grad_stage))) return ADACOMP_ERR_NULL;
+    // every check pack() makes on the host comes before the first copy: an error code means nothing was enqueued
+    if (!packed_dev || !count_dev || (n && !residue)) return ADACOMP_ERR_NULL;
+    if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
+    if (misaligned(grad_stage) || misaligned(residue) || misaligned(packed_dev) ||
+        (reinterpret_cast<uintptr_t>(count_dev) & 7u))
+        return ADACOMP_ERR_ALIGN;
+    if ((n + L_T - 1) / L_T >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (n && cudaMemcpyAsync(grad_stage, grad_host, n * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return ADACOMP_ERR_CUDA;
@@ -4572,7 +4514,10 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
         if (!d.packed_out || !d.count_out || (d.n && (!d.grad || !d.residue))) return ADACOMP_ERR_NULL;
         if (d.L_T == 0 || d.L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
         if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
-        if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out)) return ADACOMP_ERR_ALIGN;
+        if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out) ||
+            (reinterpret_cast<uintptr_t>(d.count_out) & 7u))
+            return ADACOMP_ERR_ALIGN;
+        if ((d.n + d.L_T - 1) / d.L_T >= (1ull << 31)) return ADACOMP_ERR_SIZE;
         if (states) {
             if (!states[t]) return ADACOMP_ERR_NULL;
             if (misaligned(states[t])) return ADACOMP_ERR_ALIGN;
@@ -4692,19 +4637,6 @@ int adacomp_device_status(uint32_t *host_out, void *stream)
     *host_out = v;
     return ADACOMP_OK;
 }
-
-#ifdef ADACOMP_PHASE_CLOCKS
-int adacomp_debug_phase_clocks(unsigned long long *host_out, int reset)
-{
-    if (cudaDeviceSynchronize() != cudaSuccess) return ADACOMP_ERR_CUDA;
-    if (cudaMemcpyFromSymbol(host_out, g_phase_clocks, sizeof(g_phase_clocks)) != cudaSuccess) return ADACOMP_ERR_CUDA;
-    if (reset) {
-        unsigned long long zero[16] = {0};
-        cudaMemcpyToSymbol(g_phase_clocks, zero, sizeof(zero));
-    }
-    return ADACOMP_OK;
-}
-#endif
 
 int adacomp_device_status_reset(void *stream)
 {

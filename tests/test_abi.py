@@ -130,6 +130,23 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.adacomp_compress_multi(None, 0, None) == 0
     assert lib.adacomp_compress_multi_lazy(descs, None, 1, None) == -1
     assert lib.adacomp_compress_multi_lazy(None, None, 0, None) == 0
+    # a list is checked as a whole before anything is enqueued: a misaligned count_out or an oversized layer
+    # anywhere in it is refused on the host
+    two = (binding.adacomp_layer_desc * 2)()
+    for d in two:
+        d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out = A, A, 5000, 50, A, A
+    two[1].count_out = A + 4
+    assert lib.adacomp_compress_multi(two, 2, None) == -3
+    two[1].count_out = A
+    two[1].n, two[1].L_T = 1 << 40, 1
+    assert lib.adacomp_compress_multi(two, 2, None) == -5
+    # the host-buffer form validates before its first copy
+    ch = lib.adacomp_compress_host
+    assert ch(A, A, A, 10, 0, A, A, A, 100, A, None) == -2
+    assert ch(A, A + 4, A, 10, 50, A, A, A, 100, A, None) == -3
+    assert ch(A, A, A, 10, 50, A, A + 4, A, 100, A, None) == -3
+    assert ch(A, A, A, 10, 50, None, A, A, 100, A, None) == -1
+    assert ch(A, A, A, 1 << 40, 1, A, A, A, 100, A, None) == -5
 
 
 def test_binding_refuses_cpu_tensors():

@@ -184,3 +184,136 @@ def test_full_size_2_to_30_two_learners():
     assert_stream_equal(packed[0][:int(cnt[1])].cpu().numpy(), want, "2^30 learner 0 step 1")
     assert_f32_bits_equal(res0.cpu().numpy(), r_cpu0, "2^30 residue learner 0 step 1")
     assert B.adacomp_device_status() == 0
+
+
+@pytest.mark.parametrize("L_T", [50, 500])
+@pytest.mark.parametrize("log2n,learners", [(26, 4), (28, 1)])
+def test_config5_upper_sweep_points_prewarmed(L_T, log2n, learners):
+    """The sweep's points above 2^24: six carried steps (five pre-warm steps and the measured one), eager
+    and lazy-scale pack() compared with the oracle byte for byte at every step, then the dense sum; all four
+    learners at 2^26, learner 0 alone at 2^28.  The gradients come from a seeded torch CUDA generator and are
+    copied to the host for the oracle."""
+    n, k = 1 << log2n, learners
+    dev = torch.device(DEV)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7000 + log2n + L_T)
+    g = torch.empty(n, device=dev)
+    r_cpu = [np.zeros(n, np.float32) for _ in range(k)]
+    res_e = [torch.zeros(n, device=dev) for _ in range(k)]
+    res_l = [torch.zeros(n, device=dev) for _ in range(k)]
+    cap = B.adacomp_packed_capacity(n, L_T)
+    packed = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(k)]
+    packed_l = torch.empty(cap, dtype=torch.uint8, device=dev)
+    cnt = torch.zeros(2, dtype=torch.int64, device=dev)
+    state = [torch.empty(B.adacomp_lazy_state_bytes(n, L_T), dtype=torch.uint8, device=dev) for _ in range(k)]
+    for s in state:
+        B.adacomp_lazy_state_init(s, n, L_T)
+    last = [None] * k
+    for step in range(6):
+        for l in range(k):
+            g.normal_(0.0, 1e-3, generator=gen)
+            want = cref.pack(g.cpu().numpy(), r_cpu[l], L_T)
+            B.adacomp_compress(g, res_e[l], n, L_T, packed[l], cnt)
+            torch.cuda.synchronize()
+            assert_stream_equal(packed[l][:int(cnt[1])].cpu().numpy(), want, f"eager step {step} learner {l}")
+            B.adacomp_compress_lazy(g, res_l[l], state[l], n, L_T, packed_l, cnt)
+            torch.cuda.synchronize()
+            assert_stream_equal(packed_l[:int(cnt[1])].cpu().numpy(), want, f"lazy step {step} learner {l}")
+            last[l] = want.raw
+    for l in range(k):
+        assert_f32_bits_equal(res_e[l].cpu().numpy(), r_cpu[l], f"eager residue learner {l}")
+        B.adacomp_residue_flush(res_l[l], state[l], n, L_T)
+        assert_f32_bits_equal(res_l[l].cpu().numpy(), r_cpu[l], f"flushed lazy residue learner {l}")
+    del res_e, res_l, state, g
+    dst = torch.empty(n, device=dev)
+    B.adacomp_decompress_accumulate_ex(packed, k, dst, n, L_T)
+    torch.cuda.synchronize()
+    assert_f32_bits_equal(dst.cpu().numpy(), cref.unpack_sum(last, n), "dense sum")
+    assert B.adacomp_device_status() == 0
+
+
+def test_full_size_2_to_30_lazy_scale_two_carried_steps_and_flush():
+    """The entry point that meets the bandwidth target at 2^30, adacomp_compress_lazy, against the oracle:
+    two carried steps (the second applies the first one's pending subtraction while it loads), every stream
+    byte for byte, then the flush that turns the buffer into the paper's residue."""
+    n, L_T = 1 << 30, 50
+    dev = torch.device(DEV)
+    gen = torch.Generator(device=dev)
+    g = torch.empty(n, device=dev)
+    res = torch.zeros(n, device=dev)
+    r_cpu = np.zeros(n, np.float32)
+    pk = torch.empty(B.adacomp_packed_capacity(n, L_T), dtype=torch.uint8, device=dev)
+    cnt = torch.zeros(2, dtype=torch.int64, device=dev)
+    state = torch.empty(B.adacomp_lazy_state_bytes(n, L_T), dtype=torch.uint8, device=dev)
+    B.adacomp_lazy_state_init(state, n, L_T)
+    for step in range(2):
+        gen.manual_seed(1200 + step)
+        g.normal_(0.0, 1e-3, generator=gen)
+        want = cref.pack(g.cpu().numpy(), r_cpu, L_T)
+        B.adacomp_compress_lazy(g, res, state, n, L_T, pk, cnt)
+        torch.cuda.synchronize()
+        assert int(cnt[0]) == want.n_sel
+        assert_stream_equal(pk[:int(cnt[1])].cpu().numpy(), want, f"2^30 lazy step {step}")
+        del want
+    B.adacomp_residue_flush(res, state, n, L_T)
+    torch.cuda.synchronize()
+    assert_f32_bits_equal(res.cpu().numpy(), r_cpu, "2^30 lazy residue after the flush")
+    assert B.adacomp_device_status() == 0
+
+
+def test_full_size_2_to_30_bins_of_500_and_the_fused_update():
+    """2^30 elements at L_T = 500 (16-bit words): two learners' eager pack() and the dense sum against the
+    oracle; then, at L_T = 50, the fused unpack + average + SGD step of the same size, compared in slices with
+    the oracle's averageGradients() / updateWeights() so that the host never holds more than a few full-size
+    arrays."""
+    n = 1 << 30
+    dev = torch.device(DEV)
+    gen = torch.Generator(device=dev)
+    g = torch.empty(n, device=dev)
+    cnt = torch.zeros(2, dtype=torch.int64, device=dev)
+    for L_T in (500, 50):
+        cap = B.adacomp_packed_capacity(n, L_T)
+        packed, raws = [], []
+        for l in range(2):
+            gen.manual_seed(1300 + l + L_T)
+            g.normal_(0.0, 1e-3, generator=gen)
+            r_cpu = np.zeros(n, np.float32)
+            want = cref.pack(g.cpu().numpy(), r_cpu, L_T)
+            res = torch.zeros(n, device=dev)
+            pk = torch.empty(cap, dtype=torch.uint8, device=dev)
+            B.adacomp_compress(g, res, n, L_T, pk, cnt)
+            torch.cuda.synchronize()
+            assert_stream_equal(pk[:int(cnt[1])].cpu().numpy(), want, f"2^30 L_T={L_T} learner {l}")
+            assert_f32_bits_equal(res.cpu().numpy(), r_cpu, f"2^30 L_T={L_T} residue learner {l}")
+            packed.append(pk)
+            raws.append(want.raw)
+            del res, r_cpu, want
+        want_sum = cref.unpack_sum(raws, n)
+        if L_T == 500:
+            dst = torch.empty(n, device=dev)
+            B.adacomp_decompress_accumulate_ex(packed, 2, dst, n, L_T)
+            torch.cuda.synchronize()
+            assert_f32_bits_equal(dst.cpu().numpy(), want_sum, "2^30 L_T=500 dense sum")
+            del dst
+        else:
+            # weights and momentum that are cheap to make on both sides and exact in binary32
+            idx = torch.arange(n, device=dev, dtype=torch.int32)
+            w = ((idx % 1021).to(torch.float32) - 510.0) * (1.0 / 1024.0)
+            v = ((idx % 509).to(torch.float32) - 254.0) * (1.0 / 4096.0)
+            del idx
+            B.adacomp_decompress_average_sgd(packed, 2, w, v, n, L_T, 0.1, 0.9)
+            torch.cuda.synchronize()
+            w_gpu, v_gpu = w.cpu().numpy(), v.cpu().numpy()
+            del w, v
+            f = np.float32
+            step = 1 << 26
+            for lo in range(0, n, step):
+                i = np.arange(lo, lo + step, dtype=np.int64)
+                w0 = ((i % 1021).astype(np.float32) - f(510.0)) * f(1.0 / 1024.0)
+                v0 = ((i % 509).astype(np.float32) - f(254.0)) * f(1.0 / 4096.0)
+                w1, v1 = cref.sgd_step(want_sum[lo:lo + step], 2, w0, v0, 0.1, 0.9)
+                assert_f32_bits_equal(v_gpu[lo:lo + step], v1, f"2^30 fused update, momentum from {lo}")
+                assert_f32_bits_equal(w_gpu[lo:lo + step], w1, f"2^30 fused update, weights from {lo}")
+        del packed, raws, want_sum
+    assert B.adacomp_device_status() == 0
+

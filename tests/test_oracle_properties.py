@@ -328,3 +328,26 @@ def test_decoder_rejects_reserved_code_and_mismatched_streams():
     q = cref.pack(_gauss(250), np.zeros(250, np.float32), 50)
     with pytest.raises(RuntimeError, match="-4"):
         cref.unpack_sum([p.raw, q.raw], 200)
+
+
+def test_pack_on_several_threads_gives_the_same_bytes():
+    """The all-cores mode of the oracle (used only as a timed baseline) spreads pack()'s loops over
+    threads; bins are independent and the scale's sum is exact, so nothing may change."""
+    rng = np.random.default_rng(99)
+    assert cref.get_threads() == 1
+    try:
+        for L_T, n, flags, factor in [(50, 100352, 0, 0.0), (500, 147456 + 3, 0, 0.0), (7, 30011, 1, 0.0),
+                                      (5000, 123457, 0, 1.5), (64, 64 * 33 + 1, 0, 0.0), (50, 0, 0, 0.0)]:
+            dW = rng.normal(0, 1e-3, n).astype(np.float32)
+            r0 = rng.normal(0, 2e-3, n).astype(np.float32)
+            cref.set_threads(1)
+            r1 = r0.copy()
+            one = cref.pack(dW, r1, L_T, flags=flags, factor=factor)
+            cref.set_threads(5)
+            r5 = r0.copy()
+            many = cref.pack(dW, r5, L_T, flags=flags, factor=factor)
+            assert np.array_equal(one.raw, many.raw), (L_T, n)
+            assert np.array_equal(r1.view(np.uint32), r5.view(np.uint32)), (L_T, n)
+    finally:
+        cref.set_threads(1)
+

@@ -72,6 +72,48 @@ def test_static_scratch_matches_adacomp_compress_on_two_calls_in_a_row(L_T, n):
 
 
 @pytest.mark.gpu
+def test_static_scratch_stale_contents_of_another_shape_never_leak():
+    """The shared array keeps whatever the last call left.  A dense call with many tiles (every element sent)
+    fills its counts and word slots; the sparse calls after it, each of another shape, must come out exactly
+    as the CPU oracle packs them - streams, counts and residues byte for byte - so a count or a slot that some
+    path forgot to rewrite would show.  Also the empty tensor and a tensor of a single short tile."""
+    from oracle import cref
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(2024)
+
+    def static_call(dW, res, L_T):
+        n = dW.size
+        g = torch.from_numpy(dW).to(dev) if n else torch.zeros(4, device=dev)
+        r = torch.from_numpy(res).to(dev) if n else torch.zeros(4, device=dev)
+        packed = torch.full((max(stream_bound(n, L_T), 64),), 0xCD, dtype=torch.uint8, device=dev)
+        cnt = torch.zeros(2, dtype=torch.int64, device=dev)
+        B.adacomp_compress_static(g, r, n, L_T, packed, cnt)
+        torch.cuda.synchronize()
+        n_sel, used = (int(v) for v in cnt.cpu())
+        return packed[:used].cpu().numpy(), n_sel, r[:n].cpu().numpy()
+
+    def dense_call():
+        n = 4000 * 600 + 37                  # every element ties for its bin's maximum: all of them are sent
+        dW = (np.where(rng.random(n) < 0.5, -1.0, 1.0) * 0.25).astype(np.float32)
+        raw, n_sel, _ = static_call(dW, np.zeros(n, np.float32), 50)
+        assert n_sel == n
+        return raw
+
+    dense_call()
+    for L_T, n in [(500, 4000 * 150 + 11), (7, 30011), (5000, 5000 * 40 + 123), (50, 100352), (50, 0), (50, 37), (500, 499)]:
+        dW = rng.normal(0, 1e-3, n).astype(np.float32)
+        res = rng.normal(0, 2e-3, n).astype(np.float32)
+        want_res = res.copy()
+        want = cref.pack(dW, want_res, L_T)
+        raw, n_sel, got_res = static_call(dW, res, L_T)
+        assert n_sel == want.n_sel and raw.size == want.bytes_used, (L_T, n)
+        assert np.array_equal(raw, want.raw), f"L_T={L_T} n={n}: stream differs from the oracle's"
+        assert np.array_equal(got_res.view(np.uint32), want_res.view(np.uint32)), f"L_T={L_T} n={n}: residue"
+        dense_call()                         # and dirty the array again before the next shape
+    assert B.adacomp_device_status() == 0
+
+
+@pytest.mark.gpu
 def test_static_scratch_largest_supported_and_first_refused_size():
     dev = torch.device("cuda:0")
     # largest n whose scratch still fits the array (the scratch grows with n), by bisection
