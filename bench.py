@@ -763,6 +763,114 @@ def measure_config(cfg, steps, warmup, prewarm_steps, pack_only=False):
     return line
 
 
+def run_exchange(a):
+    """Algorithm 1's communication path with every rank a learner: pack() of the rank's own gradient,
+    exchange() (all-gather of the variable-length streams: their sizes first, then the streams padded to the
+    longest, received into this rank's own memory), and the decode-sum of all ranks' streams in rank order on
+    every rank.  Weak scaling: each rank brings its own n elements; the decode has as many streams as ranks."""
+    import zlib
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_1712_02679_b200 import binding as B
+    from paper_1712_02679_b200 import ranks
+    from paper_1712_02679_b200.exchange import exchange
+
+    rank, world, local = ranks.rank_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    if os.environ.get("ADACOMP_BENCH_SHARE_GPU") == "1":
+        local %= torch.cuda.device_count()
+    backend = os.environ.get("ADACOMP_BENCH_BACKEND", "nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    B.adacomp_set_device(local)
+    if world > 1:
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n, L_T = 1 << min(a.log2n, 28), a.L_T
+    K, W = a.steps, max(a.warmup, 3)
+    stream = torch.cuda.current_stream()
+    gen = torch.Generator(device=dev)
+    cap = B.adacomp_packed_capacity(n, L_T)
+    residue = torch.zeros(n, device=dev)
+    packed = torch.empty(cap, dtype=torch.uint8, device=dev)
+    count = torch.zeros(2, dtype=torch.int64, device=dev)
+    recv = torch.empty(world * cap, dtype=torch.uint8, device=dev) if world > 1 else None
+    dW = torch.empty(n, device=dev)
+    dst = torch.empty(n, device=dev)
+    for step in range(PREWARM_STEPS + 1):
+        gen.manual_seed(ranks.learner_seed(rank, 0, step))
+        dW.normal_(0.0, SIGMA, generator=gen)
+        if step < PREWARM_STEPS:
+            B.adacomp_compress(dW, residue, n, L_T, packed, count, stream)
+    snap = residue.clone()
+    torch.cuda.synchronize()
+    gpu_index = (torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                 else os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    sampler = ClockSampler(gpu_index)
+    if rank == 0:
+        sampler.start()
+    evs, wire = [], 0
+    for it in range(W + K):
+        if it == W:
+            barrier()
+        residue.copy_(snap)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record(stream)
+        B.adacomp_compress(dW, residue, n, L_T, packed, count, stream)
+        e[1].record(stream)
+        used = int(count[1])                    # exchange() sends the sizes first: the host needs this one
+        streams = exchange(packed, used, recv=recv)
+        e[2].record(stream)
+        B.adacomp_decompress_accumulate_ex(streams, world, dst, n, L_T, stream)
+        e[3].record(stream)
+        wire = sum(int(t.numel()) for t in streams)
+        if it >= W:
+            evs.append(e)
+    barrier()
+    clocks = ClockSampler.merge([sampler.stop()]) if rank == 0 else None
+    t = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs) for i in range(3)]
+    total_ms = sum(e[0].elapsed_time(e[3]) for e in evs)
+    v = ranks.max_over_ranks([total_ms] + t, device=dev if backend == "nccl" else None)
+    crc = zlib.crc32(dst.cpu().numpy().tobytes())
+    same = True
+    if world > 1:
+        mine = torch.tensor([crc], dtype=torch.int64, device=dev if backend == "nccl" else None)
+        every = torch.empty(world, dtype=torch.int64, device=mine.device)
+        dist.all_gather_into_tensor(every, mine)
+        same = len({int(c) for c in every.cpu()}) == 1
+    status = B.adacomp_device_status(stream)
+    if rank == 0:
+        ms = v[0] / K
+        line = {
+            "metric": METRIC, "value": ranks.whole_job_throughput(4.0 * n, world, ms), "unit": "GB/s", "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"pack -> exchange -> decode-sum with every rank a learner: flat fp32 gradient n=2^{n.bit_length() - 1} "
+                                   f"per rank, L_T={L_T}, dW~N(0,1e-3), residue pre-warmed {PREWARM_STEPS} steps",
+                       "exchange": f"all-gather of the sizes, then of the streams padded to the longest ({backend}); received "
+                                   "streams land in the rank's own memory before the decoder reads them",
+                       "l2": "arrays far beyond the 126 MB L2" if 4 * n > (1 << 29) else "small case"},
+            "pack_ms": v[1], "exchange_ms": v[2], "decode_sum_ms": v[3], "stream_bytes_received_per_rank": wire,
+            "same_sum_on_every_rank": same, "device_status": status, "clocks": clocks,
+            "gpu_launches": K * 4,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_rate_curve(a):
     """Compression rate against the bin length L_T (the axis of the paper's rate figures) on the synthetic
     Gaussian run: for each L_T, k learners are pre-warmed PREWARM_STEPS steps from a zero residue, then one
@@ -833,6 +941,8 @@ def main():
         run_reference(a)
     elif a.workload == "ratecurve":
         run_rate_curve(a)
+    elif a.workload == "exchange":
+        run_exchange(a)
     elif a.workload != "sweep":
         run_multi_workload(a)
     else:

@@ -44,8 +44,12 @@ def exchange(packed: torch.Tensor, bytes_used: int, group=None,
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
         return [packed[:bytes_used]]
     world = dist.get_world_size(group)
-    mine = torch.tensor([int(bytes_used)], dtype=torch.int64, device=packed.device)
-    sizes_t = torch.empty(world, dtype=torch.int64, device=packed.device)
+    # gloo gathers host tensors only: device streams are staged through the host for it (how the ranks of a
+    # one-GPU machine are tested); NCCL gathers device tensors in place
+    staged = packed.is_cuda and dist.get_backend(group) == "gloo"
+    wire = torch.device("cpu") if staged else packed.device
+    mine = torch.tensor([int(bytes_used)], dtype=torch.int64, device=wire)
+    sizes_t = torch.empty(world, dtype=torch.int64, device=wire)
     dist.all_gather_into_tensor(sizes_t, mine, group=group)
     sizes = [int(v) for v in sizes_t.cpu()]
     step = padded_size(sizes)
@@ -55,6 +59,10 @@ def exchange(packed: torch.Tensor, bytes_used: int, group=None,
         recv = torch.empty(world * step, dtype=torch.uint8, device=packed.device)
     elif recv.numel() < world * step or recv.dtype != torch.uint8 or recv.device != packed.device:
         raise ValueError("recv buffer too small, of the wrong type or on another device")
-    if step:
+    if step and staged:
+        host = torch.empty(world * step, dtype=torch.uint8)
+        dist.all_gather_into_tensor(host, packed[:step].cpu(), group=group)
+        recv[:world * step].copy_(host)
+    elif step:
         dist.all_gather_into_tensor(recv[:world * step], packed[:step], group=group)
     return [recv[r * step:r * step + sizes[r]] for r in range(world)]
