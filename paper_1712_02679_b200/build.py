@@ -1,43 +1,70 @@
-"""Build libadacomp.so in-tree with nvcc for sm_100a (no GPU needed to compile)."""
+"""Build libadacomp.so in-tree with nvcc for sm_100a (no GPU needed to compile).
+
+The library is several translation units (paper_1712_02679_b200/csrc/*.cu) compiled side by side (whole-program
+device code each, no relocatable device code) and linked into one shared object."""
 from __future__ import annotations
 
+import glob
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SRC = os.path.join(HERE, "csrc", "adacomp.cu")
+CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libadacomp.so")
+OBJ = os.path.join(HERE, "build")
 
+ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+    *ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
     # IEEE arithmetic: no fast-math, denormals kept; the kernels use explicit
     # __fadd_rn / __fsub_rn so no multiply-add contraction can change a result.
     "-ftz=false", "-prec-div=true", "-prec-sqrt=true",
 ]
 
 
-def _sources():
-    out = [SRC, os.path.join(INCLUDE, "adacomp.h")]
-    return [p for p in out if os.path.exists(p)]
+def _units():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    newest = max(os.path.getmtime(p) for p in _sources())
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
-        return LIB
+def _headers():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h"))
+                  + [os.path.join(INCLUDE, "adacomp.h")])
+
+
+def build(force: bool = False, verbose: bool = False, extra=()) -> str:
+    units = _units()
+    newest_header = max(os.path.getmtime(p) for p in _headers())
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    todo, objs = [], []
+    for src in units:
+        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        objs.append(obj)
+        stale = (force or not os.path.exists(obj)
+                 or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header))
+        if stale:
+            todo.append((src, obj))
+    if not todo and os.path.exists(LIB) and os.path.getmtime(LIB) >= max(os.path.getmtime(o) for o in objs):
+        return LIB
+
+    def compile_one(job):
+        src, obj = job
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", INCLUDE, "-I", CSRC, "-c", "-o", obj, src]
+        if verbose:
+            cmd[1:1] = ["-Xptxas", "-v"]
+        subprocess.run(cmd, check=True)
+
+    with ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 4) or 1) as pool:
+        list(pool.map(compile_one, todo))
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-o", tmp, SRC]
-    if verbose:
-        cmd[1:1] = ["-Xptxas", "-v"]
-    subprocess.run(cmd, check=True)
+    subprocess.run([nvcc, *ARCH, "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-o", tmp, *objs], check=True)
     os.replace(tmp, LIB)
     return LIB
 
 
 if __name__ == "__main__":
     import sys
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force="-f" in sys.argv or "-v" in sys.argv, verbose="-v" in sys.argv))
