@@ -84,6 +84,11 @@ extern "C" {
 #define ADACOMP_FLAG_LITERAL 1u       /* Algorithm 2 as printed: |H| >= g_max only */
 #define ADACOMP_FLAG_GENERIC_PATH 256u /* use the any-L_T kernel even where a specialised one exists */
 
+/* gradient formats (adacomp_options.grad_type): values narrower than binary32 are widened exactly as they are read */
+#define ADACOMP_GRAD_F32 0u
+#define ADACOMP_GRAD_BF16 1u
+#define ADACOMP_GRAD_F16 2u
+
 /* Library ABI version (ADACOMP_VERSION).  Host only, no CUDA call. */
 int adacomp_version(void);
 
@@ -178,6 +183,39 @@ int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint3
  */
 int adacomp_compress_bf16(const void *grad_bf16, float *residue, uint64_t n, uint32_t L_T,
                           void *packed_out, uint64_t *count_out, void *stream);
+
+/*
+ * The same for a gradient in IEEE binary16 (half precision): every value, subnormals, infinities and NaNs
+ * included, has an exact binary32 counterpart, which is what Algorithm 2 then sees.
+ *   grad_f16   device, n binary16 values (uint16 bit patterns), 16-byte aligned; read-only.
+ */
+int adacomp_compress_f16(const void *grad_f16, float *residue, uint64_t n, uint32_t L_T,
+                         void *packed_out, uint64_t *count_out, void *stream);
+
+/*
+ * pack() with every option at once: the variants above are this call with one field set.
+ *   flags       ADACOMP_FLAG_* bits (adacomp_compress_ex).
+ *   grad_type   ADACOMP_GRAD_*: what `grad` points to (adacomp_compress_bf16 / _f16).
+ *   factor      0: Algorithm 2's H = G + dW; else H = residue + factor * dW (adacomp_compress_scaled).
+ *   lazy_state  NULL, or the layer's lazy-scale state (adacomp_compress_lazy).
+ * Combinations: a factor and a 16-bit gradient go with lazy-scale mode wherever that mode exists
+ * (L_T 41..1000 and the multiples of 4 up to 4000), except a 16-bit gradient at a bin length whose tiles
+ * are an odd multiple of 4 elements (L_T 43, 45, 47, ... : their 16-bit tiles do not start on the 16-byte
+ * boundaries that bulk copies need; eager mode takes the any-L_T kernel there, lazy-scale mode returns
+ * ADACOMP_ERR_UNSUPPORTED); flags exclude lazy-scale mode.  `opt` NULL means all zero.  Other arguments,
+ * results and errors as for adacomp_compress.
+ */
+typedef struct {
+    uint32_t flags;
+    uint32_t grad_type;
+    float factor;
+    uint32_t reserved;      /* must be 0 */
+    void *lazy_state;
+} adacomp_options;
+
+int adacomp_compress_opt(const void *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                         uint64_t *count_out, const adacomp_options *opt, void *stream);
+
 
 /*
  * unpack() of k learners' streams and their sum (Algorithm 1: unpack(), and the

@@ -187,6 +187,19 @@ def pack_bf16(dW_bits: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0
     return pack(bf16_to_f32(dW_bits), residue, L_T, flags=flags, want_gmax=want_gmax)
 
 
+def f16_to_f32(bits: np.ndarray) -> np.ndarray:
+    """IEEE binary16 bit patterns (uint16) as float32 values.  Every binary16 value (subnormals, infinities
+    and NaNs included) is a binary32 value, so the conversion is exact; numpy's cast is that conversion."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return b.view(np.float16).astype(np.float32)
+
+
+def pack_f16(dW_bits: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0, want_gmax: bool = False,
+             factor: float = 0.0) -> Packed:
+    """pack() for a gradient that arrives in binary16: widened exactly, then Algorithm 2 as for any binary32 gradient."""
+    return pack(f16_to_f32(dW_bits), residue, L_T, flags=flags, want_gmax=want_gmax, factor=factor)
+
+
 def average_adam(streams: Sequence[np.ndarray], n: int, weights: np.ndarray, m: np.ndarray, v: np.ndarray,
                  step_size: float, beta1: float, beta2: float, eps: float):
     """unpack(), averageGradients() and an Adam step for one layer (the paper reports AdaComp with Adam too,

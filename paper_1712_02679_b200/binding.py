@@ -38,6 +38,14 @@ class adacomp_layer_desc(C.Structure):
                 ("count_out", C.c_void_p)]
 
 
+class adacomp_options(C.Structure):
+    _fields_ = [("flags", C.c_uint32), ("grad_type", C.c_uint32), ("factor", C.c_float), ("reserved", C.c_uint32),
+                ("lazy_state", C.c_void_p)]
+
+
+ADACOMP_GRAD_F32, ADACOMP_GRAD_BF16, ADACOMP_GRAD_F16 = 0, 1, 2
+_GRAD_DTYPES = {ADACOMP_GRAD_F32: torch.float32, ADACOMP_GRAD_BF16: torch.bfloat16, ADACOMP_GRAD_F16: torch.float16}
+
 _lib: Optional[C.CDLL] = None
 
 
@@ -77,6 +85,12 @@ def lib() -> C.CDLL:
         L.adacomp_decompress_average_adam_multi.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                                             C.c_void_p, C.c_void_p, C.c_uint32, C.c_float, C.c_float,
                                                             C.c_float, C.c_float, C.c_void_p]
+        L.adacomp_compress_f16.restype = C.c_int
+        L.adacomp_compress_f16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]
+        L.adacomp_compress_opt.restype = C.c_int
+        L.adacomp_compress_opt.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
+                                           C.POINTER(adacomp_options), C.c_void_p]
         L.adacomp_compress_bf16.restype = C.c_int
         L.adacomp_compress_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p]
@@ -202,6 +216,27 @@ def adacomp_compress_bf16(grad_bf16, residue, n: int, L_T: int, packed_out, coun
                                        _dev_ptr(packed_out, "packed_out", torch.uint8),
                                        _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
            "adacomp_compress_bf16")
+
+
+def adacomp_compress_f16(grad_f16, residue, n: int, L_T: int, packed_out, count_out, stream=None) -> None:
+    """pack() of a binary16 gradient (widened exactly on load); residue and stream as for a binary32 gradient."""
+    _check(lib().adacomp_compress_f16(_dev_ptr(grad_f16, "grad_f16", torch.float16),
+                                      _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                      _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                      _dev_ptr(count_out, "count_out", torch.int64), _stream(stream)),
+           "adacomp_compress_f16")
+
+
+def adacomp_compress_opt(grad, residue, n: int, L_T: int, packed_out, count_out, flags: int = 0,
+                         grad_type: int = ADACOMP_GRAD_F32, factor: float = 0.0, lazy_state=None, stream=None) -> None:
+    """pack() with every option at once (flags, gradient format, the selection's factor, lazy-scale state)."""
+    opt = adacomp_options(int(flags), int(grad_type), float(factor), 0,
+                          _dev_ptr(lazy_state, "lazy_state", torch.uint8) if lazy_state is not None else None)
+    _check(lib().adacomp_compress_opt(_dev_ptr(grad, "grad", _GRAD_DTYPES.get(int(grad_type))),
+                                      _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
+                                      _dev_ptr(packed_out, "packed_out", torch.uint8),
+                                      _dev_ptr(count_out, "count_out", torch.int64), C.byref(opt), _stream(stream)),
+           "adacomp_compress_opt")
 
 
 def adacomp_compress_scaled(grad, residue, n: int, L_T: int, packed_out, count_out, factor: float, stream=None) -> None:

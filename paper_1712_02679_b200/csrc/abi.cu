@@ -374,7 +374,24 @@ int adacomp_compress_bf16(const void *grad_bf16, float *residue, uint64_t n, uin
                           uint64_t *count_out, void *stream)
 {
     return compress_impl(static_cast<const float *>(grad_bf16), residue, n, L_T, packed_out, count_out, stream, 0, nullptr,
-                         nullptr, 0.f, true);
+                         nullptr, 0.f, ADACOMP_GRAD_BF16);
+}
+
+int adacomp_compress_f16(const void *grad_f16, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                         uint64_t *count_out, void *stream)
+{
+    return compress_impl(static_cast<const float *>(grad_f16), residue, n, L_T, packed_out, count_out, stream, 0, nullptr,
+                         nullptr, 0.f, ADACOMP_GRAD_F16);
+}
+
+int adacomp_compress_opt(const void *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
+                         uint64_t *count_out, const adacomp_options *opt, void *stream)
+{
+    const adacomp_options none = {0u, ADACOMP_GRAD_F32, 0.f, 0u, nullptr};
+    const adacomp_options &o = opt ? *opt : none;
+    if (o.reserved != 0u) return ADACOMP_ERR_FLAGS;
+    return compress_impl(static_cast<const float *>(grad), residue, n, L_T, packed_out, count_out, stream, o.flags, nullptr,
+                         o.lazy_state, o.factor, o.grad_type);
 }
 
 int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,

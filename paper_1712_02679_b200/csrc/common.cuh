@@ -2,6 +2,7 @@
 // helpers, and the mbarrier / bulk-copy (TMA) wrappers (no cluster multicast anywhere).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -83,9 +84,11 @@ __host__ __device__ inline Geometry make_geometry(u64 n, u32 L_T)
 __device__ inline void raise_status(u32 bits) { atomicOr(&g_status, bits); }
 
 // Element i of a gradient that is binary32, or bfloat16 widened exactly (sixteen zero bits appended).
-__device__ inline float load_grad(const float *grad, u64 i, u32 bf16)
+__device__ inline float load_grad(const float *grad, u64 i, u32 grad_type)
 {
-    return bf16 ? __uint_as_float((u32)reinterpret_cast<const unsigned short *>(grad)[i] << 16) : grad[i];
+    if (grad_type == ADACOMP_GRAD_BF16) return __uint_as_float((u32)reinterpret_cast<const unsigned short *>(grad)[i] << 16);
+    if (grad_type == ADACOMP_GRAD_F16) return __half2float(__ushort_as_half(reinterpret_cast<const unsigned short *>(grad)[i]));
+    return grad[i];
 }
 
 __device__ inline u32 warp_inclusive_scan(u32 v, int lane)

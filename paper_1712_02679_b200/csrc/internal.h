@@ -31,8 +31,8 @@ void init_decode_batch_info(DeviceInfo &d);     // decode_batch.cu
 
 // pack_fast_a.cu .. pack_fast_d.cu: the instances of the pipelined tile pass, a few bin lengths per file.
 // With `args` null: allows the kernels their dynamic shared memory (false: some kernel cannot be launched).
-// Else: launches the kernel that takes args->geo.L_T (lazy-scale when args->lazy_state is set, bfloat16
-// gradient when args->grad_bf16 is) and returns true, or returns false when the bin length is another file's.
+// Else: launches the kernel that takes args->geo.L_T (lazy-scale when args->lazy_state is set, the gradient
+// format of args->grad_type) and returns true, or returns false when the bin length is another file's.
 bool fast_tile_pass_a(const PassArgs *args, unsigned grid, cudaStream_t st);
 bool fast_tile_pass_b(const PassArgs *args, unsigned grid, cudaStream_t st);
 bool fast_tile_pass_c(const PassArgs *args, unsigned grid, cudaStream_t st);
@@ -41,7 +41,7 @@ bool fast_tile_pass_d(const PassArgs *args, unsigned grid, cudaStream_t st);
 // pack.cu
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
-                  void *lazy_state = nullptr, float factor = 0.f, bool grad_bf16 = false,
+                  void *lazy_state = nullptr, float factor = 0.f, uint32_t grad_type = ADACOMP_GRAD_F32,
                   unsigned char *own_scratch = nullptr);
 int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                          uint64_t *count_out, void *stream);

@@ -107,12 +107,13 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 // `own_scratch` (optional): the scratch to use in place of the one behind the stream in packed_out.
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events, void *lazy_state,
-                  float factor, bool grad_bf16, unsigned char *own_scratch)
+                  float factor, uint32_t grad_type, unsigned char *own_scratch)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
     if (flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
     if (factor != 0.f && !(factor > 0.f && factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
+    if (grad_type > ADACOMP_GRAD_F16) return ADACOMP_ERR_FLAGS;
     if (misaligned(grad) || misaligned(residue) || misaligned(packed_out) ||
         (reinterpret_cast<uintptr_t>(count_out) & 7u))
         return ADACOMP_ERR_ALIGN;
@@ -120,7 +121,9 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     if (geo.n_bins >= (1ull << 31)) return ADACOMP_ERR_SIZE;
     unsigned char *lazy = static_cast<unsigned char *>(lazy_state);
     if (lazy) {
-        if (!(fast_L_T(L_T) || any_fast_L_T(L_T)) || flags != 0 || factor != 0.f || grad_bf16) return ADACOMP_ERR_UNSUPPORTED;
+        if (!(fast_L_T(L_T) || any_fast_L_T(L_T)) || flags != 0) return ADACOMP_ERR_UNSUPPORTED;
+        // (16-bit gradients: the any-bin form needs tiles of them to start on 16-byte boundaries)
+        if (grad_type != ADACOMP_GRAD_F32 && !fast_L_T(L_T) && geo.tile_elems % 8u != 0) return ADACOMP_ERR_UNSUPPORTED;
         if (misaligned(lazy)) return ADACOMP_ERR_ALIGN;
     }
 
@@ -140,11 +143,12 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_bf16 ? 1u : 0u};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_type};
         const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
         // (one-bin tiles fill the pipelined kernel's 4000-element stages only in part: below 2800 elements the
         // warp-per-part kernel is faster, measured; lazy-scale mode exists in the pipelined kernel only)
-        const bool any_fast = any_fast_L_T(L_T) && flags == 0 && !grad_bf16 && info->fast_ready &&
+        const bool any_fast = any_fast_L_T(L_T) && flags == 0 && info->fast_ready &&
+                              (grad_type == ADACOMP_GRAD_F32 || geo.tile_elems % 8u == 0) &&
                               (lazy || L_T <= 1000u || L_T >= 2800u);
         if (fast || any_fast) {
             const u64 cap = (u64)info->sms * 2;
@@ -219,7 +223,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
         g_static_scratch_addr[dev] = ptr;
     }
     // the same kernels, in the same order, as adacomp_compress: only the scratch is elsewhere
-    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, nullptr, 0.f, false,
+    return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, nullptr, 0.f, ADACOMP_GRAD_F32,
                          g_static_scratch_addr[dev]);
 }
 

@@ -6,22 +6,31 @@
 
 namespace adacomp_impl {
 
-// eager / lazy-scale / bfloat16-gradient forms of the kernel for one bin length
-template <int SPB, typename Word>
-inline bool fast_forms_allow()
+// the forms of the kernel for one bin length: eager / lazy-scale, each for the three gradient formats
+template <int SPB, typename Word, bool LAZY>
+inline bool fast_formats_allow()
 {
     const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
     const int bytes = (int)FastSmem::kBytes;
-    return cudaFuncSetAttribute(tile_pass_fast<SPB, Word, false, false>, at, bytes) == cudaSuccess &&
-           cudaFuncSetAttribute(tile_pass_fast<SPB, Word, true, false>, at, bytes) == cudaSuccess &&
-           cudaFuncSetAttribute(tile_pass_fast<SPB, Word, false, true>, at, bytes) == cudaSuccess;
+    return cudaFuncSetAttribute(tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_F32>, at, bytes) == cudaSuccess &&
+           cudaFuncSetAttribute(tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_BF16>, at, bytes) == cudaSuccess &&
+           cudaFuncSetAttribute(tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_F16>, at, bytes) == cudaSuccess;
+}
+template <int SPB, typename Word>
+inline bool fast_forms_allow() { return fast_formats_allow<SPB, Word, false>() && fast_formats_allow<SPB, Word, true>(); }
+
+template <int SPB, typename Word, bool LAZY>
+inline void fast_formats_launch(const PassArgs &a, unsigned grid, cudaStream_t st)
+{
+    if (a.grad_type == ADACOMP_GRAD_BF16) tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_BF16><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
+    else if (a.grad_type == ADACOMP_GRAD_F16) tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_F16><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
+    else tile_pass_fast<SPB, Word, LAZY, ADACOMP_GRAD_F32><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
 }
 template <int SPB, typename Word>
 inline void fast_forms_launch(const PassArgs &a, unsigned grid, cudaStream_t st)
 {
-    if (a.lazy_state) tile_pass_fast<SPB, Word, true, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
-    else if (a.grad_bf16) tile_pass_fast<SPB, Word, false, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
-    else tile_pass_fast<SPB, Word, false, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(a);
+    if (a.lazy_state) fast_formats_launch<SPB, Word, true>(a, grid, st);
+    else fast_formats_launch<SPB, Word, false>(a, grid, st);
 }
 
 }  // namespace adacomp_impl

@@ -6,23 +6,15 @@ namespace adacomp_impl {
 bool fast_tile_pass_d(const PassArgs *args, unsigned grid, cudaStream_t st)
 {
     if (!args)
-        return fast_forms_allow<40, unsigned short>() &&
-               cudaFuncSetAttribute(tile_pass_fast<0, unsigned char, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FastSmem::kBytes) == cudaSuccess &&
-               cudaFuncSetAttribute(tile_pass_fast<0, unsigned short, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FastSmem::kBytes) == cudaSuccess &&
-               cudaFuncSetAttribute(tile_pass_fast<0, unsigned char, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FastSmem::kBytes) == cudaSuccess &&
-               cudaFuncSetAttribute(tile_pass_fast<0, unsigned short, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FastSmem::kBytes) == cudaSuccess;
+        return fast_forms_allow<40, unsigned short>() && fast_forms_allow<0, unsigned char>() && fast_forms_allow<0, unsigned short>();
     switch (args->geo.L_T) {
     case 1000u: fast_forms_launch<40, unsigned short>(*args, grid, st); return true;
     default:
-        // every other bin length of the pipelined kernel: its any-bin form (fp32 gradient)
-        if (!any_fast_L_T(args->geo.L_T) || args->grad_bf16) return false;
-        if (args->geo.L_T <= 64u) {
-            if (args->lazy_state) tile_pass_fast<0, unsigned char, true, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(*args);
-            else tile_pass_fast<0, unsigned char, false, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(*args);
-        } else {
-            if (args->lazy_state) tile_pass_fast<0, unsigned short, true, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(*args);
-            else tile_pass_fast<0, unsigned short, false, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(*args);
-        }
+        // every other bin length of the pipelined kernel: its any-bin form (16-bit gradients only where a tile of
+        // them is a multiple of 16 bytes, which the caller has checked)
+        if (!any_fast_L_T(args->geo.L_T)) return false;
+        if (args->geo.L_T <= 64u) fast_forms_launch<0, unsigned char>(*args, grid, st);
+        else fast_forms_launch<0, unsigned short>(*args, grid, st);
         return true;
     }
 }

@@ -32,7 +32,7 @@ struct PassArgs {
     u32 literal;
     unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
     float factor;               // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW (Section 2.4's scale-factor)
-    u32 grad_bf16;              // `grad` points to bfloat16 values (widened exactly on load)
+    u32 grad_type;              // ADACOMP_GRAD_*: `grad` points to binary32 values, or to bfloat16 / binary16 ones (widened exactly on load)
 };
 
 // Lazy-mode state: 64-byte header, then one u32 per 25-element segment (bit j = element j
@@ -64,8 +64,9 @@ struct FastSmem {
 };
 static_assert(FastSmem::kAccAt % 8 == 0, "accumulator must be 8-byte aligned");
 
-// BF16: the gradient arrives as bfloat16 (8000-byte tiles, widened as they are read).
-template <int SPB, typename Word, bool LAZY, bool BF16 = false>
+// GT: ADACOMP_GRAD_F32, or the gradient arrives in 16 bits per value (bfloat16 / binary16: tiles of half the
+// bytes, widened exactly as they are read).
+template <int SPB, typename Word, bool LAZY, int GT = 0>
 __global__ void __launch_bounds__(kFastThreads, 2)
 tile_pass_fast(PassArgs a)
 {
@@ -83,7 +84,7 @@ tile_pass_fast(PassArgs a)
     const bool service = warp == 5;
     const Geometry &geo = a.geo;
     constexpr bool ANY = SPB == 0;
-    static_assert(!ANY || !BF16, "the any-L_T form takes fp32 gradients");
+    constexpr bool G16 = GT != 0;       // 16-bit gradient values (ANY: the launcher sees to it that a tile of them is a multiple of 16 bytes)
     constexpr int kBins = ANY ? kSmallBins : kTileSegs / (ANY ? 1 : SPB);
     const int T = ANY ? (int)geo.tile_elems : kFastTile;            // elements of a tile (a multiple of 4)
     const int TB = ANY ? (int)geo.tile_bins : kBins;
@@ -146,7 +147,7 @@ tile_pass_fast(PassArgs a)
         if (i >= my_tiles || tile >= full_tiles) return;
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        const u32 grad_bytes = BF16 ? kTileBytes / 2 : tile_bytes;
+        const u32 grad_bytes = G16 ? tile_bytes / 2 : tile_bytes;
         mbar_arrive_expect_tx(bar, grad_bytes + tile_bytes + (LAZY ? kMaskBytes : 0u));
         bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)grad_bytes, grad_bytes, bar);
         bulk_load(st + kTileBytes, a.residue + tile * (u64)T, tile_bytes, bar);
@@ -178,8 +179,13 @@ tile_pass_fast(PassArgs a)
             // the ragged last tile of the tensor: plain loads, zero fill past the end
             for (int e = tid; e < kFastTile; e += kFastThreads) {
                 float d = 0.f, r = 0.f;
-                if (e < elems) { d = load_grad(a.grad, base + e, BF16); r = a.residue[base + e]; }
-                if (BF16) reinterpret_cast<unsigned short *>(s_d)[e] = (unsigned short)(__float_as_uint(d) >> 16);
+                unsigned short d16 = 0;
+                if (e < elems) {
+                    if (G16) d16 = reinterpret_cast<const unsigned short *>(a.grad)[base + e];
+                    else d = a.grad[base + e];
+                    r = a.residue[base + e];
+                }
+                if (G16) reinterpret_cast<unsigned short *>(s_d)[e] = d16;
                 else s_d[e] = d;
                 s_r[e] = r;
             }
@@ -197,11 +203,11 @@ tile_pass_fast(PassArgs a)
             const float *pr = s_r + tid * kSeg;
             float m = 0.f, m1 = 0.f;
             const u32 prev = LAZY ? s_prev[tid] : 0u;
-            // bfloat16: the segment's 50 bytes start on a 4-byte boundary for even threads and two bytes
+            // 16-bit values: the segment's 50 bytes start on a 4-byte boundary for even threads and two bytes
             // past one for odd threads; thirteen aligned 32-bit loads cover them either way, and a funnel
             // shift by 0 or 16 bits lines the pairs up (half as many shared-memory accesses as 25 16-bit loads)
-            u32 pair[BF16 ? 13 : 1];
-            if (BF16) {
+            u32 pair[G16 ? 13 : 1];
+            if (G16) {
                 const u32 *pw = reinterpret_cast<const u32 *>(s_d) + ((tid * kSeg) >> 1);
                 const u32 sh = (tid & 1) * 16u;
                 u32 w[14];
@@ -213,7 +219,10 @@ tile_pass_fast(PassArgs a)
             }
 #pragma unroll
             for (int j = 0; j < kSeg; j++) {
-                float d = BF16 ? __uint_as_float((j & 1) ? pair[j >> 1] & 0xffff0000u : pair[j >> 1] << 16) : pd[j];
+                float d;
+                if (GT == ADACOMP_GRAD_BF16) d = __uint_as_float((j & 1) ? pair[j >> 1] & 0xffff0000u : pair[j >> 1] << 16);
+                else if (GT == ADACOMP_GRAD_F16) d = __half2float(__ushort_as_half((unsigned short)((j & 1) ? pair[j >> 1] >> 16 : pair[j >> 1] & 0xffffu)));
+                else d = pd[j];
                 float r = pr[j];
                 if (ANY && j >= vcount) d = r = 0.f;        // past the tile's end
                 if (LAZY) {
@@ -377,7 +386,7 @@ struct TileIo {                 // the buffers of one layer, as the generic tile
     unsigned char *packed, *scratch;
     u32 literal;
     float factor;               // as in PassArgs
-    u32 grad_bf16;
+    u32 grad_type;
 };
 
 template <typename Word>
@@ -407,7 +416,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
 
     // G and H of the tile: four elements a thread and step where 4 divides the tile's length (every tile, and
     // the G array behind the H array in shared memory, then start on a 16-byte boundary)
-    const int quads = (T & 3) == 0 && !a.grad_bf16 ? elems >> 2 : 0;
+    const int quads = (T & 3) == 0 && !a.grad_type ? elems >> 2 : 0;
     for (int i = tid; i < quads; i += kGenericThreads) {
         const float4 d = reinterpret_cast<const float4 *>(a.grad + base)[i];
         const float4 r = reinterpret_cast<const float4 *>(a.residue + base)[i];
@@ -423,7 +432,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
     }
     for (int i = 4 * quads + tid; i < T; i += kGenericThreads) {
         float d = 0.f, r = 0.f;
-        if (i < elems) { d = load_grad(a.grad, base + i, a.grad_bf16); r = a.residue[base + i]; }
+        if (i < elems) { d = load_grad(a.grad, base + i, a.grad_type); r = a.residue[base + i]; }
         const float g = __fadd_rn(r, d);
         s_g[i] = g;
         s_d[i] = a.factor != 0.f ? __fadd_rn(r, __fmul_rn(a.factor, d)) : __fadd_rn(g, d);      // H: dW is not needed again
@@ -550,7 +559,7 @@ __device__ void generic_tile_one_bin(const TileIo &a, const Geometry &geo, u64 t
     };
     float m = 0.f;
     // (four elements a step where the bin starts on a 16-byte boundary)
-    const int quads = (base & 3u) == 0 && !a.grad_bf16 ? elems >> 2 : 0;
+    const int quads = (base & 3u) == 0 && !a.grad_type ? elems >> 2 : 0;
     for (int i = tid; i < quads; i += kGenericThreads) {
         const float4 d = reinterpret_cast<const float4 *>(a.grad + base)[i];
         const float4 r = reinterpret_cast<const float4 *>(a.residue + base)[i];
@@ -567,7 +576,7 @@ __device__ void generic_tile_one_bin(const TileIo &a, const Geometry &geo, u64 t
         float k = 0.f;
         if (i < elems) {
             float g;
-            k = key_of(a.residue[base + i], load_grad(a.grad, base + i, a.grad_bf16), g);
+            k = key_of(a.residue[base + i], load_grad(a.grad, base + i, a.grad_type), g);
             m = fmaxf(m, fabsf(g));
             a.residue[base + i] = g;
         }
@@ -635,7 +644,7 @@ tile_pass_generic(PassArgs a)
     const int tid = threadIdx.x;
     if (tid < kWindows + 1) s_acc[tid] = 0;
     __syncthreads();
-    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_bf16};
+    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_type};
     for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x) {
         if (a.geo.tile_bins == 1u && sizeof(Word) == 2) generic_tile_one_bin<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
         else generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
