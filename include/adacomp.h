@@ -399,6 +399,18 @@ int adacomp_compress_multi_lazy(const adacomp_layer_desc *layers, void *const *s
                                 void *stream);
 
 /*
+ * adacomp_compress_multi with options per layer: opts (HOST array of n_layers adacomp_options, or NULL for
+ * none) gives layer t its gradient format (layers[t].grad then points to values of that format), the factor of
+ * its selection test and, when lazy_state is set, lazy-scale mode with that state.  opts[t].flags must be 0:
+ * a layer's flags are those of its descriptor.  Layers share launches as in adacomp_compress_multi; a list
+ * in which only some layers have a lazy-scale state is packed layer by layer.  Results are those of
+ * adacomp_compress_opt layer by layer, bit for bit; every layer is checked before anything is launched.
+ */
+int adacomp_compress_multi_opt(const adacomp_layer_desc *layers, const adacomp_options *opts, uint32_t n_layers,
+                               void *stream);
+
+
+/*
  * unpack()-and-sum of every layer: packed[t * k_streams + l] (HOST array) is
  * learner l's stream of layer t, dst[t] (HOST array of device pointers) its output.
  */

@@ -88,6 +88,9 @@ def lib() -> C.CDLL:
         L.adacomp_compress_f16.restype = C.c_int
         L.adacomp_compress_f16.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                            C.c_void_p]
+        L.adacomp_compress_multi_opt.restype = C.c_int
+        L.adacomp_compress_multi_opt.argtypes = [C.POINTER(adacomp_layer_desc), C.POINTER(adacomp_options), C.c_uint32,
+                                                 C.c_void_p]
         L.adacomp_compress_opt.restype = C.c_int
         L.adacomp_compress_opt.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p,
                                            C.POINTER(adacomp_options), C.c_void_p]
@@ -419,7 +422,7 @@ def make_layer_descs(layers: Sequence[dict]):
     """HOST array of adacomp_layer_desc from dicts with the struct's field names."""
     arr = (adacomp_layer_desc * max(len(layers), 1))()
     for i, d in enumerate(layers):
-        arr[i].grad = _dev_ptr(d["grad"], "grad", torch.float32)
+        arr[i].grad = _dev_ptr(d["grad"], "grad", _GRAD_DTYPES.get(int(d.get("grad_type", 0))))
         arr[i].residue = _dev_ptr(d["residue"], "residue", torch.float32)
         arr[i].n = int(d["n"])
         arr[i].L_T = int(d["L_T"])
@@ -445,6 +448,17 @@ def adacomp_compress_multi_lazy(layers, states, n_layers: int, stream=None) -> N
         states = make_pointer_array(states, torch.uint8)
     _check(lib().adacomp_compress_multi_lazy(layers, states, int(n_layers), _stream(stream)),
            "adacomp_compress_multi_lazy")
+
+
+def adacomp_compress_multi_opt(layers: Sequence[dict], n_layers: int, stream=None) -> None:
+    """layers: dicts with the descriptor's fields and, optionally, grad_type, factor and lazy_state."""
+    descs = make_layer_descs(layers)
+    opts = (adacomp_options * max(len(layers), 1))()
+    for i, d in enumerate(layers):
+        st = d.get("lazy_state")
+        opts[i] = adacomp_options(0, int(d.get("grad_type", 0)), float(d.get("factor", 0.0)), 0,
+                                  _dev_ptr(st, "lazy_state", torch.uint8) if st is not None else None)
+    _check(lib().adacomp_compress_multi_opt(descs, opts, int(n_layers), _stream(stream)), "adacomp_compress_multi_opt")
 
 
 def make_pointer_array(tensors: Sequence[torch.Tensor], dtype):

@@ -283,12 +283,30 @@ int adacomp_decompress_accumulate_host(const void *const *packed_host, const uin
     return cudaStreamSynchronize(st) == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 
-// `states` (optional): lazy-scale mode, states[t] the state of layer t.
-static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *states, uint32_t n_layers, void *stream)
+// `states` (optional): lazy-scale mode, states[t] the state of layer t.  `opts` (optional): per layer the gradient
+// format and the selection's factor (and, in place of `states`, the lazy-scale state); its flags are not used,
+// the layer's own are.
+static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *states, uint32_t n_layers, void *stream,
+                               const adacomp_options *opts = nullptr)
 {
     if (n_layers && !layers) return ADACOMP_ERR_NULL;
+    auto state_of = [&](uint32_t t) -> void * { return states ? states[t] : opts ? opts[t].lazy_state : nullptr; };
+    auto factor_of = [&](uint32_t t) { return opts ? opts[t].factor : 0.f; };
+    auto type_of = [&](uint32_t t) { return opts ? opts[t].grad_type : (uint32_t)ADACOMP_GRAD_F32; };
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
+        if (opts) {
+            const adacomp_options &o = opts[t];
+            if (o.reserved != 0u || o.flags != 0u || o.grad_type > ADACOMP_GRAD_F16) return ADACOMP_ERR_FLAGS;
+            if (o.factor != 0.f && !(o.factor > 0.f && o.factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
+            if (o.lazy_state) {
+                if (misaligned(o.lazy_state)) return ADACOMP_ERR_ALIGN;
+                if (d.flags != 0 || !(fast_L_T(d.L_T) || any_fast_L_T(d.L_T))) return ADACOMP_ERR_UNSUPPORTED;
+                if (o.grad_type != ADACOMP_GRAD_F32 && !fast_L_T(d.L_T) && d.L_T >= 1u && d.L_T <= ADACOMP_MAX_L_T &&
+                    make_geometry(d.n, d.L_T).tile_elems % 8u != 0)
+                    return ADACOMP_ERR_UNSUPPORTED;
+            }
+        }
         if (!d.packed_out || !d.count_out || (d.n && (!d.grad || !d.residue))) return ADACOMP_ERR_NULL;
         if (d.L_T == 0 || d.L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
         if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
@@ -311,12 +329,21 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
     static thread_local BatchArgs batch;
     batch.n_layers = 0;
     batch.total_tiles = 0;
+    // (a batch is eager or lazy-scale as a whole: with per-layer options the layers of either kind go to the
+    // single-layer path unless all of them are lazy-scale or none is)
+    bool any_lazy = false, all_lazy = n_layers > 0;
+    for (uint32_t t = 0; t < n_layers; t++) {
+        any_lazy = any_lazy || state_of(t) != nullptr;
+        all_lazy = all_lazy && state_of(t) != nullptr;
+    }
+    const bool batch_lazy = any_lazy && all_lazy, mixed = any_lazy && !all_lazy;
     auto batched = [&](const adacomp_layer_desc &d) {
-        return info->batch_per_sm > 0 && batchable(d, *info) && (!states || info->batch_fast_ready);
+        return !mixed && info->batch_per_sm > 0 && batchable(d, *info) && (!batch_lazy || info->batch_fast_ready);
     };
     // (more layers than a table holds: batches of equal size, so that none is left with a layer or two)
     uint32_t to_batch = 0;
     for (uint32_t t = 0; t < n_layers; t++) to_batch += batched(layers[t]) ? 1u : 0u;
+    // (without the pipelined batch kernel the batch runs the any-L_T tile code, which takes every format too)
     const uint32_t n_batches = (to_batch + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
     const uint32_t per_batch = n_batches ? (to_batch + n_batches - 1) / n_batches : (uint32_t)kBatchMax;
     for (uint32_t t = 0; t < n_layers; t++) {
@@ -329,22 +356,29 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
             L.count_out = reinterpret_cast<u64 *>(d.count_out);
             L.geo = make_geometry(d.n, d.L_T);
             L.tile_first = batch.total_tiles;
+            L.grad_type = type_of(t);
+            L.factor = factor_of(t);
             L.pad = 0;
-            L.lazy = states ? static_cast<unsigned char *>(states[t]) : nullptr;
+            L.lazy = static_cast<unsigned char *>(state_of(t));
             batch.total_tiles += (u32)L.geo.n_tiles;
             if (batch.n_layers == per_batch) {
-                rc = launch_batch(batch, *info, st, states != nullptr);
+                rc = launch_batch(batch, *info, st, batch_lazy);
                 if (rc != ADACOMP_OK) return rc;
                 batch.n_layers = 0;
                 batch.total_tiles = 0;
             }
         } else {
             rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags, nullptr,
-                               states ? states[t] : nullptr);
+                               state_of(t), factor_of(t), type_of(t));
             if (rc != ADACOMP_OK) return rc;
         }
     }
-    return launch_batch(batch, *info, st, states != nullptr);
+    return launch_batch(batch, *info, st, batch_lazy);
+}
+
+int adacomp_compress_multi_opt(const adacomp_layer_desc *layers, const adacomp_options *opts, uint32_t n_layers, void *stream)
+{
+    return compress_multi_impl(layers, nullptr, n_layers, stream, opts);
 }
 
 int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream)

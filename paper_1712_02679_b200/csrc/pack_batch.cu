@@ -50,7 +50,7 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
             cur = li;
         }
         const BatchLayer &L = b.layer[li];
-        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, 0.f, 0u};
+        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, L.factor, L.grad_type};
         if (L.geo.w == 1u) generic_tile<unsigned char>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
         else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
     }
@@ -65,7 +65,9 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
 // to that layer's windows when the CTA leaves the layer.  Every layer here has 41 <= L_T <= 1000.
 // LAZY: lazy-scale mode, every layer with its own state (see tile_pass_fast); a layer whose state is not its
 // own is flagged, left untouched and reports empty tiles.
-template <int N, bool LAZY>
+// OPTS: some layer has a 16-bit gradient or a factor (else both are compile-time constants: plain lists keep
+// the shorter code).
+template <int N, bool LAZY, bool OPTS>
 __global__ void __launch_bounds__(kFastThreads, 2)
 batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
 {
@@ -73,6 +75,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     unsigned char *s_words = smem + FastSmem::kWordsAt;
     u32 *s_incl = reinterpret_cast<u32 *>(smem + FastSmem::kInclAt);
     u32 *s_wtot = reinterpret_cast<u32 *>(smem + FastSmem::kWtotAt);
+    float *s_segmax = reinterpret_cast<float *>(smem + FastSmem::kSegmaxAt);   // (layers whose bins are whole segments) the segments' maxima
     u32 *s_anymax = reinterpret_cast<u32 *>(smem + FastSmem::kBinmaxAt);    // [2][kSmallBins] bits of the bin maxima, by tile parity
     u32 *s_anycnt = s_anymax + 2 * kSmallBins;                               // [2][kSmallBins] words per bin
     u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
@@ -116,10 +119,13 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
         if (LAZY && !load_ok) return;                   // nothing of such a layer is read
         const u32 lt = gt - L.tile_first, T = L.geo.tile_elems;
         if ((u64)lt >= L.geo.n / T) return;             // a ragged last tile is read with plain loads
+        const bool g16 = OPTS && L.grad_type != ADACOMP_GRAD_F32;
+        if (g16 && T % 8u != 0) return;                 // 16-bit tiles off the 16-byte boundaries: plain loads as well
+        const u32 gbytes = g16 ? 2u * T : 4u * T;
         unsigned char *st = smem + (i % kStages) * kStageBytes;
         u64 *bar = &s_full[i % kStages];
-        mbar_arrive_expect_tx(bar, 8u * T + (LAZY ? kMaskBytes : 0u));
-        bulk_load(st, L.grad + (u64)lt * T, 4u * T, bar);
+        mbar_arrive_expect_tx(bar, gbytes + 4u * T + (LAZY ? kMaskBytes : 0u));
+        bulk_load(st, reinterpret_cast<const unsigned char *>(L.grad) + (u64)lt * gbytes, gbytes, bar);
         bulk_load(st + kTileBytes, L.residue + (u64)lt * T, 4u * T, bar);
         if (LAZY) bulk_load(st + 2 * kTileBytes, L.lazy + kLazyHeaderBytes + (u64)lt * kMaskBytes, kMaskBytes, bar);
         issued = i + 1;
@@ -133,6 +139,9 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     u32 phase = 0;                      // bit s: parity of stage s's next completion (ragged tiles use no barrier)
     int T = 0, TB = 0, b0 = 0, cut = kSeg, off0 = 0, vcount = 0;
     u32 full_tiles = 0, wbytes = 1;
+    u32 gtype = 0;                      // the layer's gradient format
+    float factor = 0.f;                 // the layer's factor of the selection test (0: two additions)
+    int SPB = 0;                        // (aligned) segments per bin
     bool aligned = false;               // every segment of the layer's tiles lies in one bin and exists whole
     bool layer_ok = true;               // (LAZY) the layer's state is its own
     u32 prev_scale_bits = 0;            // (LAZY) last step's scale of the layer
@@ -165,7 +174,16 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             off0 = e0 - b0 * Lt;
             cut = min(kSeg, Lt - off0);
             vcount = max(0, min(kSeg, T - e0));
+#ifdef ADACOMP_BATCH_NO_ALIGNED_FORM
+            aligned = false;
+#else
             aligned = T == kFastTile && Lt % kSeg == 0;     // (then cut = vcount = 25 in every thread)
+#endif
+            SPB = Lt / kSeg;
+            gtype = OPTS ? L.grad_type : (u32)ADACOMP_GRAD_F32;
+            factor = OPTS ? L.factor : 0.f;
+            // (16-bit gradient tiles that do not start on 16-byte boundaries: every tile by plain loads)
+            if (gtype != ADACOMP_GRAD_F32 && T % 8 != 0) full_tiles = 0;
             if (LAZY) {
                 layer_ok = state_ok(L);
                 if (layer_ok) {
@@ -197,7 +215,7 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
         float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
         float *s_r = s_d + kFastTile;
         const bool whole = lt < full_tiles;
-        const int elems = whole ? T : (int)(geo.n - base);
+        const int elems = whole ? T : (int)min((u64)T, geo.n - base);      // (plain loads: the ragged last tile, or 16-bit tiles off the 16-byte boundaries)
         u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
 
         if (whole) {
@@ -211,8 +229,14 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             // the ragged last tile of a layer: plain loads, zero fill past the end
             for (int e = tid; e < kFastTile; e += kFastThreads) {
                 float d = 0.f, r = 0.f;
-                if (e < elems) { d = L.grad[base + e]; r = L.residue[base + e]; }
-                s_d[e] = d;
+                unsigned short d16 = 0;
+                if (e < elems) {
+                    if (OPTS && gtype != ADACOMP_GRAD_F32) d16 = reinterpret_cast<const unsigned short *>(L.grad)[base + e];
+                    else d = L.grad[base + e];
+                    r = L.residue[base + e];
+                }
+                if (OPTS && gtype != ADACOMP_GRAD_F32) reinterpret_cast<unsigned short *>(s_d)[e] = d16;
+                else s_d[e] = d;
                 s_r[e] = r;
             }
             if (LAZY && tid < kTileSegs) reinterpret_cast<u32 *>(s_r + kFastTile)[tid] = lazy_mask[(u64)lt * kTileSegs + tid];
@@ -230,12 +254,30 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             const u32 prev = LAZY ? reinterpret_cast<const u32 *>(s_r + kFastTile)[tid] : 0u;
             // (the loop twice: where the segments line up with the bins, as in the lists' bin lengths 50 and
             // 500, the tests on `vcount` and `cut` fold away)
-            auto form = [&](auto lined_up) {
-                constexpr bool AL = decltype(lined_up)::value;
+            auto form = [&](auto lined_up, auto sixteen) {
+                constexpr bool AL = decltype(lined_up)::value, G16 = decltype(sixteen)::value;
                 const int vc = AL ? kSeg : vcount, ct = AL ? kSeg : cut;
+                // 16-bit values: thirteen aligned 32-bit loads cover the segment's 50 bytes, a funnel shift lines the pairs up
+                u32 pair[G16 ? 13 : 1];
+                if (G16) {
+                    const u32 *pw = reinterpret_cast<const u32 *>(s_d) + ((tid * kSeg) >> 1);
+                    const u32 sh = (tid & 1) * 16u;
+                    u32 w[14];
+#pragma unroll
+                    for (int q = 0; q < 13; q++) w[q] = pw[q];
+                    w[13] = 0;
+#pragma unroll
+                    for (int q = 0; q < 13; q++) pair[q] = __funnelshift_r(w[q], w[q + 1], sh);
+                }
 #pragma unroll
                 for (int j = 0; j < kSeg; j++) {
-                    float d = pd[j], r = pr[j];
+                    float d, r = pr[j];
+                    if (G16) {
+                        const u32 v16 = (j & 1) ? pair[j >> 1] >> 16 : pair[j >> 1] & 0xffffu;
+                        d = gtype == ADACOMP_GRAD_BF16 ? __uint_as_float(v16 << 16) : __half2float(__ushort_as_half((unsigned short)v16));
+                    } else {
+                        d = pd[j];
+                    }
                     if (j >= vc) d = r = 0.f;               // past the tile's end
                     if (LAZY) {
                         // r holds last step's G: finish "residue = G - sign(G) * scale" where it was sent
@@ -244,27 +286,39 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                         r = (prev >> j & 1u) ? fixed : r;
                     }
                     g[j] = __fadd_rn(r, d);
-                    const float h = __fadd_rn(g[j], d);
+                    const float h = OPTS && factor != 0.f ? __fadd_rn(r, __fmul_rn(factor, d)) : __fadd_rn(g[j], d);
                     if (j >= ct) m1 = fmaxf(m1, fabsf(g[j]));
                     else m = fmaxf(m, fabsf(g[j]));
                     key[j] = fmaxf(fabsf(h), fabsf(g[j]));
                 }
             };
-            if (aligned) form(TrueType{});
-            else form(FalseType{});
-            // (non-negative floats order like their bits)
-            if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
-            if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
+            if (!OPTS || gtype == ADACOMP_GRAD_F32) {
+                if (aligned) form(TrueType{}, FalseType{});
+                else form(FalseType{}, FalseType{});
+            } else {
+                if (aligned) form(TrueType{}, TrueType{});
+                else form(FalseType{}, TrueType{});
+            }
+            if (aligned) {
+                // a bin is SPB whole segments: no atomics, the maximum goes through a shuffle (two segments)
+                // or through the segments' maxima in shared memory
+                if (SPB == 2) gm = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+                else s_segmax[tid] = m;
+            } else {
+                // (non-negative floats order like their bits)
+                if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
+                if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
+            }
         }
-        __syncthreads();                                            // barrier A
-        // the other parity's buffers are free: tile i - 1 is done with them, tile i + 1 starts after barrier D
-        if (tid < kSmallBins) {
-            s_anymax[((i & 1) ^ 1) * kSmallBins + tid] = 0;
-            s_anycnt[((i & 1) ^ 1) * kSmallBins + tid] = 0;
-        }
+        if (!(aligned && SPB == 2)) __syncthreads();                // barrier A (uniform: the layer's shape)
         if (!service) {
-            gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
-            gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
+            if (!aligned) {
+                gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
+                gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
+            } else if (SPB != 2) {
+                const int s0 = b0 * SPB;
+                for (int sgm = 0; sgm < SPB; sgm++) gm = fmaxf(gm, s_segmax[s0 + sgm]);
+            }
             // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
             if (aligned) {
 #pragma unroll
@@ -276,22 +330,32 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                     if (key[j] >= (j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
             }
             cnt = __popc(selmask);
-            const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
-            if (c0) atomicAdd(&any_cnt[b0], c0);
-            if (cnt - c0) atomicAdd(&any_cnt[b0 + 1], cnt - c0);
+            if (!aligned) {
+                const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
+                if (c0) atomicAdd(&any_cnt[b0], c0);
+                if (cnt - c0) atomicAdd(&any_cnt[b0 + 1], cnt - c0);
+            } else if (tid == b0 * SPB) {
+                any_max[b0] = __float_as_uint(gm);                  // for the exact sum (the service warp reads it after barrier B)
+            }
             incl = warp_inclusive_scan(cnt, lane);
             s_incl[tid] = incl;
             if (lane == 31) s_wtot[warp] = incl;
         }
         __syncthreads();                                            // barrier B
+        // the other parity's buffers are free: tile i - 1 is done with them, tile i + 1 starts after barrier D
+        if (tid < kSmallBins) {
+            s_anymax[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+            s_anycnt[((i & 1) ^ 1) * kSmallBins + tid] = 0;
+        }
 
         u32 total = 0;
         if (!service) {
             // ---- words into the staging area, G back into the residue stage ----
-            u32 wpre = 0;
+            u32 wpre_all[6];
+            wpre_all[0] = 0;
 #pragma unroll
-            for (int wv = 0; wv < 5; wv++)
-                if (wv < warp) wpre += s_wtot[wv];
+            for (int wv = 0; wv < 5; wv++) wpre_all[wv + 1] = wpre_all[wv] + s_wtot[wv];
+            const u32 wpre = wpre_all[warp];
             float *pr = s_r + tid * kSeg;
 #pragma unroll
             for (int j = 0; j < kSeg; j++) pr[j] = g[j];
@@ -308,7 +372,19 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 at++;
             }
             if (LAZY) lazy_mask[(u64)lt * kTileSegs + tid] = selmask;
-            if (tid < TB) {
+            if (aligned) {
+                // the bin's first thread: the words between its own first one and the last one of the bin's last segment
+                if (tid == b0 * SPB) {
+                    const u64 bin = (u64)lt * (u64)TB + (u32)b0;
+                    const int t1 = tid + SPB - 1;
+                    const u32 last = wpre_all[t1 >> 5] + s_incl[t1], count = last - (wpre + incl) + cnt;
+                    if (bin < geo.n_bins) {
+                        unsigned char *bc = L.packed + geo.bin_cnt_at;
+                        if (wbytes == 1u) bc[bin] = (unsigned char)count;
+                        else reinterpret_cast<unsigned short *>(bc)[bin] = (unsigned short)count;
+                    }
+                }
+            } else if (tid < TB) {
                 const u64 bin = (u64)lt * (u64)TB + tid;
                 if (bin < geo.n_bins) {
                     unsigned char *bc = L.packed + geo.bin_cnt_at;
@@ -381,7 +457,7 @@ __global__ void __launch_bounds__(1024)
 batch_finalize(const __grid_constant__ BatchArgsT<N> b)
 {
     const BatchLayer &L = b.layer[blockIdx.x];
-    finalize_body(L.packed, L.packed + L.geo.scratch_at, L.geo, 0u, L.count_out, L.lazy);
+    finalize_body(L.packed, L.packed + L.geo.scratch_at, L.geo, L.factor != 0.f ? kFlagFactor : 0u, L.count_out, L.lazy);
 }
 
 // FIXUP: also finishes the sent elements' residues (eager mode; lazy-scale mode leaves G).
@@ -414,10 +490,14 @@ void init_pack_batch_info(DeviceInfo &d)
         d.batch_per_sm = per;
     }
     d.batch_fast_ready = d.fast_ready &&
-                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false>, at, bytes) == cudaSuccess &&
-                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false>, at, bytes) == cudaSuccess &&
-                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true>, at, bytes) == cudaSuccess &&
-                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true>, at, bytes) == cudaSuccess;
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false, false>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false, false>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true, false>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, false>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false, true>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false, true>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true, true>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, true>, at, bytes) == cudaSuccess;
 }
 
 // lazy: lazy-scale mode (every layer carries its state; needs the pipelined batch tile pass).
@@ -429,8 +509,12 @@ int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStrea
         if (info.batch_fast_ready) {
             const u64 cap = (u64)info.sms * 2;
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
-            if (lazy) batch_tile_pass_fast<N, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
-            else batch_tile_pass_fast<N, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            bool opts = false;
+            for (u32 i = 0; i < b.n_layers; i++) opts = opts || b.layer[i].grad_type != ADACOMP_GRAD_F32 || b.layer[i].factor != 0.f;
+            if (lazy && opts) batch_tile_pass_fast<N, true, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            else if (lazy) batch_tile_pass_fast<N, true, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            else if (opts) batch_tile_pass_fast<N, false, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            else batch_tile_pass_fast<N, false, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
         } else {
             const u64 cap = (u64)info.sms * info.batch_per_sm;
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
@@ -454,7 +538,7 @@ int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st, bo
     if (b.n_layers == 1) {      // a batch of one gains nothing over the single-layer kernels
         const BatchLayer &L = b.layer[0];
         return compress_impl(L.grad, L.residue, L.geo.n, L.geo.L_T, L.packed, reinterpret_cast<uint64_t *>(L.count_out),
-                             st, 0, nullptr, L.lazy);
+                             st, 0, nullptr, L.lazy, L.factor, L.grad_type);
     }
     if (b.n_layers <= (u32)kBatchSmall) {
         BatchArgsT<kBatchSmall> small;

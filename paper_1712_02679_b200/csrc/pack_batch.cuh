@@ -12,7 +12,7 @@ namespace adacomp_impl {
 // Layers of 42 <= L_T <= 1000 (tiles of at most 4000 elements and 96 bins) qualify.
 // ---------------------------------------------------------------------------------
 
-constexpr int kBatchMax = 184;                       // layers per batched launch (the table is 32392 of the 32764 bytes of kernel parameters)
+constexpr int kBatchMax = 176;                       // layers per batched launch (the table is 32392 of the 32764 bytes of kernel parameters)
 constexpr u64 kBatchLayerMaxElems = 1ull << 22;      // decode: larger layers take the single-layer kernels
 // pack(): layers up to this size share a batch's launches when the pipelined batch tile pass is there (a
 // layer alone ramps its pipeline up and down over a few tiles per CTA and pays four launches and a finalize
@@ -27,8 +27,10 @@ struct BatchLayer {
     u64 *count_out;
     Geometry geo;
     u32 tile_first;                                  // global index of the layer's first tile
-    u32 pad;
+    u32 grad_type;                                   // ADACOMP_GRAD_*: what `grad` points to
     unsigned char *lazy;                             // lazy-scale mode: the layer's state (else null)
+    float factor;                                    // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW
+    u32 pad;
 };
 
 // The table comes in two sizes: kernel parameters are copied at every launch, and a launch with the

@@ -132,3 +132,70 @@ def test_unsupported_combinations_are_refused_on_the_host():
     with pytest.raises(B.AdaCompError) as e:
         B.adacomp_compress_opt(res, res, n, L_T, packed, cnt, grad_type=7)
     assert e.value.code == -6
+
+
+def _list_case(rng, lazy):
+    """A parameter list whose layers differ in bin length, gradient format and factor."""
+    shapes = [(50, 4000 * 13 + 17, B.ADACOMP_GRAD_F32, 0.0), (500, 4000 * 6 + 499, B.ADACOMP_GRAD_BF16, 0.0),
+              (50, 4000 * 3, B.ADACOMP_GRAD_F16, 1.5), (100, 4000 * 4 + 1, B.ADACOMP_GRAD_F32, 3.0),
+              (64, 3840 * 5 + 9, B.ADACOMP_GRAD_F16, 0.0), (400, 3200 * 3 + 77, B.ADACOMP_GRAD_BF16, 1.5),
+              (500, 864, B.ADACOMP_GRAD_F32, 0.0), (50, 10, B.ADACOMP_GRAD_F16, 0.0), (200, 4000 * 2 + 150, B.ADACOMP_GRAD_F16, 0.0)]
+    if not lazy:
+        shapes.append((43, 3956 * 3 + 5, B.ADACOMP_GRAD_BF16, 0.0))      # 16-bit tiles off the 16-byte boundaries: plain loads
+    layers = []
+    for L_T, n, gt, factor in shapes:
+        r_cpu = rng.normal(0, 2e-3, n).astype(np.float32)
+        res = torch.zeros(max(n, 4), device=DEV)
+        res[:n] = torch.from_numpy(r_cpu)
+        d = dict(n=n, L_T=L_T, grad_type=gt, factor=factor, residue=res, r_cpu=r_cpu,
+                 packed_out=torch.empty(B.adacomp_packed_capacity(n, L_T), dtype=torch.uint8, device=DEV),
+                 count_out=torch.zeros(2, dtype=torch.int64, device=DEV))
+        if lazy:
+            d["lazy_state"] = torch.empty(B.adacomp_lazy_state_bytes(n, L_T), dtype=torch.uint8, device=DEV)
+            B.adacomp_lazy_state_init(d["lazy_state"], n, L_T)
+        layers.append(d)
+    return layers
+
+
+@pytest.mark.parametrize("lazy", [False, True])
+def test_parameter_list_with_per_layer_options(lazy):
+    rng = np.random.default_rng(4242 + lazy)
+    layers = _list_case(rng, lazy)
+    for step in range(3):
+        wants = []
+        for d in layers:
+            d["grad"], g_cpu = make_grad(rng, d["n"], d["grad_type"])
+            wants.append(cref.pack(g_cpu, d["r_cpu"], d["L_T"], factor=d["factor"]))
+            d["packed_out"].fill_(0xAB)
+        B.adacomp_compress_multi_opt(layers, len(layers))
+        torch.cuda.synchronize()
+        for i, (d, want) in enumerate(zip(layers, wants)):
+            what = f"layer {i} L_T={d['L_T']} n={d['n']} step {step} lazy={lazy}"
+            assert int(d["count_out"][0]) == want.n_sel, what
+            assert_stream_equal(d["packed_out"][:int(d["count_out"][1])].cpu().numpy(), want, what)
+            if not lazy:
+                assert_f32_bits_equal(d["residue"][:d["n"]].cpu().numpy(), d["r_cpu"], what + " residue")
+    if lazy:
+        for d in layers:
+            B.adacomp_residue_flush(d["residue"], d["lazy_state"], d["n"], d["L_T"])
+        torch.cuda.synchronize()
+        for i, d in enumerate(layers):
+            assert_f32_bits_equal(d["residue"][:d["n"]].cpu().numpy(), d["r_cpu"], f"layer {i} residue after the flush")
+    assert B.adacomp_device_status() == 0
+
+
+def test_parameter_list_where_only_some_layers_are_lazy():
+    rng = np.random.default_rng(77)
+    layers = _list_case(rng, True)
+    for d in layers[::2]:
+        del d["lazy_state"]
+    for step in range(2):
+        wants = []
+        for d in layers:
+            d["grad"], g_cpu = make_grad(rng, d["n"], d["grad_type"])
+            wants.append(cref.pack(g_cpu, d["r_cpu"], d["L_T"], factor=d["factor"]))
+        B.adacomp_compress_multi_opt(layers, len(layers))
+        torch.cuda.synchronize()
+        for i, (d, want) in enumerate(zip(layers, wants)):
+            assert_stream_equal(d["packed_out"][:int(d["count_out"][1])].cpu().numpy(), want, f"layer {i} step {step}")
+    assert B.adacomp_device_status() == 0
