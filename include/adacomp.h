@@ -431,6 +431,23 @@ int adacomp_set_device(int device);
  */
 int adacomp_device_status(uint32_t *host_out, void *stream);
 
+/*
+ * Testing aid for the bounded device-side waits (every wait of a kernel on a copy in flight gives up after a
+ * limit, raises ADACOMP_DEV_TIMEOUT, lets the copies it did start land and returns; no kernel spins without a
+ * limit).  This call lets a test see that path run without anything being wrong with the device:
+ *   wait_cycles            the limit, in GPU clock cycles, of the waits in adacomp_compress* (single layer,
+ *                          pipelined tile pass) and in adacomp_decompress_* (single tensor, L_T above 40);
+ *                          0 restores the default of about two seconds.
+ *   withhold_pack_tile     CTA 0 of the next tile passes announces the copies of its tile number i (i >= 1,
+ *                          counted over the CTA's own tiles) and never starts them; 0: none.
+ *   withhold_decode_item   the same for work item i of CTA 0 of the next decodes; 0: none.
+ * A kernel that meets a withheld copy times out: the tiles / items its CTA 0 had not finished are reported as
+ * empty (pack) or left unwritten (decode), every other CTA's work is complete, and the kernels behind stay
+ * inside their buffers.  Host only; the settings are process-wide and stay until the next call.  Not meant
+ * for production code.  (The paper has no counterpart.)
+ */
+int adacomp_debug_waits(uint64_t wait_cycles, uint32_t withhold_pack_tile, uint32_t withhold_decode_item);
+
 /* Enqueues a clear of the sticky bits on `stream`. */
 int adacomp_device_status_reset(void *stream);
 

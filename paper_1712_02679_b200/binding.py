@@ -488,5 +488,12 @@ def adacomp_device_status(stream=None) -> int:
     return int(out.value)
 
 
+def adacomp_debug_waits(wait_cycles: int = 0, withhold_pack_tile: int = 0, withhold_decode_item: int = 0) -> None:
+    """Testing aid: the limit of the device-side waits and one withheld copy (see include/adacomp.h)."""
+    f = lib().adacomp_debug_waits
+    f.restype, f.argtypes = C.c_int, [C.c_uint64, C.c_uint32, C.c_uint32]
+    _check(f(int(wait_cycles), int(withhold_pack_tile), int(withhold_decode_item)), "adacomp_debug_waits")
+
+
 def adacomp_device_status_reset(stream=None) -> None:
     _check(lib().adacomp_device_status_reset(_stream(stream)), "adacomp_device_status_reset")

@@ -7,6 +7,9 @@ namespace adacomp_impl {
 
 DeviceInfo g_info[64];
 
+DebugWaits g_debug_waits = {kWaitCycles, 0u, 0u};
+const DebugWaits &debug_waits() { return g_debug_waits; }
+
 int device_info(DeviceInfo *&out)
 {
     int dev = 0;
@@ -450,6 +453,14 @@ int adacomp_decompress_average_adam(const void *const *packed, uint32_t k_stream
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
     const Epilogue ep = {weights, m, v, step_size, beta1, beta2, eps, 0.f, 1u, 0.f};
     return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
+}
+
+int adacomp_debug_waits(uint64_t wait_cycles, uint32_t withhold_pack_tile, uint32_t withhold_decode_item)
+{
+    g_debug_waits.limit = wait_cycles ? (long long)(wait_cycles < (1ull << 40) ? wait_cycles : (1ull << 40)) : kWaitCycles;
+    g_debug_waits.withhold_pack = withhold_pack_tile;
+    g_debug_waits.withhold_decode = withhold_decode_item;
+    return ADACOMP_OK;
 }
 
 int adacomp_set_device(int device)

@@ -226,16 +226,24 @@ __device__ inline void mbar_arrive(u64 *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
-// Bounded wait: false if the phase did not complete within kWaitCycles.
-__device__ inline bool mbar_wait(u64 *bar, u32 parity)
+// Bounded wait: false if the phase did not complete within `limit` cycles.
+__device__ inline bool mbar_wait(u64 *bar, u32 parity, long long limit = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
+
+// What adacomp_debug_waits sets (a testing aid, see include/adacomp.h): the bound of the waits of the single-layer
+// tile pass and of the single-tensor warp decoder, and which of CTA 0's loads its copy engine is to leave out
+// (0: none) so that a wait runs out without anything being wrong with the device.
+struct DebugWaits {
+    long long limit;
+    u32 withhold_pack, withhold_decode;
+};
 
 __device__ inline void bulk_load(void *smem_dst, const void *gmem_src, u32 bytes, u64 *bar)
 {

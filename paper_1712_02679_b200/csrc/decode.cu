@@ -67,6 +67,8 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
     args.k = k;
     args.hint_n = hint_n;
     args.hint_L_T = hint_L_T;
+    args.wait_limit = debug_waits().limit;
+    args.withhold = debug_waits().withhold_decode;
     DeviceInfo *info = nullptr;
     int rc = device_info(info);
     if (rc != ADACOMP_OK) return rc;

@@ -76,6 +76,8 @@ struct DecodeArgs {
     u32 pairs;          // the kernel of pair_path() is launched too: its shapes are left to it
     u32 hint_L_T;       // 0: the caller did not say; else the streams must carry exactly this shape
     u64 hint_n;
+    long long wait_limit;   // cycles a wait for a slot may take (kWaitCycles unless a test shortened it)
+    u32 withhold;           // testing aid: CTA 0's loader starts no copies for its item number `withhold` (0: none)
 };
 
 // Work items of the decoder for a tensor: output tiles, split into chunks where a tile is larger.
@@ -1146,7 +1148,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                 // the item's bin counts start `clead` bytes behind a 16-byte boundary: the copy starts at the boundary
                 const u32 clead = ONE ? ia >> 24 : (u32)(bin0 * sizeof(Word)) & 15u;
                 const u32 cbytes = (u32)align_up(clead + live * (u32)sizeof(Word), 16);
-                if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u)) {
+                if (use > 0 && !mbar_wait(&ws.empty[s], (use - 1u) & 1u, a.wait_limit)) {
                     ws.abort = 1;
                     raise_status(ADACOMP_DEV_TIMEOUT);
                     failed = true;      // the decoding warps time out on the full barrier in turn
@@ -1200,10 +1202,12 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
                     if ((u32)lane + 32u * h < staged) expect += cbytes + wbytes[h];
                 if (expect) mbar_arrive_expect_tx(&ws.full[s], expect);
                 else mbar_arrive(&ws.full[s]);
+                // (testing aid) bytes are expected and never sent: the decoding warps' wait for this slot runs out
+                const bool hold = a.withhold != 0u && blockIdx.x == 0 && it == (u64)a.withhold;
 #pragma unroll
                 for (int h = 0; h < 2; h++) {
                     const u32 j = (u32)lane + 32u * h;
-                    if (j < staged) {
+                    if (j < staged && !hold) {
                         bulk_load(sl + coff[h], a.stream[l0 + j] + geo.bin_cnt_at + (bin0 * sizeof(Word) - clead), cbytes, &ws.full[s]);
                         if (wbytes[h])
                             bulk_load(sl + coff[h] + count_bytes, reinterpret_cast<const void *>(src[h] & ~(u64)15u), wbytes[h],
@@ -1225,7 +1229,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
         if (*reinterpret_cast<volatile u32 *>(&ws.abort)) {
             // after a timeout the copies already started must land (or time out in turn) before
             // this CTA's shared memory is given back
-            for (u64 j = issued > S ? issued - S : 0; j < issued; j++) mbar_wait(&ws.full[j % S], (u32)(j / S) & 1u);    // (rare)
+            for (u64 j = issued > S ? issued - S : 0; j < issued; j++) mbar_wait(&ws.full[j % S], (u32)(j / S) & 1u, a.wait_limit);    // (rare)
         }
         return;
     }
@@ -1272,7 +1276,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             if (OPT == 2) bulk_load(uq, a.ep.second + out0, quarter * 4u, &ws.wv_full[warp]);
         }
         for (u32 r = 0; r < NR; r++, s = s + 1u == S ? 0u : s + 1u, use += s == 0u) {
-            if (!mbar_wait(&ws.full[s], use & 1u)) {
+            if (!mbar_wait(&ws.full[s], use & 1u, a.wait_limit)) {
                 ws.abort = 1;
                 bad |= ADACOMP_DEV_TIMEOUT;
                 failed = true;
@@ -1344,7 +1348,7 @@ __device__ void decode_warps(const DecodeArgs &a, const Geometry &geo, float *s_
             // averageGradients() + updateWeights() on the warp's quarter, in shared memory; two bulk
             // copies take the new weights and momentum back
             if (whole) {
-                if (!mbar_wait(&ws.wv_full[warp], wv_use & 1u)) {
+                if (!mbar_wait(&ws.wv_full[warp], wv_use & 1u, a.wait_limit)) {
                     ws.abort = 1;
                     bad |= ADACOMP_DEV_TIMEOUT;
                     break;

@@ -38,6 +38,9 @@ bool fast_tile_pass_b(const PassArgs *args, unsigned grid, cudaStream_t st);
 bool fast_tile_pass_c(const PassArgs *args, unsigned grid, cudaStream_t st);
 bool fast_tile_pass_d(const PassArgs *args, unsigned grid, cudaStream_t st);
 
+// abi.cu: what adacomp_debug_waits last set (the defaults: kWaitCycles, nothing withheld)
+const DebugWaits &debug_waits();
+
 // pack.cu
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,

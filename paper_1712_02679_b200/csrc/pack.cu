@@ -143,7 +143,8 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 
     mark(0);
     if (geo.n_tiles) {
-        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_type};
+        PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_type,
+                      debug_waits().limit, debug_waits().withhold_pack};
         const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
         // (one-bin tiles fill the pipelined kernel's 4000-element stages only in part: below 2800 elements the
         // warp-per-part kernel is faster, measured; lazy-scale mode exists in the pipelined kernel only)

@@ -33,6 +33,8 @@ struct PassArgs {
     unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
     float factor;               // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW (Section 2.4's scale-factor)
     u32 grad_type;              // ADACOMP_GRAD_*: `grad` points to binary32 values, or to bfloat16 / binary16 ones (widened exactly on load)
+    long long wait_limit;       // cycles a wait for a stage may take (kWaitCycles unless a test shortened it)
+    u32 withhold;               // testing aid: CTA 0 starts no copies for its tile number `withhold` (0: none)
 };
 
 // Lazy-mode state: 64-byte header, then one u32 per 25-element segment (bit j = element j
@@ -149,6 +151,10 @@ tile_pass_fast(PassArgs a)
         u64 *bar = &s_full[i % kStages];
         const u32 grad_bytes = G16 ? tile_bytes / 2 : tile_bytes;
         mbar_arrive_expect_tx(bar, grad_bytes + tile_bytes + (LAZY ? kMaskBytes : 0u));
+        if (a.withhold != 0u && blockIdx.x == 0 && i == (u64)a.withhold) {
+            issued = i + 1;             // (testing aid) bytes are expected and never sent: the wait for this stage runs out
+            return;
+        }
         bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)grad_bytes, grad_bytes, bar);
         bulk_load(st + kTileBytes, a.residue + tile * (u64)T, tile_bytes, bar);
         if (LAZY) bulk_load(st + 2 * kTileBytes, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
@@ -171,7 +177,7 @@ tile_pass_fast(PassArgs a)
         u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
 
         if (whole) {
-            if (!mbar_wait(&s_full[i % kStages], (u32)(i / kStages) & 1u)) {
+            if (!mbar_wait(&s_full[i % kStages], (u32)(i / kStages) & 1u, a.wait_limit)) {
                 *s_abort = 1;                      // every thread that times out says so
                 raise_status(ADACOMP_DEV_TIMEOUT);
             }
@@ -361,7 +367,7 @@ tile_pass_fast(PassArgs a)
                 // after a timeout: loads still in flight must land (or time out in turn) before
                 // this CTA's shared memory is given back, and the tiles it never finished count
                 // as empty so that the kernels after this one stay inside their buffers
-                for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % kStages], (u32)(j / kStages) & 1u);
+                for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % kStages], (u32)(j / kStages) & 1u, a.wait_limit);
                 for (u64 j = i; j < my_tiles; j++) tile_cnt[first + j * stride] = 0;
             }
         }
