@@ -189,9 +189,22 @@ static uint32_t sent_places_of_bin(const float *G, const float *H, uint64_t lo, 
  * two forms can differ in the last place, which is why they are kept apart).  Factor 1 makes H = G:
  * only the bin maxima are sent, which is the local selection without the soft threshold that the
  * paper compares against (Section 5, "LS").  Streams made with a factor carry bit 1 in the header's flags.
+ *
+ * `quantiser`: Section 2.5 notes that the method is not tied to one quantisation function.  0 is the
+ * paper's: sign(G) times the average of the g_max vector over all bins.  1 keeps the sign and the one value
+ * per layer but takes for it the average |G| of the elements that are sent (the value that makes the
+ * squared error of the sent elements smallest): the exact sum of those |G|, rounded once to double,
+ * divided by their number in double and rounded to binary32; 0 when nothing is sent.  The selection does
+ * not depend on the quantiser.  Streams made with quantiser 1 carry bit 2 in the header's flags.
  */
+int adacomp_oracle_pack_general(const float *dW, float *residue, uint64_t n, uint32_t L_T, uint32_t flags,
+                                float factor, uint32_t quantiser, uint8_t *out, uint64_t out_cap, float *g_max_out);
+
 int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint32_t L_T,
-                               uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out);
+                               uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out)
+{
+    return adacomp_oracle_pack_general(dW, residue, n, L_T, flags, factor, 0u, out, out_cap, g_max_out);
+}
 
 int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_T,
                         uint32_t flags, uint8_t *out, uint64_t out_cap, float *g_max_out)
@@ -199,12 +212,13 @@ int adacomp_oracle_pack(const float *dW, float *residue, uint64_t n, uint32_t L_
     return adacomp_oracle_pack_scaled(dW, residue, n, L_T, flags, 0.0f, out, out_cap, g_max_out);
 }
 
-int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint32_t L_T,
-                               uint32_t flags, float factor, uint8_t *out, uint64_t out_cap, float *g_max_out)
+int adacomp_oracle_pack_general(const float *dW, float *residue, uint64_t n, uint32_t L_T, uint32_t flags,
+                                float factor, uint32_t quantiser, uint8_t *out, uint64_t out_cap, float *g_max_out)
 {
     if (L_T == 0 || L_T > 16384u || !out || (n && (!dW || !residue))) return -1;
     if (factor != 0.0f && !(factor > 0.0f && factor <= 1e30f)) return -1;
-    flags = (flags & 1u) | (factor != 0.0f ? 2u : 0u);
+    if (quantiser > 1u) return -1;
+    flags = (flags & 1u) | (factor != 0.0f ? 2u : 0u) | (quantiser == 1u ? 4u : 0u);
     const int literal = (flags & 1u) != 0;
     const int threads = oracle_threads;
     (void)threads;
@@ -260,6 +274,25 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
     const uint64_t bytes_used = geo.payload_at + align16(n_sel * geo.w);
     const int overflow = bytes_used > out_cap;
 
+    if (quantiser == 1u) {
+        /* the other quantiser: the average |G| of the elements that are sent */
+        scale = 0.0f;
+        if (n_sel) {
+            float *sent_abs = (float *)malloc(n_sel * sizeof(float));
+            if (!sent_abs) { free(G); free(H); free(g_max); free(first_word); return -2; }
+#pragma omp parallel for num_threads(threads) if (threads > 1)
+            for (int64_t b = 0; b < bins; b++) {
+                uint64_t lo = (uint64_t)b * L_T, hi = lo + L_T < n ? lo + L_T : n;
+                uint16_t places[16384];
+                const uint32_t sent = sent_places_of_bin(G, H, lo, hi, g_max[b], literal, places);
+                for (uint32_t j = 0; j < sent; j++) sent_abs[first_word[b] + j] = fabsf(G[lo + places[j]]);
+            }
+            double S = adacomp_oracle_exact_sum(sent_abs, n_sel);
+            scale = (float)(S / (double)n_sel);
+            free(sent_abs);
+        }
+    }
+
     /* bin by bin: the counts, the words of the sent elements, and everybody's new residue */
     memset(out, 0, geo.payload_at);
     uint8_t *tile_off = out + geo.tile_off_at;
@@ -293,7 +326,7 @@ int adacomp_oracle_pack_scaled(const float *dW, float *residue, uint64_t n, uint
     put_u32(out + 0, ORACLE_MAGIC);
     put_u16(out + 4, 1);
     out[6] = (uint8_t)geo.w;
-    out[7] = (uint8_t)(flags & 3u);
+    out[7] = (uint8_t)(flags & 7u);
     put_u32(out + 8, L_T);
     put_u32(out + 12, geo.tile_bins);
     put_u64(out + 16, n);

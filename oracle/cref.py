@@ -34,6 +34,9 @@ def lib() -> C.CDLL:
         _lib.adacomp_oracle_set_threads.argtypes = [C.c_int]
         _lib.adacomp_oracle_get_threads.restype = C.c_int
         _lib.adacomp_oracle_get_threads.argtypes = []
+        _lib.adacomp_oracle_pack_general.restype = C.c_int
+        _lib.adacomp_oracle_pack_general.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
+                                                     C.c_float, C.c_uint32, C.c_void_p, C.c_uint64, C.c_void_p]
         _lib.adacomp_oracle_unpack_sum.restype = C.c_int
         _lib.adacomp_oracle_unpack_sum.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
     return _lib
@@ -109,9 +112,10 @@ def parse(raw: np.ndarray) -> Packed:
 
 
 def pack(dW: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0,
-         want_gmax: bool = False, factor: float = 0.0) -> Packed:
+         want_gmax: bool = False, factor: float = 0.0, quantiser: int = 0) -> Packed:
     """Run Algorithm 2 on one layer.  `residue` (float32, contiguous) is updated in place.
-    `factor` (0: the paper's H = G + dW) selects H = residue + factor * dW, see the C source."""
+    `factor` (0: the paper's H = G + dW) selects H = residue + factor * dW, `quantiser` (0: the paper's mean of
+    the bin maxima) the layer's reconstruction value, see the C source."""
     assert dW.dtype == np.float32 and residue.dtype == np.float32
     assert dW.flags.c_contiguous and residue.flags.c_contiguous and dW.shape == residue.shape
     n = dW.size
@@ -119,9 +123,9 @@ def pack(dW: np.ndarray, residue: np.ndarray, L_T: int, flags: int = 0,
     out = np.empty(cap, dtype=np.uint8)
     n_bins = (n + L_T - 1) // L_T
     gmax = np.empty(max(n_bins, 1), dtype=np.float32) if want_gmax else None
-    rc = lib().adacomp_oracle_pack_scaled(_ptr(dW) if n else None, _ptr(residue) if n else None, n, L_T,
-                                          flags, C.c_float(factor), _ptr(out), cap,
-                                          _ptr(gmax) if want_gmax else None)
+    rc = lib().adacomp_oracle_pack_general(_ptr(dW) if n else None, _ptr(residue) if n else None, n, L_T,
+                                           flags, C.c_float(factor), int(quantiser), _ptr(out), cap,
+                                           _ptr(gmax) if want_gmax else None)
     if rc != 0:
         raise RuntimeError(f"adacomp_oracle_pack failed: {rc}")
     p = parse(out)

@@ -20,9 +20,12 @@ def _tile_bins(L_T: int) -> int:
     return 4 * (1000 // L_T) if L_T <= 1000 else 1
 
 
-def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool = False, factor: float = 0.0):
+def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool = False, factor: float = 0.0,
+         quantiser: int = 0):
     """Returns (bin_cnt, words, scale, new_residue, g_max).  `factor` other than 0 replaces the paper's
-    H = G + dW by H = residue + factor * dW (the scale-factor of Section 2.4; 1 = local selection only)."""
+    H = G + dW by H = residue + factor * dW (the scale-factor of Section 2.4; 1 = local selection only).
+    `quantiser` 1 replaces the mean of the bin maxima by the mean |G| of the sent elements (Section 2.5 leaves
+    the quantisation function open)."""
     n = len(dW)
     dW = [f32(x) for x in dW]
     residue = [f32(x) for x in residue]
@@ -42,6 +45,17 @@ def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool 
         scale = f32(S / float(n_bins))
     else:
         scale = f32(0)
+    def is_sent(index, i):
+        g, h, m = G[index], H[index], g_max[i]
+        return bool(m > 0 and g != 0 and (abs(h) >= m or (not literal and abs(g) == m)))
+
+    if quantiser == 1:
+        sent = [abs(G[i * L_T + j]) for i in range(n_bins) for j in range(L_T) if i * L_T + j < n and is_sent(i * L_T + j, i)]
+        if sent:
+            total = sum((Fraction(float(x)) for x in sent), Fraction(0))
+            scale = f32(float(total) / float(len(sent)))
+        else:
+            scale = f32(0)
     bin_cnt: List[int] = []
     words: List[int] = []
     new_residue = list(G)
@@ -64,7 +78,7 @@ def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool 
 
 
 def to_stream(n: int, L_T: int, bin_cnt: Sequence[int], words: Sequence[int], scale,
-              literal: bool = False, factor: float = 0.0) -> bytes:
+              literal: bool = False, factor: float = 0.0, quantiser: int = 0) -> bytes:
     """Serialise to the wire layout: header, tile directory, bin counts, words."""
     w = 1 if L_T <= 64 else 2
     tb = _tile_bins(L_T)
@@ -78,7 +92,7 @@ def to_stream(n: int, L_T: int, bin_cnt: Sequence[int], words: Sequence[int], sc
     body += pad16(struct.pack(f"<{len(words)}{fmt}", *words))
     bytes_used = 64 + len(body)
     scale_bits = struct.unpack("<I", struct.pack("<f", float(scale)))[0]
-    head = struct.pack("<IHBBIIQQQQIIQ", 0x31434441, 1, w, (1 if literal else 0) | (2 if factor != 0.0 else 0), L_T, tb, n, n_bins,
+    head = struct.pack("<IHBBIIQQQQIIQ", 0x31434441, 1, w, (1 if literal else 0) | (2 if factor != 0.0 else 0) | (4 if quantiser == 1 else 0), L_T, tb, n, n_bins,
                        n_tiles, len(words), scale_bits, 0, bytes_used)
     return head + body
 
