@@ -89,6 +89,10 @@ extern "C" {
 #define ADACOMP_GRAD_BF16 1u
 #define ADACOMP_GRAD_F16 2u
 
+/* quantisers (adacomp_options.quantiser): what the one value per layer, sent with the words, is */
+#define ADACOMP_QUANT_BIN_MAX_MEAN 0u  /* the paper's (Section 2.5): the average of the bin maxima over all bins */
+#define ADACOMP_QUANT_SENT_MEAN 1u     /* the average |G| of the elements that are sent (Section 2.5 leaves the function open) */
+
 /* Library ABI version (ADACOMP_VERSION).  Host only, no CUDA call. */
 int adacomp_version(void);
 
@@ -197,6 +201,12 @@ int adacomp_compress_f16(const void *grad_f16, float *residue, uint64_t n, uint3
  *   flags       ADACOMP_FLAG_* bits (adacomp_compress_ex).
  *   grad_type   ADACOMP_GRAD_*: what `grad` points to (adacomp_compress_bf16 / _f16).
  *   factor      0: Algorithm 2's H = G + dW; else H = residue + factor * dW (adacomp_compress_scaled).
+ *   quantiser   ADACOMP_QUANT_*: the value Q = sign(G) * scale is made with.  The paper's scale is the average of
+ *               the bin maxima over all bins; ADACOMP_QUANT_SENT_MEAN takes the average |G| of the sent elements
+ *               instead (an exact sum, rounded once to double, divided by their number, rounded to binary32; 0
+ *               when nothing is sent), which makes the squared error of the sent elements smallest.  The
+ *               selection, the words and the decoder do not change; the stream's header carries bit 2 in its
+ *               flags byte.
  *   lazy_state  NULL, or the layer's lazy-scale state (adacomp_compress_lazy).
  * Combinations: a factor and a 16-bit gradient go with lazy-scale mode wherever that mode exists
  * (L_T 41..1000 and the multiples of 4 up to 4000), except a 16-bit gradient at a bin length whose tiles
@@ -209,7 +219,7 @@ typedef struct {
     uint32_t flags;
     uint32_t grad_type;
     float factor;
-    uint32_t reserved;      /* must be 0 */
+    uint32_t quantiser;
     void *lazy_state;
 } adacomp_options;
 

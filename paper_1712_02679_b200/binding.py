@@ -39,11 +39,12 @@ class adacomp_layer_desc(C.Structure):
 
 
 class adacomp_options(C.Structure):
-    _fields_ = [("flags", C.c_uint32), ("grad_type", C.c_uint32), ("factor", C.c_float), ("reserved", C.c_uint32),
+    _fields_ = [("flags", C.c_uint32), ("grad_type", C.c_uint32), ("factor", C.c_float), ("quantiser", C.c_uint32),
                 ("lazy_state", C.c_void_p)]
 
 
 ADACOMP_GRAD_F32, ADACOMP_GRAD_BF16, ADACOMP_GRAD_F16 = 0, 1, 2
+ADACOMP_QUANT_BIN_MAX_MEAN, ADACOMP_QUANT_SENT_MEAN = 0, 1
 _GRAD_DTYPES = {ADACOMP_GRAD_F32: torch.float32, ADACOMP_GRAD_BF16: torch.bfloat16, ADACOMP_GRAD_F16: torch.float16}
 
 _lib: Optional[C.CDLL] = None
@@ -231,9 +232,10 @@ def adacomp_compress_f16(grad_f16, residue, n: int, L_T: int, packed_out, count_
 
 
 def adacomp_compress_opt(grad, residue, n: int, L_T: int, packed_out, count_out, flags: int = 0,
-                         grad_type: int = ADACOMP_GRAD_F32, factor: float = 0.0, lazy_state=None, stream=None) -> None:
-    """pack() with every option at once (flags, gradient format, the selection's factor, lazy-scale state)."""
-    opt = adacomp_options(int(flags), int(grad_type), float(factor), 0,
+                         grad_type: int = ADACOMP_GRAD_F32, factor: float = 0.0, lazy_state=None, quantiser: int = 0,
+                         stream=None) -> None:
+    """pack() with every option at once (flags, gradient format, the selection's factor, quantiser, lazy-scale state)."""
+    opt = adacomp_options(int(flags), int(grad_type), float(factor), int(quantiser),
                           _dev_ptr(lazy_state, "lazy_state", torch.uint8) if lazy_state is not None else None)
     _check(lib().adacomp_compress_opt(_dev_ptr(grad, "grad", _GRAD_DTYPES.get(int(grad_type))),
                                       _dev_ptr(residue, "residue", torch.float32), int(n), int(L_T),
@@ -456,7 +458,7 @@ def adacomp_compress_multi_opt(layers: Sequence[dict], n_layers: int, stream=Non
     opts = (adacomp_options * max(len(layers), 1))()
     for i, d in enumerate(layers):
         st = d.get("lazy_state")
-        opts[i] = adacomp_options(0, int(d.get("grad_type", 0)), float(d.get("factor", 0.0)), 0,
+        opts[i] = adacomp_options(0, int(d.get("grad_type", 0)), float(d.get("factor", 0.0)), int(d.get("quantiser", 0)),
                                   _dev_ptr(st, "lazy_state", torch.uint8) if st is not None else None)
     _check(lib().adacomp_compress_multi_opt(descs, opts, int(n_layers), _stream(stream)), "adacomp_compress_multi_opt")
 

@@ -296,11 +296,12 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
     auto state_of = [&](uint32_t t) -> void * { return states ? states[t] : opts ? opts[t].lazy_state : nullptr; };
     auto factor_of = [&](uint32_t t) { return opts ? opts[t].factor : 0.f; };
     auto type_of = [&](uint32_t t) { return opts ? opts[t].grad_type : (uint32_t)ADACOMP_GRAD_F32; };
+    auto quant_of = [&](uint32_t t) { return opts ? opts[t].quantiser : (uint32_t)ADACOMP_QUANT_BIN_MAX_MEAN; };
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
         if (opts) {
             const adacomp_options &o = opts[t];
-            if (o.reserved != 0u || o.flags != 0u || o.grad_type > ADACOMP_GRAD_F16) return ADACOMP_ERR_FLAGS;
+            if (o.quantiser > ADACOMP_QUANT_SENT_MEAN || o.flags != 0u || o.grad_type > ADACOMP_GRAD_F16) return ADACOMP_ERR_FLAGS;
             if (o.factor != 0.f && !(o.factor > 0.f && o.factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
             if (o.lazy_state) {
                 if (misaligned(o.lazy_state)) return ADACOMP_ERR_ALIGN;
@@ -340,18 +341,20 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
         all_lazy = all_lazy && state_of(t) != nullptr;
     }
     const bool batch_lazy = any_lazy && all_lazy, mixed = any_lazy && !all_lazy;
-    auto batched = [&](const adacomp_layer_desc &d) {
-        return !mixed && info->batch_per_sm > 0 && batchable(d, *info) && (!batch_lazy || info->batch_fast_ready);
+    // (the batch kernels know the paper's quantiser only: a layer with the other one is packed on its own)
+    auto batched_at = [&](uint32_t t) {
+        return !mixed && quant_of(t) == ADACOMP_QUANT_BIN_MAX_MEAN && info->batch_per_sm > 0 && batchable(layers[t], *info) &&
+               (!batch_lazy || info->batch_fast_ready);
     };
     // (more layers than a table holds: batches of equal size, so that none is left with a layer or two)
     uint32_t to_batch = 0;
-    for (uint32_t t = 0; t < n_layers; t++) to_batch += batched(layers[t]) ? 1u : 0u;
+    for (uint32_t t = 0; t < n_layers; t++) to_batch += batched_at(t) ? 1u : 0u;
     // (without the pipelined batch kernel the batch runs the any-L_T tile code, which takes every format too)
     const uint32_t n_batches = (to_batch + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
     const uint32_t per_batch = n_batches ? (to_batch + n_batches - 1) / n_batches : (uint32_t)kBatchMax;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (batched(d)) {
+        if (batched_at(t)) {
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
@@ -372,7 +375,7 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
             }
         } else {
             rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags, nullptr,
-                               state_of(t), factor_of(t), type_of(t));
+                               state_of(t), factor_of(t), type_of(t), nullptr, quant_of(t));
             if (rc != ADACOMP_OK) return rc;
         }
     }
@@ -424,11 +427,10 @@ int adacomp_compress_f16(const void *grad_f16, float *residue, uint64_t n, uint3
 int adacomp_compress_opt(const void *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                          uint64_t *count_out, const adacomp_options *opt, void *stream)
 {
-    const adacomp_options none = {0u, ADACOMP_GRAD_F32, 0.f, 0u, nullptr};
+    const adacomp_options none = {0u, ADACOMP_GRAD_F32, 0.f, ADACOMP_QUANT_BIN_MAX_MEAN, nullptr};
     const adacomp_options &o = opt ? *opt : none;
-    if (o.reserved != 0u) return ADACOMP_ERR_FLAGS;
     return compress_impl(static_cast<const float *>(grad), residue, n, L_T, packed_out, count_out, stream, o.flags, nullptr,
-                         o.lazy_state, o.factor, o.grad_type);
+                         o.lazy_state, o.factor, o.grad_type, nullptr, o.quantiser);
 }
 
 int adacomp_compress_scaled(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,

@@ -15,6 +15,8 @@ typedef unsigned int u32;
 
 constexpr u32 kMagic = 0x31434441u;
 constexpr u32 kFlagFactor = 2u;       // header flag (set by the library): the stream was made with a scale-factor
+constexpr u32 kFlagQuant = 4u;        // header flag (set by the library): the scale is the mean |G| of the sent elements
+constexpr u32 kCtlSentSumAt = 128;    // control block: the nine windows of the exact sum of the sent |G| (second quantiser)
 constexpr u32 kHeaderBytes = 64;
 constexpr u32 kCtlBytes = 256;       // control block at the start of the scratch area
 constexpr int kWindows = 9;          // 32-bit windows of the exact g_max accumulator
@@ -191,6 +193,29 @@ __device__ inline void warp_accumulate(u64 *acc, float gm, bool valid)
         atomicAdd(&acc[window + 1], hi);
     }
     __syncwarp();
+}
+
+// The same into an accumulator that several warps of the CTA share (shared-memory atomics).
+__device__ inline void warp_accumulate_shared(u64 *acc, float v, bool valid)
+{
+    const u32 full = 0xffffffffu;
+    u32 window = 0;
+    u64 lo = 0, hi = 0;
+    valid = valid && split_for_sum(v, window, lo, hi);
+    const u32 vm = __ballot_sync(full, valid);
+    if (vm == 0) return;
+    const u32 w0 = __shfl_sync(full, window, __ffs(vm) - 1);
+    if (__all_sync(full, !valid || window == w0)) {
+        if (!valid) { lo = 0; hi = 0; }
+        for (int d = 16; d > 0; d >>= 1) {
+            lo += __shfl_down_sync(full, lo, d);
+            hi += __shfl_down_sync(full, hi, d);
+        }
+        if ((threadIdx.x & 31) == 0) { atomicAdd(&acc[w0], lo); atomicAdd(&acc[w0 + 1], hi); }
+    } else if (valid) {
+        atomicAdd(&acc[window], lo);
+        atomicAdd(&acc[window + 1], hi);
+    }
 }
 
 // ---- mbarrier / bulk-copy (TMA) wrappers; no cluster multicast anywhere ----

@@ -45,7 +45,7 @@ const DebugWaits &debug_waits();
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events = nullptr,
                   void *lazy_state = nullptr, float factor = 0.f, uint32_t grad_type = ADACOMP_GRAD_F32,
-                  unsigned char *own_scratch = nullptr);
+                  unsigned char *own_scratch = nullptr, uint32_t quantiser = ADACOMP_QUANT_BIN_MAX_MEAN);
 int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                          uint64_t *count_out, void *stream);
 int lazy_state_init(void *state, uint64_t n, uint32_t L_T, void *stream);

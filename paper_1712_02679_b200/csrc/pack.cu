@@ -107,13 +107,13 @@ int launch_generic(const PassArgs &args, const DeviceInfo &info, cudaStream_t st
 // `own_scratch` (optional): the scratch to use in place of the one behind the stream in packed_out.
 int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, void *packed_out,
                   uint64_t *count_out, void *stream, uint32_t flags, void *const *events, void *lazy_state,
-                  float factor, uint32_t grad_type, unsigned char *own_scratch)
+                  float factor, uint32_t grad_type, unsigned char *own_scratch, uint32_t quantiser)
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
     if (flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
     if (factor != 0.f && !(factor > 0.f && factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
-    if (grad_type > ADACOMP_GRAD_F16) return ADACOMP_ERR_FLAGS;
+    if (grad_type > ADACOMP_GRAD_F16 || quantiser > ADACOMP_QUANT_SENT_MEAN) return ADACOMP_ERR_FLAGS;
     if (misaligned(grad) || misaligned(residue) || misaligned(packed_out) ||
         (reinterpret_cast<uintptr_t>(count_out) & 7u))
         return ADACOMP_ERR_ALIGN;
@@ -144,7 +144,7 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     mark(0);
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_type,
-                      debug_waits().limit, debug_waits().withhold_pack};
+                      quantiser, debug_waits().limit, debug_waits().withhold_pack};
         const bool fast = fast_L_T(L_T) && flags == 0 && info->fast_ready;
         // (one-bin tiles fill the pipelined kernel's 4000-element stages only in part: below 2800 elements the
         // warp-per-part kernel is faster, measured; lazy-scale mode exists in the pipelined kernel only)
@@ -164,7 +164,8 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         }
     }
     mark(1);
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags | (factor != 0.f ? kFlagFactor : 0u), reinterpret_cast<u64 *>(count_out), lazy);
+    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags | (factor != 0.f ? kFlagFactor : 0u) | (quantiser ? kFlagQuant : 0u),
+                                 reinterpret_cast<u64 *>(count_out), lazy);
     mark(2);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
@@ -225,7 +226,7 @@ int compress_static_impl(const float *grad, float *residue, uint64_t n, uint32_t
     }
     // the same kernels, in the same order, as adacomp_compress: only the scratch is elsewhere
     return compress_impl(grad, residue, n, L_T, packed_out, count_out, stream, 0, nullptr, nullptr, 0.f, ADACOMP_GRAD_F32,
-                         g_static_scratch_addr[dev]);
+                         g_static_scratch_addr[dev], ADACOMP_QUANT_BIN_MAX_MEAN);
 }
 
 

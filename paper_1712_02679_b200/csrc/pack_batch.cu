@@ -50,7 +50,7 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
             cur = li;
         }
         const BatchLayer &L = b.layer[li];
-        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, L.factor, L.grad_type};
+        const TileIo io{L.grad, L.residue, L.packed, L.packed + L.geo.scratch_at, 0u, L.factor, L.grad_type, 0u, nullptr};
         if (L.geo.w == 1u) generic_tile<unsigned char>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
         else generic_tile<unsigned short>(io, L.geo, gt - L.tile_first, smem_raw, s_tmp, s_acc);
     }

@@ -33,6 +33,7 @@ struct PassArgs {
     unsigned char *lazy_state;  // lazy mode: header + per-segment masks of the elements sent last step
     float factor;               // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW (Section 2.4's scale-factor)
     u32 grad_type;              // ADACOMP_GRAD_*: `grad` points to binary32 values, or to bfloat16 / binary16 ones (widened exactly on load)
+    u32 quantiser;              // 0: scale = mean of the bin maxima (Section 2.5); 1: mean |G| of the sent elements
     long long wait_limit;       // cycles a wait for a stage may take (kWaitCycles unless a test shortened it)
     u32 withhold;               // testing aid: CTA 0 starts no copies for its tile number `withhold` (0: none)
 };
@@ -60,7 +61,8 @@ struct FastSmem {
     static constexpr u32 kSegmaxAt = kWtotAt + 4 * 8;
     static constexpr u32 kBinmaxAt = kSegmaxAt + 4 * kTileSegs;
     static constexpr u32 kAccAt = kBinmaxAt + 4 * 4 * kSmallBins;     // (SPB = 0: two buffers each of bin maxima and counts) 8-byte aligned
-    static constexpr u32 kBarAt = kAccAt + 8 * (kWindows + 1);
+    static constexpr u32 kAcc2At = kAccAt + 8 * (kWindows + 1);       // (second quantiser) exact sum of the sent |G|
+    static constexpr u32 kBarAt = kAcc2At + 8 * (kWindows + 1);
     static constexpr u32 kAbortAt = kBarAt + 8 * kStages;
     static constexpr u32 kBytes = kAbortAt + 16;
 };
@@ -79,6 +81,7 @@ tile_pass_fast(PassArgs a)
     float *s_segmax = reinterpret_cast<float *>(smem + FastSmem::kSegmaxAt);
     float *s_binmax = reinterpret_cast<float *>(smem + FastSmem::kBinmaxAt);
     u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
+    u64 *s_acc2 = reinterpret_cast<u64 *>(smem + FastSmem::kAcc2At);
     u64 *s_full = reinterpret_cast<u64 *>(smem + FastSmem::kBarAt);
     volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FastSmem::kAbortAt);
 
@@ -133,7 +136,7 @@ tile_pass_fast(PassArgs a)
         lazy_mask = reinterpret_cast<u32 *>(a.lazy_state + kLazyHeaderBytes);
     }
 
-    if (tid < kWindows + 1) s_acc[tid] = 0;
+    if (tid < kWindows + 1) s_acc[tid] = s_acc2[tid] = 0;
     if (ANY)
         for (int b = tid; b < 4 * kSmallBins; b += kFastThreads) s_anymax[b] = 0;
     if (tid == 0) {
@@ -312,6 +315,17 @@ tile_pass_fast(PassArgs a)
                 const u32 idx = ANY && j >= cut ? (u32)(j - cut) : seg_in_bin + j;      // the element's place in its bin
                 s_words[at++] = (Word)((idx << 2) | 1u | (neg << 1));
             }
+            if (a.quantiser) {
+                // the second quantiser: the exact sum of |G| over the sent elements, a sent element per lane and round
+                const u32 rounds = __reduce_max_sync(0xffffffffu, cnt);
+                u32 left = selmask;
+                for (u32 r = 0; r < rounds; r++) {
+                    const bool have = left != 0u;
+                    const int j = have ? __ffs(left) - 1 : 0;
+                    left &= left - 1u;
+                    warp_accumulate_shared(s_acc2, fabsf(pr[j]), have);
+                }
+            }
             if (LAZY) lazy_mask[tile * (u64)kTileSegs + tid] = selmask;
             if (ANY) {
                 if (tid < TB) {
@@ -372,8 +386,9 @@ tile_pass_fast(PassArgs a)
             }
         }
         if (lane < kWindows) {
-            const u64 v = s_acc[lane];
+            const u64 v = s_acc[lane], v2 = s_acc2[lane];
             if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + lane, v);
+            if (v2) atomicAdd(reinterpret_cast<u64 *>(a.scratch + kCtlSentSumAt) + lane, v2);
         }
     }
 }
@@ -393,6 +408,8 @@ struct TileIo {                 // the buffers of one layer, as the generic tile
     u32 literal;
     float factor;               // as in PassArgs
     u32 grad_type;
+    u32 quantiser;              // as in PassArgs (then s_acc2 collects the exact sum of the sent |G|)
+    u64 *s_acc2;
 };
 
 template <typename Word>
@@ -518,6 +535,7 @@ __device__ void generic_tile(const TileIo &a, const Geometry &geo, u64 tile, uns
                 const u32 pos = at + __popc(mask & ((1u << lane) - 1u));
                 s_words[pos] = (Word)(((u32)j << 2) | (g < 0.f ? 3u : 1u));
             }
+            if (a.quantiser && mask) warp_accumulate_shared(a.s_acc2, fabsf(g), sel);
             at += __popc(mask);
         }
     }
@@ -620,6 +638,8 @@ __device__ void generic_tile_one_bin(const TileIo &a, const Geometry &geo, u64 t
             const bool sel = fabsf(k) >= m && k != 0.f;
             const u32 mask = __ballot_sync(0xffffffffu, sel);
             if (sel) s_words[at + __popc(mask & ((1u << lane) - 1u))] = (Word)(((u32)j << 2) | (k < 0.f ? 3u : 1u));
+            // (the second quantiser needs |G| itself: it was written through to the residue before the last barrier)
+            if (a.quantiser && mask) warp_accumulate_shared(a.s_acc2, sel ? fabsf(a.residue[base + j]) : 0.f, sel);
             at += __popc(mask);
         }
     __syncthreads();
@@ -646,18 +666,19 @@ tile_pass_generic(PassArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u32 s_tmp[33];
-    __shared__ u64 s_acc[kWindows + 1];
+    __shared__ u64 s_acc[kWindows + 1], s_acc2[kWindows + 1];
     const int tid = threadIdx.x;
-    if (tid < kWindows + 1) s_acc[tid] = 0;
+    if (tid < kWindows + 1) s_acc[tid] = s_acc2[tid] = 0;
     __syncthreads();
-    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_type};
+    const TileIo io{a.grad, a.residue, a.packed, a.scratch, a.literal, a.factor, a.grad_type, a.quantiser, s_acc2};
     for (u64 tile = blockIdx.x; tile < a.geo.n_tiles; tile += gridDim.x) {
         if (a.geo.tile_bins == 1u && sizeof(Word) == 2) generic_tile_one_bin<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
         else generic_tile<Word>(io, a.geo, tile, smem_raw, s_tmp, s_acc);
     }
     if (tid < kWindows) {
-        const u64 v = s_acc[tid];
+        const u64 v = s_acc[tid], v2 = s_acc2[tid];
         if (v) atomicAdd(reinterpret_cast<u64 *>(a.scratch) + tid, v);
+        if (v2) atomicAdd(reinterpret_cast<u64 *>(a.scratch + kCtlSentSumAt) + tid, v2);
     }
 }
 
@@ -742,7 +763,10 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
         tile_off[geo.n_tiles] = n_sel;
         const u64 *win = reinterpret_cast<const u64 *>(scratch);
         float scale = 0.f;
-        if (geo.n_bins) {
+        if (flags & kFlagQuant) {
+            // the second quantiser: the mean |G| of the sent elements
+            if (n_sel) scale = __double2float_rn(__ddiv_rn(windows_to_double(win + kCtlSentSumAt / 8), (double)n_sel));
+        } else if (geo.n_bins) {
             const double S = windows_to_double(win);
             scale = __double2float_rn(__ddiv_rn(S, (double)geo.n_bins));
         }
@@ -750,7 +774,7 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
         u32 *h32 = reinterpret_cast<u32 *>(packed);
         u64 *h64 = reinterpret_cast<u64 *>(packed);
         h32[0] = kMagic;
-        h32[1] = 1u | (geo.w << 16) | ((flags & (ADACOMP_FLAG_LITERAL | kFlagFactor)) << 24);
+        h32[1] = 1u | (geo.w << 16) | ((flags & (ADACOMP_FLAG_LITERAL | kFlagFactor | kFlagQuant)) << 24);
         h32[2] = geo.L_T;
         h32[3] = geo.tile_bins;
         h64[2] = geo.n;
