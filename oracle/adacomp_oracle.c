@@ -343,6 +343,151 @@ int adacomp_oracle_pack_general(const float *dW, float *residue, uint64_t n, uin
     return overflow ? -3 : 0;
 }
 
+/* ---- stream version 2: the bins are told apart by a flag in the words -------- */
+/*
+ * The paper's rate figures count the words alone (Section "Experiment Results": 8 or 16 bits per sent
+ * element), i.e. they leave out whatever tells the receiver which bin a word belongs to.  Version 1 spends a
+ * count per bin on that (1 or 2 bytes per L_T elements).  Version 2 spends nothing but one of the word's two
+ * spare bits: the first word of every bin carries a flag.  Layout: the 64-byte header (version field 2; bytes
+ * 52..55 hold the number of bins that send nothing), the tile directory (u64 word offsets, as in version 1,
+ * counted in version-2 words), the words, zero-padded to 16 bytes.  There is no count section.
+ *   word = (index_in_bin << 2) | (first_of_bin << 1) | negative
+ * A bin that sends nothing is one marker word with first_of_bin set and the index L_T (one past the bin), so that
+ * every bin owns exactly one flagged word.  Words are 8 bits wide for L_T <= 63 (the marker's index must fit
+ * 6 bits) and 16 bits up to 16383; L_T = 16384 has no version-2 form.
+ */
+static uint32_t v2_word_bytes(uint32_t L_T) { return L_T <= 63u ? 1u : 2u; }
+
+uint64_t adacomp_oracle_v2_bytes(uint64_t n, uint32_t L_T, uint64_t n_words)
+{
+    geometry g = geometry_of(n, L_T);
+    return align16(ORACLE_HEADER_BYTES + 8u * (g.n_tiles + 1u)) + align16(n_words * v2_word_bytes(L_T));
+}
+
+/* Version 1 stream in, version 2 stream out.  Returns 0, -1 bad argument, -3 out_cap too small, -4 malformed input. */
+int adacomp_oracle_to_v2(const uint8_t *v1, uint8_t *out, uint64_t out_cap)
+{
+    if (!v1 || !out) return -1;
+    if (get_u32(v1) != ORACLE_MAGIC || get_u16(v1 + 4) != 1) return -4;
+    const uint32_t L_T = get_u32(v1 + 8);
+    const uint64_t n = get_u64(v1 + 16), n_sel = get_u64(v1 + 40);
+    if (L_T == 0 || L_T >= 16384u) return -1;
+    geometry g = geometry_of(n, L_T);
+    const uint32_t w2 = v2_word_bytes(L_T);
+    const uint8_t *bin_cnt = v1 + g.bin_cnt_at, *words = v1 + g.payload_at;
+    uint64_t empty = 0;
+    for (uint64_t b = 0; b < g.n_bins; b++) empty += (g.w == 1u ? bin_cnt[b] : get_u16(bin_cnt + 2u * b)) == 0;
+    const uint64_t n_words = n_sel + empty, pay2 = align16(ORACLE_HEADER_BYTES + 8u * (g.n_tiles + 1u));
+    const uint64_t bytes_used = pay2 + align16(n_words * w2);
+    if (bytes_used > out_cap) return -3;
+    memset(out, 0, bytes_used);
+    memcpy(out, v1, ORACLE_HEADER_BYTES);
+    put_u16(out + 4, 2);
+    out[6] = (uint8_t)w2;
+    put_u32(out + 52, (uint32_t)empty);
+    put_u64(out + 56, bytes_used);
+    uint64_t at1 = 0, at2 = 0;
+    for (uint64_t b = 0; b < g.n_bins; b++) {
+        if (b % g.tile_bins == 0) put_u64(out + ORACLE_HEADER_BYTES + 8u * (b / g.tile_bins), at2);
+        const uint32_t count = g.w == 1u ? bin_cnt[b] : get_u16(bin_cnt + 2u * b);
+        if (count == 0) {                                       /* the marker of a bin that sends nothing */
+            const uint32_t word = (L_T << 2) | 2u;
+            if (w2 == 1u) out[pay2 + at2] = (uint8_t)word; else put_u16(out + pay2 + 2u * at2, (uint16_t)word);
+            at2++;
+        }
+        for (uint32_t j = 0; j < count; j++, at1++, at2++) {
+            if (at1 >= n_sel) return -4;
+            const uint32_t word1 = g.w == 1u ? words[at1] : get_u16(words + 2u * at1);
+            const uint32_t code = word1 & 3u;
+            if (code != 1u && code != 3u) return -4;
+            const uint32_t word = (word1 & ~3u) | (j == 0 ? 2u : 0u) | (code == 3u ? 1u : 0u);
+            if (w2 == 1u) out[pay2 + at2] = (uint8_t)word; else put_u16(out + pay2 + 2u * at2, (uint16_t)word);
+        }
+    }
+    put_u64(out + ORACLE_HEADER_BYTES + 8u * g.n_tiles, at2);
+    return at1 == n_sel ? 0 : -4;
+}
+
+/* Version 2 stream in, version 1 stream out (the inverse of the above).  Same return codes. */
+int adacomp_oracle_from_v2(const uint8_t *v2, uint8_t *out, uint64_t out_cap)
+{
+    if (!v2 || !out) return -1;
+    if (get_u32(v2) != ORACLE_MAGIC || get_u16(v2 + 4) != 2) return -4;
+    const uint32_t L_T = get_u32(v2 + 8);
+    const uint64_t n = get_u64(v2 + 16), n_sel = get_u64(v2 + 40), empty = get_u32(v2 + 52);
+    if (L_T == 0 || L_T >= 16384u) return -1;
+    geometry g = geometry_of(n, L_T);
+    const uint32_t w2 = v2_word_bytes(L_T);
+    if (v2[6] != w2) return -4;
+    const uint64_t pay2 = align16(ORACLE_HEADER_BYTES + 8u * (g.n_tiles + 1u)), n_words = n_sel + empty;
+    const uint64_t bytes_used = g.payload_at + align16(n_sel * g.w);
+    if (bytes_used > out_cap) return -3;
+    memset(out, 0, bytes_used);
+    memcpy(out, v2, ORACLE_HEADER_BYTES);
+    put_u16(out + 4, 1);
+    out[6] = (uint8_t)g.w;
+    put_u32(out + 52, 0);
+    put_u64(out + 56, bytes_used);
+    uint8_t *tile_off = out + g.tile_off_at, *bin_cnt = out + g.bin_cnt_at, *words = out + g.payload_at;
+    uint64_t at1 = 0, bin = 0;           /* `bin`: bins opened so far */
+    uint32_t count = 0;
+    for (uint64_t at2 = 0; at2 < n_words; at2++) {
+        const uint32_t word = w2 == 1u ? v2[pay2 + at2] : get_u16(v2 + pay2 + 2u * at2);
+        if (word & 2u) {                                        /* a new bin starts */
+            if (bin > 0) { if (g.w == 1u) bin_cnt[bin - 1] = (uint8_t)count; else put_u16(bin_cnt + 2u * (bin - 1), (uint16_t)count); }
+            if (bin >= g.n_bins) return -4;
+            if (bin % g.tile_bins == 0) put_u64(tile_off + 8u * (bin / g.tile_bins), at1);
+            bin++;
+            count = 0;
+        } else if (bin == 0) {
+            return -4;
+        }
+        if ((word >> 2) == L_T) { if (!(word & 2u)) return -4; continue; }      /* the marker of an empty bin */
+        if ((word >> 2) > L_T || at1 >= n_sel) return -4;
+        const uint32_t word1 = (word & ~3u) | ((word & 1u) ? 3u : 1u);
+        if (g.w == 1u) words[at1] = (uint8_t)word1; else put_u16(words + 2u * at1, (uint16_t)word1);
+        at1++;
+        count++;
+    }
+    if (bin > 0) { if (g.w == 1u) bin_cnt[bin - 1] = (uint8_t)count; else put_u16(bin_cnt + 2u * (bin - 1), (uint16_t)count); }
+    put_u64(tile_off + 8u * g.n_tiles, at1);
+    return (bin == g.n_bins && at1 == n_sel) ? 0 : -4;
+}
+
+/* unpack() and sum of version-2 streams, decoded from the flags alone (no counts are rebuilt): the same ordered
+ * sum as adacomp_oracle_unpack_sum gives for the version-1 forms of the streams. */
+int adacomp_oracle_unpack_sum_v2(const uint8_t *const *streams, uint32_t k, float *dst, uint64_t n)
+{
+    if (!streams || k == 0 || (n && !dst)) return -1;
+    for (uint64_t i = 0; i < n; i++) dst[i] = 0.0f;
+    for (uint32_t l = 0; l < k; l++) {
+        const uint8_t *s = streams[l];
+        if (get_u32(s) != ORACLE_MAGIC || get_u16(s + 4) != 2 || get_u64(s + 16) != n) return -4;
+        const uint32_t L_T = get_u32(s + 8), w2 = v2_word_bytes(L_T);
+        if (L_T == 0 || L_T >= 16384u || s[6] != w2) return -4;
+        geometry g = geometry_of(n, L_T);
+        const uint64_t pay2 = align16(ORACLE_HEADER_BYTES + 8u * (g.n_tiles + 1u));
+        const uint64_t n_words = get_u64(s + 40) + get_u32(s + 52);
+        uint32_t scale_bits = get_u32(s + 48);
+        float scale;
+        memcpy(&scale, &scale_bits, 4);
+        uint64_t bin = 0;                /* bins opened so far: the current one is bin - 1 */
+        for (uint64_t at = 0; at < n_words; at++) {
+            const uint32_t word = w2 == 1u ? s[pay2 + at] : get_u16(s + pay2 + 2u * at);
+            if (word & 2u) bin++;
+            if (bin == 0 || bin > g.n_bins) return -4;
+            const uint32_t idx = word >> 2;
+            if (idx == L_T) continue;
+            const uint64_t index = (bin - 1) * L_T + idx;
+            if (idx > L_T || index >= n) return -4;
+            if (word & 1u) dst[index] = dst[index] - scale;
+            else dst[index] = dst[index] + scale;
+        }
+        if (bin != g.n_bins) return -4;
+    }
+    return 0;
+}
+
 /* ---- unpack() and sum ----------------------------------------------------- */
 /*
  * dst[n] is overwritten with the sum over the k streams, taken in stream

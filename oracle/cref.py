@@ -37,6 +37,13 @@ def lib() -> C.CDLL:
         _lib.adacomp_oracle_pack_general.restype = C.c_int
         _lib.adacomp_oracle_pack_general.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
                                                      C.c_float, C.c_uint32, C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.adacomp_oracle_v2_bytes.restype = C.c_uint64
+        _lib.adacomp_oracle_v2_bytes.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
+        for name in ("adacomp_oracle_to_v2", "adacomp_oracle_from_v2"):
+            getattr(_lib, name).restype = C.c_int
+            getattr(_lib, name).argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        _lib.adacomp_oracle_unpack_sum_v2.restype = C.c_int
+        _lib.adacomp_oracle_unpack_sum_v2.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
         _lib.adacomp_oracle_unpack_sum.restype = C.c_int
         _lib.adacomp_oracle_unpack_sum.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64]
     return _lib
@@ -142,6 +149,42 @@ def unpack_sum(streams: Sequence[np.ndarray], n: int) -> np.ndarray:
     rc = lib().adacomp_oracle_unpack_sum(ptrs, len(keep), _ptr(dst) if n else None, n)
     if rc != 0:
         raise RuntimeError(f"adacomp_oracle_unpack_sum failed: {rc}")
+    return dst
+
+
+def to_v2(raw_v1: np.ndarray) -> np.ndarray:
+    """A version-1 stream re-encoded as version 2 (the bins told apart by a flag in the words; no count section)."""
+    v1 = np.ascontiguousarray(raw_v1, dtype=np.uint8)
+    p = parse(v1)
+    n_empty = int(np.count_nonzero(p.bin_cnt == 0))
+    cap = int(lib().adacomp_oracle_v2_bytes(p.n, p.L_T, p.n_sel + n_empty))
+    out = np.empty(cap, dtype=np.uint8)
+    rc = lib().adacomp_oracle_to_v2(_ptr(v1), _ptr(out), cap)
+    if rc != 0:
+        raise RuntimeError(f"adacomp_oracle_to_v2 failed: {rc}")
+    return out
+
+
+def from_v2(raw_v2: np.ndarray) -> np.ndarray:
+    """The version-1 form of a version-2 stream."""
+    v2 = np.ascontiguousarray(raw_v2, dtype=np.uint8)
+    L_T, n, n_sel = struct.unpack_from("<I", v2, 8)[0], struct.unpack_from("<Q", v2, 16)[0], struct.unpack_from("<Q", v2, 40)[0]
+    cap = stream_bytes(n, L_T, n_sel)
+    out = np.empty(cap, dtype=np.uint8)
+    rc = lib().adacomp_oracle_from_v2(_ptr(v2), _ptr(out), cap)
+    if rc != 0:
+        raise RuntimeError(f"adacomp_oracle_from_v2 failed: {rc}")
+    return out
+
+
+def unpack_sum_v2(streams: Sequence[np.ndarray], n: int) -> np.ndarray:
+    """Sum k version-2 streams, in order, into a dense float32 vector (decoded from the flags alone)."""
+    keep: List[np.ndarray] = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    ptrs = (C.c_void_p * len(keep))(*[_ptr(s) for s in keep])
+    dst = np.empty(n, dtype=np.float32)
+    rc = lib().adacomp_oracle_unpack_sum_v2(ptrs, len(keep), _ptr(dst) if n else None, n)
+    if rc != 0:
+        raise RuntimeError(f"adacomp_oracle_unpack_sum_v2 failed: {rc}")
     return dst
 
 

@@ -115,3 +115,38 @@ def unpack_sum(streams: Sequence[Tuple[Sequence[int], Sequence[int], float]], n:
                 elif code == 2:
                     raise ValueError("reserved ternary code")
     return dst
+
+
+def to_stream_v2(n: int, L_T: int, bin_cnt: Sequence[int], words: Sequence[int], scale,
+                 literal: bool = False, factor: float = 0.0, quantiser: int = 0) -> bytes:
+    """Serialise to stream version 2: no counts; the first word of every bin carries a flag, a bin that sends
+    nothing is one marker word (flag set, index L_T).  word = (index << 2) | (first << 1) | negative."""
+    w = 1 if L_T <= 63 else 2
+    tb = _tile_bins(L_T)
+    n_bins = len(bin_cnt)
+    n_tiles = -(-n_bins // tb)
+    out_words: List[int] = []
+    tile_off: List[int] = []
+    at = 0
+    for b, count in enumerate(bin_cnt):
+        if b % tb == 0:
+            tile_off.append(len(out_words))
+        if count == 0:
+            out_words.append((L_T << 2) | 2)
+        for j in range(count):
+            word = words[at]
+            at += 1
+            out_words.append((word & ~3) | (2 if j == 0 else 0) | (1 if (word & 3) == 3 else 0))
+    tile_off.append(len(out_words))
+    fmt = "B" if w == 1 else "H"
+    pad16 = lambda b: b + bytes((-len(b)) % 16)
+    dir_bytes = struct.pack(f"<{n_tiles + 1}Q", *tile_off)
+    body = bytes((-(64 + len(dir_bytes))) % 16)
+    body = dir_bytes + body + pad16(struct.pack(f"<{len(out_words)}{fmt}", *out_words))
+    bytes_used = 64 + len(body)
+    scale_bits = struct.unpack("<I", struct.pack("<f", float(scale)))[0]
+    flags = (1 if literal else 0) | (2 if factor != 0.0 else 0) | (4 if quantiser == 1 else 0)
+    head = struct.pack("<IHBBIIQQQQIIQ", 0x31434441, 2, w, flags, L_T, tb, n, n_bins, n_tiles, len(words), scale_bits,
+                       sum(1 for c in bin_cnt if c == 0), bytes_used)
+    return head + body
+
