@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-lazy", action="store_true")
     ap.add_argument("--no-update", action="store_true", help="skip the fused unpack + average + SGD measurement")
+    ap.add_argument("--wire-version", type=int, default=2, choices=[1, 2],
+                    help="exchange workload: the stream version on the wire (2: first-of-bin flags, no per-bin counts)")
     ap.add_argument("--no-configs", action="store_true", help="skip the parameter-list configs appended to the default line")
     ap.add_argument("--cpu-log2n", type=int, default=26, help="oracle sample size (cpu_baseline)")
     ap.add_argument("--workload", default="sweep", choices=["sweep", "config1", "config2", "config3", "config4", "lstm", "ratecurve", "exchange"],
@@ -775,7 +777,7 @@ def run_exchange(a):
 
     from paper_1712_02679_b200 import binding as B
     from paper_1712_02679_b200 import ranks
-    from paper_1712_02679_b200.exchange import exchange
+    from paper_1712_02679_b200.exchange import exchange, exchange_v2
 
     rank, world, local = ranks.rank_env()
     if not torch.cuda.is_available():
@@ -806,6 +808,11 @@ def run_exchange(a):
     packed = torch.empty(cap, dtype=torch.uint8, device=dev)
     count = torch.zeros(2, dtype=torch.int64, device=dev)
     recv = torch.empty(world * cap, dtype=torch.uint8, device=dev) if world > 1 else None
+    v2 = a.wire_version == 2 and L_T < 16384
+    if v2:
+        wire_buf = torch.empty(B.adacomp_v2_capacity(n, L_T), dtype=torch.uint8, device=dev)
+        recv_wire = torch.empty(world * wire_buf.numel(), dtype=torch.uint8, device=dev) if world > 1 else None
+        recv_packed = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(world)]
     dW = torch.empty(n, device=dev)
     dst = torch.empty(n, device=dev)
     for step in range(PREWARM_STEPS + 1):
@@ -830,11 +837,16 @@ def run_exchange(a):
         B.adacomp_compress(dW, residue, n, L_T, packed, count, stream)
         e[1].record(stream)
         used = int(count[1])                    # exchange() sends the sizes first: the host needs this one
-        streams = exchange(packed, used, recv=recv)
+        if v2:
+            streams, wire_bytes = exchange_v2(packed, n, L_T, wire_buf, recv_wire, recv_packed)
+        else:
+            streams = exchange(packed, used, recv=recv)
+            wire_bytes = [int(t.numel()) for t in streams]
         e[2].record(stream)
         B.adacomp_decompress_accumulate_ex(streams, world, dst, n, L_T, stream)
         e[3].record(stream)
-        wire = sum(int(t.numel()) for t in streams)
+        wire = sum(wire_bytes)
+        v1_bytes = sum(int(t.numel()) for t in streams)
         if it >= W:
             evs.append(e)
     barrier()
@@ -859,9 +871,13 @@ def run_exchange(a):
             "config": {"workload": f"pack -> exchange -> decode-sum with every rank a learner: flat fp32 gradient n=2^{n.bit_length() - 1} "
                                    f"per rank, L_T={L_T}, dW~N(0,1e-3), residue pre-warmed {PREWARM_STEPS} steps",
                        "exchange": f"all-gather of the sizes, then of the streams padded to the longest ({backend}); received "
-                                   "streams land in the rank's own memory before the decoder reads them",
+                                   "streams land in the rank's own memory before the decoder reads them; on the wire: stream version "
+                                   + ("2 (first-of-bin flags, no per-bin counts; re-encoded by adacomp_stream_to_v2 / _from_v2 on either side)"
+                                      if v2 else "1"),
                        "l2": "arrays far beyond the 126 MB L2" if 4 * n > (1 << 29) else "small case"},
             "pack_ms": v[1], "exchange_ms": v[2], "decode_sum_ms": v[3], "stream_bytes_received_per_rank": wire,
+            "version_1_bytes_of_the_same_streams": v1_bytes,
+            "rate_on_the_wire": 4.0 * n * world / max(wire, 1), "rate_version_1": 4.0 * n * world / max(v1_bytes, 1),
             "same_sum_on_every_rank": same, "device_status": status, "clocks": clocks,
             "gpu_launches": K * 4,
         }
@@ -918,9 +934,17 @@ def run_rate_curve(a):
                 t_c.append(ev[0].elapsed_time(ev[1]) / k)
                 t_d.append(ev[1].elapsed_time(ev[2]))
         n_sel, used = (int(v) for v in count[0].cpu())
+        used_v2 = None
+        if L_T < 16384:
+            wire_buf = torch.empty(B.adacomp_v2_capacity(n, L_T), dtype=torch.uint8, device=dev)
+            c2 = torch.zeros(2, dtype=torch.int64, device=dev)
+            B.adacomp_stream_to_v2(packed[0], wire_buf, c2, n, L_T)
+            used_v2 = int(c2[1])
+            del wire_buf
         word_bits = 8 if L_T <= 64 else 16
         rows.append({"L_T": L_T, "selected_fraction": n_sel / n,
                      "rate_paper_accounting": 32.0 * n / max(word_bits * n_sel, 1), "rate_on_the_wire": 4.0 * n / used,
+                     "rate_on_the_wire_version_2": (4.0 * n / used_v2) if used_v2 else None,
                      "pack_ms": statistics.mean(t_c), "pack_gbs": 4.0 * n / (statistics.mean(t_c) * 1e-3) / 1e9,
                      "decode_sum_ms": statistics.mean(t_d),
                      "decode_sum_gbs": (4.0 * n + sum(int(c[1]) for c in count)) / (statistics.mean(t_d) * 1e-3) / 1e9})

@@ -442,6 +442,34 @@ int adacomp_set_device(int device);
 int adacomp_device_status(uint32_t *host_out, void *stream);
 
 /*
+ * Stream version 2, for the wire.  The paper's rate figures (Section "Experiment Results": 8 or 16 bits per sent
+ * element, 40x at L_T = 50 and 200x at L_T = 500) count the words alone; the streams above also carry a count per bin
+ * so that a decoder can find a word's bin (1 or 2 bytes per L_T elements: 29.3x on the wire against 34.9x by the
+ * paper's accounting at L_T = 50).  Version 2 tells the bins apart with one of the word's own spare bits instead:
+ *   word = (index_in_bin << 2) | (first_of_bin << 1) | negative
+ * and a bin that sends nothing is one marker word (first_of_bin set, index L_T), so every bin owns exactly one
+ * flagged word.  Layout: the 64-byte header (version 2; bytes 52..55: bins that send nothing), the tile directory
+ * (u64 offsets in version-2 words), the words, zero-padded to 16 bytes; no count section.  Words are 8 bits wide for
+ * L_T <= 63 and 16 bits up to 16383 (the marker's index must fit); L_T = 16384 has no version-2 form.
+ * The decoders read version 1; these two calls re-encode a stream either way (three small kernels each), so that
+ * exchange() can put version 2 on the wire:
+ *   adacomp_stream_to_v2    packed: device, a version-1 stream of shape (n, L_T) as adacomp_compress* leaves it;
+ *                           out_v2: device, out_capacity >= adacomp_v2_capacity(n, L_T) bytes, 16-byte aligned;
+ *                           count_out: device, uint64_t[2] {words incl. markers, bytes_used} (may be NULL).
+ *   adacomp_stream_from_v2  in_v2: device, a version-2 stream; packed_out: device, out_capacity >= the stream part
+ *                           of adacomp_packed_capacity(n, L_T) (that value always suffices); receives the
+ *                           version-1 stream, byte for byte what the sender converted.
+ * A header that is not of the given shape and version sets ADACOMP_DEV_HEADER_MISMATCH and nothing else is written;
+ * a stream that contradicts itself sets ADACOMP_DEV_BAD_STREAM and every write stays inside the output.
+ * Host errors as for adacomp_compress (ADACOMP_ERR_SIZE: out_capacity too small; ADACOMP_ERR_L_T also for 16384).
+ */
+size_t adacomp_v2_capacity(uint64_t n, uint32_t L_T);
+int adacomp_stream_to_v2(const void *packed, void *out_v2, uint64_t out_capacity, uint64_t *count_out, uint64_t n,
+                         uint32_t L_T, void *stream);
+int adacomp_stream_from_v2(const void *in_v2, void *packed_out, uint64_t out_capacity, uint64_t n, uint32_t L_T,
+                           void *stream);
+
+/*
  * Testing aid for the bounded device-side waits (every wait of a kernel on a copy in flight gives up after a
  * limit, raises ADACOMP_DEV_TIMEOUT, lets the copies it did start land and returns; no kernel spins without a
  * limit).  This call lets a test see that path run without anything being wrong with the device:

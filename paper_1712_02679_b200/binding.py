@@ -490,6 +490,31 @@ def adacomp_device_status(stream=None) -> int:
     return int(out.value)
 
 
+def adacomp_v2_capacity(n: int, L_T: int) -> int:
+    f = lib().adacomp_v2_capacity
+    f.restype, f.argtypes = C.c_size_t, [C.c_uint64, C.c_uint32]
+    return int(f(int(n), int(L_T)))
+
+
+def adacomp_stream_to_v2(packed, out_v2, count_out, n: int, L_T: int, stream=None) -> None:
+    """A version-1 stream re-encoded as version 2 (first-of-bin flags, no counts): the form for the wire."""
+    f = lib().adacomp_stream_to_v2
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p]
+    _check(f(_dev_ptr(packed, "packed", torch.uint8), _dev_ptr(out_v2, "out_v2", torch.uint8), int(out_v2.numel()),
+             _dev_ptr(count_out, "count_out", torch.int64) if count_out is not None else None, int(n), int(L_T),
+             _stream(stream)), "adacomp_stream_to_v2")
+
+
+def adacomp_stream_from_v2(in_v2, packed_out, n: int, L_T: int, stream=None) -> None:
+    """A version-2 stream re-encoded as version 1, which the decoders read."""
+    f = lib().adacomp_stream_from_v2
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p]
+    _check(f(_dev_ptr(in_v2, "in_v2", torch.uint8), _dev_ptr(packed_out, "packed_out", torch.uint8),
+             int(packed_out.numel()), int(n), int(L_T), _stream(stream)), "adacomp_stream_from_v2")
+
+
 def adacomp_debug_waits(wait_cycles: int = 0, withhold_pack_tile: int = 0, withhold_decode_item: int = 0) -> None:
     """Testing aid: the limit of the device-side waits and one withheld copy (see include/adacomp.h)."""
     f = lib().adacomp_debug_waits

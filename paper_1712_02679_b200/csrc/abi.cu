@@ -457,6 +457,25 @@ int adacomp_decompress_average_adam(const void *const *packed, uint32_t k_stream
     return decompress_impl(packed, k_streams, nullptr, stream, n, L_T, &ep);
 }
 
+size_t adacomp_v2_capacity(uint64_t n, uint32_t L_T)
+{
+    if (L_T == 0 || L_T >= ADACOMP_MAX_L_T) return 0;
+    const Geometry g = make_geometry(n, L_T);
+    return (size_t)(align_up(kHeaderBytes + 8 * (g.n_tiles + 1), 16) + align_up(n * (L_T <= 63u ? 1u : 2u), 16));
+}
+
+int adacomp_stream_to_v2(const void *packed, void *out_v2, uint64_t out_capacity, uint64_t *count_out, uint64_t n,
+                         uint32_t L_T, void *stream)
+{
+    return stream_convert(packed, out_v2, out_capacity, count_out, n, L_T, true, stream);
+}
+
+int adacomp_stream_from_v2(const void *in_v2, void *packed_out, uint64_t out_capacity, uint64_t n, uint32_t L_T,
+                           void *stream)
+{
+    return stream_convert(in_v2, packed_out, out_capacity, nullptr, n, L_T, false, stream);
+}
+
 int adacomp_debug_waits(uint64_t wait_cycles, uint32_t withhold_pack_tile, uint32_t withhold_decode_item)
 {
     g_debug_waits.limit = wait_cycles ? (long long)(wait_cycles < (1ull << 40) ? wait_cycles : (1ull << 40)) : kWaitCycles;
@@ -483,7 +502,8 @@ int adacomp_device_status(uint32_t *host_out, void *stream)
                     status_read_pack_batch(&v) &&
                     status_read_decode(&v) &&
                     status_read_decode_opt(&v) &&
-                    status_read_decode_batch(&v);
+                    status_read_decode_batch(&v) &&
+                    status_read_wire(&v);
     if (!ok) return ADACOMP_ERR_CUDA;
     *host_out = v;
     return ADACOMP_OK;
@@ -501,6 +521,7 @@ int adacomp_device_status_reset(void *stream)
     status_reset_decode(st);
     status_reset_decode_opt(st);
     status_reset_decode_batch(st);
+    status_reset_wire(st);
     return cudaGetLastError() == cudaSuccess ? ADACOMP_OK : ADACOMP_ERR_CUDA;
 }
 

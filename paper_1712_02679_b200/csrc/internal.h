@@ -60,6 +60,10 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
 int launch_decode_opt(const DecodeArgs &args, const Epilogue &ep, const DeviceInfo &info, uint64_t hint_n,
                       uint32_t hint_L_T, cudaStream_t st);
 
+// wire.cu: a packed stream re-encoded as version 2 (to_v2) or back as version 1
+int stream_convert(const void *in, void *out, uint64_t out_capacity, uint64_t *count_out, uint64_t n, uint32_t L_T,
+                   bool to_v2, void *stream);
+
 // decode_batch.cu
 int launch_decode_batch(const DecodeBatchArgs &batch, u64 batch_tiles, const DeviceInfo &info, cudaStream_t st);
 
@@ -78,5 +82,6 @@ ADACOMP_STATUS_DECLARE(pack_batch)
 ADACOMP_STATUS_DECLARE(decode)
 ADACOMP_STATUS_DECLARE(decode_opt)
 ADACOMP_STATUS_DECLARE(decode_batch)
+ADACOMP_STATUS_DECLARE(wire)
 
 }  // namespace adacomp_impl

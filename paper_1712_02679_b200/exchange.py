@@ -7,8 +7,11 @@ streams padded to the longest one (rounded up to 16 bytes, which keeps every rec
 the 16-byte boundary the decoder asks for).  The received streams land in this rank's own memory
 before any kernel reads them; nothing here reads a peer's memory directly.
 
-This module only moves bytes: packing and decoding stay in the library's kernels
-(`adacomp_compress*`, `adacomp_decompress_accumulate*`, `adacomp_decompress_average_sgd`).
+`exchange` only moves bytes: packing and decoding stay in the library's kernels (`adacomp_compress*`,
+`adacomp_decompress_accumulate*`, `adacomp_decompress_average_sgd`).  `exchange_v2` puts stream version 2 on the
+wire (first-of-bin flags in place of the per-bin counts: the bytes the paper's rate figures count, plus a small
+directory): the sender re-encodes its stream with `adacomp_stream_to_v2`, the receiver turns every stream it gets
+back into version 1 with `adacomp_stream_from_v2`, which is what the decoders read.
 """
 from __future__ import annotations
 
@@ -66,3 +69,33 @@ def exchange(packed: torch.Tensor, bytes_used: int, group=None,
     elif step:
         dist.all_gather_into_tensor(recv[:world * step], packed[:step], group=group)
     return [recv[r * step:r * step + sizes[r]] for r in range(world)]
+
+
+def exchange_v2(packed: torch.Tensor, n: int, L_T: int, wire: torch.Tensor, recv_wire: Optional[torch.Tensor],
+                recv_packed: Sequence[torch.Tensor], group=None):
+    """exchange() with version-2 streams on the wire.
+
+    packed       this learner's version-1 stream (device, as adacomp_compress* left it).
+    wire         device uint8 scratch of adacomp_v2_capacity(n, L_T) bytes for this learner's version-2 stream.
+    recv_wire    device uint8 buffer of world_size * len(wire) bytes (None: allocated) for the gathered streams.
+    recv_packed  world_size device uint8 buffers of at least adacomp_packed_capacity(n, L_T) bytes each: they
+                 receive the learners' version-1 streams, in rank order, ready for the decoders.
+    Returns (streams, wire_bytes): the world_size version-1 streams (views of recv_packed, trimmed) and the bytes
+    each rank put on the wire (their version-2 lengths).
+    """
+    from . import binding as B
+
+    count = torch.zeros(2, dtype=torch.int64, device=packed.device)
+    B.adacomp_stream_to_v2(packed, wire, count, n, L_T)
+    used = int(count[1])
+    got = exchange(wire, used, group=group, recv=recv_wire)
+    streams = []
+    for r, v2 in enumerate(got):
+        # (a gathered slice starts on a 16-byte boundary: the padded size is a multiple of 16)
+        B.adacomp_stream_from_v2(v2, recv_packed[r], n, L_T)
+    torch.cuda.synchronize(packed.device)
+    for r in range(len(got)):
+        bytes_used = int(recv_packed[r][56:64].view(torch.int64)[0])
+        streams.append(recv_packed[r][:bytes_used])
+    return streams, [int(g.numel()) for g in got]
+

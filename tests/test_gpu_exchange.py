@@ -27,7 +27,7 @@ WORKER = textwrap.dedent("""
     from oracle import cref
     from paper_1712_02679_b200 import binding as B
     from paper_1712_02679_b200 import ranks
-    from paper_1712_02679_b200.exchange import exchange
+    from paper_1712_02679_b200.exchange import exchange, exchange_v2
     rank, world, local = ranks.rank_env()
     dist.init_process_group("gloo")
     dev = torch.device("cuda", 0)            # every rank on the one GPU
@@ -47,6 +47,9 @@ WORKER = textwrap.dedent("""
         packed = torch.empty(cap, dtype=torch.uint8, device=dev)
         count = torch.zeros(2, dtype=torch.int64, device=dev)
         recv = torch.empty(world * cap, dtype=torch.uint8, device=dev)
+        wire = torch.empty(B.adacomp_v2_capacity(n, L_T), dtype=torch.uint8, device=dev)
+        recv_wire = torch.empty(world * wire.numel(), dtype=torch.uint8, device=dev)
+        recv_packed = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(world)]
         w = torch.from_numpy(w_true.copy()).to(dev)
         v = torch.zeros(n, device=dev)
         dst = torch.empty(n, device=dev)
@@ -60,6 +63,14 @@ WORKER = textwrap.dedent("""
                 assert got[r].is_cuda and got[r].data_ptr() % 16 == 0
                 assert np.array_equal(got[r].cpu().numpy(), want[r]), (step, r)
             B.adacomp_decompress_accumulate_ex(got, world, dst, n, L_T)
+            torch.cuda.synchronize()
+            assert np.array_equal(dst.cpu().numpy().view(np.uint32), cref.unpack_sum(want, n).view(np.uint32)), step
+            # the same exchange with version-2 streams on the wire: fewer bytes, the same streams on arrival
+            streams2, wire_bytes = exchange_v2(packed, n, L_T, wire, recv_wire, recv_packed)
+            for r in range(world):
+                assert np.array_equal(streams2[r].cpu().numpy(), want[r]), (step, r)
+                assert wire_bytes[r] == cref.to_v2(want[r]).size < want[r].size
+            B.adacomp_decompress_accumulate_ex(streams2, world, dst, n, L_T)
             torch.cuda.synchronize()
             assert np.array_equal(dst.cpu().numpy().view(np.uint32), cref.unpack_sum(want, n).view(np.uint32)), step
             B.adacomp_decompress_average_sgd(got, world, w, v, n, L_T, 0.1, 0.9)
