@@ -83,6 +83,7 @@ extern "C" {
 /* flags of adacomp_compress_ex */
 #define ADACOMP_FLAG_LITERAL 1u       /* Algorithm 2 as printed: |H| >= g_max only */
 #define ADACOMP_FLAG_GENERIC_PATH 256u /* use the any-L_T kernel even where a specialised one exists */
+#define ADACOMP_FLAG_STREAMING 512u    /* use the streaming kernels even for a layer small enough for the one-kernel form */
 
 /* gradient formats (adacomp_options.grad_type): values narrower than binary32 are widened exactly as they are read */
 #define ADACOMP_GRAD_F32 0u
@@ -157,7 +158,12 @@ int adacomp_compress(const float *grad, float *residue, uint64_t n, uint32_t L_T
 int adacomp_compress_static(const float *grad, float *residue, uint64_t n, uint32_t L_T,
                             void *packed_out, uint64_t *count_out, void *stream);
 
-/* As adacomp_compress, with ADACOMP_FLAG_* bits. */
+/* As adacomp_compress, with ADACOMP_FLAG_* bits.
+ * Which kernels run never changes a byte of the result.  A layer of one of the bin lengths 50, 100, 125, 200,
+ * 250, 500, 1000 whose 4000-element tiles all fit in the shared memory of the CTAs that are resident together
+ * (4 tiles per CTA, 2 CTAs per SM: 4.7 M elements on 148 SMs) is packed by one cooperative kernel that visits
+ * the residue once; ADACOMP_FLAG_STREAMING takes the streaming kernels instead (a tile pass, the scale, and a
+ * second visit of the sent elements), which larger layers always take. */
 int adacomp_compress_ex(const float *grad, float *residue, uint64_t n, uint32_t L_T,
                         void *packed_out, uint64_t *count_out, void *stream, uint32_t flags);
 

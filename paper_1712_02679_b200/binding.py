@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libadacomp.so")
 
 ADACOMP_FLAG_LITERAL = 1
 ADACOMP_FLAG_GENERIC_PATH = 256
+ADACOMP_FLAG_STREAMING = 512
 ADACOMP_MAX_STREAMS = 64
 
 ADACOMP_DEV_NONFINITE = 1

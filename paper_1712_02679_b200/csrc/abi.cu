@@ -24,6 +24,7 @@ int device_info(DeviceInfo *&out)
         init_decode_info(d);
         init_pack_info(d);
         init_pack_batch_info(d);        // (after init_pack_info: it needs fast_ready)
+        init_pack_onchip_info(d);
         init_decode_batch_info(d);
         d.sms = sms;
     }
@@ -313,7 +314,7 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
         }
         if (!d.packed_out || !d.count_out || (d.n && (!d.grad || !d.residue))) return ADACOMP_ERR_NULL;
         if (d.L_T == 0 || d.L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-        if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
+        if (d.flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH | ADACOMP_FLAG_STREAMING)) return ADACOMP_ERR_FLAGS;
         if (misaligned(d.grad) || misaligned(d.residue) || misaligned(d.packed_out) ||
             (reinterpret_cast<uintptr_t>(d.count_out) & 7u))
             return ADACOMP_ERR_ALIGN;
@@ -352,9 +353,11 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
     // (without the pipelined batch kernel the batch runs the any-L_T tile code, which takes every format too)
     const uint32_t n_batches = (to_batch + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
     const uint32_t per_batch = n_batches ? (to_batch + n_batches - 1) / n_batches : (uint32_t)kBatchMax;
+    // (a lone layer gains nothing from the batch kernels, and the single-layer path may pack it in one kernel)
+    const bool lone = to_batch == 1;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (batched_at(t)) {
+        if (batched_at(t) && !lone) {
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
@@ -500,6 +503,7 @@ int adacomp_device_status(uint32_t *host_out, void *stream)
                     status_read_pack_fast_c(&v) &&
                     status_read_pack_fast_d(&v) &&
                     status_read_pack_batch(&v) &&
+                    status_read_pack_onchip(&v) &&
                     status_read_decode(&v) &&
                     status_read_decode_opt(&v) &&
                     status_read_decode_batch(&v) &&
@@ -518,6 +522,7 @@ int adacomp_device_status_reset(void *stream)
     status_reset_pack_fast_c(st);
     status_reset_pack_fast_d(st);
     status_reset_pack_batch(st);
+    status_reset_pack_onchip(st);
     status_reset_decode(st);
     status_reset_decode_opt(st);
     status_reset_decode_batch(st);

@@ -19,6 +19,7 @@ struct DeviceInfo {
     int dec_batch_per_sm = 0;   // 0: batched decode unavailable on this device
     int dec_batch_warps_per_sm[3] = {0, 0, 0};      // CTAs of the batched warp decoder per SM, by optimizer form
     bool fast_ready = false;
+    int onchip_ctas = 0;        // CTAs of the one-kernel pack() that are resident together; 0: unavailable on this device
 };
 
 
@@ -26,6 +27,7 @@ struct DeviceInfo {
 int device_info(DeviceInfo *&out);
 void init_pack_info(DeviceInfo &d);             // pack.cu, pack_fast_*.cu
 void init_pack_batch_info(DeviceInfo &d);       // pack_batch.cu
+void init_pack_onchip_info(DeviceInfo &d);      // pack_onchip.cu
 void init_decode_info(DeviceInfo &d);           // decode.cu, decode_opt.cu
 void init_decode_batch_info(DeviceInfo &d);     // decode_batch.cu
 
@@ -60,6 +62,10 @@ int decompress_impl(const void *const *packed, uint32_t k, float *dst, void *str
 int launch_decode_opt(const DecodeArgs &args, const Epilogue &ep, const DeviceInfo &info, uint64_t hint_n,
                       uint32_t hint_L_T, cudaStream_t st);
 
+// pack_onchip.cu: pack() of a layer whose tiles all fit in the resident CTAs' shared memory, in one kernel
+u64 onchip_tile_capacity(const DeviceInfo &d);
+int launch_pack_onchip(PassArgs &args, u64 *count_out, u32 header_flags, const DeviceInfo &info, cudaStream_t st);
+
 // wire.cu: a packed stream re-encoded as version 2 (to_v2) or back as version 1
 int stream_convert(const void *in, void *out, uint64_t out_capacity, uint64_t *count_out, uint64_t n, uint32_t L_T,
                    bool to_v2, void *stream);
@@ -79,6 +85,7 @@ ADACOMP_STATUS_DECLARE(pack_fast_b)
 ADACOMP_STATUS_DECLARE(pack_fast_c)
 ADACOMP_STATUS_DECLARE(pack_fast_d)
 ADACOMP_STATUS_DECLARE(pack_batch)
+ADACOMP_STATUS_DECLARE(pack_onchip)
 ADACOMP_STATUS_DECLARE(decode)
 ADACOMP_STATUS_DECLARE(decode_opt)
 ADACOMP_STATUS_DECLARE(decode_batch)

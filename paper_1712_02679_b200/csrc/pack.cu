@@ -111,7 +111,9 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
 {
     if (!packed_out || !count_out || (n && (!grad || !residue))) return ADACOMP_ERR_NULL;
     if (L_T == 0 || L_T > ADACOMP_MAX_L_T) return ADACOMP_ERR_L_T;
-    if (flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH)) return ADACOMP_ERR_FLAGS;
+    if (flags & ~(ADACOMP_FLAG_LITERAL | ADACOMP_FLAG_GENERIC_PATH | ADACOMP_FLAG_STREAMING)) return ADACOMP_ERR_FLAGS;
+    const bool streaming = (flags & ADACOMP_FLAG_STREAMING) != 0;       // (the flag chooses among kernels that give the same bytes)
+    flags &= ~ADACOMP_FLAG_STREAMING;
     if (factor != 0.f && !(factor > 0.f && factor <= 1e30f)) return ADACOMP_ERR_FLAGS;
     if (grad_type > ADACOMP_GRAD_F16 || quantiser > ADACOMP_QUANT_SENT_MEAN) return ADACOMP_ERR_FLAGS;
     if (misaligned(grad) || misaligned(residue) || misaligned(packed_out) ||
@@ -142,6 +144,17 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
     auto mark = [&](int i) { if (events) cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st); };
 
     mark(0);
+    // a layer whose tiles all fit in the shared memory of the CTAs that are resident together: one kernel, the
+    // residue visited once (pack_onchip.cu)
+    if (!lazy && !streaming && flags == 0 && fast_L_T(L_T) && grad_type == ADACOMP_GRAD_F32 && quantiser == 0 && geo.n_tiles != 0 &&
+        geo.n_tiles <= onchip_tile_capacity(*info) && debug_waits().withhold_pack == 0) {
+        PassArgs args{grad, residue, packed, scratch, geo, 0u, nullptr, factor, grad_type, quantiser, debug_waits().limit, 0u};
+        rc = launch_pack_onchip(args, reinterpret_cast<u64 *>(count_out), factor != 0.f ? kFlagFactor : 0u, *info, st);
+        mark(1);
+        mark(2);
+        mark(3);
+        return rc;
+    }
     if (geo.n_tiles) {
         PassArgs args{grad, residue, packed, scratch, geo, flags & ADACOMP_FLAG_LITERAL, lazy, factor, grad_type,
                       quantiser, debug_waits().limit, debug_waits().withhold_pack};
