@@ -28,9 +28,10 @@ int launch_decode_opt(const DecodeArgs &args, const Epilogue &ep_ref, const Devi
     const DeviceInfo *info = &info_ref;
 
         // (the optimizer entry points always pass the shape)
-        // (eight warps where they divide the tile's bins, unless four can work a lane per bin)
+        // (eight warps where they divide the tile's bins, unless four can work a lane per bin; Adam's two CTAs per
+        // SM need the eight all the same: 7.0 against 6.1 ms at 2^30 elements, L_T = 50)
         const Geometry og = make_geometry(hint_n, hint_L_T ? hint_L_T : 1u);
-        const bool eight = hint_L_T && og.tile_bins % 8u == 0 && !lanes_shape(og.tile_bins, 4u, og.w);
+        const bool eight = hint_L_T && og.tile_bins % 8u == 0 && (ep->adam || !lanes_shape(og.tile_bins, 4u, og.w));
         const int per = info->decode_opt_per_sm[ep->adam ? 1 : 0][eight ? 1 : 0];
         if (!per) return ADACOMP_ERR_CUDA;
         u64 grid_s = (u64)info->sms * per;
