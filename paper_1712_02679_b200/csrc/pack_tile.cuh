@@ -54,8 +54,10 @@ __host__ __device__ inline u64 lazy_state_bytes(const Geometry &g)
     return kLazyHeaderBytes + align_up(g.n_tiles * (u64)kMaskBytes, 16);
 }
 
-struct FastSmem {
-    static constexpr u32 kWordsAt = kStages * kStageBytes;            // 96000
+// Shared memory of the pipelined tile pass: NS stages of STAGE bytes, then the tile's words and the small tables.
+template <int NS, u32 STAGE>
+struct FastSmemT {
+    static constexpr u32 kWordsAt = NS * STAGE;                       // (3 stages of 32640: 97920)
     static constexpr u32 kInclAt = kWordsAt + 2 * kFastTile;          // + 8000 (16-bit words)
     static constexpr u32 kWtotAt = kInclAt + 4 * kTileSegs;
     static constexpr u32 kSegmaxAt = kWtotAt + 4 * 8;
@@ -63,27 +65,40 @@ struct FastSmem {
     static constexpr u32 kAccAt = kBinmaxAt + 4 * 4 * kSmallBins;     // (SPB = 0: two buffers each of bin maxima and counts) 8-byte aligned
     static constexpr u32 kAcc2At = kAccAt + 8 * (kWindows + 1);       // (second quantiser) exact sum of the sent |G|
     static constexpr u32 kBarAt = kAcc2At + 8 * (kWindows + 1);
-    static constexpr u32 kAbortAt = kBarAt + 8 * kStages;
+    static constexpr u32 kAbortAt = kBarAt + 8 * NS;
     static constexpr u32 kBytes = kAbortAt + 16;
 };
+typedef FastSmemT<kStages, kStageBytes> FastSmem;
 static_assert(FastSmem::kAccAt % 8 == 0, "accumulator must be 8-byte aligned");
+// The form with three CTAs per SM (16-bit gradients): two stages, the 8000-byte gradient tile packed against the residue.
+constexpr u32 kStageBytes16 = kTileBytes / 2 + kTileBytes + kMaskBytes;     // 24640
+typedef FastSmemT<2, kStageBytes16> FastSmem3;
+static_assert(FastSmem3::kAccAt % 8 == 0 && kStageBytes16 % 16 == 0 && 3 * (FastSmem3::kBytes + 1024) <= 227 * 1024, "three CTAs per SM");
 
 // GT: ADACOMP_GRAD_F32, or the gradient arrives in 16 bits per value (bfloat16 / binary16: tiles of half the
 // bytes, widened exactly as they are read).
-template <int SPB, typename Word, bool LAZY, int GT = 0>
-__global__ void __launch_bounds__(kFastThreads, 2)
+// CTAS: CTAs per SM the kernel is built for.  2: three stages of a whole gradient tile and a residue tile.  3 (16-bit
+// gradients only): two stages with the half-size gradient tile packed against the residue; the next tile's load
+// is then issued at the top of a tile instead of at its end, so that it has the whole tile to land.
+template <int SPB, typename Word, bool LAZY, int GT = 0, int CTAS = 2>
+__global__ void __launch_bounds__(kFastThreads, CTAS)
 tile_pass_fast(PassArgs a)
 {
+    static_assert(CTAS == 2 || (CTAS == 3 && GT != 0), "three CTAs per SM: 16-bit gradients");
+    constexpr int NS = CTAS == 3 ? 2 : kStages;
+    constexpr u32 STAGE = CTAS == 3 ? kStageBytes16 : kStageBytes;
+    constexpr u32 kResAt = CTAS == 3 ? kTileBytes / 2 : kTileBytes, kMaskAt = kResAt + kTileBytes;     // inside a stage
+    typedef FastSmemT<NS, STAGE> FS;
     extern __shared__ __align__(128) unsigned char smem[];
-    Word *s_words = reinterpret_cast<Word *>(smem + FastSmem::kWordsAt);
-    u32 *s_incl = reinterpret_cast<u32 *>(smem + FastSmem::kInclAt);
-    u32 *s_wtot = reinterpret_cast<u32 *>(smem + FastSmem::kWtotAt);
-    float *s_segmax = reinterpret_cast<float *>(smem + FastSmem::kSegmaxAt);
-    float *s_binmax = reinterpret_cast<float *>(smem + FastSmem::kBinmaxAt);
-    u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
-    u64 *s_acc2 = reinterpret_cast<u64 *>(smem + FastSmem::kAcc2At);
-    u64 *s_full = reinterpret_cast<u64 *>(smem + FastSmem::kBarAt);
-    volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FastSmem::kAbortAt);
+    Word *s_words = reinterpret_cast<Word *>(smem + FS::kWordsAt);
+    u32 *s_incl = reinterpret_cast<u32 *>(smem + FS::kInclAt);
+    u32 *s_wtot = reinterpret_cast<u32 *>(smem + FS::kWtotAt);
+    float *s_segmax = reinterpret_cast<float *>(smem + FS::kSegmaxAt);
+    float *s_binmax = reinterpret_cast<float *>(smem + FS::kBinmaxAt);
+    u64 *s_acc = reinterpret_cast<u64 *>(smem + FS::kAccAt);
+    u64 *s_acc2 = reinterpret_cast<u64 *>(smem + FS::kAcc2At);
+    u64 *s_full = reinterpret_cast<u64 *>(smem + FS::kBarAt);
+    volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FS::kAbortAt);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == 5;
@@ -141,7 +156,7 @@ tile_pass_fast(PassArgs a)
         for (int b = tid; b < 4 * kSmallBins; b += kFastThreads) s_anymax[b] = 0;
     if (tid == 0) {
         *s_abort = 0;
-        for (int s = 0; s < kStages; s++) mbar_init(&s_full[s], 1);
+        for (int s = 0; s < NS; s++) mbar_init(&s_full[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -150,8 +165,8 @@ tile_pass_fast(PassArgs a)
     auto issue_load = [&](u64 i) {
         const u64 tile = first + i * stride;
         if (i >= my_tiles || tile >= full_tiles) return;
-        unsigned char *st = smem + (i % kStages) * kStageBytes;
-        u64 *bar = &s_full[i % kStages];
+        unsigned char *st = smem + (i % NS) * STAGE;
+        u64 *bar = &s_full[i % NS];
         const u32 grad_bytes = G16 ? tile_bytes / 2 : tile_bytes;
         mbar_arrive_expect_tx(bar, grad_bytes + tile_bytes + (LAZY ? kMaskBytes : 0u));
         if (a.withhold != 0u && blockIdx.x == 0 && i == (u64)a.withhold) {
@@ -159,28 +174,32 @@ tile_pass_fast(PassArgs a)
             return;
         }
         bulk_load(st, reinterpret_cast<const unsigned char *>(a.grad) + tile * (u64)grad_bytes, grad_bytes, bar);
-        bulk_load(st + kTileBytes, a.residue + tile * (u64)T, tile_bytes, bar);
-        if (LAZY) bulk_load(st + 2 * kTileBytes, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
+        bulk_load(st + kResAt, a.residue + tile * (u64)T, tile_bytes, bar);
+        if (LAZY) bulk_load(st + kMaskAt, lazy_mask + tile * (u64)kTileSegs, kMaskBytes, bar);
         issued = i + 1;
     };
     if (service && lane == 0) {
         issue_load(0);
-        issue_load(1);
+        if (NS > 2) issue_load(1);
     }
 
     u64 i = 0;
     for (; i < my_tiles; i++) {
         const u64 tile = first + i * stride;
         const u64 base = tile * (u64)T;
-        float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
-        float *s_r = s_d + kFastTile;
+        float *s_d = reinterpret_cast<float *>(smem + (i % NS) * STAGE);
+        float *s_r = reinterpret_cast<float *>(smem + (i % NS) * STAGE + kResAt);
         const u32 *s_prev = reinterpret_cast<const u32 *>(s_r + kFastTile);
         const bool whole = tile < full_tiles;
         const int elems = whole ? T : (int)(geo.n - base);
         u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
+        if (NS == 2 && service && lane == 0) {
+            bulk_wait_read_all();        // the store of tile i - 1 has drained the other stage
+            issue_load(i + 1);
+        }
 
         if (whole) {
-            if (!mbar_wait(&s_full[i % kStages], (u32)(i / kStages) & 1u, a.wait_limit)) {
+            if (!mbar_wait(&s_full[i % NS], (u32)(i / NS) & 1u, a.wait_limit)) {
                 *s_abort = 1;                      // every thread that times out says so
                 raise_status(ADACOMP_DEV_TIMEOUT);
             }
@@ -346,7 +365,7 @@ tile_pass_fast(PassArgs a)
                 const bool valid = b < TB && tile * (u64)TB + b < geo.n_bins;
                 warp_accumulate(s_acc, valid ? (ANY ? __uint_as_float(any_max[b]) : s_binmax[b]) : 0.f, valid);
             }
-            if (lane == 0) {
+            if (NS > 2 && lane == 0) {
                 bulk_wait_read_all();    // the store of tile i - 1 has drained its stage
                 issue_load(i + 2);
             }
@@ -381,7 +400,7 @@ tile_pass_fast(PassArgs a)
                 // after a timeout: loads still in flight must land (or time out in turn) before
                 // this CTA's shared memory is given back, and the tiles it never finished count
                 // as empty so that the kernels after this one stay inside their buffers
-                for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % kStages], (u32)(j / kStages) & 1u, a.wait_limit);
+                for (u64 j = i + 1; j < issued; j++) mbar_wait(&s_full[j % NS], (u32)(j / NS) & 1u, a.wait_limit);
                 for (u64 j = i; j < my_tiles; j++) tile_cnt[first + j * stride] = 0;
             }
         }
