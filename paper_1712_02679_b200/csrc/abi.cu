@@ -347,17 +347,43 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
         return !mixed && quant_of(t) == ADACOMP_QUANT_BIN_MAX_MEAN && info->batch_per_sm > 0 && batchable(layers[t], *info) &&
                (!batch_lazy || info->batch_fast_ready);
     };
-    // (more layers than a table holds: batches of equal size, so that none is left with a layer or two)
+    // (a lone layer gains nothing from the batch kernels, and the single-layer path may pack it in one kernel)
     uint32_t to_batch = 0;
     for (uint32_t t = 0; t < n_layers; t++) to_batch += batched_at(t) ? 1u : 0u;
-    // (without the pipelined batch kernel the batch runs the any-L_T tile code, which takes every format too)
-    const uint32_t n_batches = (to_batch + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
-    const uint32_t per_batch = n_batches ? (to_batch + n_batches - 1) / n_batches : (uint32_t)kBatchMax;
-    // (a lone layer gains nothing from the batch kernels, and the single-layer path may pack it in one kernel)
     const bool lone = to_batch == 1;
     for (uint32_t t = 0; t < n_layers; t++) {
         const adacomp_layer_desc &d = layers[t];
-        if (batched_at(t) && !lone) {
+        if (batched_at(t) && !lone) continue;
+        rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags, nullptr,
+                           state_of(t), factor_of(t), type_of(t), nullptr, quant_of(t));
+        if (rc != ADACOMP_OK) return rc;
+    }
+    if (lone || to_batch == 0) return ADACOMP_OK;
+    // A batch whose layers all have the bin length 50, or all 500, runs a tile pass with the tile's shape compiled
+    // in (pack_batch.cu).  The layers of such a bin length get batches of their own when they are worth the extra
+    // launches (a few thousand tiles: the shorter tile code saves about a microsecond per tile and CTA, a batch
+    // costs four launches); layers are independent, so the order in which they are packed is free.
+    constexpr u64 kOwnBatchTiles = 3000;     // (of the bin length 50: the form for 500 measured no faster than the mixed one)
+    u64 tiles_of[2] = {0, 0};           // [L_T 500, L_T 50]
+    uint32_t others = 0;
+    for (uint32_t t = 0; t < n_layers; t++) {
+        if (!batched_at(t)) continue;
+        const u32 lt = layers[t].L_T;
+        if (lt == 500u || lt == 50u) tiles_of[lt == 50u] += make_geometry(layers[t].n, lt).n_tiles;
+        else others++;
+    }
+    const bool own[2] = {false, tiles_of[1] >= kOwnBatchTiles && (tiles_of[0] != 0 || others != 0)};
+    auto class_of = [&](uint32_t t) { return layers[t].L_T == 500u && own[0] ? 0 : layers[t].L_T == 50u && own[1] ? 1 : 2; };
+    for (int cls = 0; cls < 3; cls++) {
+        // (more layers than a table holds: batches of equal size, so that none is left with a layer or two)
+        uint32_t members = 0;
+        for (uint32_t t = 0; t < n_layers; t++) members += batched_at(t) && class_of(t) == cls ? 1u : 0u;
+        if (!members) continue;
+        const uint32_t n_batches = (members + (uint32_t)kBatchMax - 1) / (uint32_t)kBatchMax;
+        const uint32_t per_batch = (members + n_batches - 1) / n_batches;
+        for (uint32_t t = 0; t < n_layers; t++) {
+            if (!batched_at(t) || class_of(t) != cls) continue;
+            const adacomp_layer_desc &d = layers[t];
             BatchLayer &L = batch.layer[batch.n_layers++];
             L.grad = d.grad;
             L.residue = d.residue;
@@ -367,7 +393,7 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
             L.tile_first = batch.total_tiles;
             L.grad_type = type_of(t);
             L.factor = factor_of(t);
-            L.pad = 0;
+            L.inv_L_T = (u32)(((1ull << 32) + d.L_T - 1) / d.L_T);
             L.lazy = static_cast<unsigned char *>(state_of(t));
             batch.total_tiles += (u32)L.geo.n_tiles;
             if (batch.n_layers == per_batch) {
@@ -376,13 +402,13 @@ static int compress_multi_impl(const adacomp_layer_desc *layers, void *const *st
                 batch.n_layers = 0;
                 batch.total_tiles = 0;
             }
-        } else {
-            rc = compress_impl(d.grad, d.residue, d.n, d.L_T, d.packed_out, d.count_out, stream, d.flags, nullptr,
-                               state_of(t), factor_of(t), type_of(t), nullptr, quant_of(t));
-            if (rc != ADACOMP_OK) return rc;
         }
+        rc = launch_batch(batch, *info, st, batch_lazy);
+        if (rc != ADACOMP_OK) return rc;
+        batch.n_layers = 0;
+        batch.total_tiles = 0;
     }
-    return launch_batch(batch, *info, st, batch_lazy);
+    return ADACOMP_OK;
 }
 
 int adacomp_compress_multi_opt(const adacomp_layer_desc *layers, const adacomp_options *opts, uint32_t n_layers, void *stream)

@@ -67,10 +67,15 @@ batch_tile_pass(const __grid_constant__ BatchArgsT<N> b)
 // own is flagged, left untouched and reports empty tiles.
 // OPTS: some layer has a 16-bit gradient or a factor (else both are compile-time constants: plain lists keep
 // the shorter code).
-template <int N, bool LAZY, bool OPTS>
+// USPB: not 0 when every layer of the batch has the bin length 25 * USPB (tiles of exactly 4000 elements, a bin
+// USPB whole segments): the tile's shape, a thread's place among the bins and the word width are then
+// compile-time constants, as in the single-layer kernel, and the tile code is two thirds as long.
+template <int N, bool LAZY, bool OPTS, int USPB = 0>
 __global__ void __launch_bounds__(kFastThreads, 2)
 batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
 {
+    constexpr bool UNI = USPB != 0;
+    constexpr int USPB1 = UNI ? USPB : 1;           // (a divisor that is never 0)
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *s_words = smem + FastSmem::kWordsAt;
     u32 *s_incl = reinterpret_cast<u32 *>(smem + FastSmem::kInclAt);
@@ -81,14 +86,18 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
     u64 *s_acc = reinterpret_cast<u64 *>(smem + FastSmem::kAccAt);
     u64 *s_full = reinterpret_cast<u64 *>(smem + FastSmem::kBarAt);
     volatile u32 *s_abort = reinterpret_cast<volatile u32 *>(smem + FastSmem::kAbortAt);
+    // the layers' first tiles, copied out of the kernel parameters: a CTA's next tile is often several layers on, and a
+    // walk through the parameter table is a chain of dependent constant-cache misses that every warp waits for
+    u32 *s_tile_first = reinterpret_cast<u32 *>(smem + FastSmem::kBytes);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == 5;
     const u32 first = blockIdx.x, stride = gridDim.x;
     const u32 my_tiles = b.total_tiles > first ? (b.total_tiles - first + stride - 1) / stride : 0;
     const int n_layers = (int)b.n_layers;
+    for (int l = tid; l < n_layers; l += kFastThreads) s_tile_first[l] = b.layer[l].tile_first;
     auto seek = [&](u32 gt, int &li) {      // (tiles only go up)
-        while (li + 1 < n_layers && b.layer[li + 1].tile_first <= gt) li++;
+        while (li + 1 < n_layers && s_tile_first[li + 1] <= gt) li++;
     };
     auto state_ok = [&](const BatchLayer &L) {      // (LAZY) the state is this layer's
         const LazyHeader *lh = reinterpret_cast<const LazyHeader *>(L.lazy);
@@ -118,7 +127,8 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
         }
         if (LAZY && !load_ok) return;                   // nothing of such a layer is read
         const u32 lt = gt - L.tile_first, T = L.geo.tile_elems;
-        if ((u64)lt >= L.geo.n / T) return;             // a ragged last tile is read with plain loads
+        // a ragged last tile is read with plain loads (no division: the layer's tiles cover n exactly or all but the last are whole)
+        if ((u64)lt + 1 >= L.geo.n_tiles && L.geo.n != L.geo.n_tiles * (u64)T) return;
         const bool g16 = OPTS && L.grad_type != ADACOMP_GRAD_F32;
         if (g16 && T % 8u != 0) return;                 // 16-bit tiles off the 16-byte boundaries: plain loads as well
         const u32 gbytes = g16 ? 2u * T : 4u * T;
@@ -165,12 +175,12 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             at_li = li;
             T = (int)geo.tile_elems;
             TB = (int)geo.tile_bins;
-            full_tiles = (u32)(geo.n / (u64)T);
+            full_tiles = (u32)geo.n_tiles - (geo.n != geo.n_tiles * (u64)T ? 1u : 0u);      // (no division)
             wbytes = geo.w;
             // the thread's elements [0, cut) lie in bin b0 of the tile, from place off0 of it on, the others
             // in bin b0 + 1; only the first `vcount` of them exist (tiles of less than 4000 elements)
             const int Lt = (int)geo.L_T, e0 = tid * kSeg;
-            b0 = e0 / Lt;
+            b0 = (int)__umulhi((u32)e0, L.inv_L_T);         // e0 / L_T (the host's ceil(2^32 / L_T): exact for e0 < 4000, L_T <= 1000)
             off0 = e0 - b0 * Lt;
             cut = min(kSeg, Lt - off0);
             vcount = max(0, min(kSeg, T - e0));
@@ -194,6 +204,11 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 }
             }
         }
+        // (UNI: what the layer-change block worked out is known at compile time)
+        const int kT = UNI ? kFastTile : T, kTB = UNI ? kTileSegs / USPB1 : TB, kSPB = UNI ? USPB : SPB;
+        const bool kAl = UNI || aligned;
+        const u32 kWb = UNI ? (USPB == 2 ? 1u : 2u) : wbytes;
+        const int kB0 = UNI ? tid / USPB1 : b0, kCut = UNI ? kSeg : cut, kOff0 = UNI ? (tid % USPB1) * kSeg : off0;
         unsigned char *scratch = L.packed + geo.scratch_at;
         const u32 lt = gt - L.tile_first;
         if (LAZY && !layer_ok) {
@@ -211,11 +226,11 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             __syncthreads();
             continue;
         }
-        const u64 base = (u64)lt * (u64)T;
+        const u64 base = (u64)lt * (u64)kT;
         float *s_d = reinterpret_cast<float *>(smem + (i % kStages) * kStageBytes);
         float *s_r = s_d + kFastTile;
         const bool whole = lt < full_tiles;
-        const int elems = whole ? T : (int)min((u64)T, geo.n - base);      // (plain loads: the ragged last tile, or 16-bit tiles off the 16-byte boundaries)
+        const int elems = whole ? kT : (int)min((u64)kT, geo.n - base);      // (plain loads: the ragged last tile, or 16-bit tiles off the 16-byte boundaries)
         u32 *const any_max = s_anymax + (i & 1) * kSmallBins, *const any_cnt = s_anycnt + (i & 1) * kSmallBins;
 
         if (whole) {
@@ -226,18 +241,29 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             }
             phase ^= 1u << stage;
         } else {
-            // the ragged last tile of a layer: plain loads, zero fill past the end
-            for (int e = tid; e < kFastTile; e += kFastThreads) {
-                float d = 0.f, r = 0.f;
-                unsigned short d16 = 0;
+            // the ragged last tile of a layer: plain loads, zero fill past the end (all of a thread's loads are
+            // started before the first value is used: one trip to memory, not twenty-one)
+            constexpr int kPer = (kFastTile + kFastThreads - 1) / kFastThreads;
+            float dv[kPer], rv[kPer];
+            const bool g16 = OPTS && gtype != ADACOMP_GRAD_F32;
+#pragma unroll
+            for (int q = 0; q < kPer; q++) {
+                const int e = tid + q * kFastThreads;
+                dv[q] = rv[q] = 0.f;
                 if (e < elems) {
-                    if (OPTS && gtype != ADACOMP_GRAD_F32) d16 = reinterpret_cast<const unsigned short *>(L.grad)[base + e];
-                    else d = L.grad[base + e];
-                    r = L.residue[base + e];
+                    if (g16) dv[q] = __uint_as_float((u32) reinterpret_cast<const unsigned short *>(L.grad)[base + e]);    // (the 16 bits, as they are)
+                    else dv[q] = L.grad[base + e];
+                    rv[q] = L.residue[base + e];
                 }
-                if (OPTS && gtype != ADACOMP_GRAD_F32) reinterpret_cast<unsigned short *>(s_d)[e] = d16;
-                else s_d[e] = d;
-                s_r[e] = r;
+            }
+#pragma unroll
+            for (int q = 0; q < kPer; q++) {
+                const int e = tid + q * kFastThreads;
+                if (e < kFastTile) {
+                    if (g16) reinterpret_cast<unsigned short *>(s_d)[e] = (unsigned short)__float_as_uint(dv[q]);
+                    else s_d[e] = dv[q];
+                    s_r[e] = rv[q];
+                }
             }
             if (LAZY && tid < kTileSegs) reinterpret_cast<u32 *>(s_r + kFastTile)[tid] = lazy_mask[(u64)lt * kTileSegs + tid];
             __syncthreads();
@@ -253,11 +279,11 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
             float m = 0.f, m1 = 0.f;
             const u32 prev = LAZY ? reinterpret_cast<const u32 *>(s_r + kFastTile)[tid] : 0u;
             // (the loop twice: where the segments line up with the bins, as in the lists' bin lengths 50 and
-            // 500, the tests on `vcount` and `cut` fold away)
+            // 500, the tests on `vcount` and `kCut` fold away)
             auto form = [&](auto lined_up, auto sixteen) {
                 constexpr bool AL = decltype(lined_up)::value, G16 = decltype(sixteen)::value;
-                const int vc = AL ? kSeg : vcount, ct = AL ? kSeg : cut;
-                // 16-bit values: thirteen aligned 32-bit loads cover the segment's 50 bytes, a funnel shift lines the pairs up
+                const int vc = AL ? kSeg : vcount, ct = AL ? kSeg : kCut;
+                // 16-bit values: thirteen kAl 32-bit loads cover the segment's 50 bytes, a funnel shift lines the pairs up
                 u32 pair[G16 ? 13 : 1];
                 if (G16) {
                     const u32 *pw = reinterpret_cast<const u32 *>(s_d) + ((tid * kSeg) >> 1);
@@ -293,49 +319,49 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 }
             };
             if (!OPTS || gtype == ADACOMP_GRAD_F32) {
-                if (aligned) form(TrueType{}, FalseType{});
+                if (kAl) form(TrueType{}, FalseType{});
                 else form(FalseType{}, FalseType{});
             } else {
-                if (aligned) form(TrueType{}, TrueType{});
+                if (kAl) form(TrueType{}, TrueType{});
                 else form(FalseType{}, TrueType{});
             }
-            if (aligned) {
-                // a bin is SPB whole segments: no atomics, the maximum goes through a shuffle (two segments)
+            if (kAl) {
+                // a bin is kSPB whole segments: no atomics, the maximum goes through a shuffle (two segments)
                 // or through the segments' maxima in shared memory
-                if (SPB == 2) gm = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+                if (kSPB == 2) gm = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
                 else s_segmax[tid] = m;
             } else {
                 // (non-negative floats order like their bits)
-                if (m > 0.f && b0 < TB) atomicMax(&any_max[b0], __float_as_uint(m));
-                if (m1 > 0.f && b0 + 1 < TB) atomicMax(&any_max[b0 + 1], __float_as_uint(m1));
+                if (m > 0.f && kB0 < kTB) atomicMax(&any_max[kB0], __float_as_uint(m));
+                if (m1 > 0.f && kB0 + 1 < kTB) atomicMax(&any_max[kB0 + 1], __float_as_uint(m1));
             }
         }
-        if (!(aligned && SPB == 2)) __syncthreads();                // barrier A (uniform: the layer's shape)
+        if (!(kAl && kSPB == 2)) __syncthreads();                // barrier A (uniform: the layer's shape)
         if (!service) {
-            if (!aligned) {
-                gm = b0 < TB ? __uint_as_float(any_max[b0]) : 0.f;
-                gm1 = b0 + 1 < TB ? __uint_as_float(any_max[b0 + 1]) : 0.f;
-            } else if (SPB != 2) {
-                const int s0 = b0 * SPB;
-                for (int sgm = 0; sgm < SPB; sgm++) gm = fmaxf(gm, s_segmax[s0 + sgm]);
+            if (!kAl) {
+                gm = kB0 < kTB ? __uint_as_float(any_max[kB0]) : 0.f;
+                gm1 = kB0 + 1 < kTB ? __uint_as_float(any_max[kB0 + 1]) : 0.f;
+            } else if (kSPB != 2) {
+                const int s0 = kB0 * kSPB;
+                for (int sgm = 0; sgm < kSPB; sgm++) gm = fmaxf(gm, s_segmax[s0 + sgm]);
             }
             // ---- selection (a zero bin has G == 0 everywhere and sends nothing) ----
-            if (aligned) {
+            if (kAl) {
 #pragma unroll
                 for (int j = 0; j < kSeg; j++)
                     if (key[j] >= gm && g[j] != 0.f) selmask |= 1u << j;
             } else {
 #pragma unroll
                 for (int j = 0; j < kSeg; j++)
-                    if (key[j] >= (j >= cut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
+                    if (key[j] >= (j >= kCut ? gm1 : gm) && g[j] != 0.f) selmask |= 1u << j;
             }
             cnt = __popc(selmask);
-            if (!aligned) {
-                const u32 c0 = __popc(selmask & ((1u << cut) - 1u));
-                if (c0) atomicAdd(&any_cnt[b0], c0);
-                if (cnt - c0) atomicAdd(&any_cnt[b0 + 1], cnt - c0);
-            } else if (tid == b0 * SPB) {
-                any_max[b0] = __float_as_uint(gm);                  // for the exact sum (the service warp reads it after barrier B)
+            if (!kAl) {
+                const u32 c0 = __popc(selmask & ((1u << kCut) - 1u));
+                if (c0) atomicAdd(&any_cnt[kB0], c0);
+                if (cnt - c0) atomicAdd(&any_cnt[kB0 + 1], cnt - c0);
+            } else if (tid == kB0 * kSPB) {
+                any_max[kB0] = __float_as_uint(gm);                  // for the exact sum (the service warp reads it after barrier B)
             }
             incl = warp_inclusive_scan(cnt, lane);
             s_incl[tid] = incl;
@@ -365,39 +391,39 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
                 const int j = __ffs(mask) - 1;
                 mask &= mask - 1;
                 const u32 neg = __float_as_uint(pr[j]) >> 31;
-                const u32 idx = j >= cut ? (u32)(j - cut) : (u32)(off0 + j);        // the element's place in its bin
+                const u32 idx = j >= kCut ? (u32)(j - kCut) : (u32)(kOff0 + j);        // the element's place in its bin
                 const u32 word = (idx << 2) | 1u | (neg << 1);
-                if (wbytes == 1u) s_words[at] = (unsigned char)word;
+                if (kWb == 1u) s_words[at] = (unsigned char)word;
                 else reinterpret_cast<unsigned short *>(s_words)[at] = (unsigned short)word;
                 at++;
             }
             if (LAZY) lazy_mask[(u64)lt * kTileSegs + tid] = selmask;
-            if (aligned) {
+            if (kAl) {
                 // the bin's first thread: the words between its own first one and the last one of the bin's last segment
-                if (tid == b0 * SPB) {
-                    const u64 bin = (u64)lt * (u64)TB + (u32)b0;
-                    const int t1 = tid + SPB - 1;
+                if (tid == kB0 * kSPB) {
+                    const u64 bin = (u64)lt * (u64)kTB + (u32)kB0;
+                    const int t1 = tid + kSPB - 1;
                     const u32 last = wpre_all[t1 >> 5] + s_incl[t1], count = last - (wpre + incl) + cnt;
                     if (bin < geo.n_bins) {
                         unsigned char *bc = L.packed + geo.bin_cnt_at;
-                        if (wbytes == 1u) bc[bin] = (unsigned char)count;
+                        if (kWb == 1u) bc[bin] = (unsigned char)count;
                         else reinterpret_cast<unsigned short *>(bc)[bin] = (unsigned short)count;
                     }
                 }
-            } else if (tid < TB) {
-                const u64 bin = (u64)lt * (u64)TB + tid;
+            } else if (tid < kTB) {
+                const u64 bin = (u64)lt * (u64)kTB + tid;
                 if (bin < geo.n_bins) {
                     unsigned char *bc = L.packed + geo.bin_cnt_at;
-                    if (wbytes == 1u) bc[bin] = (unsigned char)any_cnt[tid];
+                    if (kWb == 1u) bc[bin] = (unsigned char)any_cnt[tid];
                     else reinterpret_cast<unsigned short *>(bc)[bin] = (unsigned short)any_cnt[tid];
                 }
             }
             fence_async_smem();          // the bulk store below reads what was just written
         } else {
             total = s_wtot[0] + s_wtot[1] + s_wtot[2] + s_wtot[3] + s_wtot[4];
-            for (int bb = 0; bb < TB; bb += 32) {       // every lane takes part each round
+            for (int bb = 0; bb < kTB; bb += 32) {       // every lane takes part each round
                 const int bq = bb + lane;
-                const bool valid = bq < TB && (u64)lt * (u64)TB + bq < geo.n_bins;
+                const bool valid = bq < kTB && (u64)lt * (u64)kTB + bq < geo.n_bins;
                 warp_accumulate(s_acc, valid ? __uint_as_float(any_max[bq]) : 0.f, valid);
             }
             if (lane == 0) {
@@ -411,14 +437,14 @@ batch_tile_pass_fast(const __grid_constant__ BatchArgsT<N> b)
         if (service && !aborted) {
             if (whole) {
                 if (lane == 0) {
-                    bulk_store(L.residue + base, s_r, 4u * (u32)T);
+                    bulk_store(L.residue + base, s_r, 4u * (u32)kT);
                     bulk_commit();
                 }
             } else {
                 for (int e = lane; e < elems; e += 32) L.residue[base + e] = s_r[e];
             }
             uint4 *slot = reinterpret_cast<uint4 *>(scratch + geo.slots_at + (u64)lt * geo.slot_bytes);
-            const int chunks = (int)((total * wbytes + 15) / 16);
+            const int chunks = (int)((total * kWb + 15) / 16);
             for (int c = lane; c < chunks; c += 32) slot[c] = reinterpret_cast<uint4 *>(s_words)[c];
             if (lane == 0) {
                 reinterpret_cast<u32 *>(scratch + geo.tile_cnt_at)[lt] = total;
@@ -482,7 +508,7 @@ batch_gather(const __grid_constant__ BatchArgsT<N> b)
 void init_pack_batch_info(DeviceInfo &d)
 {
     const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    const int bytes = (int)FastSmem::kBytes;
+    const int bytes = (int)FastSmem::kBytes + 4 * kBatchMax;
     if (cudaFuncSetAttribute(batch_tile_pass<kBatchMax>, at, (int)kBatchSmemBytes) == cudaSuccess &&
         cudaFuncSetAttribute(batch_tile_pass<kBatchSmall>, at, (int)kBatchSmemBytes) == cudaSuccess) {
         int per = 0;
@@ -497,7 +523,15 @@ void init_pack_batch_info(DeviceInfo &d)
                          cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false, true>, at, bytes) == cudaSuccess &&
                          cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false, true>, at, bytes) == cudaSuccess &&
                          cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true, true>, at, bytes) == cudaSuccess &&
-                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, true>, at, bytes) == cudaSuccess;
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, true>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false, false, 2>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false, false, 2>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true, false, 2>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, false, 2>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, false, false, 20>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, false, false, 20>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchMax, true, false, 20>, at, bytes) == cudaSuccess &&
+                         cudaFuncSetAttribute(batch_tile_pass_fast<kBatchSmall, true, false, 20>, at, bytes) == cudaSuccess;
 }
 
 // lazy: lazy-scale mode (every layer carries its state; needs the pipelined batch tile pass).
@@ -511,10 +545,17 @@ int launch_batch_sized(const BatchArgsT<N> &b, const DeviceInfo &info, cudaStrea
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);
             bool opts = false;
             for (u32 i = 0; i < b.n_layers; i++) opts = opts || b.layer[i].grad_type != ADACOMP_GRAD_F32 || b.layer[i].factor != 0.f;
-            if (lazy && opts) batch_tile_pass_fast<N, true, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
-            else if (lazy) batch_tile_pass_fast<N, true, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
-            else if (opts) batch_tile_pass_fast<N, false, true><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
-            else batch_tile_pass_fast<N, false, false><<<grid, kFastThreads, FastSmem::kBytes, st>>>(b);
+            // (one bin length, 50 or 500, throughout the batch: the form with the tile's shape compiled in)
+            u32 lt_all = b.layer[0].geo.L_T;
+            for (u32 i = 1; i < b.n_layers; i++) lt_all = b.layer[i].geo.L_T == lt_all ? lt_all : 0u;
+            if (lazy && opts) batch_tile_pass_fast<N, true, true><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (opts) batch_tile_pass_fast<N, false, true><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (lazy && lt_all == 50u) batch_tile_pass_fast<N, true, false, 2><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (lazy && lt_all == 500u) batch_tile_pass_fast<N, true, false, 20><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (lazy) batch_tile_pass_fast<N, true, false><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (lt_all == 50u) batch_tile_pass_fast<N, false, false, 2><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else if (lt_all == 500u) batch_tile_pass_fast<N, false, false, 20><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
+            else batch_tile_pass_fast<N, false, false><<<grid, kFastThreads, FastSmem::kBytes + 4 * N, st>>>(b);
         } else {
             const u64 cap = (u64)info.sms * info.batch_per_sm;
             const unsigned grid = (unsigned)(b.total_tiles < cap ? b.total_tiles : cap);

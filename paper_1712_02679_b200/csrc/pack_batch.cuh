@@ -30,7 +30,7 @@ struct BatchLayer {
     u32 grad_type;                                   // ADACOMP_GRAD_*: what `grad` points to
     unsigned char *lazy;                             // lazy-scale mode: the layer's state (else null)
     float factor;                                    // 0: H = G + dW (Algorithm 2); else H = residue + factor * dW
-    u32 pad;
+    u32 inv_L_T;                                     // ceil(2^32 / L_T): a thread's first bin without a division
 };
 
 // The table comes in two sizes: kernel parameters are copied at every launch, and a launch with the
