@@ -93,6 +93,16 @@ def test_lstm_parameter_list_eight_learners():
     _multi_tensor_case(6, specs, learners=8)
 
 
+def test_mixed_list_whose_layers_of_bin_length_50_get_batches_of_their_own():
+    # 3000 tiles and more of bin length 50 beside other bin lengths: the 50s are packed by the batch form with
+    # the tile's shape compiled in, the others by the any-bin form; the order of the layers in the list stays free
+    T = synth.TensorSpec
+    specs = [T("fc_a", 4000 * 1100 + 37, 50, "fc"), T("conv_a", 4000 * 40 + 499, 500, "conv"), T("fc_b", 4000 * 1000, 50, "fc"),
+             T("bn", 256, 500, "bn"), T("other", 4000 * 30 + 50, 100, "conv"), T("fc_c", 4000 * 950 + 1, 50, "fc"),
+             T("fc_bias", 1000, 50, "fc"), T("conv_b", 4000 * 25, 500, "conv")]
+    _multi_tensor_case(7, specs, learners=2, heavy_sigma=1e-3)
+
+
 @pytest.mark.parametrize("L_T", [50, 500])
 @pytest.mark.parametrize("log2n", [20, 22, 24])
 def test_config5_sweep_point_prewarmed_eager_and_lazy(L_T, log2n):
