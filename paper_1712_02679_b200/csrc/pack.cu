@@ -177,14 +177,25 @@ int compress_impl(const float *grad, float *residue, uint64_t n, uint32_t L_T, v
         }
     }
     mark(1);
-    finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, flags | (factor != 0.f ? kFlagFactor : 0u) | (quantiser ? kFlagQuant : 0u),
-                                 reinterpret_cast<u64 *>(count_out), lazy);
+    const u32 header_flags = flags | (factor != 0.f ? kFlagFactor : 0u) | (quantiser ? kFlagQuant : 0u);
+    // (layers of at most kFoldGroups groups of tiles: the gather does finalize's work itself, a launch fewer)
+    const bool fold = geo.n_tiles != 0 && geo.tile_bins <= (u32)kSmallBins && geo.n_groups <= (u64)kFoldGroups;
+    if (!fold) finalize<<<1, 1024, 0, st>>>(packed, scratch, geo, header_flags, reinterpret_cast<u64 *>(count_out), lazy);
     mark(2);
     if (geo.n_tiles) {
         if (geo.tile_bins <= (u32)kSmallBins) {
             const u64 want = (geo.n_tiles + 3) / 4, cap = (u64)info->sms * 16;
             const unsigned grid = (unsigned)(want < cap ? want : cap);
-            if (lazy) {     // the residue keeps G; only the words move
+            u64 *const co = reinterpret_cast<u64 *>(count_out);
+            if (fold) {
+                if (lazy) {     // the residue keeps G; only the words move
+                    if (geo.w == 1u) gather_fixup_fold<unsigned char, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo, header_flags, co, lazy);
+                    else gather_fixup_fold<unsigned short, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo, header_flags, co, lazy);
+                } else {
+                    if (geo.w == 1u) gather_fixup_fold<unsigned char, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo, header_flags, co, lazy);
+                    else gather_fixup_fold<unsigned short, true><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo, header_flags, co, lazy);
+                }
+            } else if (lazy) {
                 if (geo.w == 1u) gather_fixup_small<unsigned char, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
                 else gather_fixup_small<unsigned short, false><<<grid, kGatherThreads, 0, st>>>(residue, packed, scratch, geo);
             } else {

@@ -739,15 +739,22 @@ __device__ inline double windows_to_double(const u64 *win)
     return scalbn((double)mant, low - 149);
 }
 
-__device__ inline void finalize_body(unsigned char *packed, unsigned char *scratch, const Geometry &geo, u32 flags,
-                              u64 *count_out, unsigned char *lazy_state)
+// The whole CTA (any number of whole warps).  `prefix`: where the groups' running sums go: null for "in place, over the
+// counts" (the finalize kernel), else an array of n_groups entries that the counts are scanned into (a gather
+// kernel that does this work itself, every CTA into its own shared memory).  `head`: this CTA writes the header,
+// count_out, the gaps and the lazy-scale state (exactly one CTA of a launch does).  Returns the scale (in thread 0).
+__device__ inline float finalize_body(unsigned char *packed, unsigned char *scratch, const Geometry &geo, u32 flags,
+                                      u64 *count_out, unsigned char *lazy_state, u64 *prefix = nullptr, bool head = true)
 {
     __shared__ u64 s_warp[33];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    u64 *group = reinterpret_cast<u64 *>(scratch + geo.group_at);
+    const u64 *group = reinterpret_cast<const u64 *>(scratch + geo.group_at);
+    u64 *const sums = prefix ? prefix : reinterpret_cast<u64 *>(scratch + geo.group_at);
+    if (tid < 33) s_warp[tid] = 0;
+    __syncthreads();
 
-    // in-place exclusive scan of the per-group word counts
-    const u64 per = (geo.n_groups + 1023) / 1024;
+    // exclusive scan of the per-group word counts
+    const u64 per = (geo.n_groups + blockDim.x - 1) / blockDim.x;
     const u64 lo = min((u64)tid * per, geo.n_groups), hi = min(lo + per, geo.n_groups);
     u64 sum = 0;
     for (u64 i = lo; i < hi; i++) sum += group[i];
@@ -772,16 +779,14 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
     u64 run = s_warp[warp] + inc - sum;
     for (u64 i = lo; i < hi; i++) {
         const u64 c = group[i];
-        group[i] = run;
+        sums[i] = run;
         run += c;
     }
     const u64 n_sel = s_warp[32];
 
+    float scale = 0.f;
     if (tid == 0) {
-        u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
-        tile_off[geo.n_tiles] = n_sel;
         const u64 *win = reinterpret_cast<const u64 *>(scratch);
-        float scale = 0.f;
         if (flags & kFlagQuant) {
             // the second quantiser: the mean |G| of the sent elements
             if (n_sel) scale = __double2float_rn(__ddiv_rn(windows_to_double(win + kCtlSentSumAt / 8), (double)n_sel));
@@ -789,6 +794,11 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
             const double S = windows_to_double(win);
             scale = __double2float_rn(__ddiv_rn(S, (double)geo.n_bins));
         }
+    }
+    if (!head) return scale;
+    if (tid == 0) {
+        u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
+        tile_off[geo.n_tiles] = n_sel;
         const u64 bytes_used = geo.payload_at + align_up(n_sel * geo.w, 16);
         u32 *h32 = reinterpret_cast<u32 *>(packed);
         u64 *h64 = reinterpret_cast<u64 *>(packed);
@@ -821,6 +831,7 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
     if ((u64)tid < geo.bin_cnt_at - dir_end) packed[dir_end + tid] = 0;
     const u64 cnt_end = geo.bin_cnt_at + geo.n_bins * geo.w;
     if ((u64)tid < geo.payload_at - cnt_end) packed[cnt_end + tid] = 0;
+    return scale;
 }
 
 // ---------------------------------------------------------------------------------
@@ -832,10 +843,10 @@ __device__ inline void finalize_body(unsigned char *packed, unsigned char *scrat
 // Words before `tile`: its group's scanned offset plus the counts of the tiles before it
 // in the group.  Warp-collective; also returns the tile's own count.
 __device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &geo, u64 tile, int lane,
-                                  u32 &count)
+                                  u32 &count, const u64 *group_sums = nullptr)
 {
     const u32 *tile_cnt = reinterpret_cast<const u32 *>(scratch + geo.tile_cnt_at);
-    const u64 *group = reinterpret_cast<const u64 *>(scratch + geo.group_at);
+    const u64 *group = group_sums ? group_sums : reinterpret_cast<const u64 *>(scratch + geo.group_at);
     const u64 g = tile / kGroupTiles;
     const int me = (int)(tile % kGroupTiles);
     const u64 t = g * kGroupTiles + lane;
@@ -847,17 +858,20 @@ __device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &
 }
 
 // One tile of at most 96 bins, handled by one warp.
+// group_sums / scale_bits: null / unused where a finalize kernel ran before (the groups' running sums are in the
+// scratch, the scale in the header); else the CTA's own copies.
 template <typename Word, bool FIXUP>
 __device__ void gather_tile_small(float *residue, unsigned char *packed, const unsigned char *scratch,
-                                  const Geometry &geo, u64 tile, int lane, u32 *s_pre)
+                                  const Geometry &geo, u64 tile, int lane, u32 *s_pre, const u64 *group_sums = nullptr,
+                                  u32 scale_bits = 0u)
 {
     const int TB = (int)geo.tile_bins;
     u64 *tile_off = reinterpret_cast<u64 *>(packed + geo.tile_off_at);
     const Word *bin_cnt = reinterpret_cast<const Word *>(packed + geo.bin_cnt_at);
     Word *payload = reinterpret_cast<Word *>(packed + geo.payload_at);
-    const float scale = __uint_as_float(reinterpret_cast<const u32 *>(packed)[12]);
+    const float scale = __uint_as_float(group_sums ? scale_bits : reinterpret_cast<const u32 *>(packed)[12]);
     u32 cnt;
-    const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt);
+    const u64 off0 = tile_offset(scratch, geo, tile, lane, cnt, group_sums);
     if (lane == 0) tile_off[tile] = off0;
     if (cnt == 0) return;
     // exclusive scan of the tile's bin counts, three bins per lane (only the fix-up needs bins)
@@ -928,6 +942,27 @@ gather_fixup_small(float *residue, unsigned char *packed, const unsigned char *s
     // L2 still holds when this kernel starts.
     for (u64 item = (u64)blockIdx.x * (kGatherThreads / 32) + warp; item < geo.n_tiles; item += warps)
         gather_tile_small<Word, FIXUP>(residue, packed, scratch, geo, geo.n_tiles - 1 - item, lane, s_pre_all[warp]);
+}
+
+// The same with finalize's work done here, for layers of at most kFoldGroups groups of 32 tiles (2^27 elements): every
+// CTA scans the groups' counts into its shared memory and works the scale out (8 KB read from L2 and a microsecond,
+// all CTAs at once) instead of waiting for a kernel of one CTA to do it; the first CTA also writes the header.
+constexpr u32 kFoldGroups = 1024;
+template <typename Word, bool FIXUP>
+__global__ void __launch_bounds__(kGatherThreads)
+gather_fixup_fold(float *residue, unsigned char *packed, unsigned char *scratch, Geometry geo, u32 flags, u64 *count_out,
+                  unsigned char *lazy_state)
+{
+    __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
+    __shared__ u64 s_sums[kFoldGroups];
+    __shared__ u32 s_scale_bits;
+    const float scale = finalize_body(packed, scratch, geo, flags, count_out, lazy_state, s_sums, blockIdx.x == 0);
+    if (threadIdx.x == 0) s_scale_bits = __float_as_uint(scale);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const u64 warps = (u64)gridDim.x * (kGatherThreads / 32);
+    for (u64 item = (u64)blockIdx.x * (kGatherThreads / 32) + warp; item < geo.n_tiles; item += warps)
+        gather_tile_small<Word, FIXUP>(residue, packed, scratch, geo, geo.n_tiles - 1 - item, lane, s_pre_all[warp], s_sums, s_scale_bits);
 }
 
 // Any tile shape: one CTA per tile.
