@@ -494,7 +494,9 @@ batch_gather(const __grid_constant__ BatchArgsT<N> b)
     __shared__ u32 s_pre_all[kGatherThreads / 32][kSmallBins + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const u32 warps = gridDim.x * (kGatherThreads / 32);
-    for (u32 gt = blockIdx.x * (kGatherThreads / 32) + warp; gt < b.total_tiles; gt += warps) {
+    // Last tile first: the tile pass wrote the residues front to back, so the tail is what the L2 still holds.
+    for (u32 item = blockIdx.x * (kGatherThreads / 32) + warp; item < b.total_tiles; item += warps) {
+        const u32 gt = b.total_tiles - 1u - item;
         const BatchLayer &L = b.layer[batch_layer_of(b, gt)];
         const unsigned char *scratch = L.packed + L.geo.scratch_at;
         if (L.geo.w == 1u)
