@@ -857,6 +857,11 @@ __device__ inline u64 tile_offset(const unsigned char *scratch, const Geometry &
     return group[g] + before;
 }
 
+#ifndef ADACOMP_GATHER_AHEAD
+#define ADACOMP_GATHER_AHEAD 8
+#endif
+constexpr int kGatherAhead = ADACOMP_GATHER_AHEAD;     // words a lane of the gather has in flight
+
 // One tile of at most 96 bins, handled by one warp.
 // group_sums / scale_bits: null / unused where a finalize kernel ran before (the groups' running sums are in the
 // scratch, the scale in the header); else the CTA's own copies.
@@ -898,13 +903,13 @@ __device__ void gather_tile_small(float *residue, unsigned char *packed, const u
     }
     const Word *slot = reinterpret_cast<const Word *>(scratch + geo.slots_at + tile * geo.slot_bytes);
     const u64 base = tile * (u64)geo.tile_elems;
-    for (u32 j0 = 0; j0 < cnt; j0 += 128) {
-        // four words per lane per round: their residue loads overlap
-        u32 word[4];
-        u64 pos[4];
-        float g[4];
+    for (u32 j0 = 0; j0 < cnt; j0 += 32 * kGatherAhead) {
+        // kGatherAhead words per lane per round: their residue loads overlap
+        u32 word[kGatherAhead];
+        u64 pos[kGatherAhead];
+        float g[kGatherAhead];
 #pragma unroll
-        for (int q = 0; q < 4; q++) {
+        for (int q = 0; q < kGatherAhead; q++) {
             const u32 j = j0 + q * 32 + lane;
             word[q] = 0;
             pos[q] = 0;
@@ -919,7 +924,7 @@ __device__ void gather_tile_small(float *residue, unsigned char *packed, const u
             }
         }
 #pragma unroll
-        for (int q = 0; q < 4; q++) {
+        for (int q = 0; q < kGatherAhead; q++) {
             const u32 j = j0 + q * 32 + lane;
             if (j < cnt) {
                 if (FIXUP) residue[pos[q]] = (word[q] & 2u) ? __fadd_rn(g[q], scale) : __fsub_rn(g[q], scale);
