@@ -25,6 +25,7 @@ int device_info(DeviceInfo *&out)
         init_pack_info(d);
         init_pack_batch_info(d);        // (after init_pack_info: it needs fast_ready)
         init_pack_onchip_info(d);
+        init_pack_onchip_list_info(d);
         init_decode_batch_info(d);
         d.sms = sms;
     }
@@ -530,6 +531,7 @@ int adacomp_device_status(uint32_t *host_out, void *stream)
                     status_read_pack_fast_d(&v) &&
                     status_read_pack_batch(&v) &&
                     status_read_pack_onchip(&v) &&
+                    status_read_pack_onchip_list(&v) &&
                     status_read_decode(&v) &&
                     status_read_decode_opt(&v) &&
                     status_read_decode_batch(&v) &&
@@ -549,6 +551,7 @@ int adacomp_device_status_reset(void *stream)
     status_reset_pack_fast_d(st);
     status_reset_pack_batch(st);
     status_reset_pack_onchip(st);
+    status_reset_pack_onchip_list(st);
     status_reset_decode(st);
     status_reset_decode_opt(st);
     status_reset_decode_batch(st);

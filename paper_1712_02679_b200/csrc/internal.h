@@ -20,6 +20,7 @@ struct DeviceInfo {
     int dec_batch_warps_per_sm[3] = {0, 0, 0};      // CTAs of the batched warp decoder per SM, by optimizer form
     bool fast_ready = false;
     int onchip_ctas = 0;        // CTAs of the one-kernel pack() that are resident together; 0: unavailable on this device
+    int onchip_list_ctas = 0;   // the same for the one-kernel pack() of a parameter list
 };
 
 
@@ -28,6 +29,7 @@ int device_info(DeviceInfo *&out);
 void init_pack_info(DeviceInfo &d);             // pack.cu, pack_fast_*.cu
 void init_pack_batch_info(DeviceInfo &d);       // pack_batch.cu
 void init_pack_onchip_info(DeviceInfo &d);      // pack_onchip.cu
+void init_pack_onchip_list_info(DeviceInfo &d); // pack_onchip_list.cu (after init_pack_onchip_info)
 void init_decode_info(DeviceInfo &d);           // decode.cu, decode_opt.cu
 void init_decode_batch_info(DeviceInfo &d);     // decode_batch.cu
 
@@ -66,6 +68,10 @@ int launch_decode_opt(const DecodeArgs &args, const Epilogue &ep, const DeviceIn
 u64 onchip_tile_capacity(const DeviceInfo &d);
 int launch_pack_onchip(PassArgs &args, u64 *count_out, u32 header_flags, const DeviceInfo &info, cudaStream_t st);
 
+// pack_onchip_list.cu: the same for a batch of layers (the layers' control blocks cleared before)
+bool onchip_list_takes(const BatchArgs &b, const DeviceInfo &info);
+int launch_pack_onchip_list(const BatchArgs &b, const DeviceInfo &info, long long wait_limit, cudaStream_t st);
+
 // wire.cu: a packed stream re-encoded as version 2 (to_v2) or back as version 1
 int stream_convert(const void *in, void *out, uint64_t out_capacity, uint64_t *count_out, uint64_t n, uint32_t L_T,
                    bool to_v2, void *stream);
@@ -86,6 +92,7 @@ ADACOMP_STATUS_DECLARE(pack_fast_c)
 ADACOMP_STATUS_DECLARE(pack_fast_d)
 ADACOMP_STATUS_DECLARE(pack_batch)
 ADACOMP_STATUS_DECLARE(pack_onchip)
+ADACOMP_STATUS_DECLARE(pack_onchip_list)
 ADACOMP_STATUS_DECLARE(decode)
 ADACOMP_STATUS_DECLARE(decode_opt)
 ADACOMP_STATUS_DECLARE(decode_batch)

@@ -583,14 +583,20 @@ int launch_batch(const BatchArgs &b, const DeviceInfo &info, cudaStream_t st, bo
         return compress_impl(L.grad, L.residue, L.geo.n, L.geo.L_T, L.packed, reinterpret_cast<uint64_t *>(L.count_out),
                              st, 0, nullptr, L.lazy, L.factor, L.grad_type);
     }
+    // a list that fits on the chip: the control blocks cleared, then one kernel (pack_onchip_list.cu)
+    const bool onchip = !lazy && debug_waits().withhold_pack == 0 && onchip_list_takes(b, info);
     if (b.n_layers <= (u32)kBatchSmall) {
         BatchArgsT<kBatchSmall> small;
         small.n_layers = b.n_layers;
         small.total_tiles = b.total_tiles;
         for (u32 i = 0; i < b.n_layers; i++) small.layer[i] = b.layer[i];
-        return launch_batch_sized(small, info, st, lazy);
+        if (!onchip) return launch_batch_sized(small, info, st, lazy);
+        batch_clear<kBatchSmall><<<small.n_layers, 128, 0, st>>>(small);
+    } else {
+        if (!onchip) return launch_batch_sized(b, info, st, lazy);
+        batch_clear<kBatchMax><<<b.n_layers, 128, 0, st>>>(b);
     }
-    return launch_batch_sized(b, info, st, lazy);
+    return launch_pack_onchip_list(b, info, debug_waits().limit, st);
 }
 
 

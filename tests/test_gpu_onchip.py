@@ -134,3 +134,89 @@ def test_through_the_entry_point_with_its_own_scratch():
     torch.cuda.synchronize()
     assert_stream_equal(packed[:int(cnt[1])].cpu().numpy(), want, "own scratch")
     assert_f32_bits_equal(res.cpu().numpy(), r_cpu, "own scratch residue")
+
+
+# ---- a whole parameter list in one kernel ----
+
+def run_list(shapes, steps=2, factors=None, seed=3):
+    """shapes: (L_T, n) per layer; every step and layer against the oracle."""
+    rng = np.random.default_rng(seed)
+    layers, r_cpu = [], []
+    for t, (L_T, n) in enumerate(shapes):
+        r = rng.normal(0, 2e-3, n).astype(np.float32)
+        res = torch.zeros(max(n, 4), device=DEV)
+        res[:n] = torch.from_numpy(r)
+        r_cpu.append(r)
+        layers.append(dict(grad=torch.zeros(max(n, 4), device=DEV), residue=res, n=n, L_T=L_T,
+                           packed_out=torch.empty(B.adacomp_packed_capacity(n, L_T), dtype=torch.uint8, device=DEV),
+                           count_out=torch.zeros(2, dtype=torch.int64, device=DEV),
+                           factor=0.0 if factors is None else factors[t]))
+    for step in range(steps):
+        want = []
+        for t, (L_T, n) in enumerate(shapes):
+            g = rng.normal(0, 1e-3, n).astype(np.float32)
+            layers[t]["grad"][:n].copy_(torch.from_numpy(g))
+            want.append(cref.pack(g, r_cpu[t], L_T, factor=layers[t]["factor"]))
+        if factors is None:
+            B.adacomp_compress_multi(layers, len(layers))
+        else:
+            B.adacomp_compress_multi_opt(layers, len(layers))
+        torch.cuda.synchronize()
+        for t, (L_T, n) in enumerate(shapes):
+            what = f"step {step} layer {t} L_T={L_T} n={n}"
+            used = int(layers[t]["count_out"][1])
+            assert_stream_equal(layers[t]["packed_out"][:used].cpu().numpy(), want[t], what)
+            assert_f32_bits_equal(layers[t]["residue"][:n].cpu().numpy(), r_cpu[t], what + " residue")
+    assert B.adacomp_device_status() == 0
+
+
+def test_list_in_one_kernel_mixed_bin_lengths_ragged_and_tiny_layers():
+    run_list([(500, 4000 * 7 + 3), (50, 4000 * 5 + 49), (500, 64), (50, 1), (500, 4000 * 2), (50, 4000), (500, 3999),
+              (50, 4000 * 30 + 1999), (500, 4000 * 41 + 1)], steps=3)
+
+
+def test_list_in_one_kernel_with_factors():
+    run_list([(500, 4000 * 6 + 7), (50, 4000 * 9 + 11), (500, 4000 * 3)], factors=[1.5, 0.0, 3.0])
+
+
+def test_list_at_the_capacity_of_the_one_kernel_form_and_beyond():
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    cap_tiles = sms * 2 * 4
+    half = cap_tiles // 2
+    run_list([(50, 4000 * half), (500, 4000 * (cap_tiles - half) - 17)], steps=2)           # exactly the capacity
+    run_list([(50, 4000 * half), (500, 4000 * (cap_tiles - half) + 1)], steps=2)            # one tile more: the batch kernels
+
+
+def test_list_with_another_bin_length_takes_the_batch_kernels():
+    run_list([(500, 4000 * 6 + 7), (100, 4000 * 4 + 50), (50, 4000 * 3 + 1)], steps=2)
+
+
+def test_list_in_one_kernel_under_a_cuda_graph():
+    shapes = [(500, 4000 * 11 + 5), (50, 4000 * 6 + 3), (500, 1000)]
+    rng = np.random.default_rng(21)
+    layers, r_cpu = [], []
+    for L_T, n in shapes:
+        r_cpu.append(np.zeros(n, np.float32))
+        layers.append(dict(grad=torch.zeros(n, device=DEV), residue=torch.zeros(n, device=DEV), n=n, L_T=L_T,
+                           packed_out=torch.empty(B.adacomp_packed_capacity(n, L_T), dtype=torch.uint8, device=DEV),
+                           count_out=torch.zeros(2, dtype=torch.int64, device=DEV)))
+    descs = B.make_layer_descs(layers)
+    B.adacomp_compress_multi(descs, len(layers))            # (first call outside the capture)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            B.adacomp_compress_multi(descs, len(layers), stream=s.cuda_stream)
+    for step in range(3):
+        want = []
+        for t, (L_T, n) in enumerate(shapes):
+            g = rng.normal(0, 1e-3, n).astype(np.float32)
+            layers[t]["grad"].copy_(torch.from_numpy(g))
+            want.append(cref.pack(g, r_cpu[t], L_T))
+        graph.replay()
+        torch.cuda.synchronize()
+        for t, (L_T, n) in enumerate(shapes):
+            used = int(layers[t]["count_out"][1])
+            assert_stream_equal(layers[t]["packed_out"][:used].cpu().numpy(), want[t], f"replay {step} layer {t}")
+            assert_f32_bits_equal(layers[t]["residue"].cpu().numpy(), r_cpu[t], f"replay {step} layer {t} residue")
