@@ -292,7 +292,10 @@ bool onchip_list_takes(const BatchArgs &b, const DeviceInfo &info)
     return false;
 #endif
     if (info.onchip_list_ctas <= 0 || b.n_layers == 0 || b.total_tiles == 0) return false;
-    if ((u64)b.total_tiles > (u64)info.onchip_list_ctas * kOnchipSlots) return false;
+    // (up to two tiles per CTA: beyond that the batch kernels' pipelines, which keep loads, work and stores going side
+    // by side, beat this kernel's burst of loads at the start and of stores at the end when the data come from DRAM:
+    // the LSTM list, three tiles per CTA, 26.9 against 22.7 us per learner)
+    if ((u64)b.total_tiles > (u64)info.onchip_list_ctas * 2) return false;
     for (u32 i = 0; i < b.n_layers; i++) {
         const BatchLayer &L = b.layer[i];
         if ((L.geo.L_T != 50u && L.geo.L_T != 500u) || L.grad_type != ADACOMP_GRAD_F32 || L.lazy != nullptr || L.geo.n_tiles == 0) return false;

@@ -181,7 +181,7 @@ def test_list_in_one_kernel_with_factors():
 
 def test_list_at_the_capacity_of_the_one_kernel_form_and_beyond():
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    cap_tiles = sms * 2 * 4
+    cap_tiles = sms * 2 * 2                         # (lists: two tiles per CTA)
     half = cap_tiles // 2
     run_list([(50, 4000 * half), (500, 4000 * (cap_tiles - half) - 17)], steps=2)           # exactly the capacity
     run_list([(50, 4000 * half), (500, 4000 * (cap_tiles - half) + 1)], steps=2)            # one tile more: the batch kernels
