@@ -399,7 +399,14 @@ typedef struct {
     uint64_t *count_out;
 } adacomp_layer_desc;
 
-/* pack() of every layer in `layers` (HOST array of n_layers descriptors) on one stream. */
+/*
+ * pack() of every layer in `layers` (HOST array of n_layers descriptors) on one stream.  Every layer gets what
+ * adacomp_compress would give it, bit for bit; the layers are independent, and the order in which the kernels
+ * take them is not the list's.  Layers share launches: a small list (bin lengths 50 and 500, at most two
+ * 4000-element tiles per resident CTA in all) is packed by two launches, lists of layers with bin lengths 42..1000
+ * and fewer than 2^25 elements each by four launches per batch of up to 176 layers, other layers one by one.
+ * The descriptors are read during the call only.
+ */
 int adacomp_compress_multi(const adacomp_layer_desc *layers, uint32_t n_layers, void *stream);
 
 /*
