@@ -29,14 +29,14 @@ def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool 
     n = len(dW)
     dW = [f32(x) for x in dW]
     residue = [f32(x) for x in residue]
-    G = [f32(residue[i] + dW[i]) for i in range(n)]          # G <- residue + dW
+    G = [f32(residue[i] + dW[i]) for i in range(n)]          # this step's accumulated gradient
     if factor == 0.0:
-        H = [f32(G[i] + dW[i]) for i in range(n)]            # H <- G + dW
+        H = [f32(G[i] + dW[i]) for i in range(n)]            # the latest gradient counted twice (the selection's look-ahead)
     else:
         H = [f32(residue[i] + f32(f32(factor) * dW[i])) for i in range(n)]
     n_bins = -(-n // L_T)
     g_max = []
-    for i in range(n_bins):                                  # over all bins
+    for i in range(n_bins):                                  # first sweep: each bin's largest |G|
         members = G[i * L_T:(i + 1) * L_T]
         g_max.append(max((abs(x) for x in members), default=f32(0)))
     if n_bins:
@@ -59,9 +59,9 @@ def pack(dW: Sequence[float], residue: Sequence[float], L_T: int, literal: bool 
     bin_cnt: List[int] = []
     words: List[int] = []
     new_residue = list(G)
-    for i in range(n_bins):                                  # over all bins
+    for i in range(n_bins):                                  # second sweep: bin by bin,
         count = 0
-        for j in range(L_T):                                 # over all indices within the bin
+        for j in range(L_T):                                 # place by place
             index = i * L_T + j
             if index >= n:
                 break
