@@ -357,7 +357,8 @@ decode_batch_warps(const __grid_constant__ DecodeBatchArgs b, u32 ring_bytes)
         seek(gt, li);
         const BatchLayerCtx &c = sm.ctx[li];
         if (li != at_li) {
-            if (at_li != 0xffffffffu) {
+            // (layers of one bin length and word width, as most neighbours in a list are, cut the tile alike)
+            if (at_li != 0xffffffffu && !(c.L_T == L_T && (int)c.TB == TB && c.w == wb)) {
                 // a warp's share of the output tile moves with the bin length: every warp has stored and
                 // zeroed its old share before any adds into its new one (a bounded wait, as all of them)
                 __syncwarp();
