@@ -220,3 +220,11 @@ def test_list_in_one_kernel_under_a_cuda_graph():
             used = int(layers[t]["count_out"][1])
             assert_stream_equal(layers[t]["packed_out"][:used].cpu().numpy(), want[t], f"replay {step} layer {t}")
             assert_f32_bits_equal(layers[t]["residue"].cpu().numpy(), r_cpu[t], f"replay {step} layer {t} residue")
+
+
+def test_list_in_one_kernel_with_more_layers_than_the_small_table():
+    rng = np.random.default_rng(77)
+    shapes = [(500 if t % 3 else 50, int(rng.integers(1, 3 * 4000))) for t in range(60)]
+    run_list(shapes, steps=2, seed=78)
+    shapes = [(50 if t % 2 else 500, int(rng.integers(1, 2 * 4000))) for t in range(200)]      # two batches
+    run_list(shapes, steps=1, seed=79)
